@@ -1,0 +1,464 @@
+#!/usr/bin/env python
+"""Benchmark of the fused operator groups on B200.
+
+One "step" is one pass of the whole hot path over synthetic inputs shaped like the five
+configurations: tiny fp32 MLP layer (forward + gradient), the bf16 broadcast-elementwise group
+(forward + gradient group), the 3-layer bf16 MLP (forward + full backward), the 3x3 conv2d
+(forward + dX + dW + db) and the LSTM sequence.  Every group is timed with CUDA events on the
+launching stream; the line printed at the end carries the tensor-bound aggregate as `value`
+(TFLOP/s over the dense + conv2d groups), the memory-bound aggregate (GB/s over the elementwise
+groups), a per-group table, the roofline of the dominant kernel, the end-to-end figure with
+host buffers, and the CPU oracle timed on a bounded sample.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--groups a,b,..]
+
+With N > 1 (under torchrun) every rank runs an independent replica on its own GPU: the path
+has no exchange step, so there is no collective on the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+METRIC = "fused-group TFLOP/s (dense/conv) and HBM GB/s (ewise/reduce) on 1 B200 vs roofline"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+ALL_GROUPS = ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"]
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        d["source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["source"] = "fallback"
+    return d
+
+
+# ---------------------------------------------------------------------------------------------------
+# clocks sampling (nvidia-smi in the background during the timed region)
+# ---------------------------------------------------------------------------------------------------
+class ClockSampler:
+    Q = "clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown," \
+        "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap"
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx = float(r[1])
+            except Exception:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------------------------------
+# the groups
+# ---------------------------------------------------------------------------------------------------
+class Timer:
+    """CUDA-event timing of labelled regions on the current stream."""
+
+    def __init__(self):
+        self.pending, self.ms = [], {}
+
+    def region(self, label):
+        t = self
+
+        class R:
+            def __enter__(self_inner):
+                self_inner.a = torch.cuda.Event(enable_timing=True); self_inner.b = torch.cuda.Event(enable_timing=True)
+                self_inner.a.record()
+
+            def __exit__(self_inner, *exc):
+                self_inner.b.record()
+                t.pending.append((label, self_inner.a, self_inner.b))
+        return R()
+
+    def collect(self):
+        torch.cuda.synchronize()
+        for label, a, b in self.pending:
+            self.ms.setdefault(label, []).append(a.elapsed_time(b))
+        self.pending = []
+
+
+class Workload:
+    def __init__(self, dev, groups, small=False):
+        from paper_1810_00952_b200 import binding as B
+        from relay_workloads import inputs as I
+        from relay_workloads import program as P
+        self.B, self.I, self.P, self.dev, self.groups = B, I, P, dev, groups
+        self.host, self.devt, self.out = {}, {}, {}
+        ws_bytes = 16
+        if "cfg1" in groups:
+            self.host["cfg1"] = I.cfg1_tiny_mlp()
+        if "cfg2" in groups:
+            self.host["cfg2"] = I.cfg2_ewise(*((512, 1024) if small else (8192, 8192)))
+        if "cfg3" in groups:
+            self.host["cfg3"] = I.cfg3_mlp(*((256, 256) if small else (4096, 4096)))
+        if "cfg4" in groups:
+            self.host["cfg4"] = I.cfg4_conv(*((2, 32, 14, 14, 32) if small else (32, 256, 56, 56, 256)))
+        if "cfg5" in groups:
+            self.host["cfg5"] = I.cfg5_lstm(*((8, 8, 64, 64) if small else (128, 64, 1024, 1024)))
+        for g, d in self.host.items():
+            self.host[g] = {k: v.pin_memory() for k, v in d.items()}
+            self.devt[g] = {k: torch.empty_like(v, device=dev) for k, v in d.items()}
+        E = lambda *s, dt=torch.bfloat16: torch.empty(*s, dtype=dt, device=dev)
+        f32 = torch.float32
+        if "cfg1" in groups:
+            self.out["cfg1"] = dict(y=E(8, 32, dt=f32), dx=E(8, 64, dt=f32), dw=E(64, 32, dt=f32), db=E(32, dt=f32))
+            ws_bytes = max(ws_bytes, B.relay_workspace_bytes_dense_act_grad(self.devt["cfg1"]["x"], self.devt["cfg1"]["w"]))
+        if "cfg2" in groups:
+            r, c = self.host["cfg2"]["x"].shape
+            self.out["cfg2"] = dict(out=E(r, c), dx=E(r, c), da=E(c, dt=f32), db=E(1, c, dt=f32))
+            self.fwd_prog, self.fwd_outs = P.tanh_affine_residual_fwd(P.BF16)
+            self.grad_prog, ids = P.tanh_affine_residual_grad(P.BF16)
+            self.grad_specs = [(ids[0], B.RED_NONE, 0, 0), (ids[1], B.RED_SUM, 1, 0), (ids[2], B.RED_SUM, 1, 1)]
+            d = self.devt["cfg2"]
+            ws_bytes = max(ws_bytes, B.relay_workspace_bytes_reduce([d["dout"], d["x"], d["a"], d["b"]], self.grad_specs))
+        if "cfg3" in groups:
+            m, k = self.host["cfg3"]["x"].shape
+            o = dict()
+            for l in range(3):
+                o[f"y{l}"] = E(m, k); o[f"dx{l}"] = E(m, k); o[f"dw{l}"] = E(k, k); o[f"db{l}"] = E(k, dt=f32)
+            self.out["cfg3"] = o
+            ws_bytes = max(ws_bytes, B.relay_workspace_bytes_dense_act_grad(self.devt["cfg3"]["x"], self.devt["cfg3"]["w0"]))
+        if "cfg4" in groups:
+            d = self.devt["cfg4"]
+            self.out["cfg4"] = dict(y=torch.empty_like(d["dy"]), dx=torch.empty_like(d["x"]), dw=torch.empty_like(d["w"]),
+                                    db=E(d["w"].shape[0], dt=f32))
+            ws_bytes = max(ws_bytes, B.relay_workspace_bytes_conv2d_act(d["x"], d["w"], 1, 1),
+                           B.relay_workspace_bytes_conv2d_act_grad(d["x"], d["w"], 1, 1))
+        if "cfg5" in groups:
+            d = self.devt["cfg5"]
+            T, Bn, _ = d["x"].shape
+            H = d["w_hh"].shape[0]
+            self.out["cfg5"] = dict(h_all=E(T, Bn, H, dt=f32), c=E(Bn, H, dt=f32))
+            ws_bytes = max(ws_bytes, B.relay_workspace_bytes_lstm(d["x"], d["w_ih"], d["w_hh"]))
+        self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+        self.flush_buf = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+        self.pinned_out = {g: {k: torch.empty_like(v, device="cpu").pin_memory() for k, v in o.items()} for g, o in self.out.items()}
+        self.upload()
+
+    # -- data movement ---------------------------------------------------------------------------------
+    def upload(self):
+        n = 0
+        for g, d in self.host.items():
+            for k, v in d.items():
+                self.devt[g][k].copy_(v, non_blocking=True)
+                n += v.numel() * v.element_size()
+        return n
+
+    def download(self):
+        n = 0
+        for g, o in self.out.items():
+            for k, v in o.items():
+                self.pinned_out[g][k].copy_(v, non_blocking=True)
+                n += v.numel() * v.element_size()
+        return n
+
+    def flush_l2(self):
+        self.flush_buf.fill_(1)   # 256 MiB written: larger than the 126 MB L2
+
+    # -- one pass of the hot path ------------------------------------------------------------------------
+    def step(self, tm: Timer):
+        B, ws = self.B, self.ws
+        if "cfg1" in self.groups:
+            d, o = self.devt["cfg1"], self.out["cfg1"]
+            with tm.region("cfg1.fwd"):
+                B.relay_fused_dense_act(d["x"], d["w"], d["b"], B.ACT_RELU, o["y"], ws)
+            with tm.region("cfg1.grad"):
+                B.relay_fused_dense_act_grad(d["x"], d["w"], o["y"], d["dy"], B.ACT_RELU, o["dx"], o["dw"], o["db"], ws)
+        if "cfg2" in self.groups:
+            d, o = self.devt["cfg2"], self.out["cfg2"]
+            self.flush_l2()
+            with tm.region("cfg2.fwd"):
+                B.relay_fused_ewise(self.fwd_prog.arrays(), [d["x"], d["a"], d["b"]], self.fwd_outs, [o["out"]], ws)
+            self.flush_l2()
+            with tm.region("cfg2.grad"):
+                B.relay_fused_reduce(self.grad_prog.arrays(), [d["dout"], d["x"], d["a"], d["b"]], self.grad_specs,
+                                     [o["dx"], o["da"], o["db"]], ws)
+        if "cfg3" in self.groups:
+            d, o = self.devt["cfg3"], self.out["cfg3"]
+            self.flush_l2()
+            acts = [d["x"], o["y0"], o["y1"], o["y2"]]
+            with tm.region("cfg3.fwd"):
+                for l in range(3):
+                    with tm.region("cfg3.fwd.layer"):
+                        B.relay_fused_dense_act(acts[l], d[f"w{l}"], d[f"b{l}"], B.ACT_RELU, acts[l + 1], ws)
+            with tm.region("cfg3.bwd"):
+                g = d["dy"]
+                for l in (2, 1, 0):
+                    B.relay_fused_dense_act_grad(acts[l], d[f"w{l}"], acts[l + 1], g, B.ACT_RELU, o[f"dx{l}"], o[f"dw{l}"],
+                                                 o[f"db{l}"], ws)
+                    g = o[f"dx{l}"]
+        if "cfg4" in self.groups:
+            d, o = self.devt["cfg4"], self.out["cfg4"]
+            self.flush_l2()
+            with tm.region("cfg4.fwd"):
+                B.relay_fused_conv2d_act(d["x"], d["w"], d["b"], 1, 1, B.ACT_RELU, o["y"], ws)
+            with tm.region("cfg4.grad"):
+                B.relay_fused_conv2d_act_grad(d["x"], d["w"], o["y"], d["dy"], 1, 1, B.ACT_RELU, o["dx"], o["dw"], o["db"], ws)
+        if "cfg5" in self.groups:
+            d, o = self.devt["cfg5"], self.out["cfg5"]
+            self.flush_l2()
+            with tm.region("cfg5.lstm"):
+                B.relay_lstm_cell_seq(d["x"], d["w_ih"], d["w_hh"], d["b"], d["h0"], d["c0"], o["h_all"], o["c"], ws)
+
+    # -- algorithmic work per step -------------------------------------------------------------------------
+    def work(self):
+        w = {}
+        if "cfg1" in self.groups:
+            w["cfg1.fwd"] = dict(flop=2 * 8 * 64 * 32); w["cfg1.grad"] = dict(flop=2 * 2 * 8 * 64 * 32 + 8 * 32 * 2)
+        if "cfg2" in self.groups:
+            r, c = self.host["cfg2"]["x"].shape
+            w["cfg2.fwd"] = dict(bytes=2 * r * c * 2 + 2 * c * 2)
+            w["cfg2.grad"] = dict(bytes=3 * r * c * 2 + 2 * c * 2 + 2 * c * 4)
+        if "cfg3" in self.groups:
+            m, k = self.host["cfg3"]["x"].shape
+            w["cfg3.fwd"] = dict(flop=3 * 2 * m * k * k); w["cfg3.bwd"] = dict(flop=6 * 2 * m * k * k)
+            w["cfg3.fwd.layer"] = dict(flop=2 * m * k * k)
+        if "cfg4" in self.groups:
+            n, c, h, wd = self.host["cfg4"]["x"].shape
+            o = self.host["cfg4"]["w"].shape[0]
+            f = 2 * n * h * wd * o * c * 9
+            w["cfg4.fwd"] = dict(flop=f); w["cfg4.grad"] = dict(flop=2 * f)
+        if "cfg5" in self.groups:
+            T, Bn, In = self.host["cfg5"]["x"].shape
+            H = self.host["cfg5"]["w_hh"].shape[0]
+            w["cfg5.lstm"] = dict(flop=2 * T * Bn * (In + H) * 4 * H)
+        return w
+
+
+# ---------------------------------------------------------------------------------------------------
+# CPU oracle on a bounded sample (single thread); also the `--impl reference` arm
+# ---------------------------------------------------------------------------------------------------
+def oracle_sample(rows3=48, rows2=192):
+    """Times the fp64 oracle, as it stands, on slices of the same workload along the independent
+    dimension.  Returns (tflops, gbs, seconds, description)."""
+    import oracle
+    from relay_workloads import inputs as I
+    from relay_workloads import program as P
+    t3 = I.cfg3_mlp(batch=rows3)
+    x, w, b, dy = (I.as_f64(t3[k]) for k in ("x", "w0", "b0", "dy"))
+    t0 = time.perf_counter()
+    y = oracle.dense_act(x, w, b, oracle.ACT_RELU, oracle.BF16)
+    oracle.dense_act_grad(x, w, y, dy, oracle.ACT_RELU, oracle.BF16, oracle.BF16, oracle.F32)
+    s3 = time.perf_counter() - t0
+    flop3 = 3 * 2 * rows3 * 4096 * 4096
+    t2 = I.cfg2_ewise(rows=rows2)
+    prog, outs = P.tanh_affine_residual_fwd(P.BF16)
+    ins = [I.as_f64(t2[k]) for k in ("x", "a", "b")]
+    t0 = time.perf_counter()
+    oracle.ewise(prog.arrays(), ins, outs)
+    s2 = time.perf_counter() - t0
+    bytes2 = 2 * rows2 * 8192 * 2
+    desc = (f"cfg3 layer forward+gradient on the first {rows3} batch rows ({flop3 / 1e9:.1f} GFLOP, {s3:.1f} s) and "
+            f"cfg2 forward on the first {rows2} rows ({bytes2 / 1e6:.1f} MB, {s2:.1f} s)")
+    return flop3 / s3 / 1e12, bytes2 / s2 / 1e9, s3 + s2, desc
+
+
+def run_reference(args, rank, world):
+    if rank != 0:
+        return
+    vals = []
+    for i in range(args.warmup + args.steps):
+        tf, gb, sec, desc = oracle_sample(rows3=16, rows2=64)
+        if i >= args.warmup:
+            vals.append((tf, gb, sec))
+    tf = float(np.mean([v[0] for v in vals])); gb = float(np.mean([v[1] for v in vals])); sec = float(np.mean([v[2] for v in vals]))
+    line = {"impl": "reference", "metric": METRIC, "value": tf, "unit": "TFLOP/s", "hbm_gbs": gb, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "all five configurations; each step = the oracle on a bounded sample: " + desc},
+            "cpu_baseline": {"value": tf, "unit": "TFLOP/s", "cores": 1, "kind": "oracle", "sample": desc},
+            "e2e": {"value": tf, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}, "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--groups", default=",".join(ALL_GROUPS))
+    ap.add_argument("--small", action="store_true", help="reduced shapes (for profiler captures and quick checks)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0")); world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        return run_reference(args, rank, world)
+    if args.warmup < 3:
+        args.warmup = 3 if not args.small else args.warmup
+
+    from paper_1810_00952_b200 import binding as B
+    B.lib()   # fails loudly if the CUDA library is missing
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device"
+    dev = torch.device(f"cuda:{local}")
+    torch.cuda.set_device(dev)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    groups = [g for g in args.groups.split(",") if g]
+    wl = Workload(dev, groups, small=args.small)
+    work = wl.work()
+    peaks = load_peaks()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    tm = Timer()
+    for _ in range(args.warmup):
+        wl.step(tm)
+    tm.collect(); tm.ms = {}
+    B.relay_poll_status()
+
+    sampler = ClockSampler(local); sampler.start()
+    barrier()
+    n0 = B.relay_launch_count()
+    t_all0 = torch.cuda.Event(enable_timing=True); t_all1 = torch.cuda.Event(enable_timing=True)
+    t_all0.record()
+    for _ in range(args.steps):
+        wl.step(tm)
+    t_all1.record()
+    barrier()
+    launches = (B.relay_launch_count() - n0) // max(args.steps, 1)
+    tm.collect()
+    clocks = sampler.stop()
+    B.relay_poll_status()
+
+    # per-group device time (sum of the groups' regions; L2 flushes between groups are not counted)
+    top = [k for k in tm.ms if k.count(".") == 1]
+    med = {k: float(np.median(v)) for k, v in tm.ms.items()}
+    step_ms = sum(float(np.mean(tm.ms[k])) for k in top)
+    step_ms_t = torch.tensor([step_ms], device=dev)
+    if dist is not None:
+        dist.all_reduce(step_ms_t, op=dist.ReduceOp.MAX)
+    step_ms_max = float(step_ms_t.item())
+
+    tensor_keys = [k for k in top if k.startswith(("cfg3", "cfg4"))]
+    hbm_keys = [k for k in top if k.startswith("cfg2")]
+    t_ms = sum(float(np.mean(tm.ms[k])) for k in tensor_keys)
+    h_ms = sum(float(np.mean(tm.ms[k])) for k in hbm_keys)
+    tflops = world * sum(work[k]["flop"] for k in tensor_keys) / (t_ms * 1e-3) / 1e12 if t_ms else None
+    gbs = world * sum(work[k]["bytes"] for k in hbm_keys) / (h_ms * 1e-3) / 1e9 if h_ms else None
+
+    table = {}
+    for k in sorted(tm.ms):
+        ms = float(np.mean(tm.ms[k])) if k.count(".") == 1 else float(np.mean(tm.ms[k]))
+        e = {"ms": round(ms, 5), "ms_median": round(med[k], 5), "ms_best": round(float(np.min(tm.ms[k])), 5)}
+        if "flop" in work.get(k, {}):
+            e["tflops"] = work[k]["flop"] / (ms * 1e-3) / 1e12
+            e["frac_of_measured_bf16_peak"] = e["tflops"] / peaks["bf16_tflops"]
+        if "bytes" in work.get(k, {}):
+            e["gbs"] = work[k]["bytes"] / (ms * 1e-3) / 1e9
+            e["frac_of_measured_hbm"] = e["gbs"] / peaks["hbm_gbs"]
+        table[k] = e
+
+    # roofline of the dominant kernel: the dense contraction kernel, one launch per forward layer call
+    roofline = None
+    if "cfg3.fwd.layer" in table:
+        a = table["cfg3.fwd.layer"]["tflops"]
+        roofline = {"kernel": "dense contraction (forward layer call = one launch)", "bound": "tensor", "achieved": a,
+                    "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": a / peaks["bf16_tflops"], "traffic": None,
+                    "peak_source": peaks["source"] + " (burst)"}
+    elif "cfg2.fwd" in table:
+        a = table["cfg2.fwd"]["gbs"]
+        roofline = {"kernel": "ewise2d<tanh_affine_residual_fwd>", "bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": a / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]}
+
+    # end to end: pinned host inputs -> device, the step, results -> pinned host, all inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        tm2 = Timer()
+        h2d = d2h = 0
+        for _ in range(2):
+            wl.upload(); wl.step(tm2); wl.download()
+        barrier()
+        a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+        n_e2e = max(2, min(args.steps, 5))
+        a.record()
+        for _ in range(n_e2e):
+            h2d = wl.upload(); wl.step(tm2); d2h = wl.download()
+        b.record()
+        barrier()
+        e_ms = a.elapsed_time(b) / n_e2e
+        et = torch.tensor([e_ms], device=dev)
+        if dist is not None:
+            dist.all_reduce(et, op=dist.ReduceOp.MAX)
+        e_ms = float(et.item())
+        flop_all = sum(work[k]["flop"] for k in tensor_keys)
+        e2e = {"value": world * flop_all / (e_ms * 1e-3) / 1e12 if flop_all else None, "unit": "TFLOP/s", "ms_per_step": e_ms,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "note": "whole step incl. L2 flushes and all five configurations; dense+conv FLOPs over that time"}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        tf, gb, sec, desc = oracle_sample()
+        cpu = {"value": tf, "unit": "TFLOP/s", "hbm_gbs": gb, "cores": 1, "kind": "oracle", "sample": desc,
+               "host_cores_available": os.cpu_count()}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": tflops if tflops is not None else gbs, "unit": "TFLOP/s" if tflops is not None else "GB/s",
+                "hbm_gbs": gbs, "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms_max,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 (fp32 accumulate); cfg1 f32",
+                "data": "synthetic",
+                "config": {"workload": ("reduced shapes" if args.small else "all five configurations at full size")
+                           + ": step = cfg1 fwd+grad, cfg2 fwd+grad, cfg3 3-layer fwd+bwd, cfg4 conv fwd+dX+dW+db, cfg5 LSTM",
+                           "value_covers": "dense + conv2d groups (cfg3 + cfg4) FLOPs / their device time; hbm_gbs covers cfg2",
+                           "groups": groups, "l2": "256 MiB written between groups (L2 flush); cfg2 inputs exceed L2",
+                           "replicas": world},
+                "groups": table, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
+                "clocks": clocks, "peaks": {k: peaks.get(k) for k in ("hbm_gbs", "bf16_tflops", "bf16_tflops_sustained", "source")}}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

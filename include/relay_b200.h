@@ -1,0 +1,282 @@
+/*
+ * relay_b200.h -- C ABI of the fused primitive-operator groups that a Relay program executes.
+ *
+ * Background (Relay, arXiv 1810.00952).  Relay declares primitive operators as externally
+ * implemented functions with a tensor type ("operator <GlobalId> : <Type>", Section 3, Fig. 1),
+ * registers them with its runtime (Section 4.1) and instantiates them per concrete tensor
+ * type, i.e. per base type and static shape (Section 5.1).  Every value is a tensor whose
+ * type is Tensor(BaseType, Shape(d1..dn)) (Fig. 1; Fig. 4 rules BaseType-T, Shape-T,
+ * Tensor-T).  This library is that operator layer for one B200 GPU: each entry point checks
+ * the operand types against the operator's type relation on the host (Section 4.3: shapes live
+ * in types, so the check needs no data), then enqueues hand-written sm_100a kernels.
+ *
+ * Common rules for every compute entry point
+ *   - Tensors are dense and row-major in the order of `shape` (NCHW / OIHW are row-major over
+ *     those four axes).  `data` is a DEVICE pointer aligned to 16 bytes.  The caller owns all
+ *     buffers; the library allocates no device memory and keeps no pointer after return.
+ *   - `ws` is caller-provided device scratch of `ws_bytes` bytes (16-byte aligned); the needed
+ *     size comes from the matching relay_workspace_bytes_* query (0 means `ws` may be NULL).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls only enqueue
+ *     work and return without synchronising.  Inputs are read-only; outputs must not overlap
+ *     inputs or each other.
+ *   - All descriptor errors are found before anything is launched and leave outputs untouched.
+ *     Rules are checked in the order: null -> rank -> dtype -> layout -> shape -> attributes ->
+ *     alignment/overlap -> workspace; the first failing rule decides the status.
+ *     relay_last_error() returns a thread-local description of the last failure.
+ *   - Kernels that wait on hardware barriers give up after a bounded number of polls and set a
+ *     device-side error word instead of hanging; relay_poll_status() reads (and clears) it.
+ */
+#ifndef RELAY_B200_H_
+#define RELAY_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define RELAY_MAX_RANK 6
+#define RELAY_MAX_INPUTS 8
+#define RELAY_MAX_OUTPUTS 8
+#define RELAY_MAX_INSTR 32
+
+typedef enum {
+    RELAY_OK = 0,
+    RELAY_ERR_NULL = 1,        /* a required pointer is NULL */
+    RELAY_ERR_RANK = 2,        /* rank outside what the operator's type allows */
+    RELAY_ERR_SHAPE = 3,       /* shapes violate the operator's type relation */
+    RELAY_ERR_DTYPE = 4,       /* base types violate the operator's type relation */
+    RELAY_ERR_LAYOUT = 5,      /* layout tag not accepted by the operator */
+    RELAY_ERR_ALIGN = 6,       /* data pointer not 16-byte aligned */
+    RELAY_ERR_ATTR = 7,        /* bad attribute, malformed program, overlapping buffers */
+    RELAY_ERR_UNSUPPORTED = 8, /* well-typed, but no kernel instance exists for it */
+    RELAY_ERR_WORKSPACE = 9,   /* workspace missing, misaligned or too small */
+    RELAY_ERR_CUDA = 10,       /* a CUDA runtime/driver call failed */
+    RELAY_ERR_TIMEOUT = 11     /* a bounded device-side wait expired */
+} relay_status_t;
+
+/* Base types (Fig. 1 <BaseType>).  The paper's FloatType(width) carries only a width; the
+ * 16-bit float here is bfloat16 (8 exponent, 7 fraction bits).  Bool is stored as one byte
+ * holding 0 or 1. */
+typedef enum { RELAY_F32 = 0, RELAY_BF16 = 1, RELAY_I32 = 2, RELAY_I64 = 3, RELAY_BOOL = 4 } relay_dtype_t;
+
+typedef enum { RELAY_ROWMAJOR = 0, RELAY_NCHW = 1, RELAY_NHWC = 2, RELAY_OIHW = 3 } relay_layout_t;
+
+typedef enum { RELAY_ACT_NONE = 0, RELAY_ACT_RELU = 1, RELAY_ACT_TANH = 2, RELAY_ACT_SIGMOID = 3 } relay_act_t;
+
+/* A typed tensor value: Tensor(dtype, Shape(shape[0..rank))) plus its device address. */
+typedef struct relay_tensor {
+    void *data;
+    int32_t dtype;  /* relay_dtype_t */
+    int32_t rank;   /* 0..RELAY_MAX_RANK; rank 0 is a scalar (all values are tensors) */
+    int64_t shape[RELAY_MAX_RANK];
+    int32_t layout; /* relay_layout_t */
+    int32_t reserved;
+} relay_tensor_t;
+
+/* ---------------------------------------------------------------------------------------------
+ * Elementwise programs.  A fused elementwise group is a let-list (Fig. 1 "let") of at most
+ * RELAY_MAX_INSTR instructions.  Value ids: 0..n_in-1 are the group's inputs, n_in+j is the
+ * result of instruction j; an instruction may only name earlier values; unused operands are -1.
+ * Opcodes are Fig. 1's BinOp / UnaryOp productions, the cast production, and the elementwise
+ * library operators of Fig. 3.  Typing follows Fig. 5 after an explicit NumPy-style broadcast
+ * of all inputs to one shape: arithmetic needs equal float base types and yields that type
+ * (Type-Noncomp-BinaryOp, Type-UnaryOp); comparisons need equal base types and yield Bool
+ * (Type-Comp-BinaryOp); select needs a Bool condition and equal branch types; cast yields the
+ * named type; const is a literal of the named type.  `dtype` states the result type of each
+ * instruction and is checked against these rules.
+ * Arithmetic is carried out in fp32; a result whose type is bf16 is rounded to bf16 (nearest
+ * even).  Integer types may appear only as sources or targets of cast.
+ * ------------------------------------------------------------------------------------------- */
+typedef enum {
+    RELAY_OP_ADD = 0, RELAY_OP_SUB = 1, RELAY_OP_MUL = 2, RELAY_OP_DIV = 3,
+    RELAY_OP_NEG = 4, RELAY_OP_SQ = 5,
+    RELAY_OP_NE = 6, RELAY_OP_EQ = 7, RELAY_OP_LT = 8, RELAY_OP_LE = 9, RELAY_OP_GT = 10, RELAY_OP_GE = 11,
+    RELAY_OP_SELECT = 12, /* a ? b : c */
+    RELAY_OP_RELU = 13, RELAY_OP_TANH = 14, RELAY_OP_SIGMOID = 15,
+    RELAY_OP_CAST = 16, RELAY_OP_CONST = 17, RELAY_OP_EXP = 18, RELAY_OP_LOG = 19,
+    RELAY_OP_MAX = 20, RELAY_OP_MIN = 21,
+    RELAY_OP_COUNT_ = 22
+} relay_opcode_t;
+
+typedef struct relay_instr {
+    int32_t op;    /* relay_opcode_t */
+    int32_t a, b, c;
+    int32_t dtype; /* result type */
+    int32_t reserved;
+    double imm;    /* literal of RELAY_OP_CONST */
+} relay_instr_t;
+
+typedef struct relay_ewise_prog {
+    int32_t n_instr;
+    int32_t reserved;
+    const relay_instr_t *instr; /* HOST pointer; read during the call only */
+} relay_ewise_prog_t;
+
+typedef enum { RELAY_RED_NONE = 0, RELAY_RED_SUM = 1, RELAY_RED_MAX = 2, RELAY_RED_MEAN = 3, RELAY_RED_ARGMAX = 4 } relay_reduce_op_t;
+
+/* One result of a reduce group: program value `value`, reduced with `red_op` over the axes
+ * whose bit is set in `axes_mask` (bit d = axis d of the broadcast shape).  RELAY_RED_NONE
+ * returns the value unreduced.  With keepdims the reduced axes stay as extent 1. */
+typedef struct relay_out_spec {
+    int32_t value;
+    int32_t red_op;    /* relay_reduce_op_t */
+    int32_t axes_mask;
+    int32_t keepdims;
+} relay_out_spec_t;
+
+typedef struct relay_conv2d_attrs {
+    int32_t stride;   /* same in both spatial axes, >= 1 */
+    int32_t pad;      /* zero padding on every side, >= 0 */
+    int32_t dilation; /* must be 1 */
+    int32_t groups;   /* must be 1 */
+} relay_conv2d_attrs_t;
+
+/* ---------------------------------------------------------------------------------------------
+ * Type relations, host only (no GPU needed).  Each fills `out` (dtype, rank, shape, layout;
+ * data = NULL) with the result type the operator's relation gives for the argument types,
+ * the way Fig. 5 derives the type of an expression from the types of its parts.
+ * ------------------------------------------------------------------------------------------- */
+
+/* dense: Tensor(t,(M,K)) x Tensor(t,(K,N)) -> Tensor(t,(M,N)), t in {f32, bf16} (Fig. 3 relay.linear). */
+relay_status_t relay_infer_dense(const relay_tensor_t *x, const relay_tensor_t *w, relay_tensor_t *out);
+
+/* conv2d: x:(N,C,H,W) NCHW, w:(O,C,R,S) OIHW -> (N,O,P,Q) with P = floor((H+2p-R)/s)+1
+ * (Fig. 3 relay.conv2d). */
+relay_status_t relay_infer_conv2d(const relay_tensor_t *x, const relay_tensor_t *w,
+                                  const relay_conv2d_attrs_t *attrs, relay_tensor_t *out);
+
+/* NumPy-style broadcast of two shapes (the explicit step that precedes Fig. 5's same-shape
+ * rules): right-align, each axis pair equal or one of them 1.  dtype/layout copied from a. */
+relay_status_t relay_infer_broadcast(const relay_tensor_t *a, const relay_tensor_t *b, relay_tensor_t *out);
+
+/* Type of value `value` of an elementwise program over the given inputs (Fig. 5 rules applied
+ * instruction by instruction after broadcasting all inputs to one shape). */
+relay_status_t relay_infer_ewise(const relay_ewise_prog_t *prog, const relay_tensor_t *const *inputs,
+                                 int32_t n_in, int32_t value, relay_tensor_t *out);
+
+/* Reduction result: axes in axes_mask removed (or kept as 1).  out_dtype: f32 for sum/max/mean
+ * of float input, i64 for argmax. */
+relay_status_t relay_infer_reduce(const relay_tensor_t *in, int32_t red_op, int32_t axes_mask,
+                                  int32_t keepdims, relay_tensor_t *out);
+
+/* Tensor literal (Fig. 5 Type-Tensor-Literal): m tensors of type Tensor(b, Shape(d1..dn))
+ * stack to Tensor(b, Shape(m, d1..dn)). */
+relay_status_t relay_infer_stack(const relay_tensor_t *elem, int64_t m, relay_tensor_t *out);
+
+/* LSTM sequence: x:(T,B,I), w_ih:(I,4H), w_hh:(H,4H) -> h_all:(T,B,H) f32, c_final:(B,H) f32. */
+relay_status_t relay_infer_lstm(const relay_tensor_t *x, const relay_tensor_t *w_ih, const relay_tensor_t *w_hh,
+                                relay_tensor_t *h_all, relay_tensor_t *c_final);
+
+/* ---------------------------------------------------------------------------------------------
+ * Workspace queries, host only.  Return the scratch bytes the matching call needs for these
+ * argument types (0 if the types are invalid; the call itself reports why).
+ * ------------------------------------------------------------------------------------------- */
+size_t relay_workspace_bytes_dense_act(const relay_tensor_t *x, const relay_tensor_t *w);
+size_t relay_workspace_bytes_dense_act_grad(const relay_tensor_t *x, const relay_tensor_t *w);
+size_t relay_workspace_bytes_conv2d_act(const relay_tensor_t *x, const relay_tensor_t *w,
+                                        const relay_conv2d_attrs_t *attrs);
+size_t relay_workspace_bytes_conv2d_act_grad(const relay_tensor_t *x, const relay_tensor_t *w,
+                                             const relay_conv2d_attrs_t *attrs);
+size_t relay_workspace_bytes_reduce(const relay_tensor_t *const *inputs, int32_t n_in,
+                                    const relay_out_spec_t *specs, int32_t n_out);
+size_t relay_workspace_bytes_lstm(const relay_tensor_t *x, const relay_tensor_t *w_ih, const relay_tensor_t *w_hh);
+
+/* ---------------------------------------------------------------------------------------------
+ * Compute entry points.
+ * ------------------------------------------------------------------------------------------- */
+
+/* Dense anchor fused with broadcast bias and elementwise activation (Fig. 3: relay.linear
+ * followed by an elementwise operator; fusion of such chains is the optimisation Section 5.2
+ * names):   y[m,n] = act( sum_k x[m,k] * w[k,n] + b[n] ).
+ *   x:(M,K)  w:(K,N)  b:(N) or NULL  ->  y:(M,N); x, w, y share one dtype t in {f32, bf16};
+ *   b has dtype t or f32.  f32 runs in true fp32 (FMA); bf16 multiplies bf16 and accumulates
+ *   in fp32, rounding once on the store of y. */
+relay_status_t relay_fused_dense_act(const relay_tensor_t *x, const relay_tensor_t *w, const relay_tensor_t *b,
+                                     int32_t act, const relay_tensor_t *y, void *ws, size_t ws_bytes, void *stream);
+
+/* Gradient group of the dense anchor (Section 4.2: reverse mode; `dy` is the partial of the
+ * program's final scalar with respect to y, each returned tensor the partial with respect to
+ * the argument of the same name; the pair (forward call, this call) is what `Grad` returns:
+ * the original result bundled with all partials).
+ *   dZ = dy (.) act'(y)  with act' taken from the SAVED forward output y:
+ *        relu' = 1[y>0] (so relu'(0)=0), tanh' = 1-y^2, sigmoid' = y(1-y);
+ *   dx[m,k] = sum_n dZ[m,n] w[k,n];   dw[k,n] = sum_m x[m,k] dZ[m,n];   db[n] = sum_m dZ[m,n].
+ *   dx, db may be NULL (not wanted); dw is required.  dx, dw have dtype t; db is f32 (or t for
+ *   t = f32).  Sums are deterministic (fixed order, no float atomics). */
+relay_status_t relay_fused_dense_act_grad(const relay_tensor_t *x, const relay_tensor_t *w, const relay_tensor_t *y,
+                                          const relay_tensor_t *dy, int32_t act, const relay_tensor_t *dx,
+                                          const relay_tensor_t *dw, const relay_tensor_t *db, void *ws,
+                                          size_t ws_bytes, void *stream);
+
+/* conv2d anchor (Fig. 3 relay.conv2d) as cross-correlation with zero padding, run as an
+ * implicit GEMM and fused with per-channel bias and activation:
+ *   y[n,o,p,q] = act( b[o] + sum_{c,r,s} x[n,c,p*st-pad+r,q*st-pad+s] * w[o,c,r,s] ).
+ *   x:(N,C,H,W) NCHW  w:(O,C,R,S) OIHW  b:(O) or NULL  ->  y:(N,O,P,Q) NCHW. */
+relay_status_t relay_fused_conv2d_act(const relay_tensor_t *x, const relay_tensor_t *w, const relay_tensor_t *b,
+                                      const relay_conv2d_attrs_t *attrs, int32_t act, const relay_tensor_t *y,
+                                      void *ws, size_t ws_bytes, void *stream);
+
+/* Gradient group of the conv2d anchor (Section 4.2), dZ = dy (.) act'(y) as above:
+ *   dx[n,c,i,j]  = sum_{o,r,s} dZ[n,o,p,q] w[o,c,r,s]   over (p,q) with p*st-pad+r=i, q*st-pad+s=j
+ *   dw[o,c,r,s]  = sum_{n,p,q} dZ[n,o,p,q] x[n,c,p*st-pad+r,q*st-pad+s]
+ *   db[o]        = sum_{n,p,q} dZ[n,o,p,q]
+ *   dx, db may be NULL; dw is required. */
+relay_status_t relay_fused_conv2d_act_grad(const relay_tensor_t *x, const relay_tensor_t *w, const relay_tensor_t *y,
+                                           const relay_tensor_t *dy, const relay_conv2d_attrs_t *attrs, int32_t act,
+                                           const relay_tensor_t *dx, const relay_tensor_t *dw,
+                                           const relay_tensor_t *db, void *ws, size_t ws_bytes, void *stream);
+
+/* Fused broadcast-elementwise group (Fig. 1 BinOp/UnaryOp/cast; Fig. 5 typing; Section 5.2
+ * operator fusion): evaluates `prog` at every index of the broadcast shape and stores the
+ * values named in out_values[0..n_out) to outputs[k], whose type must equal the value's
+ * inferred type (full broadcast shape). */
+relay_status_t relay_fused_ewise(const relay_ewise_prog_t *prog, const relay_tensor_t *const *inputs, int32_t n_in,
+                                 const int32_t *out_values, const relay_tensor_t *const *outputs, int32_t n_out,
+                                 void *ws, size_t ws_bytes, void *stream);
+
+/* Fused elementwise + reduce group (Fig. 3 relay.argmax and the reduction inside
+ * softmax_cross_entropy; the column sums a gradient program needs where a value was broadcast,
+ * Section 5.2 "summing in the correct places"): evaluates `prog` (may have 0 instructions) and
+ * for each spec stores the value unreduced or reduced.  sum/max/mean outputs are f32 (bf16
+ * allowed for unreduced values per their type); argmax outputs are i64 positions inside the
+ * reduced axes, the first maximum winning.  Reductions are deterministic. */
+relay_status_t relay_fused_reduce(const relay_ewise_prog_t *prog, const relay_tensor_t *const *inputs, int32_t n_in,
+                                  const relay_out_spec_t *specs, const relay_tensor_t *const *outputs,
+                                  int32_t n_out, void *ws, size_t ws_bytes, void *stream);
+
+/* LSTM cell applied over a sequence (a recursive program over time composed of the dense
+ * anchor and elementwise gates; recursion is what Section 3.1 adds over dataflow graphs).
+ * Gate blocks along the 4H axis are [ i | f | g | o ]:
+ *   z = x_t w_ih + bf16(h) w_hh + b;  i,f,o = sigmoid(z_i,z_f,z_o);  g = tanh(z_g);
+ *   c = f (.) c + i (.) g;  h = o (.) tanh(c)                      (c, h kept in f32)
+ *   x:(T,B,I) bf16  w_ih:(I,4H) bf16  w_hh:(H,4H) bf16  b:(4H) f32  h0,c0:(B,H) f32
+ *   -> h_all:(T,B,H) f32, c_final:(B,H) f32. */
+relay_status_t relay_lstm_cell_seq(const relay_tensor_t *x, const relay_tensor_t *w_ih, const relay_tensor_t *w_hh,
+                                   const relay_tensor_t *b, const relay_tensor_t *h0, const relay_tensor_t *c0,
+                                   const relay_tensor_t *h_all, const relay_tensor_t *c_final, void *ws,
+                                   size_t ws_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Status helpers.
+ * ------------------------------------------------------------------------------------------- */
+
+/* Thread-local text describing the last non-OK status returned on this thread ("" if none). */
+const char *relay_last_error(void);
+
+/* Synchronises `stream`, then reads and clears the device-side error word of the current
+ * device: RELAY_ERR_TIMEOUT if a bounded wait expired in any kernel since the last poll,
+ * RELAY_ERR_CUDA if the stream reports an error, else RELAY_OK. */
+relay_status_t relay_poll_status(void *stream);
+
+/* Number of kernels this library has launched on this process so far (monotonic counter). */
+int64_t relay_launch_count(void);
+
+/* Library version string. */
+const char *relay_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RELAY_B200_H_ */

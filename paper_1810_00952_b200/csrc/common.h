@@ -1,0 +1,99 @@
+// Internal helpers shared by the host-side entry points: status reporting, descriptor checks
+// (the type relations of Fig. 4 / Fig. 5 applied to concrete tensors), launch accounting.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdarg>
+#include <cstdint>
+#include <cstdio>
+
+#include "../../include/relay_b200.h"
+
+namespace relay {
+
+// ---- status -----------------------------------------------------------------------------------
+relay_status_t fail(relay_status_t st, const char *fmt, ...);  // records text, returns st
+void clear_error();
+void count_launch(int n = 1);
+
+#define RELAY_TRY(expr)                                   \
+    do {                                                  \
+        relay_status_t st__ = (expr);                     \
+        if (st__ != RELAY_OK) return st__;                \
+    } while (0)
+
+#define RELAY_CUDA(expr)                                                                        \
+    do {                                                                                        \
+        cudaError_t e__ = (expr);                                                               \
+        if (e__ != cudaSuccess)                                                                 \
+            return ::relay::fail(RELAY_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e__)); \
+    } while (0)
+
+// checks the launch that was just issued
+relay_status_t check_launch(const char *what);
+
+// ---- descriptors --------------------------------------------------------------------------------
+inline size_t dtype_size(int32_t dt)
+{
+    switch (dt) {
+    case RELAY_F32: return 4;
+    case RELAY_BF16: return 2;
+    case RELAY_I32: return 4;
+    case RELAY_I64: return 8;
+    case RELAY_BOOL: return 1;
+    default: return 0;
+    }
+}
+inline bool is_float(int32_t dt) { return dt == RELAY_F32 || dt == RELAY_BF16; }
+inline const char *dtype_name(int32_t dt)
+{
+    switch (dt) {
+    case RELAY_F32: return "f32";
+    case RELAY_BF16: return "bf16";
+    case RELAY_I32: return "i32";
+    case RELAY_I64: return "i64";
+    case RELAY_BOOL: return "bool";
+    default: return "?";
+    }
+}
+
+inline int64_t numel(const relay_tensor_t *t)
+{
+    int64_t n = 1;
+    for (int d = 0; d < t->rank; ++d) n *= t->shape[d];
+    return n;
+}
+inline size_t nbytes(const relay_tensor_t *t) { return (size_t)numel(t) * dtype_size(t->dtype); }
+
+// Tensor-T / Shape-T / BaseType-T on a concrete descriptor: known base type, rank in range,
+// extents natural numbers.  Does not look at `data`.
+relay_status_t check_type(const relay_tensor_t *t, const char *name);
+
+// Stage-wise checks used by the entry points so that the first failing rule is reported in the
+// documented order.
+relay_status_t check_not_null(const void *p, const char *name);
+relay_status_t check_rank(const relay_tensor_t *t, int rank, const char *name);
+relay_status_t check_dtype(const relay_tensor_t *t, int32_t dt, const char *name);
+relay_status_t check_layout(const relay_tensor_t *t, int32_t a, int32_t b, const char *name);
+relay_status_t check_shape(const relay_tensor_t *t, std::initializer_list<int64_t> want, const char *name);
+relay_status_t check_data(const relay_tensor_t *t, const char *name);  // non-null (if numel>0), 16 B aligned
+relay_status_t check_workspace(const void *ws, size_t have, size_t need);
+
+struct Span { const char *lo, *hi; };
+inline Span span_of(const relay_tensor_t *t)
+{
+    const char *p = (const char *)t->data;
+    return Span{p, p + nbytes(t)};
+}
+// outputs must not overlap inputs or each other
+relay_status_t check_no_overlap(const relay_tensor_t *const *outs, int n_out, const relay_tensor_t *const *ins,
+                                int n_in);
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// device-side error word (set by kernels whose bounded waits expire)
+int *device_error_word();  // device address of the word on the current device (nullptr on failure)
+
+}  // namespace relay

@@ -1,0 +1,28 @@
+// Shapes of one conv2d instance and the kernel tiers that run it.
+#pragma once
+#include "common.h"
+
+namespace relay {
+
+struct ConvDims {
+    int64_t Nb = 0, C = 0, H = 0, W = 0, O = 0, R = 0, S = 0, P = 0, Q = 0;
+    int32_t stride = 1, pad = 0, dt = RELAY_F32;
+};
+
+// direct (SIMT) tier: any stride / pad / window, fp32 accumulation in a fixed order
+relay_status_t launch_conv_fwd_direct(const ConvDims &d, const void *x, const void *w, const void *b, int32_t b_dt, int act,
+                                      void *y, cudaStream_t st);
+relay_status_t launch_conv_dx_direct(const ConvDims &d, const void *dz, const void *w, void *dx, cudaStream_t st);
+relay_status_t launch_conv_dw_direct(const ConvDims &d, const void *dz, const void *x, void *dw, cudaStream_t st);
+relay_status_t launch_conv_db(const ConvDims &d, const void *dz, float *db, cudaStream_t st);
+
+// implicit-GEMM tensor-core tier (3x3, stride 1, pad 1, bf16)
+bool conv_tc_eligible(const ConvDims &d);
+size_t conv_tc_fwd_workspace(const ConvDims &d);
+size_t conv_tc_grad_workspace(const ConvDims &d);
+relay_status_t launch_conv_fwd_tc(const ConvDims &d, const void *x, const void *w, const void *b, int32_t b_dt, int act, void *y,
+                                  void *ws, cudaStream_t st);
+relay_status_t launch_conv_dx_tc(const ConvDims &d, const void *dz, const void *w, void *dx, void *ws, cudaStream_t st);
+relay_status_t launch_conv_dw_tc(const ConvDims &d, const void *dz, const void *x, void *dw, void *ws, cudaStream_t st);
+
+}  // namespace relay

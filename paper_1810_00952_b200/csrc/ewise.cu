@@ -1,0 +1,691 @@
+// Memory-bound groups: fused broadcast-elementwise (relay_fused_ewise) and fused
+// elementwise + reduce (relay_fused_reduce).
+//
+// Two tiers of kernels, both on the GPU:
+//   * pre-compiled bodies over a collapsed 2-D view [rows, cols]: 128-bit loads/stores, operands
+//     that are broadcast down the rows kept in registers, several rows in flight per thread,
+//     column sums as per-thread accumulators -> shared-memory combine -> per-slice partials ->
+//     a second fixed-order pass (deterministic, no float atomics);
+//   * a generic evaluator that interprets any well-typed program for any broadcast pattern and
+//     any axes mask (one element per thread; one warp or one block per reduced result).
+#include <algorithm>
+#include <cstring>
+#include <string>
+
+#include "ewise_host.h"
+#include "ewise_kernels.cuh"
+#include "ewise_prog.h"
+
+namespace relay {
+
+// =================================================================================================
+// kernels
+// =================================================================================================
+constexpr int kTX = 32, kTY = 8, kUnroll = 4;
+
+template <typename Body, typename T, bool FAST>
+__global__ void __launch_bounds__(kTX *kTY, Body::NIN >= 4 ? 2 : 3) ewise2d_kernel(const Args2D<Body::NIN, Body::NOUT> A)
+{
+    constexpr int V = VecN<T>::N, NIN = Body::NIN, NOUT = Body::NOUT;
+    const int tx = threadIdx.x, ty = threadIdx.y;
+    const int64_t col0 = ((int64_t)blockIdx.x * kTX + tx) * V;
+    const bool active = col0 < A.cols;
+
+    float fixed[NIN][V];  // operands that do not change from row to row
+#pragma unroll
+    for (int i = 0; i < NIN; ++i) {
+        if (Body::kind(i) == KIND_ROWVEC && active) {
+            unpack(ld_stream((const T *)A.in[i] + col0), fixed[i]);
+        } else if (Body::kind(i) == KIND_SCALAR) {
+            float s;
+            if constexpr (sizeof(T) == 2) s = __bfloat162float(*(const __nv_bfloat16 *)A.in[i]);
+            else s = *(const float *)A.in[i];
+#pragma unroll
+            for (int v = 0; v < V; ++v) fixed[i][v] = s;
+        } else {
+#pragma unroll
+            for (int v = 0; v < V; ++v) fixed[i][v] = 0.0f;
+        }
+    }
+
+    float acc[NOUT][V];
+#pragma unroll
+    for (int k = 0; k < NOUT; ++k)
+#pragma unroll
+        for (int v = 0; v < V; ++v) acc[k][v] = 0.0f;
+
+    const int64_t r0 = (int64_t)blockIdx.y * A.rows_per_slice;
+    const int64_t r1 = min(A.rows, r0 + (int64_t)A.rows_per_slice);
+
+    if (active) {
+        for (int64_t r = r0 + ty; r < r1; r += kTY * kUnroll) {
+            uint4 raw[kUnroll][NIN];
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                const int64_t rr = r + u * kTY;
+#pragma unroll
+                for (int i = 0; i < NIN; ++i)
+                    if (Body::kind(i) == KIND_FULL && rr < r1) raw[u][i] = ld_stream((const T *)A.in[i] + rr * A.cols + col0);
+            }
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                const int64_t rr = r + u * kTY;
+                if (rr >= r1) break;
+                float vin[NIN][V];
+#pragma unroll
+                for (int i = 0; i < NIN; ++i) {
+                    if (Body::kind(i) == KIND_FULL) unpack(raw[u][i], vin[i]);
+                    else {
+#pragma unroll
+                        for (int v = 0; v < V; ++v) vin[i][v] = fixed[i][v];
+                    }
+                }
+                float vout[NOUT][V];
+#pragma unroll
+                for (int v = 0; v < V; ++v) {
+                    float ein[NIN], eout[NOUT];
+#pragma unroll
+                    for (int i = 0; i < NIN; ++i) ein[i] = vin[i][v];
+                    Body::template apply<FAST>(ein, eout, A.aux);
+#pragma unroll
+                    for (int k = 0; k < NOUT; ++k) vout[k][v] = eout[k];
+                }
+#pragma unroll
+                for (int k = 0; k < NOUT; ++k) {
+                    if (Body::col_sum(k)) {
+#pragma unroll
+                        for (int v = 0; v < V; ++v) acc[k][v] += vout[k][v];
+                    }
+                    if (A.out[k] != nullptr) st_stream((T *)A.out[k] + rr * A.cols + col0, pack(vout[k]));
+                }
+            }
+        }
+    }
+
+    // combine the kTY row-threads of each column, in ty order, and publish one partial per slice
+    constexpr bool any_sum = []() { bool s = false; for (int k = 0; k < NOUT; ++k) s = s || Body::col_sum(k); return s; }();
+    if constexpr (any_sum) {
+        __shared__ float sm[kTY][kTX * V + 1];
+#pragma unroll
+        for (int k = 0; k < NOUT; ++k) {
+            if (!Body::col_sum(k)) continue;
+#pragma unroll
+            for (int v = 0; v < V; ++v) sm[ty][tx * V + v] = acc[k][v];
+            __syncthreads();
+            if (ty == 0 && active && A.partial[k] != nullptr) {
+#pragma unroll
+                for (int v = 0; v < V; ++v) {
+                    float s = 0.0f;
+#pragma unroll
+                    for (int j = 0; j < kTY; ++j) s += sm[j][tx * V + v];
+                    A.partial[k][(int64_t)blockIdx.y * A.cols + col0 + v] = s;
+                }
+            }
+            __syncthreads();
+        }
+    }
+}
+
+// second pass of a column sum: adds the per-slice partials in slice order
+__global__ void colsum_finalize_kernel(const float *__restrict__ partial, int n_slices, int64_t cols, float scale,
+                                       float *__restrict__ out)
+{
+    int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= cols) return;
+    float s = 0.0f;
+    for (int j = 0; j < n_slices; ++j) s += partial[(int64_t)j * cols + c];
+    out[c] = s * scale;
+}
+
+// reduction over the last axis of a [rows, cols] tensor: one warp per row, 128-bit loads
+template <typename T, int RED>
+__global__ void __launch_bounds__(256) rowreduce_kernel(const T *__restrict__ in, int64_t rows, int64_t cols, float scale,
+                                                         void *__restrict__ out)
+{
+    constexpr int V = VecN<T>::N;
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    const T *p = in + row * cols;
+    const int64_t nvec = cols / V;
+    float best = RED == RELAY_RED_SUM ? 0.0f : -INFINITY;
+    int64_t pos = 0;
+    for (int64_t j = lane; j < nvec; j += 32 * kUnroll) {
+        uint4 raw[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+            if (j + u * 32 < nvec) raw[u] = ld_stream(p + (j + u * 32) * V);
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            if (j + u * 32 >= nvec) break;
+            float f[V];
+            unpack(raw[u], f);
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+                if (RED == RELAY_RED_SUM) best += f[v];
+                else if (f[v] > best) { best = f[v]; pos = (j + u * 32) * V + v; }
+            }
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        float ob = __shfl_xor_sync(0xffffffffu, best, o);
+        int64_t op = __shfl_xor_sync(0xffffffffu, pos, o);
+        if (RED == RELAY_RED_SUM) best += ob;
+        else if (ob > best || (ob == best && op < pos)) { best = ob; pos = op; }
+    }
+    if (lane == 0) {
+        if (RED == RELAY_RED_ARGMAX) ((int64_t *)out)[row] = pos;
+        else ((float *)out)[row] = best * scale;
+    }
+}
+
+struct DevOutputs {
+    int32_t n_out;
+    int32_t value[RELAY_MAX_OUTPUTS];
+    int32_t dtype[RELAY_MAX_OUTPUTS];
+    void *ptr[RELAY_MAX_OUTPUTS];
+};
+
+__global__ void __launch_bounds__(256) ewise_generic_kernel(const DevProgram P, const DevOutputs O, int64_t total)
+{
+    float vals[kDevMaxValues];
+    int64_t idx[RELAY_MAX_RANK];
+    for (int64_t lin = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; lin < total; lin += (int64_t)gridDim.x * blockDim.x) {
+        unravel(lin, P.rank, P.shape, idx);
+        eval_program(P, idx, vals);
+        for (int k = 0; k < O.n_out; ++k) store_from_float(O.ptr[k], lin, O.dtype[k], vals[O.value[k]]);
+    }
+}
+
+struct DevReduce {
+    int32_t red_op, value, n_kept, n_red;
+    int32_t kept_axis[RELAY_MAX_RANK], red_axis[RELAY_MAX_RANK];
+    int64_t kept_elems, red_elems;
+    void *out;
+    float scale;
+    int32_t group;  // threads that share one result: 32 (a warp) or 256 (the block)
+};
+
+__device__ __forceinline__ void combine(int red_op, float &best, int64_t &pos, float ob, int64_t op)
+{
+    if (red_op == RELAY_RED_SUM || red_op == RELAY_RED_MEAN) best += ob;
+    else if (ob > best || (ob == best && op < pos)) { best = ob; pos = op; }
+}
+
+// one warp (group 32) or one block (group 256) per reduced result; fixed combine order
+__global__ void __launch_bounds__(256) reduce_generic_kernel(const DevProgram P, const DevReduce R)
+{
+    __shared__ float sbest[8];
+    __shared__ long long spos[8];
+    float vals[kDevMaxValues];
+    int64_t idx[RELAY_MAX_RANK];
+    const int lane_in_group = threadIdx.x % R.group;
+    const int groups_per_block = blockDim.x / R.group;
+    const int64_t kept = (int64_t)blockIdx.x * groups_per_block + threadIdx.x / R.group;
+    const bool live = kept < R.kept_elems;
+    const bool is_sum = R.red_op == RELAY_RED_SUM || R.red_op == RELAY_RED_MEAN;
+    float best = is_sum ? 0.0f : -INFINITY;
+    int64_t pos = 0;
+    if (live) {
+        int64_t rem = kept;
+        for (int i = R.n_kept - 1; i >= 0; --i) {
+            int ax = R.kept_axis[i];
+            idx[ax] = rem % P.shape[ax];
+            rem /= P.shape[ax];
+        }
+        for (int64_t j = lane_in_group; j < R.red_elems; j += R.group) {
+            int64_t rj = j;
+            for (int i = R.n_red - 1; i >= 0; --i) {
+                int ax = R.red_axis[i];
+                idx[ax] = rj % P.shape[ax];
+                rj /= P.shape[ax];
+            }
+            eval_program(P, idx, vals);
+            float v = vals[R.value];
+            if (is_sum) best += v;
+            else if (v > best) { best = v; pos = j; }
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        float ob = __shfl_xor_sync(0xffffffffu, best, o);
+        int64_t op = __shfl_xor_sync(0xffffffffu, pos, o);
+        combine(R.red_op, best, pos, ob, op);
+    }
+    if (R.group > 32) {
+        const int warp = threadIdx.x >> 5;
+        if ((threadIdx.x & 31) == 0) { sbest[warp] = best; spos[warp] = pos; }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            best = sbest[0]; pos = spos[0];
+            for (int w = 1; w < (int)(blockDim.x >> 5); ++w) combine(R.red_op, best, pos, sbest[w], spos[w]);
+        }
+    }
+    if (live && lane_in_group == 0) {
+        if (R.red_op == RELAY_RED_ARGMAX) ((int64_t *)R.out)[kept] = pos;
+        else ((float *)R.out)[kept] = best * R.scale;
+    }
+}
+
+// =================================================================================================
+// host: canonical form of a program value, used to pick a pre-compiled body
+// =================================================================================================
+static bool commutative(int op)
+{
+    return op == RELAY_OP_ADD || op == RELAY_OP_MUL || op == RELAY_OP_MAX || op == RELAY_OP_MIN || op == RELAY_OP_EQ || op == RELAY_OP_NE;
+}
+
+// Expression tree of a value written as text, operands of commutative operators sorted, so
+// that two programs that compute the same expression compare equal whatever their let order.
+static std::string canon(const TypedProgram &tp, int v, int depth = 0)
+{
+    if (depth > 24) return "?";
+    char buf[64];
+    if (v < tp.n_in) { snprintf(buf, sizeof buf, "i%d:%d", v, tp.dtype[v]); return buf; }
+    const relay_instr_t &in = tp.instr[v - tp.n_in];
+    if (in.op == RELAY_OP_CONST) { snprintf(buf, sizeof buf, "k%.9g:%d", in.imm, in.dtype); return buf; }
+    std::string args[3];
+    int n = 0;
+    if (in.a >= 0) args[n++] = canon(tp, in.a, depth + 1);
+    if (in.b >= 0) args[n++] = canon(tp, in.b, depth + 1);
+    if (in.c >= 0) args[n++] = canon(tp, in.c, depth + 1);
+    if (commutative(in.op) && n == 2 && args[1] < args[0]) std::swap(args[0], args[1]);
+    snprintf(buf, sizeof buf, "o%d:%d(", in.op, in.dtype);
+    std::string s = buf;
+    for (int i = 0; i < n; ++i) { if (i) s += ","; s += args[i]; if (s.size() > 4096) return "?"; }
+    return s + ")";
+}
+
+// canonical text of the benchmark groups' values, produced from the same typed-program machinery
+static void build(TypedProgram &tp, int n_in, int32_t in_dt)
+{
+    tp = TypedProgram();
+    tp.n_in = n_in;
+    for (int i = 0; i < n_in; ++i) tp.dtype[i] = in_dt;
+}
+static int emit(TypedProgram &tp, int op, int a, int b, int c, int dt, double imm = 0.0)
+{
+    relay_instr_t &in = tp.instr[tp.n_instr];
+    in.op = op; in.a = a; in.b = b; in.c = c; in.dtype = dt; in.imm = imm; in.reserved = 0;
+    tp.dtype[tp.n_in + tp.n_instr] = dt;
+    tp.n_values = tp.n_in + tp.n_instr + 1;
+    return tp.n_in + tp.n_instr++;
+}
+
+struct KnownFwd { std::string out; };
+struct KnownGrad { std::string dx, da, db; };
+
+static KnownFwd known_tanh_affine_fwd(int32_t st)
+{
+    TypedProgram p; build(p, 3, st);
+    const int F = RELAY_F32;
+    int x = emit(p, RELAY_OP_CAST, 0, -1, -1, F), a = emit(p, RELAY_OP_CAST, 1, -1, -1, F), b = emit(p, RELAY_OP_CAST, 2, -1, -1, F);
+    int u = emit(p, RELAY_OP_ADD, emit(p, RELAY_OP_MUL, a, x, -1, F), b, -1, F);
+    int o = emit(p, RELAY_OP_ADD, emit(p, RELAY_OP_TANH, u, -1, -1, F), x, -1, F);
+    return KnownFwd{canon(p, emit(p, RELAY_OP_CAST, o, -1, -1, st))};
+}
+static KnownGrad known_tanh_affine_grad(int32_t st)
+{
+    TypedProgram p; build(p, 4, st);
+    const int F = RELAY_F32;
+    int d = emit(p, RELAY_OP_CAST, 0, -1, -1, F), x = emit(p, RELAY_OP_CAST, 1, -1, -1, F);
+    int a = emit(p, RELAY_OP_CAST, 2, -1, -1, F), b = emit(p, RELAY_OP_CAST, 3, -1, -1, F);
+    int t = emit(p, RELAY_OP_TANH, emit(p, RELAY_OP_ADD, emit(p, RELAY_OP_MUL, a, x, -1, F), b, -1, F), -1, -1, F);
+    int one = emit(p, RELAY_OP_CONST, -1, -1, -1, F, 1.0);
+    int s = emit(p, RELAY_OP_SUB, one, emit(p, RELAY_OP_SQ, t, -1, -1, F), -1, F);
+    int g = emit(p, RELAY_OP_ADD, emit(p, RELAY_OP_MUL, a, s, -1, F), one, -1, F);
+    int dx = emit(p, RELAY_OP_CAST, emit(p, RELAY_OP_MUL, d, g, -1, F), -1, -1, st);
+    int ds = emit(p, RELAY_OP_MUL, d, s, -1, F);
+    int da = emit(p, RELAY_OP_MUL, ds, x, -1, F);
+    return KnownGrad{canon(p, dx), canon(p, da), canon(p, ds)};
+}
+
+// =================================================================================================
+// host: launches
+// =================================================================================================
+static void fill_dev_program(const TypedProgram &tp, const relay_tensor_t *const *inputs, DevProgram *P)
+{
+    memset(P, 0, sizeof(*P));
+    P->n_in = tp.n_in; P->n_instr = tp.n_instr; P->rank = tp.rank;
+    for (int d = 0; d < tp.rank; ++d) P->shape[d] = tp.shape[d];
+    for (int i = 0; i < tp.n_in; ++i) {
+        int64_t stride = 1;
+        for (int d = tp.rank - 1; d >= 0; --d) {
+            P->in_stride[i][d] = tp.in_shape[i][d] == 1 ? 0 : stride;
+            stride *= tp.in_shape[i][d];
+        }
+        P->in_ptr[i] = inputs[i]->data;
+        P->in_dtype[i] = (int8_t)inputs[i]->dtype;
+    }
+    for (int j = 0; j < tp.n_instr; ++j) {
+        P->op[j] = (int8_t)tp.instr[j].op; P->a[j] = (int8_t)tp.instr[j].a; P->b[j] = (int8_t)tp.instr[j].b;
+        P->c[j] = (int8_t)tp.instr[j].c; P->dt[j] = (int8_t)tp.instr[j].dtype; P->imm[j] = (float)tp.instr[j].imm;
+    }
+}
+
+// 2-D view: is every input either full-shape, constant down the rows, or a scalar, all in one
+// float storage type, with whole 16-byte vectors per row?
+struct View2D { bool ok; int64_t rows, cols; int kind[RELAY_MAX_INPUTS]; int32_t storage; };
+
+static View2D view2d(const TypedProgram &tp)
+{
+    View2D v{};
+    v.ok = false;
+    if (tp.rank < 1 || tp.n_in < 1 || tp.total == 0) return v;
+    v.cols = tp.shape[tp.rank - 1];
+    v.rows = tp.total / v.cols;
+    v.storage = tp.dtype[0];
+    if (!is_float(v.storage)) return v;
+    const int vec = v.storage == RELAY_BF16 ? 8 : 4;
+    if (v.cols % vec != 0) return v;
+    for (int i = 0; i < tp.n_in; ++i) {
+        if (tp.dtype[i] != v.storage) return v;
+        bool full = true, lead1 = true;
+        for (int d = 0; d < tp.rank; ++d) {
+            if (tp.in_shape[i][d] != tp.shape[d]) full = false;
+            if (d < tp.rank - 1 && tp.in_shape[i][d] != 1) lead1 = false;
+        }
+        if (full) v.kind[i] = KIND_FULL;
+        else if (lead1 && tp.in_shape[i][tp.rank - 1] == v.cols) v.kind[i] = KIND_ROWVEC;
+        else if (lead1 && tp.in_shape[i][tp.rank - 1] == 1) v.kind[i] = KIND_SCALAR;
+        else return v;
+    }
+    v.ok = true;
+    return v;
+}
+
+template <typename Body>
+static bool kinds_match(const View2D &v)
+{
+    for (int i = 0; i < Body::NIN; ++i)
+        if (v.kind[i] != Body::kind(i)) return false;
+    return true;
+}
+
+int colsum_slices(int64_t rows, int64_t cols, int32_t storage)
+{
+    const int vec = storage == RELAY_BF16 ? 8 : 4;
+    const int64_t gx = (cols + (int64_t)kTX * vec - 1) / (kTX * vec);
+    // about 8 blocks of 256 threads per SM in total, but at least 32 rows per slice
+    int64_t want = std::max<int64_t>(1, (148 * 8) / gx);
+    int64_t max_by_rows = std::max<int64_t>(1, rows / 32);
+    return (int)std::max<int64_t>(1, std::min(want, max_by_rows));
+}
+
+template <typename Body>
+relay_status_t launch_body2d(int32_t storage, const Args2D<Body::NIN, Body::NOUT> &A0, int n_slices, cudaStream_t st,
+                             const char *what)
+{
+    Args2D<Body::NIN, Body::NOUT> A = A0;
+    const int vec = storage == RELAY_BF16 ? 8 : 4;
+    dim3 block(kTX, kTY);
+    dim3 grid((unsigned)((A.cols + (int64_t)kTX * vec - 1) / (kTX * vec)), (unsigned)n_slices);
+    A.rows_per_slice = (int)((A.rows + n_slices - 1) / n_slices);
+    if (storage == RELAY_BF16) ewise2d_kernel<Body, __nv_bfloat16, true><<<grid, block, 0, st>>>(A);
+    else ewise2d_kernel<Body, float, false><<<grid, block, 0, st>>>(A);
+    return check_launch(what);
+}
+
+relay_status_t launch_colsum_finalize(const float *partial, int n_slices, int64_t cols, float scale, float *out,
+                                      cudaStream_t st)
+{
+    colsum_finalize_kernel<<<(unsigned)((cols + 255) / 256), 256, 0, st>>>(partial, n_slices, cols, scale, out);
+    return check_launch("colsum_finalize");
+}
+
+// dZ = dy (.) act'(y) stored to dz, and (if db) db = column sums of dZ; used by the dense gradient group
+relay_status_t launch_act_grad(int32_t storage, const void *dy, const void *y, void *dz, float *db, float *partials,
+                               int64_t rows, int64_t cols, int act, cudaStream_t st)
+{
+    Args2D<2, 2> A{};
+    A.in[0] = dy; A.in[1] = y;
+    A.out[0] = dz; A.out[1] = nullptr;
+    A.partial[0] = nullptr; A.partial[1] = db ? partials : nullptr;
+    A.rows = rows; A.cols = cols; A.aux = act;
+    const int ns = colsum_slices(rows, cols, storage);
+    RELAY_TRY(launch_body2d<BodyActGrad>(storage, A, ns, st, "act_grad"));
+    if (db) RELAY_TRY(launch_colsum_finalize(partials, ns, cols, 1.0f, db, st));
+    return RELAY_OK;
+}
+
+static relay_status_t check_output(const relay_tensor_t *o, int32_t dtype, int rank, const int64_t *shape, int k)
+{
+    char name[32];
+    snprintf(name, sizeof name, "outputs[%d]", k);
+    RELAY_TRY(check_type(o, name));
+    RELAY_TRY(check_rank(o, rank, name));
+    RELAY_TRY(check_dtype(o, dtype, name));
+    for (int d = 0; d < rank; ++d)
+        if (o->shape[d] != shape[d])
+            return fail(RELAY_ERR_SHAPE, "%s: axis %d has extent %lld, the group's type gives %lld", name, d, (long long)o->shape[d],
+                        (long long)shape[d]);
+    return RELAY_OK;
+}
+
+static unsigned grid_for(int64_t total, int threads)
+{
+    int64_t g = (total + threads - 1) / threads;
+    return (unsigned)std::max<int64_t>(1, std::min<int64_t>(g, 148 * 16));
+}
+
+}  // namespace relay
+
+using namespace relay;
+
+extern "C" relay_status_t relay_fused_ewise(const relay_ewise_prog_t *prog, const relay_tensor_t *const *inputs, int32_t n_in,
+                                            const int32_t *out_values, const relay_tensor_t *const *outputs, int32_t n_out,
+                                            void *ws, size_t ws_bytes, void *stream)
+{
+    (void)ws; (void)ws_bytes;
+    clear_error();
+    TypedProgram tp;
+    RELAY_TRY(check_not_null(out_values, "out_values"));
+    RELAY_TRY(check_not_null(outputs, "outputs"));
+    if (n_out < 1 || n_out > RELAY_MAX_OUTPUTS) return fail(RELAY_ERR_ATTR, "%d outputs, 1..%d allowed", n_out, RELAY_MAX_OUTPUTS);
+    for (int k = 0; k < n_out; ++k) RELAY_TRY(check_not_null(outputs[k], "outputs[k]"));
+    RELAY_TRY(type_program(prog, inputs, n_in, &tp));
+    if (n_in < 1) return fail(RELAY_ERR_ATTR, "an elementwise group needs at least one input");
+    for (int k = 0; k < n_out; ++k) {
+        if (out_values[k] < 0 || out_values[k] >= tp.n_values) return fail(RELAY_ERR_ATTR, "out_values[%d] = %d names no value", k, out_values[k]);
+        RELAY_TRY(check_output(outputs[k], tp.dtype[out_values[k]], tp.rank, tp.shape, k));
+    }
+    for (int i = 0; i < n_in; ++i) RELAY_TRY(check_data(inputs[i], "input"));
+    for (int k = 0; k < n_out; ++k) RELAY_TRY(check_data(outputs[k], "output"));
+    RELAY_TRY(check_no_overlap(outputs, n_out, inputs, n_in));
+    if (tp.total == 0) return RELAY_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+
+    // pre-compiled body?
+    View2D v = view2d(tp);
+    if (v.ok && n_out == 1 && n_in == 3 && outputs[0]->dtype == v.storage && kinds_match<BodyTanhAffineResidualFwd>(v) &&
+        canon(tp, out_values[0]) == known_tanh_affine_fwd(v.storage).out) {
+        Args2D<3, 1> A{};
+        for (int i = 0; i < 3; ++i) A.in[i] = inputs[i]->data;
+        A.out[0] = outputs[0]->data; A.partial[0] = nullptr;
+        A.rows = v.rows; A.cols = v.cols; A.aux = 0;
+        const int vec = v.storage == RELAY_BF16 ? 8 : 4;
+        const int64_t gx = (v.cols + (int64_t)kTX * vec - 1) / (kTX * vec);
+        int ns = (int)std::max<int64_t>(1, std::min<int64_t>((148 * 16) / gx, (v.rows + kTY * kUnroll - 1) / (kTY * kUnroll)));
+        return launch_body2d<BodyTanhAffineResidualFwd>(v.storage, A, ns, st, "ewise2d<tanh_affine_residual_fwd>");
+    }
+
+    DevProgram P;
+    fill_dev_program(tp, inputs, &P);
+    DevOutputs O{};
+    O.n_out = n_out;
+    for (int k = 0; k < n_out; ++k) { O.value[k] = out_values[k]; O.dtype[k] = outputs[k]->dtype; O.ptr[k] = outputs[k]->data; }
+    ewise_generic_kernel<<<grid_for(tp.total, 256), 256, 0, st>>>(P, O, tp.total);
+    return check_launch("ewise_generic");
+}
+
+// ---- reduce ----------------------------------------------------------------------------------------
+namespace relay {
+
+struct ReducePlan {
+    TypedProgram tp;
+    View2D v;
+    bool fast_grad = false;     // pre-compiled tanh-affine gradient group
+    bool fast_colsum = false;   // identity column sum / mean over all leading axes
+    bool fast_row = false;      // identity reduction over the last axis
+    int n_slices = 1;
+    size_t ws_need = 0;
+    int64_t red_shape[RELAY_MAX_OUTPUTS][RELAY_MAX_RANK];
+    int red_rank[RELAY_MAX_OUTPUTS];
+    int32_t out_dtype[RELAY_MAX_OUTPUTS];
+};
+
+static relay_status_t plan_reduce(const relay_ewise_prog_t *prog, const relay_tensor_t *const *inputs, int32_t n_in,
+                                  const relay_out_spec_t *specs, int32_t n_out, ReducePlan *pl)
+{
+    static const relay_ewise_prog_t empty = {0, 0, nullptr};
+    if (!prog) prog = &empty;
+    RELAY_TRY(check_not_null(specs, "specs"));
+    if (n_out < 1 || n_out > RELAY_MAX_OUTPUTS) return fail(RELAY_ERR_ATTR, "%d outputs, 1..%d allowed", n_out, RELAY_MAX_OUTPUTS);
+    RELAY_TRY(type_program(prog, inputs, n_in, &pl->tp));
+    const TypedProgram &tp = pl->tp;
+    if (n_in < 1) return fail(RELAY_ERR_ATTR, "a reduce group needs at least one input");
+    for (int k = 0; k < n_out; ++k) {
+        const relay_out_spec_t &s = specs[k];
+        if (s.value < 0 || s.value >= tp.n_values) return fail(RELAY_ERR_ATTR, "specs[%d].value = %d names no value", k, s.value);
+        relay_tensor_t vt{}, rt{};
+        vt.dtype = tp.dtype[s.value]; vt.rank = tp.rank; vt.layout = RELAY_ROWMAJOR;
+        for (int d = 0; d < tp.rank; ++d) vt.shape[d] = tp.shape[d];
+        if (s.red_op != RELAY_RED_NONE && !is_float(vt.dtype))
+            return fail(RELAY_ERR_DTYPE, "specs[%d]: reduction of a %s value is not defined here", k, dtype_name(vt.dtype));
+        RELAY_TRY(relay_infer_reduce(&vt, s.red_op, s.axes_mask, s.keepdims, &rt));
+        pl->red_rank[k] = rt.rank;
+        pl->out_dtype[k] = rt.dtype;
+        for (int d = 0; d < rt.rank; ++d) pl->red_shape[k][d] = rt.shape[d];
+    }
+    pl->v = view2d(tp);
+    const View2D &v = pl->v;
+    const int32_t lead_mask = tp.rank >= 2 ? ((1 << (tp.rank - 1)) - 1) : 0;
+    const int32_t last_mask = tp.rank >= 1 ? (1 << (tp.rank - 1)) : 0;
+    if (v.ok && tp.rank >= 2 && n_out == 3 && n_in == 4 && kinds_match<BodyTanhAffineResidualGrad>(v) && specs[0].red_op == RELAY_RED_NONE &&
+        tp.dtype[specs[0].value] == v.storage && specs[1].red_op == RELAY_RED_SUM && specs[2].red_op == RELAY_RED_SUM &&
+        specs[1].axes_mask == lead_mask && specs[2].axes_mask == lead_mask) {
+        KnownGrad kg = known_tanh_affine_grad(v.storage);
+        if (canon(tp, specs[0].value) == kg.dx && canon(tp, specs[1].value) == kg.da && canon(tp, specs[2].value) == kg.db)
+            pl->fast_grad = true;
+    }
+    if (!pl->fast_grad && v.ok && tp.rank >= 2 && n_out == 1 && n_in == 1 && tp.n_instr == 0 && v.kind[0] == KIND_FULL &&
+        (specs[0].red_op == RELAY_RED_SUM || specs[0].red_op == RELAY_RED_MEAN) && specs[0].axes_mask == lead_mask)
+        pl->fast_colsum = true;
+    if (v.ok && tp.rank >= 1 && n_out == 1 && n_in == 1 && tp.n_instr == 0 && v.kind[0] == KIND_FULL &&
+        specs[0].red_op != RELAY_RED_NONE && specs[0].axes_mask == last_mask)
+        pl->fast_row = true;
+    if (pl->fast_grad || pl->fast_colsum) {
+        pl->n_slices = colsum_slices(v.rows, v.cols, v.storage);
+        pl->ws_need = (size_t)(pl->fast_grad ? 2 : 1) * pl->n_slices * (size_t)v.cols * sizeof(float);
+    }
+    return RELAY_OK;
+}
+
+}  // namespace relay
+
+extern "C" size_t relay_workspace_bytes_reduce(const relay_tensor_t *const *inputs, int32_t n_in, const relay_out_spec_t *specs,
+                                               int32_t n_out)
+{
+    // The workspace depends on the shapes and on which results are column sums, not on the
+    // program body: an upper bound that holds for every program over these inputs.
+    clear_error();
+    if (!inputs || !specs || n_in < 1 || n_in > RELAY_MAX_INPUTS || n_out < 1) return 0;
+    static const relay_ewise_prog_t empty = {0, 0, nullptr};
+    TypedProgram tp;
+    if (type_program(&empty, inputs, n_in, &tp) != RELAY_OK) return 0;
+    View2D v = view2d(tp);
+    if (!v.ok) return 0;
+    int n_sum = 0;
+    for (int k = 0; k < n_out; ++k) n_sum += specs[k].red_op != RELAY_RED_NONE;
+    return (size_t)n_sum * colsum_slices(v.rows, v.cols, v.storage) * (size_t)v.cols * sizeof(float);
+}
+
+extern "C" relay_status_t relay_fused_reduce(const relay_ewise_prog_t *prog, const relay_tensor_t *const *inputs, int32_t n_in,
+                                             const relay_out_spec_t *specs, const relay_tensor_t *const *outputs, int32_t n_out,
+                                             void *ws, size_t ws_bytes, void *stream)
+{
+    clear_error();
+    RELAY_TRY(check_not_null(outputs, "outputs"));
+    if (n_out >= 1 && n_out <= RELAY_MAX_OUTPUTS)
+        for (int k = 0; k < n_out; ++k) RELAY_TRY(check_not_null(outputs[k], "outputs[k]"));
+    ReducePlan pl;
+    RELAY_TRY(plan_reduce(prog, inputs, n_in, specs, n_out, &pl));
+    const TypedProgram &tp = pl.tp;
+    for (int k = 0; k < n_out; ++k) RELAY_TRY(check_output(outputs[k], pl.out_dtype[k], pl.red_rank[k], pl.red_shape[k], k));
+    for (int i = 0; i < n_in; ++i) RELAY_TRY(check_data(inputs[i], "input"));
+    for (int k = 0; k < n_out; ++k) RELAY_TRY(check_data(outputs[k], "output"));
+    RELAY_TRY(check_no_overlap(outputs, n_out, inputs, n_in));
+    RELAY_TRY(check_workspace(ws, ws_bytes, pl.ws_need));
+    if (tp.total == 0) return RELAY_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    const View2D &v = pl.v;
+
+    if (pl.fast_grad) {
+        Args2D<4, 3> A{};
+        for (int i = 0; i < 4; ++i) A.in[i] = inputs[i]->data;
+        float *part = (float *)ws;
+        A.out[0] = outputs[0]->data; A.out[1] = A.out[2] = nullptr;
+        A.partial[0] = nullptr; A.partial[1] = part; A.partial[2] = part + (size_t)pl.n_slices * v.cols;
+        A.rows = v.rows; A.cols = v.cols; A.aux = 0;
+        RELAY_TRY(launch_body2d<BodyTanhAffineResidualGrad>(v.storage, A, pl.n_slices, st, "ewise2d<tanh_affine_residual_grad>"));
+        RELAY_TRY(launch_colsum_finalize(A.partial[1], pl.n_slices, v.cols, 1.0f, (float *)outputs[1]->data, st));
+        RELAY_TRY(launch_colsum_finalize(A.partial[2], pl.n_slices, v.cols, 1.0f, (float *)outputs[2]->data, st));
+        return RELAY_OK;
+    }
+    if (pl.fast_colsum) {
+        Args2D<1, 1> A{};
+        A.in[0] = inputs[0]->data; A.out[0] = nullptr; A.partial[0] = (float *)ws;
+        A.rows = v.rows; A.cols = v.cols; A.aux = 0;
+        RELAY_TRY(launch_body2d<BodyIdentityColSum>(v.storage, A, pl.n_slices, st, "ewise2d<identity_colsum>"));
+        const float scale = specs[0].red_op == RELAY_RED_MEAN ? 1.0f / (float)v.rows : 1.0f;
+        return launch_colsum_finalize(A.partial[0], pl.n_slices, v.cols, scale, (float *)outputs[0]->data, st);
+    }
+    if (pl.fast_row) {
+        const unsigned grid = (unsigned)((v.rows + 7) / 8);
+        const float scale = specs[0].red_op == RELAY_RED_MEAN ? 1.0f / (float)v.cols : 1.0f;
+        const int op = specs[0].red_op == RELAY_RED_MEAN ? RELAY_RED_SUM : specs[0].red_op;
+#define ROWRED(T, OP) rowreduce_kernel<T, OP><<<grid, 256, 0, st>>>((const T *)inputs[0]->data, v.rows, v.cols, scale, outputs[0]->data)
+        if (v.storage == RELAY_BF16) {
+            if (op == RELAY_RED_SUM) ROWRED(__nv_bfloat16, RELAY_RED_SUM);
+            else if (op == RELAY_RED_MAX) ROWRED(__nv_bfloat16, RELAY_RED_MAX);
+            else ROWRED(__nv_bfloat16, RELAY_RED_ARGMAX);
+        } else {
+            if (op == RELAY_RED_SUM) ROWRED(float, RELAY_RED_SUM);
+            else if (op == RELAY_RED_MAX) ROWRED(float, RELAY_RED_MAX);
+            else ROWRED(float, RELAY_RED_ARGMAX);
+        }
+#undef ROWRED
+        return check_launch("rowreduce");
+    }
+
+    // generic: one evaluator pass for the unreduced results, one reduction launch per reduced result
+    DevProgram P;
+    fill_dev_program(tp, inputs, &P);
+    DevOutputs O{};
+    for (int k = 0; k < n_out; ++k)
+        if (specs[k].red_op == RELAY_RED_NONE) {
+            O.value[O.n_out] = specs[k].value; O.dtype[O.n_out] = outputs[k]->dtype; O.ptr[O.n_out] = outputs[k]->data;
+            ++O.n_out;
+        }
+    if (O.n_out > 0) {
+        ewise_generic_kernel<<<grid_for(tp.total, 256), 256, 0, st>>>(P, O, tp.total);
+        RELAY_TRY(check_launch("ewise_generic"));
+    }
+    for (int k = 0; k < n_out; ++k) {
+        if (specs[k].red_op == RELAY_RED_NONE) continue;
+        DevReduce R{};
+        R.red_op = specs[k].red_op; R.value = specs[k].value; R.out = outputs[k]->data;
+        R.kept_elems = 1; R.red_elems = 1;
+        for (int d = 0; d < tp.rank; ++d) {
+            if (specs[k].axes_mask >> d & 1) { R.red_axis[R.n_red++] = d; R.red_elems *= tp.shape[d]; }
+            else { R.kept_axis[R.n_kept++] = d; R.kept_elems *= tp.shape[d]; }
+        }
+        R.scale = specs[k].red_op == RELAY_RED_MEAN ? 1.0f / (float)R.red_elems : 1.0f;
+        R.group = (R.kept_elems < 148 * 8 && R.red_elems >= 1024) ? 256 : 32;
+        const int per_block = 256 / R.group;
+        reduce_generic_kernel<<<(unsigned)((R.kept_elems + per_block - 1) / per_block), 256, 0, st>>>(P, R);
+        RELAY_TRY(check_launch("reduce_generic"));
+    }
+    return RELAY_OK;
+}

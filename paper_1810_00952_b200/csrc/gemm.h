@@ -1,0 +1,30 @@
+// One description for every contraction the groups need, so that the forward product, the
+// input gradient and the weight gradient run without materialising a transpose:
+//   C[m,n] = epilogue( sum_k A(m,k) * B(k,n) ),  A(m,k) = a[m*a_sm + k*a_sk],  B(k,n) = b[k*b_sk + n*b_sn]
+// where exactly one stride of each operand is 1 (the other is its leading dimension).
+#pragma once
+#include "common.h"
+
+namespace relay {
+
+struct GemmDesc {
+    int64_t M = 0, N = 0, K = 0;
+    const void *a = nullptr; int64_t a_sm = 0, a_sk = 0;
+    const void *b = nullptr; int64_t b_sk = 0, b_sn = 0;
+    void *c = nullptr;       int64_t ldc = 0;      // C row-major, leading dimension ldc
+    int32_t in_dtype = RELAY_F32;                   // dtype of A and B
+    int32_t out_dtype = RELAY_F32;                  // dtype of C
+    const void *bias = nullptr; int32_t bias_dtype = RELAY_F32;  // per column n, or nullptr
+    int32_t act = RELAY_ACT_NONE;
+};
+
+// Picks the tensor-core kernel when the description fits it, else the SIMT kernel (both on the
+// GPU).  Enqueues on `st`.
+relay_status_t launch_gemm(const GemmDesc &g, cudaStream_t st);
+
+// the two tiers, callable directly
+relay_status_t launch_gemm_simt(const GemmDesc &g, cudaStream_t st);
+bool gemm_tc_eligible(const GemmDesc &g);
+relay_status_t launch_gemm_tc(const GemmDesc &g, cudaStream_t st);
+
+}  // namespace relay

@@ -1,0 +1,151 @@
+"""GPU parity: conv2d anchor (+bias +activation) with its gradient group, and the LSTM sequence."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1810_00952_b200 import binding as B
+from relay_workloads import inputs as I
+
+from parity import Guarded, assert_bf16, assert_f32, to_np, workspace
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+F64 = 5
+
+
+def conv_fwd(x, w, b, stride, pad, act):
+    d = B.relay_infer_conv2d(B.desc(x, B.NCHW), B.desc(w, B.OIHW), stride, pad)
+    y = Guarded(B._shape(d), x.dtype, DEV)
+    ws = workspace(B.relay_workspace_bytes_conv2d_act(x, w, stride, pad), DEV)
+    B.relay_fused_conv2d_act(x.to(DEV), w.to(DEV), None if b is None else b.to(DEV), stride, pad, act, y.t, ws)
+    torch.cuda.synchronize()
+    return y.check()
+
+
+def conv_grad(x, w, y, dy, stride, pad, act, want_dx=True, want_db=True):
+    dx = Guarded(tuple(x.shape), x.dtype, DEV) if want_dx else None
+    dw = Guarded(tuple(w.shape), x.dtype, DEV)
+    db = Guarded((w.shape[0],), torch.float32, DEV) if want_db else None
+    ws = workspace(B.relay_workspace_bytes_conv2d_act_grad(x, w, stride, pad), DEV)
+    B.relay_fused_conv2d_act_grad(x.to(DEV), w.to(DEV), y.to(DEV), dy.to(DEV), stride, pad, act, dx.t if dx else None, dw.t,
+                                  db.t if db else None, ws)
+    torch.cuda.synchronize()
+    return (dx.check() if dx else None), dw.check(), (db.check() if db else None)
+
+
+@pytest.mark.parametrize("N,C,H,W,O,R,stride,pad", [(2, 3, 7, 6, 4, 3, 1, 1), (1, 5, 9, 9, 3, 3, 2, 1), (2, 2, 8, 5, 6, 5, 1, 0),
+                                                     (1, 4, 6, 6, 2, 1, 1, 0), (3, 8, 10, 12, 16, 3, 2, 2), (1, 1, 1, 1, 1, 3, 1, 1)])
+@pytest.mark.parametrize("tdt", [torch.float32, torch.bfloat16])
+def test_conv_small_shapes_forward_and_gradient(N, C, H, W, O, R, stride, pad, tdt):
+    t = I.cfg4_conv(N, C, H, W, O, R, R, dtype=tdt, salt=H)
+    act = B.ACT_RELU
+    y = conv_fwd(t["x"], t["w"], t["b"], stride, pad, act)
+    xo, wo, bo = (I.as_f64(t[k]) for k in ("x", "w", "b"))
+    want = oracle.conv2d_act(xo, wo, bo, stride, pad, act, F64)
+    chk = assert_f32 if tdt == torch.float32 else assert_bf16
+    chk(y, want, what="y")
+    dy = I.normal(4, 3, tuple(y.shape), 1.0, tdt, salt=H)
+    dx, dw, db = conv_grad(t["x"], t["w"], y, dy, stride, pad, act)
+    odx, odw, odb = oracle.conv2d_act_grad(xo, wo, to_np(y), I.as_f64(dy), stride, pad, act, F64, F64, F64)
+    chk(dx, odx, what="dx"); chk(dw, odw, what="dw")
+    (assert_f32 if tdt == torch.float32 else (lambda g, o, what: assert_bf16(g, o, stored_bf16=False, what=what)))(db, odb, what="db")
+
+
+def test_conv_reduced_config_bf16_3x3():
+    """Configuration 4's structure (3x3, stride 1, pad 1, NCHW/OIHW, bf16) at N=2, C=64, 28x28, O=64."""
+    t = I.cfg4_conv(2, 64, 28, 28, 64)
+    y = conv_fwd(t["x"], t["w"], t["b"], 1, 1, B.ACT_RELU)
+    xo, wo, bo, dyo = (I.as_f64(t[k]) for k in ("x", "w", "b", "dy"))
+    assert_bf16(y, oracle.conv2d_act(xo, wo, bo, 1, 1, B.ACT_RELU, F64), what="y")
+    dx, dw, db = conv_grad(t["x"], t["w"], y, t["dy"], 1, 1, B.ACT_RELU)
+    odx, odw, odb = oracle.conv2d_act_grad(xo, wo, to_np(y), dyo, 1, 1, B.ACT_RELU, F64, F64, F64)
+    assert_bf16(dx, odx, what="dx"); assert_bf16(dw, odw, what="dw"); assert_bf16(db, odb, stored_bf16=False, what="db")
+
+
+def test_conv_rejections():
+    x = torch.zeros(2, 3, 8, 8, dtype=torch.bfloat16, device=DEV); w = torch.zeros(5, 3, 3, 3, dtype=torch.bfloat16, device=DEV)
+    y = torch.zeros(2, 5, 8, 8, dtype=torch.bfloat16, device=DEV)
+    n0 = B.relay_launch_count()
+    with pytest.raises(B.RelayError) as e:
+        B.relay_fused_conv2d_act(x, w, None, 1, 1, B.ACT_RELU, torch.zeros(2, 5, 8, 7, dtype=torch.bfloat16, device=DEV))
+    assert e.value.status_name == "ERR_SHAPE"
+    with pytest.raises(B.RelayError) as e:
+        B.relay_fused_conv2d_act(x, w, torch.zeros(4, device=DEV), 1, 1, B.ACT_RELU, y)
+    assert e.value.status_name == "ERR_SHAPE"
+    with pytest.raises(B.RelayError) as e:
+        B.relay_fused_conv2d_act(x, w.float(), None, 1, 1, B.ACT_RELU, y)
+    assert e.value.status_name == "ERR_DTYPE"
+    assert B.relay_launch_count() == n0
+
+
+def test_conv_full_size_sampled():
+    """Configuration 4 at full size: the oracle recomputes one whole image of y and dx, and a block
+    of dW (8 output x 8 input channels, all taps, all 32 images), from the GPU's stored y."""
+    t = I.cfg4_conv()
+    y = conv_fwd(t["x"], t["w"], t["b"], 1, 1, B.ACT_RELU)
+    dx, dw, db = conv_grad(t["x"], t["w"], y, t["dy"], 1, 1, B.ACT_RELU)
+    wo, bo = I.as_f64(t["w"]), I.as_f64(t["b"])
+    n = 17
+    xo = I.as_f64(t["x"][n:n + 1])
+    assert_bf16(y[n:n + 1], oracle.conv2d_act(xo, wo, bo, 1, 1, B.ACT_RELU, F64), what="y")
+    odx, _, _ = oracle.conv2d_act_grad(xo, wo, to_np(y[n:n + 1]), I.as_f64(t["dy"][n:n + 1]), 1, 1, B.ACT_RELU, F64, F64, F64,
+                                       want_dw=False, want_db=False)
+    assert_bf16(dx[n:n + 1], odx, what="dx")
+    oc, ic = slice(120, 128), slice(248, 256)
+    _, odw, odb = oracle.conv2d_act_grad(I.as_f64(t["x"][:, ic]), wo[oc, ic], to_np(y[:, oc]), I.as_f64(t["dy"][:, oc]), 1, 1,
+                                         B.ACT_RELU, F64, F64, F64, want_dx=False)
+    assert_bf16(dw[oc, ic], odw, what="dw")
+    assert_bf16(db[oc], odb, stored_bf16=False, what="db")
+
+
+# ---- LSTM -------------------------------------------------------------------------------------------
+def lstm(t):
+    T_, Bn, _ = t["x"].shape
+    H = t["w_hh"].shape[0]
+    h_all = Guarded((T_, Bn, H), torch.float32, DEV)
+    c_fin = Guarded((Bn, H), torch.float32, DEV)
+    ws = workspace(B.relay_workspace_bytes_lstm(t["x"], t["w_ih"], t["w_hh"]), DEV)
+    B.relay_lstm_cell_seq(*(t[k].to(DEV) for k in ("x", "w_ih", "w_hh", "b", "h0", "c0")), h_all.t, c_fin.t, ws)
+    B.relay_poll_status()
+    return h_all.check(), c_fin.check()
+
+
+@pytest.mark.parametrize("T,Bn,In,H", [(1, 1, 8, 8), (5, 3, 20, 24), (8, 16, 128, 256), (3, 70, 40, 72), (12, 9, 64, 128)])
+def test_lstm_small_shapes(T, Bn, In, H):
+    t = I.cfg5_lstm(T, Bn, In, H, salt=T)
+    g = torch.Generator().manual_seed(T)
+    t["h0"] = torch.randn(Bn, H, generator=g) * 0.3
+    t["c0"] = torch.randn(Bn, H, generator=g) * 0.3
+    h_all, c_fin = lstm(t)
+    oh, oc = oracle.lstm_cell_seq(*(I.as_f64(t[k]) for k in ("x", "w_ih", "w_hh", "b", "h0", "c0")))
+    # bf16 GEMM inputs with fp32 accumulation and fp32 state: the bf16-path tolerance, results in f32
+    assert_bf16(h_all, oh, stored_bf16=False, what="h_all"); assert_bf16(c_fin, oc, stored_bf16=False, what="c_final")
+    assert bool((h_all.abs() < 1).all())
+
+
+def test_lstm_full_size_sampled_batch_rows():
+    """Configuration 5 at full size; batch rows are independent, so the oracle runs 3 of the 64
+    rows through all 128 steps."""
+    t = I.cfg5_lstm()
+    h_all, c_fin = lstm(t)
+    rows = [0, 31, 63]
+    sub = {k: I.as_f64(t[k]) for k in ("w_ih", "w_hh", "b")}
+    oh, oc = oracle.lstm_cell_seq(I.as_f64(t["x"][:, rows]), sub["w_ih"], sub["w_hh"], sub["b"], I.as_f64(t["h0"][rows]), I.as_f64(t["c0"][rows]))
+    assert_bf16(h_all[:, rows], oh, stored_bf16=False, what="h_all"); assert_bf16(c_fin[rows], oc, stored_bf16=False, what="c_final")
+    assert bool((h_all.abs() < 1).all()) and bool((c_fin.abs() <= 128).all())
+
+
+def test_lstm_rejections():
+    t = {k: v.to(DEV) for k, v in I.cfg5_lstm(2, 2, 8, 8).items()}
+    h_all = torch.empty(2, 2, 8, device=DEV); c = torch.empty(2, 8, device=DEV)
+    ws = workspace(B.relay_workspace_bytes_lstm(t["x"], t["w_ih"], t["w_hh"]), DEV)
+    with pytest.raises(B.RelayError) as e:
+        B.relay_lstm_cell_seq(t["x"], t["w_ih"], t["w_hh"], t["b"][:31].contiguous(), t["h0"], t["c0"], h_all, c, ws)
+    assert e.value.status_name == "ERR_SHAPE"
+    with pytest.raises(B.RelayError) as e:
+        B.relay_lstm_cell_seq(t["x"], t["w_ih"], t["w_hh"], t["b"], t["h0"].bfloat16(), t["c0"], h_all, c, ws)
+    assert e.value.status_name == "ERR_DTYPE"
+    with pytest.raises(B.RelayError) as e:
+        B.relay_lstm_cell_seq(t["x"], t["w_ih"], t["w_hh"], t["b"], t["h0"], t["c0"], h_all, c, None)
+    assert e.value.status_name == "ERR_WORKSPACE"

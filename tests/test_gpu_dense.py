@@ -1,0 +1,150 @@
+"""GPU parity: dense anchor (+bias +activation) and its gradient group against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1810_00952_b200 import binding as B
+from relay_workloads import inputs as I
+
+from parity import Guarded, assert_bf16, assert_f32, to_np, workspace
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+ACTS = (B.ACT_NONE, B.ACT_RELU, B.ACT_TANH, B.ACT_SIGMOID)
+F64 = 5
+
+
+def run_fwd(x, w, b, act):
+    y = Guarded((x.shape[0], w.shape[1]), x.dtype, DEV)
+    ws = workspace(B.relay_workspace_bytes_dense_act(x, w), DEV)
+    B.relay_fused_dense_act(x.to(DEV), w.to(DEV), None if b is None else b.to(DEV), act, y.t, ws)
+    torch.cuda.synchronize()
+    return y.check()
+
+
+def run_grad(x, w, y, dy, act, want_dx=True, want_db=True):
+    M, K = x.shape
+    N = w.shape[1]
+    dx = Guarded((M, K), x.dtype, DEV) if want_dx else None
+    dw = Guarded((K, N), x.dtype, DEV)
+    db = Guarded((N,), torch.float32, DEV) if want_db else None
+    ws = workspace(B.relay_workspace_bytes_dense_act_grad(x, w), DEV)
+    B.relay_fused_dense_act_grad(x.to(DEV), w.to(DEV), y.to(DEV), dy.to(DEV), act, dx.t if dx else None, dw.t,
+                                 db.t if db else None, ws)
+    torch.cuda.synchronize()
+    return (dx.check() if dx else None), dw.check(), (db.check() if db else None)
+
+
+@pytest.mark.parametrize("act", ACTS)
+def test_tiny_mlp_layer_fp32_forward_and_gradient(act):
+    """Configuration 1: x[8,64] W[64,32] b[32] dy[8,32], fp32, max relative error <= 1e-4."""
+    t = I.cfg1_tiny_mlp()
+    y = run_fwd(t["x"], t["w"], t["b"], act)
+    xo, wo, bo, dyo = (I.as_f64(t[k]) for k in ("x", "w", "b", "dy"))
+    assert_f32(y, oracle.dense_act(xo, wo, bo, act, F64), what="y")
+    if act == B.ACT_RELU:
+        z = xo @ wo + bo
+        assert bool((y.cpu()[torch.from_numpy(z < -1e-3)] == 0).all())      # exact zeros stay exact
+    dx, dw, db = run_grad(t["x"], t["w"], y, t["dy"], act)
+    odx, odw, odb = oracle.dense_act_grad(xo, wo, to_np(y), dyo, act, F64, F64, F64)   # the saved y decides the mask
+    assert_f32(dx, odx, what="dx"); assert_f32(dw, odw, what="dw"); assert_f32(db, odb, what="db")
+
+
+@pytest.mark.parametrize("M,K,N", [(1, 1, 1), (37, 53, 29), (130, 70, 200), (64, 64, 64), (5, 300, 8)])
+@pytest.mark.parametrize("tdt", [torch.float32, torch.bfloat16])
+def test_odd_shapes_forward_and_gradient(M, K, N, tdt):
+    t = I.cfg1_tiny_mlp(M, K, N, salt=M)
+    x, w, b, dy = (t[k].to(tdt) for k in ("x", "w", "b", "dy"))
+    w = (w / np.sqrt(K)).to(tdt)
+    act = B.ACT_TANH
+    y = run_fwd(x, w, b, act)
+    xo, wo, bo, dyo = (v.double().numpy() for v in (x, w, b, dy))
+    chk = assert_f32 if tdt == torch.float32 else assert_bf16
+    chk(y, oracle.dense_act(xo, wo, bo, act, F64), what="y")
+    dx, dw, db = run_grad(x, w, y, dy, act)
+    odx, odw, odb = oracle.dense_act_grad(xo, wo, to_np(y), dyo, act, F64, F64, F64)
+    chk(dx, odx, what="dx"); chk(dw, odw, what="dw")
+    if tdt == torch.float32:
+        assert_f32(db, odb, what="db")
+    else:
+        assert_bf16(db, odb, stored_bf16=False, what="db")
+
+
+def test_optional_outputs_no_bias_and_f32_bias():
+    t = I.cfg3_mlp(batch=96, width=128, layers=1)
+    x, w, dy = t["x"], t["w0"], t["dy"]
+    y = run_fwd(x, w, None, B.ACT_RELU)
+    xo, wo, dyo = (I.as_f64(v) for v in (x, w, dy))
+    assert_bf16(y, oracle.dense_act(xo, wo, None, B.ACT_RELU, F64))
+    bias32 = torch.linspace(-1, 1, 128)
+    y2 = run_fwd(x, w, bias32, B.ACT_NONE)
+    assert_bf16(y2, oracle.dense_act(xo, wo, bias32.double().numpy(), B.ACT_NONE, F64))
+    dx, dw, db = run_grad(x, w, y, dy, B.ACT_RELU, want_dx=False, want_db=False)
+    assert dx is None and db is None
+    _, odw, _ = oracle.dense_act_grad(xo, wo, to_np(y), dyo, B.ACT_RELU, F64, F64, F64)
+    assert_bf16(dw, odw)
+
+
+def test_three_layer_mlp_chain_reduced_size_group_by_group():
+    """Configuration 3's structure at width 256 / batch 192: every group is checked against the
+    oracle fed with the GPU's stored inputs of that group (so relu masks are identical)."""
+    t = I.cfg3_mlp(batch=192, width=256, layers=3)
+    acts = [t["x"]]
+    for l in range(3):
+        y = run_fwd(acts[-1].to(DEV), t[f"w{l}"], t[f"b{l}"], B.ACT_RELU)
+        assert_bf16(y, oracle.dense_act(to_np(acts[-1]), I.as_f64(t[f"w{l}"]), I.as_f64(t[f"b{l}"]), B.ACT_RELU, F64), what=f"y{l}")
+        acts.append(y)
+    g = t["dy"]
+    for l in (2, 1, 0):
+        dx, dw, db = run_grad(acts[l], t[f"w{l}"], acts[l + 1], g, B.ACT_RELU)
+        odx, odw, odb = oracle.dense_act_grad(to_np(acts[l]), I.as_f64(t[f"w{l}"]), to_np(acts[l + 1]), to_np(g), B.ACT_RELU, F64, F64, F64)
+        assert_bf16(dx, odx, what=f"dx{l}"); assert_bf16(dw, odw, what=f"dw{l}"); assert_bf16(db, odb, stored_bf16=False, what=f"db{l}")
+        g = dx
+
+
+def test_dense_rejections_leave_outputs_untouched():
+    x = torch.zeros(8, 64, device=DEV); w = torch.zeros(64, 32, device=DEV); y = torch.full((8, 32), 5.0, device=DEV)
+    n0 = B.relay_launch_count()
+    cases = [(x, torch.zeros(63, 32, device=DEV), None, y, "ERR_SHAPE"), (x, w.bfloat16(), None, y, "ERR_DTYPE"),
+             (x, w, torch.zeros(31, device=DEV), y, "ERR_SHAPE"), (x, w, None, torch.zeros(8, 31, device=DEV), "ERR_SHAPE"),
+             (x, w, None, y.bfloat16(), "ERR_DTYPE"), (x, w, torch.zeros(32, dtype=torch.bfloat16, device=DEV), y, "ERR_DTYPE")]
+    for xx, ww, bb, yy, status in cases:
+        with pytest.raises(B.RelayError) as e:
+            B.relay_fused_dense_act(xx, ww, bb, B.ACT_RELU, yy)
+        assert e.value.status_name == status, str(e.value)
+    with pytest.raises(B.RelayError) as e:
+        B.relay_fused_dense_act(x, w, None, 9, y)
+    assert e.value.status_name == "ERR_ATTR"
+    with pytest.raises(B.RelayError) as e:     # gradient group without workspace
+        B.relay_fused_dense_act_grad(x, w, y, y.clone(), B.ACT_RELU, torch.empty_like(x), torch.empty_like(w), None, None)
+    assert e.value.status_name == "ERR_WORKSPACE"
+    torch.cuda.synchronize()
+    assert B.relay_launch_count() == n0 and bool((y == 5.0).all())
+
+
+def test_full_size_mlp_layer_sampled_rows_and_columns():
+    """Configuration 3 at full size (4096^3 per contraction, bf16, fp32 accumulate), all three
+    layers forward and backward; the oracle recomputes sampled rows of y / dx (all columns) and
+    sampled rows of dW (all columns) plus db, each from the GPU's stored inputs of that group."""
+    t = I.cfg3_mlp()
+    rng = np.random.default_rng(5)
+    rows = np.unique(np.concatenate([[0, 127, 128, 4095], rng.integers(0, 4096, 8)]))
+    acts = [t["x"].to(DEV)]
+    for l in range(3):
+        acts.append(run_fwd(acts[-1], t[f"w{l}"], t[f"b{l}"], B.ACT_RELU))
+        want = oracle.dense_act(to_np(acts[l][rows]), I.as_f64(t[f"w{l}"]), I.as_f64(t[f"b{l}"]), B.ACT_RELU, F64)
+        assert_bf16(acts[-1][rows], want, what=f"y{l}")
+    g = t["dy"].to(DEV)
+    for l in (2, 1, 0):
+        dx, dw, db = run_grad(acts[l], t[f"w{l}"], acts[l + 1], g, B.ACT_RELU)
+        wo = I.as_f64(t[f"w{l}"])
+        odx, _, _ = oracle.dense_act_grad(to_np(acts[l][rows]), wo, to_np(acts[l + 1][rows]), to_np(g[rows]), B.ACT_RELU, F64, F64, F64,
+                                          want_dw=False, want_db=False)
+        assert_bf16(dx[rows], odx, what=f"dx{l}")
+        # dW rows k in `rows`: needs x[:, rows] over the whole batch
+        _, odw, odb = oracle.dense_act_grad(to_np(acts[l][:, rows]), wo[rows], to_np(acts[l + 1]), to_np(g), B.ACT_RELU, F64, F64, F64,
+                                            want_dx=False)
+        assert_bf16(dw[rows], odw, what=f"dw{l}")
+        assert_bf16(db, odb, stored_bf16=False, what=f"db{l}")
+        g = dx
