@@ -55,10 +55,9 @@ class Guarded:
         n = int(np.prod(shape)) if len(shape) else 1
         item = torch.empty((), dtype=dtype).element_size()
         m = (margin * 16) // item          # keeps the view 16-byte aligned
-        self.full = torch.full((n + 2 * m,), 7, dtype=dtype, device=device) if dtype != torch.int64 else \
-            torch.full((n + 2 * m,), 7, dtype=dtype, device=device)
+        self.full = torch.full((n + 2 * m,), 7, dtype=dtype, device=device)
         self.m, self.n = m, n
-        self.t = self.full[m:m + n].view(*shape) if n else self.full[m:m].view(*shape)
+        self.t = self.full[m:m + n].view(tuple(shape))
 
     def check(self):
         assert bool((self.full[:self.m] == 7).all()) and bool((self.full[self.m + self.n:] == 7).all()), "out-of-range write"
