@@ -246,6 +246,27 @@ relay_status_t relay_fused_reduce(const relay_ewise_prog_t *prog, const relay_te
                                   const relay_out_spec_t *specs, const relay_tensor_t *const *outputs,
                                   int32_t n_out, void *ws, size_t ws_bytes, void *stream);
 
+/* The same group as relay_fused_reduce, for callers that cannot allocate device memory (the paper
+ * has no counterpart; this is a convenience of this library).  Some users of this ABI run where
+ * cudaMalloc is not an option: inside a host framework whose memory pool they may not touch, in
+ * a plug-in that is handed only its input and output buffers, or in a phase of a program where
+ * allocation is forbidden.  They still pass inputs and outputs, but no workspace: the scratch for
+ * the per-slice partial sums is a fixed array of RELAY_STATIC_SCRATCH_BYTES inside the library's
+ * device image (each GPU that loads the library holds one copy until the process exits).
+ *   - A group whose relay_workspace_bytes_reduce() exceeds RELAY_STATIC_SCRATCH_BYTES is rejected
+ *     with RELAY_ERR_WORKSPACE before anything is launched; use relay_fused_reduce then.
+ *   - The call allocates nothing, on the device or through any allocating library routine.
+ *   - The first call on each device looks up the array's device address (a one-time set-up with
+ *     that device current); make that first call outside any stream capture.
+ *   - All calls share the one array, and it keeps whatever the last call left there.  A call
+ *     overwrites every word it later reads, so no clearing is needed between calls; but two
+ *     calls that overlap in time on the same GPU (different streams or threads) race on it --
+ *     serialise them. */
+#define RELAY_STATIC_SCRATCH_BYTES (8u << 20)
+relay_status_t relay_fused_reduce_static_scratch(const relay_ewise_prog_t *prog, const relay_tensor_t *const *inputs,
+                                                 int32_t n_in, const relay_out_spec_t *specs,
+                                                 const relay_tensor_t *const *outputs, int32_t n_out, void *stream);
+
 /* LSTM cell applied over a sequence (a recursive program over time composed of the dense
  * anchor and elementwise gates; recursion is what Section 3.1 adds over dataflow graphs).
  * Gate blocks along the 4H axis are [ i | f | g | o ]:

@@ -276,6 +276,21 @@ def relay_fused_reduce(prog: Optional[dict], inputs, specs, outputs, ws=None):
                                     _desc_array(outs), len(outs), wp, wb, _stream()))
 
 
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def relay_fused_reduce_static_scratch(prog: Optional[dict], inputs, specs, outputs):
+    """relay_fused_reduce without a workspace argument: for callers that may not allocate device
+    memory, the partial sums go to a fixed STATIC_SCRATCH_BYTES array inside the library.  Calls
+    that overlap on one GPU race on that array; larger groups are rejected (ERR_WORKSPACE)."""
+    p = make_prog(prog) if prog is not None else None
+    ins = [desc(t) for t in inputs]
+    outs = [desc(t) for t in outputs]
+    sp = (OutSpec * max(len(specs), 1))(*[OutSpec(*s) for s in specs])
+    _check(lib().relay_fused_reduce_static_scratch(ctypes.byref(p) if p is not None else None, _desc_array(ins), len(ins), sp,
+                                                   _desc_array(outs), len(outs), _stream()))
+
+
 def relay_lstm_cell_seq(x, w_ih, w_hh, b, h0, c0, h_all, c_final, ws=None):
     wp, wb = _ws(ws)
     _check(lib().relay_lstm_cell_seq(_ref(desc(x)), _ref(desc(w_ih)), _ref(desc(w_hh)), _ref(desc(b)), _ref(desc(h0)),
