@@ -243,7 +243,7 @@ def dense_act(x, w, b, act_code: int, y_dtype: int) -> np.ndarray:
 
 
 def dense_act_grad(x, w, y, dy, act_code: int, dx_dtype: int, dw_dtype: int, db_dtype: int,
-                   want_dx=True, want_dw=True, want_db=True):
+                   want_dx=True, want_dw=True, want_db=True, dz_dtype: int = F64):
     x, w, y, dy = _f64(x), _f64(w), _f64(y), _f64(dy)
     M, K = x.shape
     _, N = w.shape
@@ -253,7 +253,7 @@ def dense_act_grad(x, w, y, dy, act_code: int, dx_dtype: int, dw_dtype: int, db_
     db = np.empty((N,)) if want_db else None
     i64 = ctypes.c_int64
     rc = _L().orc_dense_act_grad(
-        _ptr(x), _ptr(w), _ptr(y), _ptr(dy), i64(M), i64(K), i64(N), int(act_code),
+        _ptr(x), _ptr(w), _ptr(y), _ptr(dy), i64(M), i64(K), i64(N), int(act_code), int(dz_dtype),
         int(dx_dtype), int(dw_dtype), int(db_dtype), _ptr(dx), _ptr(dw), _ptr(db),
     )
     assert rc == 0
@@ -278,7 +278,8 @@ def conv2d_act(x, wt, b, stride: int, pad: int, act_code: int, y_dtype: int) -> 
 
 
 def conv2d_act_grad(x, wt, y, dy, stride: int, pad: int, act_code: int, dx_dtype: int,
-                    dw_dtype: int, db_dtype: int, want_dx=True, want_dw=True, want_db=True):
+                    dw_dtype: int, db_dtype: int, want_dx=True, want_dw=True, want_db=True,
+                    dz_dtype: int = F64):
     x, wt, y, dy = _f64(x), _f64(wt), _f64(y), _f64(dy)
     Nb, C, H, W = x.shape
     O, _, R, S = wt.shape
@@ -288,8 +289,8 @@ def conv2d_act_grad(x, wt, y, dy, stride: int, pad: int, act_code: int, dx_dtype
     i64 = ctypes.c_int64
     rc = _L().orc_conv2d_act_grad(
         _ptr(x), _ptr(wt), _ptr(y), _ptr(dy), i64(Nb), i64(C), i64(H), i64(W), i64(O), i64(R),
-        i64(S), i64(stride), i64(pad), int(act_code), int(dx_dtype), int(dw_dtype), int(db_dtype),
-        _ptr(dx), _ptr(dw), _ptr(db),
+        i64(S), i64(stride), i64(pad), int(act_code), int(dz_dtype), int(dx_dtype), int(dw_dtype),
+        int(db_dtype), _ptr(dx), _ptr(dw), _ptr(db),
     )
     assert rc == 0
     return dx, dw, db

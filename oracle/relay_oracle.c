@@ -328,15 +328,19 @@ int orc_dense_act(const double *x, const double *w, const double *b, int64_t M, 
  *   dx[m,k] = sum_n dZ[m,n] W[k,n]
  *   dW[k,n] = sum_m x[m,k] dZ[m,n]
  *   db[n]   = sum_m dZ[m,n]
+ * dZ is itself a typed value: the elementwise product of two tensors of base type t has type t
+ * (Fig. 5, Type-Noncomp-BinaryOp), so it is rounded to dz_dtype before the contractions consume it
+ * (dz_dtype = fp64 code keeps it exact).
  * Any of dx, dw, db may be NULL (not requested).  Results are stored in the given dtypes.
  * ---------------------------------------------------------------------------------------- */
 int orc_dense_act_grad(const double *x, const double *w, const double *y, const double *dy,
-                       int64_t M, int64_t K, int64_t N, int act, int dx_dtype, int dw_dtype,
-                       int db_dtype, double *dx, double *dw, double *db)
+                       int64_t M, int64_t K, int64_t N, int act, int dz_dtype, int dx_dtype,
+                       int dw_dtype, int db_dtype, double *dx, double *dw, double *db)
 {
     double *dz = (double *)malloc(sizeof(double) * (size_t)(M * N ? M * N : 1));
     if (!dz) return -1;
-    for (int64_t i = 0; i < M * N; ++i) dz[i] = dy[i] * orc_act_grad_from_output(y[i], act);
+    for (int64_t i = 0; i < M * N; ++i)
+        dz[i] = orc_cast(dy[i] * orc_act_grad_from_output(y[i], act), dz_dtype);
     if (dx) {
         for (int64_t m = 0; m < M; ++m)
             for (int64_t k = 0; k < K; ++k) {
@@ -408,14 +412,14 @@ int orc_conv2d_act(const double *x, const double *wt, const double *b, int64_t N
 }
 
 /* conv2d gradient group (Section 4.2):
- *   dZ = dy (.) act'(y)
+ *   dZ = cast(dy (.) act'(y), dz_dtype)      (a typed value, as in the dense gradient group)
  *   dx[n,c,i,j]   = sum_{o,r,s} dZ[n,o,p,q] Wt[o,c,r,s]  over the (p,q) with p*st-pad+r = i, q*st-pad+s = j
  *   dWt[o,c,r,s]  = sum_{n,p,q} dZ[n,o,p,q] x[n,c,p*st-pad+r,q*st-pad+s]   (in-range taps only)
  *   db[o]         = sum_{n,p,q} dZ[n,o,p,q]
  */
 int orc_conv2d_act_grad(const double *x, const double *wt, const double *y, const double *dy,
                         int64_t Nb, int64_t C, int64_t H, int64_t W, int64_t O, int64_t R,
-                        int64_t S, int64_t stride, int64_t pad, int act, int dx_dtype,
+                        int64_t S, int64_t stride, int64_t pad, int act, int dz_dtype, int dx_dtype,
                         int dw_dtype, int db_dtype, double *dx, double *dw, double *db)
 {
     int64_t P, Q;
@@ -424,7 +428,8 @@ int orc_conv2d_act_grad(const double *x, const double *wt, const double *y, cons
     int64_t ny = Nb * O * P * Q;
     double *dz = (double *)malloc(sizeof(double) * (size_t)(ny ? ny : 1));
     if (!dz) return -1;
-    for (int64_t i = 0; i < ny; ++i) dz[i] = dy[i] * orc_act_grad_from_output(y[i], act);
+    for (int64_t i = 0; i < ny; ++i)
+        dz[i] = orc_cast(dy[i] * orc_act_grad_from_output(y[i], act), dz_dtype);
     if (dx) {
         for (int64_t n = 0; n < Nb; ++n)
             for (int64_t c = 0; c < C; ++c)

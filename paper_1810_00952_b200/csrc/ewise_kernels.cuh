@@ -238,6 +238,7 @@ struct BodyActGrad {
     __device__ __forceinline__ static void apply(const float (&in)[NIN], float (&out)[NOUT], int act)
     {
         float dz = in[0] * act_grad_from_output(in[1], act);
+        if constexpr (FAST) dz = round_bf16(dz);   // bf16 storage: dZ is a bf16 value; db sums what is stored
         out[0] = dz;
         out[1] = dz;
     }

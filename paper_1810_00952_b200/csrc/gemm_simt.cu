@@ -1,6 +1,9 @@
-// SIMT contraction kernel: true fp32 FMA accumulation in k order.  It is the fp32 path of the
-// dense groups (tensor cores would round the operands) and the path for shapes the
-// tensor-core kernel does not take.
+// SIMT contraction kernel, sums in k order.  It is the fp32 path of the dense groups (tensor cores
+// would round the operands to tf32) and the path for shapes the tensor-core kernel does not take.
+// fp32 operands are accumulated in fp64 and rounded once on the store, so that results that suffer
+// cancellation still meet the fp32 tolerance; bf16 operands are accumulated in fp32.
+#include <type_traits>
+
 #include "ewise_kernels.cuh"
 #include "gemm.h"
 
@@ -22,7 +25,8 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmDesc g)
     const int tid = threadIdx.x;
     const int64_t m0 = (int64_t)blockIdx.x * BM, n0 = (int64_t)blockIdx.y * BN;
     const int tm = (tid / 16) * 4, tn = (tid % 16) * 4;
-    float acc[4][4] = {};
+    using Acc = typename std::conditional<sizeof(TIN) == 4, double, float>::type;
+    Acc acc[4][4] = {};
     // loader index order follows the unit stride of each operand so that loads coalesce
     const bool a_k_fast = g.a_sk == 1, b_n_fast = g.b_sn == 1;
     for (int64_t k0 = 0; k0 < g.K; k0 += BK) {
@@ -47,7 +51,7 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmDesc g)
 #pragma unroll
             for (int i = 0; i < 4; ++i)
 #pragma unroll
-                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+                for (int j = 0; j < 4; ++j) acc[i][j] = fma((Acc)av[i], (Acc)bv[j], acc[i][j]);
         }
         __syncthreads();
     }
@@ -60,8 +64,9 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmDesc g)
         for (int j = 0; j < 4; ++j) {
             int64_t n = n0 + tn + j;
             if (n >= g.N) continue;
-            float z = acc[i][j];
-            if (g.bias) z += g.bias_dtype == RELAY_BF16 ? __bfloat162float(((const __nv_bfloat16 *)g.bias)[n]) : ((const float *)g.bias)[n];
+            Acc zz = acc[i][j];
+            if (g.bias) zz += (Acc)(g.bias_dtype == RELAY_BF16 ? __bfloat162float(((const __nv_bfloat16 *)g.bias)[n]) : ((const float *)g.bias)[n]);
+            const float z = (float)zz;
             float y = act_fwd<FAST>(z, g.act);
             if constexpr (sizeof(TOUT) == 2) C[m * g.ldc + n] = __float2bfloat16_rn(y);
             else C[m * g.ldc + n] = y;

@@ -1,9 +1,276 @@
-// Tensor-core contraction kernel (tcgen05 + TMEM + TMA) -- placeholder until the kernel lands.
+// Tensor-core contraction for bf16 operands with fp32 accumulation (sm_100a):
+//   TMA tile loads (128-byte swizzle) -> 4-stage shared-memory ring -> tcgen05.mma issued by one
+//   thread into a double-buffered TMEM accumulator -> epilogue warps read TMEM (tcgen05.ld), add the
+//   bias, apply the activation, round once and store.
+// One persistent block per SM walks the 128 x 256 output tiles.  Roles: warp 0 = TMA producer,
+// warp 1 = TMEM owner + MMA issuer, warps 2..5 = epilogue (one TMEM lane quarter each), so the
+// epilogue of tile i overlaps the main loop of tile i+1.
+//
+// Operands are described by strides (gemm.h): an operand whose contraction index is contiguous is
+// "K-major", one whose M/N index is contiguous is "MN-major"; both are fed to the MMA unit as they
+// lie in memory, so forward (x K-major, W MN-major), input gradient (dZ K-major, W K-major) and
+// weight gradient (x MN-major, dZ MN-major) need no transpose pass.
+#include <mutex>
+
+#include "ewise_kernels.cuh"
 #include "gemm.h"
+#include "tc_common.cuh"
 
 namespace relay {
 
-bool gemm_tc_eligible(const GemmDesc &) { return false; }
-relay_status_t launch_gemm_tc(const GemmDesc &, cudaStream_t) { return fail(RELAY_ERR_UNSUPPORTED, "tensor-core contraction not built"); }
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int MN_BOX_BYTES = 64 * BK * 2;   // one TMA box of an MN-major operand: 64 (M/N) x 64 (k)
+constexpr int TMEM_COLS = 512;              // two accumulators of 256 fp32 columns
+constexpr int NUM_THREADS = 192;
+constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_BYTES + 256;
+
+struct Params {
+    int M, N, K;
+    void *c;
+    long long ldc;
+    const void *bias;
+    int bias_bf16, act, out_f32;
+    int tiles_m, tiles_n, k_blocks;
+    int *err;
+};
+
+template <bool A_MN, bool B_MN>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const Params p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + (size_t)STAGES * STAGE_BYTES);
+    uint64_t *full = bars, *empty = bars + STAGES, *tmem_full = bars + 2 * STAGES, *tmem_empty = bars + 2 * STAGES + 2;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 4);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_tiles = p.tiles_m * p.tiles_n;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { tc::mbar_init(&tmem_full[b], 1); tc::mbar_init(&tmem_empty[b], 4); }
+        *abort_flag = 0;
+        tc::fence_barrier_init();
+        tc::prefetch_tmap(&tm_a);
+        tc::prefetch_tmap(&tm_b);
+    }
+    if (warp == 1) {
+        tc::tmem_alloc(tmem_slot, TMEM_COLS);
+        tc::tmem_relinquish();
+    }
+    tc::tc_fence_before_sync();
+    __syncthreads();
+    tc::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+                const int m0 = (tile % p.tiles_m) * BM, n0 = (tile / p.tiles_m) * BN;
+                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    if (!tc::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
+                    uint8_t *sa = smem + (size_t)s * STAGE_BYTES, *sb = sa + A_BYTES;
+                    tc::mbar_expect_tx(&full[s], STAGE_BYTES);
+                    const int k0 = kb * BK;
+                    if (A_MN) {
+#pragma unroll
+                        for (int i = 0; i < BM / 64; ++i) tc::tma_load_2d(sa + i * MN_BOX_BYTES, &tm_a, &full[s], m0 + i * 64, k0);
+                    } else {
+                        tc::tma_load_2d(sa, &tm_a, &full[s], k0, m0);
+                    }
+                    if (B_MN) {
+#pragma unroll
+                        for (int i = 0; i < BN / 64; ++i) tc::tma_load_2d(sb + i * MN_BOX_BYTES, &tm_b, &full[s], n0 + i * 64, k0);
+                    } else {
+                        tc::tma_load_2d(sb, &tm_b, &full[s], k0, n0);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            constexpr uint32_t idesc = tc::instr_desc_bf16(BM, BN, A_MN, B_MN);
+            // K-major: 8-row atoms 1024 B apart, one MMA (16 k) = 32 bytes along the swizzled row;
+            // MN-major: 64-wide M/N groups one TMA box apart, 8-k atoms 1024 B apart, one MMA = 2 atoms.
+            constexpr uint32_t a_lbo = A_MN ? MN_BOX_BYTES : 16, b_lbo = B_MN ? MN_BOX_BYTES : 16;
+            constexpr uint32_t a_step = A_MN ? 2048 : 32, b_step = B_MN ? 2048 : 32;
+            uint32_t it = 0, t_local = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++t_local) {
+                const int buf = t_local & 1;
+                if (!tc::mbar_wait(&tmem_empty[buf], ((t_local >> 1) & 1) ^ 1, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) break;
+                tc::tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + buf * BN;
+                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    if (!tc::mbar_wait(&full[s], (it / STAGES) & 1, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
+                    tc::tc_fence_after_sync();
+                    const uint32_t sa = tc::smem_u32(smem + (size_t)s * STAGE_BYTES), sb = sa + A_BYTES;
+#pragma unroll
+                    for (int kk = 0; kk < BK / 16; ++kk) {
+                        const uint64_t da = tc::smem_desc(sa + kk * a_step, a_lbo, 1024);
+                        const uint64_t db = tc::smem_desc(sb + kk * b_step, b_lbo, 1024);
+                        tc::mma_bf16(d_tmem, da, db, idesc, (kb | kk) != 0);
+                    }
+                    tc::mma_commit(&empty[s]);          // the stage is free once these MMAs have read it
+                }
+                if (ok) tc::mma_commit(&tmem_full[buf]);  // the accumulator is complete
+            }
+        }
+    } else {
+        // ---------------- epilogue (4 warps, 128 threads) ----------------
+        const int quarter = warp & 3;                     // TMEM lanes [32*quarter, 32*quarter+32)
+        uint32_t t_local = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++t_local) {
+            const int buf = t_local & 1;
+            const int m0 = (tile % p.tiles_m) * BM, n0 = (tile / p.tiles_m) * BN;
+            // one lane polls, the warp follows its verdict (keeps the warp converged for tcgen05.ld)
+            int ok = 1;
+            if (lane == 0) ok = tc::mbar_wait(&tmem_full[buf], (t_local >> 1) & 1, abort_flag, p.err, tc::ERR_WAIT_TMEM_FULL) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            tc::tc_fence_after_sync();
+            const int row = m0 + quarter * 32 + lane;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * BN;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t r[32];
+                tc::tmem_ld_32x32(taddr + c * 32, r);
+                tc::tmem_ld_wait();
+                const int nc = n0 + c * 32;
+                // lane j fetches the bias of column nc + j; every lane then reads all 32 by shuffle
+                float bias_lane = 0.0f;
+                if (p.bias != nullptr && nc + lane < p.N)
+                    bias_lane = p.bias_bf16 ? __bfloat162float(((const __nv_bfloat16 *)p.bias)[nc + lane]) : ((const float *)p.bias)[nc + lane];
+                float v[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) + __shfl_sync(0xffffffffu, bias_lane, j);
+                if (row < p.M && nc < p.N) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const float z = v[j];
+                        v[j] = p.out_f32 ? act_fwd<false>(z, p.act) : act_fwd<true>(z, p.act);
+                    }
+                    if (p.out_f32) {
+                        float *dst = (float *)p.c + (long long)row * p.ldc + nc;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            if (nc + j < p.N) *reinterpret_cast<float4 *>(dst + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                    } else {
+                        __nv_bfloat16 *dst = (__nv_bfloat16 *)p.c + (long long)row * p.ldc + nc;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8)
+                            if (nc + j < p.N)
+                                *reinterpret_cast<uint4 *>(dst + j) = make_uint4(pack2(v[j], v[j + 1]), pack2(v[j + 2], v[j + 3]),
+                                                                                 pack2(v[j + 4], v[j + 5]), pack2(v[j + 6], v[j + 7]));
+                    }
+                }
+            }
+            tc::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(&tmem_empty[buf]);
+        }
+    }
+
+    tc::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc::tc_fence_after_sync();
+        tc::tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ---- host ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    });
+    return fn;
+}
+
+}  // namespace
+
+// 2-D bf16 tensor map: `inner` contiguous elements per row, `outer` rows `row_stride` elements apart,
+// box = box_inner x box_outer, 128-byte swizzle, out-of-range elements read as zero
+relay_status_t make_tmap_2d_bf16(CUtensorMap *m, const void *base, uint64_t inner, uint64_t outer, uint64_t row_stride,
+                                 uint32_t box_inner, uint32_t box_outer)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return fail(RELAY_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    cuuint64_t dims[2] = {inner, outer};
+    cuuint64_t strides[1] = {row_stride * 2};
+    cuuint32_t box[2] = {box_inner, box_outer};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(RELAY_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    return RELAY_OK;
+}
+
+bool gemm_tc_eligible(const GemmDesc &g)
+{
+    if (g.in_dtype != RELAY_BF16) return false;
+    if (g.out_dtype != RELAY_BF16 && g.out_dtype != RELAY_F32) return false;
+    if (g.M % 8 || g.N % 8 || g.K % 8 || g.ldc % 8) return false;
+    if (g.M < 64 || g.N < 64 || g.K < 64) return false;                 // too small to fill a tile: SIMT kernel
+    if (g.M > (1ll << 30) || g.N > (1ll << 30) || g.K > (1ll << 30)) return false;
+    if (((uintptr_t)g.a | (uintptr_t)g.b | (uintptr_t)g.c) & 15) return false;
+    const bool a_ok = (g.a_sk == 1 && g.a_sm % 8 == 0) || (g.a_sm == 1 && g.a_sk % 8 == 0);
+    const bool b_ok = (g.b_sk == 1 && g.b_sn % 8 == 0) || (g.b_sn == 1 && g.b_sk % 8 == 0);
+    return a_ok && b_ok;
+}
+
+relay_status_t launch_gemm_tc(const GemmDesc &g, cudaStream_t st)
+{
+    const bool a_mn = g.a_sk != 1, b_mn = g.b_sk != 1;
+    CUtensorMap tm_a, tm_b;
+    if (a_mn) RELAY_TRY(make_tmap_2d_bf16(&tm_a, g.a, g.M, g.K, g.a_sk, 64, BK));       // rows = k, inner = m
+    else RELAY_TRY(make_tmap_2d_bf16(&tm_a, g.a, g.K, g.M, g.a_sm, BK, BM));             // rows = m, inner = k
+    if (b_mn) RELAY_TRY(make_tmap_2d_bf16(&tm_b, g.b, g.N, g.K, g.b_sk, 64, BK));       // rows = k, inner = n
+    else RELAY_TRY(make_tmap_2d_bf16(&tm_b, g.b, g.K, g.N, g.b_sn, BK, BN));             // rows = n, inner = k
+    Params p{};
+    p.M = (int)g.M; p.N = (int)g.N; p.K = (int)g.K;
+    p.c = g.c; p.ldc = g.ldc;
+    p.bias = g.bias; p.bias_bf16 = g.bias_dtype == RELAY_BF16; p.act = g.act; p.out_f32 = g.out_dtype == RELAY_F32;
+    p.tiles_m = (int)((g.M + BM - 1) / BM); p.tiles_n = (int)((g.N + BN - 1) / BN); p.k_blocks = (int)((g.K + BK - 1) / BK);
+    p.err = device_error_word();
+    if (!p.err) return fail(RELAY_ERR_CUDA, "no device error word");
+    int dev = 0, sms = 148;
+    RELAY_CUDA(cudaGetDevice(&dev));
+    RELAY_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const int grid = std::min(p.tiles_m * p.tiles_n, sms);
+#define LAUNCH(AMN, BMN)                                                                                          \
+    do {                                                                                                          \
+        RELAY_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<AMN, BMN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES)); \
+        gemm_tc_kernel<AMN, BMN><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tm_a, tm_b, p);                           \
+    } while (0)
+    if (a_mn && b_mn) LAUNCH(true, true);
+    else if (a_mn) LAUNCH(true, false);
+    else if (b_mn) LAUNCH(false, true);
+    else LAUNCH(false, false);
+#undef LAUNCH
+    return check_launch("gemm_tc");
+}
 
 }  // namespace relay

@@ -47,7 +47,8 @@ def test_conv_small_shapes_forward_and_gradient(N, C, H, W, O, R, stride, pad, t
     chk(y, want, what="y")
     dy = I.normal(4, 3, tuple(y.shape), 1.0, tdt, salt=H)
     dx, dw, db = conv_grad(t["x"], t["w"], y, dy, stride, pad, act)
-    odx, odw, odb = oracle.conv2d_act_grad(xo, wo, to_np(y), I.as_f64(dy), stride, pad, act, F64, F64, F64)
+    odx, odw, odb = oracle.conv2d_act_grad(xo, wo, to_np(y), I.as_f64(dy), stride, pad, act, F64, F64, F64,
+                                           dz_dtype=oracle.F32 if tdt == torch.float32 else oracle.BF16)
     chk(dx, odx, what="dx"); chk(dw, odw, what="dw")
     (assert_f32 if tdt == torch.float32 else (lambda g, o, what: assert_bf16(g, o, stored_bf16=False, what=what)))(db, odb, what="db")
 

@@ -47,11 +47,12 @@ def test_tiny_mlp_layer_fp32_forward_and_gradient(act):
         z = xo @ wo + bo
         assert bool((y.cpu()[torch.from_numpy(z < -1e-3)] == 0).all())      # exact zeros stay exact
     dx, dw, db = run_grad(t["x"], t["w"], y, t["dy"], act)
-    odx, odw, odb = oracle.dense_act_grad(xo, wo, to_np(y), dyo, act, F64, F64, F64)   # the saved y decides the mask
+    odx, odw, odb = oracle.dense_act_grad(xo, wo, to_np(y), dyo, act, F64, F64, F64, dz_dtype=oracle.F32)   # the saved y decides the mask
     assert_f32(dx, odx, what="dx"); assert_f32(dw, odw, what="dw"); assert_f32(db, odb, what="db")
 
 
-@pytest.mark.parametrize("M,K,N", [(1, 1, 1), (37, 53, 29), (130, 70, 200), (64, 64, 64), (5, 300, 8)])
+@pytest.mark.parametrize("M,K,N", [(1, 1, 1), (37, 53, 29), (130, 70, 200), (64, 64, 64), (5, 300, 8),
+                                   (128, 64, 256), (200, 136, 264), (384, 512, 320), (72, 1032, 520)])
 @pytest.mark.parametrize("tdt", [torch.float32, torch.bfloat16])
 def test_odd_shapes_forward_and_gradient(M, K, N, tdt):
     t = I.cfg1_tiny_mlp(M, K, N, salt=M)
@@ -63,7 +64,9 @@ def test_odd_shapes_forward_and_gradient(M, K, N, tdt):
     chk = assert_f32 if tdt == torch.float32 else assert_bf16
     chk(y, oracle.dense_act(xo, wo, bo, act, F64), what="y")
     dx, dw, db = run_grad(x, w, y, dy, act)
-    odx, odw, odb = oracle.dense_act_grad(xo, wo, to_np(y), dyo, act, F64, F64, F64)
+    # dZ is a value of the operand type (stored in bf16 / fp32 before the contractions read it)
+    odx, odw, odb = oracle.dense_act_grad(xo, wo, to_np(y), dyo, act, F64, F64, F64,
+                                          dz_dtype=oracle.F32 if tdt == torch.float32 else oracle.BF16)
     chk(dx, odx, what="dx"); chk(dw, odw, what="dw")
     if tdt == torch.float32:
         assert_f32(db, odb, what="db")
