@@ -36,7 +36,8 @@ static void flat_view(int64_t total, int32_t dt, int64_t *rows, int64_t *cols)
 static size_t conv_grad_ws(const ConvDims &d, size_t *dz_bytes)
 {
     *dz_bytes = align_up((size_t)(d.Nb * d.O * d.P * d.Q) * dtype_size(d.dt), 256);
-    return *dz_bytes + (conv_tc_eligible(d) ? align_up(conv_tc_grad_workspace(d), 256) : 0);
+    if (conv_tc_eligible(d)) return conv_tc_grad_workspace(d);   // the tensor-core tier keeps dZ in its own layout
+    return *dz_bytes;
 }
 
 }  // namespace relay
@@ -137,16 +138,14 @@ extern "C" relay_status_t relay_fused_conv2d_act_grad(const relay_tensor_t *x, c
         if (db && numel(db)) RELAY_CUDA(cudaMemsetAsync(db->data, 0, nbytes(db), st));
         return RELAY_OK;
     }
+    if (conv_tc_eligible(d))
+        return launch_conv_grad_tc(d, x->data, w->data, y->data, dy->data, act, dx ? dx->data : nullptr, dw->data,
+                                   db ? (float *)db->data : nullptr, ws, st);
     void *dz = ws;
-    void *tc_ws = (char *)ws + dz_bytes;
     int64_t rows, cols;
     flat_view(ny, d.dt, &rows, &cols);
     RELAY_TRY(act_grad_any(d.dt, dy->data, y->data, dz, nullptr, nullptr, rows, cols, act, st));
     if (db) RELAY_TRY(launch_conv_db(d, dz, (float *)db->data, st));
-    if (conv_tc_eligible(d)) {
-        if (dx) RELAY_TRY(launch_conv_dx_tc(d, dz, w->data, dx->data, tc_ws, st));
-        return launch_conv_dw_tc(d, dz, x->data, dw->data, tc_ws, st);
-    }
     if (dx) RELAY_TRY(launch_conv_dx_direct(d, dz, w->data, dx->data, st));
     return launch_conv_dw_direct(d, dz, x->data, dw->data, st);
 }

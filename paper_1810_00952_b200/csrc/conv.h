@@ -22,7 +22,8 @@ size_t conv_tc_fwd_workspace(const ConvDims &d);
 size_t conv_tc_grad_workspace(const ConvDims &d);
 relay_status_t launch_conv_fwd_tc(const ConvDims &d, const void *x, const void *w, const void *b, int32_t b_dt, int act, void *y,
                                   void *ws, cudaStream_t st);
-relay_status_t launch_conv_dx_tc(const ConvDims &d, const void *dz, const void *w, void *dx, void *ws, cudaStream_t st);
-relay_status_t launch_conv_dw_tc(const ConvDims &d, const void *dz, const void *x, void *dw, void *ws, cudaStream_t st);
+// whole gradient group: dZ = dy (.) act'(y) (kept in NHWC), db, dx (if wanted), dw
+relay_status_t launch_conv_grad_tc(const ConvDims &d, const void *x, const void *w, const void *y, const void *dy, int act, void *dx,
+                                   void *dw, float *db, void *ws, cudaStream_t st);
 
 }  // namespace relay

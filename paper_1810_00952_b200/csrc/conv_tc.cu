@@ -1,22 +1,535 @@
-// Implicit-GEMM tensor-core conv2d kernels -- placeholder until the kernels land.
+// conv2d 3x3 / stride 1 / "same" padding as implicit GEMM on the tensor cores (bf16, fp32 accumulate).
+//
+// Layout change first (Section 5.2 of the paper lists change of layout among the optimisations a
+// whole-program IR enables): the NCHW boundary tensors are repacked once per call into NHWC, where
+// a filter tap is a shift along NON-innermost tensor-map axes, so every TMA tile load starts on a
+// 16-byte boundary and the zero padding is the tensor map's out-of-range fill.
+//
+//   forward / input gradient ("fprop" kernel):   D[o, pixel] = sum_{tap, c} Wp[o, tap, c] * Xn[pixel + tap, c]
+//     A = packed weights [O][R*S*C] (K-major), B = NHWC activations (K-major, one 4-D box of
+//     rows_per_tile image rows x W pixels x 64 channels per stage); the accumulator row is an output
+//     channel, so the epilogue writes whole runs of an NCHW image plane with bias + activation fused.
+//     The input gradient is the same kernel on dZ with the taps mirrored and the channel roles swapped.
+//   weight gradient ("wgrad" kernel):             D[o, c] = sum_{pixel} dZn[pixel, o] * Xn[pixel + tap, c]
+//     both operands MN-major (rows are pixels); one work unit = (tap, 128 output channels, slice of the
+//     batch); slices are summed afterwards in a fixed order (split-K without atomics).
+#include <algorithm>
+
 #include "conv.h"
+#include "ewise_host.h"
+#include "ewise_kernels.cuh"
+#include "tc_common.cuh"
 
 namespace relay {
 
-bool conv_tc_eligible(const ConvDims &) { return false; }
-size_t conv_tc_fwd_workspace(const ConvDims &) { return 0; }
-size_t conv_tc_grad_workspace(const ConvDims &) { return 0; }
-relay_status_t launch_conv_fwd_tc(const ConvDims &, const void *, const void *, const void *, int32_t, int, void *, void *, cudaStream_t)
+relay_status_t make_tmap_2d_bf16(CUtensorMap *m, const void *base, uint64_t inner, uint64_t outer, uint64_t row_stride,
+                                 uint32_t box_inner, uint32_t box_outer);
+relay_status_t make_tmap_nhwc_bf16(CUtensorMap *m, const void *base, uint64_t C, uint64_t W, uint64_t H, uint64_t N,
+                                   uint32_t box_c, uint32_t box_w, uint32_t box_h);
+
+namespace {
+
+constexpr int BM = 128, BK = 64;
+constexpr int NUM_THREADS = 192;
+constexpr int TMEM_COLS = 512;
+
+// ---------------------------------------------------------------------------------------------------
+// layout kernels
+// ---------------------------------------------------------------------------------------------------
+// out[n][hw][c] = in[n][c][hw]  (GRAD: in = dy, multiplied by act'(y) on the way: dZ in NHWC)
+template <bool GRAD>
+__global__ void __launch_bounds__(256) nchw_to_nhwc_kernel(const __nv_bfloat16 *__restrict__ in, const __nv_bfloat16 *__restrict__ y,
+                                                            __nv_bfloat16 *__restrict__ out, int C, int HW, int act)
 {
-    return fail(RELAY_ERR_UNSUPPORTED, "tensor-core conv2d not built");
+    __shared__ __nv_bfloat16 tile[64][66];
+    const int n = blockIdx.z, c0 = blockIdx.y * 64, p0 = blockIdx.x * 64;
+    const size_t img = (size_t)n * C * HW;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int idx = threadIdx.x + i * 256;
+        const int cl = idx >> 5, p2 = (idx & 31) * 2;
+        const int c = c0 + cl, p = p0 + p2;
+        float v0 = 0.0f, v1 = 0.0f;
+        if (c < C && p < HW) {   // HW is even, so p + 1 < HW as well
+            const size_t off = img + (size_t)c * HW + p;
+            const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162 *>(in + off);
+            v0 = __low2float(a); v1 = __high2float(a);
+            if (GRAD) {
+                const __nv_bfloat162 yy = *reinterpret_cast<const __nv_bfloat162 *>(y + off);
+                v0 *= act_grad_from_output(__low2float(yy), act);
+                v1 *= act_grad_from_output(__high2float(yy), act);
+            }
+        }
+        tile[cl][p2] = __float2bfloat16_rn(v0);
+        tile[cl][p2 + 1] = __float2bfloat16_rn(v1);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int idx = threadIdx.x + i * 256;
+        const int pl = idx >> 5, c2 = (idx & 31) * 2;
+        const int c = c0 + c2, p = p0 + pl;
+        if (c < C && p < HW) {
+            __nv_bfloat162 v;
+            v.x = tile[c2][pl]; v.y = tile[c2 + 1][pl];
+            *reinterpret_cast<__nv_bfloat162 *>(out + ((size_t)n * HW + p) * C + c) = v;
+        }
+    }
 }
-relay_status_t launch_conv_dx_tc(const ConvDims &, const void *, const void *, void *, void *, cudaStream_t)
+
+// wf[o][tap][c] = w[o][c][tap];   wb[c][mirror(tap)][o] = w[o][c][tap]   (either may be null)
+__global__ void pack_weights_kernel(const __nv_bfloat16 *__restrict__ w, __nv_bfloat16 *__restrict__ wf,
+                                    __nv_bfloat16 *__restrict__ wb, int O, int C, int R, int S)
 {
-    return fail(RELAY_ERR_UNSUPPORTED, "tensor-core conv2d not built");
+    const int64_t total = (int64_t)O * C * R * S;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int s = (int)(i % S);
+        int64_t t = i / S;
+        const int r = (int)(t % R); t /= R;
+        const int c = (int)(t % C);
+        const int o = (int)(t / C);
+        const __nv_bfloat16 v = w[i];
+        if (wf) wf[((int64_t)o * (R * S) + r * S + s) * C + c] = v;
+        if (wb) wb[((int64_t)c * (R * S) + (R - 1 - r) * S + (S - 1 - s)) * O + o] = v;
+    }
 }
-relay_status_t launch_conv_dw_tc(const ConvDims &, const void *, const void *, void *, void *, cudaStream_t)
+
+// dw[o][c][tap] = bf16( sum over slices, in slice order, of part[slice][tap][o][c] )
+__global__ void wgrad_reduce_kernel(const float *__restrict__ part, int n_slices, __nv_bfloat16 *__restrict__ dw, int O, int C, int taps)
 {
-    return fail(RELAY_ERR_UNSUPPORTED, "tensor-core conv2d not built");
+    const int64_t per_slice = (int64_t)taps * O * C;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < per_slice; i += (int64_t)gridDim.x * blockDim.x) {
+        const int tap = (int)(i % taps);          // i enumerates the OUTPUT (o, c, tap) so that stores coalesce
+        const int64_t oc = i / taps;
+        const int c = (int)(oc % C);
+        const int o = (int)(oc / C);
+        float s = 0.0f;
+        for (int j = 0; j < n_slices; ++j) s += part[(size_t)j * per_slice + ((int64_t)tap * O + o) * C + c];
+        dw[i] = __float2bfloat16_rn(s);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// fprop kernel: 128 output channels x (rows_per_tile * W) pixels per tile
+// ---------------------------------------------------------------------------------------------------
+struct FpropParams {
+    int Cin, Cout, H, W, Nb, taps_r, taps_s, pad;
+    int rows_per_tile, nt;      // nt = rows_per_tile * W = UMMA N
+    int m_tiles, tiles_per_img, n_tiles_total, k_blocks, stages;
+    __nv_bfloat16 *out;         // NCHW [Nb][Cout][H][W]
+    const void *bias;           // per output channel, or null
+    int bias_bf16, act;
+    int *err;
+};
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+conv_fprop_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, const FpropParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int a_bytes = BM * BK * 2, b_bytes = p.nt * BK * 2;
+    const int stage_bytes = a_bytes + ((b_bytes + 1023) & ~1023);
+    const int STAGES = p.stages;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + (size_t)STAGES * stage_bytes);
+    uint64_t *full = bars, *empty = bars + STAGES, *tmem_full = bars + 2 * STAGES, *tmem_empty = bars + 2 * STAGES + 2;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 4);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_tiles = p.m_tiles * p.n_tiles_total;
+    const int cblocks = p.Cin / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { tc::mbar_init(&tmem_full[b], 1); tc::mbar_init(&tmem_empty[b], 4); }
+        *abort_flag = 0;
+        tc::fence_barrier_init();
+        tc::prefetch_tmap(&tm_w);
+        tc::prefetch_tmap(&tm_x);
+    }
+    if (warp == 1) { tc::tmem_alloc(tmem_slot, TMEM_COLS); tc::tmem_relinquish(); }
+    tc::tc_fence_before_sync();
+    __syncthreads();
+    tc::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+                const int m0 = (tile % p.m_tiles) * BM;
+                const int nt_idx = tile / p.m_tiles;
+                const int img = nt_idx / p.tiles_per_img, h0 = (nt_idx % p.tiles_per_img) * p.rows_per_tile;
+                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    if (!tc::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
+                    uint8_t *sa = smem + (size_t)s * stage_bytes, *sb = sa + a_bytes;
+                    tc::mbar_expect_tx(&full[s], a_bytes + b_bytes);
+                    const int tap = kb / cblocks, cb = kb % cblocks;
+                    const int r = tap / p.taps_s, sft = tap % p.taps_s;
+                    tc::tma_load_2d(sa, &tm_w, &full[s], kb * BK, m0);
+                    tc::tma_load_4d(sb, &tm_x, &full[s], cb * BK, sft - p.pad, h0 + r - p.pad, img);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = tc::instr_desc_bf16(BM, p.nt, false, false);
+            uint32_t it = 0, t_local = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++t_local) {
+                const int buf = t_local & 1;
+                if (!tc::mbar_wait(&tmem_empty[buf], ((t_local >> 1) & 1) ^ 1, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) break;
+                tc::tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + buf * 256;
+                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    if (!tc::mbar_wait(&full[s], (it / STAGES) & 1, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
+                    tc::tc_fence_after_sync();
+                    const uint32_t sa = tc::smem_u32(smem + (size_t)s * stage_bytes), sb = sa + a_bytes;
+#pragma unroll
+                    for (int kk = 0; kk < BK / 16; ++kk)
+                        tc::mma_bf16(d_tmem, tc::smem_desc(sa + kk * 32, 16, 1024), tc::smem_desc(sb + kk * 32, 16, 1024), idesc,
+                                     (kb | kk) != 0);
+                    tc::mma_commit(&empty[s]);
+                }
+                if (ok) tc::mma_commit(&tmem_full[buf]);
+            }
+        }
+    } else {
+        const int quarter = warp & 3;
+        uint32_t t_local = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++t_local) {
+            const int buf = t_local & 1;
+            const int m0 = (tile % p.m_tiles) * BM;
+            const int nt_idx = tile / p.m_tiles;
+            const int img = nt_idx / p.tiles_per_img, h0 = (nt_idx % p.tiles_per_img) * p.rows_per_tile;
+            int ok = 1;
+            if (lane == 0) ok = tc::mbar_wait(&tmem_full[buf], (t_local >> 1) & 1, abort_flag, p.err, tc::ERR_WAIT_TMEM_FULL) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            tc::tc_fence_after_sync();
+            const int o = m0 + quarter * 32 + lane;
+            float bias = 0.0f;
+            if (p.bias != nullptr && o < p.Cout)
+                bias = p.bias_bf16 ? __bfloat162float(((const __nv_bfloat16 *)p.bias)[o]) : ((const float *)p.bias)[o];
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * 256;
+            __nv_bfloat16 *dst = p.out + (((size_t)img * p.Cout + o) * p.H + h0) * p.W;
+#pragma unroll 1
+            for (int c = 0; c < p.nt / 32; ++c) {
+                uint32_t r[32];
+                tc::tmem_ld_32x32(taddr + c * 32, r);
+                tc::tmem_ld_wait();
+                if (o < p.Cout) {
+                    float v[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = act_fwd<true>(__uint_as_float(r[j]) + bias, p.act);
+#pragma unroll
+                    for (int j = 0; j < 32; j += 8)
+                        *reinterpret_cast<uint4 *>(dst + c * 32 + j) = make_uint4(pack2(v[j], v[j + 1]), pack2(v[j + 2], v[j + 3]),
+                                                                                 pack2(v[j + 4], v[j + 5]), pack2(v[j + 6], v[j + 7]));
+                }
+            }
+            tc::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(&tmem_empty[buf]);
+        }
+    }
+    tc::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) { tc::tc_fence_after_sync(); tc::tmem_dealloc(tmem_base, TMEM_COLS); }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// wgrad kernel: one work unit = (tap, 128 output channels, NT input channels, batch slice)
+// ---------------------------------------------------------------------------------------------------
+struct WgradParams {
+    int C, O, H, W, Nb, taps_r, taps_s, pad;
+    int rows_per_kblock, kpix;           // kpix = rows_per_kblock * W pixels per k-block
+    int nt;                              // input channels per unit (UMMA N)
+    int m_tiles, c_tiles, n_slices, imgs_per_slice, stages;
+    float *part;                         // [slice][tap][O][C]
+    int *err;
+};
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_dz, const __grid_constant__ CUtensorMap tm_x, const WgradParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int box_bytes = p.kpix * 128;                 // 64 channels x kpix pixel rows
+    const int a_bytes = (BM / 64) * box_bytes, b_bytes = (p.nt / 64) * box_bytes;
+    const int stage_bytes = a_bytes + b_bytes;
+    const int STAGES = p.stages;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + (size_t)STAGES * stage_bytes);
+    uint64_t *full = bars, *empty = bars + STAGES, *tmem_full = bars + 2 * STAGES;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 2);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // decode the work unit of this block
+    int u = blockIdx.x;
+    const int slice = u % p.n_slices; u /= p.n_slices;
+    const int ct = u % p.c_tiles; u /= p.c_tiles;
+    const int mt = u % p.m_tiles; u /= p.m_tiles;
+    const int tap = u;
+    const int r = tap / p.taps_s, sft = tap % p.taps_s;
+    const int img0 = slice * p.imgs_per_slice, img1 = min(p.Nb, img0 + p.imgs_per_slice);
+    const int kb_per_img = p.H / p.rows_per_kblock;
+    const int k_blocks = max(0, img1 - img0) * kb_per_img;
+    const int o0 = mt * BM, c0 = ct * p.nt;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
+        tc::mbar_init(&tmem_full[0], 1);
+        *abort_flag = 0;
+        tc::fence_barrier_init();
+        tc::prefetch_tmap(&tm_dz);
+        tc::prefetch_tmap(&tm_x);
+    }
+    if (warp == 1) { tc::tmem_alloc(tmem_slot, 256); tc::tmem_relinquish(); }
+    tc::tc_fence_before_sync();
+    __syncthreads();
+    tc::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int kb = 0; kb < k_blocks; ++kb) {
+                const int s = kb % STAGES;
+                if (!tc::mbar_wait(&empty[s], ((kb / STAGES) & 1) ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) break;
+                uint8_t *sa = smem + (size_t)s * stage_bytes, *sb = sa + a_bytes;
+                tc::mbar_expect_tx(&full[s], stage_bytes);
+                const int img = img0 + kb / kb_per_img, h0 = (kb % kb_per_img) * p.rows_per_kblock;
+                for (int i = 0; i < BM / 64; ++i) tc::tma_load_4d(sa + i * box_bytes, &tm_dz, &full[s], o0 + i * 64, 0, h0, img);
+                for (int j = 0; j < p.nt / 64; ++j)
+                    tc::tma_load_4d(sb + j * box_bytes, &tm_x, &full[s], c0 + j * 64, sft - p.pad, h0 + r - p.pad, img);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = tc::instr_desc_bf16(BM, p.nt, true, true);
+            bool ok = true;
+            for (int kb = 0; kb < k_blocks; ++kb) {
+                const int s = kb % STAGES;
+                if (!tc::mbar_wait(&full[s], (kb / STAGES) & 1, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
+                tc::tc_fence_after_sync();
+                const uint32_t sa = tc::smem_u32(smem + (size_t)s * stage_bytes), sb = sa + a_bytes;
+                for (int kk = 0; kk < p.kpix / 16; ++kk)
+                    tc::mma_bf16(tmem_base, tc::smem_desc(sa + kk * 2048, box_bytes, 1024), tc::smem_desc(sb + kk * 2048, box_bytes, 1024),
+                                 idesc, (kb | kk) != 0);
+                tc::mma_commit(&empty[s]);
+            }
+            if (ok) tc::mma_commit(&tmem_full[0]);
+        }
+    } else {
+        const int quarter = warp & 3;
+        int ok = 1;
+        if (k_blocks > 0) {
+            if (lane == 0) ok = tc::mbar_wait(&tmem_full[0], 0, abort_flag, p.err, tc::ERR_WAIT_TMEM_FULL) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+        }
+        if (ok) {
+            tc::tc_fence_after_sync();
+            const int o = o0 + quarter * 32 + lane;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+            float *dst = p.part + (((size_t)slice * (p.taps_r * p.taps_s) + tap) * p.O + o) * p.C + c0;
+#pragma unroll 1
+            for (int c = 0; c < p.nt / 32; ++c) {
+                uint32_t v[32];
+                if (k_blocks > 0) {
+                    tc::tmem_ld_32x32(taddr + c * 32, v);
+                    tc::tmem_ld_wait();
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = 0u;
+                }
+                if (o < p.O) {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4)
+                        *reinterpret_cast<uint4 *>(dst + c * 32 + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                }
+            }
+        }
+    }
+    tc::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) { tc::tc_fence_after_sync(); tc::tmem_dealloc(tmem_base, 256); }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// host plans
+// ---------------------------------------------------------------------------------------------------
+struct TcPlan {
+    bool ok = false;
+    int rows_per_tile = 0;   // fprop: image rows per tile (rows*W <= 256, multiple of 32)
+    int rows_per_kblock = 0; // wgrad: image rows per k-block (rows*W multiple of 16, <= 128)
+    int wg_nt = 0, wg_c_tiles = 0, wg_m_tiles = 0, wg_slices = 0, wg_imgs_per_slice = 0, wg_stages = 0;
+    int fp_stages = 0;
+    size_t x_nhwc = 0, dz_nhwc = 0, wpack = 0, part = 0, db_part = 0;
+};
+
+constexpr size_t kSmemLimit = 227 * 1024 - 2048;
+
+TcPlan plan(const ConvDims &d)
+{
+    TcPlan pl;
+    if (d.dt != RELAY_BF16 || d.stride != 1 || d.R != 3 || d.S != 3 || d.pad != 1) return pl;
+    if (d.C % 128 || d.O % 128 || d.W % 8 || d.W > 256 || d.H < 1 || d.Nb < 1) return pl;
+    if (d.Nb > 65535 || d.H * d.W > (1 << 24)) return pl;
+    for (int rt = (int)std::min<int64_t>(d.H, 256 / d.W); rt >= 1; --rt)
+        if (d.H % rt == 0 && (rt * d.W) % 32 == 0) { pl.rows_per_tile = rt; break; }
+    for (int rk = (int)std::min<int64_t>(d.H, 128 / d.W); rk >= 1; --rk)
+        if (d.H % rk == 0 && (rk * d.W) % 16 == 0) { pl.rows_per_kblock = rk; break; }
+    if (!pl.rows_per_tile || !pl.rows_per_kblock) return pl;
+    // fprop stages
+    const size_t fp_stage = BM * BK * 2 + (((size_t)pl.rows_per_tile * d.W * BK * 2 + 1023) & ~size_t(1023));
+    pl.fp_stages = (int)std::min<size_t>(6, (kSmemLimit - 1024) / fp_stage);
+    if (pl.fp_stages < 2) return pl;
+    // wgrad tiling
+    pl.wg_nt = (int)std::min<int64_t>(256, d.C);
+    const size_t box = (size_t)pl.rows_per_kblock * d.W * 128;
+    auto wg_stage = [&](int nt) { return (size_t)(BM / 64 + nt / 64) * box; };
+    while (pl.wg_nt > 64 && (kSmemLimit - 1024) / wg_stage(pl.wg_nt) < 2) pl.wg_nt -= 64;
+    if ((kSmemLimit - 1024) / wg_stage(pl.wg_nt) < 2 || d.C % pl.wg_nt) return pl;
+    pl.wg_stages = (int)std::min<size_t>(4, (kSmemLimit - 1024) / wg_stage(pl.wg_nt));
+    pl.wg_c_tiles = (int)(d.C / pl.wg_nt);
+    pl.wg_m_tiles = (int)(d.O / BM);
+    const int base_units = 9 * pl.wg_m_tiles * pl.wg_c_tiles;
+    int slices = std::max(1, 148 / base_units);
+    slices = (int)std::min<int64_t>(slices, d.Nb);
+    pl.wg_imgs_per_slice = (int)((d.Nb + slices - 1) / slices);
+    pl.wg_slices = (int)((d.Nb + pl.wg_imgs_per_slice - 1) / pl.wg_imgs_per_slice);
+    pl.x_nhwc = align_up((size_t)d.Nb * d.C * d.H * d.W * 2, 1024);
+    pl.dz_nhwc = align_up((size_t)d.Nb * d.O * d.H * d.W * 2, 1024);
+    pl.wpack = align_up((size_t)d.O * d.C * 9 * 2, 1024);
+    pl.part = align_up((size_t)pl.wg_slices * 9 * d.O * d.C * sizeof(float), 1024);
+    pl.db_part = align_up((size_t)colsum_slices(d.Nb * d.H * d.W, d.O, RELAY_BF16) * d.O * sizeof(float), 1024);
+    pl.ok = true;
+    return pl;
+}
+
+relay_status_t launch_fprop(const ConvDims &d, const TcPlan &pl, const void *act_nhwc, int Cin, const void *wpacked, int Cout,
+                            const void *bias, int32_t b_dt, int act, void *out_nchw, cudaStream_t st)
+{
+    CUtensorMap tm_w, tm_x;
+    RELAY_TRY(make_tmap_2d_bf16(&tm_w, wpacked, (uint64_t)9 * Cin, Cout, (uint64_t)9 * Cin, BK, BM));
+    RELAY_TRY(make_tmap_nhwc_bf16(&tm_x, act_nhwc, Cin, d.W, d.H, d.Nb, BK, (uint32_t)d.W, pl.rows_per_tile));
+    FpropParams p{};
+    p.Cin = Cin; p.Cout = Cout; p.H = (int)d.H; p.W = (int)d.W; p.Nb = (int)d.Nb; p.taps_r = 3; p.taps_s = 3; p.pad = 1;
+    p.rows_per_tile = pl.rows_per_tile; p.nt = pl.rows_per_tile * (int)d.W;
+    p.m_tiles = Cout / BM; p.tiles_per_img = (int)d.H / pl.rows_per_tile; p.n_tiles_total = (int)d.Nb * p.tiles_per_img;
+    p.k_blocks = 9 * Cin / BK; p.stages = pl.fp_stages;
+    p.out = (__nv_bfloat16 *)out_nchw; p.bias = bias; p.bias_bf16 = b_dt == RELAY_BF16; p.act = act;
+    p.err = device_error_word();
+    if (!p.err) return fail(RELAY_ERR_CUDA, "no device error word");
+    const size_t stage = BM * BK * 2 + (((size_t)p.nt * BK * 2 + 1023) & ~size_t(1023));
+    const size_t smem = 1024 + (size_t)p.stages * stage + 256;
+    RELAY_CUDA(cudaFuncSetAttribute(conv_fprop_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int dev = 0, sms = 148;
+    RELAY_CUDA(cudaGetDevice(&dev));
+    RELAY_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const int grid = std::min(p.m_tiles * p.n_tiles_total, sms);
+    conv_fprop_tc_kernel<<<grid, NUM_THREADS, smem, st>>>(tm_w, tm_x, p);
+    return check_launch("conv_fprop_tc");
+}
+
+relay_status_t launch_transpose(bool grad, const void *in, const void *y, void *out, int64_t Nb, int64_t C, int64_t HW, int act,
+                                cudaStream_t st)
+{
+    dim3 grid((unsigned)((HW + 63) / 64), (unsigned)((C + 63) / 64), (unsigned)Nb);
+    if (grad) nchw_to_nhwc_kernel<true><<<grid, 256, 0, st>>>((const __nv_bfloat16 *)in, (const __nv_bfloat16 *)y, (__nv_bfloat16 *)out, (int)C, (int)HW, act);
+    else nchw_to_nhwc_kernel<false><<<grid, 256, 0, st>>>((const __nv_bfloat16 *)in, nullptr, (__nv_bfloat16 *)out, (int)C, (int)HW, act);
+    return check_launch("nchw_to_nhwc");
+}
+
+}  // namespace
+
+relay_status_t make_tmap_nhwc_bf16(CUtensorMap *m, const void *base, uint64_t C, uint64_t W, uint64_t H, uint64_t N,
+                                   uint32_t box_c, uint32_t box_w, uint32_t box_h)
+{
+    typedef CUresult (*Fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                           const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                           CUtensorMapFloatOOBfill);
+    void *fp = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fp, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess)
+        return fail(RELAY_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    cuuint64_t dims[4] = {C, W, H, N};
+    cuuint64_t strides[3] = {C * 2, W * C * 2, H * W * C * 2};
+    cuuint32_t box[4] = {box_c, box_w, box_h, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = ((Fn)fp)(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(RELAY_ERR_CUDA, "cuTensorMapEncodeTiled (NHWC) failed with code %d", (int)r);
+    return RELAY_OK;
+}
+
+bool conv_tc_eligible(const ConvDims &d) { return plan(d).ok; }
+
+size_t conv_tc_fwd_workspace(const ConvDims &d)
+{
+    TcPlan pl = plan(d);
+    return pl.ok ? pl.x_nhwc + pl.wpack : 0;
+}
+
+size_t conv_tc_grad_workspace(const ConvDims &d)
+{
+    TcPlan pl = plan(d);
+    return pl.ok ? pl.x_nhwc + pl.dz_nhwc + pl.wpack + pl.part + pl.db_part : 0;
+}
+
+relay_status_t launch_conv_fwd_tc(const ConvDims &d, const void *x, const void *w, const void *b, int32_t b_dt, int act, void *y,
+                                  void *ws, cudaStream_t st)
+{
+    TcPlan pl = plan(d);
+    char *base = (char *)ws;
+    void *x_nhwc = base, *wf = base + pl.x_nhwc;
+    RELAY_TRY(launch_transpose(false, x, nullptr, x_nhwc, d.Nb, d.C, d.H * d.W, 0, st));
+    pack_weights_kernel<<<256, 256, 0, st>>>((const __nv_bfloat16 *)w, (__nv_bfloat16 *)wf, nullptr, (int)d.O, (int)d.C, 3, 3);
+    RELAY_TRY(check_launch("pack_weights"));
+    return launch_fprop(d, pl, x_nhwc, (int)d.C, wf, (int)d.O, b, b_dt, act, y, st);
+}
+
+relay_status_t launch_conv_grad_tc(const ConvDims &d, const void *x, const void *w, const void *y, const void *dy, int act, void *dx,
+                                   void *dw, float *db, void *ws, cudaStream_t st)
+{
+    TcPlan pl = plan(d);
+    char *base = (char *)ws;
+    void *x_nhwc = base;
+    void *dz_nhwc = base + pl.x_nhwc;
+    void *wb = base + pl.x_nhwc + pl.dz_nhwc;
+    float *part = (float *)(base + pl.x_nhwc + pl.dz_nhwc + pl.wpack);
+    float *db_part = (float *)(base + pl.x_nhwc + pl.dz_nhwc + pl.wpack + pl.part);
+    const int64_t HW = d.H * d.W;
+    // dZ = dy (.) act'(y), written straight into NHWC; x into NHWC
+    RELAY_TRY(launch_transpose(true, dy, y, dz_nhwc, d.Nb, d.O, HW, act, st));
+    RELAY_TRY(launch_transpose(false, x, nullptr, x_nhwc, d.Nb, d.C, HW, 0, st));
+    if (db) RELAY_TRY(launch_colsum_bf16(dz_nhwc, d.Nb * HW, d.O, db_part, db, st));
+    if (dx) {
+        pack_weights_kernel<<<256, 256, 0, st>>>((const __nv_bfloat16 *)w, nullptr, (__nv_bfloat16 *)wb, (int)d.O, (int)d.C, 3, 3);
+        RELAY_TRY(check_launch("pack_weights"));
+        RELAY_TRY(launch_fprop(d, pl, dz_nhwc, (int)d.O, wb, (int)d.C, nullptr, RELAY_F32, RELAY_ACT_NONE, dx, st));
+    }
+    CUtensorMap tm_dz, tm_x;
+    RELAY_TRY(make_tmap_nhwc_bf16(&tm_dz, dz_nhwc, d.O, d.W, d.H, d.Nb, 64, (uint32_t)d.W, pl.rows_per_kblock));
+    RELAY_TRY(make_tmap_nhwc_bf16(&tm_x, x_nhwc, d.C, d.W, d.H, d.Nb, 64, (uint32_t)d.W, pl.rows_per_kblock));
+    WgradParams p{};
+    p.C = (int)d.C; p.O = (int)d.O; p.H = (int)d.H; p.W = (int)d.W; p.Nb = (int)d.Nb; p.taps_r = 3; p.taps_s = 3; p.pad = 1;
+    p.rows_per_kblock = pl.rows_per_kblock; p.kpix = pl.rows_per_kblock * (int)d.W; p.nt = pl.wg_nt;
+    p.m_tiles = pl.wg_m_tiles; p.c_tiles = pl.wg_c_tiles; p.n_slices = pl.wg_slices; p.imgs_per_slice = pl.wg_imgs_per_slice;
+    p.stages = pl.wg_stages; p.part = part; p.err = device_error_word();
+    if (!p.err) return fail(RELAY_ERR_CUDA, "no device error word");
+    const size_t stage = (size_t)(BM / 64 + p.nt / 64) * p.kpix * 128;
+    const size_t smem = 1024 + (size_t)p.stages * stage + 256;
+    RELAY_CUDA(cudaFuncSetAttribute(conv_wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const int grid = 9 * p.m_tiles * p.c_tiles * p.n_slices;
+    conv_wgrad_tc_kernel<<<grid, NUM_THREADS, smem, st>>>(tm_dz, tm_x, p);
+    RELAY_TRY(check_launch("conv_wgrad_tc"));
+    wgrad_reduce_kernel<<<(unsigned)std::min<int64_t>(148 * 8, (9 * d.O * d.C + 255) / 256), 256, 0, st>>>(part, p.n_slices, (__nv_bfloat16 *)dw,
+                                                                                                          (int)d.O, (int)d.C, 9);
+    return check_launch("wgrad_reduce");
 }
 
 }  // namespace relay

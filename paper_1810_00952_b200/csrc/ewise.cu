@@ -449,6 +449,16 @@ relay_status_t launch_act_grad(int32_t storage, const void *dy, const void *y, v
     return RELAY_OK;
 }
 
+relay_status_t launch_colsum_bf16(const void *in, int64_t rows, int64_t cols, float *partials, float *out, cudaStream_t st)
+{
+    Args2D<1, 1> A{};
+    A.in[0] = in; A.out[0] = nullptr; A.partial[0] = partials;
+    A.rows = rows; A.cols = cols; A.aux = 0;
+    const int ns = colsum_slices(rows, cols, RELAY_BF16);
+    RELAY_TRY(launch_body2d<BodyIdentityColSum>(RELAY_BF16, A, ns, st, "ewise2d<identity_colsum>"));
+    return launch_colsum_finalize(partials, ns, cols, 1.0f, out, st);
+}
+
 static relay_status_t check_output(const relay_tensor_t *o, int32_t dtype, int rank, const int64_t *shape, int k)
 {
     char name[32];

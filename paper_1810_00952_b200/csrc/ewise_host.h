@@ -14,6 +14,10 @@ int colsum_slices(int64_t rows, int64_t cols, int32_t storage);
 relay_status_t launch_act_grad(int32_t storage, const void *dy, const void *y, void *dz, float *db, float *partials,
                                int64_t rows, int64_t cols, int act, cudaStream_t st);
 
+// out[c] = sum_r in[r,c] for a bf16 [rows, cols] tensor (cols a multiple of 8); `partials` holds
+// colsum_slices(rows, cols, RELAY_BF16) * cols floats
+relay_status_t launch_colsum_bf16(const void *in, int64_t rows, int64_t cols, float *partials, float *out, cudaStream_t st);
+
 relay_status_t launch_colsum_finalize(const float *partial, int n_slices, int64_t cols, float scale, float *out,
                                       cudaStream_t st);
 

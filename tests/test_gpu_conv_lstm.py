@@ -53,15 +53,25 @@ def test_conv_small_shapes_forward_and_gradient(N, C, H, W, O, R, stride, pad, t
     (assert_f32 if tdt == torch.float32 else (lambda g, o, what: assert_bf16(g, o, stored_bf16=False, what=what)))(db, odb, what="db")
 
 
-def test_conv_reduced_config_bf16_3x3():
-    """Configuration 4's structure (3x3, stride 1, pad 1, NCHW/OIHW, bf16) at N=2, C=64, 28x28, O=64."""
-    t = I.cfg4_conv(2, 64, 28, 28, 64)
+@pytest.mark.parametrize("N,C,H,W,O", [(2, 64, 28, 28, 64), (2, 128, 16, 16, 128), (3, 128, 12, 24, 256), (1, 128, 56, 56, 128)])
+def test_conv_reduced_config_bf16_3x3(N, C, H, W, O):
+    """Configuration 4's structure (3x3, stride 1, pad 1, NCHW/OIHW, bf16) at reduced sizes; the shapes
+    with C and O multiples of 128 take the implicit-GEMM tensor-core kernels (several tiles, batch
+    slices of unequal size), the first one the direct kernels."""
+    t = I.cfg4_conv(N, C, H, W, O, salt=C + W)
     y = conv_fwd(t["x"], t["w"], t["b"], 1, 1, B.ACT_RELU)
     xo, wo, bo, dyo = (I.as_f64(t[k]) for k in ("x", "w", "b", "dy"))
     assert_bf16(y, oracle.conv2d_act(xo, wo, bo, 1, 1, B.ACT_RELU, F64), what="y")
     dx, dw, db = conv_grad(t["x"], t["w"], y, t["dy"], 1, 1, B.ACT_RELU)
-    odx, odw, odb = oracle.conv2d_act_grad(xo, wo, to_np(y), dyo, 1, 1, B.ACT_RELU, F64, F64, F64)
+    odx, odw, odb = oracle.conv2d_act_grad(xo, wo, to_np(y), dyo, 1, 1, B.ACT_RELU, F64, F64, F64, dz_dtype=oracle.BF16)
     assert_bf16(dx, odx, what="dx"); assert_bf16(dw, odw, what="dw"); assert_bf16(db, odb, stored_bf16=False, what="db")
+    # tanh epilogue and no bias / no dx / no db through the same kernels
+    y2 = conv_fwd(t["x"], t["w"], None, 1, 1, B.ACT_TANH)
+    assert_bf16(y2, oracle.conv2d_act(xo, wo, None, 1, 1, B.ACT_TANH, F64), what="y tanh")
+    _, dw2, _ = conv_grad(t["x"], t["w"], y2, t["dy"], 1, 1, B.ACT_TANH, want_dx=False, want_db=False)
+    _, odw2, _ = oracle.conv2d_act_grad(xo, wo, to_np(y2), dyo, 1, 1, B.ACT_TANH, F64, F64, F64, want_dx=False, want_db=False,
+                                        dz_dtype=oracle.BF16)
+    assert_bf16(dw2, odw2, what="dw tanh")
 
 
 def test_conv_rejections():
