@@ -6,6 +6,7 @@
 // h_all[t-1] is the running hidden state.
 #include "ewise_kernels.cuh"
 #include "gemm.h"
+#include "lstm.h"
 
 namespace relay {
 
@@ -80,7 +81,11 @@ static relay_status_t check_lstm(const relay_tensor_t *x, const relay_tensor_t *
     return RELAY_OK;
 }
 
-static size_t lstm_ws(const LstmDims &d) { return align_up((size_t)d.T * d.B * 4 * d.H * sizeof(float), 256); }
+static size_t lstm_zx_bytes(const LstmDims &d) { return align_up((size_t)d.T * d.B * 4 * d.H * sizeof(float), 1024); }
+static size_t lstm_ws(const LstmDims &d)
+{
+    return lstm_zx_bytes(d) + (lstm_tc_eligible(d.T, d.B, d.H) ? lstm_tc_workspace(d.B, d.H) : 0);
+}
 
 }  // namespace relay
 
@@ -136,7 +141,10 @@ extern "C" relay_status_t relay_lstm_cell_seq(const relay_tensor_t *x, const rel
     g.act = RELAY_ACT_NONE;
     RELAY_TRY(launch_gemm(g, st));
 
-    // (2) the dependent steps
+    // (2) the dependent steps: one persistent kernel when the shape fits it, else one launch per step
+    if (lstm_tc_eligible(d.T, d.B, d.H))
+        return launch_lstm_tc(d.T, d.B, d.H, zx, w_hh->data, (const float *)h0->data, (const float *)c0->data, (float *)h_all->data,
+                              (float *)c_final->data, (char *)ws + lstm_zx_bytes(d), st);
     dim3 grid((unsigned)((d.H + 255) / 256), (unsigned)((d.B + kRowsPerBlock - 1) / kRowsPerBlock));
     float *hall = (float *)h_all->data;
     for (int64_t t = 0; t < d.T; ++t) {

@@ -1,0 +1,15 @@
+// Persistent tensor-core kernel for the recurrent half of the LSTM sequence.
+#pragma once
+#include "common.h"
+
+namespace relay {
+
+// B <= 128, H a multiple of 64 and <= 1024 (the block's slice of W_hh must fit in shared memory),
+// H / 16 blocks co-resident on the device
+bool lstm_tc_eligible(int64_t T, int64_t B, int64_t H);
+size_t lstm_tc_workspace(int64_t B, int64_t H);
+// zx: [T*B][4H] fp32 (input projection + bias); runs all T steps
+relay_status_t launch_lstm_tc(int64_t T, int64_t B, int64_t H, const float *zx, const void *w_hh, const float *h0, const float *c0,
+                              float *h_all, float *c_final, void *ws, cudaStream_t st);
+
+}  // namespace relay

@@ -1,0 +1,285 @@
+// Recurrent half of the LSTM sequence as ONE persistent cooperative kernel (sm_100a).
+//
+// Block j owns 16 hidden units (64 gate columns: i, f, g, o of those units).  Its slice of W_hh
+// (64 columns x H, bf16) is loaded once by TMA and stays in shared memory for all T steps; the
+// running cell state of its units lives in registers.  Each step:
+//   loader warps copy bf16(h_{t-1}) [B x H] from the exchange buffer in L2 into a 4-stage shared
+//   memory ring (128-byte swizzle written by hand)  ->  one thread issues tcgen05.mma
+//   (D[batch row, 64 gate columns] in TMEM)  ->  epilogue warps add the precomputed input projection,
+//   apply the gates, update c, write h_t (fp32 to h_all, bf16 to the exchange buffer)  ->  grid barrier.
+// The grid barrier is a counter in global memory with a bounded spin; the kernel is launched
+// cooperatively so that all blocks are resident.
+#include <cooperative_groups.h>
+
+#include "ewise_kernels.cuh"
+#include "lstm.h"
+#include "tc_common.cuh"
+
+namespace relay {
+
+relay_status_t make_tmap_2d_bf16(CUtensorMap *m, const void *base, uint64_t inner, uint64_t outer, uint64_t row_stride,
+                                 uint32_t box_inner, uint32_t box_outer);
+
+namespace {
+
+constexpr int UNITS = 16, NCOL = 4 * UNITS;      // hidden units and gate columns per block
+constexpr int BK = 64, STAGES = 4;
+constexpr int A_STAGE = 128 * BK * 2;            // 128 batch rows (rows >= B stay zero) x 64 k
+constexpr int W_KB = NCOL * BK * 2;              // one k-block of the resident W slice
+constexpr int NUM_THREADS = 256;                 // warps 0-3 epilogue, warp 4 MMA, warps 5-7 loaders
+constexpr int N_LOADERS = 96;
+
+struct Params {
+    int T, B, H, n_blocks, k_blocks;
+    const float *zx;                 // [T*B][4H] input projection + bias
+    const float *h0, *c0;            // [B][H]
+    float *h_all, *c_final;          // [T][B][H], [B][H]
+    __nv_bfloat16 *hq;               // [2][B][H] exchange buffer for bf16(h)
+    unsigned int *counter;           // grid barrier
+    int *err;
+};
+
+__device__ __forceinline__ unsigned int ld_acquire(const unsigned int *p)
+{
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void red_release_add(unsigned int *p, unsigned int v)
+{
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ float fast_sigmoid(float x) { return __fdividef(1.0f, 1.0f + __expf(-x)); }
+__device__ __forceinline__ float fast_tanh(float x) { return 1.0f - __fdividef(2.0f, 1.0f + __expf(2.0f * x)); }
+
+__global__ void __launch_bounds__(NUM_THREADS, 1) lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const Params p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t *w_s = smem;                                           // [k_blocks][64 cols x 128 B]
+    uint8_t *a_s = smem + (size_t)p.k_blocks * W_KB;               // [STAGES][128 rows x 128 B]
+    uint64_t *bars = reinterpret_cast<uint64_t *>(a_s + (size_t)STAGES * A_STAGE);
+    uint64_t *full = bars, *empty = bars + STAGES, *w_full = bars + 2 * STAGES, *tmem_full = bars + 2 * STAGES + 1;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 2);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int j0 = blockIdx.x * UNITS;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], N_LOADERS); tc::mbar_init(&empty[s], 1); }
+        tc::mbar_init(w_full, 1);
+        tc::mbar_init(tmem_full, 1);
+        *abort_flag = 0;
+        tc::fence_barrier_init();
+        tc::prefetch_tmap(&tm_w);
+    }
+    // rows >= B of every ring stage are zero for the whole kernel
+    for (int i = threadIdx.x; i < STAGES * A_STAGE / 16; i += NUM_THREADS) reinterpret_cast<uint4 *>(a_s)[i] = make_uint4(0, 0, 0, 0);
+    tc::fence_proxy_async();
+    if (warp == 4) { tc::tmem_alloc(tmem_slot, 64); tc::tmem_relinquish(); }
+    tc::tc_fence_before_sync();
+    __syncthreads();
+    tc::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp < 4) {
+        // ------------------------------ epilogue / state owners ------------------------------
+        const int b = warp * 32 + lane;               // batch row = TMEM lane
+        const bool live = b < p.B;
+        float c[UNITS];
+#pragma unroll
+        for (int i = 0; i < UNITS; ++i) c[i] = live ? p.c0[(size_t)b * p.H + j0 + i] : 0.0f;
+        // publish bf16(h0) of the owned units, then arrive for "step -1"
+        if (live) {
+            uint32_t packed[UNITS / 2];
+#pragma unroll
+            for (int i = 0; i < UNITS; i += 2) packed[i / 2] = pack2(p.h0[(size_t)b * p.H + j0 + i], p.h0[(size_t)b * p.H + j0 + i + 1]);
+            uint4 *dst = reinterpret_cast<uint4 *>(p.hq + (size_t)b * p.H + j0);
+            dst[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+            dst[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+        }
+        // every epilogue warp arrives on the grid barrier by itself (no block-level barrier that a
+        // warp which has given up could leave the others waiting on)
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) red_release_add(p.counter, 1u);
+
+        for (int t = 0; t < p.T; ++t) {
+            // the input projection does not depend on h: fetch it while the recurrent product runs
+            float zx[4][UNITS];
+            if (live) {
+                const float *zrow = p.zx + ((size_t)t * p.B + b) * 4 * p.H + j0;
+#pragma unroll
+                for (int g = 0; g < 4; ++g)
+#pragma unroll
+                    for (int i = 0; i < UNITS; i += 4) {
+                        const float4 v = *reinterpret_cast<const float4 *>(zrow + (size_t)g * p.H + i);
+                        zx[g][i] = v.x; zx[g][i + 1] = v.y; zx[g][i + 2] = v.z; zx[g][i + 3] = v.w;
+                    }
+            }
+            int ok = 1;
+            if (lane == 0) ok = tc::mbar_wait(tmem_full, t & 1, abort_flag, p.err, tc::ERR_WAIT_TMEM_FULL) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            tc::tc_fence_after_sync();
+            uint32_t d0[32], d1[32];
+            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16);
+            tc::tmem_ld_32x32(taddr, d0);
+            tc::tmem_ld_32x32(taddr + 32, d1);
+            tc::tmem_ld_wait();
+            tc::tc_fence_before_sync();
+            if (live) {
+                float hn[UNITS];
+#pragma unroll
+                for (int i = 0; i < UNITS; ++i) {
+                    const float zi = __uint_as_float(d0[i]) + zx[0][i];
+                    const float zf = __uint_as_float(d0[16 + i]) + zx[1][i];
+                    const float zg = __uint_as_float(d1[i]) + zx[2][i];
+                    const float zo = __uint_as_float(d1[16 + i]) + zx[3][i];
+                    const float cn = fmaf(fast_sigmoid(zf), c[i], fast_sigmoid(zi) * fast_tanh(zg));
+                    c[i] = cn;
+                    hn[i] = fast_sigmoid(zo) * fast_tanh(cn);
+                }
+                float4 *ho = reinterpret_cast<float4 *>(p.h_all + ((size_t)t * p.B + b) * p.H + j0);
+#pragma unroll
+                for (int i = 0; i < UNITS; i += 4) ho[i / 4] = make_float4(hn[i], hn[i + 1], hn[i + 2], hn[i + 3]);
+                uint4 *hq = reinterpret_cast<uint4 *>(p.hq + ((size_t)((t + 1) & 1) * p.B + b) * p.H + j0);
+                hq[0] = make_uint4(pack2(hn[0], hn[1]), pack2(hn[2], hn[3]), pack2(hn[4], hn[5]), pack2(hn[6], hn[7]));
+                hq[1] = make_uint4(pack2(hn[8], hn[9]), pack2(hn[10], hn[11]), pack2(hn[12], hn[13]), pack2(hn[14], hn[15]));
+            }
+            __threadfence();
+            __syncwarp();
+            if (lane == 0) red_release_add(p.counter, 1u);
+        }
+        if (live) {
+#pragma unroll
+            for (int i = 0; i < UNITS; ++i) p.c_final[(size_t)b * p.H + j0 + i] = c[i];
+        }
+    } else if (warp == 4) {
+        // ------------------------------ W slice load + MMA issue ------------------------------
+        if (lane == 0) {
+            tc::mbar_expect_tx(w_full, (uint32_t)(p.k_blocks * W_KB));
+            for (int kb = 0; kb < p.k_blocks; ++kb) tc::tma_load_2d(w_s + (size_t)kb * W_KB, &tm_w, w_full, kb * BK, blockIdx.x * NCOL);
+            bool ok = tc::mbar_wait(w_full, 0, abort_flag, p.err, tc::ERR_WAIT_FULL);
+            const uint32_t idesc = tc::instr_desc_bf16(128, NCOL, false, false);
+            uint32_t it = 0;
+            for (int t = 0; t < p.T && ok; ++t) {
+                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    if (!tc::mbar_wait(&full[s], (it / STAGES) & 1, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
+                    tc::tc_fence_after_sync();
+                    const uint32_t sa = tc::smem_u32(a_s + (size_t)s * A_STAGE), sb = tc::smem_u32(w_s + (size_t)kb * W_KB);
+#pragma unroll
+                    for (int kk = 0; kk < BK / 16; ++kk)
+                        tc::mma_bf16(tmem_base, tc::smem_desc(sa + kk * 32, 16, 1024), tc::smem_desc(sb + kk * 32, 16, 1024), idesc,
+                                     (kb | kk) != 0);
+                    tc::mma_commit(&empty[s]);
+                }
+                if (ok) tc::mma_commit(tmem_full);
+            }
+        }
+    } else {
+        // ------------------------------ loaders: bf16(h_{t-1}) -> swizzled ring ------------------------------
+        const int lt = threadIdx.x - 160;                         // 0..95
+        const int chunks_per_kb = p.B * 8;                        // 16-byte chunks of one k-block (B rows x 128 B)
+        uint32_t it = 0;
+        bool ok = true;
+        for (int t = 0; t < p.T && ok; ++t) {
+            // grid barrier: every block has published its part of h_{t-1}
+            if (lt == 0) {
+                const unsigned int target = 4u * (unsigned int)p.n_blocks * (unsigned int)(t + 1);   // 4 epilogue warps per block
+                const long long t0 = clock64();
+                unsigned spins = 0;
+                while (ld_acquire(p.counter) < target) {
+                    if ((++spins & 255u) == 0 && (*abort_flag || clock64() - t0 > tc::kWaitLimitCycles)) {
+                        if (!*abort_flag) { *abort_flag = 1; atomicCAS(p.err, 0, tc::ERR_WAIT_STEP); }
+                        break;
+                    }
+                }
+            }
+            asm volatile("bar.sync 2, 96;" ::: "memory");
+            if (*abort_flag) break;
+            const __nv_bfloat16 *hsrc = p.hq + (size_t)(t & 1) * p.B * p.H;
+            for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                const int s = it % STAGES;
+                if (!tc::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
+                uint8_t *dst = a_s + (size_t)s * A_STAGE;
+                for (int ch = lt; ch < chunks_per_kb; ch += N_LOADERS) {
+                    const int row = ch >> 3, c16 = ch & 7;
+                    uint4 v;
+                    const void *src = hsrc + (size_t)row * p.H + kb * BK + c16 * 8;
+                    asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(src) : "memory");
+                    *reinterpret_cast<uint4 *>(dst + row * 128 + ((c16 ^ (row & 7)) << 4)) = v;
+                }
+                tc::fence_proxy_async();
+                tc::mbar_arrive(&full[s]);
+            }
+        }
+    }
+    tc::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 4) { tc::tc_fence_after_sync(); tc::tmem_dealloc(tmem_base, 64); }
+}
+
+// wp[blk][g*16 + i][k] = w_hh[k][g*H + blk*16 + i]
+__global__ void __launch_bounds__(256) pack_whh_kernel(const __nv_bfloat16 *__restrict__ w_hh, __nv_bfloat16 *__restrict__ wp, int H)
+{
+    __shared__ __nv_bfloat16 tile[64][66];     // [k local][column local]
+    const int blk = blockIdx.x, k0 = blockIdx.y * 64;
+    for (int e = threadIdx.x; e < 64 * 64; e += 256) {
+        const int kl = e >> 6, n = e & 63;
+        const int g = n >> 4, i = n & 15;
+        tile[kl][n] = w_hh[(size_t)(k0 + kl) * 4 * H + (size_t)g * H + blk * 16 + i];
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < 64 * 64; e += 256) {
+        const int n = e >> 6, kl = e & 63;
+        wp[((size_t)blk * 64 + n) * H + k0 + kl] = tile[kl][n];
+    }
+}
+
+}  // namespace
+
+bool lstm_tc_eligible(int64_t T, int64_t B, int64_t H)
+{
+    if (T < 1 || B < 1 || B > 128 || H % 64 || H < 64 || H > 1024) return false;
+    int dev = 0, sms = 0, coop = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+    return coop && H / UNITS <= sms;
+}
+
+size_t lstm_tc_workspace(int64_t B, int64_t H)
+{
+    return align_up((size_t)H * 4 * H * 2, 1024) /* packed W_hh */ + align_up((size_t)2 * B * H * 2, 1024) /* exchange */ + 1024 /* counter */;
+}
+
+relay_status_t launch_lstm_tc(int64_t T, int64_t B, int64_t H, const float *zx, const void *w_hh, const float *h0, const float *c0,
+                              float *h_all, float *c_final, void *ws, cudaStream_t st)
+{
+    char *base = (char *)ws;
+    __nv_bfloat16 *wp = (__nv_bfloat16 *)base;
+    __nv_bfloat16 *hq = (__nv_bfloat16 *)(base + align_up((size_t)H * 4 * H * 2, 1024));
+    unsigned int *counter = (unsigned int *)((char *)hq + align_up((size_t)2 * B * H * 2, 1024));
+    const int n_blocks = (int)(H / UNITS);
+    pack_whh_kernel<<<dim3(n_blocks, (unsigned)(H / 64)), 256, 0, st>>>((const __nv_bfloat16 *)w_hh, wp, (int)H);
+    RELAY_TRY(check_launch("pack_whh"));
+    RELAY_CUDA(cudaMemsetAsync(counter, 0, 1024, st));
+    CUtensorMap tm_w;
+    RELAY_TRY(make_tmap_2d_bf16(&tm_w, wp, (uint64_t)H, (uint64_t)n_blocks * NCOL, (uint64_t)H, BK, NCOL));
+    Params p{};
+    p.T = (int)T; p.B = (int)B; p.H = (int)H; p.n_blocks = n_blocks; p.k_blocks = (int)(H / BK);
+    p.zx = zx; p.h0 = h0; p.c0 = c0; p.h_all = h_all; p.c_final = c_final; p.hq = hq; p.counter = counter;
+    p.err = device_error_word();
+    if (!p.err) return fail(RELAY_ERR_CUDA, "no device error word");
+    const size_t smem = 1024 + (size_t)p.k_blocks * W_KB + (size_t)STAGES * A_STAGE + 256;
+    RELAY_CUDA(cudaFuncSetAttribute(lstm_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    void *args[] = {(void *)&tm_w, (void *)&p};
+    RELAY_CUDA(cudaLaunchCooperativeKernel((const void *)lstm_persistent_kernel, dim3(n_blocks), dim3(NUM_THREADS), args, smem, st));
+    count_launch();
+    return RELAY_OK;
+}
+
+}  // namespace relay
