@@ -3,8 +3,8 @@
 // Block j owns 16 hidden units (64 gate columns: i, f, g, o of those units).  Its slice of W_hh
 // (64 columns x H, bf16) is loaded once by TMA and stays in shared memory for all T steps; the
 // running cell state of its units lives in registers.  Each step:
-//   loader warps copy bf16(h_{t-1}) [B x H] from the exchange buffer in L2 into a 4-stage shared
-//   memory ring (128-byte swizzle written by hand)  ->  one thread issues tcgen05.mma
+//   one thread streams bf16(h_{t-1}) [B x H] from the exchange buffer in L2 through a 4-stage shared
+//   memory ring by TMA (all k-blocks in flight at once)  ->  one thread issues tcgen05.mma
 //   (D[batch row, 64 gate columns] in TMEM)  ->  epilogue warps add the precomputed input projection,
 //   apply the gates, update c, write h_t (fp32 to h_all, bf16 to the exchange buffer)  ->  grid barrier.
 // The grid barrier is a counter in global memory with a bounded spin; the kernel is launched
@@ -23,11 +23,10 @@ relay_status_t make_tmap_2d_bf16(CUtensorMap *m, const void *base, uint64_t inne
 namespace {
 
 constexpr int UNITS = 16, NCOL = 4 * UNITS;      // hidden units and gate columns per block
-constexpr int BK = 64, STAGES = 4;
+constexpr int BK = 64, STAGES = 6;
 constexpr int A_STAGE = 128 * BK * 2;            // 128 batch rows (rows >= B stay zero) x 64 k
 constexpr int W_KB = NCOL * BK * 2;              // one k-block of the resident W slice
-constexpr int NUM_THREADS = 256;                 // warps 0-3 epilogue, warp 4 MMA, warps 5-7 loaders
-constexpr int N_LOADERS = 96;
+constexpr int NUM_THREADS = 192;                 // warps 0-3 epilogue, warp 4 MMA, warp 5 h loader
 
 struct Params {
     int T, B, H, n_blocks, k_blocks;
@@ -52,7 +51,9 @@ __device__ __forceinline__ void red_release_add(unsigned int *p, unsigned int v)
 __device__ __forceinline__ float fast_sigmoid(float x) { return __fdividef(1.0f, 1.0f + __expf(-x)); }
 __device__ __forceinline__ float fast_tanh(float x) { return 1.0f - __fdividef(2.0f, 1.0f + __expf(2.0f * x)); }
 
-__global__ void __launch_bounds__(NUM_THREADS, 1) lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const Params p)
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_h0,
+                       const __grid_constant__ CUtensorMap tm_h1, const Params p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -67,12 +68,14 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) lstm_persistent_kernel(const _
     const int j0 = blockIdx.x * UNITS;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], N_LOADERS); tc::mbar_init(&empty[s], 1); }
+        for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
         tc::mbar_init(w_full, 1);
         tc::mbar_init(tmem_full, 1);
         *abort_flag = 0;
         tc::fence_barrier_init();
         tc::prefetch_tmap(&tm_w);
+        tc::prefetch_tmap(&tm_h0);
+        tc::prefetch_tmap(&tm_h1);
     }
     // rows >= B of every ring stage are zero for the whole kernel
     for (int i = threadIdx.x; i < STAGES * A_STAGE / 16; i += NUM_THREADS) reinterpret_cast<uint4 *>(a_s)[i] = make_uint4(0, 0, 0, 0);
@@ -100,7 +103,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) lstm_persistent_kernel(const _
             dst[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
         }
         // every epilogue warp arrives on the grid barrier by itself (no block-level barrier that a
-        // warp which has given up could leave the others waiting on)
+        // warp which has given up could leave the others waiting on); the exchange buffer is read
+        // by TMA (async proxy), so the generic-proxy stores are fenced for it before the release
+        asm volatile("fence.proxy.async.global;" ::: "memory");
         __threadfence();
         __syncwarp();
         if (lane == 0) red_release_add(p.counter, 1u);
@@ -148,6 +153,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) lstm_persistent_kernel(const _
                 hq[0] = make_uint4(pack2(hn[0], hn[1]), pack2(hn[2], hn[3]), pack2(hn[4], hn[5]), pack2(hn[6], hn[7]));
                 hq[1] = make_uint4(pack2(hn[8], hn[9]), pack2(hn[10], hn[11]), pack2(hn[12], hn[13]), pack2(hn[14], hn[15]));
             }
+            asm volatile("fence.proxy.async.global;" ::: "memory");
             __threadfence();
             __syncwarp();
             if (lane == 0) red_release_add(p.counter, 1u);
@@ -180,40 +186,31 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) lstm_persistent_kernel(const _
             }
         }
     } else {
-        // ------------------------------ loaders: bf16(h_{t-1}) -> swizzled ring ------------------------------
-        const int lt = threadIdx.x - 160;                         // 0..95
-        const int chunks_per_kb = p.B * 8;                        // 16-byte chunks of one k-block (B rows x 128 B)
-        uint32_t it = 0;
-        bool ok = true;
-        for (int t = 0; t < p.T && ok; ++t) {
-            // grid barrier: every block has published its part of h_{t-1}
-            if (lt == 0) {
+        // ------------------------------ h loader: bf16(h_{t-1}) -> ring, by TMA ------------------------------
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int t = 0; t < p.T && ok; ++t) {
+                // grid barrier: every block has published its part of h_{t-1}
                 const unsigned int target = 4u * (unsigned int)p.n_blocks * (unsigned int)(t + 1);   // 4 epilogue warps per block
                 const long long t0 = clock64();
                 unsigned spins = 0;
                 while (ld_acquire(p.counter) < target) {
                     if ((++spins & 255u) == 0 && (*abort_flag || clock64() - t0 > tc::kWaitLimitCycles)) {
                         if (!*abort_flag) { *abort_flag = 1; atomicCAS(p.err, 0, tc::ERR_WAIT_STEP); }
+                        ok = false;
                         break;
                     }
                 }
-            }
-            asm volatile("bar.sync 2, 96;" ::: "memory");
-            if (*abort_flag) break;
-            const __nv_bfloat16 *hsrc = p.hq + (size_t)(t & 1) * p.B * p.H;
-            for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
-                const int s = it % STAGES;
-                if (!tc::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
-                uint8_t *dst = a_s + (size_t)s * A_STAGE;
-                for (int ch = lt; ch < chunks_per_kb; ch += N_LOADERS) {
-                    const int row = ch >> 3, c16 = ch & 7;
-                    uint4 v;
-                    const void *src = hsrc + (size_t)row * p.H + kb * BK + c16 * 8;
-                    asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(src) : "memory");
-                    *reinterpret_cast<uint4 *>(dst + row * 128 + ((c16 ^ (row & 7)) << 4)) = v;
+                if (!ok) break;
+                asm volatile("fence.proxy.async.global;" ::: "memory");
+                const CUtensorMap *tm_h = (t & 1) ? &tm_h1 : &tm_h0;
+                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    if (!tc::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
+                    tc::mbar_expect_tx(&full[s], (uint32_t)(p.B * 128));
+                    tc::tma_load_2d(a_s + (size_t)s * A_STAGE, tm_h, &full[s], kb * BK, 0);   // rows 0..B-1; the rest stay zero
                 }
-                tc::fence_proxy_async();
-                tc::mbar_arrive(&full[s]);
             }
         }
     }
@@ -267,8 +264,10 @@ relay_status_t launch_lstm_tc(int64_t T, int64_t B, int64_t H, const float *zx, 
     pack_whh_kernel<<<dim3(n_blocks, (unsigned)(H / 64)), 256, 0, st>>>((const __nv_bfloat16 *)w_hh, wp, (int)H);
     RELAY_TRY(check_launch("pack_whh"));
     RELAY_CUDA(cudaMemsetAsync(counter, 0, 1024, st));
-    CUtensorMap tm_w;
+    CUtensorMap tm_w, tm_h0, tm_h1;
     RELAY_TRY(make_tmap_2d_bf16(&tm_w, wp, (uint64_t)H, (uint64_t)n_blocks * NCOL, (uint64_t)H, BK, NCOL));
+    RELAY_TRY(make_tmap_2d_bf16(&tm_h0, hq, (uint64_t)H, (uint64_t)B, (uint64_t)H, BK, (uint32_t)B));
+    RELAY_TRY(make_tmap_2d_bf16(&tm_h1, hq + (size_t)B * H, (uint64_t)H, (uint64_t)B, (uint64_t)H, BK, (uint32_t)B));
     Params p{};
     p.T = (int)T; p.B = (int)B; p.H = (int)H; p.n_blocks = n_blocks; p.k_blocks = (int)(H / BK);
     p.zx = zx; p.h0 = h0; p.c0 = c0; p.h_all = h_all; p.c_final = c_final; p.hq = hq; p.counter = counter;
@@ -276,7 +275,7 @@ relay_status_t launch_lstm_tc(int64_t T, int64_t B, int64_t H, const float *zx, 
     if (!p.err) return fail(RELAY_ERR_CUDA, "no device error word");
     const size_t smem = 1024 + (size_t)p.k_blocks * W_KB + (size_t)STAGES * A_STAGE + 256;
     RELAY_CUDA(cudaFuncSetAttribute(lstm_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    void *args[] = {(void *)&tm_w, (void *)&p};
+    void *args[] = {(void *)&tm_w, (void *)&tm_h0, (void *)&tm_h1, (void *)&p};
     RELAY_CUDA(cudaLaunchCooperativeKernel((const void *)lstm_persistent_kernel, dim3(n_blocks), dim3(NUM_THREADS), args, smem, st));
     count_launch();
     return RELAY_OK;
