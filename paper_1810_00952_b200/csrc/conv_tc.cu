@@ -36,61 +36,71 @@ constexpr int TMEM_COLS = 512;
 // ---------------------------------------------------------------------------------------------------
 // layout kernels
 // ---------------------------------------------------------------------------------------------------
-// out[n][hw][c] = in[n][c][hw]  (GRAD: in = dy, multiplied by act'(y) on the way: dZ in NHWC)
+// out[n][hw][c] = in[n][c][hw]  (GRAD: in = dy, multiplied by act'(y) on the way: dZ in NHWC).
+// 64 channels x 64 pixels per block, 16-byte global accesses on both sides (HW % 8 == 0, C % 8 == 0).
 template <bool GRAD>
 __global__ void __launch_bounds__(256) nchw_to_nhwc_kernel(const __nv_bfloat16 *__restrict__ in, const __nv_bfloat16 *__restrict__ y,
                                                             __nv_bfloat16 *__restrict__ out, int C, int HW, int act)
 {
-    __shared__ __nv_bfloat16 tile[64][66];
+    __shared__ __align__(16) __nv_bfloat16 tile[64][72];   // [channel][pixel], rows 144 B apart
     const int n = blockIdx.z, c0 = blockIdx.y * 64, p0 = blockIdx.x * 64;
     const size_t img = (size_t)n * C * HW;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
+    for (int i = 0; i < 2; ++i) {
         const int idx = threadIdx.x + i * 256;
-        const int cl = idx >> 5, p2 = (idx & 31) * 2;
-        const int c = c0 + cl, p = p0 + p2;
-        float v0 = 0.0f, v1 = 0.0f;
-        if (c < C && p < HW) {   // HW is even, so p + 1 < HW as well
+        const int cl = idx >> 3, chunk = idx & 7;
+        const int c = c0 + cl, p = p0 + chunk * 8;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (c < C && p < HW) {
             const size_t off = img + (size_t)c * HW + p;
-            const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162 *>(in + off);
-            v0 = __low2float(a); v1 = __high2float(a);
+            v = ld_stream(in + off);
             if (GRAD) {
-                const __nv_bfloat162 yy = *reinterpret_cast<const __nv_bfloat162 *>(y + off);
-                v0 *= act_grad_from_output(__low2float(yy), act);
-                v1 *= act_grad_from_output(__high2float(yy), act);
+                const uint4 yy = ld_stream(y + off);
+                float a[8], b[8];
+                unpack(v, a);
+                unpack(yy, b);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) a[j] *= act_grad_from_output(b[j], act);
+                v = pack(a);
             }
         }
-        tile[cl][p2] = __float2bfloat16_rn(v0);
-        tile[cl][p2 + 1] = __float2bfloat16_rn(v1);
+        *reinterpret_cast<uint4 *>(&tile[cl][chunk * 8]) = v;
     }
     __syncthreads();
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
+    for (int i = 0; i < 2; ++i) {
         const int idx = threadIdx.x + i * 256;
-        const int pl = idx >> 5, c2 = (idx & 31) * 2;
-        const int c = c0 + c2, p = p0 + pl;
+        const int pl = idx & 63, cchunk = idx >> 6;          // a warp reads 32 consecutive pixels of one channel row
+        const int c = c0 + cchunk * 8, p = p0 + pl;
         if (c < C && p < HW) {
-            __nv_bfloat162 v;
-            v.x = tile[c2][pl]; v.y = tile[c2 + 1][pl];
-            *reinterpret_cast<__nv_bfloat162 *>(out + ((size_t)n * HW + p) * C + c) = v;
+            __align__(16) __nv_bfloat16 e[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) e[j] = tile[cchunk * 8 + j][pl];
+            *reinterpret_cast<uint4 *>(out + ((size_t)n * HW + p) * C + c) = *reinterpret_cast<const uint4 *>(e);
         }
     }
 }
 
-// wf[o][tap][c] = w[o][c][tap];   wb[c][mirror(tap)][o] = w[o][c][tap]   (either may be null)
+// wf[o][tap][c] = w[o][c][tap];   wb[c][mirror(tap)][o] = w[o][c][tap]   (either may be null); one thread
+// per OUTPUT element so that the stores coalesce (the 1 MB source stays in L2)
 __global__ void pack_weights_kernel(const __nv_bfloat16 *__restrict__ w, __nv_bfloat16 *__restrict__ wf,
                                     __nv_bfloat16 *__restrict__ wb, int O, int C, int R, int S)
 {
-    const int64_t total = (int64_t)O * C * R * S;
+    const int taps = R * S;
+    const int64_t total = (int64_t)O * C * taps;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-        const int s = (int)(i % S);
-        int64_t t = i / S;
-        const int r = (int)(t % R); t /= R;
-        const int c = (int)(t % C);
-        const int o = (int)(t / C);
-        const __nv_bfloat16 v = w[i];
-        if (wf) wf[((int64_t)o * (R * S) + r * S + s) * C + c] = v;
-        if (wb) wb[((int64_t)c * (R * S) + (R - 1 - r) * S + (S - 1 - s)) * O + o] = v;
+        if (wf) {
+            const int c = (int)(i % C);
+            const int tap = (int)((i / C) % taps);
+            const int o = (int)(i / ((int64_t)C * taps));
+            wf[i] = w[((int64_t)o * C + c) * taps + tap];
+        }
+        if (wb) {
+            const int o = (int)(i % O);
+            const int tap2 = (int)((i / O) % taps);
+            const int c = (int)(i / ((int64_t)O * taps));
+            wb[i] = w[((int64_t)o * C + c) * taps + (taps - 1 - tap2)];
+        }
     }
 }
 
@@ -487,7 +497,7 @@ relay_status_t launch_conv_fwd_tc(const ConvDims &d, const void *x, const void *
     char *base = (char *)ws;
     void *x_nhwc = base, *wf = base + pl.x_nhwc;
     RELAY_TRY(launch_transpose(false, x, nullptr, x_nhwc, d.Nb, d.C, d.H * d.W, 0, st));
-    pack_weights_kernel<<<256, 256, 0, st>>>((const __nv_bfloat16 *)w, (__nv_bfloat16 *)wf, nullptr, (int)d.O, (int)d.C, 3, 3);
+    pack_weights_kernel<<<(unsigned)((d.O * d.C * 9 + 255) / 256), 256, 0, st>>>((const __nv_bfloat16 *)w, (__nv_bfloat16 *)wf, nullptr, (int)d.O, (int)d.C, 3, 3);
     RELAY_TRY(check_launch("pack_weights"));
     return launch_fprop(d, pl, x_nhwc, (int)d.C, wf, (int)d.O, b, b_dt, act, y, st);
 }
@@ -508,7 +518,7 @@ relay_status_t launch_conv_grad_tc(const ConvDims &d, const void *x, const void 
     RELAY_TRY(launch_transpose(false, x, nullptr, x_nhwc, d.Nb, d.C, HW, 0, st));
     if (db) RELAY_TRY(launch_colsum_bf16(dz_nhwc, d.Nb * HW, d.O, db_part, db, st));
     if (dx) {
-        pack_weights_kernel<<<256, 256, 0, st>>>((const __nv_bfloat16 *)w, nullptr, (__nv_bfloat16 *)wb, (int)d.O, (int)d.C, 3, 3);
+        pack_weights_kernel<<<(unsigned)((d.O * d.C * 9 + 255) / 256), 256, 0, st>>>((const __nv_bfloat16 *)w, nullptr, (__nv_bfloat16 *)wb, (int)d.O, (int)d.C, 3, 3);
         RELAY_TRY(check_launch("pack_weights"));
         RELAY_TRY(launch_fprop(d, pl, dz_nhwc, (int)d.O, wb, (int)d.C, nullptr, RELAY_F32, RELAY_ACT_NONE, dx, st));
     }

@@ -126,15 +126,28 @@ __global__ void __launch_bounds__(kTX *kTY, Body::NIN >= 4 ? 2 : 3) ewise2d_kern
     }
 }
 
-// second pass of a column sum: adds the per-slice partials in slice order
-__global__ void colsum_finalize_kernel(const float *__restrict__ partial, int n_slices, int64_t cols, float scale,
-                                       float *__restrict__ out)
+// second pass of a column sum: thread (tx, ty) adds the partials of slices ty, ty+8, ... of its column in
+// slice order, then the 8 row-threads are combined in ty order (fixed order, so reruns are bit-identical).
+// grid.y indexes the summed result k: partials at partial + k * n_slices * cols, output out[k].
+struct FinalizeOuts { float *out[RELAY_MAX_OUTPUTS]; };
+__global__ void __launch_bounds__(256) colsum_finalize_kernel(const float *__restrict__ partial, int n_slices, int64_t cols, float scale,
+                                                               const FinalizeOuts outs)
 {
-    int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (c >= cols) return;
+    __shared__ float sm[8][33];
+    const int tx = threadIdx.x, ty = threadIdx.y;
+    const int64_t c = (int64_t)blockIdx.x * 32 + tx;
+    const float *p = partial + (size_t)blockIdx.y * n_slices * cols;
     float s = 0.0f;
-    for (int j = 0; j < n_slices; ++j) s += partial[(int64_t)j * cols + c];
-    out[c] = s * scale;
+    if (c < cols)
+        for (int j = ty; j < n_slices; j += 8) s += p[(int64_t)j * cols + c];
+    sm[ty][tx] = s;
+    __syncthreads();
+    if (ty == 0 && c < cols) {
+        float t = 0.0f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) t += sm[j][tx];
+        outs.out[blockIdx.y][c] = t * scale;
+    }
 }
 
 // reduction over the last axis of a [rows, cols] tensor: one warp per row, 128-bit loads
@@ -427,11 +440,20 @@ relay_status_t launch_body2d(int32_t storage, const Args2D<Body::NIN, Body::NOUT
     return check_launch(what);
 }
 
+// finalises n_out column sums whose partials lie one after another ([k][n_slices][cols])
+relay_status_t launch_colsum_finalize_n(const float *partial, int n_slices, int64_t cols, float scale, float *const *out, int n_out,
+                                        cudaStream_t st)
+{
+    FinalizeOuts fo{};
+    for (int k = 0; k < n_out; ++k) fo.out[k] = out[k];
+    colsum_finalize_kernel<<<dim3((unsigned)((cols + 31) / 32), (unsigned)n_out), dim3(32, 8), 0, st>>>(partial, n_slices, cols, scale, fo);
+    return check_launch("colsum_finalize");
+}
+
 relay_status_t launch_colsum_finalize(const float *partial, int n_slices, int64_t cols, float scale, float *out,
                                       cudaStream_t st)
 {
-    colsum_finalize_kernel<<<(unsigned)((cols + 255) / 256), 256, 0, st>>>(partial, n_slices, cols, scale, out);
-    return check_launch("colsum_finalize");
+    return launch_colsum_finalize_n(partial, n_slices, cols, scale, &out, 1, st);
 }
 
 // dZ = dy (.) act'(y) stored to dz, and (if db) db = column sums of dZ; used by the dense gradient group
@@ -639,9 +661,8 @@ extern "C" relay_status_t relay_fused_reduce(const relay_ewise_prog_t *prog, con
         A.partial[0] = nullptr; A.partial[1] = part; A.partial[2] = part + (size_t)pl.n_slices * v.cols;
         A.rows = v.rows; A.cols = v.cols; A.aux = 0;
         RELAY_TRY(launch_body2d<BodyTanhAffineResidualGrad>(v.storage, A, pl.n_slices, st, "ewise2d<tanh_affine_residual_grad>"));
-        RELAY_TRY(launch_colsum_finalize(A.partial[1], pl.n_slices, v.cols, 1.0f, (float *)outputs[1]->data, st));
-        RELAY_TRY(launch_colsum_finalize(A.partial[2], pl.n_slices, v.cols, 1.0f, (float *)outputs[2]->data, st));
-        return RELAY_OK;
+        float *sums[2] = {(float *)outputs[1]->data, (float *)outputs[2]->data};
+        return launch_colsum_finalize_n(A.partial[1], pl.n_slices, v.cols, 1.0f, sums, 2, st);
     }
     if (pl.fast_colsum) {
         Args2D<1, 1> A{};
