@@ -61,7 +61,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE, text=True)
+                                          "--format=csv,noheader,nounits", "-lms", "20"], stdout=subprocess.PIPE, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except Exception:
@@ -273,7 +273,7 @@ class Workload:
 # ---------------------------------------------------------------------------------------------------
 # CPU oracle on a bounded sample (single thread); also the `--impl reference` arm
 # ---------------------------------------------------------------------------------------------------
-def oracle_sample(rows3=48, rows2=192):
+def oracle_sample(rows3=192, rows2=1024):
     """Times the fp64 oracle, as it stands, on slices of the same workload along the independent
     dimension.  Returns (tflops, gbs, seconds, description)."""
     import oracle
@@ -320,7 +320,7 @@ def run_reference(args, rank, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--groups", default=",".join(ALL_GROUPS))
