@@ -2,9 +2,14 @@
 //   TMA tile loads (128-byte swizzle) -> 4-stage shared-memory ring -> tcgen05.mma issued by one
 //   thread into a double-buffered TMEM accumulator -> epilogue warps read TMEM (tcgen05.ld), add the
 //   bias, apply the activation, round once and store.
-// One persistent block per SM walks the 128 x 256 output tiles.  Roles: warp 0 = TMA producer,
-// warp 1 = TMEM owner + MMA issuer, warps 2..5 = epilogue (one TMEM lane quarter each), so the
-// epilogue of tile i overlaps the main loop of tile i+1.
+// One persistent block per SM walks the output tiles.  Roles: warp 0 = TMA producer, warp 1 = TMEM
+// owner + MMA issuer, the remaining warps = epilogue (one TMEM lane quarter each).
+// Two tile shapes (template parameter MH = number of 128-row halves):
+//   MH = 1: 128 x 256 tiles, 4 stages, the two 256-column TMEM accumulators alternate between tiles so
+//           that the epilogue of tile i overlaps the main loop of tile i+1;
+//   MH = 2: 256 x 256 tiles (two MMAs per k-step share the B tile in shared memory, which cuts the
+//           bytes fetched per FLOP by a third), 3 stages, one accumulator per half, each half drained
+//           by its own four epilogue warps and released separately.
 //
 // Operands are described by strides (gemm.h): an operand whose contraction index is contiguous is
 // "K-major", one whose M/N index is contiguous is "MN-major"; both are fed to the MMA unit as they
@@ -20,12 +25,21 @@ namespace relay {
 
 namespace {
 
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
-constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int BN = 256, BK = 64;
+constexpr int B_BYTES = BN * BK * 2;
 constexpr int MN_BOX_BYTES = 64 * BK * 2;   // one TMA box of an MN-major operand: 64 (M/N) x 64 (k)
 constexpr int TMEM_COLS = 512;              // two accumulators of 256 fp32 columns
-constexpr int NUM_THREADS = 192;
-constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_BYTES + 256;
+
+template <int MH> struct Cfg {
+    static constexpr int BM = 128 * MH;
+    static constexpr int STAGES = MH == 1 ? 4 : 3;
+    static constexpr int A_BYTES = BM * BK * 2;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int NUM_THREADS = 64 + 128 * MH;
+    static constexpr int STORE_BUFS = MH == 1 ? 2 : 1;                 // 4 KB staging buffers per epilogue warp
+    static constexpr int STAGING_BYTES = 4 * MH * STORE_BUFS * 4096;
+    static constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_BYTES + STAGING_BYTES + 256;
+};
 
 struct Params {
     int M, N, K;
@@ -37,13 +51,72 @@ struct Params {
     int *err;
 };
 
-template <bool A_MN, bool B_MN>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const Params p)
+// One warp drains its 32 accumulator rows (256 columns): TMEM -> registers -> bias + activation ->
+// rounding -> swizzled staging buffer -> TMA tile store of 32 rows x 128 bytes at a time.
+template <bool OUT_F32, int BUFS>
+__device__ __forceinline__ void epilogue_rows(const Params &p, const CUtensorMap *tm_c, uint32_t taddr, uint8_t *stage, int lane,
+                                              int row0, int n0)
 {
+    constexpr int COLS = OUT_F32 ? 32 : 64;             // columns per 128-byte block
+#pragma unroll 1
+    for (int blk = 0; blk < BN / COLS; ++blk) {
+        const int nc = n0 + blk * COLS;
+        if (nc >= p.N) break;                            // warp-uniform
+        uint4 piece[8];
+#pragma unroll
+        for (int sub = 0; sub < COLS / 32; ++sub) {
+            uint32_t r[32];
+            tc::tmem_ld_32x32(taddr + blk * COLS + sub * 32, r);
+            tc::tmem_ld_wait();
+            const int c0 = nc + sub * 32;
+            // lane j fetches the bias of column c0 + j; every lane then reads all 32 by shuffle
+            float bias_lane = 0.0f;
+            if (p.bias != nullptr && c0 + lane < p.N)
+                bias_lane = p.bias_bf16 ? __bfloat162float(((const __nv_bfloat16 *)p.bias)[c0 + lane]) : ((const float *)p.bias)[c0 + lane];
+            float v[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) + __shfl_sync(0xffffffffu, bias_lane, j);
+            switch (p.act) {                             // hoisted out of the element loop
+            case RELAY_ACT_RELU:
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.0f);
+                break;
+            case RELAY_ACT_TANH:
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = OUT_F32 ? tanh_<false>(v[j]) : tanh_<true>(v[j]);
+                break;
+            case RELAY_ACT_SIGMOID:
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = OUT_F32 ? sigmoid_<false>(v[j]) : sigmoid_<true>(v[j]);
+                break;
+            default: break;
+            }
+            if (OUT_F32) {
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    piece[c] = make_uint4(__float_as_uint(v[4 * c]), __float_as_uint(v[4 * c + 1]), __float_as_uint(v[4 * c + 2]),
+                                          __float_as_uint(v[4 * c + 3]));
+            } else {
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    piece[sub * 4 + c] = make_uint4(pack2(v[8 * c], v[8 * c + 1]), pack2(v[8 * c + 2], v[8 * c + 3]),
+                                                    pack2(v[8 * c + 4], v[8 * c + 5]), pack2(v[8 * c + 6], v[8 * c + 7]));
+            }
+        }
+        tc::warp_store_block<BUFS - 1>(tm_c, stage + (blk % BUFS) * 4096, piece, lane, nc, row0);
+    }
+}
+
+template <bool A_MN, bool B_MN, int MH>
+__global__ void __launch_bounds__(Cfg<MH>::NUM_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+               const __grid_constant__ CUtensorMap tm_c, const Params p)
+{
+    constexpr int BM = Cfg<MH>::BM, STAGES = Cfg<MH>::STAGES, A_BYTES = Cfg<MH>::A_BYTES, STAGE_BYTES = Cfg<MH>::STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + (size_t)STAGES * STAGE_BYTES);
+    uint8_t *staging = smem + (size_t)STAGES * STAGE_BYTES;            // [epilogue warp][STORE_BUFS][4 KB]
+    uint64_t *bars = reinterpret_cast<uint64_t *>(staging + Cfg<MH>::STAGING_BYTES);
     uint64_t *full = bars, *empty = bars + STAGES, *tmem_full = bars + 2 * STAGES, *tmem_empty = bars + 2 * STAGES + 2;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 4);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
@@ -58,6 +131,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         tc::fence_barrier_init();
         tc::prefetch_tmap(&tm_a);
         tc::prefetch_tmap(&tm_b);
+        tc::prefetch_tmap(&tm_c);
     }
     if (warp == 1) {
         tc::tmem_alloc(tmem_slot, TMEM_COLS);
@@ -85,7 +159,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 #pragma unroll
                         for (int i = 0; i < BM / 64; ++i) tc::tma_load_2d(sa + i * MN_BOX_BYTES, &tm_a, &full[s], m0 + i * 64, k0);
                     } else {
-                        tc::tma_load_2d(sa, &tm_a, &full[s], k0, m0);
+                        tc::tma_load_2d(sa, &tm_a, &full[s], k0, m0);     // one box of BM rows
                     }
                     if (B_MN) {
 #pragma unroll
@@ -99,7 +173,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            constexpr uint32_t idesc = tc::instr_desc_bf16(BM, BN, A_MN, B_MN);
+            constexpr uint32_t idesc = tc::instr_desc_bf16(128, BN, A_MN, B_MN);
             // K-major: 8-row atoms 1024 B apart, one MMA (16 k) = 32 bytes along the swizzled row;
             // MN-major: 64-wide M/N groups one TMA box apart, 8-k atoms 1024 B apart, one MMA = 2 atoms.
             constexpr uint32_t a_lbo = A_MN ? MN_BOX_BYTES : 16, b_lbo = B_MN ? MN_BOX_BYTES : 16;
@@ -107,8 +181,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             uint32_t it = 0, t_local = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++t_local) {
-                const int buf = t_local & 1;
-                if (!tc::mbar_wait(&tmem_empty[buf], ((t_local >> 1) & 1) ^ 1, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) break;
+                // MH = 1: accumulator t_local & 1;  MH = 2: accumulator h for half h, both used by every tile
+                const int buf = MH == 1 ? (t_local & 1) : 0;
+                const uint32_t empty_parity = MH == 1 ? (((t_local >> 1) & 1) ^ 1) : ((t_local & 1) ^ 1);
+                if (!tc::mbar_wait(&tmem_empty[buf], empty_parity, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) break;
                 tc::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * BN;
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
@@ -118,63 +194,46 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     const uint32_t sa = tc::smem_u32(smem + (size_t)s * STAGE_BYTES), sb = sa + A_BYTES;
 #pragma unroll
                     for (int kk = 0; kk < BK / 16; ++kk) {
-                        const uint64_t da = tc::smem_desc(sa + kk * a_step, a_lbo, 1024);
                         const uint64_t db = tc::smem_desc(sb + kk * b_step, b_lbo, 1024);
-                        tc::mma_bf16(d_tmem, da, db, idesc, (kb | kk) != 0);
+#pragma unroll
+                        for (int h = 0; h < MH; ++h) {
+                            if (MH == 2 && h == 1 && kb == 0 && kk == 0) {   // the second half may still be draining
+                                if (!tc::mbar_wait(&tmem_empty[1], empty_parity, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) { ok = false; break; }
+                                tc::tc_fence_after_sync();
+                            }
+                            const uint64_t da = tc::smem_desc(sa + h * (128 * BK * 2) + kk * a_step, a_lbo, 1024);
+                            tc::mma_bf16(d_tmem + h * BN, da, db, idesc, (kb | kk) != 0);
+                        }
+                        if (!ok) break;
                     }
+                    if (!ok) break;
                     tc::mma_commit(&empty[s]);          // the stage is free once these MMAs have read it
                 }
-                if (ok) tc::mma_commit(&tmem_full[buf]);  // the accumulator is complete
+                if (ok) tc::mma_commit(&tmem_full[buf]);  // the accumulator(s) are complete
             }
         }
     } else {
-        // ---------------- epilogue (4 warps, 128 threads) ----------------
+        // ---------------- epilogue (4 warps per 128-row half) ----------------
         const int quarter = warp & 3;                     // TMEM lanes [32*quarter, 32*quarter+32)
+        const int half = (warp - 2) >> 2;                 // which 128-row half this warp drains (MH = 2)
         uint32_t t_local = 0;
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++t_local) {
-            const int buf = t_local & 1;
-            const int m0 = (tile % p.tiles_m) * BM, n0 = (tile / p.tiles_m) * BN;
+            const int buf = MH == 1 ? (t_local & 1) : half;          // accumulator to read
+            const int fbar = MH == 1 ? (t_local & 1) : 0;            // barrier that announces it
+            const uint32_t full_parity = MH == 1 ? ((t_local >> 1) & 1) : (t_local & 1);
+            const int m0 = (tile % p.tiles_m) * BM + half * 128, n0 = (tile / p.tiles_m) * BN;
             // one lane polls, the warp follows its verdict (keeps the warp converged for tcgen05.ld)
             int ok = 1;
-            if (lane == 0) ok = tc::mbar_wait(&tmem_full[buf], (t_local >> 1) & 1, abort_flag, p.err, tc::ERR_WAIT_TMEM_FULL) ? 1 : 0;
+            if (lane == 0) ok = tc::mbar_wait(&tmem_full[fbar], full_parity, abort_flag, p.err, tc::ERR_WAIT_TMEM_FULL) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
             tc::tc_fence_after_sync();
-            const int row = m0 + quarter * 32 + lane;
+            const int row0 = m0 + quarter * 32;                 // this warp's 32 rows; lane = row within them
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * BN;
-#pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t r[32];
-                tc::tmem_ld_32x32(taddr + c * 32, r);
-                tc::tmem_ld_wait();
-                const int nc = n0 + c * 32;
-                // lane j fetches the bias of column nc + j; every lane then reads all 32 by shuffle
-                float bias_lane = 0.0f;
-                if (p.bias != nullptr && nc + lane < p.N)
-                    bias_lane = p.bias_bf16 ? __bfloat162float(((const __nv_bfloat16 *)p.bias)[nc + lane]) : ((const float *)p.bias)[nc + lane];
-                float v[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) + __shfl_sync(0xffffffffu, bias_lane, j);
-                if (row < p.M && nc < p.N) {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const float z = v[j];
-                        v[j] = p.out_f32 ? act_fwd<false>(z, p.act) : act_fwd<true>(z, p.act);
-                    }
-                    if (p.out_f32) {
-                        float *dst = (float *)p.c + (long long)row * p.ldc + nc;
-#pragma unroll
-                        for (int j = 0; j < 32; j += 4)
-                            if (nc + j < p.N) *reinterpret_cast<float4 *>(dst + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                    } else {
-                        __nv_bfloat16 *dst = (__nv_bfloat16 *)p.c + (long long)row * p.ldc + nc;
-#pragma unroll
-                        for (int j = 0; j < 32; j += 8)
-                            if (nc + j < p.N)
-                                *reinterpret_cast<uint4 *>(dst + j) = make_uint4(pack2(v[j], v[j + 1]), pack2(v[j + 2], v[j + 3]),
-                                                                                 pack2(v[j + 4], v[j + 5]), pack2(v[j + 6], v[j + 7]));
-                    }
-                }
+            uint8_t *my_stage = staging + (size_t)(warp - 2) * Cfg<MH>::STORE_BUFS * 4096;
+            if (row0 < p.M) {
+                if (p.out_f32) epilogue_rows<true, Cfg<MH>::STORE_BUFS>(p, &tm_c, taddr, my_stage, lane, row0, n0);
+                else epilogue_rows<false, Cfg<MH>::STORE_BUFS>(p, &tm_c, taddr, my_stage, lane, row0, n0);
             }
             tc::tc_fence_before_sync();
             __syncwarp();
@@ -182,6 +241,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         }
     }
 
+    if (warp >= 2 && lane == 0) tc::tma_store_wait_all<0>();   // this lane's tile stores have landed
     tc::tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {
@@ -210,22 +270,28 @@ EncodeTiledFn encode_fn()
 
 }  // namespace
 
-// 2-D bf16 tensor map: `inner` contiguous elements per row, `outer` rows `row_stride` elements apart,
-// box = box_inner x box_outer, 128-byte swizzle, out-of-range elements read as zero
-relay_status_t make_tmap_2d_bf16(CUtensorMap *m, const void *base, uint64_t inner, uint64_t outer, uint64_t row_stride,
-                                 uint32_t box_inner, uint32_t box_outer)
+// 2-D tensor map (bf16 or f32): `inner` contiguous elements per row, `outer` rows `row_stride` elements
+// apart, box = box_inner x box_outer, 128-byte swizzle, out-of-range elements read as zero / not written
+relay_status_t make_tmap_2d(CUtensorMap *m, bool f32, const void *base, uint64_t inner, uint64_t outer, uint64_t row_stride,
+                            uint32_t box_inner, uint32_t box_outer)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return fail(RELAY_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
     cuuint64_t dims[2] = {inner, outer};
-    cuuint64_t strides[1] = {row_stride * 2};
+    cuuint64_t strides[1] = {row_stride * (f32 ? 4 : 2)};
     cuuint32_t box[2] = {box_inner, box_outer};
     cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+    CUresult r = fn(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(RELAY_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
     return RELAY_OK;
+}
+
+relay_status_t make_tmap_2d_bf16(CUtensorMap *m, const void *base, uint64_t inner, uint64_t outer, uint64_t row_stride,
+                                 uint32_t box_inner, uint32_t box_outer)
+{
+    return make_tmap_2d(m, false, base, inner, outer, row_stride, box_inner, box_outer);
 }
 
 bool gemm_tc_eligible(const GemmDesc &g)
@@ -244,31 +310,47 @@ bool gemm_tc_eligible(const GemmDesc &g)
 relay_status_t launch_gemm_tc(const GemmDesc &g, cudaStream_t st)
 {
     const bool a_mn = g.a_sk != 1, b_mn = g.b_sk != 1;
+    // 256 x 256 tiles fetch a third fewer bytes per FLOP but their epilogue is not overlapped; take them
+    // when they do not cost an extra round of tiles over the SMs
+    int dev = 0, sms = 148;
+    RELAY_CUDA(cudaGetDevice(&dev));
+    RELAY_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const int64_t t1 = ((g.M + 127) / 128) * ((g.N + BN - 1) / BN), t2 = ((g.M + 255) / 256) * ((g.N + BN - 1) / BN);
+    const double cost1 = (double)((t1 + sms - 1) / sms), cost2 = 1.85 * (double)((t2 + sms - 1) / sms);
+    const int mh = (g.M >= 256 && cost2 < cost1) ? 2 : 1;
+    const int bm = 128 * mh;
     CUtensorMap tm_a, tm_b;
     if (a_mn) RELAY_TRY(make_tmap_2d_bf16(&tm_a, g.a, g.M, g.K, g.a_sk, 64, BK));       // rows = k, inner = m
-    else RELAY_TRY(make_tmap_2d_bf16(&tm_a, g.a, g.K, g.M, g.a_sm, BK, BM));             // rows = m, inner = k
+    else RELAY_TRY(make_tmap_2d_bf16(&tm_a, g.a, g.K, g.M, g.a_sm, BK, bm));             // rows = m, inner = k
     if (b_mn) RELAY_TRY(make_tmap_2d_bf16(&tm_b, g.b, g.N, g.K, g.b_sk, 64, BK));       // rows = k, inner = n
     else RELAY_TRY(make_tmap_2d_bf16(&tm_b, g.b, g.K, g.N, g.b_sn, BK, BN));             // rows = n, inner = k
     Params p{};
     p.M = (int)g.M; p.N = (int)g.N; p.K = (int)g.K;
     p.c = g.c; p.ldc = g.ldc;
     p.bias = g.bias; p.bias_bf16 = g.bias_dtype == RELAY_BF16; p.act = g.act; p.out_f32 = g.out_dtype == RELAY_F32;
-    p.tiles_m = (int)((g.M + BM - 1) / BM); p.tiles_n = (int)((g.N + BN - 1) / BN); p.k_blocks = (int)((g.K + BK - 1) / BK);
+    p.tiles_m = (int)((g.M + bm - 1) / bm); p.tiles_n = (int)((g.N + BN - 1) / BN); p.k_blocks = (int)((g.K + BK - 1) / BK);
     p.err = device_error_word();
     if (!p.err) return fail(RELAY_ERR_CUDA, "no device error word");
-    int dev = 0, sms = 148;
-    RELAY_CUDA(cudaGetDevice(&dev));
-    RELAY_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    CUtensorMap tm_c;
+    const bool f32 = g.out_dtype == RELAY_F32;
+    RELAY_TRY(make_tmap_2d(&tm_c, f32, g.c, g.N, g.M, g.ldc, f32 ? 32 : 64, 32));
     const int grid = std::min(p.tiles_m * p.tiles_n, sms);
-#define LAUNCH(AMN, BMN)                                                                                          \
-    do {                                                                                                          \
-        RELAY_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<AMN, BMN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES)); \
-        gemm_tc_kernel<AMN, BMN><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tm_a, tm_b, p);                           \
+#define LAUNCH(AMN, BMN, MHV)                                                                                             \
+    do {                                                                                                                  \
+        RELAY_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<AMN, BMN, MHV>, cudaFuncAttributeMaxDynamicSharedMemorySize,       \
+                                        (int)Cfg<MHV>::SMEM_BYTES));                                                      \
+        gemm_tc_kernel<AMN, BMN, MHV><<<grid, Cfg<MHV>::NUM_THREADS, Cfg<MHV>::SMEM_BYTES, st>>>(tm_a, tm_b, tm_c, p);          \
     } while (0)
-    if (a_mn && b_mn) LAUNCH(true, true);
-    else if (a_mn) LAUNCH(true, false);
-    else if (b_mn) LAUNCH(false, true);
-    else LAUNCH(false, false);
+#define LAUNCH_MH(AMN, BMN)          \
+    do {                             \
+        if (mh == 2) LAUNCH(AMN, BMN, 2); \
+        else LAUNCH(AMN, BMN, 1);    \
+    } while (0)
+    if (a_mn && b_mn) LAUNCH_MH(true, true);
+    else if (a_mn) LAUNCH_MH(true, false);
+    else if (b_mn) LAUNCH_MH(false, true);
+    else LAUNCH_MH(false, false);
+#undef LAUNCH_MH
 #undef LAUNCH
     return check_launch("gemm_tc");
 }

@@ -92,6 +92,38 @@ __device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *m, uin
                  : "memory");
 }
 
+// 2-D tile store from shared memory (tracked as a bulk async-group of the issuing thread); elements
+// outside the tensor are not written, so ragged tile edges need no guard
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *m, const void *src, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(src)), "r"(x), "r"(y)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// waits until at most N of this thread's store groups still READ their shared-memory source
+template <int N> __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+template <int N> __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory"); }
+
+// One warp hands a 32-row x 128-byte block (lane = row, eight 16-byte pieces per lane) to a TMA tile
+// store: pieces go to a 4 KB staging buffer in the 128-byte swizzle pattern (conflict-free), then one
+// lane issues the store of the whole block at tensor coordinates (x, y).  `reuse_wait` is the number of
+// younger store groups that may still be reading OTHER staging buffers when this one is refilled.
+template <int OTHER_BUFFERS_IN_FLIGHT>
+__device__ __forceinline__ void warp_store_block(const CUtensorMap *m, uint8_t *stage, const uint4 (&piece)[8], int lane, int x, int y)
+{
+    if (lane == 0) tma_store_wait_read<OTHER_BUFFERS_IN_FLIGHT>();
+    __syncwarp();
+#pragma unroll
+    for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4 *>(stage + lane * 128 + ((c ^ (lane & 7)) << 4)) = piece[c];
+    fence_proxy_async();
+    __syncwarp();
+    if (lane == 0) {
+        tma_store_2d(m, stage, x, y);
+        tma_store_commit();
+    }
+}
+
 // ---- tcgen05 ----------------------------------------------------------------------------------------
 __device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t cols)
 {
