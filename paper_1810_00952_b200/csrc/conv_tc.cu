@@ -26,6 +26,8 @@ relay_status_t make_tmap_2d_bf16(CUtensorMap *m, const void *base, uint64_t inne
                                  uint32_t box_inner, uint32_t box_outer);
 relay_status_t make_tmap_nhwc_bf16(CUtensorMap *m, const void *base, uint64_t C, uint64_t W, uint64_t H, uint64_t N,
                                    uint32_t box_c, uint32_t box_w, uint32_t box_h);
+relay_status_t make_tmap_2d(CUtensorMap *m, bool f32, const void *base, uint64_t inner, uint64_t outer, uint64_t row_stride,
+                            uint32_t box_inner, uint32_t box_outer, bool swizzle128);
 
 namespace {
 
@@ -120,32 +122,67 @@ __global__ void wgrad_reduce_kernel(const float *__restrict__ part, int n_slices
 }
 
 // ---------------------------------------------------------------------------------------------------
-// fprop kernel: 128 output channels x (rows_per_tile * W) pixels per tile
+// fprop kernel.  Work items are output tiles of (rows_per_tile * W) pixels by 128 * mh output channels:
+//   MH = 1: every item is 128 channels wide; the two TMEM accumulators alternate between items, so the
+//           epilogue of one item overlaps the main loop of the next;
+//   MH = 2: "pairs" (256 channels: two MMAs per k-step share the activation tile in shared memory, a third
+//           fewer bytes per FLOP) fill whole rounds over the SMs, and what is left runs as single
+//           128-channel items so that the last round is half as long.  One accumulator per half, each
+//           drained by its own four epilogue warps.
+// The epilogue goes through a staging buffer and TMA tile stores into the NCHW output viewed as a 2-D
+// tensor [Nb * Cout rows][H * W columns] (the pixels of consecutive image rows are contiguous there).
 // ---------------------------------------------------------------------------------------------------
 struct FpropParams {
     int Cin, Cout, H, W, Nb, taps_r, taps_s, pad;
     int rows_per_tile, nt;      // nt = rows_per_tile * W = UMMA N
-    int m_tiles, tiles_per_img, n_tiles_total, k_blocks, stages;
-    __nv_bfloat16 *out;         // NCHW [Nb][Cout][H][W]
+    int tiles_per_img, n_tiles_total, k_blocks, stages;
+    int n_pairs, pairs_per_ntile, n_items;   // items [0, n_pairs) are pairs, the rest singles (MH = 2); MH = 1: all singles
     const void *bias;           // per output channel, or null
     int bias_bf16, act;
     int *err;
 };
 
-__global__ void __launch_bounds__(NUM_THREADS, 1)
-conv_fprop_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, const FpropParams p)
+struct FpropItem { int m0, mh, img, h0; };
+
+template <int MH>
+__device__ __forceinline__ FpropItem fprop_item(const FpropParams &p, int item)
+{
+    FpropItem it;
+    int nt_idx;
+    if (MH == 2 && item < p.n_pairs) {
+        it.mh = 2;
+        it.m0 = (item % p.pairs_per_ntile) * 256;
+        nt_idx = item / p.pairs_per_ntile;
+    } else {
+        const int singles_per_ntile = p.Cout / BM;
+        const int j = item - (MH == 2 ? p.n_pairs : 0);
+        const int base = MH == 2 ? p.n_pairs / p.pairs_per_ntile : 0;
+        it.mh = 1;
+        it.m0 = (j % singles_per_ntile) * BM;
+        nt_idx = base + j / singles_per_ntile;
+    }
+    it.img = nt_idx / p.tiles_per_img;
+    it.h0 = (nt_idx % p.tiles_per_img) * p.rows_per_tile;
+    return it;
+}
+
+template <int MH>
+__global__ void __launch_bounds__(64 + 128 * MH, 1)
+conv_fprop_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
+                     const __grid_constant__ CUtensorMap tm_y, const FpropParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const int a_bytes = BM * BK * 2, b_bytes = p.nt * BK * 2;
+    constexpr int a_bytes = MH * BM * BK * 2;
+    const int b_bytes = p.nt * BK * 2;
     const int stage_bytes = a_bytes + ((b_bytes + 1023) & ~1023);
     const int STAGES = p.stages;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + (size_t)STAGES * stage_bytes);
+    uint8_t *staging = smem + (size_t)STAGES * stage_bytes;                 // [epilogue warp][2][2 KB]
+    uint64_t *bars = reinterpret_cast<uint64_t *>(staging + 4 * MH * 4096);
     uint64_t *full = bars, *empty = bars + STAGES, *tmem_full = bars + 2 * STAGES, *tmem_empty = bars + 2 * STAGES + 2;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 4);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_tiles = p.m_tiles * p.n_tiles_total;
     const int cblocks = p.Cin / BK;
 
     if (threadIdx.x == 0) {
@@ -155,6 +192,7 @@ conv_fprop_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
         tc::fence_barrier_init();
         tc::prefetch_tmap(&tm_w);
         tc::prefetch_tmap(&tm_x);
+        tc::prefetch_tmap(&tm_y);
     }
     if (warp == 1) { tc::tmem_alloc(tmem_slot, TMEM_COLS); tc::tmem_relinquish(); }
     tc::tc_fence_before_sync();
@@ -166,19 +204,17 @@ conv_fprop_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-                const int m0 = (tile % p.m_tiles) * BM;
-                const int nt_idx = tile / p.m_tiles;
-                const int img = nt_idx / p.tiles_per_img, h0 = (nt_idx % p.tiles_per_img) * p.rows_per_tile;
+            for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
+                const FpropItem wi = fprop_item<MH>(p, item);
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
                     const int s = it % STAGES;
                     if (!tc::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
                     uint8_t *sa = smem + (size_t)s * stage_bytes, *sb = sa + a_bytes;
-                    tc::mbar_expect_tx(&full[s], a_bytes + b_bytes);
+                    tc::mbar_expect_tx(&full[s], wi.mh * (BM * BK * 2) + b_bytes);
                     const int tap = kb / cblocks, cb = kb % cblocks;
                     const int r = tap / p.taps_s, sft = tap % p.taps_s;
-                    tc::tma_load_2d(sa, &tm_w, &full[s], kb * BK, m0);
-                    tc::tma_load_4d(sb, &tm_x, &full[s], cb * BK, sft - p.pad, h0 + r - p.pad, img);
+                    for (int h = 0; h < wi.mh; ++h) tc::tma_load_2d(sa + h * (BM * BK * 2), &tm_w, &full[s], kb * BK, wi.m0 + h * BM);
+                    tc::tma_load_4d(sb, &tm_x, &full[s], cb * BK, sft - p.pad, wi.h0 + r - p.pad, wi.img);
                 }
             }
         }
@@ -187,9 +223,12 @@ conv_fprop_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
             const uint32_t idesc = tc::instr_desc_bf16(BM, p.nt, false, false);
             uint32_t it = 0, t_local = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++t_local) {
-                const int buf = t_local & 1;
-                if (!tc::mbar_wait(&tmem_empty[buf], ((t_local >> 1) & 1) ^ 1, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) break;
+            for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x, ++t_local) {
+                const FpropItem wi = fprop_item<MH>(p, item);
+                const int buf = MH == 1 ? (t_local & 1) : 0;
+                const uint32_t empty_parity = MH == 1 ? (((t_local >> 1) & 1) ^ 1) : ((t_local & 1) ^ 1);
+                if (!tc::mbar_wait(&tmem_empty[buf], empty_parity, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) break;
+                if (MH == 2 && !tc::mbar_wait(&tmem_empty[1], empty_parity, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) break;
                 tc::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * 256;
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
@@ -198,9 +237,11 @@ conv_fprop_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
                     tc::tc_fence_after_sync();
                     const uint32_t sa = tc::smem_u32(smem + (size_t)s * stage_bytes), sb = sa + a_bytes;
 #pragma unroll
-                    for (int kk = 0; kk < BK / 16; ++kk)
-                        tc::mma_bf16(d_tmem, tc::smem_desc(sa + kk * 32, 16, 1024), tc::smem_desc(sb + kk * 32, 16, 1024), idesc,
-                                     (kb | kk) != 0);
+                    for (int kk = 0; kk < BK / 16; ++kk) {
+                        const uint64_t db = tc::smem_desc(sb + kk * 32, 16, 1024);
+                        for (int h = 0; h < wi.mh; ++h)
+                            tc::mma_bf16(d_tmem + h * 256, tc::smem_desc(sa + h * (BM * BK * 2) + kk * 32, 16, 1024), db, idesc, (kb | kk) != 0);
+                    }
                     tc::mma_commit(&empty[s]);
                 }
                 if (ok) tc::mma_commit(&tmem_full[buf]);
@@ -208,42 +249,71 @@ conv_fprop_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
         }
     } else {
         const int quarter = warp & 3;
-        uint32_t t_local = 0;
-        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++t_local) {
-            const int buf = t_local & 1;
-            const int m0 = (tile % p.m_tiles) * BM;
-            const int nt_idx = tile / p.m_tiles;
-            const int img = nt_idx / p.tiles_per_img, h0 = (nt_idx % p.tiles_per_img) * p.rows_per_tile;
+        const int half = (warp - 2) >> 2;                  // MH = 2: which accumulator this warp drains
+        uint8_t *my_stage = staging + (size_t)(warp - 2) * 4096;
+        uint32_t t_local = 0, blk_count = 0;
+        for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++t_local) {
+            const FpropItem wi = fprop_item<MH>(p, item);
+            const int buf = MH == 1 ? (t_local & 1) : half;
+            const int fbar = MH == 1 ? (t_local & 1) : 0;
+            const uint32_t full_parity = MH == 1 ? ((t_local >> 1) & 1) : (t_local & 1);
             int ok = 1;
-            if (lane == 0) ok = tc::mbar_wait(&tmem_full[buf], (t_local >> 1) & 1, abort_flag, p.err, tc::ERR_WAIT_TMEM_FULL) ? 1 : 0;
+            if (lane == 0) ok = tc::mbar_wait(&tmem_full[fbar], full_parity, abort_flag, p.err, tc::ERR_WAIT_TMEM_FULL) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
             tc::tc_fence_after_sync();
-            const int o = m0 + quarter * 32 + lane;
-            float bias = 0.0f;
-            if (p.bias != nullptr && o < p.Cout)
-                bias = p.bias_bf16 ? __bfloat162float(((const __nv_bfloat16 *)p.bias)[o]) : ((const float *)p.bias)[o];
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * 256;
-            __nv_bfloat16 *dst = p.out + (((size_t)img * p.Cout + o) * p.H + h0) * p.W;
+            if (half < wi.mh) {                            // a single item leaves the second accumulator unused
+                const int o0 = wi.m0 + half * BM + quarter * 32;   // this warp's 32 output channels; lane = channel
+                const int o = o0 + lane;
+                float bias = 0.0f;
+                if (p.bias != nullptr && o < p.Cout)
+                    bias = p.bias_bf16 ? __bfloat162float(((const __nv_bfloat16 *)p.bias)[o]) : ((const float *)p.bias)[o];
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * 256;
 #pragma unroll 1
-            for (int c = 0; c < p.nt / 32; ++c) {
-                uint32_t r[32];
-                tc::tmem_ld_32x32(taddr + c * 32, r);
-                tc::tmem_ld_wait();
-                if (o < p.Cout) {
+                for (int c = 0; c < p.nt / 32; ++c, ++blk_count) {
+                    uint32_t r[32];
+                    tc::tmem_ld_32x32(taddr + c * 32, r);
+                    tc::tmem_ld_wait();
                     float v[32];
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = act_fwd<true>(__uint_as_float(r[j]) + bias, p.act);
+                    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) + bias;
+                    switch (p.act) {
+                    case RELAY_ACT_RELU:
 #pragma unroll
-                    for (int j = 0; j < 32; j += 8)
-                        *reinterpret_cast<uint4 *>(dst + c * 32 + j) = make_uint4(pack2(v[j], v[j + 1]), pack2(v[j + 2], v[j + 3]),
-                                                                                 pack2(v[j + 4], v[j + 5]), pack2(v[j + 6], v[j + 7]));
+                        for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.0f);
+                        break;
+                    case RELAY_ACT_TANH:
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = tanh_<true>(v[j]);
+                        break;
+                    case RELAY_ACT_SIGMOID:
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = sigmoid_<true>(v[j]);
+                        break;
+                    default: break;
+                    }
+                    // 32 channels x 32 pixels (64 bytes per row) -> staging (2 buffers of 2 KB) -> TMA tile store
+                    uint8_t *st = my_stage + (blk_count & 1) * 2048;
+                    if (lane == 0) tc::tma_store_wait_read<1>();
+                    __syncwarp();
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        *reinterpret_cast<uint4 *>(st + lane * 64 + q * 16) =
+                            make_uint4(pack2(v[8 * q], v[8 * q + 1]), pack2(v[8 * q + 2], v[8 * q + 3]), pack2(v[8 * q + 4], v[8 * q + 5]),
+                                       pack2(v[8 * q + 6], v[8 * q + 7]));
+                    tc::fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tc::tma_store_2d(&tm_y, st, wi.h0 * p.W + c * 32, wi.img * p.Cout + o0);
+                        tc::tma_store_commit();
+                    }
                 }
             }
             tc::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) tc::mbar_arrive(&tmem_empty[buf]);
         }
+        if (lane == 0) tc::tma_store_wait_all<0>();
     }
     tc::tc_fence_before_sync();
     __syncthreads();
@@ -263,7 +333,8 @@ struct WgradParams {
 };
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_dz, const __grid_constant__ CUtensorMap tm_x, const WgradParams p)
+conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_dz, const __grid_constant__ CUtensorMap tm_x,
+                     const __grid_constant__ CUtensorMap tm_part, const WgradParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -271,7 +342,8 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_dz, const __grid_con
     const int a_bytes = (BM / 64) * box_bytes, b_bytes = (p.nt / 64) * box_bytes;
     const int stage_bytes = a_bytes + b_bytes;
     const int STAGES = p.stages;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + (size_t)STAGES * stage_bytes);
+    uint8_t *staging = smem + (size_t)STAGES * stage_bytes;           // [epilogue warp][2][4 KB]
+    uint64_t *bars = reinterpret_cast<uint64_t *>(staging + 4 * 8192);
     uint64_t *full = bars, *empty = bars + STAGES, *tmem_full = bars + 2 * STAGES;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 2);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
@@ -341,9 +413,9 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_dz, const __grid_con
         }
         if (ok) {
             tc::tc_fence_after_sync();
-            const int o = o0 + quarter * 32 + lane;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
-            float *dst = p.part + (((size_t)slice * (p.taps_r * p.taps_s) + tap) * p.O + o) * p.C + c0;
+            uint8_t *my_stage = staging + (size_t)(warp - 2) * 8192;
+            const int row0 = (slice * (p.taps_r * p.taps_s) + tap) * p.O + o0 + quarter * 32;   // row of the [slice][tap][O] x [C] partial
 #pragma unroll 1
             for (int c = 0; c < p.nt / 32; ++c) {
                 uint32_t v[32];
@@ -354,12 +426,12 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_dz, const __grid_con
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0u;
                 }
-                if (o < p.O) {
+                uint4 piece[8];
 #pragma unroll
-                    for (int j = 0; j < 32; j += 4)
-                        *reinterpret_cast<uint4 *>(dst + c * 32 + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                }
+                for (int q = 0; q < 8; ++q) piece[q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                tc::warp_store_block<1>(&tm_part, my_stage + (c & 1) * 4096, piece, lane, c0 + c * 32, row0);
             }
+            if (lane == 0) tc::tma_store_wait_all<0>();
         }
     }
     tc::tc_fence_before_sync();
@@ -400,9 +472,10 @@ TcPlan plan(const ConvDims &d)
     pl.wg_nt = (int)std::min<int64_t>(256, d.C);
     const size_t box = (size_t)pl.rows_per_kblock * d.W * 128;
     auto wg_stage = [&](int nt) { return (size_t)(BM / 64 + nt / 64) * box; };
-    while (pl.wg_nt > 64 && (kSmemLimit - 1024) / wg_stage(pl.wg_nt) < 2) pl.wg_nt -= 64;
-    if ((kSmemLimit - 1024) / wg_stage(pl.wg_nt) < 2 || d.C % pl.wg_nt) return pl;
-    pl.wg_stages = (int)std::min<size_t>(4, (kSmemLimit - 1024) / wg_stage(pl.wg_nt));
+    constexpr size_t wg_fixed = 1024 + 4 * 8192;   // alignment slack + store staging
+    while (pl.wg_nt > 64 && (kSmemLimit - wg_fixed) / wg_stage(pl.wg_nt) < 2) pl.wg_nt -= 64;
+    if ((kSmemLimit - wg_fixed) / wg_stage(pl.wg_nt) < 2 || d.C % pl.wg_nt) return pl;
+    pl.wg_stages = (int)std::min<size_t>(4, (kSmemLimit - wg_fixed) / wg_stage(pl.wg_nt));
     pl.wg_c_tiles = (int)(d.C / pl.wg_nt);
     pl.wg_m_tiles = (int)(d.O / BM);
     const int base_units = 9 * pl.wg_m_tiles * pl.wg_c_tiles;
@@ -422,25 +495,43 @@ TcPlan plan(const ConvDims &d)
 relay_status_t launch_fprop(const ConvDims &d, const TcPlan &pl, const void *act_nhwc, int Cin, const void *wpacked, int Cout,
                             const void *bias, int32_t b_dt, int act, void *out_nchw, cudaStream_t st)
 {
-    CUtensorMap tm_w, tm_x;
+    CUtensorMap tm_w, tm_x, tm_y;
     RELAY_TRY(make_tmap_2d_bf16(&tm_w, wpacked, (uint64_t)9 * Cin, Cout, (uint64_t)9 * Cin, BK, BM));
     RELAY_TRY(make_tmap_nhwc_bf16(&tm_x, act_nhwc, Cin, d.W, d.H, d.Nb, BK, (uint32_t)d.W, pl.rows_per_tile));
-    FpropParams p{};
-    p.Cin = Cin; p.Cout = Cout; p.H = (int)d.H; p.W = (int)d.W; p.Nb = (int)d.Nb; p.taps_r = 3; p.taps_s = 3; p.pad = 1;
-    p.rows_per_tile = pl.rows_per_tile; p.nt = pl.rows_per_tile * (int)d.W;
-    p.m_tiles = Cout / BM; p.tiles_per_img = (int)d.H / pl.rows_per_tile; p.n_tiles_total = (int)d.Nb * p.tiles_per_img;
-    p.k_blocks = 9 * Cin / BK; p.stages = pl.fp_stages;
-    p.out = (__nv_bfloat16 *)out_nchw; p.bias = bias; p.bias_bf16 = b_dt == RELAY_BF16; p.act = act;
-    p.err = device_error_word();
-    if (!p.err) return fail(RELAY_ERR_CUDA, "no device error word");
-    const size_t stage = BM * BK * 2 + (((size_t)p.nt * BK * 2 + 1023) & ~size_t(1023));
-    const size_t smem = 1024 + (size_t)p.stages * stage + 256;
-    RELAY_CUDA(cudaFuncSetAttribute(conv_fprop_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    // output NCHW as [Nb * Cout rows][H * W columns]; 32 x 32 boxes, rows of 64 bytes, no swizzle
+    RELAY_TRY(make_tmap_2d(&tm_y, false, out_nchw, (uint64_t)(d.H * d.W), (uint64_t)d.Nb * Cout, (uint64_t)(d.H * d.W), 32, 32, false));
     int dev = 0, sms = 148;
     RELAY_CUDA(cudaGetDevice(&dev));
     RELAY_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    const int grid = std::min(p.m_tiles * p.n_tiles_total, sms);
-    conv_fprop_tc_kernel<<<grid, NUM_THREADS, smem, st>>>(tm_w, tm_x, p);
+    FpropParams p{};
+    p.Cin = Cin; p.Cout = Cout; p.H = (int)d.H; p.W = (int)d.W; p.Nb = (int)d.Nb; p.taps_r = 3; p.taps_s = 3; p.pad = 1;
+    p.rows_per_tile = pl.rows_per_tile; p.nt = pl.rows_per_tile * (int)d.W;
+    p.tiles_per_img = (int)d.H / pl.rows_per_tile; p.n_tiles_total = (int)d.Nb * p.tiles_per_img;
+    p.k_blocks = 9 * Cin / BK;
+    p.bias = bias; p.bias_bf16 = b_dt == RELAY_BF16; p.act = act;
+    p.err = device_error_word();
+    if (!p.err) return fail(RELAY_ERR_CUDA, "no device error word");
+    // pairs fill whole rounds over the SMs; the remainder runs as singles
+    const int64_t total_pairs = Cout % 256 == 0 ? (int64_t)p.n_tiles_total * (Cout / 256) : 0;
+    const int mh = total_pairs >= sms ? 2 : 1;
+    const size_t b_stage = ((size_t)p.nt * BK * 2 + 1023) & ~size_t(1023);
+    const size_t stage = (size_t)mh * BM * BK * 2 + b_stage;
+    const size_t staging = (size_t)4 * mh * 4096;
+    p.stages = (int)std::min<size_t>(6, (kSmemLimit - 1024 - staging) / stage);
+    if (p.stages < 2) return fail(RELAY_ERR_UNSUPPORTED, "conv2d tile does not fit in shared memory");
+    const size_t smem = 1024 + (size_t)p.stages * stage + staging + 256;
+    if (mh == 2) {
+        p.pairs_per_ntile = Cout / 256;
+        const int64_t ntiles_as_pairs = (total_pairs / sms) * sms / p.pairs_per_ntile;   // whole n-tiles only
+        p.n_pairs = (int)(ntiles_as_pairs * p.pairs_per_ntile);
+        p.n_items = p.n_pairs + (int)((p.n_tiles_total - ntiles_as_pairs) * (Cout / BM));
+        RELAY_CUDA(cudaFuncSetAttribute(conv_fprop_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        conv_fprop_tc_kernel<2><<<std::min(p.n_items, sms), 64 + 256, smem, st>>>(tm_w, tm_x, tm_y, p);
+    } else {
+        p.pairs_per_ntile = 1; p.n_pairs = 0; p.n_items = p.n_tiles_total * (Cout / BM);
+        RELAY_CUDA(cudaFuncSetAttribute(conv_fprop_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        conv_fprop_tc_kernel<1><<<std::min(p.n_items, sms), 64 + 128, smem, st>>>(tm_w, tm_x, tm_y, p);
+    }
     return check_launch("conv_fprop_tc");
 }
 
@@ -532,10 +623,12 @@ relay_status_t launch_conv_grad_tc(const ConvDims &d, const void *x, const void 
     p.stages = pl.wg_stages; p.part = part; p.err = device_error_word();
     if (!p.err) return fail(RELAY_ERR_CUDA, "no device error word");
     const size_t stage = (size_t)(BM / 64 + p.nt / 64) * p.kpix * 128;
-    const size_t smem = 1024 + (size_t)p.stages * stage + 256;
+    const size_t smem = 1024 + (size_t)p.stages * stage + 4 * 8192 + 256;
     RELAY_CUDA(cudaFuncSetAttribute(conv_wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    CUtensorMap tm_part;
+    RELAY_TRY(make_tmap_2d(&tm_part, true, part, (uint64_t)d.C, (uint64_t)p.n_slices * 9 * d.O, (uint64_t)d.C, 32, 32, true));
     const int grid = 9 * p.m_tiles * p.c_tiles * p.n_slices;
-    conv_wgrad_tc_kernel<<<grid, NUM_THREADS, smem, st>>>(tm_dz, tm_x, p);
+    conv_wgrad_tc_kernel<<<grid, NUM_THREADS, smem, st>>>(tm_dz, tm_x, tm_part, p);
     RELAY_TRY(check_launch("conv_wgrad_tc"));
     wgrad_reduce_kernel<<<(unsigned)std::min<int64_t>(148 * 8, (9 * d.O * d.C + 255) / 256), 256, 0, st>>>(part, p.n_slices, (__nv_bfloat16 *)dw,
                                                                                                           (int)d.O, (int)d.C, 9);

@@ -273,7 +273,7 @@ EncodeTiledFn encode_fn()
 // 2-D tensor map (bf16 or f32): `inner` contiguous elements per row, `outer` rows `row_stride` elements
 // apart, box = box_inner x box_outer, 128-byte swizzle, out-of-range elements read as zero / not written
 relay_status_t make_tmap_2d(CUtensorMap *m, bool f32, const void *base, uint64_t inner, uint64_t outer, uint64_t row_stride,
-                            uint32_t box_inner, uint32_t box_outer)
+                            uint32_t box_inner, uint32_t box_outer, bool swizzle128)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return fail(RELAY_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
@@ -282,8 +282,8 @@ relay_status_t make_tmap_2d(CUtensorMap *m, bool f32, const void *base, uint64_t
     cuuint32_t box[2] = {box_inner, box_outer};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(RELAY_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
     return RELAY_OK;
 }
@@ -291,7 +291,7 @@ relay_status_t make_tmap_2d(CUtensorMap *m, bool f32, const void *base, uint64_t
 relay_status_t make_tmap_2d_bf16(CUtensorMap *m, const void *base, uint64_t inner, uint64_t outer, uint64_t row_stride,
                                  uint32_t box_inner, uint32_t box_outer)
 {
-    return make_tmap_2d(m, false, base, inner, outer, row_stride, box_inner, box_outer);
+    return make_tmap_2d(m, false, base, inner, outer, row_stride, box_inner, box_outer, true);
 }
 
 bool gemm_tc_eligible(const GemmDesc &g)
@@ -333,7 +333,7 @@ relay_status_t launch_gemm_tc(const GemmDesc &g, cudaStream_t st)
     if (!p.err) return fail(RELAY_ERR_CUDA, "no device error word");
     CUtensorMap tm_c;
     const bool f32 = g.out_dtype == RELAY_F32;
-    RELAY_TRY(make_tmap_2d(&tm_c, f32, g.c, g.N, g.M, g.ldc, f32 ? 32 : 64, 32));
+    RELAY_TRY(make_tmap_2d(&tm_c, f32, g.c, g.N, g.M, g.ldc, f32 ? 32 : 64, 32, true));
     const int grid = std::min(p.tiles_m * p.tiles_n, sms);
 #define LAUNCH(AMN, BMN, MHV)                                                                                             \
     do {                                                                                                                  \
