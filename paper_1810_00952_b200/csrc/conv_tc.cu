@@ -202,26 +202,32 @@ conv_fprop_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
 
     if (warp == 0) {
         if (lane == 0) {
-            uint32_t it = 0;
+            int s = 0;
+            uint32_t phase = 0;
             bool ok = true;
             for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
                 const FpropItem wi = fprop_item<MH>(p, item);
-                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    if (!tc::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
-                    uint8_t *sa = smem + (size_t)s * stage_bytes, *sb = sa + a_bytes;
-                    tc::mbar_expect_tx(&full[s], wi.mh * (BM * BK * 2) + b_bytes);
-                    const int tap = kb / cblocks, cb = kb % cblocks;
-                    const int r = tap / p.taps_s, sft = tap % p.taps_s;
-                    for (int h = 0; h < wi.mh; ++h) tc::tma_load_2d(sa + h * (BM * BK * 2), &tm_w, &full[s], kb * BK, wi.m0 + h * BM);
-                    tc::tma_load_4d(sb, &tm_x, &full[s], cb * BK, sft - p.pad, wi.h0 + r - p.pad, wi.img);
-                }
+                const uint32_t tx = wi.mh * (BM * BK * 2) + b_bytes;
+                int kb = 0;
+                for (int r = 0; r < p.taps_r && ok; ++r)
+                    for (int sft = 0; sft < p.taps_s && ok; ++sft)
+                        for (int cb = 0; cb < cblocks; ++cb, ++kb) {
+                            if (!tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
+                            uint8_t *sa = smem + (size_t)s * stage_bytes, *sb = sa + a_bytes;
+                            tc::mbar_expect_tx(&full[s], tx);
+                            tc::tma_load_2d(sa, &tm_w, &full[s], kb * BK, wi.m0);
+                            if (MH == 2 && wi.mh == 2) tc::tma_load_2d(sa + BM * BK * 2, &tm_w, &full[s], kb * BK, wi.m0 + BM);
+                            tc::tma_load_4d(sb, &tm_x, &full[s], cb * BK, sft - p.pad, wi.h0 + r - p.pad, wi.img);
+                            if (++s == STAGES) { s = 0; phase ^= 1; }
+                        }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = tc::instr_desc_bf16(BM, p.nt, false, false);
-            uint32_t it = 0, t_local = 0;
+            const uint64_t desc_a0 = tc::smem_desc(tc::smem_u32(smem), 16, 1024), desc_b0 = tc::smem_desc(tc::smem_u32(smem) + a_bytes, 16, 1024);
+            uint32_t t_local = 0, phase = 0, stage_off = 0;   // stage_off = s * stage_bytes in 16-byte units
+            int s = 0;
             bool ok = true;
             for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x, ++t_local) {
                 const FpropItem wi = fprop_item<MH>(p, item);
@@ -231,18 +237,26 @@ conv_fprop_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
                 if (MH == 2 && !tc::mbar_wait(&tmem_empty[1], empty_parity, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) break;
                 tc::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * 256;
-                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    if (!tc::mbar_wait(&full[s], (it / STAGES) & 1, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    if (!tc::mbar_wait(&full[s], phase, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
                     tc::tc_fence_after_sync();
-                    const uint32_t sa = tc::smem_u32(smem + (size_t)s * stage_bytes), sb = sa + a_bytes;
+                    // descriptors differ from the stage-0 ones only in the start address field (16-byte units),
+                    // so the issuing thread spends one add per MMA instead of rebuilding them
+                    const uint64_t da = desc_a0 + stage_off, db = desc_b0 + stage_off;
+                    const uint32_t acc = kb != 0;
+                    if (MH == 2 && wi.mh == 2) {
 #pragma unroll
-                    for (int kk = 0; kk < BK / 16; ++kk) {
-                        const uint64_t db = tc::smem_desc(sb + kk * 32, 16, 1024);
-                        for (int h = 0; h < wi.mh; ++h)
-                            tc::mma_bf16(d_tmem + h * 256, tc::smem_desc(sa + h * (BM * BK * 2) + kk * 32, 16, 1024), db, idesc, (kb | kk) != 0);
+                        for (int kk = 0; kk < BK / 16; ++kk) {
+                            tc::mma_bf16(d_tmem, da + kk * 2, db + kk * 2, idesc, acc | (kk != 0));
+                            tc::mma_bf16(d_tmem + 256, da + (BM * BK * 2 >> 4) + kk * 2, db + kk * 2, idesc, acc | (kk != 0));
+                        }
+                    } else {
+#pragma unroll
+                        for (int kk = 0; kk < BK / 16; ++kk) tc::mma_bf16(d_tmem, da + kk * 2, db + kk * 2, idesc, acc | (kk != 0));
                     }
                     tc::mma_commit(&empty[s]);
+                    stage_off += (uint32_t)stage_bytes >> 4;
+                    if (++s == STAGES) { s = 0; phase ^= 1; stage_off = 0; }
                 }
                 if (ok) tc::mma_commit(&tmem_full[buf]);
             }
@@ -397,9 +411,9 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_dz, const __grid_con
                 if (!tc::mbar_wait(&full[s], (kb / STAGES) & 1, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
                 tc::tc_fence_after_sync();
                 const uint32_t sa = tc::smem_u32(smem + (size_t)s * stage_bytes), sb = sa + a_bytes;
-                for (int kk = 0; kk < p.kpix / 16; ++kk)
-                    tc::mma_bf16(tmem_base, tc::smem_desc(sa + kk * 2048, box_bytes, 1024), tc::smem_desc(sb + kk * 2048, box_bytes, 1024),
-                                 idesc, (kb | kk) != 0);
+                const uint64_t da = tc::smem_desc(sa, box_bytes, 1024), db = tc::smem_desc(sb, box_bytes, 1024);
+                const uint32_t acc = kb != 0;
+                for (int kk = 0; kk < p.kpix / 16; ++kk) tc::mma_bf16(tmem_base, da + kk * 128, db + kk * 128, idesc, acc | (kk != 0));
                 tc::mma_commit(&empty[s]);
             }
             if (ok) tc::mma_commit(&tmem_full[0]);

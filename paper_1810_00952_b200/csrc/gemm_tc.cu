@@ -145,13 +145,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            uint32_t it = 0;
+            int s = 0;
+            uint32_t phase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
                 const int m0 = (tile % p.tiles_m) * BM, n0 = (tile / p.tiles_m) * BN;
-                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    if (!tc::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    if (!tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
                     uint8_t *sa = smem + (size_t)s * STAGE_BYTES, *sb = sa + A_BYTES;
                     tc::mbar_expect_tx(&full[s], STAGE_BYTES);
                     const int k0 = kb * BK;
@@ -167,6 +167,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     } else {
                         tc::tma_load_2d(sb, &tm_b, &full[s], k0, n0);
                     }
+                    if (++s == STAGES) { s = 0; phase ^= 1; }
                 }
             }
         }
@@ -178,36 +179,36 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             // MN-major: 64-wide M/N groups one TMA box apart, 8-k atoms 1024 B apart, one MMA = 2 atoms.
             constexpr uint32_t a_lbo = A_MN ? MN_BOX_BYTES : 16, b_lbo = B_MN ? MN_BOX_BYTES : 16;
             constexpr uint32_t a_step = A_MN ? 2048 : 32, b_step = B_MN ? 2048 : 32;
-            uint32_t it = 0, t_local = 0;
+            // descriptors of a stage differ from the stage-0 ones only in the start-address field (16-byte
+            // units): the issuing thread spends one add per MMA instead of rebuilding them
+            const uint64_t desc_a0 = tc::smem_desc(tc::smem_u32(smem), a_lbo, 1024);
+            const uint64_t desc_b0 = tc::smem_desc(tc::smem_u32(smem) + A_BYTES, b_lbo, 1024);
+            uint32_t t_local = 0, phase = 0, stage_off = 0;
+            int s = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++t_local) {
                 // MH = 1: accumulator t_local & 1;  MH = 2: accumulator h for half h, both used by every tile
                 const int buf = MH == 1 ? (t_local & 1) : 0;
                 const uint32_t empty_parity = MH == 1 ? (((t_local >> 1) & 1) ^ 1) : ((t_local & 1) ^ 1);
                 if (!tc::mbar_wait(&tmem_empty[buf], empty_parity, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) break;
+                if (MH == 2 && !tc::mbar_wait(&tmem_empty[1], empty_parity, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) break;
                 tc::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * BN;
-                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    if (!tc::mbar_wait(&full[s], (it / STAGES) & 1, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    if (!tc::mbar_wait(&full[s], phase, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
                     tc::tc_fence_after_sync();
-                    const uint32_t sa = tc::smem_u32(smem + (size_t)s * STAGE_BYTES), sb = sa + A_BYTES;
+                    const uint64_t da = desc_a0 + stage_off, db = desc_b0 + stage_off;
+                    const uint32_t acc = kb != 0;
 #pragma unroll
                     for (int kk = 0; kk < BK / 16; ++kk) {
-                        const uint64_t db = tc::smem_desc(sb + kk * b_step, b_lbo, 1024);
 #pragma unroll
-                        for (int h = 0; h < MH; ++h) {
-                            if (MH == 2 && h == 1 && kb == 0 && kk == 0) {   // the second half may still be draining
-                                if (!tc::mbar_wait(&tmem_empty[1], empty_parity, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) { ok = false; break; }
-                                tc::tc_fence_after_sync();
-                            }
-                            const uint64_t da = tc::smem_desc(sa + h * (128 * BK * 2) + kk * a_step, a_lbo, 1024);
-                            tc::mma_bf16(d_tmem + h * BN, da, db, idesc, (kb | kk) != 0);
-                        }
-                        if (!ok) break;
+                        for (int h = 0; h < MH; ++h)
+                            tc::mma_bf16(d_tmem + h * BN, da + ((h * (128 * BK * 2) + kk * a_step) >> 4), db + ((kk * b_step) >> 4), idesc,
+                                         acc | (kk != 0));
                     }
-                    if (!ok) break;
                     tc::mma_commit(&empty[s]);          // the stage is free once these MMAs have read it
+                    stage_off += STAGE_BYTES >> 4;
+                    if (++s == STAGES) { s = 0; phase ^= 1; stage_off = 0; }
                 }
                 if (ok) tc::mma_commit(&tmem_full[buf]);  // the accumulator(s) are complete
             }
