@@ -40,9 +40,12 @@ constexpr int TMEM_COLS = 512;
 // ---------------------------------------------------------------------------------------------------
 // out[n][hw][c] = in[n][c][hw]  (GRAD: in = dy, multiplied by act'(y) on the way: dZ in NHWC).
 // 64 channels x 64 pixels per block, 16-byte global accesses on both sides (HW % 8 == 0, C % 8 == 0).
+// GRAD with db_part != null also writes, per block, the sums over its 64 pixels of the stored (rounded) dZ
+// of each of its 64 channels to db_part[(n * gridDim.x + blockIdx.x) * C + c]: the bias gradient's partials.
 template <bool GRAD>
 __global__ void __launch_bounds__(256) nchw_to_nhwc_kernel(const __nv_bfloat16 *__restrict__ in, const __nv_bfloat16 *__restrict__ y,
-                                                            __nv_bfloat16 *__restrict__ out, int C, int HW, int act)
+                                                            __nv_bfloat16 *__restrict__ out, int C, int HW, int act,
+                                                            float *__restrict__ db_part)
 {
     __shared__ __align__(16) __nv_bfloat16 tile[64][72];   // [channel][pixel], rows 144 B apart
     const int n = blockIdx.z, c0 = blockIdx.y * 64, p0 = blockIdx.x * 64;
@@ -67,6 +70,15 @@ __global__ void __launch_bounds__(256) nchw_to_nhwc_kernel(const __nv_bfloat16 *
             }
         }
         *reinterpret_cast<uint4 *>(&tile[cl][chunk * 8]) = v;
+        if (GRAD && db_part != nullptr) {          // the 8 lanes that share a channel row combine in a fixed order
+            float r[8];
+            unpack(v, r);
+            float sum = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
+            sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+            sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+            sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+            if (chunk == 0 && c < C) db_part[((size_t)n * gridDim.x + blockIdx.x) * C + c] = sum;
+        }
     }
     __syncthreads();
 #pragma unroll
@@ -501,7 +513,7 @@ TcPlan plan(const ConvDims &d)
     pl.dz_nhwc = align_up((size_t)d.Nb * d.O * d.H * d.W * 2, 1024);
     pl.wpack = align_up((size_t)d.O * d.C * 9 * 2, 1024);
     pl.part = align_up((size_t)pl.wg_slices * 9 * d.O * d.C * sizeof(float), 1024);
-    pl.db_part = align_up((size_t)colsum_slices(d.Nb * d.H * d.W, d.O, RELAY_BF16) * d.O * sizeof(float), 1024);
+    pl.db_part = align_up((size_t)d.Nb * ((d.H * d.W + 63) / 64) * d.O * sizeof(float), 1024);   // one partial row per repack block
     pl.ok = true;
     return pl;
 }
@@ -550,11 +562,11 @@ relay_status_t launch_fprop(const ConvDims &d, const TcPlan &pl, const void *act
 }
 
 relay_status_t launch_transpose(bool grad, const void *in, const void *y, void *out, int64_t Nb, int64_t C, int64_t HW, int act,
-                                cudaStream_t st)
+                                float *db_part, cudaStream_t st)
 {
     dim3 grid((unsigned)((HW + 63) / 64), (unsigned)((C + 63) / 64), (unsigned)Nb);
-    if (grad) nchw_to_nhwc_kernel<true><<<grid, 256, 0, st>>>((const __nv_bfloat16 *)in, (const __nv_bfloat16 *)y, (__nv_bfloat16 *)out, (int)C, (int)HW, act);
-    else nchw_to_nhwc_kernel<false><<<grid, 256, 0, st>>>((const __nv_bfloat16 *)in, nullptr, (__nv_bfloat16 *)out, (int)C, (int)HW, act);
+    if (grad) nchw_to_nhwc_kernel<true><<<grid, 256, 0, st>>>((const __nv_bfloat16 *)in, (const __nv_bfloat16 *)y, (__nv_bfloat16 *)out, (int)C, (int)HW, act, db_part);
+    else nchw_to_nhwc_kernel<false><<<grid, 256, 0, st>>>((const __nv_bfloat16 *)in, nullptr, (__nv_bfloat16 *)out, (int)C, (int)HW, act, nullptr);
     return check_launch("nchw_to_nhwc");
 }
 
@@ -601,7 +613,7 @@ relay_status_t launch_conv_fwd_tc(const ConvDims &d, const void *x, const void *
     TcPlan pl = plan(d);
     char *base = (char *)ws;
     void *x_nhwc = base, *wf = base + pl.x_nhwc;
-    RELAY_TRY(launch_transpose(false, x, nullptr, x_nhwc, d.Nb, d.C, d.H * d.W, 0, st));
+    RELAY_TRY(launch_transpose(false, x, nullptr, x_nhwc, d.Nb, d.C, d.H * d.W, 0, nullptr, st));
     pack_weights_kernel<<<(unsigned)((d.O * d.C * 9 + 255) / 256), 256, 0, st>>>((const __nv_bfloat16 *)w, (__nv_bfloat16 *)wf, nullptr, (int)d.O, (int)d.C, 3, 3);
     RELAY_TRY(check_launch("pack_weights"));
     return launch_fprop(d, pl, x_nhwc, (int)d.C, wf, (int)d.O, b, b_dt, act, y, st);
@@ -619,9 +631,10 @@ relay_status_t launch_conv_grad_tc(const ConvDims &d, const void *x, const void 
     float *db_part = (float *)(base + pl.x_nhwc + pl.dz_nhwc + pl.wpack + pl.part);
     const int64_t HW = d.H * d.W;
     // dZ = dy (.) act'(y), written straight into NHWC; x into NHWC
-    RELAY_TRY(launch_transpose(true, dy, y, dz_nhwc, d.Nb, d.O, HW, act, st));
-    RELAY_TRY(launch_transpose(false, x, nullptr, x_nhwc, d.Nb, d.C, HW, 0, st));
-    if (db) RELAY_TRY(launch_colsum_bf16(dz_nhwc, d.Nb * HW, d.O, db_part, db, st));
+    // (the same pass leaves per-block partial sums of dZ over pixels for the bias gradient)
+    RELAY_TRY(launch_transpose(true, dy, y, dz_nhwc, d.Nb, d.O, HW, act, db ? db_part : nullptr, st));
+    RELAY_TRY(launch_transpose(false, x, nullptr, x_nhwc, d.Nb, d.C, HW, 0, nullptr, st));
+    if (db) RELAY_TRY(launch_colsum_finalize(db_part, (int)(d.Nb * ((HW + 63) / 64)), d.O, 1.0f, db, st));
     if (dx) {
         pack_weights_kernel<<<(unsigned)((d.O * d.C * 9 + 255) / 256), 256, 0, st>>>((const __nv_bfloat16 *)w, nullptr, (__nv_bfloat16 *)wb, (int)d.O, (int)d.C, 3, 3);
         RELAY_TRY(check_launch("pack_weights"));
