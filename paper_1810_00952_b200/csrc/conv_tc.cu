@@ -47,7 +47,9 @@ __global__ void __launch_bounds__(256) nchw_to_nhwc_kernel(const __nv_bfloat16 *
                                                             __nv_bfloat16 *__restrict__ out, int C, int HW, int act,
                                                             float *__restrict__ db_part)
 {
-    __shared__ __align__(16) __nv_bfloat16 tile[64][72];   // [channel][pixel], rows 144 B apart
+    // [pixel][channel]; 33 words per row: the scattered 2-byte stores below are at most 2-way conflicted and
+    // the 4-byte reads of the write phase are conflict-free
+    __shared__ __align__(16) __nv_bfloat16 tile[64][66];
     const int n = blockIdx.z, c0 = blockIdx.y * 64, p0 = blockIdx.x * 64;
     const size_t img = (size_t)n * C * HW;
 #pragma unroll
@@ -69,7 +71,12 @@ __global__ void __launch_bounds__(256) nchw_to_nhwc_kernel(const __nv_bfloat16 *
                 v = pack(a);
             }
         }
-        *reinterpret_cast<uint4 *>(&tile[cl][chunk * 8]) = v;
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            tile[chunk * 8 + 2 * j][cl] = __ushort_as_bfloat16((unsigned short)(w[j] & 0xffffu));
+            tile[chunk * 8 + 2 * j + 1][cl] = __ushort_as_bfloat16((unsigned short)(w[j] >> 16));
+        }
         if (GRAD && db_part != nullptr) {          // the 8 lanes that share a channel row combine in a fixed order
             float r[8];
             unpack(v, r);
@@ -84,13 +91,11 @@ __global__ void __launch_bounds__(256) nchw_to_nhwc_kernel(const __nv_bfloat16 *
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
         const int idx = threadIdx.x + i * 256;
-        const int pl = idx & 63, cchunk = idx >> 6;          // a warp reads 32 consecutive pixels of one channel row
+        const int pl = idx >> 3, cchunk = idx & 7;           // 8 lanes write the 128 contiguous bytes of one pixel
         const int c = c0 + cchunk * 8, p = p0 + pl;
         if (c < C && p < HW) {
-            __align__(16) __nv_bfloat16 e[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) e[j] = tile[cchunk * 8 + j][pl];
-            *reinterpret_cast<uint4 *>(out + ((size_t)n * HW + p) * C + c) = *reinterpret_cast<const uint4 *>(e);
+            const uint32_t *row = reinterpret_cast<const uint32_t *>(&tile[pl][cchunk * 8]);
+            *reinterpret_cast<uint4 *>(out + ((size_t)n * HW + p) * C + c) = make_uint4(row[0], row[1], row[2], row[3]);
         }
     }
 }
@@ -100,20 +105,15 @@ __global__ void __launch_bounds__(256) nchw_to_nhwc_kernel(const __nv_bfloat16 *
 __global__ void pack_weights_kernel(const __nv_bfloat16 *__restrict__ w, __nv_bfloat16 *__restrict__ wf,
                                     __nv_bfloat16 *__restrict__ wb, int O, int C, int R, int S)
 {
-    const int taps = R * S;
-    const int64_t total = (int64_t)O * C * taps;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const unsigned taps = R * S, total = (unsigned)O * C * taps;     // < 2^31 (checked by the plan)
+    for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
         if (wf) {
-            const int c = (int)(i % C);
-            const int tap = (int)((i / C) % taps);
-            const int o = (int)(i / ((int64_t)C * taps));
-            wf[i] = w[((int64_t)o * C + c) * taps + tap];
+            const unsigned c = i % C, t = i / C, tap = t % taps, o = t / taps;
+            wf[i] = w[(o * C + c) * taps + tap];
         }
         if (wb) {
-            const int o = (int)(i % O);
-            const int tap2 = (int)((i / O) % taps);
-            const int c = (int)(i / ((int64_t)O * taps));
-            wb[i] = w[((int64_t)o * C + c) * taps + (taps - 1 - tap2)];
+            const unsigned o = i % O, t = i / O, tap2 = t % taps, c = t / taps;
+            wb[i] = w[(o * C + c) * taps + (taps - 1 - tap2)];
         }
     }
 }
@@ -484,7 +484,7 @@ TcPlan plan(const ConvDims &d)
     TcPlan pl;
     if (d.dt != RELAY_BF16 || d.stride != 1 || d.R != 3 || d.S != 3 || d.pad != 1) return pl;
     if (d.C % 128 || d.O % 128 || d.W % 8 || d.W > 256 || d.H < 1 || d.Nb < 1) return pl;
-    if (d.Nb > 65535 || d.H * d.W > (1 << 24)) return pl;
+    if (d.Nb > 65535 || d.H * d.W > (1 << 24) || d.O * d.C * 9 >= (1ll << 31)) return pl;
     for (int rt = (int)std::min<int64_t>(d.H, 256 / d.W); rt >= 1; --rt)
         if (d.H % rt == 0 && (rt * d.W) % 32 == 0) { pl.rows_per_tile = rt; break; }
     for (int rk = (int)std::min<int64_t>(d.H, 128 / d.W); rk >= 1; --rk)
