@@ -118,18 +118,18 @@ __global__ void pack_weights_kernel(const __nv_bfloat16 *__restrict__ w, __nv_bf
     }
 }
 
-// dw[o][c][tap] = bf16( sum over slices, in slice order, of part[slice][tap][o][c] )
+// dw[o][c][tap] = bf16( sum over slices, in slice order, of part[slice][tap][o][c] ); one thread per (o, c)
+// so that the partial reads coalesce along c
 __global__ void wgrad_reduce_kernel(const float *__restrict__ part, int n_slices, __nv_bfloat16 *__restrict__ dw, int O, int C, int taps)
 {
-    const int64_t per_slice = (int64_t)taps * O * C;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < per_slice; i += (int64_t)gridDim.x * blockDim.x) {
-        const int tap = (int)(i % taps);          // i enumerates the OUTPUT (o, c, tap) so that stores coalesce
-        const int64_t oc = i / taps;
-        const int c = (int)(oc % C);
-        const int o = (int)(oc / C);
-        float s = 0.0f;
-        for (int j = 0; j < n_slices; ++j) s += part[(size_t)j * per_slice + ((int64_t)tap * O + o) * C + c];
-        dw[i] = __float2bfloat16_rn(s);
+    const unsigned oc_total = (unsigned)O * C;
+    const size_t per_slice = (size_t)taps * oc_total;
+    for (unsigned oc = blockIdx.x * blockDim.x + threadIdx.x; oc < oc_total; oc += gridDim.x * blockDim.x) {
+        for (int tap = 0; tap < taps; ++tap) {
+            float s = 0.0f;
+            for (int j = 0; j < n_slices; ++j) s += part[(size_t)j * per_slice + (size_t)tap * oc_total + oc];
+            dw[(size_t)oc * taps + tap] = __float2bfloat16_rn(s);
+        }
     }
 }
 
@@ -657,7 +657,7 @@ relay_status_t launch_conv_grad_tc(const ConvDims &d, const void *x, const void 
     const int grid = 9 * p.m_tiles * p.c_tiles * p.n_slices;
     conv_wgrad_tc_kernel<<<grid, NUM_THREADS, smem, st>>>(tm_dz, tm_x, tm_part, p);
     RELAY_TRY(check_launch("conv_wgrad_tc"));
-    wgrad_reduce_kernel<<<(unsigned)std::min<int64_t>(148 * 8, (9 * d.O * d.C + 255) / 256), 256, 0, st>>>(part, p.n_slices, (__nv_bfloat16 *)dw,
+    wgrad_reduce_kernel<<<(unsigned)((d.O * d.C + 127) / 128), 128, 0, st>>>(part, p.n_slices, (__nv_bfloat16 *)dw,
                                                                                                           (int)d.O, (int)d.C, 9);
     return check_launch("wgrad_reduce");
 }

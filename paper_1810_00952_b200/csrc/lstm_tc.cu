@@ -7,9 +7,14 @@
 //   memory ring by TMA (all k-blocks in flight at once)  ->  one thread issues tcgen05.mma
 //   (D[batch row, 64 gate columns] in TMEM)  ->  epilogue warps add the precomputed input projection,
 //   apply the gates, update c, write h_t (fp32 to h_all, bf16 to the exchange buffer)  ->  grid barrier.
+// Batch rows are independent, so the batch is split into groups of rows that run as separate sets of
+// blocks (separate exchange rows, separate barrier counters) when the SM count allows: each block then
+// streams fewer rows of h per step.
 // The grid barrier is a counter in global memory with a bounded spin; the kernel is launched
 // cooperatively so that all blocks are resident.
 #include <cooperative_groups.h>
+
+#include <algorithm>
 
 #include "ewise_kernels.cuh"
 #include "lstm.h"
@@ -30,6 +35,7 @@ constexpr int NUM_THREADS = 192;                 // warps 0-3 epilogue, warp 4 M
 
 struct Params {
     int T, B, H, n_blocks, k_blocks;
+    int rows_per_group, n_epi;       // batch rows per block group; epilogue warps that own rows (ceil(rows_per_group / 32))
     const float *zx;                 // [T*B][4H] input projection + bias
     const float *h0, *c0;            // [B][H]
     float *h_all, *c_final;          // [T][B][H], [B][H]
@@ -65,7 +71,11 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int j0 = blockIdx.x * UNITS;
+    const int blk = blockIdx.x % p.n_blocks, grp = blockIdx.x / p.n_blocks;
+    const int j0 = blk * UNITS;
+    const int b_lo = grp * p.rows_per_group;                      // first batch row of this block's group
+    const int nb = min(p.rows_per_group, p.B - b_lo);             // rows the group really has
+    unsigned int *counter = p.counter + grp * 32;                 // one barrier counter per group (128 B apart)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
@@ -87,9 +97,10 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp < 4) {
+      if (warp < p.n_epi) {
         // ------------------------------ epilogue / state owners ------------------------------
-        const int b = warp * 32 + lane;               // batch row = TMEM lane
-        const bool live = b < p.B;
+        const int b = b_lo + warp * 32 + lane;        // batch row; TMEM lane = row within the group
+        const bool live = warp * 32 + lane < nb;
         float c[UNITS];
 #pragma unroll
         for (int i = 0; i < UNITS; ++i) c[i] = live ? p.c0[(size_t)b * p.H + j0 + i] : 0.0f;
@@ -108,7 +119,7 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
         asm volatile("fence.proxy.async.global;" ::: "memory");
         __threadfence();
         __syncwarp();
-        if (lane == 0) red_release_add(p.counter, 1u);
+        if (lane == 0) red_release_add(counter, 1u);
 
         for (int t = 0; t < p.T; ++t) {
             // the input projection does not depend on h: fetch it while the recurrent product runs
@@ -134,8 +145,8 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
             tc::tmem_ld_32x32(taddr + 32, d1);
             tc::tmem_ld_wait();
             tc::tc_fence_before_sync();
+            float hn[UNITS];
             if (live) {
-                float hn[UNITS];
 #pragma unroll
                 for (int i = 0; i < UNITS; ++i) {
                     const float zi = __uint_as_float(d0[i]) + zx[0][i];
@@ -146,9 +157,7 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
                     c[i] = cn;
                     hn[i] = fast_sigmoid(zo) * fast_tanh(cn);
                 }
-                float4 *ho = reinterpret_cast<float4 *>(p.h_all + ((size_t)t * p.B + b) * p.H + j0);
-#pragma unroll
-                for (int i = 0; i < UNITS; i += 4) ho[i / 4] = make_float4(hn[i], hn[i + 1], hn[i + 2], hn[i + 3]);
+                // publish bf16(h_t) first: it is what the other blocks wait for
                 uint4 *hq = reinterpret_cast<uint4 *>(p.hq + ((size_t)((t + 1) & 1) * p.B + b) * p.H + j0);
                 hq[0] = make_uint4(pack2(hn[0], hn[1]), pack2(hn[2], hn[3]), pack2(hn[4], hn[5]), pack2(hn[6], hn[7]));
                 hq[1] = make_uint4(pack2(hn[8], hn[9]), pack2(hn[10], hn[11]), pack2(hn[12], hn[13]), pack2(hn[14], hn[15]));
@@ -156,17 +165,23 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
             asm volatile("fence.proxy.async.global;" ::: "memory");
             __threadfence();
             __syncwarp();
-            if (lane == 0) red_release_add(p.counter, 1u);
+            if (lane == 0) red_release_add(counter, 1u);
+            if (live) {   // the fp32 copy for the caller is off the critical path
+                float4 *ho = reinterpret_cast<float4 *>(p.h_all + ((size_t)t * p.B + b) * p.H + j0);
+#pragma unroll
+                for (int i = 0; i < UNITS; i += 4) ho[i / 4] = make_float4(hn[i], hn[i + 1], hn[i + 2], hn[i + 3]);
+            }
         }
         if (live) {
 #pragma unroll
             for (int i = 0; i < UNITS; ++i) p.c_final[(size_t)b * p.H + j0 + i] = c[i];
         }
+      }
     } else if (warp == 4) {
         // ------------------------------ W slice load + MMA issue ------------------------------
         if (lane == 0) {
             tc::mbar_expect_tx(w_full, (uint32_t)(p.k_blocks * W_KB));
-            for (int kb = 0; kb < p.k_blocks; ++kb) tc::tma_load_2d(w_s + (size_t)kb * W_KB, &tm_w, w_full, kb * BK, blockIdx.x * NCOL);
+            for (int kb = 0; kb < p.k_blocks; ++kb) tc::tma_load_2d(w_s + (size_t)kb * W_KB, &tm_w, w_full, kb * BK, blk * NCOL);
             bool ok = tc::mbar_wait(w_full, 0, abort_flag, p.err, tc::ERR_WAIT_FULL);
             const uint32_t idesc = tc::instr_desc_bf16(128, NCOL, false, false);
             uint32_t it = 0;
@@ -192,10 +207,10 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
             bool ok = true;
             for (int t = 0; t < p.T && ok; ++t) {
                 // grid barrier: every block has published its part of h_{t-1}
-                const unsigned int target = 4u * (unsigned int)p.n_blocks * (unsigned int)(t + 1);   // 4 epilogue warps per block
+                const unsigned int target = (unsigned int)(p.n_epi * p.n_blocks) * (unsigned int)(t + 1);   // n_epi arrivals per block
                 const long long t0 = clock64();
                 unsigned spins = 0;
-                while (ld_acquire(p.counter) < target) {
+                while (ld_acquire(counter) < target) {
                     if ((++spins & 255u) == 0 && (*abort_flag || clock64() - t0 > tc::kWaitLimitCycles)) {
                         if (!*abort_flag) { *abort_flag = 1; atomicCAS(p.err, 0, tc::ERR_WAIT_STEP); }
                         ok = false;
@@ -208,8 +223,8 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
                     const int s = it % STAGES;
                     if (!tc::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
-                    tc::mbar_expect_tx(&full[s], (uint32_t)(p.B * 128));
-                    tc::tma_load_2d(a_s + (size_t)s * A_STAGE, tm_h, &full[s], kb * BK, 0);   // rows 0..B-1; the rest stay zero
+                    tc::mbar_expect_tx(&full[s], (uint32_t)(p.rows_per_group * 128));
+                    tc::tma_load_2d(a_s + (size_t)s * A_STAGE, tm_h, &full[s], kb * BK, b_lo);   // the group's rows; the rest stay zero
                 }
             }
         }
@@ -250,7 +265,7 @@ bool lstm_tc_eligible(int64_t T, int64_t B, int64_t H)
 
 size_t lstm_tc_workspace(int64_t B, int64_t H)
 {
-    return align_up((size_t)H * 4 * H * 2, 1024) /* packed W_hh */ + align_up((size_t)2 * B * H * 2, 1024) /* exchange */ + 1024 /* counter */;
+    return align_up((size_t)H * 4 * H * 2, 1024) /* packed W_hh */ + align_up((size_t)2 * B * H * 2, 1024) /* exchange */ + 1024 /* counters */;
 }
 
 relay_status_t launch_lstm_tc(int64_t T, int64_t B, int64_t H, const float *zx, const void *w_hh, const float *h0, const float *c0,
@@ -266,17 +281,25 @@ relay_status_t launch_lstm_tc(int64_t T, int64_t B, int64_t H, const float *zx, 
     RELAY_CUDA(cudaMemsetAsync(counter, 0, 1024, st));
     CUtensorMap tm_w, tm_h0, tm_h1;
     RELAY_TRY(make_tmap_2d_bf16(&tm_w, wp, (uint64_t)H, (uint64_t)n_blocks * NCOL, (uint64_t)H, BK, NCOL));
-    RELAY_TRY(make_tmap_2d_bf16(&tm_h0, hq, (uint64_t)H, (uint64_t)B, (uint64_t)H, BK, (uint32_t)B));
-    RELAY_TRY(make_tmap_2d_bf16(&tm_h1, hq + (size_t)B * H, (uint64_t)H, (uint64_t)B, (uint64_t)H, BK, (uint32_t)B));
+    // split the batch into groups of rows while every block still fits on its own SM (at least 8 rows a group)
+    int dev = 0, sms = 148;
+    RELAY_CUDA(cudaGetDevice(&dev));
+    RELAY_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    int groups = std::max(1, std::min({sms / n_blocks, (int)(B / 8), 8}));
+    const int rows_per_group = (int)((B + groups - 1) / groups);
+    groups = (int)((B + rows_per_group - 1) / rows_per_group);
+    RELAY_TRY(make_tmap_2d_bf16(&tm_h0, hq, (uint64_t)H, (uint64_t)B, (uint64_t)H, BK, (uint32_t)rows_per_group));
+    RELAY_TRY(make_tmap_2d_bf16(&tm_h1, hq + (size_t)B * H, (uint64_t)H, (uint64_t)B, (uint64_t)H, BK, (uint32_t)rows_per_group));
     Params p{};
     p.T = (int)T; p.B = (int)B; p.H = (int)H; p.n_blocks = n_blocks; p.k_blocks = (int)(H / BK);
+    p.rows_per_group = rows_per_group; p.n_epi = (rows_per_group + 31) / 32;
     p.zx = zx; p.h0 = h0; p.c0 = c0; p.h_all = h_all; p.c_final = c_final; p.hq = hq; p.counter = counter;
     p.err = device_error_word();
     if (!p.err) return fail(RELAY_ERR_CUDA, "no device error word");
     const size_t smem = 1024 + (size_t)p.k_blocks * W_KB + (size_t)STAGES * A_STAGE + 256;
     RELAY_CUDA(cudaFuncSetAttribute(lstm_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     void *args[] = {(void *)&tm_w, (void *)&tm_h0, (void *)&tm_h1, (void *)&p};
-    RELAY_CUDA(cudaLaunchCooperativeKernel((const void *)lstm_persistent_kernel, dim3(n_blocks), dim3(NUM_THREADS), args, smem, st));
+    RELAY_CUDA(cudaLaunchCooperativeKernel((const void *)lstm_persistent_kernel, dim3(n_blocks * groups), dim3(NUM_THREADS), args, smem, st));
     count_launch();
     return RELAY_OK;
 }
