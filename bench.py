@@ -316,6 +316,19 @@ def run_reference(args, rank, world):
     print(json.dumps(line))
 
 
+def max_over_ranks(value_ms: float, dist, device) -> float:
+    """Multi-GPU numbers are the MAX over ranks of the device time (replicas run independently)."""
+    t = torch.tensor([value_ms], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job(per_rank_units: float, world: int, ms: float) -> float:
+    """Weak scaling: every replica processes `per_rank_units` in `ms` (max over ranks)."""
+    return world * per_rank_units / (ms * 1e-3) if ms else 0.0
+
+
 # ---------------------------------------------------------------------------------------------------
 def main():
     ap = argparse.ArgumentParser()
@@ -378,17 +391,14 @@ def main():
     top = [k for k in tm.ms if k.count(".") == 1]
     med = {k: float(np.median(v)) for k, v in tm.ms.items()}
     step_ms = sum(float(np.mean(tm.ms[k])) for k in top)
-    step_ms_t = torch.tensor([step_ms], device=dev)
-    if dist is not None:
-        dist.all_reduce(step_ms_t, op=dist.ReduceOp.MAX)
-    step_ms_max = float(step_ms_t.item())
+    step_ms_max = max_over_ranks(step_ms, dist, dev)
 
     tensor_keys = [k for k in top if k.startswith(("cfg3", "cfg4"))]
     hbm_keys = [k for k in top if k.startswith("cfg2")]
-    t_ms = sum(float(np.mean(tm.ms[k])) for k in tensor_keys)
-    h_ms = sum(float(np.mean(tm.ms[k])) for k in hbm_keys)
-    tflops = world * sum(work[k]["flop"] for k in tensor_keys) / (t_ms * 1e-3) / 1e12 if t_ms else None
-    gbs = world * sum(work[k]["bytes"] for k in hbm_keys) / (h_ms * 1e-3) / 1e9 if h_ms else None
+    t_ms = max_over_ranks(sum(float(np.mean(tm.ms[k])) for k in tensor_keys), dist, dev)
+    h_ms = max_over_ranks(sum(float(np.mean(tm.ms[k])) for k in hbm_keys), dist, dev)
+    tflops = whole_job(sum(work[k]["flop"] for k in tensor_keys), world, t_ms) / 1e12 if t_ms else None
+    gbs = whole_job(sum(work[k]["bytes"] for k in hbm_keys), world, h_ms) / 1e9 if h_ms else None
 
     table = {}
     for k in sorted(tm.ms):
@@ -449,11 +459,7 @@ def main():
             h2d = wl.upload(); wl.step(tm2); d2h = wl.download()
         b.record()
         barrier()
-        e_ms = a.elapsed_time(b) / n_e2e
-        et = torch.tensor([e_ms], device=dev)
-        if dist is not None:
-            dist.all_reduce(et, op=dist.ReduceOp.MAX)
-        e_ms = float(et.item())
+        e_ms = max_over_ranks(a.elapsed_time(b) / n_e2e, dist, dev)
         flop_all = sum(work[k]["flop"] for k in tensor_keys)
         e2e = {"value": world * flop_all / (e_ms * 1e-3) / 1e12 if flop_all else None, "unit": "TFLOP/s", "ms_per_step": e_ms,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

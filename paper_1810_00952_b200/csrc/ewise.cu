@@ -126,26 +126,27 @@ __global__ void __launch_bounds__(kTX *kTY, Body::NIN >= 4 ? 2 : 3) ewise2d_kern
     }
 }
 
-// second pass of a column sum: thread (tx, ty) adds the partials of slices ty, ty+32, ... of its column in
-// slice order, then the 32 row-threads are combined in ty order (fixed order, so reruns are bit-identical).
+// second pass of a column sum: thread (tx, ty) adds the partials of slices ty, ty+TY, ... of its column in
+// slice order, then the TY row-threads are combined in ty order (fixed order, so reruns are bit-identical).
 // grid.y indexes the summed result k: partials at partial + k * n_slices * cols, output out[k].
 struct FinalizeOuts { float *out[RELAY_MAX_OUTPUTS]; };
-__global__ void __launch_bounds__(1024) colsum_finalize_kernel(const float *__restrict__ partial, int n_slices, int64_t cols, float scale,
-                                                                const FinalizeOuts outs)
+template <int TY>
+__global__ void __launch_bounds__(32 * TY) colsum_finalize_kernel(const float *__restrict__ partial, int n_slices, int64_t cols, float scale,
+                                                                  const FinalizeOuts outs)
 {
-    __shared__ float sm[32][33];
+    __shared__ float sm[TY][33];
     const int tx = threadIdx.x, ty = threadIdx.y;
     const int64_t c = (int64_t)blockIdx.x * 32 + tx;
     const float *p = partial + (size_t)blockIdx.y * n_slices * cols;
     float s = 0.0f;
     if (c < cols)
-        for (int j = ty; j < n_slices; j += 32) s += p[(int64_t)j * cols + c];
+        for (int j = ty; j < n_slices; j += TY) s += p[(int64_t)j * cols + c];
     sm[ty][tx] = s;
     __syncthreads();
     if (ty == 0 && c < cols) {
         float t = 0.0f;
 #pragma unroll
-        for (int j = 0; j < 32; ++j) t += sm[j][tx];
+        for (int j = 0; j < TY; ++j) t += sm[j][tx];
         outs.out[blockIdx.y][c] = t * scale;
     }
 }
@@ -446,7 +447,9 @@ relay_status_t launch_colsum_finalize_n(const float *partial, int n_slices, int6
 {
     FinalizeOuts fo{};
     for (int k = 0; k < n_out; ++k) fo.out[k] = out[k];
-    colsum_finalize_kernel<<<dim3((unsigned)((cols + 31) / 32), (unsigned)n_out), dim3(32, 32), 0, st>>>(partial, n_slices, cols, scale, fo);
+    const dim3 grid((unsigned)((cols + 31) / 32), (unsigned)n_out);
+    if (n_slices > 64) colsum_finalize_kernel<32><<<grid, dim3(32, 32), 0, st>>>(partial, n_slices, cols, scale, fo);
+    else colsum_finalize_kernel<8><<<grid, dim3(32, 8), 0, st>>>(partial, n_slices, cols, scale, fo);
     return check_launch("colsum_finalize");
 }
 
