@@ -26,5 +26,8 @@ relay_status_t launch_gemm(const GemmDesc &g, cudaStream_t st);
 relay_status_t launch_gemm_simt(const GemmDesc &g, cudaStream_t st);
 bool gemm_tc_eligible(const GemmDesc &g);
 relay_status_t launch_gemm_tc(const GemmDesc &g, cudaStream_t st);
+// two-SM (cta_group::2) variant: 256 x 256 tiles computed by pairs of blocks
+bool gemm_tc2_eligible(const GemmDesc &g, int sms);
+relay_status_t launch_gemm_tc2(const GemmDesc &g, int sms, cudaStream_t st);
 
 }  // namespace relay
