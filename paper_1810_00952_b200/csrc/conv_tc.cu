@@ -118,18 +118,16 @@ __global__ void pack_weights_kernel(const __nv_bfloat16 *__restrict__ w, __nv_bf
     }
 }
 
-// dw[o][c][tap] = bf16( sum over slices, in slice order, of part[slice][tap][o][c] ); one thread per (o, c)
-// so that the partial reads coalesce along c
+// dw[o][c][tap] = bf16( sum over slices, in slice order, of part[slice][tap][o][c] ); one thread per
+// (tap, o, c) with (o, c) fastest so that the partial reads coalesce (the 2-byte stores scatter, 1.2 MB)
 __global__ void wgrad_reduce_kernel(const float *__restrict__ part, int n_slices, __nv_bfloat16 *__restrict__ dw, int O, int C, int taps)
 {
-    const unsigned oc_total = (unsigned)O * C;
-    const size_t per_slice = (size_t)taps * oc_total;
-    for (unsigned oc = blockIdx.x * blockDim.x + threadIdx.x; oc < oc_total; oc += gridDim.x * blockDim.x) {
-        for (int tap = 0; tap < taps; ++tap) {
-            float s = 0.0f;
-            for (int j = 0; j < n_slices; ++j) s += part[(size_t)j * per_slice + (size_t)tap * oc_total + oc];
-            dw[(size_t)oc * taps + tap] = __float2bfloat16_rn(s);
-        }
+    const unsigned oc_total = (unsigned)O * C, total = oc_total * (unsigned)taps;
+    for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+        const unsigned tap = i / oc_total, oc = i - tap * oc_total;
+        float s = 0.0f;
+        for (int j = 0; j < n_slices; ++j) s += part[(size_t)j * total + i];
+        dw[(size_t)oc * taps + tap] = __float2bfloat16_rn(s);
     }
 }
 
@@ -657,7 +655,7 @@ relay_status_t launch_conv_grad_tc(const ConvDims &d, const void *x, const void 
     const int grid = 9 * p.m_tiles * p.c_tiles * p.n_slices;
     conv_wgrad_tc_kernel<<<grid, NUM_THREADS, smem, st>>>(tm_dz, tm_x, tm_part, p);
     RELAY_TRY(check_launch("conv_wgrad_tc"));
-    wgrad_reduce_kernel<<<(unsigned)((d.O * d.C + 127) / 128), 128, 0, st>>>(part, p.n_slices, (__nv_bfloat16 *)dw,
+    wgrad_reduce_kernel<<<(unsigned)((9 * d.O * d.C + 255) / 256), 256, 0, st>>>(part, p.n_slices, (__nv_bfloat16 *)dw,
                                                                                                           (int)d.O, (int)d.C, 9);
     return check_launch("wgrad_reduce");
 }

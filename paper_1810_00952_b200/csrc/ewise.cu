@@ -448,7 +448,7 @@ relay_status_t launch_colsum_finalize_n(const float *partial, int n_slices, int6
     FinalizeOuts fo{};
     for (int k = 0; k < n_out; ++k) fo.out[k] = out[k];
     const dim3 grid((unsigned)((cols + 31) / 32), (unsigned)n_out);
-    if (n_slices > 64) colsum_finalize_kernel<32><<<grid, dim3(32, 32), 0, st>>>(partial, n_slices, cols, scale, fo);
+    if (n_slices > 256) colsum_finalize_kernel<32><<<grid, dim3(32, 32), 0, st>>>(partial, n_slices, cols, scale, fo);
     else colsum_finalize_kernel<8><<<grid, dim3(32, 8), 0, st>>>(partial, n_slices, cols, scale, fo);
     return check_launch("colsum_finalize");
 }
