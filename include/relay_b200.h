@@ -291,6 +291,13 @@ const char *relay_last_error(void);
  * RELAY_ERR_CUDA if the stream reports an error, else RELAY_OK. */
 relay_status_t relay_poll_status(void *stream);
 
+/* Self-test of the time-out path (no counterpart in the paper): enqueues a one-block kernel that
+ * waits, for at most `limit_us` microseconds (1..1000000), on a hardware barrier that nothing ever
+ * signals, then gives up, records the time-out in the device error word and exits normally.  The next
+ * relay_poll_status() therefore returns RELAY_ERR_TIMEOUT and clears the word; the context stays usable.
+ * It shows a caller that an expired wait in any kernel of this library is reported rather than hung on. */
+relay_status_t relay_debug_expire_wait(int32_t limit_us, void *stream);
+
 /* Number of kernels this library has launched on this process so far (monotonic counter). */
 int64_t relay_launch_count(void);
 

@@ -306,6 +306,10 @@ def relay_poll_status():
     _check(lib().relay_poll_status(_stream()))
 
 
+def relay_debug_expire_wait(limit_us: int = 1000):
+    _check(lib().relay_debug_expire_wait(int(limit_us), _stream()))
+
+
 def relay_launch_count() -> int:
     return int(lib().relay_launch_count())
 

@@ -6,6 +6,7 @@
 
 #include "common.h"
 #include "ewise_prog.h"
+#include "tc_common.cuh"
 
 namespace relay {
 
@@ -136,6 +137,20 @@ int *device_error_word()
     return addr[dev];
 }
 
+// waits on a barrier that nobody signals, for at most limit_cycles, then reports the time-out
+__global__ void expire_wait_kernel(long long limit_cycles, int *err)
+{
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        tc::mbar_init(&bar, 1);
+        tc::fence_barrier_init();
+        const long long t0 = clock64();
+        bool done = false;
+        while (!(done = tc::mbar_try_wait(&bar, 0)) && clock64() - t0 < limit_cycles) {}
+        if (!done) atomicCAS(err, 0, tc::ERR_WAIT_STEP);
+    }
+}
+
 static void fill_out(relay_tensor_t *out, int32_t dtype, int32_t layout, int rank, const int64_t *shape)
 {
     std::memset(out, 0, sizeof(*out));
@@ -171,6 +186,19 @@ relay_status_t relay_poll_status(void *stream)
         return fail(RELAY_ERR_TIMEOUT, "a bounded device-side wait expired (code %d)", v);
     }
     return RELAY_OK;
+}
+
+relay_status_t relay_debug_expire_wait(int32_t limit_us, void *stream)
+{
+    clear_error();
+    if (limit_us < 1 || limit_us > 1000000) return fail(RELAY_ERR_ATTR, "limit_us = %d outside [1, 1000000]", limit_us);
+    int *w = device_error_word();
+    if (!w) return fail(RELAY_ERR_CUDA, "no device error word (no CUDA device?)");
+    int dev = 0, khz = 0;
+    RELAY_CUDA(cudaGetDevice(&dev));
+    RELAY_CUDA(cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, dev));
+    expire_wait_kernel<<<1, 32, 0, (cudaStream_t)stream>>>((long long)limit_us * (khz / 1000), w);
+    return check_launch("expire_wait");
 }
 
 relay_status_t relay_infer_dense(const relay_tensor_t *x, const relay_tensor_t *w, relay_tensor_t *out)
