@@ -464,6 +464,133 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_dz, const __grid_con
 }
 
 // ---------------------------------------------------------------------------------------------------
+// wgrad kernel, two-SM form: a pair of blocks owns (tap, 256 output channels, 256 input channels, batch
+// slice).  Each block loads its 128 output channels of dZ and its 128 input channels of x per k-block
+// (56 KB instead of 84 KB) and the pair's MMA (cta_group::2, M = 256) reads both halves.
+// ---------------------------------------------------------------------------------------------------
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
+conv_wgrad_tc2_kernel(const __grid_constant__ CUtensorMap tm_dz, const __grid_constant__ CUtensorMap tm_x,
+                      const __grid_constant__ CUtensorMap tm_part, const WgradParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int box_bytes = p.kpix * 128;
+    const int a_bytes = 2 * box_bytes, stage_bytes = 4 * box_bytes;      // 128 o + 128 c per block
+    const int STAGES = p.stages;
+    uint8_t *staging = smem + (size_t)STAGES * stage_bytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(staging + 4 * 8192);
+    uint64_t *full = bars, *empty = bars + STAGES, *tmem_full = bars + 2 * STAGES;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 2);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = tc::cluster_ctarank();
+
+    int u = blockIdx.x >> 1;                           // unit of the pair
+    const int slice = u % p.n_slices; u /= p.n_slices;
+    const int ct = u % p.c_tiles; u /= p.c_tiles;
+    const int mt = u % p.m_tiles; u /= p.m_tiles;      // m_tiles counts 256-channel tiles here
+    const int tap = u;
+    const int r = tap / p.taps_s, sft = tap % p.taps_s;
+    const int img0 = slice * p.imgs_per_slice, img1 = min(p.Nb, img0 + p.imgs_per_slice);
+    const int kb_per_img = p.H / p.rows_per_kblock;
+    const int k_blocks = max(0, img1 - img0) * kb_per_img;
+    const int o0 = mt * 256 + (int)rank * 128, c0 = ct * 256 + (int)rank * 128;   // this block's halves
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
+        tc::mbar_init(&tmem_full[0], 1);
+        *abort_flag = 0;
+        tc::fence_barrier_init();
+        tc::prefetch_tmap(&tm_dz);
+        tc::prefetch_tmap(&tm_x);
+        tc::prefetch_tmap(&tm_part);
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc::smem_u32(tmem_slot)), "r"(256) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc::tc_fence_before_sync();
+    __syncthreads();
+    tc::cluster_sync();
+    tc::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int s = 0;
+            uint32_t phase = 0;
+            for (int kb = 0; kb < k_blocks; ++kb) {
+                if (!tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) break;
+                uint8_t *sa = smem + (size_t)s * stage_bytes, *sb = sa + a_bytes;
+                const uint32_t bar = tc::mapa(tc::smem_u32(&full[s]), 0);
+                if (rank == 0) tc::mbar_expect_tx_cluster(bar, 2 * stage_bytes);
+                const int img = img0 + kb / kb_per_img, h0 = (kb % kb_per_img) * p.rows_per_kblock;
+#pragma unroll
+                for (int i = 0; i < 2; ++i) tc::tma_load_4d_pair(sa + i * box_bytes, &tm_dz, bar, o0 + i * 64, 0, h0, img);
+#pragma unroll
+                for (int j = 0; j < 2; ++j) tc::tma_load_4d_pair(sb + j * box_bytes, &tm_x, bar, c0 + j * 64, sft - p.pad, h0 + r - p.pad, img);
+                if (++s == STAGES) { s = 0; phase ^= 1; }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = tc::instr_desc_bf16(256, 256, true, true);
+            int s = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int kb = 0; kb < k_blocks; ++kb) {
+                if (!tc::mbar_wait(&full[s], phase, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
+                tc::tc_fence_after_sync();
+                const uint32_t sa = tc::smem_u32(smem + (size_t)s * stage_bytes), sb = sa + a_bytes;
+                const uint64_t da = tc::smem_desc(sa, box_bytes, 1024), db = tc::smem_desc(sb, box_bytes, 1024);
+                const uint32_t acc = kb != 0;
+                for (int kk = 0; kk < p.kpix / 16; ++kk) tc::mma_bf16_pair(tmem_base, da + kk * 128, db + kk * 128, idesc, acc | (kk != 0));
+                tc::mma_commit_pair(&empty[s]);
+                if (++s == STAGES) { s = 0; phase ^= 1; }
+            }
+            if (ok) tc::mma_commit_pair(&tmem_full[0]);
+        }
+    } else {
+        const int quarter = warp & 3;
+        int ok = 1;
+        if (k_blocks > 0) {
+            if (lane == 0) ok = tc::mbar_wait(&tmem_full[0], 0, abort_flag, p.err, tc::ERR_WAIT_TMEM_FULL) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+        }
+        if (ok) {
+            tc::tc_fence_after_sync();
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+            uint8_t *my_stage = staging + (size_t)(warp - 2) * 8192;
+            const int row0 = (slice * (p.taps_r * p.taps_s) + tap) * p.O + o0 + quarter * 32;
+            const int col0 = ct * 256;                  // the accumulator row holds all 256 input channels of the tile
+#pragma unroll 1
+            for (int c = 0; c < 256 / 32; ++c) {
+                uint32_t v[32];
+                if (k_blocks > 0) {
+                    tc::tmem_ld_32x32(taddr + c * 32, v);
+                    tc::tmem_ld_wait();
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = 0u;
+                }
+                uint4 piece[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) piece[q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                tc::warp_store_block<1>(&tm_part, my_stage + (c & 1) * 4096, piece, lane, col0 + c * 32, row0);
+            }
+            if (lane == 0) tc::tma_store_wait_all<0>();
+        }
+    }
+    tc::tc_fence_before_sync();
+    __syncthreads();
+    tc::cluster_sync();
+    if (warp == 1) {
+        tc::tc_fence_after_sync();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
 // host plans
 // ---------------------------------------------------------------------------------------------------
 struct TcPlan {
@@ -471,6 +598,7 @@ struct TcPlan {
     int rows_per_tile = 0;   // fprop: image rows per tile (rows*W <= 256, multiple of 32)
     int rows_per_kblock = 0; // wgrad: image rows per k-block (rows*W multiple of 16, <= 128)
     int wg_nt = 0, wg_c_tiles = 0, wg_m_tiles = 0, wg_slices = 0, wg_imgs_per_slice = 0, wg_stages = 0;
+    bool wg_pair = false;    // two-SM wgrad: units of 256 output x 256 input channels computed by pairs of blocks
     int fp_stages = 0;
     size_t x_nhwc = 0, dz_nhwc = 0, wpack = 0, part = 0, db_part = 0;
 };
@@ -502,8 +630,18 @@ TcPlan plan(const ConvDims &d)
     pl.wg_stages = (int)std::min<size_t>(4, (kSmemLimit - wg_fixed) / wg_stage(pl.wg_nt));
     pl.wg_c_tiles = (int)(d.C / pl.wg_nt);
     pl.wg_m_tiles = (int)(d.O / BM);
+    int workers = 148;
+    const size_t pair_stage = 4 * box;
+    if (d.O % 256 == 0 && d.C % 256 == 0 && (kSmemLimit - wg_fixed) / pair_stage >= 2) {
+        pl.wg_pair = true;
+        pl.wg_nt = 256;
+        pl.wg_c_tiles = (int)(d.C / 256);
+        pl.wg_m_tiles = (int)(d.O / 256);
+        pl.wg_stages = (int)std::min<size_t>(4, (kSmemLimit - wg_fixed) / pair_stage);
+        workers = 74;
+    }
     const int base_units = 9 * pl.wg_m_tiles * pl.wg_c_tiles;
-    int slices = std::max(1, 148 / base_units);
+    int slices = std::max(1, workers / base_units);
     slices = (int)std::min<int64_t>(slices, d.Nb);
     pl.wg_imgs_per_slice = (int)((d.Nb + slices - 1) / slices);
     pl.wg_slices = (int)((d.Nb + pl.wg_imgs_per_slice - 1) / pl.wg_imgs_per_slice);
@@ -649,11 +787,17 @@ relay_status_t launch_conv_grad_tc(const ConvDims &d, const void *x, const void 
     if (!p.err) return fail(RELAY_ERR_CUDA, "no device error word");
     const size_t stage = (size_t)(BM / 64 + p.nt / 64) * p.kpix * 128;
     const size_t smem = 1024 + (size_t)p.stages * stage + 4 * 8192 + 256;
-    RELAY_CUDA(cudaFuncSetAttribute(conv_wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     CUtensorMap tm_part;
     RELAY_TRY(make_tmap_2d(&tm_part, true, part, (uint64_t)d.C, (uint64_t)p.n_slices * 9 * d.O, (uint64_t)d.C, 32, 32, true));
     const int grid = 9 * p.m_tiles * p.c_tiles * p.n_slices;
-    conv_wgrad_tc_kernel<<<grid, NUM_THREADS, smem, st>>>(tm_dz, tm_x, tm_part, p);
+    if (pl.wg_pair) {
+        const size_t smem2 = 1024 + (size_t)p.stages * 4 * p.kpix * 128 + 4 * 8192 + 256;
+        RELAY_CUDA(cudaFuncSetAttribute(conv_wgrad_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2));
+        conv_wgrad_tc2_kernel<<<2 * grid, NUM_THREADS, smem2, st>>>(tm_dz, tm_x, tm_part, p);
+    } else {
+        RELAY_CUDA(cudaFuncSetAttribute(conv_wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        conv_wgrad_tc_kernel<<<grid, NUM_THREADS, smem, st>>>(tm_dz, tm_x, tm_part, p);
+    }
     RELAY_TRY(check_launch("conv_wgrad_tc"));
     wgrad_reduce_kernel<<<(unsigned)((9 * d.O * d.C + 255) / 256), 256, 0, st>>>(part, p.n_slices, (__nv_bfloat16 *)dw,
                                                                                                           (int)d.O, (int)d.C, 9);

@@ -35,53 +35,6 @@ constexpr int NUM_THREADS = 192;
 constexpr int STAGING_BYTES = 4 * 2 * 4096;
 constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * STAGE_BYTES + STAGING_BYTES + 256;
 
-__device__ __forceinline__ uint32_t cluster_ctarank()
-{
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ uint32_t mapa(uint32_t smem_addr, uint32_t rank)
-{
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ void cluster_sync()
-{
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t bar_cluster_addr, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(bar_cluster_addr), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr)
-{
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
-}
-// tile load whose completion is posted on a barrier that may live in the peer block of the pair
-__device__ __forceinline__ void tma_load_2d_pair(void *dst, const CUtensorMap *m, uint32_t bar_cluster_addr, int x, int y)
-{
-    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                 ::"r"(tc::smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster_addr), "r"(x), "r"(y)
-                 : "memory");
-}
-__device__ __forceinline__ void mma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}\n" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc),
-        "r"(accumulate)
-        : "memory");
-}
-// arrives on the barrier at this shared-memory offset in BOTH blocks once the pair's MMAs so far are done
-__device__ __forceinline__ void mma_commit_pair(uint64_t *bar)
-{
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(tc::smem_u32(bar)), "h"((uint16_t)3)
-                 : "memory");
-}
-
 template <bool A_MN, bool B_MN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
@@ -96,7 +49,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t rank = cluster_ctarank();          // 0 = leader
+    const uint32_t rank = tc::cluster_ctarank();          // 0 = leader
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     const int n_tiles = p.tiles_m * p.tiles_n;        // tiles of 256 x 256
 
@@ -115,7 +68,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     }
     tc::tc_fence_before_sync();
     __syncthreads();
-    cluster_sync();                                   // the peer's barriers are initialised before anyone signals them
+    tc::cluster_sync();                                   // the peer's barriers are initialised before anyone signals them
     tc::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
@@ -131,20 +84,20 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
                     if (!tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
                     uint8_t *sa = smem + (size_t)s * STAGE_BYTES, *sb = sa + A_BYTES;
-                    const uint32_t bar = mapa(tc::smem_u32(&full[s]), 0);       // the leader's barrier
-                    if (rank == 0) mbar_expect_tx_cluster(bar, 2 * STAGE_BYTES); // bytes of both blocks
+                    const uint32_t bar = tc::mapa(tc::smem_u32(&full[s]), 0);       // the leader's barrier
+                    if (rank == 0) tc::mbar_expect_tx_cluster(bar, 2 * STAGE_BYTES); // bytes of both blocks
                     const int k0 = kb * BK;
                     if (A_MN) {
 #pragma unroll
-                        for (int i = 0; i < 2; ++i) tma_load_2d_pair(sa + i * MN_BOX_BYTES, &tm_a, bar, m0 + i * 64, k0);
+                        for (int i = 0; i < 2; ++i) tc::tma_load_2d_pair(sa + i * MN_BOX_BYTES, &tm_a, bar, m0 + i * 64, k0);
                     } else {
-                        tma_load_2d_pair(sa, &tm_a, bar, k0, m0);
+                        tc::tma_load_2d_pair(sa, &tm_a, bar, k0, m0);
                     }
                     if (B_MN) {
 #pragma unroll
-                        for (int i = 0; i < 2; ++i) tma_load_2d_pair(sb + i * MN_BOX_BYTES, &tm_b, bar, n0 + i * 64, k0);
+                        for (int i = 0; i < 2; ++i) tc::tma_load_2d_pair(sb + i * MN_BOX_BYTES, &tm_b, bar, n0 + i * 64, k0);
                     } else {
-                        tma_load_2d_pair(sb, &tm_b, bar, k0, n0);
+                        tc::tma_load_2d_pair(sb, &tm_b, bar, k0, n0);
                     }
                     if (++s == STAGES) { s = 0; phase ^= 1; }
                 }
@@ -173,12 +126,12 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                     const uint32_t acc = kb != 0;
 #pragma unroll
                     for (int kk = 0; kk < BK / 16; ++kk)
-                        mma_bf16_pair(d_tmem, da + ((kk * a_step) >> 4), db + ((kk * b_step) >> 4), idesc, acc | (kk != 0));
-                    mma_commit_pair(&empty[s]);
+                        tc::mma_bf16_pair(d_tmem, da + ((kk * a_step) >> 4), db + ((kk * b_step) >> 4), idesc, acc | (kk != 0));
+                    tc::mma_commit_pair(&empty[s]);
                     stage_off += STAGE_BYTES >> 4;
                     if (++s == STAGES) { s = 0; phase ^= 1; stage_off = 0; }
                 }
-                if (ok) mma_commit_pair(&tmem_full[buf]);
+                if (ok) tc::mma_commit_pair(&tmem_full[buf]);
             }
         }
     } else {
@@ -202,14 +155,14 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             }
             tc::tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(mapa(tc::smem_u32(&tmem_empty[buf]), 0));
+            if (lane == 0) tc::mbar_arrive_cluster(tc::mapa(tc::smem_u32(&tmem_empty[buf]), 0));
         }
         if (lane == 0) tc::tma_store_wait_all<0>();
     }
 
     tc::tc_fence_before_sync();
     __syncthreads();
-    cluster_sync();                                   // neither block leaves while the other may still signal it
+    tc::cluster_sync();                                   // neither block leaves while the other may still signal it
     if (warp == 1) {
         tc::tc_fence_after_sync();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");

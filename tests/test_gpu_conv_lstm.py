@@ -53,7 +53,8 @@ def test_conv_small_shapes_forward_and_gradient(N, C, H, W, O, R, stride, pad, t
     (assert_f32 if tdt == torch.float32 else (lambda g, o, what: assert_bf16(g, o, stored_bf16=False, what=what)))(db, odb, what="db")
 
 
-@pytest.mark.parametrize("N,C,H,W,O", [(2, 64, 28, 28, 64), (2, 128, 16, 16, 128), (3, 128, 12, 24, 256), (1, 128, 56, 56, 128)])
+@pytest.mark.parametrize("N,C,H,W,O", [(2, 64, 28, 28, 64), (2, 128, 16, 16, 128), (3, 128, 12, 24, 256), (1, 128, 56, 56, 128),
+                                       (3, 256, 16, 16, 256)])
 def test_conv_reduced_config_bf16_3x3(N, C, H, W, O):
     """Configuration 4's structure (3x3, stride 1, pad 1, NCHW/OIHW, bf16) at reduced sizes; the shapes
     with C and O multiples of 128 take the implicit-GEMM tensor-core kernels (several tiles, batch
