@@ -345,6 +345,173 @@ conv_fprop_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
 }
 
 // ---------------------------------------------------------------------------------------------------
+// fprop kernel, two-SM form: a pair of blocks computes 256 output channels x (rows_per_tile * W) pixels
+// with tcgen05.mma.cta_group::2.  Each block loads the packed weights of its 128 channels and HALF of the
+// activation tile (rows_per_tile / 2 image rows), 30 KB per k-block at cfg4, so six stages fit and the two
+// TMEM accumulators alternate between tiles (the epilogue overlaps the next main loop).
+// ---------------------------------------------------------------------------------------------------
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
+conv_fprop_tc2_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
+                      const __grid_constant__ CUtensorMap tm_y, const FpropParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    constexpr int a_bytes = BM * BK * 2;
+    const int bh_bytes = (p.nt / 2) * BK * 2;                       // this block's half of the activation tile
+    const int stage_bytes = a_bytes + ((bh_bytes + 1023) & ~1023);
+    const int STAGES = p.stages;
+    uint8_t *staging = smem + (size_t)STAGES * stage_bytes;         // [epilogue warp][2][2 KB]
+    uint64_t *bars = reinterpret_cast<uint64_t *>(staging + 4 * 4096);
+    uint64_t *full = bars, *empty = bars + STAGES, *tmem_full = bars + 2 * STAGES, *tmem_empty = bars + 2 * STAGES + 2;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 4);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = tc::cluster_ctarank();
+    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    const int cblocks = p.Cin / BK, half_rows = p.rows_per_tile / 2;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { tc::mbar_init(&tmem_full[b], 1); tc::mbar_init(&tmem_empty[b], 8); }
+        *abort_flag = 0;
+        tc::fence_barrier_init();
+        tc::prefetch_tmap(&tm_w);
+        tc::prefetch_tmap(&tm_x);
+        tc::prefetch_tmap(&tm_y);
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc::smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc::tc_fence_before_sync();
+    __syncthreads();
+    tc::cluster_sync();
+    tc::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int s = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int item = pair; item < p.n_items && ok; item += n_pairs) {
+                const int m0 = (item % p.pairs_per_ntile) * 256 + (int)rank * BM;
+                const int nt_idx = item / p.pairs_per_ntile;
+                const int img = nt_idx / p.tiles_per_img, h0 = (nt_idx % p.tiles_per_img) * p.rows_per_tile + (int)rank * half_rows;
+                int kb = 0;
+                for (int r = 0; r < p.taps_r && ok; ++r)
+                    for (int sft = 0; sft < p.taps_s && ok; ++sft)
+                        for (int cb = 0; cb < cblocks; ++cb, ++kb) {
+                            if (!tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
+                            uint8_t *sa = smem + (size_t)s * stage_bytes, *sb = sa + a_bytes;
+                            const uint32_t bar = tc::mapa(tc::smem_u32(&full[s]), 0);
+                            if (rank == 0) tc::mbar_expect_tx_cluster(bar, 2 * (a_bytes + bh_bytes));
+                            tc::tma_load_2d_pair(sa, &tm_w, bar, kb * BK, m0);
+                            tc::tma_load_4d_pair(sb, &tm_x, bar, cb * BK, sft - p.pad, h0 + r - p.pad, img);
+                            if (++s == STAGES) { s = 0; phase ^= 1; }
+                        }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = tc::instr_desc_bf16(256, p.nt, false, false);
+            const uint64_t desc_a0 = tc::smem_desc(tc::smem_u32(smem), 16, 1024), desc_b0 = tc::smem_desc(tc::smem_u32(smem) + a_bytes, 16, 1024);
+            uint32_t t_local = 0, phase = 0, stage_off = 0;
+            int s = 0;
+            bool ok = true;
+            for (int item = pair; item < p.n_items && ok; item += n_pairs, ++t_local) {
+                const int buf = t_local & 1;
+                if (!tc::mbar_wait(&tmem_empty[buf], ((t_local >> 1) & 1) ^ 1, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) break;
+                tc::tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + buf * 256;
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    if (!tc::mbar_wait(&full[s], phase, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
+                    tc::tc_fence_after_sync();
+                    const uint64_t da = desc_a0 + stage_off, db = desc_b0 + stage_off;
+                    const uint32_t acc = kb != 0;
+#pragma unroll
+                    for (int kk = 0; kk < BK / 16; ++kk) tc::mma_bf16_pair(d_tmem, da + kk * 2, db + kk * 2, idesc, acc | (kk != 0));
+                    tc::mma_commit_pair(&empty[s]);
+                    stage_off += (uint32_t)stage_bytes >> 4;
+                    if (++s == STAGES) { s = 0; phase ^= 1; stage_off = 0; }
+                }
+                if (ok) tc::mma_commit_pair(&tmem_full[buf]);
+            }
+        }
+    } else {
+        const int quarter = warp & 3;
+        uint8_t *my_stage = staging + (size_t)(warp - 2) * 4096;
+        uint32_t t_local = 0, blk_count = 0;
+        for (int item = pair; item < p.n_items; item += n_pairs, ++t_local) {
+            const int buf = t_local & 1;
+            const int m0 = (item % p.pairs_per_ntile) * 256 + (int)rank * BM;
+            const int nt_idx = item / p.pairs_per_ntile;
+            const int img = nt_idx / p.tiles_per_img, h0 = (nt_idx % p.tiles_per_img) * p.rows_per_tile;
+            int ok = 1;
+            if (lane == 0) ok = tc::mbar_wait(&tmem_full[buf], (t_local >> 1) & 1, abort_flag, p.err, tc::ERR_WAIT_TMEM_FULL) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            tc::tc_fence_after_sync();
+            const int o0 = m0 + quarter * 32;
+            const int o = o0 + lane;
+            float bias = 0.0f;
+            if (p.bias != nullptr && o < p.Cout)
+                bias = p.bias_bf16 ? __bfloat162float(((const __nv_bfloat16 *)p.bias)[o]) : ((const float *)p.bias)[o];
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * 256;
+#pragma unroll 1
+            for (int c = 0; c < p.nt / 32; ++c, ++blk_count) {
+                uint32_t r[32];
+                tc::tmem_ld_32x32(taddr + c * 32, r);
+                tc::tmem_ld_wait();
+                float v[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) + bias;
+                switch (p.act) {
+                case RELAY_ACT_RELU:
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.0f);
+                    break;
+                case RELAY_ACT_TANH:
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = tanh_<true>(v[j]);
+                    break;
+                case RELAY_ACT_SIGMOID:
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = sigmoid_<true>(v[j]);
+                    break;
+                default: break;
+                }
+                uint8_t *st = my_stage + (blk_count & 1) * 2048;
+                if (lane == 0) tc::tma_store_wait_read<1>();
+                __syncwarp();
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    *reinterpret_cast<uint4 *>(st + lane * 64 + q * 16) =
+                        make_uint4(pack2(v[8 * q], v[8 * q + 1]), pack2(v[8 * q + 2], v[8 * q + 3]), pack2(v[8 * q + 4], v[8 * q + 5]),
+                                   pack2(v[8 * q + 6], v[8 * q + 7]));
+                tc::fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) {
+                    tc::tma_store_2d(&tm_y, st, h0 * p.W + c * 32, img * p.Cout + o0);
+                    tc::tma_store_commit();
+                }
+            }
+            tc::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive_cluster(tc::mapa(tc::smem_u32(&tmem_empty[buf]), 0));
+        }
+        if (lane == 0) tc::tma_store_wait_all<0>();
+    }
+    tc::tc_fence_before_sync();
+    __syncthreads();
+    tc::cluster_sync();
+    if (warp == 1) {
+        tc::tc_fence_after_sync();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
 // wgrad kernel: one work unit = (tap, 128 output channels, NT input channels, batch slice)
 // ---------------------------------------------------------------------------------------------------
 struct WgradParams {
@@ -673,7 +840,21 @@ relay_status_t launch_fprop(const ConvDims &d, const TcPlan &pl, const void *act
     p.bias = bias; p.bias_bf16 = b_dt == RELAY_BF16; p.act = act;
     p.err = device_error_word();
     if (!p.err) return fail(RELAY_ERR_CUDA, "no device error word");
-    // pairs fill whole rounds over the SMs; the remainder runs as singles
+    // two-SM form: every tile is computed by a pair of blocks, each loading half of the activation tile
+    if (Cout % 256 == 0 && pl.rows_per_tile % 2 == 0 && ((p.nt / 2) * 128) % 1024 == 0 && sms >= 2 &&
+        (int64_t)p.n_tiles_total * (Cout / 256) >= sms / 2) {
+        CUtensorMap tm_xh;
+        RELAY_TRY(make_tmap_nhwc_bf16(&tm_xh, act_nhwc, Cin, d.W, d.H, d.Nb, BK, (uint32_t)d.W, pl.rows_per_tile / 2));
+        const size_t stage2 = (size_t)BM * BK * 2 + (size_t)(p.nt / 2) * 128;
+        p.stages = (int)std::min<size_t>(8, (kSmemLimit - 1024 - 4 * 4096) / stage2);
+        p.pairs_per_ntile = Cout / 256;
+        p.n_pairs = p.n_items = p.n_tiles_total * p.pairs_per_ntile;
+        const size_t smem2 = 1024 + (size_t)p.stages * stage2 + 4 * 4096 + 256;
+        RELAY_CUDA(cudaFuncSetAttribute(conv_fprop_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2));
+        conv_fprop_tc2_kernel<<<2 * std::min(p.n_items, sms / 2), NUM_THREADS, smem2, st>>>(tm_w, tm_xh, tm_y, p);
+        return check_launch("conv_fprop_tc2");
+    }
+    // one-SM form: pairs fill whole rounds over the SMs; the remainder runs as singles
     const int64_t total_pairs = Cout % 256 == 0 ? (int64_t)p.n_tiles_total * (Cout / 256) : 0;
     const int mh = total_pairs >= sms ? 2 : 1;
     const size_t b_stage = ((size_t)p.nt * BK * 2 + 1023) & ~size_t(1023);
