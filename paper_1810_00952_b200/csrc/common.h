@@ -93,6 +93,29 @@ relay_status_t check_no_overlap(const relay_tensor_t *const *outs, int n_out, co
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Launch with programmatic stream serialisation: the kernel may be scheduled while the previous kernel
+// of the stream drains, runs its set-up, and blocks in pdl_wait() until that kernel has completed and
+// its memory is visible.  Kernels launched this way call pdl_wait() before their first global access.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#ifdef __CUDACC__
+// lets the next kernel of the stream start its set-up; then waits for the previous kernel's results
+__device__ __forceinline__ void pdl_wait()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+#endif
+
 // device-side error word (set by kernels whose bounded waits expire)
 int *device_error_word();  // device address of the word on the current device (nullptr on failure)
 

@@ -52,6 +52,7 @@ __global__ void __launch_bounds__(256) nchw_to_nhwc_kernel(const __nv_bfloat16 *
     __shared__ __align__(16) __nv_bfloat16 tile[64][66];
     const int n = blockIdx.z, c0 = blockIdx.y * 64, p0 = blockIdx.x * 64;
     const size_t img = (size_t)n * C * HW;
+    pdl_wait();
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
         const int idx = threadIdx.x + i * 256;
@@ -106,6 +107,7 @@ __global__ void pack_weights_kernel(const __nv_bfloat16 *__restrict__ w, __nv_bf
                                     __nv_bfloat16 *__restrict__ wb, int O, int C, int R, int S)
 {
     const unsigned taps = R * S, total = (unsigned)O * C * taps;     // < 2^31 (checked by the plan)
+    pdl_wait();
     for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
         if (wf) {
             const unsigned c = i % C, t = i / C, tap = t % taps, o = t / taps;
@@ -123,6 +125,7 @@ __global__ void pack_weights_kernel(const __nv_bfloat16 *__restrict__ w, __nv_bf
 __global__ void wgrad_reduce_kernel(const float *__restrict__ part, int n_slices, __nv_bfloat16 *__restrict__ dw, int O, int C, int taps)
 {
     const unsigned oc_total = (unsigned)O * C, total = oc_total * (unsigned)taps;
+    pdl_wait();
     for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
         const unsigned tap = i / oc_total, oc = i - tap * oc_total;
         float s = 0.0f;
@@ -209,6 +212,7 @@ conv_fprop_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
     __syncthreads();
     tc::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();   // set-up done; from here on the kernel touches global memory
 
     if (warp == 0) {
         if (lane == 0) {
@@ -388,6 +392,7 @@ conv_fprop_tc2_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
     tc::cluster_sync();
     tc::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();   // set-up done; from here on the kernel touches global memory
 
     if (warp == 0) {
         if (lane == 0) {
@@ -565,6 +570,7 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_dz, const __grid_con
     __syncthreads();
     tc::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();   // set-up done; from here on the kernel touches global memory
 
     if (warp == 0) {
         if (lane == 0) {
@@ -681,6 +687,7 @@ conv_wgrad_tc2_kernel(const __grid_constant__ CUtensorMap tm_dz, const __grid_co
     tc::cluster_sync();
     tc::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();   // set-up done; from here on the kernel touches global memory
 
     if (warp == 0) {
         if (lane == 0) {
@@ -851,7 +858,7 @@ relay_status_t launch_fprop(const ConvDims &d, const TcPlan &pl, const void *act
         p.n_pairs = p.n_items = p.n_tiles_total * p.pairs_per_ntile;
         const size_t smem2 = 1024 + (size_t)p.stages * stage2 + 4 * 4096 + 256;
         RELAY_CUDA(cudaFuncSetAttribute(conv_fprop_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2));
-        conv_fprop_tc2_kernel<<<2 * std::min(p.n_items, sms / 2), NUM_THREADS, smem2, st>>>(tm_w, tm_xh, tm_y, p);
+        RELAY_CUDA(launch_pdl(conv_fprop_tc2_kernel, dim3(2 * std::min(p.n_items, sms / 2)), dim3(NUM_THREADS), smem2, st, tm_w, tm_xh, tm_y, p));
         return check_launch("conv_fprop_tc2");
     }
     // one-SM form: pairs fill whole rounds over the SMs; the remainder runs as singles
@@ -869,11 +876,11 @@ relay_status_t launch_fprop(const ConvDims &d, const TcPlan &pl, const void *act
         p.n_pairs = (int)(ntiles_as_pairs * p.pairs_per_ntile);
         p.n_items = p.n_pairs + (int)((p.n_tiles_total - ntiles_as_pairs) * (Cout / BM));
         RELAY_CUDA(cudaFuncSetAttribute(conv_fprop_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        conv_fprop_tc_kernel<2><<<std::min(p.n_items, sms), 64 + 256, smem, st>>>(tm_w, tm_x, tm_y, p);
+        RELAY_CUDA(launch_pdl(conv_fprop_tc_kernel<2>, dim3(std::min(p.n_items, sms)), dim3(64 + 256), smem, st, tm_w, tm_x, tm_y, p));
     } else {
         p.pairs_per_ntile = 1; p.n_pairs = 0; p.n_items = p.n_tiles_total * (Cout / BM);
         RELAY_CUDA(cudaFuncSetAttribute(conv_fprop_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        conv_fprop_tc_kernel<1><<<std::min(p.n_items, sms), 64 + 128, smem, st>>>(tm_w, tm_x, tm_y, p);
+        RELAY_CUDA(launch_pdl(conv_fprop_tc_kernel<1>, dim3(std::min(p.n_items, sms)), dim3(64 + 128), smem, st, tm_w, tm_x, tm_y, p));
     }
     return check_launch("conv_fprop_tc");
 }
@@ -882,8 +889,8 @@ relay_status_t launch_transpose(bool grad, const void *in, const void *y, void *
                                 float *db_part, cudaStream_t st)
 {
     dim3 grid((unsigned)((HW + 63) / 64), (unsigned)((C + 63) / 64), (unsigned)Nb);
-    if (grad) nchw_to_nhwc_kernel<true><<<grid, 256, 0, st>>>((const __nv_bfloat16 *)in, (const __nv_bfloat16 *)y, (__nv_bfloat16 *)out, (int)C, (int)HW, act, db_part);
-    else nchw_to_nhwc_kernel<false><<<grid, 256, 0, st>>>((const __nv_bfloat16 *)in, nullptr, (__nv_bfloat16 *)out, (int)C, (int)HW, act, nullptr);
+    if (grad) RELAY_CUDA(launch_pdl(nchw_to_nhwc_kernel<true>, grid, dim3(256), 0, st, (const __nv_bfloat16 *)in, (const __nv_bfloat16 *)y, (__nv_bfloat16 *)out, (int)C, (int)HW, act, db_part));
+    else RELAY_CUDA(launch_pdl(nchw_to_nhwc_kernel<false>, grid, dim3(256), 0, st, (const __nv_bfloat16 *)in, (const __nv_bfloat16 *)nullptr, (__nv_bfloat16 *)out, (int)C, (int)HW, act, (float *)nullptr));
     return check_launch("nchw_to_nhwc");
 }
 
@@ -931,7 +938,7 @@ relay_status_t launch_conv_fwd_tc(const ConvDims &d, const void *x, const void *
     char *base = (char *)ws;
     void *x_nhwc = base, *wf = base + pl.x_nhwc;
     RELAY_TRY(launch_transpose(false, x, nullptr, x_nhwc, d.Nb, d.C, d.H * d.W, 0, nullptr, st));
-    pack_weights_kernel<<<(unsigned)((d.O * d.C * 9 + 255) / 256), 256, 0, st>>>((const __nv_bfloat16 *)w, (__nv_bfloat16 *)wf, nullptr, (int)d.O, (int)d.C, 3, 3);
+    RELAY_CUDA(launch_pdl(pack_weights_kernel, dim3((unsigned)((d.O * d.C * 9 + 255) / 256)), dim3(256), 0, st, (const __nv_bfloat16 *)w, (__nv_bfloat16 *)wf, (__nv_bfloat16 *)nullptr, (int)d.O, (int)d.C, 3, 3));
     RELAY_TRY(check_launch("pack_weights"));
     return launch_fprop(d, pl, x_nhwc, (int)d.C, wf, (int)d.O, b, b_dt, act, y, st);
 }
@@ -953,7 +960,7 @@ relay_status_t launch_conv_grad_tc(const ConvDims &d, const void *x, const void 
     RELAY_TRY(launch_transpose(false, x, nullptr, x_nhwc, d.Nb, d.C, HW, 0, nullptr, st));
     if (db) RELAY_TRY(launch_colsum_finalize(db_part, (int)(d.Nb * ((HW + 63) / 64)), d.O, 1.0f, db, st));
     if (dx) {
-        pack_weights_kernel<<<(unsigned)((d.O * d.C * 9 + 255) / 256), 256, 0, st>>>((const __nv_bfloat16 *)w, nullptr, (__nv_bfloat16 *)wb, (int)d.O, (int)d.C, 3, 3);
+        RELAY_CUDA(launch_pdl(pack_weights_kernel, dim3((unsigned)((d.O * d.C * 9 + 255) / 256)), dim3(256), 0, st, (const __nv_bfloat16 *)w, (__nv_bfloat16 *)nullptr, (__nv_bfloat16 *)wb, (int)d.O, (int)d.C, 3, 3));
         RELAY_TRY(check_launch("pack_weights"));
         RELAY_TRY(launch_fprop(d, pl, dz_nhwc, (int)d.O, wb, (int)d.C, nullptr, RELAY_F32, RELAY_ACT_NONE, dx, st));
     }
@@ -974,14 +981,13 @@ relay_status_t launch_conv_grad_tc(const ConvDims &d, const void *x, const void 
     if (pl.wg_pair) {
         const size_t smem2 = 1024 + (size_t)p.stages * 4 * p.kpix * 128 + 4 * 8192 + 256;
         RELAY_CUDA(cudaFuncSetAttribute(conv_wgrad_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2));
-        conv_wgrad_tc2_kernel<<<2 * grid, NUM_THREADS, smem2, st>>>(tm_dz, tm_x, tm_part, p);
+        RELAY_CUDA(launch_pdl(conv_wgrad_tc2_kernel, dim3(2 * grid), dim3(NUM_THREADS), smem2, st, tm_dz, tm_x, tm_part, p));
     } else {
         RELAY_CUDA(cudaFuncSetAttribute(conv_wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        conv_wgrad_tc_kernel<<<grid, NUM_THREADS, smem, st>>>(tm_dz, tm_x, tm_part, p);
+        RELAY_CUDA(launch_pdl(conv_wgrad_tc_kernel, dim3(grid), dim3(NUM_THREADS), smem, st, tm_dz, tm_x, tm_part, p));
     }
     RELAY_TRY(check_launch("conv_wgrad_tc"));
-    wgrad_reduce_kernel<<<(unsigned)((9 * d.O * d.C + 255) / 256), 256, 0, st>>>(part, p.n_slices, (__nv_bfloat16 *)dw,
-                                                                                                          (int)d.O, (int)d.C, 9);
+    RELAY_CUDA(launch_pdl(wgrad_reduce_kernel, dim3((unsigned)((9 * d.O * d.C + 255) / 256)), dim3(256), 0, st, (const float *)part, p.n_slices, (__nv_bfloat16 *)dw, (int)d.O, (int)d.C, 9));
     return check_launch("wgrad_reduce");
 }
 

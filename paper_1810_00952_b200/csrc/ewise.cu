@@ -29,6 +29,7 @@ __global__ void __launch_bounds__(kTX *kTY, Body::NIN >= 4 ? 2 : 3) ewise2d_kern
     constexpr int V = VecN<T>::N, NIN = Body::NIN, NOUT = Body::NOUT;
     const int tx = threadIdx.x, ty = threadIdx.y;
     const int64_t col0 = ((int64_t)blockIdx.x * kTX + tx) * V;
+    pdl_wait();
     const bool active = col0 < A.cols;
 
     float fixed[NIN][V];  // operands that do not change from row to row
@@ -136,6 +137,7 @@ __global__ void __launch_bounds__(32 * TY) colsum_finalize_kernel(const float *_
 {
     __shared__ float sm[TY][33];
     const int tx = threadIdx.x, ty = threadIdx.y;
+    pdl_wait();
     const int64_t c = (int64_t)blockIdx.x * 32 + tx;
     const float *p = partial + (size_t)blockIdx.y * n_slices * cols;
     float s = 0.0f;
@@ -436,8 +438,8 @@ relay_status_t launch_body2d(int32_t storage, const Args2D<Body::NIN, Body::NOUT
     dim3 block(kTX, kTY);
     dim3 grid((unsigned)((A.cols + (int64_t)kTX * vec - 1) / (kTX * vec)), (unsigned)n_slices);
     A.rows_per_slice = (int)((A.rows + n_slices - 1) / n_slices);
-    if (storage == RELAY_BF16) ewise2d_kernel<Body, __nv_bfloat16, true><<<grid, block, 0, st>>>(A);
-    else ewise2d_kernel<Body, float, false><<<grid, block, 0, st>>>(A);
+    if (storage == RELAY_BF16) RELAY_CUDA(launch_pdl(ewise2d_kernel<Body, __nv_bfloat16, true>, grid, block, 0, st, A));
+    else RELAY_CUDA(launch_pdl(ewise2d_kernel<Body, float, false>, grid, block, 0, st, A));
     return check_launch(what);
 }
 
@@ -448,8 +450,8 @@ relay_status_t launch_colsum_finalize_n(const float *partial, int n_slices, int6
     FinalizeOuts fo{};
     for (int k = 0; k < n_out; ++k) fo.out[k] = out[k];
     const dim3 grid((unsigned)((cols + 31) / 32), (unsigned)n_out);
-    if (n_slices > 256) colsum_finalize_kernel<32><<<grid, dim3(32, 32), 0, st>>>(partial, n_slices, cols, scale, fo);
-    else colsum_finalize_kernel<8><<<grid, dim3(32, 8), 0, st>>>(partial, n_slices, cols, scale, fo);
+    if (n_slices > 256) RELAY_CUDA(launch_pdl(colsum_finalize_kernel<32>, grid, dim3(32, 32), 0, st, partial, n_slices, cols, scale, fo));
+    else RELAY_CUDA(launch_pdl(colsum_finalize_kernel<8>, grid, dim3(32, 8), 0, st, partial, n_slices, cols, scale, fo));
     return check_launch("colsum_finalize");
 }
 

@@ -75,6 +75,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     __syncthreads();
     tc::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();   // set-up done; from here on the kernel touches global memory
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
@@ -275,7 +276,7 @@ relay_status_t launch_gemm_tc(const GemmDesc &g, cudaStream_t st)
     do {                                                                                                                  \
         RELAY_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<AMN, BMN, MHV>, cudaFuncAttributeMaxDynamicSharedMemorySize,       \
                                         (int)Cfg<MHV>::SMEM_BYTES));                                                      \
-        gemm_tc_kernel<AMN, BMN, MHV><<<grid, Cfg<MHV>::NUM_THREADS, Cfg<MHV>::SMEM_BYTES, st>>>(tm_a, tm_b, tm_c, p);          \
+        RELAY_CUDA(launch_pdl(gemm_tc_kernel<AMN, BMN, MHV>, dim3(grid), dim3(Cfg<MHV>::NUM_THREADS), Cfg<MHV>::SMEM_BYTES, st, tm_a, tm_b, tm_c, p));          \
     } while (0)
 #define LAUNCH_MH(AMN, BMN)          \
     do {                             \

@@ -71,6 +71,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     tc::cluster_sync();                                   // the peer's barriers are initialised before anyone signals them
     tc::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();   // set-up done; from here on the kernel touches global memory
 
     if (warp == 0) {
         // ---------------- TMA producer (both blocks) ----------------
@@ -199,7 +200,7 @@ relay_status_t launch_gemm_tc2(const GemmDesc &g, int sms, cudaStream_t st)
 #define LAUNCH2(AMN, BMN)                                                                                                   \
     do {                                                                                                                    \
         RELAY_CUDA(cudaFuncSetAttribute(gemm_tc2_kernel<AMN, BMN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES)); \
-        gemm_tc2_kernel<AMN, BMN><<<2 * pairs, NUM_THREADS, SMEM_BYTES, st>>>(tm_a, tm_b, tm_c, p);                         \
+        RELAY_CUDA(launch_pdl(gemm_tc2_kernel<AMN, BMN>, dim3(2 * pairs), dim3(NUM_THREADS), SMEM_BYTES, st, tm_a, tm_b, tm_c, p));                         \
     } while (0)
     if (a_mn && b_mn) LAUNCH2(true, true);
     else if (a_mn) LAUNCH2(true, false);
