@@ -4,6 +4,10 @@
 // and six ring stages fit in shared memory.  No multicast load is used: every byte a block needs is
 // fetched by that block.
 //
+// Work units: whole 256 x 256 tiles for as many full rounds over the pairs as there are; the tiles left for
+// the last, partly filled round are cut into two 256 x 128 units when that lets the round end in half the
+// time (p.tail_split = 2), so the SMs are not left idle behind a few full-size tiles.
+//
 // Pair protocol (rank 0 = leader):
 //   full[s]      lives in the leader; both blocks' TMA loads complete on it (cta_group::2 form), the
 //                leader's producer posts the expected byte count of both;
@@ -35,6 +39,28 @@ constexpr int NUM_THREADS = 192;
 constexpr int STAGING_BYTES = 4 * 2 * 4096;
 constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * STAGE_BYTES + STAGING_BYTES + 256;
 
+// Work unit u of the launch: tile index, first column and width.
+struct Unit {
+    int tile_m, n0, width;
+};
+__device__ __forceinline__ Unit unit_of(const Params &p, int u)
+{
+    Unit w;
+    int tile, sub = 0;
+    w.width = BN;
+    if (u < p.full_tiles) {
+        tile = u;
+    } else {
+        const int v = u - p.full_tiles;
+        tile = p.full_tiles + v / p.tail_split;
+        sub = v % p.tail_split;
+        w.width = BN / p.tail_split;
+    }
+    w.tile_m = tile % p.tiles_m;
+    w.n0 = (tile / p.tiles_m) * BN + sub * w.width;
+    return w;
+}
+
 template <bool A_MN, bool B_MN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
@@ -51,7 +77,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = tc::cluster_ctarank();          // 0 = leader
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-    const int n_tiles = p.tiles_m * p.tiles_n;        // tiles of 256 x 256
+    const int n_units = p.full_tiles + (p.tiles_m * p.tiles_n - p.full_tiles) * p.tail_split;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
@@ -79,14 +105,17 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             int s = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
-                const int m0 = (tile % p.tiles_m) * 256 + (int)rank * 128;      // this block's rows
-                const int n0 = (tile / p.tiles_m) * BN + (int)rank * 128;       // this block's half of the B tile
+            for (int u = pair; u < n_units && ok; u += n_pairs) {
+                const Unit w = unit_of(p, u);
+                const int m0 = w.tile_m * 256 + (int)rank * 128;                // this block's rows
+                const int n0 = w.n0 + (int)rank * (w.width >> 1);               // this block's half of the B columns
+                const int b_boxes = w.width >> 7;                               // boxes of 64 columns in that half
+                const uint32_t tx = 2u * (A_BYTES + (uint32_t)b_boxes * MN_BOX_BYTES);   // bytes of both blocks
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
                     if (!tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
                     uint8_t *sa = smem + (size_t)s * STAGE_BYTES, *sb = sa + A_BYTES;
                     const uint32_t bar = tc::mapa(tc::smem_u32(&full[s]), 0);       // the leader's barrier
-                    if (rank == 0) tc::mbar_expect_tx_cluster(bar, 2 * STAGE_BYTES); // bytes of both blocks
+                    if (rank == 0) tc::mbar_expect_tx_cluster(bar, tx);
                     const int k0 = kb * BK;
                     if (A_MN) {
 #pragma unroll
@@ -94,11 +123,11 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                     } else {
                         tc::tma_load_2d_pair(sa, &tm_a, bar, k0, m0);
                     }
-                    if (B_MN) {
-#pragma unroll
-                        for (int i = 0; i < 2; ++i) tc::tma_load_2d_pair(sb + i * MN_BOX_BYTES, &tm_b, bar, n0 + i * 64, k0);
-                    } else {
-                        tc::tma_load_2d_pair(sb, &tm_b, bar, k0, n0);
+                    // B in boxes of 64 columns: MN-major boxes are 64 x 64 k anyway; K-major boxes of 64 rows stack
+                    // to the same shared-memory image as one 128-row box
+                    for (int i = 0; i < b_boxes; ++i) {
+                        if (B_MN) tc::tma_load_2d_pair(sb + i * MN_BOX_BYTES, &tm_b, bar, n0 + i * 64, k0);
+                        else tc::tma_load_2d_pair(sb + i * MN_BOX_BYTES, &tm_b, bar, k0, n0 + i * 64);
                     }
                     if (++s == STAGES) { s = 0; phase ^= 1; }
                 }
@@ -107,7 +136,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     } else if (warp == 1) {
         // ---------------- MMA issuer (leader only) ----------------
         if (lane == 0 && rank == 0) {
-            constexpr uint32_t idesc = tc::instr_desc_bf16(256, BN, A_MN, B_MN);
+            constexpr uint32_t idesc_full = tc::instr_desc_bf16(256, BN, A_MN, B_MN);
+            constexpr uint32_t idesc_half = tc::instr_desc_bf16(256, BN / 2, A_MN, B_MN);
             constexpr uint32_t a_lbo = A_MN ? MN_BOX_BYTES : 16, b_lbo = B_MN ? MN_BOX_BYTES : 16;
             constexpr uint32_t a_step = A_MN ? 2048 : 32, b_step = B_MN ? 2048 : 32;
             const uint64_t desc_a0 = tc::smem_desc(tc::smem_u32(smem), a_lbo, 1024);
@@ -115,8 +145,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             uint32_t t_local = 0, phase = 0, stage_off = 0;
             int s = 0;
             bool ok = true;
-            for (int tile = pair; tile < n_tiles && ok; tile += n_pairs, ++t_local) {
+            for (int u = pair; u < n_units && ok; u += n_pairs, ++t_local) {
                 const int buf = t_local & 1;
+                const uint32_t idesc = (u < p.full_tiles || p.tail_split == 1) ? idesc_full : idesc_half;
                 if (!tc::mbar_wait(&tmem_empty[buf], ((t_local >> 1) & 1) ^ 1, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) break;
                 tc::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * BN;
@@ -140,9 +171,10 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         const int quarter = warp & 3;
         uint8_t *my_stage = staging + (size_t)(warp - 2) * 2 * 4096;
         uint32_t t_local = 0;
-        for (int tile = pair; tile < n_tiles; tile += n_pairs, ++t_local) {
+        for (int u = pair; u < n_units; u += n_pairs, ++t_local) {
             const int buf = t_local & 1;
-            const int m0 = (tile % p.tiles_m) * 256 + (int)rank * 128, n0 = (tile / p.tiles_m) * BN;
+            const Unit w = unit_of(p, u);
+            const int m0 = w.tile_m * 256 + (int)rank * 128, n0 = w.n0;
             int ok = 1;
             if (lane == 0) ok = tc::mbar_wait(&tmem_full[buf], (t_local >> 1) & 1, abort_flag, p.err, tc::ERR_WAIT_TMEM_FULL) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -151,8 +183,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             const int row0 = m0 + quarter * 32;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * BN;
             if (row0 < p.M) {
-                if (p.out_f32) epilogue_rows<true, 2>(p, &tm_c, taddr, my_stage, lane, row0, n0);
-                else epilogue_rows<false, 2>(p, &tm_c, taddr, my_stage, lane, row0, n0);
+                if (p.out_f32) epilogue_rows<true, 2>(p, &tm_c, taddr, my_stage, lane, row0, n0, w.width);
+                else epilogue_rows<false, 2>(p, &tm_c, taddr, my_stage, lane, row0, n0, w.width);
             }
             tc::tc_fence_before_sync();
             __syncwarp();
@@ -186,7 +218,7 @@ relay_status_t launch_gemm_tc2(const GemmDesc &g, int sms, cudaStream_t st)
     if (a_mn) RELAY_TRY(make_tmap_2d_bf16(&tm_a, g.a, g.M, g.K, g.a_sk, 64, BK));
     else RELAY_TRY(make_tmap_2d_bf16(&tm_a, g.a, g.K, g.M, g.a_sm, BK, 128));
     if (b_mn) RELAY_TRY(make_tmap_2d_bf16(&tm_b, g.b, g.N, g.K, g.b_sk, 64, BK));
-    else RELAY_TRY(make_tmap_2d_bf16(&tm_b, g.b, g.K, g.N, g.b_sn, BK, 128));
+    else RELAY_TRY(make_tmap_2d_bf16(&tm_b, g.b, g.K, g.N, g.b_sn, BK, 64));
     const bool f32 = g.out_dtype == RELAY_F32;
     RELAY_TRY(make_tmap_2d(&tm_c, f32, g.c, g.N, g.M, g.ldc, f32 ? 32 : 64, 32, true));
     Params p{};
@@ -196,7 +228,12 @@ relay_status_t launch_gemm_tc2(const GemmDesc &g, int sms, cudaStream_t st)
     p.tiles_m = (int)((g.M + 255) / 256); p.tiles_n = (int)((g.N + BN - 1) / BN); p.k_blocks = (int)((g.K + BK - 1) / BK);
     p.err = device_error_word();
     if (!p.err) return fail(RELAY_ERR_CUDA, "no device error word");
-    const int pairs = std::min(p.tiles_m * p.tiles_n, sms / 2);
+    const int n_tiles = p.tiles_m * p.tiles_n;
+    const int pairs = std::min(n_tiles, sms / 2);
+    // tiles of the last, partly filled round: two half-width units each when they then still fit one round
+    const int rem = n_tiles % pairs;
+    p.tail_split = (rem > 0 && 2 * rem <= pairs) ? 2 : 1;
+    p.full_tiles = p.tail_split == 2 ? n_tiles - rem : n_tiles;
 #define LAUNCH2(AMN, BMN)                                                                                                   \
     do {                                                                                                                    \
         RELAY_CUDA(cudaFuncSetAttribute(gemm_tc2_kernel<AMN, BMN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES)); \

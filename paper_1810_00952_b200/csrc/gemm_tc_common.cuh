@@ -18,18 +18,19 @@ struct Params {
     const void *bias;
     int bias_bf16, act, out_f32;
     int tiles_m, tiles_n, k_blocks;
+    int full_tiles, tail_split;   // two-SM kernel: tiles after the first full_tiles are cut into tail_split column parts
     int *err;
 };
 
-// One warp drains its 32 accumulator rows (256 columns): TMEM -> registers -> bias + activation ->
-// rounding -> swizzled staging buffer -> TMA tile store of 32 rows x 128 bytes at a time.
+// One warp drains its 32 accumulator rows (`width` columns, 256 unless stated): TMEM -> registers -> bias +
+// activation -> rounding -> swizzled staging buffer -> TMA tile store of 32 rows x 128 bytes at a time.
 template <bool OUT_F32, int BUFS>
 __device__ __forceinline__ void epilogue_rows(const Params &p, const CUtensorMap *tm_c, uint32_t taddr, uint8_t *stage, int lane,
-                                              int row0, int n0)
+                                              int row0, int n0, int width = BN)
 {
     constexpr int COLS = OUT_F32 ? 32 : 64;             // columns per 128-byte block
 #pragma unroll 1
-    for (int blk = 0; blk < BN / COLS; ++blk) {
+    for (int blk = 0; blk < width / COLS; ++blk) {
         const int nc = n0 + blk * COLS;
         if (nc >= p.N) break;                            // warp-uniform
         uint4 piece[8];

@@ -151,3 +151,27 @@ def test_full_size_mlp_layer_sampled_rows_and_columns():
         assert_bf16(dw[rows], odw, what=f"dw{l}")
         assert_bf16(db, odb, stored_bf16=False, what=f"db{l}")
         g = dx
+
+
+def test_two_sm_kernel_ragged_edges_and_half_width_tail_units():
+    """A shape the two-SM kernel takes (more 256 x 256 tiles than SMs) with ragged M, N and K and a last
+    round that is cut into half-width units; sampled rows (all columns) of y, dx and dW, and all of db."""
+    M, K, N = 2600, 136, 3720
+    t = I.cfg1_tiny_mlp(M, K, N, salt=77)
+    x, w, b, dy = (t[k].bfloat16() for k in ("x", "w", "b", "dy"))
+    w = (t["w"] / np.sqrt(K)).bfloat16()
+    act = B.ACT_TANH
+    y = run_fwd(x, w, b, act)
+    xo, wo, bo, dyo = (v.double().numpy() for v in (x, w, b, dy))
+    rng = np.random.default_rng(11)
+    rows = np.unique(np.concatenate([[0, 127, 128, 255, 256, 2559, 2560, M - 1], rng.integers(0, M, 12)]))
+    assert_bf16(y[rows], oracle.dense_act(xo[rows], wo, bo, act, F64), what="y")
+    dx, dw, db = run_grad(x, w, y, dy, act)
+    yo = to_np(y)
+    odx, _, _ = oracle.dense_act_grad(xo[rows], wo, yo[rows], dyo[rows], act, F64, F64, F64, want_dw=False, want_db=False,
+                                      dz_dtype=oracle.BF16)
+    assert_bf16(dx[rows], odx, what="dx")
+    krows = np.unique(np.concatenate([[0, 63, 64, K - 1], rng.integers(0, K, 6)]))
+    _, odw, odb = oracle.dense_act_grad(xo[:, krows], wo[krows], yo, dyo, act, F64, F64, F64, want_dx=False, dz_dtype=oracle.BF16)
+    assert_bf16(dw[krows], odw, what="dw")
+    assert_bf16(db, odb, stored_bf16=False, what="db")
