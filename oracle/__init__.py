@@ -260,6 +260,43 @@ def dense_act_grad(x, w, y, dy, act_code: int, dx_dtype: int, dw_dtype: int, db_
     return dx, dw, db
 
 
+def softmax_xent(z, t, loss_dtype: int = F64) -> np.ndarray:
+    """loss[i] = -sum_j t[i,j] log softmax(z[i,:])_j (Fig. 3, relay.softmax_cross_entropy)."""
+    z, t = _f64(z), _f64(t)
+    Bn, C = z.shape
+    assert t.shape == (Bn, C)
+    loss = np.empty((Bn,), dtype=np.float64)
+    i64 = ctypes.c_int64
+    rc = _L().orc_softmax_xent(_ptr(z), _ptr(t), i64(Bn), i64(C), int(loss_dtype), _ptr(loss))
+    assert rc == 0
+    return loss
+
+
+def softmax_xent_grad(z, t, dloss, loss_dtype: int = F64, dz_dtype: int = F64):
+    """Returns (loss, dz): the result bundled with the partial with respect to the scores (Section 4.2)."""
+    z, t, dloss = _f64(z), _f64(t), _f64(dloss)
+    Bn, C = z.shape
+    assert t.shape == (Bn, C) and dloss.shape == (Bn,)
+    loss = np.empty((Bn,), dtype=np.float64)
+    dz = np.empty((Bn, C), dtype=np.float64)
+    i64 = ctypes.c_int64
+    rc = _L().orc_softmax_xent_grad(_ptr(z), _ptr(t), _ptr(dloss), i64(Bn), i64(C), int(loss_dtype), int(dz_dtype),
+                                    _ptr(loss), _ptr(dz))
+    assert rc == 0
+    return loss, dz
+
+
+def sgd_update(p, g, lr: float, p_dtype: int = F64) -> np.ndarray:
+    """p - lr * g stored in p_dtype (Section 4.1, relay.update_model_params)."""
+    p, g = _f64(p), _f64(g)
+    assert p.shape == g.shape
+    out = np.empty(p.shape, dtype=np.float64)
+    fn = _L().orc_sgd_update
+    fn.restype = None
+    fn(_ptr(p), _ptr(g), ctypes.c_int64(p.size), ctypes.c_double(lr), int(p_dtype), _ptr(out))
+    return out
+
+
 def conv2d_act(x, wt, b, stride: int, pad: int, act_code: int, y_dtype: int) -> np.ndarray:
     x, wt = _f64(x), _f64(wt)
     b = None if b is None else _f64(b)

@@ -370,6 +370,65 @@ int orc_dense_act_grad(const double *x, const double *w, const double *y, const 
 }
 
 /* ------------------------------------------------------------------------------------------
+ * Softmax cross-entropy loss (Fig. 3, relay.softmax_cross_entropy(scores, y); y is a Float tensor
+ * of the scores' shape, e.g. a one-hot row or any non-negative weighting of the classes).  Per row i
+ * of z[B,C] and t[B,C]:
+ *   p[i,j]  = exp(z[i,j]) / sum_k exp(z[i,k])
+ *   loss[i] = - sum_j t[i,j] * log p[i,j]
+ * written with log p[i,j] = (z[i,j] - m_i) - log sum_k exp(z[i,k] - m_i), m_i = max_k z[i,k]: the same
+ * number, without overflow of exp.  Sums run in increasing j.  loss is stored in loss_dtype.
+ * ---------------------------------------------------------------------------------------- */
+int orc_softmax_xent(const double *z, const double *t, int64_t B, int64_t C, int loss_dtype, double *loss)
+{
+    if (C <= 0) return 1;
+    for (int64_t i = 0; i < B; ++i) {
+        const double *zr = z + i * C, *tr = t + i * C;
+        double m = zr[0];
+        for (int64_t j = 1; j < C; ++j) if (zr[j] > m) m = zr[j];
+        double se = 0.0;
+        for (int64_t j = 0; j < C; ++j) se += exp(zr[j] - m);
+        double lse = log(se), l = 0.0;
+        for (int64_t j = 0; j < C; ++j) l -= tr[j] * ((zr[j] - m) - lse);
+        loss[i] = orc_cast(l, loss_dtype);
+    }
+    return 0;
+}
+
+/* Gradient group of the loss (Section 4.2: the upstream partial dloss[i] of the final scalar with respect
+ * to loss[i] is given; the result is returned alongside the partial):
+ *   dz[i,j] = dloss[i] * ( p[i,j] * sum_k t[i,k] - t[i,j] )
+ * (the derivative of -sum_j t_j (z_j - logsumexp z) with respect to z_j).  Only the partial with respect
+ * to the scores is produced; the targets are data.  loss may be NULL. */
+int orc_softmax_xent_grad(const double *z, const double *t, const double *dloss, int64_t B, int64_t C,
+                          int loss_dtype, int dz_dtype, double *loss, double *dz)
+{
+    if (C <= 0) return 1;
+    if (loss && orc_softmax_xent(z, t, B, C, loss_dtype, loss)) return 1;
+    for (int64_t i = 0; i < B; ++i) {
+        const double *zr = z + i * C, *tr = t + i * C;
+        double m = zr[0];
+        for (int64_t j = 1; j < C; ++j) if (zr[j] > m) m = zr[j];
+        double se = 0.0, st = 0.0;
+        for (int64_t j = 0; j < C; ++j) se += exp(zr[j] - m);
+        for (int64_t j = 0; j < C; ++j) st += tr[j];
+        for (int64_t j = 0; j < C; ++j) {
+            double pj = exp(zr[j] - m) / se;
+            dz[i * C + j] = orc_cast(dloss[i] * (pj * st - tr[j]), dz_dtype);
+        }
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Parameter update (Section 4.1, relay.update_model_params: vanilla stochastic gradient descent, the one
+ * place where the paper allows mutation):  p <- cast( p - lr * g ), elementwise, stored in p's dtype.
+ * ---------------------------------------------------------------------------------------- */
+void orc_sgd_update(const double *p, const double *g, int64_t n, double lr, int p_dtype, double *p_new)
+{
+    for (int64_t i = 0; i < n; ++i) p_new[i] = orc_cast(p[i] - lr * g[i], p_dtype);
+}
+
+/* ------------------------------------------------------------------------------------------
  * conv2d anchor (Fig. 3, relay.conv2d) as cross-correlation, NCHW input, OIHW weights, zero
  * padding, square stride, with per-channel bias and activation:
  *   y[n,o,p,q] = cast( act( b[o] + sum_{c,r,s} x[n,c,p*st-pad+r,q*st-pad+s] * Wt[o,c,r,s] ) )
