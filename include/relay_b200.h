@@ -280,6 +280,39 @@ relay_status_t relay_lstm_cell_seq(const relay_tensor_t *x, const relay_tensor_t
                                    size_t ws_bytes, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Loss and parameter update: the two operators that close the training step of the LeNet listing
+ * (Fig. 3: relay.softmax_cross_entropy(scores, y), relay.update_model_params(model, model_grad)).
+ * ------------------------------------------------------------------------------------------- */
+
+/* Softmax cross-entropy, one loss per row (the listing's loss is per sample; a batch adds the leading
+ * axis, Section 5.2 "auto-batching"):
+ *   p[i,j] = exp(z[i,j]) / sum_k exp(z[i,k]);   loss[i] = - sum_j t[i,j] log p[i,j]
+ *   scores z:(B,C) t in {f32, bf16};  targets t:(B,C) of base type t or f32 (a Float tensor of the scores'
+ *   shape, as in the listing: a one-hot row or any weighting of the classes);  loss:(B) f32.
+ * Arithmetic in f32.  One pass over z and t; no workspace.  B = 0 is a no-op; C = 0 is RELAY_ERR_SHAPE.
+ * Check order as everywhere: null, rank, dtype, layout, shape, alignment.  Device pointers; outputs may
+ * not overlap inputs. */
+relay_status_t relay_infer_softmax_xent(const relay_tensor_t *scores, const relay_tensor_t *targets, relay_tensor_t *loss);
+relay_status_t relay_softmax_xent(const relay_tensor_t *scores, const relay_tensor_t *targets, const relay_tensor_t *loss,
+                                  void *stream);
+
+/* Gradient group of the loss (Section 4.2: returns the result together with the partial): given the partial
+ * dloss:(B) f32 of the final scalar with respect to loss,
+ *   dscores[i,j] = dloss[i] * ( p[i,j] * sum_k t[i,k] - t[i,j] )        dscores:(B,C) of the scores' type
+ * and, if `loss` is not NULL, loss:(B) f32 as above, from the same pass over z and t. */
+relay_status_t relay_softmax_xent_grad(const relay_tensor_t *scores, const relay_tensor_t *targets, const relay_tensor_t *dloss,
+                                       const relay_tensor_t *loss, const relay_tensor_t *dscores, void *stream);
+
+/* Vanilla stochastic gradient descent on a set of parameters (Section 4.1: update_model_params is the one
+ * place where the paper exposes mutation): for k < n_params, elementwise and IN PLACE,
+ *   params[k] <- cast( params[k] - lr * grads[k] )
+ *   params[k]: any rank <= 6, f32 or bf16;  grads[k]: same shape, the parameter's base type or f32.
+ * Arithmetic in f32, one rounding to the parameter's type.  All tensors are updated by one launch per 8
+ * parameters.  A parameter may not overlap any other parameter or gradient.  n_params = 0 is a no-op. */
+relay_status_t relay_sgd_update(const relay_tensor_t *const *params, const relay_tensor_t *const *grads, int32_t n_params,
+                                float lr, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Status helpers.
  * ------------------------------------------------------------------------------------------- */
 

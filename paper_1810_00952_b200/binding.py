@@ -193,6 +193,12 @@ def relay_infer_lstm(x: TensorDesc, w_ih: TensorDesc, w_hh: TensorDesc):
     return h, c
 
 
+def relay_infer_softmax_xent(scores: TensorDesc, targets: TensorDesc) -> TensorDesc:
+    out = TensorDesc()
+    _check(lib().relay_infer_softmax_xent(_ref(scores), _ref(targets), ctypes.byref(out)))
+    return out
+
+
 def relay_infer_ewise(prog: dict, inputs: Sequence[TensorDesc], value: int) -> TensorDesc:
     out = TensorDesc()
     p = make_prog(prog)
@@ -295,6 +301,20 @@ def relay_lstm_cell_seq(x, w_ih, w_hh, b, h0, c0, h_all, c_final, ws=None):
     wp, wb = _ws(ws)
     _check(lib().relay_lstm_cell_seq(_ref(desc(x)), _ref(desc(w_ih)), _ref(desc(w_hh)), _ref(desc(b)), _ref(desc(h0)),
                                      _ref(desc(c0)), _ref(desc(h_all)), _ref(desc(c_final)), wp, wb, _stream()))
+
+
+def relay_softmax_xent(scores, targets, loss):
+    _check(lib().relay_softmax_xent(_ref(desc(scores)), _ref(desc(targets)), _ref(desc(loss)), _stream()))
+
+
+def relay_softmax_xent_grad(scores, targets, dloss, loss, dscores):
+    _check(lib().relay_softmax_xent_grad(_ref(desc(scores)), _ref(desc(targets)), _ref(desc(dloss)), _ref(desc(loss)),
+                                         _ref(desc(dscores)), _stream()))
+
+
+def relay_sgd_update(params, grads, lr: float):
+    pd, gd = [desc(p) for p in params], [desc(g) for g in grads]
+    _check(lib().relay_sgd_update(_desc_array(pd), _desc_array(gd), len(pd), ctypes.c_float(lr), _stream()))
 
 
 # ---- status helpers -----------------------------------------------------------------------------------

@@ -84,3 +84,26 @@ def cfg5_lstm(T=128, B=64, I=1024, H=1024, salt=0) -> Dict[str, torch.Tensor]:
                 w_hh=uniform(5, 2, (H, 4 * H), -k, k, bf, salt),
                 b=uniform(5, 3, (4 * H,), -k, k, f, salt),
                 h0=torch.zeros(B, H, dtype=f), c0=torch.zeros(B, H, dtype=f))
+
+
+def loss_batch(B=8192, C=8192, dtype=torch.bfloat16, target_dtype=None, one_hot=False, salt=0) -> Dict[str, torch.Tensor]:
+    """Inputs of the loss group: scores ~ N(0,2) [B,C]; targets [B,C] either one-hot rows (class drawn
+    uniformly) or U(0,1) weights; dloss ~ N(0,1) fp32 [B] (the upstream partial)."""
+    target_dtype = target_dtype or dtype
+    r = _rng(6, 1, salt)
+    if one_hot:
+        t = np.zeros((B, C))
+        if B and C:
+            t[np.arange(B), r.integers(0, C, B)] = 1.0
+    else:
+        t = r.uniform(0.0, 1.0, (B, C))
+    return dict(scores=normal(6, 0, (B, C), 2.0, dtype, salt), targets=_store(t, target_dtype),
+                dloss=normal(6, 2, (B,), 1.0, torch.float32, salt))
+
+
+def param_set(shapes, dtype=torch.bfloat16, grad_dtype=None, salt=0):
+    """Parameters ~ N(0, 0.05) and gradients ~ N(0, 1) of the given shapes (lists of CPU tensors)."""
+    grad_dtype = grad_dtype or dtype
+    ps = [normal(7, 2 * i, s, 0.05, dtype, salt) for i, s in enumerate(shapes)]
+    gs = [normal(7, 2 * i + 1, s, 1.0, grad_dtype, salt) for i, s in enumerate(shapes)]
+    return ps, gs

@@ -235,3 +235,40 @@ def test_workspace_queries_are_host_only():
     xb = torch.empty(4, 2, 8, dtype=torch.bfloat16)
     assert B.relay_workspace_bytes_lstm(xb, torch.empty(8, 16, dtype=torch.bfloat16), torch.empty(4, 16, dtype=torch.bfloat16)) >= 4 * 2 * 16 * 4
     assert B.relay_workspace_bytes_dense_act_grad(x, torch.empty(63, 32)) == 0   # ill-typed -> 0
+
+
+# ---- loss and parameter update ----------------------------------------------------------------------
+def test_infer_softmax_xent_relation_and_rejections():
+    for Bn, C in [(1, 10), (64, 1000), (0, 7), (8192, 8192)]:
+        for zt, tt in [(B.F32, B.F32), (B.BF16, B.BF16), (B.BF16, B.F32)]:
+            out = B.relay_infer_softmax_xent(T(zt, (Bn, C)), T(tt, (Bn, C)))
+            assert out.dtype == B.F32 and B._shape(out) == (Bn,)
+    cases = [(T(B.F32, (4, 10)), T(B.F32, (4, 9)), "ERR_SHAPE"), (T(B.F32, (4, 10)), T(B.F32, (5, 10)), "ERR_SHAPE"),
+             (T(B.F32, (4, 10)), T(B.BF16, (4, 10)), "ERR_DTYPE"), (T(B.I32, (4, 10)), T(B.F32, (4, 10)), "ERR_DTYPE"),
+             (T(B.F32, (4, 10, 1)), T(B.F32, (4, 10)), "ERR_RANK"), (T(B.F32, (4,)), T(B.F32, (4,)), "ERR_RANK"),
+             (T(B.F32, (4, 0)), T(B.F32, (4, 0)), "ERR_SHAPE"), (T(B.F32, (4, 10), B.NCHW), T(B.F32, (4, 10)), "ERR_LAYOUT")]
+    for z, t, status in cases:
+        with pytest.raises(B.RelayError) as e:
+            B.relay_infer_softmax_xent(z, t)
+        assert e.value.status_name == status, str(e.value)
+
+
+def test_sgd_update_descriptor_checks_run_before_any_launch():
+    """Descriptor errors are found on the host (no GPU is touched): rank, then dtype, then shape."""
+    lib = B.lib()
+
+    def call(params, grads, lr=0.1):
+        return lib.relay_sgd_update(B._desc_array(params), B._desc_array(grads), len(params), ctypes.c_float(lr), None)
+
+    ok_p, ok_g = T(B.BF16, (4, 8)), T(B.F32, (4, 8))
+    n0 = B.relay_launch_count()
+    assert call([], []) == 0                                        # nothing to update
+    def status_of(params, grads):
+        st = call(params, grads)
+        return B.RelayError(st, "").status_name
+    assert status_of([ok_p, T(B.F32, (3,))], [ok_g, T(B.F32, (3, 1))]) == "ERR_RANK"
+    assert status_of([T(B.I32, (3,))], [T(B.I32, (3,))]) == "ERR_DTYPE"
+    assert status_of([T(B.F32, (3,))], [T(B.BF16, (3,))]) == "ERR_DTYPE"       # gradient narrower than the parameter
+    assert status_of([ok_p], [T(B.F32, (4, 7))]) == "ERR_SHAPE"
+    assert status_of([ok_p], [ok_g]) == "ERR_NULL"                                # descriptors without data
+    assert B.relay_launch_count() == n0
