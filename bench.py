@@ -34,7 +34,7 @@ import torch  # noqa: E402
 
 METRIC = "fused-group TFLOP/s (dense/conv) and HBM GB/s (ewise/reduce) on 1 B200 vs roofline"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-ALL_GROUPS = ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"]
+ALL_GROUPS = ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "next"]
 
 
 def load_peaks():
@@ -138,6 +138,8 @@ class Workload:
             self.host["cfg4"] = I.cfg4_conv(*((2, 32, 14, 14, 32) if small else (32, 256, 56, 56, 256)))
         if "cfg5" in groups:
             self.host["cfg5"] = I.cfg5_lstm(*((8, 8, 64, 64) if small else (128, 64, 1024, 1024)))
+        if "next" in groups:       # loss group and parameter update (the rows that close a training step)
+            self.host["next"] = I.loss_batch(*((256, 512) if small else (8192, 8192)))
         for g, d in self.host.items():
             self.host[g] = {k: v.pin_memory() for k, v in d.items()}
             self.devt[g] = {k: torch.empty_like(v, device=dev) for k, v in d.items()}
@@ -173,6 +175,14 @@ class Workload:
             H = d["w_hh"].shape[0]
             self.out["cfg5"] = dict(h_all=E(T, Bn, H, dt=f32), c=E(Bn, H, dt=f32))
             ws_bytes = max(ws_bytes, B.relay_workspace_bytes_lstm(d["x"], d["w_ih"], d["w_hh"]))
+        if "next" in groups:
+            d = self.devt["next"]
+            self.out["next"] = dict(loss=E(d["scores"].shape[0], dt=f32), loss2=E(d["scores"].shape[0], dt=f32), dscores=torch.empty_like(d["scores"]))
+            # parameters the update mutates: device-resident state of its own (three weight matrices), so the
+            # other groups' inputs stay as generated; their gradients are generated once as well
+            n = 256 if small else 4096
+            ps, gs = I.param_set([(n, n)] * 3, torch.bfloat16, torch.bfloat16)
+            self.sgd_params, self.sgd_grads = [p.to(dev) for p in ps], [g.to(dev) for g in gs]
         self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
         self.flush_buf = torch.zeros(1024 * 1024 * 1024, dtype=torch.uint8, device=dev)
         self.pinned_out = {g: {k: torch.empty_like(v, device="cpu").pin_memory() for k, v in o.items()} for g, o in self.out.items()}
@@ -245,6 +255,18 @@ class Workload:
             with tm.region("cfg5.lstm"):
                 B.relay_lstm_cell_seq(d["x"], d["w_ih"], d["w_hh"], d["b"], d["h0"], d["c0"], o["h_all"], o["c"], ws)
 
+        if "next" in self.groups:
+            d, o = self.devt["next"], self.out["next"]
+            self.flush_l2()
+            with tm.region("next.loss"):
+                B.relay_softmax_xent(d["scores"], d["targets"], o["loss"])
+            self.flush_l2()
+            with tm.region("next.loss_grad"):
+                B.relay_softmax_xent_grad(d["scores"], d["targets"], d["dloss"], o["loss2"], o["dscores"])
+            self.flush_l2()
+            with tm.region("next.sgd"):
+                B.relay_sgd_update(self.sgd_params, self.sgd_grads, 1e-3)
+
     # -- algorithmic work per step -------------------------------------------------------------------------
     def work(self):
         w = {}
@@ -267,6 +289,11 @@ class Workload:
             T, Bn, In = self.host["cfg5"]["x"].shape
             H = self.host["cfg5"]["w_hh"].shape[0]
             w["cfg5.lstm"] = dict(flop=2 * T * Bn * (In + H) * 4 * H)
+        if "next" in self.groups:
+            r, c = self.host["next"]["scores"].shape
+            w["next.loss"] = dict(bytes=2 * r * c * 2 + r * 4)
+            w["next.loss_grad"] = dict(bytes=3 * r * c * 2 + 2 * r * 4)
+            w["next.sgd"] = dict(bytes=sum(3 * p.numel() * 2 for p in self.sgd_params))
         return w
 
 
@@ -443,6 +470,12 @@ def main():
             a = table[key]["gbs"]
             rooflines[name] = {"bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": a / peaks["hbm_gbs"],
                                "traffic": traffic_of(key), "peak_source": peaks["source"] + " (of measured)"}
+    for key, name in (("next.loss", "softmax_xent_kernel (loss)"), ("next.loss_grad", "softmax_xent_kernel (loss + partial)"),
+                      ("next.sgd", "sgd_update_kernel (3 x 4096^2 bf16)")):
+        if key in table:
+            a = table[key]["gbs"]
+            rooflines[name] = {"bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": a / peaks["hbm_gbs"],
+                               "traffic": traffic_of(key), "peak_source": peaks["source"] + " (of measured)"}
     if rooflines:
         first = next(iter(rooflines))
         roofline = dict(rooflines[first], kernel=first)
@@ -466,7 +499,7 @@ def main():
         flop_all = sum(work[k]["flop"] for k in tensor_keys)
         e2e = {"value": world * flop_all / (e_ms * 1e-3) / 1e12 if flop_all else None, "unit": "TFLOP/s", "ms_per_step": e_ms,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-               "note": "whole step incl. L2 flushes and all five configurations; dense+conv FLOPs over that time"}
+               "note": "whole step incl. L2 flushes and all groups; dense+conv FLOPs over that time"}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -480,7 +513,8 @@ def main():
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 (fp32 accumulate); cfg1 f32",
                 "data": "synthetic",
                 "config": {"workload": ("reduced shapes" if args.small else "all five configurations at full size")
-                           + ": step = cfg1 fwd+grad, cfg2 fwd+grad, cfg3 3-layer fwd+bwd, cfg4 conv fwd+dX+dW+db, cfg5 LSTM",
+                           + ": step = cfg1 fwd+grad, cfg2 fwd+grad, cfg3 3-layer fwd+bwd, cfg4 conv fwd+dX+dW+db, cfg5 LSTM"
+                           + ", then softmax cross-entropy loss / loss+partial on 8192x8192 bf16 and SGD on three 4096^2 bf16 matrices",
                            "value_covers": "dense + conv2d groups (cfg3 + cfg4) FLOPs / their device time; hbm_gbs covers cfg2",
                            "groups": groups, "l2": "1 GiB streamed through L2 between groups (flush with clean lines); cfg2 inputs also exceed L2",
                            "replicas": world},

@@ -41,49 +41,109 @@ __device__ __forceinline__ void store_vals(T *p, const float (&f)[V])
     }
 }
 
+// V consecutive values kept as loaded (packed), so that a cached bf16 vector costs 4 registers, not 8
+template <typename TT, int V>
+struct Raw {
+    static constexpr int N = (sizeof(TT) * V + 15) / 16;
+    uint4 q[N];
+};
+template <typename TT>
+struct Raw<TT, 1> {
+    float q[1];
+};
+template <typename TT, int V>
+__device__ __forceinline__ void load_raw(const TT *p, Raw<TT, V> &r)
+{
+    if constexpr (V == 1) {
+        load_vals<TT, 1>(p, r.q);
+    } else {
+#pragma unroll
+        for (int i = 0; i < Raw<TT, V>::N; ++i) r.q[i] = ld_stream(reinterpret_cast<const uint4 *>(p) + i);
+    }
+}
+template <typename TT, int V>
+__device__ __forceinline__ void to_float(const Raw<TT, V> &r, float (&f)[V])
+{
+    if constexpr (V == 1) {
+        f[0] = r.q[0];
+    } else if constexpr (Raw<TT, V>::N == 1) {
+        unpack(r.q[0], f);
+    } else {
+        float a[4], b[4];
+        unpack(r.q[0], a);
+        unpack(r.q[1], b);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { f[i] = a[i]; f[4 + i] = b[i]; }
+    }
+}
+
 template <bool FAST> __device__ __forceinline__ float exp_(float x) { return FAST ? __expf(x) : expf(x); }
 template <bool FAST> __device__ __forceinline__ float log_(float x) { return FAST ? __logf(x) : logf(x); }
 
-// Running state of one row part: maximum m, s = sum exp(z - m), st = sum t, stz = sum t (z - m).
-struct RowState {
-    float m, s, st, stz;
-};
-template <bool FAST>
-__device__ __forceinline__ void rebase(RowState &a, float m_new)
+// largest of the V values of a packed vector
+template <typename T, int V>
+__device__ __forceinline__ float raw_max(const Raw<T, V> &r)
 {
-    if (a.m != -INFINITY && m_new != a.m) {        // an empty part (m = -inf) holds zeros and needs no shift
-        a.s *= exp_<FAST>(a.m - m_new);
-        a.stz -= (m_new - a.m) * a.st;
-    }
-    a.m = m_new;
-}
-template <bool FAST>
-__device__ __forceinline__ RowState merge(RowState a, RowState b)
-{
-    const float m = fmaxf(a.m, b.m);
-    rebase<FAST>(a, m);
-    rebase<FAST>(b, m);
-    return RowState{m, a.s + b.s, a.st + b.st, a.stz + b.stz};
-}
-template <bool FAST, int V>
-__device__ __forceinline__ void absorb(RowState &a, const float (&z)[V], const float (&t)[V])
-{
-    float vm = z[0];
+    if constexpr (V == 1) {
+        return r.q[0];
+    } else if constexpr (sizeof(T) == 2) {          // bf16 pairs: the maximum of bf16 values is exact in bf16
+        const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&r.q[0]);
+        const __nv_bfloat162 m = __hmax2(__hmax2(h[0], h[1]), __hmax2(h[2], h[3]));
+        return fmaxf(__low2float(m), __high2float(m));
+    } else {
+        float f[V];
+        to_float<T, V>(r, f);
+        float m = f[0];
 #pragma unroll
-    for (int j = 1; j < V; ++j) vm = fmaxf(vm, z[j]);
-    if (vm > a.m) rebase<FAST>(a, vm);
-#pragma unroll
-    for (int j = 0; j < V; ++j) {
-        const float d = z[j] - a.m;
-        a.s += exp_<FAST>(d);
-        a.st += t[j];
-        a.stz = fmaf(t[j], d, a.stz);
+        for (int j = 1; j < V; ++j) m = fmaxf(m, f[j]);
+        return m;
     }
 }
 
-// One row per TPR threads (a warp, or the whole block).  Pass 1 reads z and t once, keeps the first kCache
-// vectors of each thread in registers and folds everything into a RowState; the states are merged in a
-// fixed order; pass 2 (gradient only) writes dz from the registers and re-reads what did not fit.
+// Combines one value per thread over the TPR threads of a row; every thread gets the result.
+// `slot` is a shared array of kThreads / 32 floats used by the block-wide form only.
+template <int TPR, bool MAX>
+__device__ __forceinline__ float row_combine(float v, float *slot)
+{
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const float o = __shfl_xor_sync(0xffffffffu, v, off);
+        v = MAX ? fmaxf(v, o) : v + o;
+    }
+    if constexpr (TPR > 32) {
+        if ((threadIdx.x & 31) == 0) slot[threadIdx.x >> 5] = v;
+        __syncthreads();
+        v = slot[0];
+#pragma unroll
+        for (int w = 1; w < kThreads / 32; ++w) v = MAX ? fmaxf(v, slot[w]) : v + slot[w];     // fixed order
+    }
+    return v;
+}
+
+// Sums of three values at once (one barrier for the three); `slot` holds 3 * kThreads / 32 floats.
+template <int TPR>
+__device__ __forceinline__ void row_sum3(float &a, float &b, float &c, float *slot)
+{
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        a += __shfl_xor_sync(0xffffffffu, a, off);
+        b += __shfl_xor_sync(0xffffffffu, b, off);
+        c += __shfl_xor_sync(0xffffffffu, c, off);
+    }
+    if constexpr (TPR > 32) {
+        constexpr int W = kThreads / 32;
+        if ((threadIdx.x & 31) == 0) { slot[threadIdx.x >> 5] = a; slot[W + (threadIdx.x >> 5)] = b; slot[2 * W + (threadIdx.x >> 5)] = c; }
+        __syncthreads();
+        a = slot[0]; b = slot[W]; c = slot[2 * W];
+#pragma unroll
+        for (int w = 1; w < W; ++w) { a += slot[w]; b += slot[W + w]; c += slot[2 * W + w]; }     // fixed order
+    }
+}
+
+// One row per TPR threads (a warp, or the whole block).  z and t are read once: the first kCache vectors
+// of each thread stay packed in registers, and only rows longer than TPR * kCache vectors re-read the
+// rest (from L2).  Phase A: row maximum m.  Phase B: s = sum exp(z - m), st = sum t, stz = sum t (z - m);
+// loss = st log s - stz.  Phase C (gradient only): dz = dl (exp(z - m) st / s - t).
 template <typename T, typename TT, int TPR, bool VEC, bool GRAD>
 __global__ void __launch_bounds__(kThreads)
 softmax_xent_kernel(const T *__restrict__ z, const TT *__restrict__ t, const float *__restrict__ dloss, float *__restrict__ loss,
@@ -92,74 +152,91 @@ softmax_xent_kernel(const T *__restrict__ z, const TT *__restrict__ t, const flo
     constexpr bool FAST = sizeof(T) == 2;
     constexpr int V = VEC ? VecN<T>::N : 1;
     constexpr int RPB = kThreads / TPR;
-    __shared__ RowState part[kThreads / 32];
+    __shared__ float slots[4][kThreads / 32];
     const int lane = threadIdx.x % TPR;
     const int64_t row = (int64_t)blockIdx.x * RPB + threadIdx.x / TPR;
     const bool live = row < B;
     const int64_t nvec = C / V;
+    const int64_t rest0 = lane + (int64_t)kCache * TPR;
     pdl_wait();
 
     const T *zr = z + (live ? row : 0) * C;
     const TT *tr = t + (live ? row : 0) * C;
-    float zc[kCache][V], tc[kCache][V];
-    RowState a{-INFINITY, 0.0f, 0.0f, 0.0f};
+    Raw<T, V> zc[kCache];
+    Raw<TT, V> tc[kCache];
+    float m = -INFINITY;
+    if (live) {
+#pragma unroll
+        for (int k = 0; k < kCache; ++k) {                  // all loads of the thread are issued before any use
+            const int64_t vi = lane + (int64_t)k * TPR;
+            if (vi < nvec) {
+                load_raw<T, V>(zr + vi * V, zc[k]);
+                load_raw<TT, V>(tr + vi * V, tc[k]);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < kCache; ++k)
+            if (lane + (int64_t)k * TPR < nvec) m = fmaxf(m, raw_max<T, V>(zc[k]));
+        for (int64_t vi = rest0; vi < nvec; vi += TPR) {
+            Raw<T, V> r;
+            load_raw<T, V>(zr + vi * V, r);
+            m = fmaxf(m, raw_max<T, V>(r));
+        }
+    }
+    m = row_combine<TPR, true>(m, slots[0]);
+
+    float s = 0.0f, st = 0.0f, stz = 0.0f;
+    auto sums = [&](const float (&zz)[V], const float (&tt)[V]) {
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+            const float d = zz[j] - m;
+            s += exp_<FAST>(d);
+            st += tt[j];
+            stz = fmaf(tt[j], d, stz);
+        }
+    };
     if (live) {
 #pragma unroll
         for (int k = 0; k < kCache; ++k) {
-            const int64_t vi = lane + (int64_t)k * TPR;
-            if (vi < nvec) {
-                load_vals<T, V>(zr + vi * V, zc[k]);
-                load_vals<TT, V>(tr + vi * V, tc[k]);
-                absorb<FAST, V>(a, zc[k], tc[k]);
+            if (lane + (int64_t)k * TPR < nvec) {
+                float zz[V], tt[V];
+                to_float<T, V>(zc[k], zz);
+                to_float<TT, V>(tc[k], tt);
+                sums(zz, tt);
             }
         }
-        for (int64_t vi = lane + (int64_t)kCache * TPR; vi < nvec; vi += TPR) {
+        for (int64_t vi = rest0; vi < nvec; vi += TPR) {
             float zz[V], tt[V];
             load_vals<T, V>(zr + vi * V, zz);
             load_vals<TT, V>(tr + vi * V, tt);
-            absorb<FAST, V>(a, zz, tt);
+            sums(zz, tt);
         }
     }
-    // merge over the threads of the row: butterfly inside a warp (every lane ends with the same state)
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        RowState b;
-        b.m = __shfl_xor_sync(0xffffffffu, a.m, off);
-        b.s = __shfl_xor_sync(0xffffffffu, a.s, off);
-        b.st = __shfl_xor_sync(0xffffffffu, a.st, off);
-        b.stz = __shfl_xor_sync(0xffffffffu, a.stz, off);
-        a = (threadIdx.x & off) ? merge<FAST>(b, a) : merge<FAST>(a, b);     // same operand order in both partners
-    }
-    if constexpr (TPR > 32) {
-        if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = a;
-        __syncthreads();
-        a = part[0];
-#pragma unroll
-        for (int w = 1; w < kThreads / 32; ++w) a = merge<FAST>(a, part[w]);
-    }
+    row_sum3<TPR>(s, st, stz, slots[1]);
     if (!live) return;
-    const float log_s = log_<FAST>(a.s);
-    if (loss != nullptr && lane == 0) loss[row] = fmaf(a.st, log_s, -a.stz);     // sum t (log s - (z - m))
+    if (loss != nullptr && lane == 0) loss[row] = fmaf(st, log_<FAST>(s), -stz);     // sum t (log s - (z - m))
     if constexpr (GRAD) {
         const float dl = dloss[row];
-        const float scale = dl * a.st / a.s;                                     // dl * sum t / sum exp
+        const float scale = dl * st / s;                                             // dl * sum t / sum exp
         T *dr = dz + row * C;
 #pragma unroll
         for (int k = 0; k < kCache; ++k) {
             const int64_t vi = lane + (int64_t)k * TPR;
             if (vi < nvec) {
-                float o[V];
+                float zz[V], tt[V], o[V];
+                to_float<T, V>(zc[k], zz);
+                to_float<TT, V>(tc[k], tt);
 #pragma unroll
-                for (int j = 0; j < V; ++j) o[j] = fmaf(scale, exp_<FAST>(zc[k][j] - a.m), -dl * tc[k][j]);
+                for (int j = 0; j < V; ++j) o[j] = fmaf(scale, exp_<FAST>(zz[j] - m), -dl * tt[j]);
                 store_vals<T, V>(dr + vi * V, o);
             }
         }
-        for (int64_t vi = lane + (int64_t)kCache * TPR; vi < nvec; vi += TPR) {
+        for (int64_t vi = rest0; vi < nvec; vi += TPR) {
             float zz[V], tt[V], o[V];
             load_vals<T, V>(zr + vi * V, zz);
             load_vals<TT, V>(tr + vi * V, tt);
 #pragma unroll
-            for (int j = 0; j < V; ++j) o[j] = fmaf(scale, exp_<FAST>(zz[j] - a.m), -dl * tt[j]);
+            for (int j = 0; j < V; ++j) o[j] = fmaf(scale, exp_<FAST>(zz[j] - m), -dl * tt[j]);
             store_vals<T, V>(dr + vi * V, o);
         }
     }
