@@ -286,6 +286,37 @@ def softmax_xent_grad(z, t, dloss, loss_dtype: int = F64, dz_dtype: int = F64):
     return loss, dz
 
 
+def max_pool2d(x, kh: int, kw: int, sh: int, sw: int):
+    """(y, idx): window maxima of an NCHW tensor and the in-plane position h*W+w of the first maximum
+    (Fig. 3, relay.max_pool)."""
+    x = _f64(x)
+    Nb, C, H, W = x.shape
+    if kh > H or kw > W or min(kh, kw, sh, sw) <= 0:
+        raise ValueError("window does not fit")
+    P, Q = (H - kh) // sh + 1, (W - kw) // sw + 1
+    y = np.empty((Nb, C, P, Q), dtype=np.float64)
+    idx = np.empty((Nb, C, P, Q), dtype=np.int32)
+    i64 = ctypes.c_int64
+    rc = _L().orc_max_pool2d(_ptr(x), i64(Nb), i64(C), i64(H), i64(W), i64(kh), i64(kw), i64(sh), i64(sw), _ptr(y),
+                             idx.ctypes.data_as(_i32p))
+    assert rc == 0
+    return y, idx
+
+
+def max_pool2d_grad(idx, dy, H: int, W: int, dx_dtype: int = F64) -> np.ndarray:
+    idx = np.asarray(idx, dtype=np.int32, order="C")
+    dy = _f64(dy)
+    Nb, C, P, Q = dy.shape
+    assert idx.shape == dy.shape
+    dx = np.empty((Nb, C, H, W), dtype=np.float64)
+    i64 = ctypes.c_int64
+    rc = _L().orc_max_pool2d_grad(idx.ctypes.data_as(_i32p), _ptr(dy), i64(Nb), i64(C), i64(H), i64(W), i64(P), i64(Q),
+                                  int(dx_dtype), _ptr(dx))
+    if rc != 0:
+        raise ValueError("index outside the plane")
+    return dx
+
+
 def sgd_update(p, g, lr: float, p_dtype: int = F64) -> np.ndarray:
     """p - lr * g stored in p_dtype (Section 4.1, relay.update_model_params)."""
     p, g = _f64(p), _f64(g)

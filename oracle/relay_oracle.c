@@ -420,6 +420,52 @@ int orc_softmax_xent_grad(const double *z, const double *t, const double *dloss,
 }
 
 /* ------------------------------------------------------------------------------------------
+ * Max pooling over windows of an NCHW tensor (Fig. 3, relay.max_pool(x, ksize, strides)), no padding:
+ *   y[n,c,p,q]   = max_{r<kh, s<kw} x[n,c,p*sh+r, q*sw+s]
+ *   idx[n,c,p,q] = (p*sh+r)*W + (q*sw+s) of the FIRST maximum in (r,s) row-major order
+ * with P = floor((H-kh)/sh)+1, Q = floor((W-kw)/sw)+1.  idx may be NULL.  Returns 1 if a window does
+ * not fit (kh > H or kw > W) or an attribute is not positive.
+ * ---------------------------------------------------------------------------------------- */
+int orc_max_pool2d(const double *x, int64_t Nb, int64_t C, int64_t H, int64_t W, int64_t kh, int64_t kw,
+                   int64_t sh, int64_t sw, double *y, int32_t *idx)
+{
+    if (kh <= 0 || kw <= 0 || sh <= 0 || sw <= 0 || kh > H || kw > W) return 1;
+    int64_t P = (H - kh) / sh + 1, Q = (W - kw) / sw + 1;
+    for (int64_t nc = 0; nc < Nb * C; ++nc) {
+        const double *xp = x + nc * H * W;
+        for (int64_t p = 0; p < P; ++p)
+            for (int64_t q = 0; q < Q; ++q) {
+                int64_t best = (p * sh) * W + q * sw;
+                for (int64_t r = 0; r < kh; ++r)
+                    for (int64_t t = 0; t < kw; ++t) {
+                        int64_t at = (p * sh + r) * W + (q * sw + t);
+                        if (xp[at] > xp[best]) best = at;        /* strict: the first maximum wins */
+                    }
+                y[(nc * P + p) * Q + q] = xp[best];
+                if (idx) idx[(nc * P + p) * Q + q] = (int32_t)best;
+            }
+    }
+    return 0;
+}
+
+/* Gradient of max pooling (Section 4.2): the partial of every input starts at zero and each window adds
+ * its dy to the input that attained the maximum (idx from the forward pass), windows visited in (p,q)
+ * order:  dx[n,c,idx[n,c,p,q]] += dy[n,c,p,q].  Stored in dx_dtype. */
+int orc_max_pool2d_grad(const int32_t *idx, const double *dy, int64_t Nb, int64_t C, int64_t H, int64_t W,
+                        int64_t P, int64_t Q, int dx_dtype, double *dx)
+{
+    for (int64_t i = 0; i < Nb * C * H * W; ++i) dx[i] = 0.0;
+    for (int64_t nc = 0; nc < Nb * C; ++nc)
+        for (int64_t o = 0; o < P * Q; ++o) {
+            int32_t at = idx[nc * P * Q + o];
+            if (at < 0 || at >= H * W) return 1;
+            dx[nc * H * W + at] += dy[nc * P * Q + o];
+        }
+    for (int64_t i = 0; i < Nb * C * H * W; ++i) dx[i] = orc_cast(dx[i], dx_dtype);
+    return 0;
+}
+
+/* ------------------------------------------------------------------------------------------
  * Parameter update (Section 4.1, relay.update_model_params: vanilla stochastic gradient descent, the one
  * place where the paper allows mutation):  p <- cast( p - lr * g ), elementwise, stored in p's dtype.
  * ---------------------------------------------------------------------------------------- */
