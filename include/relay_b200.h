@@ -133,6 +133,12 @@ typedef struct relay_conv2d_attrs {
     int32_t groups;   /* must be 1 */
 } relay_conv2d_attrs_t;
 
+/* Pooling window (Fig. 3: relay.max_pool(x, ksize=[1,kh,kw,1], strides=[1,sh,sw,1])); no padding. */
+typedef struct {
+    int32_t kh, kw;   /* window extent, >= 1, not larger than the plane */
+    int32_t sh, sw;   /* stride, >= 1 */
+} relay_pool2d_attrs_t;
+
 /* ---------------------------------------------------------------------------------------------
  * Type relations, host only (no GPU needed).  Each fills `out` (dtype, rank, shape, layout;
  * data = NULL) with the result type the operator's relation gives for the argument types,
@@ -302,6 +308,25 @@ relay_status_t relay_softmax_xent(const relay_tensor_t *scores, const relay_tens
  * and, if `loss` is not NULL, loss:(B) f32 as above, from the same pass over z and t. */
 relay_status_t relay_softmax_xent_grad(const relay_tensor_t *scores, const relay_tensor_t *targets, const relay_tensor_t *dloss,
                                        const relay_tensor_t *loss, const relay_tensor_t *dscores, void *stream);
+
+/* Max pooling of an NCHW tensor (Fig. 3 relay.max_pool), windows without padding:
+ *   y[n,c,p,q]   = max_{r<kh, s<kw} x[n,c,p*sh+r, q*sw+s],   P = floor((H-kh)/sh)+1, Q = floor((W-kw)/sw)+1
+ *   idx[n,c,p,q] = (p*sh+r)*W + (q*sw+s) of the first maximum in (r,s) row-major order   (i32, optional)
+ *   x:(N,C,H,W) f32 or bf16, NCHW;  y:(N,C,P,Q) same base type;  idx:(N,C,P,Q) i32 or NULL.
+ * y and idx are bit-exact functions of x.  H*W must fit an i32.  RELAY_ERR_ATTR for a window that is not
+ * positive or does not fit the plane. */
+relay_status_t relay_infer_max_pool2d(const relay_tensor_t *x, const relay_pool2d_attrs_t *attrs, relay_tensor_t *out);
+relay_status_t relay_max_pool2d(const relay_tensor_t *x, const relay_pool2d_attrs_t *attrs, const relay_tensor_t *y,
+                                const relay_tensor_t *idx, void *stream);
+
+/* Gradient of max pooling (Section 4.2): each window adds its dy to the input that attained the maximum,
+ * every other input gets zero:  dx[n,c,h,w] = sum over the windows (p,q) with idx[n,c,p,q] = h*W+w of dy[n,c,p,q],
+ * summed in (p,q) order (deterministic; overlapping windows may name the same input).
+ *   idx:(N,C,P,Q) i32 from the forward call;  dy:(N,C,P,Q);  dx:(N,C,H,W) of dy's base type, with the same
+ *   attrs as the forward call (P and Q must be what they give for dx's H and W).
+ * An idx entry outside its window contributes nothing. */
+relay_status_t relay_max_pool2d_grad(const relay_tensor_t *idx, const relay_tensor_t *dy, const relay_pool2d_attrs_t *attrs,
+                                     const relay_tensor_t *dx, void *stream);
 
 /* Vanilla stochastic gradient descent on a set of parameters (Section 4.1: update_model_params is the one
  * place where the paper exposes mutation): for k < n_params, elementwise and IN PLACE,

@@ -62,6 +62,10 @@ class Conv2dAttrs(ctypes.Structure):
 _lib = None
 
 
+class Pool2dAttrs(ctypes.Structure):
+    _fields_ = [("kh", ctypes.c_int32), ("kw", ctypes.c_int32), ("sh", ctypes.c_int32), ("sw", ctypes.c_int32)]
+
+
 def lib() -> ctypes.CDLL:
     """Loads the library; fails loudly if it has not been built."""
     global _lib
@@ -199,6 +203,13 @@ def relay_infer_softmax_xent(scores: TensorDesc, targets: TensorDesc) -> TensorD
     return out
 
 
+def relay_infer_max_pool2d(x: TensorDesc, kh: int, kw: int, sh: int, sw: int) -> TensorDesc:
+    out = TensorDesc()
+    at = Pool2dAttrs(kh, kw, sh, sw)
+    _check(lib().relay_infer_max_pool2d(_ref(x), ctypes.byref(at), ctypes.byref(out)))
+    return out
+
+
 def relay_infer_ewise(prog: dict, inputs: Sequence[TensorDesc], value: int) -> TensorDesc:
     out = TensorDesc()
     p = make_prog(prog)
@@ -310,6 +321,16 @@ def relay_softmax_xent(scores, targets, loss):
 def relay_softmax_xent_grad(scores, targets, dloss, loss, dscores):
     _check(lib().relay_softmax_xent_grad(_ref(desc(scores)), _ref(desc(targets)), _ref(desc(dloss)), _ref(desc(loss)),
                                          _ref(desc(dscores)), _stream()))
+
+
+def relay_max_pool2d(x, kh, kw, sh, sw, y, idx=None):
+    at = Pool2dAttrs(kh, kw, sh, sw)
+    _check(lib().relay_max_pool2d(_ref(desc(x, NCHW)), ctypes.byref(at), _ref(desc(y, NCHW)), _ref(desc(idx, NCHW)), _stream()))
+
+
+def relay_max_pool2d_grad(idx, dy, kh, kw, sh, sw, dx):
+    at = Pool2dAttrs(kh, kw, sh, sw)
+    _check(lib().relay_max_pool2d_grad(_ref(desc(idx, NCHW)), _ref(desc(dy, NCHW)), ctypes.byref(at), _ref(desc(dx, NCHW)), _stream()))
 
 
 def relay_sgd_update(params, grads, lr: float):

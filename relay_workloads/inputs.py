@@ -107,3 +107,10 @@ def param_set(shapes, dtype=torch.bfloat16, grad_dtype=None, salt=0):
     ps = [normal(7, 2 * i, s, 0.05, dtype, salt) for i, s in enumerate(shapes)]
     gs = [normal(7, 2 * i + 1, s, 1.0, grad_dtype, salt) for i, s in enumerate(shapes)]
     return ps, gs
+
+
+def pool_input(N=32, C=256, H=56, W=56, dtype=torch.bfloat16, levels=0, salt=0) -> torch.Tensor:
+    """Activations to pool: N(0,1) values, or (levels > 0) integers in [0, levels) so that windows hold ties."""
+    if levels:
+        return _store(_rng(8, 0, salt).integers(0, levels, (N, C, H, W)).astype(np.float64), dtype)
+    return normal(8, 0, (N, C, H, W), 1.0, dtype, salt)

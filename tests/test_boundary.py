@@ -272,3 +272,22 @@ def test_sgd_update_descriptor_checks_run_before_any_launch():
     assert status_of([ok_p], [T(B.F32, (4, 7))]) == "ERR_SHAPE"
     assert status_of([ok_p], [ok_g]) == "ERR_NULL"                                # descriptors without data
     assert B.relay_launch_count() == n0
+
+
+def test_infer_max_pool2d_counts_windows_and_rejects_bad_windows():
+    for H, W, kh, kw, sh, sw in itertools.product((1, 4, 7), (2, 5, 8), (1, 2, 3), (1, 2), (1, 2, 3), (1, 2)):
+        x = T(B.BF16, (2, 3, H, W), B.NCHW)
+        if kh > H or kw > W:
+            with pytest.raises(B.RelayError) as e:
+                B.relay_infer_max_pool2d(x, kh, kw, sh, sw)
+            assert e.value.status_name == "ERR_ATTR"
+            continue
+        out = B.relay_infer_max_pool2d(x, kh, kw, sh, sw)
+        P = len([p for p in range(H) if p * sh + kh <= H])
+        Q = len([q for q in range(W) if q * sw + kw <= W])
+        assert B._shape(out) == (2, 3, P, Q) and out.dtype == B.BF16
+    for x, k, status in [(T(B.F32, (2, 3, 4)), (2, 2, 2, 2), "ERR_RANK"), (T(B.I32, (1, 1, 4, 4)), (2, 2, 2, 2), "ERR_DTYPE"),
+                         (T(B.F32, (1, 1, 4, 4)), (0, 2, 2, 2), "ERR_ATTR"), (T(B.F32, (1, 1, 4, 4)), (2, 2, 2, -1), "ERR_ATTR")]:
+        with pytest.raises(B.RelayError) as e:
+            B.relay_infer_max_pool2d(x, *k)
+        assert e.value.status_name == status
