@@ -114,3 +114,16 @@ def pool_input(N=32, C=256, H=56, W=56, dtype=torch.bfloat16, levels=0, salt=0) 
     if levels:
         return _store(_rng(8, 0, salt).integers(0, levels, (N, C, H, W)).astype(np.float64), dtype)
     return normal(8, 0, (N, C, H, W), 1.0, dtype, salt)
+
+
+def lenet_batch(N=16, dtype=torch.float32, salt=0) -> Dict[str, torch.Tensor]:
+    """One batch for the LeNet-shaped model of the paper's listing: images U(0,1) [N,1,28,28], one-hot labels
+    [N,10], parameters N(0, 0.1) (the listing initialises every parameter as a small Gaussian)."""
+    r = _rng(9, 1, salt)
+    labels = np.zeros((N, 10))
+    labels[np.arange(N), r.integers(0, 10, N)] = 1.0
+    shapes = dict(w1=(20, 1, 5, 5), b1=(20,), w2=(50, 20, 5, 5), b2=(50,), w3=(800, 500), b3=(500,), w4=(500, 10), b4=(10,))
+    d = dict(x=uniform(9, 0, (N, 1, 28, 28), 0.0, 1.0, dtype, salt), labels=_store(labels, dtype))
+    for i, (k, s) in enumerate(shapes.items()):
+        d[k] = normal(9, 2 + i, s, 0.1, dtype, salt)
+    return d
