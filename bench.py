@@ -183,6 +183,12 @@ class Workload:
             n = 256 if small else 4096
             ps, gs = I.param_set([(n, n)] * 3, torch.bfloat16, torch.bfloat16)
             self.sgd_params, self.sgd_grads = [p.to(dev) for p in ps], [g.to(dev) for g in gs]
+            # max pooling 2x2 stride 2 of an activation of the conv configuration's shape (device-resident)
+            shp = (2, 32, 14, 16) if small else (32, 256, 56, 56)
+            self.pool_x = I.pool_input(*shp).to(dev)
+            ps_ = (shp[0], shp[1], shp[2] // 2, shp[3] // 2)
+            self.pool_y, self.pool_idx = E(*ps_), E(*ps_, dt=torch.int32)
+            self.pool_dy, self.pool_dx = I.normal(8, 1, ps_, 1.0, torch.bfloat16).to(dev), torch.empty_like(self.pool_x)
         self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
         self.flush_buf = torch.zeros(1024 * 1024 * 1024, dtype=torch.uint8, device=dev)
         self.pinned_out = {g: {k: torch.empty_like(v, device="cpu").pin_memory() for k, v in o.items()} for g, o in self.out.items()}
@@ -266,6 +272,12 @@ class Workload:
             self.flush_l2()
             with tm.region("next.sgd"):
                 B.relay_sgd_update(self.sgd_params, self.sgd_grads, 1e-3)
+            self.flush_l2()
+            with tm.region("next.pool"):
+                B.relay_max_pool2d(self.pool_x, 2, 2, 2, 2, self.pool_y, self.pool_idx)
+            self.flush_l2()
+            with tm.region("next.pool_grad"):
+                B.relay_max_pool2d_grad(self.pool_idx, self.pool_dy, 2, 2, 2, 2, self.pool_dx)
 
     # -- algorithmic work per step -------------------------------------------------------------------------
     def work(self):
@@ -294,6 +306,8 @@ class Workload:
             w["next.loss"] = dict(bytes=2 * r * c * 2 + r * 4)
             w["next.loss_grad"] = dict(bytes=3 * r * c * 2 + 2 * r * 4)
             w["next.sgd"] = dict(bytes=sum(3 * p.numel() * 2 for p in self.sgd_params))
+            pool_bytes = self.pool_x.numel() * 2 + self.pool_y.numel() * (2 + 4)
+            w["next.pool"] = dict(bytes=pool_bytes); w["next.pool_grad"] = dict(bytes=pool_bytes)
         return w
 
 
@@ -471,7 +485,8 @@ def main():
             rooflines[name] = {"bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": a / peaks["hbm_gbs"],
                                "traffic": traffic_of(key), "peak_source": peaks["source"] + " (of measured)"}
     for key, name in (("next.loss", "softmax_xent_kernel (loss)"), ("next.loss_grad", "softmax_xent_kernel (loss + partial)"),
-                      ("next.sgd", "sgd_update_kernel (3 x 4096^2 bf16)")):
+                      ("next.sgd", "sgd_update_kernel (3 x 4096^2 bf16)"), ("next.pool", "max_pool_2x2_kernel (32x256x56x56 bf16)"),
+                      ("next.pool_grad", "max_pool_2x2_grad_kernel (32x256x56x56 bf16)")):
         if key in table:
             a = table[key]["gbs"]
             rooflines[name] = {"bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": a / peaks["hbm_gbs"],

@@ -95,38 +95,53 @@ __device__ __forceinline__ void store8(T *p, const float (&f)[8])
     }
 }
 
+constexpr int kPer = 1;            // items a thread of the 2 x 2 kernels keeps in flight
+
 template <typename T>
 __global__ void __launch_bounds__(kThreads) max_pool_2x2_kernel(const T *__restrict__ x, T *__restrict__ y, int32_t *__restrict__ idx, PoolDims d)
 {
     const int groups = d.W >> 3;                              // threads per output row; Q = 4 * groups
     const int64_t total = d.planes * d.P * groups;
     pdl_wait();
-    for (int64_t t = (int64_t)blockIdx.x * kThreads + threadIdx.x; t < total; t += (int64_t)gridDim.x * kThreads) {
-        const int g = (int)(t % groups), p = (int)((t / groups) % d.P);
-        const int64_t plane = t / ((int64_t)groups * d.P);
-        const T *r0 = x + (plane * d.H + 2 * p) * d.W + 8 * g;
-        float a[8], b[8];
-        load8<T>(r0, a);
-        load8<T>(r0 + d.W, b);
-        const int base = (2 * p) * d.W + 8 * g;
-        float out[4];
-        int where[4];
+    for (int64_t t0 = (int64_t)blockIdx.x * (kThreads * kPer) + threadIdx.x; t0 < total; t0 += (int64_t)gridDim.x * (kThreads * kPer)) {
+        float a[kPer][8], b[kPer][8];
+        int base[kPer];
+        int64_t o[kPer];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {                         // window order: (0,0) (0,1) (1,0) (1,1), first maximum wins
-            float bv = a[2 * j];
-            int at = base + 2 * j;
-            if (a[2 * j + 1] > bv) { bv = a[2 * j + 1]; at = base + 2 * j + 1; }
-            if (b[2 * j] > bv) { bv = b[2 * j]; at = base + d.W + 2 * j; }
-            if (b[2 * j + 1] > bv) { bv = b[2 * j + 1]; at = base + d.W + 2 * j + 1; }
-            out[j] = bv; where[j] = at;
+        for (int u = 0; u < kPer; ++u) {                      // all loads first
+            const int64_t t = t0 + (int64_t)u * kThreads;
+            if (t < total) {
+                const int g = (int)(t % groups), p = (int)((t / groups) % d.P);
+                const int64_t plane = t / ((int64_t)groups * d.P);
+                const T *r0 = x + (plane * d.H + 2 * p) * d.W + 8 * g;
+                load8<T>(r0, a[u]);
+                load8<T>(r0 + d.W, b[u]);
+                base[u] = (2 * p) * d.W + 8 * g;
+                o[u] = (plane * d.P + p) * d.Q + 4 * g;
+            }
         }
-        const int64_t o = (plane * d.P + p) * d.Q + 4 * g;
-        if constexpr (sizeof(T) == 2) {
-            *reinterpret_cast<uint2 *>(y + o) = make_uint2(pack2(out[0], out[1]), pack2(out[2], out[3]));
-        } else {
-            st_stream(y + o, pack(out));
+#pragma unroll
+        for (int u = 0; u < kPer; ++u) {
+            if (t0 + (int64_t)u * kThreads < total) {
+                float out[4];
+                int where[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {                 // window order: (0,0) (0,1) (1,0) (1,1), first maximum wins
+                    float bv = a[u][2 * j];
+                    int at = base[u] + 2 * j;
+                    if (a[u][2 * j + 1] > bv) { bv = a[u][2 * j + 1]; at = base[u] + 2 * j + 1; }
+                    if (b[u][2 * j] > bv) { bv = b[u][2 * j]; at = base[u] + d.W + 2 * j; }
+                    if (b[u][2 * j + 1] > bv) { bv = b[u][2 * j + 1]; at = base[u] + d.W + 2 * j + 1; }
+                    out[j] = bv; where[j] = at;
+                }
+                if constexpr (sizeof(T) == 2) {
+                    *reinterpret_cast<uint2 *>(y + o[u]) = make_uint2(pack2(out[0], out[1]), pack2(out[2], out[3]));
+                } else {
+                    st_stream(y + o[u], pack(out));
+                }
+                if (idx) st_stream(idx + o[u], make_uint4((uint32_t)where[0], (uint32_t)where[1], (uint32_t)where[2], (uint32_t)where[3]));
+            }
         }
-        if (idx) st_stream(idx + o, make_uint4((uint32_t)where[0], (uint32_t)where[1], (uint32_t)where[2], (uint32_t)where[3]));
     }
 }
 
@@ -136,35 +151,50 @@ __global__ void __launch_bounds__(kThreads) max_pool_2x2_grad_kernel(const int32
     const int groups = d.W >> 3;
     const int64_t total = d.planes * d.P * groups;
     pdl_wait();
-    for (int64_t t = (int64_t)blockIdx.x * kThreads + threadIdx.x; t < total; t += (int64_t)gridDim.x * kThreads) {
-        const int g = (int)(t % groups), p = (int)((t / groups) % d.P);
-        const int64_t plane = t / ((int64_t)groups * d.P);
-        const int64_t o = (plane * d.P + p) * d.Q + 4 * g;
-        const uint4 wi = ld_stream(idx + o);
-        const int where[4] = {(int)wi.x, (int)wi.y, (int)wi.z, (int)wi.w};
-        float g4[4];
-        if constexpr (sizeof(T) == 2) {
-            const uint2 v = *reinterpret_cast<const uint2 *>(dy + o);
-            g4[0] = __uint_as_float(v.x << 16); g4[1] = __uint_as_float(v.x & 0xffff0000u);
-            g4[2] = __uint_as_float(v.y << 16); g4[3] = __uint_as_float(v.y & 0xffff0000u);
-        } else {
-            unpack(ld_stream(dy + o), g4);
-        }
-        const int base = (2 * p) * d.W + 8 * g;
-        float a[8], b[8];
+    for (int64_t t0 = (int64_t)blockIdx.x * (kThreads * kPer) + threadIdx.x; t0 < total; t0 += (int64_t)gridDim.x * (kThreads * kPer)) {
+        uint4 wi[kPer];
+        float g4[kPer][4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            a[2 * j] = where[j] == base + 2 * j ? g4[j] : 0.0f;
-            a[2 * j + 1] = where[j] == base + 2 * j + 1 ? g4[j] : 0.0f;
-            b[2 * j] = where[j] == base + d.W + 2 * j ? g4[j] : 0.0f;
-            b[2 * j + 1] = where[j] == base + d.W + 2 * j + 1 ? g4[j] : 0.0f;
+        for (int u = 0; u < kPer; ++u) {                      // all loads first
+            const int64_t t = t0 + (int64_t)u * kThreads;
+            if (t < total) {
+                const int g = (int)(t % groups), p = (int)((t / groups) % d.P);
+                const int64_t plane = t / ((int64_t)groups * d.P);
+                const int64_t o = (plane * d.P + p) * d.Q + 4 * g;
+                wi[u] = ld_stream(idx + o);
+                if constexpr (sizeof(T) == 2) {
+                    const uint2 v = *reinterpret_cast<const uint2 *>(dy + o);
+                    g4[u][0] = __uint_as_float(v.x << 16); g4[u][1] = __uint_as_float(v.x & 0xffff0000u);
+                    g4[u][2] = __uint_as_float(v.y << 16); g4[u][3] = __uint_as_float(v.y & 0xffff0000u);
+                } else {
+                    unpack(ld_stream(dy + o), g4[u]);
+                }
+            }
         }
-        T *r0 = dx + (plane * d.H + 2 * p) * d.W + 8 * g;
-        store8<T>(r0, a);
-        store8<T>(r0 + d.W, b);
-        if ((d.H & 1) && p == d.P - 1) {                      // the last row of an odd plane lies in no window
-            const float z[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-            store8<T>(r0 + 2 * d.W, z);
+#pragma unroll
+        for (int u = 0; u < kPer; ++u) {
+            const int64_t t = t0 + (int64_t)u * kThreads;
+            if (t < total) {
+                const int g = (int)(t % groups), p = (int)((t / groups) % d.P);
+                const int64_t plane = t / ((int64_t)groups * d.P);
+                const int where[4] = {(int)wi[u].x, (int)wi[u].y, (int)wi[u].z, (int)wi[u].w};
+                const int base = (2 * p) * d.W + 8 * g;
+                float a[8], b[8];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    a[2 * j] = where[j] == base + 2 * j ? g4[u][j] : 0.0f;
+                    a[2 * j + 1] = where[j] == base + 2 * j + 1 ? g4[u][j] : 0.0f;
+                    b[2 * j] = where[j] == base + d.W + 2 * j ? g4[u][j] : 0.0f;
+                    b[2 * j + 1] = where[j] == base + d.W + 2 * j + 1 ? g4[u][j] : 0.0f;
+                }
+                T *r0 = dx + (plane * d.H + 2 * p) * d.W + 8 * g;
+                store8<T>(r0, a);
+                store8<T>(r0 + d.W, b);
+                if ((d.H & 1) && p == d.P - 1) {              // the last row of an odd plane lies in no window
+                    const float z[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+                    store8<T>(r0 + 2 * d.W, z);
+                }
+            }
         }
     }
 }
@@ -240,7 +270,7 @@ extern "C" relay_status_t relay_max_pool2d(const relay_tensor_t *x, const relay_
     cudaStream_t st = (cudaStream_t)stream;
     int32_t *ip = idx ? (int32_t *)idx->data : nullptr;
     if (fast_2x2(d)) {
-        const unsigned grid = grid_for(d.planes * d.P * (d.W / 8));
+        const unsigned grid = grid_for((d.planes * d.P * (d.W / 8) + kPer - 1) / kPer);
         if (x->dtype == RELAY_BF16) RELAY_CUDA(launch_pdl(max_pool_2x2_kernel<__nv_bfloat16>, dim3(grid), dim3(kThreads), 0, st, (const __nv_bfloat16 *)x->data, (__nv_bfloat16 *)y->data, ip, d));
         else RELAY_CUDA(launch_pdl(max_pool_2x2_kernel<float>, dim3(grid), dim3(kThreads), 0, st, (const float *)x->data, (float *)y->data, ip, d));
     } else {
@@ -275,7 +305,7 @@ extern "C" relay_status_t relay_max_pool2d_grad(const relay_tensor_t *idx, const
     cudaStream_t st = (cudaStream_t)stream;
     const int32_t *ip = (const int32_t *)idx->data;
     if (fast_2x2(d)) {
-        const unsigned grid = grid_for(d.planes * d.P * (d.W / 8));
+        const unsigned grid = grid_for((d.planes * d.P * (d.W / 8) + kPer - 1) / kPer);
         if (dx->dtype == RELAY_BF16) RELAY_CUDA(launch_pdl(max_pool_2x2_grad_kernel<__nv_bfloat16>, dim3(grid), dim3(kThreads), 0, st, ip, (const __nv_bfloat16 *)dy->data, (__nv_bfloat16 *)dx->data, d));
         else RELAY_CUDA(launch_pdl(max_pool_2x2_grad_kernel<float>, dim3(grid), dim3(kThreads), 0, st, ip, (const float *)dy->data, (float *)dx->data, d));
     } else {
