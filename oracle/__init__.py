@@ -379,3 +379,23 @@ def lstm_cell_seq(x, w_ih, w_hh, b, h0, c0, rec_dtype: int = BF16, state_dtype: 
     )
     assert rc == 0
     return h_all, c_fin
+
+
+def lstm_cell_seq_grad(x, w_ih, w_hh, b, h0, c0, dh_all, dc_final=None, rec_dtype: int = BF16, state_dtype: int = F32,
+                       dz_dtype: int = BF16):
+    """Partials (dx, dw_ih, dw_hh, db, dh0, dc0) of sum(dh_all * h_all) + sum(dc_final * c_final), as fp64."""
+    x, w_ih, w_hh, b, h0, c0, dh_all = (_f64(v) for v in (x, w_ih, w_hh, b, h0, c0, dh_all))
+    dc_final = None if dc_final is None else _f64(dc_final)
+    T, B, I = x.shape
+    H = h0.shape[1]
+    assert w_ih.shape == (I, 4 * H) and w_hh.shape == (H, 4 * H) and b.shape == (4 * H,)
+    assert h0.shape == (B, H) and c0.shape == (B, H) and dh_all.shape == (T, B, H)
+    assert dc_final is None or dc_final.shape == (B, H)
+    dx, dwi, dwh = np.empty((T, B, I)), np.empty((I, 4 * H)), np.empty((H, 4 * H))
+    db, dh0, dc0 = np.empty((4 * H,)), np.empty((B, H)), np.empty((B, H))
+    i64 = ctypes.c_int64
+    rc = _L().orc_lstm_cell_seq_grad(
+        _ptr(x), _ptr(w_ih), _ptr(w_hh), _ptr(b), _ptr(h0), _ptr(c0), _ptr(dh_all), _ptr(dc_final), i64(T), i64(B), i64(I),
+        i64(H), int(rec_dtype), int(state_dtype), int(dz_dtype), _ptr(dx), _ptr(dwi), _ptr(dwh), _ptr(db), _ptr(dh0), _ptr(dc0))
+    assert rc == 0
+    return dx, dwi, dwh, db, dh0, dc0

@@ -648,6 +648,109 @@ int orc_lstm_cell_seq(const double *x, const double *w_ih, const double *w_hh, c
 }
 
 /* ------------------------------------------------------------------------------------------
+ * Gradient program of the LSTM sequence (Section 4.2, reverse mode through the recursion over time).
+ * Given dh_all[T,B,H] (the partial of the final scalar with respect to every emitted h_t) and
+ * dc_final[B,H] (with respect to the final cell state; NULL = zero), the forward values are recomputed
+ * exactly as orc_lstm_cell_seq computes them and kept per step, then for t = T-1 .. 0:
+ *   dh   = dh_all[t] + dh_next                 (h_t is used twice: emitted, and fed to step t+1)
+ *   do   = dh (.) tanh(c_t);        dc = dc_next + dh (.) o (.) (1 - tanh(c_t)^2)
+ *   di   = dc (.) g;   df = dc (.) c_{t-1};   dg = dc (.) i;   dc_next = dc (.) f
+ *   dz   = cast( [ di i(1-i) | df f(1-f) | dg (1-g^2) | do o(1-o) ], dz_dtype )
+ *   db  += dz;   dx[t] = dz W_ih^T;   dW_ih += x_t^T dz;   dW_hh += hq_t^T dz;   dh_next = dz W_hh^T
+ * and finally dh0 = dh_next, dc0 = dc_next.  hq_t = cast(h_{t-1}, rec_dtype) is the recurrent matmul's
+ * input; the cast is treated as the identity when differentiating.  dz is a typed value (the operand of
+ * four contractions), hence its cast.  Every partial starts from zero.  Any output pointer may be NULL.
+ * Results are stored as fp64 (the caller rounds if it wants a narrower type).
+ * ---------------------------------------------------------------------------------------- */
+int orc_lstm_cell_seq_grad(const double *x, const double *w_ih, const double *w_hh, const double *b,
+                           const double *h0, const double *c0, const double *dh_all, const double *dc_final,
+                           int64_t T, int64_t B, int64_t I, int64_t H, int rec_dtype, int state_dtype, int dz_dtype,
+                           double *dx, double *dw_ih, double *dw_hh, double *db, double *dh0, double *dc0)
+{
+    int64_t G = 4 * H, BH = B * H, BG = B * G;
+    size_t nbh = (size_t)(T * BH ? T * BH : 1), nbg = (size_t)(T * BG ? T * BG : 1);
+    double *hq = (double *)malloc(sizeof(double) * nbh);      /* hq[t] = cast(h_{t-1}) */
+    double *cs = (double *)malloc(sizeof(double) * (nbh + (size_t)(BH ? BH : 1)));   /* cs[0] = c0, cs[t+1] = c_t */
+    double *gt = (double *)malloc(sizeof(double) * nbg);      /* activated gates [i|f|g|o] per step */
+    double *h = (double *)malloc(sizeof(double) * (size_t)(BH ? BH : 1));
+    double *z = (double *)malloc(sizeof(double) * (size_t)(G ? G : 1));
+    double *dz = (double *)malloc(sizeof(double) * (size_t)(BG ? BG : 1));
+    double *dhn = (double *)malloc(sizeof(double) * (size_t)(BH ? BH : 1));
+    double *dcn = (double *)malloc(sizeof(double) * (size_t)(BH ? BH : 1));
+    if (!hq || !cs || !gt || !h || !z || !dz || !dhn || !dcn) {
+        free(hq); free(cs); free(gt); free(h); free(z); free(dz); free(dhn); free(dcn);
+        return -1;
+    }
+    /* forward, as in orc_lstm_cell_seq, keeping what the reverse sweep reads */
+    for (int64_t i = 0; i < BH; ++i) { h[i] = h0[i]; cs[i] = c0[i]; }
+    for (int64_t t = 0; t < T; ++t)
+        for (int64_t bi = 0; bi < B; ++bi) {
+            double *hqr = hq + (t * B + bi) * H, *gr = gt + (t * B + bi) * G;
+            for (int64_t j = 0; j < H; ++j) hqr[j] = orc_cast(h[bi * H + j], rec_dtype);
+            for (int64_t g = 0; g < G; ++g) z[g] = 0.0;
+            for (int64_t k = 0; k < I; ++k)
+                for (int64_t g = 0; g < G; ++g) z[g] += x[(t * B + bi) * I + k] * w_ih[k * G + g];
+            for (int64_t k = 0; k < H; ++k)
+                for (int64_t g = 0; g < G; ++g) z[g] += hqr[k] * w_hh[k * G + g];
+            for (int64_t g = 0; g < G; ++g) z[g] += b[g];
+            for (int64_t j = 0; j < H; ++j) {
+                gr[j] = sigmoid_(z[j]); gr[H + j] = sigmoid_(z[H + j]);
+                gr[2 * H + j] = tanh(z[2 * H + j]); gr[3 * H + j] = sigmoid_(z[3 * H + j]);
+                double cn = orc_cast(gr[H + j] * cs[t * BH + bi * H + j] + gr[j] * gr[2 * H + j], state_dtype);
+                cs[(t + 1) * BH + bi * H + j] = cn;
+                h[bi * H + j] = orc_cast(gr[3 * H + j] * tanh(cn), state_dtype);
+            }
+        }
+    /* reverse sweep */
+    if (dx) for (int64_t i = 0; i < T * B * I; ++i) dx[i] = 0.0;
+    if (dw_ih) for (int64_t i = 0; i < I * G; ++i) dw_ih[i] = 0.0;
+    if (dw_hh) for (int64_t i = 0; i < H * G; ++i) dw_hh[i] = 0.0;
+    if (db) for (int64_t g = 0; g < G; ++g) db[g] = 0.0;
+    for (int64_t i = 0; i < BH; ++i) { dhn[i] = 0.0; dcn[i] = dc_final ? dc_final[i] : 0.0; }
+    for (int64_t t = T - 1; t >= 0; --t) {
+        for (int64_t bi = 0; bi < B; ++bi) {
+            const double *gr = gt + (t * B + bi) * G;
+            for (int64_t j = 0; j < H; ++j) {
+                double ig = gr[j], fg = gr[H + j], gg = gr[2 * H + j], og = gr[3 * H + j];
+                double tc = tanh(cs[(t + 1) * BH + bi * H + j]);
+                double dh = dh_all[(t * B + bi) * H + j] + dhn[bi * H + j];
+                double d_o = dh * tc;
+                double dc = dcn[bi * H + j] + dh * og * (1.0 - tc * tc);
+                double d_i = dc * gg, d_f = dc * cs[t * BH + bi * H + j], d_g = dc * ig;
+                dcn[bi * H + j] = dc * fg;
+                double *dzr = dz + bi * G;
+                dzr[j] = orc_cast(d_i * ig * (1.0 - ig), dz_dtype);
+                dzr[H + j] = orc_cast(d_f * fg * (1.0 - fg), dz_dtype);
+                dzr[2 * H + j] = orc_cast(d_g * (1.0 - gg * gg), dz_dtype);
+                dzr[3 * H + j] = orc_cast(d_o * og * (1.0 - og), dz_dtype);
+            }
+        }
+        for (int64_t bi = 0; bi < B; ++bi) {
+            const double *dzr = dz + bi * G, *xr = x + (t * B + bi) * I, *hqr = hq + (t * B + bi) * H;
+            if (db) for (int64_t g = 0; g < G; ++g) db[g] += dzr[g];
+            for (int64_t k = 0; k < I; ++k) {
+                if (dx) {
+                    double s = 0.0;
+                    for (int64_t g = 0; g < G; ++g) s += dzr[g] * w_ih[k * G + g];
+                    dx[(t * B + bi) * I + k] = s;
+                }
+                if (dw_ih) for (int64_t g = 0; g < G; ++g) dw_ih[k * G + g] += xr[k] * dzr[g];
+            }
+            for (int64_t k = 0; k < H; ++k) {
+                double s = 0.0;
+                for (int64_t g = 0; g < G; ++g) s += dzr[g] * w_hh[k * G + g];
+                dhn[bi * H + k] = s;
+                if (dw_hh) for (int64_t g = 0; g < G; ++g) dw_hh[k * G + g] += hqr[k] * dzr[g];
+            }
+        }
+    }
+    if (dh0) for (int64_t i = 0; i < BH; ++i) dh0[i] = dhn[i];
+    if (dc0) for (int64_t i = 0; i < BH; ++i) dc0[i] = dcn[i];
+    free(hq); free(cs); free(gt); free(h); free(z); free(dz); free(dhn); free(dcn);
+    return 0;
+}
+
+/* ------------------------------------------------------------------------------------------
  * Integer type relations (Section 4.3: shapes live in types, so every output shape is a
  * function of the input shapes and attributes alone).
  * ---------------------------------------------------------------------------------------- */
