@@ -188,6 +188,7 @@ size_t relay_workspace_bytes_conv2d_act_grad(const relay_tensor_t *x, const rela
 size_t relay_workspace_bytes_reduce(const relay_tensor_t *const *inputs, int32_t n_in,
                                     const relay_out_spec_t *specs, int32_t n_out);
 size_t relay_workspace_bytes_lstm(const relay_tensor_t *x, const relay_tensor_t *w_ih, const relay_tensor_t *w_hh);
+size_t relay_workspace_bytes_lstm_grad(const relay_tensor_t *x, const relay_tensor_t *w_ih, const relay_tensor_t *w_hh);
 
 /* ---------------------------------------------------------------------------------------------
  * Compute entry points.
@@ -284,6 +285,26 @@ relay_status_t relay_lstm_cell_seq(const relay_tensor_t *x, const relay_tensor_t
                                    const relay_tensor_t *b, const relay_tensor_t *h0, const relay_tensor_t *c0,
                                    const relay_tensor_t *h_all, const relay_tensor_t *c_final, void *ws,
                                    size_t ws_bytes, void *stream);
+
+/* Gradient program of the LSTM sequence (Section 4.2: reverse mode through the recursion over time).
+ * Given the saved forward result h_all and the partials dh_all:(T,B,H) f32 of the final scalar with respect
+ * to every emitted h_t and dc_final:(B,H) f32 with respect to the final cell state (NULL = zero), for
+ * t = T-1 .. 0:
+ *   dh = dh_all[t] + dz_{t+1} w_hh^T;   do = dh (.) tanh(c_t);   dc = dc_next + dh (.) o (.) (1 - tanh(c_t)^2)
+ *   di = dc (.) g;  df = dc (.) c_{t-1};  dg = dc (.) i;  dc_next = dc (.) f
+ *   dz_t = bf16( [ di i(1-i) | df f(1-f) | dg (1-g^2) | do o(1-o) ] )      (the bf16 operand of four contractions)
+ * and then  dx[t] = dz_t w_ih^T,  dw_ih = sum_t x_t^T dz_t,  dw_hh = sum_t bf16(h_{t-1})^T dz_t,
+ * db = sum_t sum_rows dz_t,  dh0 = dz_0 w_hh^T,  dc0 = dc_next after t = 0.
+ *   inputs as relay_lstm_cell_seq plus h_all (its output);  dx:(T,B,I) bf16 or NULL;  dw_ih:(I,4H) bf16;
+ *   dw_hh:(H,4H) bf16;  db:(4H) f32 or NULL;  dh0, dc0:(B,H) f32 or NULL.
+ * Gates and cell states are recomputed from x and h_all (nothing else is saved by the forward call).
+ * `ws` must hold relay_workspace_bytes_lstm_grad() bytes. */
+relay_status_t relay_lstm_cell_seq_grad(const relay_tensor_t *x, const relay_tensor_t *w_ih, const relay_tensor_t *w_hh,
+                                        const relay_tensor_t *b, const relay_tensor_t *h0, const relay_tensor_t *c0,
+                                        const relay_tensor_t *h_all, const relay_tensor_t *dh_all, const relay_tensor_t *dc_final,
+                                        const relay_tensor_t *dx, const relay_tensor_t *dw_ih, const relay_tensor_t *dw_hh,
+                                        const relay_tensor_t *db, const relay_tensor_t *dh0, const relay_tensor_t *dc0, void *ws,
+                                        size_t ws_bytes, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Loss and parameter update: the two operators that close the training step of the LeNet listing

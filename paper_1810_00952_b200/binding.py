@@ -79,7 +79,7 @@ def lib() -> ctypes.CDLL:
         L.relay_launch_count.restype = ctypes.c_int64
         for name in ("relay_workspace_bytes_dense_act", "relay_workspace_bytes_dense_act_grad",
                      "relay_workspace_bytes_conv2d_act", "relay_workspace_bytes_conv2d_act_grad",
-                     "relay_workspace_bytes_reduce", "relay_workspace_bytes_lstm"):
+                     "relay_workspace_bytes_reduce", "relay_workspace_bytes_lstm", "relay_workspace_bytes_lstm_grad"):
             getattr(L, name).restype = ctypes.c_size_t
         _lib = L
     return _lib
@@ -312,6 +312,16 @@ def relay_lstm_cell_seq(x, w_ih, w_hh, b, h0, c0, h_all, c_final, ws=None):
     wp, wb = _ws(ws)
     _check(lib().relay_lstm_cell_seq(_ref(desc(x)), _ref(desc(w_ih)), _ref(desc(w_hh)), _ref(desc(b)), _ref(desc(h0)),
                                      _ref(desc(c0)), _ref(desc(h_all)), _ref(desc(c_final)), wp, wb, _stream()))
+
+
+def relay_workspace_bytes_lstm_grad(x, w_ih, w_hh) -> int:
+    return int(lib().relay_workspace_bytes_lstm_grad(_ref(desc(x)), _ref(desc(w_ih)), _ref(desc(w_hh))))
+
+
+def relay_lstm_cell_seq_grad(x, w_ih, w_hh, b, h0, c0, h_all, dh_all, dc_final, dx, dw_ih, dw_hh, db, dh0, dc0, ws=None):
+    wp, wb = _ws(ws)
+    ts = [x, w_ih, w_hh, b, h0, c0, h_all, dh_all, dc_final, dx, dw_ih, dw_hh, db, dh0, dc0]
+    _check(lib().relay_lstm_cell_seq_grad(*[_ref(desc(t)) for t in ts], wp, wb, _stream()))
 
 
 def relay_softmax_xent(scores, targets, loss):
