@@ -173,8 +173,14 @@ class Workload:
             d = self.devt["cfg5"]
             T, Bn, _ = d["x"].shape
             H = d["w_hh"].shape[0]
-            self.out["cfg5"] = dict(h_all=E(T, Bn, H, dt=f32), c=E(Bn, H, dt=f32))
-            ws_bytes = max(ws_bytes, B.relay_workspace_bytes_lstm(d["x"], d["w_ih"], d["w_hh"]))
+            In = d["x"].shape[2]
+            self.out["cfg5"] = dict(h_all=E(T, Bn, H, dt=f32), c=E(Bn, H, dt=f32), dx=E(T, Bn, In), dw_ih=E(In, 4 * H),
+                                    dw_hh=E(H, 4 * H), db=E(4 * H, dt=f32), dh0=E(Bn, H, dt=f32), dc0=E(Bn, H, dt=f32))
+            # upstream partials of the gradient program (device-resident, generated once)
+            self.lstm_dh_all = I.normal(5, 8, (T, Bn, H), 1.0, f32).to(dev)
+            self.lstm_dc_fin = I.normal(5, 9, (Bn, H), 1.0, f32).to(dev)
+            ws_bytes = max(ws_bytes, B.relay_workspace_bytes_lstm(d["x"], d["w_ih"], d["w_hh"]),
+                           B.relay_workspace_bytes_lstm_grad(d["x"], d["w_ih"], d["w_hh"]))
         if "next" in groups:
             d = self.devt["next"]
             self.out["next"] = dict(loss=E(d["scores"].shape[0], dt=f32), loss2=E(d["scores"].shape[0], dt=f32), dscores=torch.empty_like(d["scores"]))
@@ -260,6 +266,10 @@ class Workload:
             self.flush_l2()
             with tm.region("cfg5.lstm"):
                 B.relay_lstm_cell_seq(d["x"], d["w_ih"], d["w_hh"], d["b"], d["h0"], d["c0"], o["h_all"], o["c"], ws)
+            self.flush_l2()
+            with tm.region("cfg5.lstm_grad"):
+                B.relay_lstm_cell_seq_grad(d["x"], d["w_ih"], d["w_hh"], d["b"], d["h0"], d["c0"], o["h_all"], self.lstm_dh_all,
+                                           self.lstm_dc_fin, o["dx"], o["dw_ih"], o["dw_hh"], o["db"], o["dh0"], o["dc0"], ws)
 
         if "next" in self.groups:
             d, o = self.devt["next"], self.out["next"]
@@ -301,6 +311,8 @@ class Workload:
             T, Bn, In = self.host["cfg5"]["x"].shape
             H = self.host["cfg5"]["w_hh"].shape[0]
             w["cfg5.lstm"] = dict(flop=2 * T * Bn * (In + H) * 4 * H)
+            # gradient program: gate recomputation (one forward's worth), dz w_hh^T per step, dx, dw_ih, dw_hh
+            w["cfg5.lstm_grad"] = dict(flop=2 * T * Bn * (In + H) * 4 * H + 2 * T * Bn * 4 * H * (H + In) + 2 * T * Bn * 4 * H * (In + H))
         if "next" in self.groups:
             r, c = self.host["next"]["scores"].shape
             w["next.loss"] = dict(bytes=2 * r * c * 2 + r * 4)
