@@ -158,6 +158,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             const int fbar = MH == 1 ? (t_local & 1) : 0;            // barrier that announces it
             const uint32_t full_parity = MH == 1 ? ((t_local >> 1) & 1) : (t_local & 1);
             const int m0 = (tile % p.tiles_m) * BM + half * 128, n0 = (tile / p.tiles_m) * BN;
+            float bias_r[8];
+            load_bias(p, lane, n0, BN, bias_r);                 // before the wait: the loads' latency overlaps the main loop
             // one lane polls, the warp follows its verdict (keeps the warp converged for tcgen05.ld)
             int ok = 1;
             if (lane == 0) ok = tc::mbar_wait(&tmem_full[fbar], full_parity, abort_flag, p.err, tc::ERR_WAIT_TMEM_FULL) ? 1 : 0;
@@ -168,8 +170,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * BN;
             uint8_t *my_stage = staging + (size_t)(warp - 2) * Cfg<MH>::STORE_BUFS * 4096;
             if (row0 < p.M) {
-                if (p.out_f32) epilogue_rows<true, Cfg<MH>::STORE_BUFS>(p, &tm_c, taddr, my_stage, lane, row0, n0);
-                else epilogue_rows<false, Cfg<MH>::STORE_BUFS>(p, &tm_c, taddr, my_stage, lane, row0, n0);
+                if (p.out_f32) epilogue_rows<true, Cfg<MH>::STORE_BUFS>(p, &tm_c, taddr, my_stage, lane, row0, n0, bias_r, 0, BN / 32);
+                else epilogue_rows<false, Cfg<MH>::STORE_BUFS>(p, &tm_c, taddr, my_stage, lane, row0, n0, bias_r, 0, BN / 64);
             }
             tc::tc_fence_before_sync();
             __syncwarp();
@@ -220,6 +222,23 @@ relay_status_t make_tmap_2d(CUtensorMap *m, bool f32, const void *base, uint64_t
     CUresult r = fn(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(RELAY_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    return RELAY_OK;
+}
+
+// the same with 64-byte swizzle: boxes whose rows are 64 bytes (32 bf16 or 16 f32)
+relay_status_t make_tmap_2d_sw64(CUtensorMap *m, bool f32, const void *base, uint64_t inner, uint64_t outer, uint64_t row_stride,
+                                 uint32_t box_outer)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return fail(RELAY_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    cuuint64_t dims[2] = {inner, outer};
+    cuuint64_t strides[1] = {row_stride * (f32 ? 4 : 2)};
+    cuuint32_t box[2] = {f32 ? 16u : 32u, box_outer};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(RELAY_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
     return RELAY_OK;
 }

@@ -1,23 +1,35 @@
-// Two-SM tensor-core contraction: a cluster of two blocks computes one 256 x 256 tile with
-// tcgen05.mma.cta_group::2.  Each block loads its own 128 rows of A and HALF of the B tile (128 of the 256
-// columns) and the MMA unit reads both halves, so a block fetches 32 KB per 64-deep k-step instead of 48 KB
-// and six ring stages fit in shared memory.  No multicast load is used: every byte a block needs is
-// fetched by that block.
+// Two-SM tensor-core contraction: a cluster of two blocks computes 256-row work units with
+// tcgen05.mma.cta_group::2.  Each block loads its own 128 rows of A and HALF of the unit's B columns and the
+// MMA unit reads both halves.  No multicast load is used: every byte a block needs is fetched by that block.
 //
-// Work units: whole 256 x 256 tiles for as many full rounds over the pairs as there are; the tiles left for
-// the last, partly filled round are cut into two 256 x 128 units when that lets the round end in half the
-// time (p.tail_split = 2), so the SMs are not left idle behind a few full-size tiles.
+// What bounds these kernels is the number of bytes a block can pull from L2 per cycle (about 48 B per cycle and
+// SM here), so the work units are made as wide as the accumulator memory allows: a unit is 256 rows by 128, 256,
+// 384 or 512 columns ("class" 1..4 = width / 128).  The A rows of a stage are shared by all columns of the unit,
+// so a block fetches 16 KB + class x 8 KB per 64-deep k-step:
+//   class 4   two MMAs of N = 256 per 16-deep step, 48 KB stages (four), 48 B per MMA cycle: the tensor pipe stays busy;
+//   class 3   N = 256 and N = 128, 40 KB stages (four);
+//   class 2   N = 256, 32 KB stages (six);   class 1   N = 128, 24 KB stages (eight).
+// Units of class 3 and 4 own both halves of the accumulator memory (their epilogue is not overlapped with the
+// next unit's main loop), units of class 1 and 2 alternate between the halves (overlapped).
+//
+// The host cuts the output into units so that every pair of blocks gets nearly the same work in as few, as wide
+// units as possible (plan_units), sorts them widest first and passes the list as a kernel parameter; pair p
+// takes units p, p + pairs, ...  When the list would not fit, units follow a fixed scheme instead: whole rounds
+// of class-4 units, then 256 x 256 tiles, the tiles of a last, partly filled round cut in two.
+// Classes use the same ring memory with different stage sizes and their own barriers; a pair's units never grow
+// in class, and at a change of class the producer waits until every stage of the old class has been released.
 //
 // Pair protocol (rank 0 = leader):
 //   full[s]      lives in the leader; both blocks' TMA loads complete on it (cta_group::2 form), the
 //                leader's producer posts the expected byte count of both;
 //   empty[s], tmem_full[b]   live in each block; the leader's MMA thread arrives on both copies with a
 //                multicast tcgen05.commit;
-//   tmem_empty[b] lives in the leader; the eight epilogue warps of the pair arrive on it (the peer's
+//   tmem_empty[b] lives in the leader; the thirty-two epilogue warps of the pair arrive on it (the peer's
 //                remotely).
 // All waits are bounded; the only unbounded synchronisations are the two cluster barriers at the start and
 // the end, which every thread reaches unconditionally.
 #include <algorithm>
+#include <vector>
 
 #include "gemm.h"
 #include "gemm_tc_common.cuh"
@@ -26,62 +38,187 @@ namespace relay {
 
 using namespace gemm_tc;
 
-relay_status_t make_tmap_2d(CUtensorMap *m, bool f32, const void *base, uint64_t inner, uint64_t outer, uint64_t row_stride,
-                            uint32_t box_inner, uint32_t box_outer, bool swizzle128);
+relay_status_t make_tmap_2d_sw64(CUtensorMap *m, bool f32, const void *base, uint64_t inner, uint64_t outer, uint64_t row_stride,
+                                 uint32_t box_outer);
 relay_status_t make_tmap_2d_bf16(CUtensorMap *m, const void *base, uint64_t inner, uint64_t outer, uint64_t row_stride,
                                  uint32_t box_inner, uint32_t box_outer);
 
 namespace {
 
-constexpr int STAGES = 6;
-constexpr int A_BYTES = 128 * BK * 2, BH_BYTES = 128 * BK * 2, STAGE_BYTES = A_BYTES + BH_BYTES;   // 32 KB
-constexpr int NUM_THREADS = 192;
-constexpr int STAGING_BYTES = 4 * 2 * 4096;
-constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * STAGE_BYTES + STAGING_BYTES + 256;
+constexpr int A_BYTES = 128 * BK * 2;                      // this block's 128 rows of A: 16 KB
+constexpr int CHUNK_BYTES = 64 * BK * 2;                   // this block's 64 columns of one 128-column chunk: 8 KB
+constexpr int RING_BYTES = 192 * 1024;
+constexpr int NUM_THREADS = 576;                           // warp 0 producer, warp 1 MMA, warps 2-17 epilogue
+constexpr int EPI_WARPS = 16;
+constexpr int kWideMinKBlocks = 32;                        // classes 3 and 4 only for contractions at least this long
+constexpr int STAGING_BYTES = EPI_WARPS * 2048;        // one 32-row x 64-byte buffer per epilogue warp
+constexpr int BAR_BYTES = 512;
+constexpr size_t SMEM_BYTES = 1024 + (size_t)RING_BYTES + STAGING_BYTES + BAR_BYTES;
+constexpr int MAX_UNITS = 640;
 
-// Work unit u of the launch: tile index, first column and width.
+__host__ __device__ constexpr int cls_stages(int c) { return c == 1 ? 8 : c == 2 ? 6 : 4; }
+__host__ __device__ constexpr int cls_stage_bytes(int c) { return A_BYTES + c * CHUNK_BYTES; }
+__host__ __device__ constexpr int cls_bar_base(int c) { return c == 1 ? 0 : c == 2 ? 16 : c == 3 ? 28 : 36; }   // full[], then empty[]
+constexpr int BAR_TMEM = 44;                                // tmem_full[2], tmem_empty[2]
+static_assert(cls_stages(1) * cls_stage_bytes(1) <= RING_BYTES && cls_stages(2) * cls_stage_bytes(2) <= RING_BYTES &&
+              cls_stages(3) * cls_stage_bytes(3) <= RING_BYTES && cls_stages(4) * cls_stage_bytes(4) <= RING_BYTES, "ring too small");
+static_assert((BAR_TMEM + 4) * 8 + 8 <= BAR_BYTES, "barrier area too small");
+
+// unit list: row block | first 128-column chunk << 12 | class << 24, widest class first
+struct UnitTable {
+    int n;
+    uint32_t e[MAX_UNITS];
+};
+
 struct Unit {
     int tile_m, n0, width;
 };
-__device__ __forceinline__ Unit unit_of(const Params &p, int u)
+
+// Fixed scheme (no list): tiles are numbered so that 2w and 2w+1 are the two column neighbours that class-4 unit w
+// covers: tile t (t < 2 * tiles_m * (tiles_n / 2)): row block (t/2) % tiles_m, column block 2 * ((t/2) / tiles_m) + t % 2;
+// an odd last column block follows in row order.
+__device__ __forceinline__ void tile_pos(const Params &p, int t, int &tile_m, int &tile_n)
+{
+    const int paired = 2 * p.tiles_m * (p.tiles_n >> 1);
+    if (t < paired) {
+        const int w = t >> 1;
+        tile_m = w % p.tiles_m;
+        tile_n = 2 * (w / p.tiles_m) + (t & 1);
+    } else {
+        tile_m = t - paired;
+        tile_n = p.tiles_n - 1;
+    }
+}
+
+__device__ __forceinline__ Unit unit_of(const Params &p, const UnitTable &tb, int u)
 {
     Unit w;
+    if (tb.n > 0) {
+        const uint32_t e = tb.e[u];
+        w.tile_m = (int)(e & 0xFFFu);
+        w.n0 = (int)((e >> 12) & 0xFFFu) * 128;
+        w.width = (int)(e >> 24) * 128;
+        return w;
+    }
+    int tile_n;
+    if (u < p.wide_units) {
+        tile_pos(p, 2 * u, w.tile_m, tile_n);
+        w.n0 = tile_n * BN;
+        w.width = 2 * BN;
+        return w;
+    }
+    const int v = u - p.wide_units;
     int tile, sub = 0;
     w.width = BN;
-    if (u < p.full_tiles) {
-        tile = u;
+    if (v < p.full_tiles) {
+        tile = v;
     } else {
-        const int v = u - p.full_tiles;
-        tile = p.full_tiles + v / p.tail_split;
-        sub = v % p.tail_split;
+        const int x = v - p.full_tiles;
+        tile = p.full_tiles + x / p.tail_split;
+        sub = x % p.tail_split;
         w.width = BN / p.tail_split;
     }
-    w.tile_m = tile % p.tiles_m;
-    w.n0 = (tile / p.tiles_m) * BN + sub * w.width;
+    tile_pos(p, 2 * p.wide_units + tile, w.tile_m, tile_n);
+    w.n0 = tile_n * BN + sub * w.width;
     return w;
 }
 
-template <bool A_MN, bool B_MN>
+// One epilogue warp drains its 32 accumulator rows, the 32-column groups [g_begin, g_end) of an accumulator that
+// starts at column n0: both groups' TMEM loads are issued before the first is awaited (a load takes several hundred
+// cycles), then per group bias + activation + rounding, a 32-row x 64-byte staging buffer in the 64-byte swizzle
+// pattern (16-byte piece c of row r at piece c ^ ((r >> 1) & 3)) and one TMA tile store (two for f32 output).
+// The drain is spread over sixteen warps because one warp alone issues these instructions only every few cycles.
+template <bool OUT_F32, bool TRANSC>
+__device__ __forceinline__ void finish_group(const Params &p, const CUtensorMap *tm_c, uint8_t *stage, int lane, int row0, int nc,
+                                             float bias_lane, uint32_t (&r)[32])
+{
+    float v[32];
+    if (p.bias != nullptr) {                             // warp-uniform; lane j holds the bias of column nc + j
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) + __shfl_sync(0xffffffffu, bias_lane, j);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+    }
+    if (TRANSC) {                                        // tanh / sigmoid: their own instantiation (they need many registers)
+        if (p.act == RELAY_ACT_TANH) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = OUT_F32 ? tanh_<false>(v[j]) : tanh_<true>(v[j]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = OUT_F32 ? sigmoid_<false>(v[j]) : sigmoid_<true>(v[j]);
+        }
+    } else if (p.act == RELAY_ACT_RELU) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.0f);
+    }
+    const int sw = (lane >> 1) & 3;
+#pragma unroll
+    for (int h = 0; h < (OUT_F32 ? 2 : 1); ++h) {        // 64 bytes of every row at a time
+        if (lane == 0) tc::tma_store_wait_read<0>();     // the previous store has read the buffer
+        __syncwarp();
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            uint4 piece;
+            if (OUT_F32) piece = make_uint4(__float_as_uint(v[16 * h + 4 * c]), __float_as_uint(v[16 * h + 4 * c + 1]),
+                                            __float_as_uint(v[16 * h + 4 * c + 2]), __float_as_uint(v[16 * h + 4 * c + 3]));
+            else piece = make_uint4(pack2(v[8 * c], v[8 * c + 1]), pack2(v[8 * c + 2], v[8 * c + 3]), pack2(v[8 * c + 4], v[8 * c + 5]),
+                                    pack2(v[8 * c + 6], v[8 * c + 7]));
+            *reinterpret_cast<uint4 *>(stage + lane * 64 + ((c ^ sw) << 4)) = piece;
+        }
+        tc::fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) {
+            tc::tma_store_2d(tm_c, stage, nc + h * (OUT_F32 ? 16 : 0), row0);
+            tc::tma_store_commit();
+        }
+    }
+}
+
+// One epilogue warp drains its 32 accumulator rows, `per` (1 or 2) 32-column groups starting at group g0 of an
+// accumulator that starts at column n0: the TMEM loads of both groups are issued before the first is awaited (a load
+// takes several hundred cycles), then per group bias + activation + rounding, a 32-row x 64-byte staging buffer in
+// the 64-byte swizzle pattern (16-byte piece c of row r at piece c ^ ((r >> 1) & 3)) and one TMA tile store (two for
+// f32 output).  The drain is spread over sixteen warps because one warp alone issues these instructions only every
+// few cycles.
+template <bool OUT_F32, bool TRANSC>
+__device__ __forceinline__ void drain_groups(const Params &p, const CUtensorMap *tm_c, uint32_t taddr, uint8_t *stage, int lane, int row0,
+                                             int n0, const float (&bias_r)[8], int g0, int per)
+{
+    uint32_t ra[32], rb[32];
+    const int g1 = g0 + per - 1;                         // per == 1: the same group again (its copy is not used)
+    tc::tmem_ld_32x32(taddr + g0 * 32, ra);
+    tc::tmem_ld_32x32(taddr + g1 * 32, rb);
+    tc::tmem_ld_wait();
+    float bl0 = 0.0f, bl1 = 0.0f;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) { if (q == g0) bl0 = bias_r[q]; if (q == g1) bl1 = bias_r[q]; }
+    if (n0 + g0 * 32 < p.N) finish_group<OUT_F32, TRANSC>(p, tm_c, stage, lane, row0, n0 + g0 * 32, bl0, ra);
+    if (per == 2 && n0 + g1 * 32 < p.N) finish_group<OUT_F32, TRANSC>(p, tm_c, stage, lane, row0, n0 + g1 * 32, bl1, rb);
+}
+
+template <bool A_MN, bool B_MN, bool TRANSC>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                const __grid_constant__ CUtensorMap tm_c, const Params p)
+                const __grid_constant__ CUtensorMap tm_c, const Params p, const __grid_constant__ UnitTable tb)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t *staging = smem + (size_t)STAGES * STAGE_BYTES;
+    uint8_t *staging = smem + RING_BYTES;
     uint64_t *bars = reinterpret_cast<uint64_t *>(staging + STAGING_BYTES);
-    uint64_t *full = bars, *empty = bars + STAGES, *tmem_full = bars + 2 * STAGES, *tmem_empty = bars + 2 * STAGES + 2;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 4);
+    uint64_t *tmem_full = bars + BAR_TMEM, *tmem_empty = bars + BAR_TMEM + 2;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + BAR_TMEM + 4);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = tc::cluster_ctarank();          // 0 = leader
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-    const int n_units = p.full_tiles + (p.tiles_m * p.tiles_n - p.full_tiles) * p.tail_split;
+    const int n_units = tb.n > 0 ? tb.n
+                                 : p.wide_units + p.full_tiles + (p.tiles_m * p.tiles_n - 2 * p.wide_units - p.full_tiles) * p.tail_split;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { tc::mbar_init(&tmem_full[b], 1); tc::mbar_init(&tmem_empty[b], 8); }
+        for (int i = 0; i < BAR_TMEM; ++i) tc::mbar_init(&bars[i], 1);
+        for (int b = 0; b < 2; ++b) { tc::mbar_init(&tmem_full[b], 1); tc::mbar_init(&tmem_empty[b], 2 * EPI_WARPS); }
         *abort_flag = 0;
         tc::fence_barrier_init();
         tc::prefetch_tmap(&tm_a);
@@ -102,18 +239,33 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     if (warp == 0) {
         // ---------------- TMA producer (both blocks) ----------------
         if (lane == 0) {
-            int s = 0;
+            int cur = 0, s = 0, n_st = 0, st_bytes = 0;
             uint32_t phase = 0;
+            uint64_t *full = bars, *empty = bars;
             bool ok = true;
             for (int u = pair; u < n_units && ok; u += n_pairs) {
-                const Unit w = unit_of(p, u);
-                const int m0 = w.tile_m * 256 + (int)rank * 128;                // this block's rows
-                const int n0 = w.n0 + (int)rank * (w.width >> 1);               // this block's half of the B columns
-                const int b_boxes = w.width >> 7;                               // boxes of 64 columns in that half
-                const uint32_t tx = 2u * (A_BYTES + (uint32_t)b_boxes * MN_BOX_BYTES);   // bytes of both blocks
+                const Unit w = unit_of(p, tb, u);
+                const int c = w.width >> 7;
+                if (c != cur) {
+                    // the new class's stages lie over the old one's: every old stage must have been released
+                    for (int i = 0; i < n_st && ok; ++i) {
+                        if (!tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) ok = false;
+                        if (++s == n_st) { s = 0; phase ^= 1; }
+                    }
+                    if (!ok) break;
+                    cur = c; n_st = cls_stages(c); st_bytes = cls_stage_bytes(c);
+                    full = bars + cls_bar_base(c); empty = full + n_st;
+                    s = 0; phase = 0;
+                }
+                // the first MMA of a 16-deep step covers 2*h0 columns, the second 2*h1; this block holds h0 + h1 of them
+                const int h0 = c == 1 ? 64 : 128, h1 = c == 3 ? 64 : c == 4 ? 128 : 0;
+                const int m0 = w.tile_m * 256 + (int)rank * 128;
+                const int na = w.n0 + (int)rank * h0, nb = w.n0 + 2 * h0 + (int)rank * h1;
+                const int boxes0 = h0 >> 6, boxes = (h0 + h1) >> 6;
+                const uint32_t tx = 2u * (uint32_t)st_bytes;                        // bytes of both blocks
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
                     if (!tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
-                    uint8_t *sa = smem + (size_t)s * STAGE_BYTES, *sb = sa + A_BYTES;
+                    uint8_t *sa = smem + (size_t)s * st_bytes, *sb = sa + A_BYTES;
                     const uint32_t bar = tc::mapa(tc::smem_u32(&full[s]), 0);       // the leader's barrier
                     if (rank == 0) tc::mbar_expect_tx_cluster(bar, tx);
                     const int k0 = kb * BK;
@@ -124,71 +276,104 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                         tc::tma_load_2d_pair(sa, &tm_a, bar, k0, m0);
                     }
                     // B in boxes of 64 columns: MN-major boxes are 64 x 64 k anyway; K-major boxes of 64 rows stack
-                    // to the same shared-memory image as one 128-row box
-                    for (int i = 0; i < b_boxes; ++i) {
-                        if (B_MN) tc::tma_load_2d_pair(sb + i * MN_BOX_BYTES, &tm_b, bar, n0 + i * 64, k0);
-                        else tc::tma_load_2d_pair(sb + i * MN_BOX_BYTES, &tm_b, bar, k0, n0 + i * 64);
+                    // to the same shared-memory image as one taller box
+                    for (int i = 0; i < boxes; ++i) {
+                        const int n = i < boxes0 ? na + i * 64 : nb + (i - boxes0) * 64;
+                        if (B_MN) tc::tma_load_2d_pair(sb + i * MN_BOX_BYTES, &tm_b, bar, n, k0);
+                        else tc::tma_load_2d_pair(sb + i * MN_BOX_BYTES, &tm_b, bar, k0, n);
                     }
-                    if (++s == STAGES) { s = 0; phase ^= 1; }
+                    if (++s == n_st) { s = 0; phase ^= 1; }
                 }
             }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer (leader only) ----------------
         if (lane == 0 && rank == 0) {
-            constexpr uint32_t idesc_full = tc::instr_desc_bf16(256, BN, A_MN, B_MN);
-            constexpr uint32_t idesc_half = tc::instr_desc_bf16(256, BN / 2, A_MN, B_MN);
+            constexpr uint32_t idesc_256 = tc::instr_desc_bf16(256, 256, A_MN, B_MN);
+            constexpr uint32_t idesc_128 = tc::instr_desc_bf16(256, 128, A_MN, B_MN);
             constexpr uint32_t a_lbo = A_MN ? MN_BOX_BYTES : 16, b_lbo = B_MN ? MN_BOX_BYTES : 16;
             constexpr uint32_t a_step = A_MN ? 2048 : 32, b_step = B_MN ? 2048 : 32;
+            constexpr uint32_t b1_off = (2 * CHUNK_BYTES) >> 4;   // the second MMA's columns follow the first's 128 in this block
             const uint64_t desc_a0 = tc::smem_desc(tc::smem_u32(smem), a_lbo, 1024);
             const uint64_t desc_b0 = tc::smem_desc(tc::smem_u32(smem) + A_BYTES, b_lbo, 1024);
-            uint32_t t_local = 0, phase = 0, stage_off = 0;
-            int s = 0;
+            uint32_t t_local = 0, phase = 0, stage_off = 0;   // t_local counts accumulator halves handed to the epilogue
+            int cur = 0, s = 0, n_st = 0, st_bytes = 0;
+            uint64_t *full = bars, *empty = bars;
             bool ok = true;
-            for (int u = pair; u < n_units && ok; u += n_pairs, ++t_local) {
+            for (int u = pair; u < n_units && ok; u += n_pairs) {
+                const Unit w = unit_of(p, tb, u);
+                const int c = w.width >> 7;
+                if (c != cur) {
+                    cur = c; n_st = cls_stages(c); st_bytes = cls_stage_bytes(c);
+                    full = bars + cls_bar_base(c); empty = full + n_st;
+                    s = 0; phase = 0; stage_off = 0;
+                }
+                const bool both = c >= 3;                 // the unit owns both accumulator halves (t_local is even: such units come first)
                 const int buf = t_local & 1;
-                const uint32_t idesc = (u < p.full_tiles || p.tail_split == 1) ? idesc_full : idesc_half;
-                if (!tc::mbar_wait(&tmem_empty[buf], ((t_local >> 1) & 1) ^ 1, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) break;
+                const uint32_t par = ((t_local >> 1) & 1) ^ 1;
+                if (!tc::mbar_wait(&tmem_empty[buf], par, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) break;
+                if (both && !tc::mbar_wait(&tmem_empty[1], par, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) break;
                 tc::tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + buf * BN;
+                const uint32_t d0 = tmem_base + buf * BN, d1 = tmem_base + BN;
+                const uint32_t idesc0 = c == 1 ? idesc_128 : idesc_256, idesc1 = c == 3 ? idesc_128 : idesc_256;
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
                     if (!tc::mbar_wait(&full[s], phase, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
                     tc::tc_fence_after_sync();
                     const uint64_t da = desc_a0 + stage_off, db = desc_b0 + stage_off;
                     const uint32_t acc = kb != 0;
+                    if (both) {
 #pragma unroll
-                    for (int kk = 0; kk < BK / 16; ++kk)
-                        tc::mma_bf16_pair(d_tmem, da + ((kk * a_step) >> 4), db + ((kk * b_step) >> 4), idesc, acc | (kk != 0));
+                        for (int kk = 0; kk < BK / 16; ++kk) {
+                            tc::mma_bf16_pair(d0, da + ((kk * a_step) >> 4), db + ((kk * b_step) >> 4), idesc0, acc | (kk != 0));
+                            tc::mma_bf16_pair(d1, da + ((kk * a_step) >> 4), db + b1_off + ((kk * b_step) >> 4), idesc1, acc | (kk != 0));
+                        }
+                    } else {
+#pragma unroll
+                        for (int kk = 0; kk < BK / 16; ++kk)
+                            tc::mma_bf16_pair(d0, da + ((kk * a_step) >> 4), db + ((kk * b_step) >> 4), idesc0, acc | (kk != 0));
+                    }
                     tc::mma_commit_pair(&empty[s]);
-                    stage_off += STAGE_BYTES >> 4;
-                    if (++s == STAGES) { s = 0; phase ^= 1; stage_off = 0; }
+                    stage_off += (uint32_t)st_bytes >> 4;
+                    if (++s == n_st) { s = 0; phase ^= 1; stage_off = 0; }
                 }
-                if (ok) tc::mma_commit_pair(&tmem_full[buf]);
+                if (!ok) break;
+                tc::mma_commit_pair(&tmem_full[buf]);
+                if (both) tc::mma_commit_pair(&tmem_full[1]);
+                t_local += both ? 2 : 1;
             }
         }
     } else {
-        // ---------------- epilogue (both blocks: 128 rows x 256 columns each) ----------------
-        const int quarter = warp & 3;
-        uint8_t *my_stage = staging + (size_t)(warp - 2) * 2 * 4096;
+        // ---------------- epilogue (both blocks: 128 rows each; four warps per 32-row TMEM lane quarter) ----------------
+        const int quarter = warp & 3;                     // TMEM lanes [32*quarter, 32*quarter+32)
+        const int slot = (warp - 2) >> 2;                 // which quarter of an accumulator's 32-column groups this warp drains
+        uint8_t *my_stage = staging + (size_t)(warp - 2) * 2048;
         uint32_t t_local = 0;
-        for (int u = pair; u < n_units; u += n_pairs, ++t_local) {
-            const int buf = t_local & 1;
-            const Unit w = unit_of(p, u);
-            const int m0 = w.tile_m * 256 + (int)rank * 128, n0 = w.n0;
-            int ok = 1;
-            if (lane == 0) ok = tc::mbar_wait(&tmem_full[buf], (t_local >> 1) & 1, abort_flag, p.err, tc::ERR_WAIT_TMEM_FULL) ? 1 : 0;
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            if (!ok) break;
-            tc::tc_fence_after_sync();
-            const int row0 = m0 + quarter * 32;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * BN;
-            if (row0 < p.M) {
-                if (p.out_f32) epilogue_rows<true, 2>(p, &tm_c, taddr, my_stage, lane, row0, n0, w.width);
-                else epilogue_rows<false, 2>(p, &tm_c, taddr, my_stage, lane, row0, n0, w.width);
+        bool ok_all = true;
+        for (int u = pair; u < n_units && ok_all; u += n_pairs) {
+            const Unit w = unit_of(p, tb, u);
+            const int items = w.width > BN ? 2 : 1;       // accumulator halves of this unit, in the order the issuer fills them
+            for (int item = 0; item < items; ++item, ++t_local) {
+                const int buf = t_local & 1;
+                const int n0 = w.n0 + item * BN, width = item == 0 ? min(w.width, BN) : w.width - BN;
+                const int m0 = w.tile_m * 256 + (int)rank * 128;
+                float bias_r[8];
+                load_bias(p, lane, n0, width, bias_r);    // before the wait: the loads' latency overlaps the main loop
+                int ok = 1;
+                if (lane == 0) ok = tc::mbar_wait(&tmem_full[buf], (t_local >> 1) & 1, abort_flag, p.err, tc::ERR_WAIT_TMEM_FULL) ? 1 : 0;
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) { ok_all = false; break; }
+                tc::tc_fence_after_sync();
+                const int row0 = m0 + quarter * 32;
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * BN;
+                if (row0 < p.M) {
+                    const int per = width / 128;          // 32-column groups per warp: 2 for a 256-column accumulator, 1 for 128
+                    if (p.out_f32) drain_groups<true, TRANSC>(p, &tm_c, taddr, my_stage, lane, row0, n0, bias_r, slot * per, per);
+                    else drain_groups<false, TRANSC>(p, &tm_c, taddr, my_stage, lane, row0, n0, bias_r, slot * per, per);
+                }
+                tc::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive_cluster(tc::mapa(tc::smem_u32(&tmem_empty[buf]), 0));
             }
-            tc::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) tc::mbar_arrive_cluster(tc::mapa(tc::smem_u32(&tmem_empty[buf]), 0));
         }
         if (lane == 0) tc::tma_store_wait_all<0>();
     }
@@ -200,6 +385,42 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         tc::tc_fence_after_sync();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
+}
+
+// Cuts tiles_m row blocks of `cpr` 128-column chunks into units for `pairs` pairs of blocks.  A pair's share is
+// ceil(chunks / pairs) chunks; rounds over the pairs take it widest class first (4, 4, ..., then the rest), since a
+// 64-deep k-step of class c costs max(256 c MMA cycles, (16 + 8 c) KB / 48 B per cycle).  A unit never crosses a
+// row block, so what is left at the end of a row becomes a narrower unit.  Returns false when the list would not fit.
+bool plan_units(int tiles_m, int cpr, int pairs, int k_blocks, UnitTable *tb)
+{
+    const int max_c = k_blocks >= kWideMinKBlocks ? 4 : 2;
+    const long long total = (long long)tiles_m * cpr;
+    if (tiles_m > 0xFFF || cpr > 0xFFF || total > 4LL * MAX_UNITS) return false;
+    long long share = (total + pairs - 1) / pairs;
+    std::vector<int> rounds;
+    while (share > 0) {
+        const int c = (int)std::min<long long>(max_c, share);
+        rounds.push_back(c);
+        share -= c;
+    }
+    std::vector<uint32_t> units;
+    size_t r = 0;
+    int quota = pairs;
+    for (int m = 0; m < tiles_m; ++m) {
+        int at = 0;
+        while (at < cpr) {
+            const int want = r < rounds.size() ? rounds[r] : std::min(2, max_c);
+            const int c = std::min(want, cpr - at);
+            units.push_back((uint32_t)m | ((uint32_t)at << 12) | ((uint32_t)c << 24));
+            at += c;
+            if (--quota == 0) { quota = pairs; ++r; }
+        }
+    }
+    if (units.size() > (size_t)MAX_UNITS) return false;
+    std::stable_sort(units.begin(), units.end(), [](uint32_t a, uint32_t b) { return (a >> 24) > (b >> 24); });
+    tb->n = (int)units.size();
+    std::copy(units.begin(), units.end(), tb->e);
+    return true;
 }
 
 }  // namespace
@@ -220,7 +441,7 @@ relay_status_t launch_gemm_tc2(const GemmDesc &g, int sms, cudaStream_t st)
     if (b_mn) RELAY_TRY(make_tmap_2d_bf16(&tm_b, g.b, g.N, g.K, g.b_sk, 64, BK));
     else RELAY_TRY(make_tmap_2d_bf16(&tm_b, g.b, g.K, g.N, g.b_sn, BK, 64));
     const bool f32 = g.out_dtype == RELAY_F32;
-    RELAY_TRY(make_tmap_2d(&tm_c, f32, g.c, g.N, g.M, g.ldc, f32 ? 32 : 64, 32, true));
+    RELAY_TRY(make_tmap_2d_sw64(&tm_c, f32, g.c, g.N, g.M, g.ldc, 32));
     Params p{};
     p.M = (int)g.M; p.N = (int)g.N; p.K = (int)g.K;
     p.c = g.c; p.ldc = g.ldc;
@@ -230,20 +451,38 @@ relay_status_t launch_gemm_tc2(const GemmDesc &g, int sms, cudaStream_t st)
     if (!p.err) return fail(RELAY_ERR_CUDA, "no device error word");
     const int n_tiles = p.tiles_m * p.tiles_n;
     const int pairs = std::min(n_tiles, sms / 2);
-    // tiles of the last, partly filled round: two half-width units each when they then still fit one round
-    const int rem = n_tiles % pairs;
-    p.tail_split = (rem > 0 && 2 * rem <= pairs) ? 2 : 1;
-    p.full_tiles = p.tail_split == 2 ? n_tiles - rem : n_tiles;
-#define LAUNCH2(AMN, BMN)                                                                                                   \
+    static thread_local UnitTable tb;
+    tb.n = 0;
+    p.tail_split = 1;
+    if (!plan_units(p.tiles_m, (int)((g.N + 127) / 128), pairs, p.k_blocks, &tb)) {
+        // fixed scheme: class-4 units for whole rounds over the pairs (only for a contraction long enough to pay for
+        // their exposed epilogue), then 256 x 256 tiles; the tiles of a last, partly filled round become two
+        // half-width units each when they then still fit one round
+        tb.n = 0;
+        const int wide_rounds = p.k_blocks >= kWideMinKBlocks ? std::min(n_tiles / (2 * pairs), (p.tiles_m * (p.tiles_n / 2)) / pairs) : 0;
+        p.wide_units = wide_rounds * pairs;
+        const int narrow = n_tiles - 2 * p.wide_units;
+        const int rem = narrow % pairs;
+        p.tail_split = (rem > 0 && 2 * rem <= pairs) ? 2 : 1;
+        p.full_tiles = p.tail_split == 2 ? narrow - rem : narrow;
+    }
+    const bool transc = g.act == RELAY_ACT_TANH || g.act == RELAY_ACT_SIGMOID;
+#define LAUNCH3(AMN, BMN, TR)                                                                                               \
     do {                                                                                                                    \
-        RELAY_CUDA(cudaFuncSetAttribute(gemm_tc2_kernel<AMN, BMN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES)); \
-        RELAY_CUDA(launch_pdl(gemm_tc2_kernel<AMN, BMN>, dim3(2 * pairs), dim3(NUM_THREADS), SMEM_BYTES, st, tm_a, tm_b, tm_c, p));                         \
+        RELAY_CUDA(cudaFuncSetAttribute(gemm_tc2_kernel<AMN, BMN, TR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES)); \
+        RELAY_CUDA(launch_pdl(gemm_tc2_kernel<AMN, BMN, TR>, dim3(2 * pairs), dim3(NUM_THREADS), SMEM_BYTES, st, tm_a, tm_b, tm_c, p, tb));                 \
+    } while (0)
+#define LAUNCH2(AMN, BMN)            \
+    do {                             \
+        if (transc) LAUNCH3(AMN, BMN, true); \
+        else LAUNCH3(AMN, BMN, false);       \
     } while (0)
     if (a_mn && b_mn) LAUNCH2(true, true);
     else if (a_mn) LAUNCH2(true, false);
     else if (b_mn) LAUNCH2(false, true);
     else LAUNCH2(false, false);
 #undef LAUNCH2
+#undef LAUNCH3
     return check_launch("gemm_tc2");
 }
 

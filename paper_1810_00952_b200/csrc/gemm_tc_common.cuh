@@ -18,35 +18,58 @@ struct Params {
     const void *bias;
     int bias_bf16, act, out_f32;
     int tiles_m, tiles_n, k_blocks;
-    int full_tiles, tail_split;   // two-SM kernel: tiles after the first full_tiles are cut into tail_split column parts
+    // two-SM kernel: wide_units 256 x 512 units come first; of the remaining tiles, those after the first full_tiles
+    // are cut into tail_split column parts
+    int wide_units, full_tiles, tail_split;
     int *err;
 };
 
-// One warp drains its 32 accumulator rows (`width` columns, 256 unless stated): TMEM -> registers -> bias +
-// activation -> rounding -> swizzled staging buffer -> TMA tile store of 32 rows x 128 bytes at a time.
+// Bias values of up to 256 columns starting at n0, one 32-column group per register: lane j holds the bias of
+// column n0 + 32 g + j in b[g].  Fetched before the warp waits for its accumulator, so that the latency of
+// these loads is not paid per group inside the drain loop.
+__device__ __forceinline__ void load_bias(const Params &p, int lane, int n0, int width, float (&b)[8])
+{
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+        const int c = n0 + g * 32 + lane;
+        b[g] = 0.0f;
+        if (p.bias != nullptr && g * 32 < width && c < p.N)
+            b[g] = p.bias_bf16 ? __bfloat162float(((const __nv_bfloat16 *)p.bias)[c]) : ((const float *)p.bias)[c];
+    }
+}
+
+// One warp drains 32 accumulator rows, the 128-byte column blocks [blk_begin, blk_end) of an accumulator that
+// starts at column n0 (block = 64 bf16 or 32 f32 columns): TMEM -> registers -> bias + activation -> rounding ->
+// swizzled staging buffers -> TMA tile store of 32 rows x 128 bytes at a time.  `bias_r` comes from load_bias(n0).
 template <bool OUT_F32, int BUFS>
 __device__ __forceinline__ void epilogue_rows(const Params &p, const CUtensorMap *tm_c, uint32_t taddr, uint8_t *stage, int lane,
-                                              int row0, int n0, int width = BN)
+                                              int row0, int n0, const float (&bias_r)[8], int blk_begin, int blk_end)
 {
     constexpr int COLS = OUT_F32 ? 32 : 64;             // columns per 128-byte block
+    constexpr int SUBS = COLS / 32;
 #pragma unroll 1
-    for (int blk = 0; blk < width / COLS; ++blk) {
+    for (int blk = blk_begin; blk < blk_end; ++blk) {
         const int nc = n0 + blk * COLS;
         if (nc >= p.N) break;                            // warp-uniform
+        uint32_t r[SUBS][32];
+#pragma unroll
+        for (int sub = 0; sub < SUBS; ++sub) tc::tmem_ld_32x32(taddr + blk * COLS + sub * 32, r[sub]);
+        tc::tmem_ld_wait();
         uint4 piece[8];
 #pragma unroll
-        for (int sub = 0; sub < COLS / 32; ++sub) {
-            uint32_t r[32];
-            tc::tmem_ld_32x32(taddr + blk * COLS + sub * 32, r);
-            tc::tmem_ld_wait();
-            const int c0 = nc + sub * 32;
-            // lane j fetches the bias of column c0 + j; every lane then reads all 32 by shuffle
-            float bias_lane = 0.0f;
-            if (p.bias != nullptr && c0 + lane < p.N)
-                bias_lane = p.bias_bf16 ? __bfloat162float(((const __nv_bfloat16 *)p.bias)[c0 + lane]) : ((const float *)p.bias)[c0 + lane];
+        for (int sub = 0; sub < SUBS; ++sub) {
             float v[32];
+            if (p.bias != nullptr) {                     // warp-uniform
+                // every lane reads the 32 bias values of this group by shuffle (lane j holds column j's)
+                float bias_lane = 0.0f;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) + __shfl_sync(0xffffffffu, bias_lane, j);
+                for (int g = 0; g < 8; ++g) if (g == blk * SUBS + sub) bias_lane = bias_r[g];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[sub][j]) + __shfl_sync(0xffffffffu, bias_lane, j);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[sub][j]);
+            }
             switch (p.act) {                             // hoisted out of the element loop
             case RELAY_ACT_RELU:
 #pragma unroll
@@ -74,7 +97,7 @@ __device__ __forceinline__ void epilogue_rows(const Params &p, const CUtensorMap
                                                     pack2(v[8 * c + 4], v[8 * c + 5]), pack2(v[8 * c + 6], v[8 * c + 7]));
             }
         }
-        tc::warp_store_block<BUFS - 1>(tm_c, stage + (blk % BUFS) * 4096, piece, lane, nc, row0);
+        tc::warp_store_block<BUFS - 1>(tm_c, stage + ((blk - blk_begin) % BUFS) * 4096, piece, lane, nc, row0);
     }
 }
 
