@@ -129,15 +129,23 @@ __global__ void __launch_bounds__(128) colsum_any_kernel(const __nv_bfloat16 *__
 // owning a row adds dh_all, applies the gate derivatives, writes bf16(dz_t) of its 64 gate columns into
 // dZ[t] and arrives on the group's grid barrier; the carried dc stays in registers.
 constexpr int UNITS = 16;
-constexpr int BK = 64, STAGES = 6;
-constexpr int A_STAGE = 128 * BK * 2;            // 128 batch rows (rows beyond the group stay zero) x 64 k
+constexpr int BK = 64, MAX_STAGES = 32;
+constexpr int A_TILE = 128 * BK * 2;             // what one MMA reads as its A operand: 128 rows x 64 k
+constexpr int RING_BYTES = 96 * 1024;
 constexpr int W_KB = UNITS * BK * 2;             // one k-block of the resident W slice
-constexpr int NUM_THREADS = 192;                 // warps 0-3 epilogue, warp 4 MMA, warp 5 dz loader
-constexpr int TMEM_COLS = 32;
+// As in the forward kernel, ring stages are only as far apart as the rows a group really has: the MMA's rows
+// beyond the group's are whatever follows in shared memory, and the accumulator rows they produce are never read.
+constexpr int N_ISS = 4;                         // MMA-issuing threads (one lane each of warps 4, 6, 7, 8), one accumulator each
+constexpr int NUM_THREADS = 288;                 // warps 0-3 epilogue, warp 4 W loader + issuer 0, warp 5 dz loader, warps 6-8 issuers 1-3
+constexpr int TMEM_COLS = N_ISS * UNITS;
+// One thread issues a tcgen05.mma of N = 16 only every hundred cycles or so (descriptor arithmetic, barrier polling),
+// far slower than the tensor pipe runs it.  So a ring stage holds N_ISS k-blocks (one barrier round per stage), each
+// issuer takes one k-block of every stage into its own accumulator, and the epilogue adds the accumulators up.
 
 struct GradParams {
     int T, B, H, n_blocks, k_blocks;
     int rows_per_group, n_epi;
+    int tile_stride, n_stages;       // bytes between the k-block tiles of the ring (a stage is N_ISS tiles); stages in the ring
     const float *gates;              // [T*B][4H] activated gates i | f | g | o
     const float *c_all, *c0;         // [T*B][H], [B][H]
     const float *dh_all;             // [T*B][H]
@@ -172,11 +180,11 @@ lstm_grad_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __gr
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t *w_s = smem;                                           // [k_blocks][16 rows x 128 B]
-    uint8_t *a_s = smem + (size_t)p.k_blocks * W_KB;               // [STAGES][128 rows x 128 B]
-    uint64_t *bars = reinterpret_cast<uint64_t *>(a_s + (size_t)STAGES * A_STAGE);
-    uint64_t *full = bars, *empty = bars + STAGES, *w_full = bars + 2 * STAGES, *tmem_full = bars + 2 * STAGES + 1;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 2);
+    uint8_t *a_s = smem;                                           // [n_stages][rows of the group x 128 B], RING_BYTES
+    uint8_t *w_s = smem + RING_BYTES;                              // [k_blocks][16 rows x 128 B]
+    uint64_t *bars = reinterpret_cast<uint64_t *>(w_s + max(p.k_blocks * W_KB, A_TILE));
+    uint64_t *full = bars, *empty = bars + MAX_STAGES, *w_full = bars + 2 * MAX_STAGES, *tmem_full = bars + 2 * MAX_STAGES + 1;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * MAX_STAGES + 2);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -187,15 +195,15 @@ lstm_grad_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __gr
     unsigned int *counter = p.counter + grp * 32;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
+        for (int s = 0; s < p.n_stages; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], N_ISS); }
         tc::mbar_init(w_full, 1);
-        tc::mbar_init(tmem_full, 1);
+        tc::mbar_init(tmem_full, N_ISS);
         *abort_flag = 0;
         tc::fence_barrier_init();
         tc::prefetch_tmap(&tm_w);
         tc::prefetch_tmap(&tm_dz);
     }
-    for (int i = threadIdx.x; i < STAGES * A_STAGE / 16; i += NUM_THREADS) reinterpret_cast<uint4 *>(a_s)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = threadIdx.x; i < RING_BYTES / 16; i += NUM_THREADS) reinterpret_cast<uint4 *>(a_s)[i] = make_uint4(0, 0, 0, 0);
     tc::fence_proxy_async();
     if (warp == 4) { tc::tmem_alloc(tmem_slot, TMEM_COLS); tc::tmem_relinquish(); }
     tc::tc_fence_before_sync();
@@ -232,10 +240,15 @@ lstm_grad_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __gr
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) break;
                 tc::tc_fence_after_sync();
-                uint32_t d[32];
-                tc::tmem_ld_32x32(tmem_base + ((uint32_t)(warp * 32) << 16), d);     // columns 16..31 are not used
+                uint32_t d[32], d2[32];                                               // the four issuers' partial sums, 16 columns each
+                tc::tmem_ld_32x32(tmem_base + ((uint32_t)(warp * 32) << 16), d);
+                tc::tmem_ld_32x32(tmem_base + ((uint32_t)(warp * 32) << 16) + 32, d2);
                 tc::tmem_ld_wait();
                 tc::tc_fence_before_sync();
+#pragma unroll
+                for (int i = 0; i < UNITS; ++i)
+                    d[i] = __float_as_uint((__uint_as_float(d[i]) + __uint_as_float(d[UNITS + i])) +
+                                           (__uint_as_float(d2[i]) + __uint_as_float(d2[UNITS + i])));
                 if (s == p.T) {
                     if (live && p.dh0) {
                         float4 *o = reinterpret_cast<float4 *>(p.dh0 + (size_t)b * p.H + j0);
@@ -277,34 +290,13 @@ lstm_grad_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __gr
             for (int i = 0; i < UNITS; i += 4) o[i / 4] = make_float4(dc[i], dc[i + 1], dc[i + 2], dc[i + 3]);
         }
       }
-    } else if (warp == 4) {
-        // ------------------------------ W slice load + MMA issue ------------------------------
-        if (lane == 0) {
-            tc::mbar_expect_tx(w_full, (uint32_t)(p.k_blocks * W_KB));
-            for (int kb = 0; kb < p.k_blocks; ++kb) tc::tma_load_2d(w_s + (size_t)kb * W_KB, &tm_w, w_full, kb * BK, j0);
-            bool ok = tc::mbar_wait(w_full, 0, abort_flag, p.err, tc::ERR_WAIT_FULL);
-            const uint32_t idesc = tc::instr_desc_bf16(128, UNITS, false, false);
-            uint32_t it = 0;
-            for (int s = 1; s <= p.T && ok; ++s) {
-                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
-                    const int st = it % STAGES;
-                    if (!tc::mbar_wait(&full[st], (it / STAGES) & 1, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
-                    tc::tc_fence_after_sync();
-                    const uint32_t sa = tc::smem_u32(a_s + (size_t)st * A_STAGE), sb = tc::smem_u32(w_s + (size_t)kb * W_KB);
-#pragma unroll
-                    for (int kk = 0; kk < BK / 16; ++kk)
-                        tc::mma_bf16(tmem_base, tc::smem_desc(sa + kk * 32, 16, 1024), tc::smem_desc(sb + kk * 32, 16, 1024), idesc,
-                                     (kb | kk) != 0);
-                    tc::mma_commit(&empty[st]);
-                }
-                if (ok) tc::mma_commit(tmem_full);
-            }
-        }
-    } else {
+    } else if (warp == 5) {
         // ------------------------------ dz loader: dZ[T-s] rows of the group -> ring, by TMA ------------------------------
         if (lane == 0) {
-            uint32_t it = 0;
+            int st = 0;
+            uint32_t phase = 0;
             bool ok = true;
+            const uint32_t stage_bytes = (uint32_t)(N_ISS * p.rows_per_group * 128);
             for (int s = 1; s <= p.T && ok; ++s) {
                 // grid barrier: every block of the group has written its columns of dZ[T-s]
                 const unsigned int target = (unsigned int)(p.n_epi * p.n_blocks) * (unsigned int)s;
@@ -320,12 +312,47 @@ lstm_grad_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __gr
                 if (!ok) break;
                 asm volatile("fence.proxy.async.global;" ::: "memory");
                 const int row0 = (p.T - s) * p.B + b_lo;
-                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
-                    const int st = it % STAGES;
-                    if (!tc::mbar_wait(&empty[st], ((it / STAGES) & 1) ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
-                    tc::mbar_expect_tx(&full[st], (uint32_t)(p.rows_per_group * 128));
-                    tc::tma_load_2d(a_s + (size_t)st * A_STAGE, &tm_dz, &full[st], kb * BK, row0);
+                for (int kb = 0; kb < p.k_blocks; kb += N_ISS) {
+                    if (!tc::mbar_wait(&empty[st], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
+                    tc::mbar_expect_tx(&full[st], stage_bytes);
+                    uint8_t *dst = a_s + (size_t)st * N_ISS * p.tile_stride;
+#pragma unroll
+                    for (int i = 0; i < N_ISS; ++i) tc::tma_load_2d(dst + (size_t)i * p.tile_stride, &tm_dz, &full[st], (kb + i) * BK, row0);
+                    if (++st == p.n_stages) { st = 0; phase ^= 1; }
                 }
+            }
+        }
+    } else {
+        // ------------------------------ MMA issuers (warp 4 also loads the W slice) ------------------------------
+        if (lane == 0) {
+            const int iss = warp == 4 ? 0 : warp - 5;                 // warps 4, 6, 7, 8 -> issuers 0..3
+            if (iss == 0) {
+                tc::mbar_expect_tx(w_full, (uint32_t)(p.k_blocks * W_KB));
+                for (int kb = 0; kb < p.k_blocks; ++kb) tc::tma_load_2d(w_s + (size_t)kb * W_KB, &tm_w, w_full, kb * BK, j0);
+            }
+            bool ok = tc::mbar_wait(w_full, 0, abort_flag, p.err, tc::ERR_WAIT_FULL);
+            const uint32_t idesc = tc::instr_desc_bf16(128, UNITS, false, false);
+            // descriptors differ from the first one only in the start-address field (16-byte units): one add per MMA
+            const uint64_t desc_a0 = tc::smem_desc(tc::smem_u32(a_s) + (uint32_t)(iss * p.tile_stride), 16, 1024);
+            const uint64_t desc_b0 = tc::smem_desc(tc::smem_u32(w_s) + (uint32_t)(iss * W_KB), 16, 1024);
+            const uint32_t a_stage = (uint32_t)(N_ISS * p.tile_stride) >> 4, b_stage = (uint32_t)(N_ISS * W_KB) >> 4;
+            const uint32_t d_tmem = tmem_base + iss * UNITS;
+            int st = 0;
+            uint32_t phase = 0, a_off = 0;
+            for (int s = 1; s <= p.T && ok; ++s) {
+                uint32_t b_off = 0;
+                for (int kb = 0; kb < p.k_blocks; kb += N_ISS) {       // this issuer's k-block of the stage: kb + iss
+                    if (!tc::mbar_wait(&full[st], phase, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
+                    tc::tc_fence_after_sync();
+                    const uint64_t da = desc_a0 + a_off, db = desc_b0 + b_off;
+                    const uint32_t acc = kb != 0;
+#pragma unroll
+                    for (int kk = 0; kk < BK / 16; ++kk) tc::mma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, acc | (kk != 0));
+                    tc::mma_commit(&empty[st]);
+                    a_off += a_stage; b_off += b_stage;
+                    if (++st == p.n_stages) { st = 0; phase ^= 1; a_off = 0; }
+                }
+                if (ok) tc::mma_commit(tmem_full);
             }
         }
     }
@@ -395,7 +422,10 @@ relay_status_t run_steps_tc(const GradDims &d, const GradPlan &pl, char *ws, con
     p.counter = counter;
     p.err = device_error_word();
     if (!p.err) return fail(RELAY_ERR_CUDA, "no device error word");
-    const size_t smem = 1024 + (size_t)p.k_blocks * W_KB + (size_t)STAGES * A_STAGE + 256;
+    p.tile_stride = (int)align_up((size_t)rows_per_group * 128, 1024);
+    p.n_stages = std::min(MAX_STAGES, RING_BYTES / (N_ISS * p.tile_stride));
+    // what follows the ring is at least one A tile long, so the rows an MMA reads past the last stage stay inside the allocation
+    const size_t smem = 1024 + (size_t)RING_BYTES + std::max<size_t>((size_t)p.k_blocks * W_KB, A_TILE) + 1024;
     RELAY_CUDA(cudaFuncSetAttribute(lstm_grad_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     void *args[] = {(void *)&tm_w, (void *)&tm_dz, (void *)&p};
     RELAY_CUDA(cudaLaunchCooperativeKernel((const void *)lstm_grad_persistent_kernel, dim3(n_blocks * groups), dim3(NUM_THREADS), args, smem, st));

@@ -3,8 +3,8 @@
 // Block j owns 16 hidden units (64 gate columns: i, f, g, o of those units).  Its slice of W_hh
 // (64 columns x H, bf16) is loaded once by TMA and stays in shared memory for all T steps; the
 // running cell state of its units lives in registers.  Each step:
-//   one thread streams bf16(h_{t-1}) [B x H] from the exchange buffer in L2 through a 4-stage shared
-//   memory ring by TMA (all k-blocks in flight at once)  ->  one thread issues tcgen05.mma
+//   one thread streams bf16(h_{t-1}) [B x H] from the exchange buffer in L2 through a shared memory
+//   ring by TMA (as many k-blocks in flight as the ring holds)  ->  one thread issues tcgen05.mma
 //   (D[batch row, 64 gate columns] in TMEM)  ->  epilogue warps add the precomputed input projection,
 //   apply the gates, update c, write h_t (fp32 to h_all, bf16 to the exchange buffer)  ->  grid barrier.
 // Batch rows are independent, so the batch is split into groups of rows that run as separate sets of
@@ -28,14 +28,27 @@ relay_status_t make_tmap_2d_bf16(CUtensorMap *m, const void *base, uint64_t inne
 namespace {
 
 constexpr int UNITS = 16, NCOL = 4 * UNITS;      // hidden units and gate columns per block
-constexpr int BK = 64, STAGES = 6;
-constexpr int A_STAGE = 128 * BK * 2;            // 128 batch rows (rows >= B stay zero) x 64 k
+constexpr int BK = 64, MAX_STAGES = 32;
+constexpr int A_TILE = 128 * BK * 2;             // what one MMA reads as its A operand: 128 rows x 64 k
+constexpr int RING_BYTES = 96 * 1024;
 constexpr int W_KB = NCOL * BK * 2;              // one k-block of the resident W slice
-constexpr int NUM_THREADS = 192;                 // warps 0-3 epilogue, warp 4 MMA, warp 5 h loader
+// Ring stages are only as far apart as the rows a group really has (rounded up to the 1024-byte swizzle atom):
+// the MMA reads 128 rows from a stage's start, so its rows beyond the group's are whatever follows in shared
+// memory (later stages, then the W slice).  Row r of the product depends on row r of A alone, and the epilogue
+// reads only the group's rows, so those accumulator rows are never looked at; the ring holds four times as many
+// bytes in flight as it would with zero-padded 128-row stages.
+constexpr int NUM_THREADS = 224;                 // warps 0-3 epilogue, warp 4 W loader + MMA issuer 0, warp 5 h loader, warp 6 issuer 1
+constexpr int MAX_ISS = 2;
+// One thread issues a tcgen05.mma only every hundred cycles or so (descriptor arithmetic, barrier polling), slower
+// than the tensor pipe runs an N = 64 one.  With an even number of k-blocks a ring stage therefore holds two of
+// them (one barrier round per stage), each of two issuers takes one into its own accumulator, and the epilogue
+// adds the two accumulators up.
 
 struct Params {
     int T, B, H, n_blocks, k_blocks;
     int rows_per_group, n_epi;       // batch rows per block group; epilogue warps that own rows (ceil(rows_per_group / 32))
+    int tile_stride, n_stages;       // bytes between the k-block tiles of the ring (a stage is n_iss tiles); stages in the ring
+    int n_iss;                       // MMA issuers = k-blocks per stage = accumulators (1 or 2)
     const float *zx;                 // [T*B][4H] input projection + bias
     const float *h0, *c0;            // [B][H]
     float *h_all, *c_final;          // [T][B][H], [B][H]
@@ -63,11 +76,11 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t *w_s = smem;                                           // [k_blocks][64 cols x 128 B]
-    uint8_t *a_s = smem + (size_t)p.k_blocks * W_KB;               // [STAGES][128 rows x 128 B]
-    uint64_t *bars = reinterpret_cast<uint64_t *>(a_s + (size_t)STAGES * A_STAGE);
-    uint64_t *full = bars, *empty = bars + STAGES, *w_full = bars + 2 * STAGES, *tmem_full = bars + 2 * STAGES + 1;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 2);
+    uint8_t *a_s = smem;                                           // [n_stages][rows of the group x 128 B], RING_BYTES
+    uint8_t *w_s = smem + RING_BYTES;                              // [k_blocks][64 cols x 128 B] (at least A_TILE bytes: see above)
+    uint64_t *bars = reinterpret_cast<uint64_t *>(w_s + max(p.k_blocks * W_KB, A_TILE));
+    uint64_t *full = bars, *empty = bars + MAX_STAGES, *w_full = bars + 2 * MAX_STAGES, *tmem_full = bars + 2 * MAX_STAGES + 1;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * MAX_STAGES + 2);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -78,19 +91,19 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
     unsigned int *counter = p.counter + grp * 32;                 // one barrier counter per group (128 B apart)
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
+        for (int s = 0; s < p.n_stages; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], p.n_iss); }
         tc::mbar_init(w_full, 1);
-        tc::mbar_init(tmem_full, 1);
+        tc::mbar_init(tmem_full, p.n_iss);
         *abort_flag = 0;
         tc::fence_barrier_init();
         tc::prefetch_tmap(&tm_w);
         tc::prefetch_tmap(&tm_h0);
         tc::prefetch_tmap(&tm_h1);
     }
-    // rows >= B of every ring stage are zero for the whole kernel
-    for (int i = threadIdx.x; i < STAGES * A_STAGE / 16; i += NUM_THREADS) reinterpret_cast<uint4 *>(a_s)[i] = make_uint4(0, 0, 0, 0);
+    // the ring starts as zeros (finite values for the accumulator rows nobody reads)
+    for (int i = threadIdx.x; i < RING_BYTES / 16; i += NUM_THREADS) reinterpret_cast<uint4 *>(a_s)[i] = make_uint4(0, 0, 0, 0);
     tc::fence_proxy_async();
-    if (warp == 4) { tc::tmem_alloc(tmem_slot, 64); tc::tmem_relinquish(); }
+    if (warp == 4) { tc::tmem_alloc(tmem_slot, MAX_ISS * NCOL); tc::tmem_relinquish(); }
     tc::tc_fence_before_sync();
     __syncthreads();
     tc::tc_fence_after_sync();
@@ -143,7 +156,19 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
             const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16);
             tc::tmem_ld_32x32(taddr, d0);
             tc::tmem_ld_32x32(taddr + 32, d1);
-            tc::tmem_ld_wait();
+            if (p.n_iss == 2) {                           // warp-uniform: the second issuer's partial sums
+                uint32_t e0[32], e1[32];
+                tc::tmem_ld_32x32(taddr + NCOL, e0);
+                tc::tmem_ld_32x32(taddr + NCOL + 32, e1);
+                tc::tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    d0[i] = __float_as_uint(__uint_as_float(d0[i]) + __uint_as_float(e0[i]));
+                    d1[i] = __float_as_uint(__uint_as_float(d1[i]) + __uint_as_float(e1[i]));
+                }
+            } else {
+                tc::tmem_ld_wait();
+            }
             tc::tc_fence_before_sync();
             float hn[UNITS];
             if (live) {
@@ -177,34 +202,13 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
             for (int i = 0; i < UNITS; ++i) p.c_final[(size_t)b * p.H + j0 + i] = c[i];
         }
       }
-    } else if (warp == 4) {
-        // ------------------------------ W slice load + MMA issue ------------------------------
-        if (lane == 0) {
-            tc::mbar_expect_tx(w_full, (uint32_t)(p.k_blocks * W_KB));
-            for (int kb = 0; kb < p.k_blocks; ++kb) tc::tma_load_2d(w_s + (size_t)kb * W_KB, &tm_w, w_full, kb * BK, blk * NCOL);
-            bool ok = tc::mbar_wait(w_full, 0, abort_flag, p.err, tc::ERR_WAIT_FULL);
-            const uint32_t idesc = tc::instr_desc_bf16(128, NCOL, false, false);
-            uint32_t it = 0;
-            for (int t = 0; t < p.T && ok; ++t) {
-                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    if (!tc::mbar_wait(&full[s], (it / STAGES) & 1, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
-                    tc::tc_fence_after_sync();
-                    const uint32_t sa = tc::smem_u32(a_s + (size_t)s * A_STAGE), sb = tc::smem_u32(w_s + (size_t)kb * W_KB);
-#pragma unroll
-                    for (int kk = 0; kk < BK / 16; ++kk)
-                        tc::mma_bf16(tmem_base, tc::smem_desc(sa + kk * 32, 16, 1024), tc::smem_desc(sb + kk * 32, 16, 1024), idesc,
-                                     (kb | kk) != 0);
-                    tc::mma_commit(&empty[s]);
-                }
-                if (ok) tc::mma_commit(tmem_full);
-            }
-        }
-    } else {
+    } else if (warp == 5) {
         // ------------------------------ h loader: bf16(h_{t-1}) -> ring, by TMA ------------------------------
         if (lane == 0) {
-            uint32_t it = 0;
+            int s = 0;
+            uint32_t phase = 0;
             bool ok = true;
+            const uint32_t stage_bytes = (uint32_t)(p.n_iss * p.rows_per_group * 128);
             for (int t = 0; t < p.T && ok; ++t) {
                 // grid barrier: every block has published its part of h_{t-1}
                 const unsigned int target = (unsigned int)(p.n_epi * p.n_blocks) * (unsigned int)(t + 1);   // n_epi arrivals per block
@@ -220,18 +224,53 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
                 if (!ok) break;
                 asm volatile("fence.proxy.async.global;" ::: "memory");
                 const CUtensorMap *tm_h = (t & 1) ? &tm_h1 : &tm_h0;
-                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    if (!tc::mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
-                    tc::mbar_expect_tx(&full[s], (uint32_t)(p.rows_per_group * 128));
-                    tc::tma_load_2d(a_s + (size_t)s * A_STAGE, tm_h, &full[s], kb * BK, b_lo);   // the group's rows; the rest stay zero
+                for (int kb = 0; kb < p.k_blocks; kb += p.n_iss) {
+                    if (!tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
+                    tc::mbar_expect_tx(&full[s], stage_bytes);
+                    uint8_t *dst = a_s + (size_t)s * p.n_iss * p.tile_stride;
+                    for (int i = 0; i < p.n_iss; ++i)
+                        tc::tma_load_2d(dst + (size_t)i * p.tile_stride, tm_h, &full[s], (kb + i) * BK, b_lo);   // the group's rows only
+                    if (++s == p.n_stages) { s = 0; phase ^= 1; }
                 }
+            }
+        }
+    } else {
+        // ------------------------------ MMA issuers (warp 4 also loads the W slice) ------------------------------
+        const int iss = warp == 4 ? 0 : 1;
+        if (lane == 0 && iss < p.n_iss) {
+            if (iss == 0) {
+                tc::mbar_expect_tx(w_full, (uint32_t)(p.k_blocks * W_KB));
+                for (int kb = 0; kb < p.k_blocks; ++kb) tc::tma_load_2d(w_s + (size_t)kb * W_KB, &tm_w, w_full, kb * BK, blk * NCOL);
+            }
+            bool ok = tc::mbar_wait(w_full, 0, abort_flag, p.err, tc::ERR_WAIT_FULL);
+            const uint32_t idesc = tc::instr_desc_bf16(128, NCOL, false, false);
+            // descriptors differ from the first one only in the start-address field (16-byte units): one add per MMA
+            const uint64_t desc_a0 = tc::smem_desc(tc::smem_u32(a_s) + (uint32_t)(iss * p.tile_stride), 16, 1024);
+            const uint64_t desc_b0 = tc::smem_desc(tc::smem_u32(w_s) + (uint32_t)(iss * W_KB), 16, 1024);
+            const uint32_t a_stage = (uint32_t)(p.n_iss * p.tile_stride) >> 4, b_stage = (uint32_t)(p.n_iss * W_KB) >> 4;
+            const uint32_t d_tmem = tmem_base + iss * NCOL;
+            int s = 0;
+            uint32_t phase = 0, a_off = 0;
+            for (int t = 0; t < p.T && ok; ++t) {
+                uint32_t b_off = 0;
+                for (int kb = 0; kb < p.k_blocks; kb += p.n_iss) {     // this issuer's k-block of the stage: kb + iss
+                    if (!tc::mbar_wait(&full[s], phase, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
+                    tc::tc_fence_after_sync();
+                    const uint64_t da = desc_a0 + a_off, db = desc_b0 + b_off;
+                    const uint32_t acc = kb != 0;
+#pragma unroll
+                    for (int kk = 0; kk < BK / 16; ++kk) tc::mma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, acc | (kk != 0));
+                    tc::mma_commit(&empty[s]);
+                    a_off += a_stage; b_off += b_stage;
+                    if (++s == p.n_stages) { s = 0; phase ^= 1; a_off = 0; }
+                }
+                if (ok) tc::mma_commit(tmem_full);
             }
         }
     }
     tc::tc_fence_before_sync();
     __syncthreads();
-    if (warp == 4) { tc::tc_fence_after_sync(); tc::tmem_dealloc(tmem_base, 64); }
+    if (warp == 4) { tc::tc_fence_after_sync(); tc::tmem_dealloc(tmem_base, MAX_ISS * NCOL); }
 }
 
 // wp[blk][g*16 + i][k] = w_hh[k][g*H + blk*16 + i]
@@ -296,7 +335,11 @@ relay_status_t launch_lstm_tc(int64_t T, int64_t B, int64_t H, const float *zx, 
     p.zx = zx; p.h0 = h0; p.c0 = c0; p.h_all = h_all; p.c_final = c_final; p.hq = hq; p.counter = counter;
     p.err = device_error_word();
     if (!p.err) return fail(RELAY_ERR_CUDA, "no device error word");
-    const size_t smem = 1024 + (size_t)p.k_blocks * W_KB + (size_t)STAGES * A_STAGE + 256;
+    p.n_iss = p.k_blocks % 2 == 0 ? 2 : 1;
+    p.tile_stride = (int)align_up((size_t)rows_per_group * 128, 1024);
+    p.n_stages = std::min(MAX_STAGES, RING_BYTES / (p.n_iss * p.tile_stride));
+    // what follows the ring is at least one A tile long, so the rows an MMA reads past the last stage stay inside the allocation
+    const size_t smem = 1024 + (size_t)RING_BYTES + std::max<size_t>((size_t)p.k_blocks * W_KB, A_TILE) + 1024;
     RELAY_CUDA(cudaFuncSetAttribute(lstm_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     void *args[] = {(void *)&tm_w, (void *)&tm_h0, (void *)&tm_h1, (void *)&p};
     RELAY_CUDA(cudaLaunchCooperativeKernel((const void *)lstm_persistent_kernel, dim3(n_blocks * groups), dim3(NUM_THREADS), args, smem, st));
