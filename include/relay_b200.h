@@ -145,7 +145,9 @@ typedef struct {
  * the way Fig. 5 derives the type of an expression from the types of its parts.
  * ------------------------------------------------------------------------------------------- */
 
-/* dense: Tensor(t,(M,K)) x Tensor(t,(K,N)) -> Tensor(t,(M,N)), t in {f32, bf16} (Fig. 3 relay.linear). */
+/* dense: Tensor(t,(M,K)) x Tensor(t,(K,N)) -> Tensor(t,(M,N)), t in {f32, bf16} (Fig. 3 relay.linear).
+ * x may carry leading batch axes (Section 5.2: batching a program adds a leading axis to its tensors):
+ * Tensor(t,(B1,..,Bk,M,K)) x Tensor(t,(K,N)) -> Tensor(t,(B1,..,Bk,M,N)), rank at most RELAY_MAX_RANK. */
 relay_status_t relay_infer_dense(const relay_tensor_t *x, const relay_tensor_t *w, relay_tensor_t *out);
 
 /* conv2d: x:(N,C,H,W) NCHW, w:(O,C,R,S) OIHW -> (N,O,P,Q) with P = floor((H+2p-R)/s)+1
@@ -199,7 +201,9 @@ size_t relay_workspace_bytes_lstm_grad(const relay_tensor_t *x, const relay_tens
  * names):   y[m,n] = act( sum_k x[m,k] * w[k,n] + b[n] ).
  *   x:(M,K)  w:(K,N)  b:(N) or NULL  ->  y:(M,N); x, w, y share one dtype t in {f32, bf16};
  *   b has dtype t or f32.  f32 runs in true fp32 (FMA); bf16 multiplies bf16 and accumulates
- *   in fp32, rounding once on the store of y. */
+ *   in fp32, rounding once on the store of y.
+ *   x and y may carry the same leading batch axes, x:(B1,..,Bk,M,K) -> y:(B1,..,Bk,M,N): the batch
+ *   elements share w and b, so the call is one product over the B1*..*Bk*M stacked rows. */
 relay_status_t relay_fused_dense_act(const relay_tensor_t *x, const relay_tensor_t *w, const relay_tensor_t *b,
                                      int32_t act, const relay_tensor_t *y, void *ws, size_t ws_bytes, void *stream);
 
@@ -211,7 +215,9 @@ relay_status_t relay_fused_dense_act(const relay_tensor_t *x, const relay_tensor
  *        relu' = 1[y>0] (so relu'(0)=0), tanh' = 1-y^2, sigmoid' = y(1-y);
  *   dx[m,k] = sum_n dZ[m,n] w[k,n];   dw[k,n] = sum_m x[m,k] dZ[m,n];   db[n] = sum_m dZ[m,n].
  *   dx, db may be NULL (not wanted); dw is required.  dx, dw have dtype t; db is f32 (or t for
- *   t = f32).  Sums are deterministic (fixed order, no float atomics). */
+ *   t = f32).  Sums are deterministic (fixed order, no float atomics).
+ *   With leading batch axes on x, y, dy and dx, m runs over all batch elements' rows: dw and db are
+ *   summed over the batch (one weight, used by every element: its partials add up, Section 4.2). */
 relay_status_t relay_fused_dense_act_grad(const relay_tensor_t *x, const relay_tensor_t *w, const relay_tensor_t *y,
                                           const relay_tensor_t *dy, int32_t act, const relay_tensor_t *dx,
                                           const relay_tensor_t *dw, const relay_tensor_t *db, void *ws,
@@ -220,7 +226,11 @@ relay_status_t relay_fused_dense_act_grad(const relay_tensor_t *x, const relay_t
 /* conv2d anchor (Fig. 3 relay.conv2d) as cross-correlation with zero padding, run as an
  * implicit GEMM and fused with per-channel bias and activation:
  *   y[n,o,p,q] = act( b[o] + sum_{c,r,s} x[n,c,p*st-pad+r,q*st-pad+s] * w[o,c,r,s] ).
- *   x:(N,C,H,W) NCHW  w:(O,C,R,S) OIHW  b:(O) or NULL  ->  y:(N,O,P,Q) NCHW. */
+ *   x:(N,C,H,W) NCHW  w:(O,C,R,S) OIHW  b:(O) or NULL  ->  y:(N,O,P,Q) NCHW.
+ * Layout-tagged activations (Section 5.2 names layout change among the operator-level optimisations): x may
+ * instead be tagged RELAY_NHWC with shape (N,H,W,C); then y is NHWC of shape (N,P,Q,O) (and in the gradient
+ * group y, dy, dx are NHWC too); w stays OIHW.  Same values, other memory order: the call converts through
+ * the workspace (the bf16 3x3 tensor-core instance reads an NHWC x as it is). */
 relay_status_t relay_fused_conv2d_act(const relay_tensor_t *x, const relay_tensor_t *w, const relay_tensor_t *b,
                                       const relay_conv2d_attrs_t *attrs, int32_t act, const relay_tensor_t *y,
                                       void *ws, size_t ws_bytes, void *stream);

@@ -226,14 +226,14 @@ def relay_workspace_bytes_dense_act_grad(x, w) -> int:
     return int(lib().relay_workspace_bytes_dense_act_grad(_ref(desc(x)), _ref(desc(w))))
 
 
-def relay_workspace_bytes_conv2d_act(x, w, stride, pad) -> int:
+def relay_workspace_bytes_conv2d_act(x, w, stride, pad, layout=NCHW) -> int:
     at = Conv2dAttrs(stride, pad, 1, 1)
-    return int(lib().relay_workspace_bytes_conv2d_act(_ref(desc(x, NCHW)), _ref(desc(w, OIHW)), ctypes.byref(at)))
+    return int(lib().relay_workspace_bytes_conv2d_act(_ref(desc(x, layout)), _ref(desc(w, OIHW)), ctypes.byref(at)))
 
 
-def relay_workspace_bytes_conv2d_act_grad(x, w, stride, pad) -> int:
+def relay_workspace_bytes_conv2d_act_grad(x, w, stride, pad, layout=NCHW) -> int:
     at = Conv2dAttrs(stride, pad, 1, 1)
-    return int(lib().relay_workspace_bytes_conv2d_act_grad(_ref(desc(x, NCHW)), _ref(desc(w, OIHW)), ctypes.byref(at)))
+    return int(lib().relay_workspace_bytes_conv2d_act_grad(_ref(desc(x, layout)), _ref(desc(w, OIHW)), ctypes.byref(at)))
 
 
 def relay_workspace_bytes_reduce(inputs, specs) -> int:
@@ -258,18 +258,19 @@ def relay_fused_dense_act_grad(x, w, y, dy, act, dx, dw, db, ws=None):
                                             _ref(desc(dx)), _ref(desc(dw)), _ref(desc(db)), wp, wb, _stream()))
 
 
-def relay_fused_conv2d_act(x, w, b, stride, pad, act, y, ws=None):
+def relay_fused_conv2d_act(x, w, b, stride, pad, act, y, ws=None, layout=NCHW):
+    """`layout` tags x and y: NCHW tensors of shape (N,C,H,W) or NHWC tensors of shape (N,H,W,C)."""
     wp, wb = _ws(ws)
     at = Conv2dAttrs(stride, pad, 1, 1)
-    _check(lib().relay_fused_conv2d_act(_ref(desc(x, NCHW)), _ref(desc(w, OIHW)), _ref(desc(b)), ctypes.byref(at), int(act),
-                                        _ref(desc(y, NCHW)), wp, wb, _stream()))
+    _check(lib().relay_fused_conv2d_act(_ref(desc(x, layout)), _ref(desc(w, OIHW)), _ref(desc(b)), ctypes.byref(at), int(act),
+                                        _ref(desc(y, layout)), wp, wb, _stream()))
 
 
-def relay_fused_conv2d_act_grad(x, w, y, dy, stride, pad, act, dx, dw, db, ws=None):
+def relay_fused_conv2d_act_grad(x, w, y, dy, stride, pad, act, dx, dw, db, ws=None, layout=NCHW):
     wp, wb = _ws(ws)
     at = Conv2dAttrs(stride, pad, 1, 1)
-    _check(lib().relay_fused_conv2d_act_grad(_ref(desc(x, NCHW)), _ref(desc(w, OIHW)), _ref(desc(y, NCHW)),
-                                             _ref(desc(dy, NCHW)), ctypes.byref(at), int(act), _ref(desc(dx, NCHW)),
+    _check(lib().relay_fused_conv2d_act_grad(_ref(desc(x, layout)), _ref(desc(w, OIHW)), _ref(desc(y, layout)),
+                                             _ref(desc(dy, layout)), ctypes.byref(at), int(act), _ref(desc(dx, layout)),
                                              _ref(desc(dw, OIHW)), _ref(desc(db)), wp, wb, _stream()))
 
 

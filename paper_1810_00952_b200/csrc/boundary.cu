@@ -85,6 +85,16 @@ relay_status_t check_shape(const relay_tensor_t *t, std::initializer_list<int64_
     return RELAY_OK;
 }
 
+relay_status_t check_shape_n(const relay_tensor_t *t, const int64_t *want, int rank, const char *name)
+{
+    if (t->rank != rank) return fail(RELAY_ERR_RANK, "%s: rank %d, operator type needs rank %d", name, t->rank, rank);
+    for (int d = 0; d < rank; ++d)
+        if (t->shape[d] != want[d])
+            return fail(RELAY_ERR_SHAPE, "%s: axis %d has extent %lld, operator type needs %lld", name, d, (long long)t->shape[d],
+                        (long long)want[d]);
+    return RELAY_OK;
+}
+
 relay_status_t check_data(const relay_tensor_t *t, const char *name)
 {
     if (numel(t) == 0) return RELAY_OK;
@@ -209,17 +219,20 @@ relay_status_t relay_infer_dense(const relay_tensor_t *x, const relay_tensor_t *
     RELAY_TRY(check_not_null(out, "out"));
     RELAY_TRY(check_type(x, "x"));
     RELAY_TRY(check_type(w, "w"));
-    RELAY_TRY(check_rank(x, 2, "x"));
+    if (x->rank < 2) return fail(RELAY_ERR_RANK, "x: rank %d, operator type needs rank 2 or more (batch axes, M, K)", x->rank);
     RELAY_TRY(check_rank(w, 2, "w"));
     if (!is_float(x->dtype)) return fail(RELAY_ERR_DTYPE, "x: dense needs a float base type, got %s", dtype_name(x->dtype));
     RELAY_TRY(check_dtype(w, x->dtype, "w"));
     RELAY_TRY(check_layout(x, RELAY_ROWMAJOR, RELAY_ROWMAJOR, "x"));
     RELAY_TRY(check_layout(w, RELAY_ROWMAJOR, RELAY_ROWMAJOR, "w"));
-    if (x->shape[1] != w->shape[0])
-        return fail(RELAY_ERR_SHAPE, "dense: x is (%lld,%lld) but w is (%lld,%lld): inner extents differ",
-                    (long long)x->shape[0], (long long)x->shape[1], (long long)w->shape[0], (long long)w->shape[1]);
-    int64_t s[2] = {x->shape[0], w->shape[1]};
-    fill_out(out, x->dtype, RELAY_ROWMAJOR, 2, s);
+    const int r = x->rank;
+    if (x->shape[r - 1] != w->shape[0])
+        return fail(RELAY_ERR_SHAPE, "dense: x is (..,%lld,%lld) but w is (%lld,%lld): inner extents differ",
+                    (long long)x->shape[r - 2], (long long)x->shape[r - 1], (long long)w->shape[0], (long long)w->shape[1]);
+    int64_t s[RELAY_MAX_RANK];
+    for (int d = 0; d < r - 1; ++d) s[d] = x->shape[d];
+    s[r - 1] = w->shape[1];
+    fill_out(out, x->dtype, RELAY_ROWMAJOR, r, s);
     return RELAY_OK;
 }
 
@@ -237,21 +250,23 @@ relay_status_t relay_infer_conv2d(const relay_tensor_t *x, const relay_tensor_t 
     RELAY_TRY(check_rank(w, 4, "w"));
     if (!is_float(x->dtype)) return fail(RELAY_ERR_DTYPE, "x: conv2d needs a float base type, got %s", dtype_name(x->dtype));
     RELAY_TRY(check_dtype(w, x->dtype, "w"));
-    RELAY_TRY(check_layout(x, RELAY_NCHW, RELAY_NCHW, "x"));
+    RELAY_TRY(check_layout(x, RELAY_NCHW, RELAY_NHWC, "x"));
     RELAY_TRY(check_layout(w, RELAY_OIHW, RELAY_OIHW, "w"));
-    if (x->shape[1] != w->shape[1])
-        return fail(RELAY_ERR_SHAPE, "conv2d: x has %lld channels, w expects %lld", (long long)x->shape[1],
-                    (long long)w->shape[1]);
+    const bool nhwc = x->layout == RELAY_NHWC;            // shape is (N,H,W,C) then: tensors are row-major in the order of `shape`
+    const int64_t xc = nhwc ? x->shape[3] : x->shape[1];
+    if (xc != w->shape[1])
+        return fail(RELAY_ERR_SHAPE, "conv2d: x has %lld channels, w expects %lld", (long long)xc, (long long)w->shape[1]);
     if (attrs->stride < 1 || attrs->pad < 0) return fail(RELAY_ERR_ATTR, "conv2d: stride %d / pad %d invalid", attrs->stride, attrs->pad);
     if (attrs->dilation != 1 || attrs->groups != 1)
         return fail(RELAY_ERR_ATTR, "conv2d: dilation %d / groups %d: only 1 is defined here", attrs->dilation, attrs->groups);
-    int64_t H = x->shape[2], W = x->shape[3], R = w->shape[2], S = w->shape[3];
+    int64_t H = nhwc ? x->shape[1] : x->shape[2], W = nhwc ? x->shape[2] : x->shape[3], R = w->shape[2], S = w->shape[3];
     if (R < 1 || S < 1 || H + 2 * attrs->pad < R || W + 2 * attrs->pad < S)
         return fail(RELAY_ERR_SHAPE, "conv2d: %lldx%lld window does not fit the padded %lldx%lld image", (long long)R,
                     (long long)S, (long long)(H + 2 * attrs->pad), (long long)(W + 2 * attrs->pad));
-    int64_t s[4] = {x->shape[0], w->shape[0], (H + 2 * attrs->pad - R) / attrs->stride + 1,
-                    (W + 2 * attrs->pad - S) / attrs->stride + 1};
-    fill_out(out, x->dtype, RELAY_NCHW, 4, s);
+    const int64_t P = (H + 2 * attrs->pad - R) / attrs->stride + 1, Q = (W + 2 * attrs->pad - S) / attrs->stride + 1;
+    int64_t s[4] = {x->shape[0], w->shape[0], P, Q};
+    if (nhwc) { s[1] = P; s[2] = Q; s[3] = w->shape[0]; }
+    fill_out(out, x->dtype, nhwc ? RELAY_NHWC : RELAY_NCHW, 4, s);
     return RELAY_OK;
 }
 

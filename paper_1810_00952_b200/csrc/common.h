@@ -78,6 +78,7 @@ relay_status_t check_rank(const relay_tensor_t *t, int rank, const char *name);
 relay_status_t check_dtype(const relay_tensor_t *t, int32_t dt, const char *name);
 relay_status_t check_layout(const relay_tensor_t *t, int32_t a, int32_t b, const char *name);
 relay_status_t check_shape(const relay_tensor_t *t, std::initializer_list<int64_t> want, const char *name);
+relay_status_t check_shape_n(const relay_tensor_t *t, const int64_t *want, int rank, const char *name);
 relay_status_t check_data(const relay_tensor_t *t, const char *name);  // non-null (if numel>0), 16 B aligned
 relay_status_t check_workspace(const void *ws, size_t have, size_t need);
 

@@ -7,7 +7,12 @@ namespace relay {
 struct ConvDims {
     int64_t Nb = 0, C = 0, H = 0, W = 0, O = 0, R = 0, S = 0, P = 0, Q = 0;
     int32_t stride = 1, pad = 0, dt = RELAY_F32;
+    bool nhwc = false;                // x, y, dy, dx are (N,H,W,C) tensors; the kernels below work on NCHW
 };
+
+// layout change: out[b][s][r] = in[b][r][s] for `batch` matrices of R x S elements of 2 or 4 bytes
+// (NCHW -> NHWC: R = C, S = H*W;  NHWC -> NCHW: R = H*W, S = C)
+relay_status_t launch_layout_change(int32_t dt, const void *in, void *out, int64_t batch, int64_t R, int64_t S, cudaStream_t st);
 
 // direct (SIMT) tier: any stride / pad / window, fp32 accumulation in a fixed order
 relay_status_t launch_conv_fwd_direct(const ConvDims &d, const void *x, const void *w, const void *b, int32_t b_dt, int act,
@@ -20,8 +25,9 @@ relay_status_t launch_conv_db(const ConvDims &d, const void *dz, float *db, cuda
 bool conv_tc_eligible(const ConvDims &d);
 size_t conv_tc_fwd_workspace(const ConvDims &d);
 size_t conv_tc_grad_workspace(const ConvDims &d);
-relay_status_t launch_conv_fwd_tc(const ConvDims &d, const void *x, const void *w, const void *b, int32_t b_dt, int act, void *y,
-                                  void *ws, cudaStream_t st);
+// `x_is_nhwc`: x is already in the kernel's own activation layout, the repack pass is skipped (y is NCHW either way)
+relay_status_t launch_conv_fwd_tc(const ConvDims &d, const void *x, bool x_is_nhwc, const void *w, const void *b, int32_t b_dt, int act,
+                                  void *y, void *ws, cudaStream_t st);
 // whole gradient group: dZ = dy (.) act'(y) (kept in NHWC), db, dx (if wanted), dw
 relay_status_t launch_conv_grad_tc(const ConvDims &d, const void *x, const void *w, const void *y, const void *dy, int act, void *dx,
                                    void *dw, float *db, void *ws, cudaStream_t st);

@@ -166,4 +166,31 @@ relay_status_t launch_conv_db(const ConvDims &d, const void *dz, float *db, cuda
     return check_launch("conv_db");
 }
 
+// ---- layout change (NCHW <-> NHWC): batched transpose through a 32 x 33 shared-memory tile --------------------
+template <typename T>
+__global__ void __launch_bounds__(256) layout_change_kernel(const T *__restrict__ in, T *__restrict__ out, int64_t R, int64_t S)
+{
+    __shared__ T tile[32][33];
+    const int64_t b = blockIdx.z;
+    const int64_t r0 = (int64_t)blockIdx.y * 32, s0 = (int64_t)blockIdx.x * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const T *src = in + b * R * S;
+    T *dst = out + b * R * S;
+    for (int i = ty; i < 32; i += 8)
+        if (r0 + i < R && s0 + tx < S) tile[i][tx] = src[(r0 + i) * S + s0 + tx];
+    __syncthreads();
+    for (int i = ty; i < 32; i += 8)
+        if (s0 + i < S && r0 + tx < R) dst[(s0 + i) * R + r0 + tx] = tile[tx][i];
+}
+
+relay_status_t launch_layout_change(int32_t dt, const void *in, void *out, int64_t batch, int64_t R, int64_t S, cudaStream_t st)
+{
+    if (batch == 0 || R == 0 || S == 0) return RELAY_OK;
+    if (batch > 65535 || (R + 31) / 32 > 65535) return fail(RELAY_ERR_UNSUPPORTED, "layout change: extent exceeds the grid limit");
+    dim3 grid((unsigned)((S + 31) / 32), (unsigned)((R + 31) / 32), (unsigned)batch);
+    if (dtype_size(dt) == 2) layout_change_kernel<<<grid, 256, 0, st>>>((const uint16_t *)in, (uint16_t *)out, R, S);
+    else layout_change_kernel<<<grid, 256, 0, st>>>((const uint32_t *)in, (uint32_t *)out, R, S);
+    return check_launch("layout_change");
+}
+
 }  // namespace relay

@@ -931,13 +931,17 @@ size_t conv_tc_grad_workspace(const ConvDims &d)
     return pl.ok ? pl.x_nhwc + pl.dz_nhwc + pl.wpack + pl.part + pl.db_part : 0;
 }
 
-relay_status_t launch_conv_fwd_tc(const ConvDims &d, const void *x, const void *w, const void *b, int32_t b_dt, int act, void *y,
-                                  void *ws, cudaStream_t st)
+relay_status_t launch_conv_fwd_tc(const ConvDims &d, const void *x, bool x_is_nhwc, const void *w, const void *b, int32_t b_dt, int act,
+                                  void *y, void *ws, cudaStream_t st)
 {
     TcPlan pl = plan(d);
     char *base = (char *)ws;
-    void *x_nhwc = base, *wf = base + pl.x_nhwc;
-    RELAY_TRY(launch_transpose(false, x, nullptr, x_nhwc, d.Nb, d.C, d.H * d.W, 0, nullptr, st));
+    void *wf = base + pl.x_nhwc;
+    const void *x_nhwc = x;
+    if (!x_is_nhwc) {
+        RELAY_TRY(launch_transpose(false, x, nullptr, base, d.Nb, d.C, d.H * d.W, 0, nullptr, st));
+        x_nhwc = base;
+    }
     RELAY_CUDA(launch_pdl(pack_weights_kernel, dim3((unsigned)((d.O * d.C * 9 + 255) / 256)), dim3(256), 0, st, (const __nv_bfloat16 *)w, (__nv_bfloat16 *)wf, (__nv_bfloat16 *)nullptr, (int)d.O, (int)d.C, 3, 3));
     RELAY_TRY(check_launch("pack_weights"));
     return launch_fprop(d, pl, x_nhwc, (int)d.C, wf, (int)d.O, b, b_dt, act, y, st);

@@ -52,7 +52,15 @@ relay_status_t act_grad_any(int32_t dt, const void *dy, const void *y, void *dz,
     return RELAY_OK;
 }
 
-struct DenseDims { int64_t M, K, N; int32_t dt; };
+// M counts the rows of all leading batch axes together: a batch of products with one weight matrix is one
+// product over the stacked rows (Section 5.2: batching adds a leading axis to every tensor of the program)
+struct DenseDims {
+    int64_t M, K, N;
+    int32_t dt;
+    int rank;                         // of x, y, dy, dx
+    int64_t xs[RELAY_MAX_RANK];       // x's shape;  ys: the same with N as last extent
+    int64_t ys[RELAY_MAX_RANK];
+};
 
 // type relation of the dense anchor on concrete descriptors, in the documented check order
 static relay_status_t check_dense(const relay_tensor_t *x, const relay_tensor_t *w, const relay_tensor_t *b, DenseDims *d)
@@ -66,7 +74,10 @@ static relay_status_t check_dense(const relay_tensor_t *x, const relay_tensor_t 
             return fail(RELAY_ERR_DTYPE, "b: base type %s, needs %s or f32", dtype_name(b->dtype), dtype_name(x->dtype));
         RELAY_TRY(check_shape(b, {w->shape[1]}, "b"));
     }
-    d->M = x->shape[0]; d->K = x->shape[1]; d->N = w->shape[1]; d->dt = x->dtype;
+    d->rank = x->rank;
+    d->M = 1;
+    for (int i = 0; i < x->rank; ++i) { d->xs[i] = x->shape[i]; d->ys[i] = yt.shape[i]; if (i < x->rank - 1) d->M *= x->shape[i]; }
+    d->K = x->shape[x->rank - 1]; d->N = w->shape[1]; d->dt = x->dtype;
     return RELAY_OK;
 }
 
@@ -103,10 +114,10 @@ extern "C" relay_status_t relay_fused_dense_act(const relay_tensor_t *x, const r
     DenseDims d{};
     RELAY_TRY(check_dense(x, w, b, &d));
     RELAY_TRY(check_type(y, "y"));
-    RELAY_TRY(check_rank(y, 2, "y"));
+    RELAY_TRY(check_rank(y, d.rank, "y"));
     RELAY_TRY(check_dtype(y, d.dt, "y"));
     RELAY_TRY(check_layout(y, RELAY_ROWMAJOR, RELAY_ROWMAJOR, "y"));
-    RELAY_TRY(check_shape(y, {d.M, d.N}, "y"));
+    RELAY_TRY(check_shape_n(y, d.ys, d.rank, "y"));
     if (act < RELAY_ACT_NONE || act > RELAY_ACT_SIGMOID) return fail(RELAY_ERR_ATTR, "unknown activation %d", act);
     RELAY_TRY(check_data(x, "x"));
     RELAY_TRY(check_data(w, "w"));
@@ -140,16 +151,16 @@ extern "C" relay_status_t relay_fused_dense_act_grad(const relay_tensor_t *x, co
     RELAY_TRY(check_dense(x, w, nullptr, &d));
     const relay_tensor_t *mn[2] = {y, dy};
     const char *mn_name[2] = {"y", "dy"};
-    for (int i = 0; i < 2; ++i) { RELAY_TRY(check_type(mn[i], mn_name[i])); RELAY_TRY(check_rank(mn[i], 2, mn_name[i])); }
-    if (dx) { RELAY_TRY(check_type(dx, "dx")); RELAY_TRY(check_rank(dx, 2, "dx")); }
+    for (int i = 0; i < 2; ++i) { RELAY_TRY(check_type(mn[i], mn_name[i])); RELAY_TRY(check_rank(mn[i], d.rank, mn_name[i])); }
+    if (dx) { RELAY_TRY(check_type(dx, "dx")); RELAY_TRY(check_rank(dx, d.rank, "dx")); }
     RELAY_TRY(check_type(dw, "dw")); RELAY_TRY(check_rank(dw, 2, "dw"));
     if (db) { RELAY_TRY(check_type(db, "db")); RELAY_TRY(check_rank(db, 1, "db")); }
     for (int i = 0; i < 2; ++i) RELAY_TRY(check_dtype(mn[i], d.dt, mn_name[i]));
     if (dx) RELAY_TRY(check_dtype(dx, d.dt, "dx"));
     RELAY_TRY(check_dtype(dw, d.dt, "dw"));
     if (db) RELAY_TRY(check_dtype(db, RELAY_F32, "db"));
-    for (int i = 0; i < 2; ++i) RELAY_TRY(check_shape(mn[i], {d.M, d.N}, mn_name[i]));
-    if (dx) RELAY_TRY(check_shape(dx, {d.M, d.K}, "dx"));
+    for (int i = 0; i < 2; ++i) RELAY_TRY(check_shape_n(mn[i], d.ys, d.rank, mn_name[i]));
+    if (dx) RELAY_TRY(check_shape_n(dx, d.xs, d.rank, "dx"));
     RELAY_TRY(check_shape(dw, {d.K, d.N}, "dw"));
     if (db) RELAY_TRY(check_shape(db, {d.N}, "db"));
     if (act < RELAY_ACT_NONE || act > RELAY_ACT_SIGMOID) return fail(RELAY_ERR_ATTR, "unknown activation %d", act);

@@ -48,7 +48,7 @@ namespace {
 constexpr int A_BYTES = 128 * BK * 2;                      // this block's 128 rows of A: 16 KB
 constexpr int CHUNK_BYTES = 64 * BK * 2;                   // this block's 64 columns of one 128-column chunk: 8 KB
 constexpr int RING_BYTES = 192 * 1024;
-constexpr int NUM_THREADS = 576;                           // warp 0 producer, warp 1 MMA, warps 2-17 epilogue
+constexpr int NUM_THREADS = 608;                           // warp 0 A producer, warp 1 MMA, warps 2-17 epilogue, warp 18 B producer
 constexpr int EPI_WARPS = 16;
 constexpr int kWideMinKBlocks = 32;                        // classes 3 and 4 only for contractions at least this long
 constexpr int STAGING_BYTES = EPI_WARPS * 2048;        // one 32-row x 64-byte buffer per epilogue warp
@@ -236,8 +236,10 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     const uint32_t tmem_base = *tmem_slot;
     pdl_wait();   // set-up done; from here on the kernel touches global memory
 
-    if (warp == 0) {
-        // ---------------- TMA producer (both blocks) ----------------
+    if (warp == 0 || warp == 18) {
+        // ---------------- TMA producers (both blocks): warp 0 loads A and posts the byte count, warp 18 loads B ----------------
+        // (one thread issues only a few instructions per hundred cycles; two threads keep the ring fed)
+        const bool load_a = warp == 0;
         if (lane == 0) {
             int cur = 0, s = 0, n_st = 0, st_bytes = 0;
             uint32_t phase = 0;
@@ -267,20 +269,23 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                     if (!tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
                     uint8_t *sa = smem + (size_t)s * st_bytes, *sb = sa + A_BYTES;
                     const uint32_t bar = tc::mapa(tc::smem_u32(&full[s]), 0);       // the leader's barrier
-                    if (rank == 0) tc::mbar_expect_tx_cluster(bar, tx);
                     const int k0 = kb * BK;
-                    if (A_MN) {
+                    if (load_a) {
+                        if (rank == 0) tc::mbar_expect_tx_cluster(bar, tx);
+                        if (A_MN) {
 #pragma unroll
-                        for (int i = 0; i < 2; ++i) tc::tma_load_2d_pair(sa + i * MN_BOX_BYTES, &tm_a, bar, m0 + i * 64, k0);
+                            for (int i = 0; i < 2; ++i) tc::tma_load_2d_pair(sa + i * MN_BOX_BYTES, &tm_a, bar, m0 + i * 64, k0);
+                        } else {
+                            tc::tma_load_2d_pair(sa, &tm_a, bar, k0, m0);
+                        }
                     } else {
-                        tc::tma_load_2d_pair(sa, &tm_a, bar, k0, m0);
-                    }
-                    // B in boxes of 64 columns: MN-major boxes are 64 x 64 k anyway; K-major boxes of 64 rows stack
-                    // to the same shared-memory image as one taller box
-                    for (int i = 0; i < boxes; ++i) {
-                        const int n = i < boxes0 ? na + i * 64 : nb + (i - boxes0) * 64;
-                        if (B_MN) tc::tma_load_2d_pair(sb + i * MN_BOX_BYTES, &tm_b, bar, n, k0);
-                        else tc::tma_load_2d_pair(sb + i * MN_BOX_BYTES, &tm_b, bar, k0, n);
+                        // B in boxes of 64 columns: MN-major boxes are 64 x 64 k anyway; K-major boxes of 64 rows stack
+                        // to the same shared-memory image as one taller box
+                        for (int i = 0; i < boxes; ++i) {
+                            const int n = i < boxes0 ? na + i * 64 : nb + (i - boxes0) * 64;
+                            if (B_MN) tc::tma_load_2d_pair(sb + i * MN_BOX_BYTES, &tm_b, bar, n, k0);
+                            else tc::tma_load_2d_pair(sb + i * MN_BOX_BYTES, &tm_b, bar, k0, n);
+                        }
                     }
                     if (++s == n_st) { s = 0; phase ^= 1; }
                 }

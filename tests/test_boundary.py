@@ -60,13 +60,18 @@ def test_infer_dense_relation():
         for dt in (B.F32, B.BF16):
             out = B.relay_infer_dense(T(dt, (M, K)), T(dt, (K, N)))
             assert B._shape(out) == (M, N) and out.dtype == dt and out.rank == 2
+    # leading batch axes are carried through (batching adds a leading axis to every tensor, Section 5.2)
+    for lead in [(3,), (2, 5), (1, 1, 1, 4)]:
+        out = B.relay_infer_dense(T(B.BF16, lead + (7, 16)), T(B.BF16, (16, 24)))
+        assert B._shape(out) == lead + (7, 24) and out.rank == len(lead) + 2
 
 
 @pytest.mark.parametrize("x,w,status", [
     (T(B.F32, (8, 64)), T(B.F32, (63, 32)), "ERR_SHAPE"),
     (T(B.F32, (8, 64)), T(B.BF16, (64, 32)), "ERR_DTYPE"),
     (T(B.I32, (8, 64)), T(B.I32, (64, 32)), "ERR_DTYPE"),
-    (T(B.F32, (8, 64, 1)), T(B.F32, (64, 32)), "ERR_RANK"),
+    (T(B.F32, (8, 64, 1)), T(B.F32, (64, 32)), "ERR_SHAPE"),     # a batch of 8 with K = 1, not 64
+    (T(B.F32, (64,)), T(B.F32, (64, 32)), "ERR_RANK"),
     (T(B.F32, (8, 64)), T(B.F32, (64,)), "ERR_RANK"),
     (T(B.F32, (8, 64), B.NCHW), T(B.F32, (64, 32)), "ERR_LAYOUT"),
     (T(B.F32, (8, -1)), T(B.F32, (64, 32)), "ERR_SHAPE"),
@@ -93,6 +98,22 @@ def test_rule_order_rank_before_dtype_before_shape():
 
 
 # ---- conv2d -----------------------------------------------------------------------------------------
+def test_infer_conv2d_nhwc_tag_permutes_the_relation():
+    """An NHWC-tagged x has shape (N,H,W,C); the result is NHWC with the same extents as the NCHW relation gives."""
+    for H, W_, R, p, s in [(7, 6, 3, 1, 1), (9, 9, 3, 1, 2), (8, 5, 5, 0, 1), (56, 56, 3, 1, 1)]:
+        a = B.relay_infer_conv2d(T(B.BF16, (2, 3, H, W_), B.NCHW), T(B.BF16, (5, 3, R, R), B.OIHW), s, p)
+        b = B.relay_infer_conv2d(T(B.BF16, (2, H, W_, 3), B.NHWC), T(B.BF16, (5, 3, R, R), B.OIHW), s, p)
+        n, o, pp, q = B._shape(a)
+        assert B._shape(b) == (n, pp, q, o) and b.layout == B.NHWC and a.layout == B.NCHW
+    with pytest.raises(B.RelayError) as e:          # channels are the LAST axis of an NHWC tensor
+        B.relay_infer_conv2d(T(B.BF16, (2, 3, 7, 6), B.NHWC), T(B.BF16, (5, 3, 3, 3), B.OIHW), 1, 1)
+    assert e.value.status_name == "ERR_SHAPE"
+    with pytest.raises(B.RelayError) as e:
+        B.relay_infer_conv2d(T(B.BF16, (2, 3, 7, 6), B.ROWMAJOR), T(B.BF16, (5, 3, 3, 3), B.OIHW), 1, 1)
+    assert e.value.status_name == "ERR_LAYOUT"
+
+
+
 def test_infer_conv2d_matches_window_counting():
     for H, W_, R, p, s in itertools.product(range(1, 7), (1, 4, 6), (1, 2, 3, 5), (0, 1, 2), (1, 2, 3)):
         x, w = T(B.BF16, (2, 3, H, W_), B.NCHW), T(B.BF16, (5, 3, R, R), B.OIHW)

@@ -1,4 +1,6 @@
 """GPU parity: conv2d anchor (+bias +activation) with its gradient group, and the LSTM sequence."""
+import ctypes
+
 import numpy as np
 import pytest
 import torch
@@ -73,6 +75,47 @@ def test_conv_reduced_config_bf16_3x3(N, C, H, W, O):
     _, odw2, _ = oracle.conv2d_act_grad(xo, wo, to_np(y2), dyo, 1, 1, B.ACT_TANH, F64, F64, F64, want_dx=False, want_db=False,
                                         dz_dtype=oracle.BF16)
     assert_bf16(dw2, odw2, what="dw tanh")
+
+
+@pytest.mark.parametrize("N,C,H,W,O,R,stride,pad,tdt", [(2, 3, 7, 6, 4, 3, 1, 1, torch.float32), (1, 5, 9, 9, 3, 3, 2, 1, torch.bfloat16),
+                                                         (2, 128, 16, 16, 128, 3, 1, 1, torch.bfloat16),      # tensor-core instance
+                                                         (3, 128, 12, 24, 256, 3, 1, 1, torch.bfloat16)])
+def test_conv_nhwc_tagged_activations(N, C, H, W, O, R, stride, pad, tdt):
+    """Layout-tagged activations: x, y, dy, dx are NHWC tensors of shape (N,H,W,C); the values are those of the NCHW
+    definition (the oracle is given the same tensors permuted on the host)."""
+    t = I.cfg4_conv(N, C, H, W, O, R, R, dtype=tdt, salt=H + 1)
+    act = B.ACT_RELU
+    x_nhwc = t["x"].permute(0, 2, 3, 1).contiguous()
+    d = B.relay_infer_conv2d(B.desc(x_nhwc, B.NHWC), B.desc(t["w"], B.OIHW), stride, pad)
+    assert d.layout == B.NHWC and B._shape(d)[3] == O
+    y = Guarded(B._shape(d), tdt, DEV)
+    ws = workspace(B.relay_workspace_bytes_conv2d_act(x_nhwc, t["w"], stride, pad, layout=B.NHWC), DEV)
+    B.relay_fused_conv2d_act(x_nhwc.to(DEV), t["w"].to(DEV), t["b"].to(DEV), stride, pad, act, y.t, ws, layout=B.NHWC)
+    torch.cuda.synchronize()
+    yg = y.check()
+    xo, wo, bo = (I.as_f64(t[k]) for k in ("x", "w", "b"))
+    want = oracle.conv2d_act(xo, wo, bo, stride, pad, act, F64)                     # NCHW
+    chk = assert_f32 if tdt == torch.float32 else assert_bf16
+    chk(yg.permute(0, 3, 1, 2), want, what="y")
+    dy = I.normal(4, 3, tuple(want.shape), 1.0, tdt, salt=H + 1)                      # NCHW values
+    dy_nhwc = dy.permute(0, 2, 3, 1).contiguous()
+    dx, dw, db = Guarded(tuple(x_nhwc.shape), tdt, DEV), Guarded(tuple(t["w"].shape), tdt, DEV), Guarded((O,), torch.float32, DEV)
+    ws = workspace(B.relay_workspace_bytes_conv2d_act_grad(x_nhwc, t["w"], stride, pad, layout=B.NHWC), DEV)
+    B.relay_fused_conv2d_act_grad(x_nhwc.to(DEV), t["w"].to(DEV), yg.to(DEV), dy_nhwc.to(DEV), stride, pad, act, dx.t, dw.t, db.t, ws,
+                                  layout=B.NHWC)
+    torch.cuda.synchronize()
+    odx, odw, odb = oracle.conv2d_act_grad(xo, wo, to_np(yg.permute(0, 3, 1, 2)), I.as_f64(dy), stride, pad, act, F64, F64, F64,
+                                           dz_dtype=oracle.F32 if tdt == torch.float32 else oracle.BF16)
+    chk(dx.check().permute(0, 3, 1, 2), odx, what="dx"); chk(dw.check(), odw, what="dw")
+    (assert_f32 if tdt == torch.float32 else (lambda g, o, what: assert_bf16(g, o, stored_bf16=False, what=what)))(db.check(), odb, what="db")
+    # an NCHW-tagged y for an NHWC x is a layout error; nothing is written
+    bad = torch.full(B._shape(d), 5.0, dtype=tdt, device=DEV)
+    at = B.Conv2dAttrs(stride, pad, 1, 1)
+    xd, wd, yd = B.desc(x_nhwc.to(DEV), B.NHWC), B.desc(t["w"].to(DEV), B.OIHW), B.desc(bad, B.NCHW)
+    with pytest.raises(B.RelayError) as e:
+        B._check(B.lib().relay_fused_conv2d_act(ctypes.byref(xd), ctypes.byref(wd), None, ctypes.byref(at), int(act), ctypes.byref(yd),
+                                                 None, 0, None))
+    assert e.value.status_name == "ERR_LAYOUT" and bool((bad == 5.0).all())
 
 
 def test_conv_rejections():

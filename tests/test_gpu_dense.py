@@ -89,6 +89,48 @@ def test_optional_outputs_no_bias_and_f32_bias():
     assert_bf16(dw, odw)
 
 
+@pytest.mark.parametrize("lead,M,K,N,tdt", [((3,), 8, 64, 32, torch.float32), ((2, 5), 24, 72, 40, torch.bfloat16),
+                                            ((4,), 128, 256, 512, torch.bfloat16), ((0,), 8, 16, 8, torch.float32)])
+def test_leading_batch_axes(lead, M, K, N, tdt):
+    """Batching adds a leading axis to every tensor of the program (Section 5.2): the oracle runs the dense anchor
+    and its gradient group once per batch element; the partials of the shared w and b add up over the batch."""
+    nb = int(np.prod(lead))
+    t = I.cfg1_tiny_mlp(max(nb * M, 1), K, N, salt=77)
+    w, b = (t["w"] / np.sqrt(K)).to(tdt), t["b"].to(tdt)
+    x = t["x"][:nb * M].to(tdt).reshape(lead + (M, K)); dy = t["dy"][:nb * M].to(tdt).reshape(lead + (M, N))
+    y = Guarded(lead + (M, N), tdt, DEV)
+    B.relay_fused_dense_act(x.to(DEV), w.to(DEV), b.to(DEV), B.ACT_TANH, y.t, None)
+    dx, dw, db = Guarded(lead + (M, K), tdt, DEV), Guarded((K, N), tdt, DEV), Guarded((N,), torch.float32, DEV)
+    ws = workspace(B.relay_workspace_bytes_dense_act_grad(x, w), DEV)
+    B.relay_fused_dense_act_grad(x.to(DEV), w.to(DEV), y.t, dy.to(DEV), B.ACT_TANH, dx.t, dw.t, db.t, ws)
+    torch.cuda.synchronize()
+    yg, dxg, dwg, dbg = y.check(), dx.check(), dw.check(), db.check()
+    wo, bo = w.double().numpy(), b.double().numpy()
+    xe, dye, yge = x.reshape(nb, M, K), dy.reshape(nb, M, N), yg.reshape(nb, M, N)
+    want_y, want_dx = np.zeros((nb, M, N)), np.zeros((nb, M, K))
+    want_dw, want_db = np.zeros((K, N)), np.zeros(N)
+    dzt = oracle.F32 if tdt == torch.float32 else oracle.BF16
+    for e in range(nb):
+        xo = xe[e].double().numpy()
+        want_y[e] = oracle.dense_act(xo, wo, bo, B.ACT_TANH, F64)
+        odx, odw, odb = oracle.dense_act_grad(xo, wo, to_np(yge[e]), dye[e].double().numpy(), B.ACT_TANH, F64, F64, F64, dz_dtype=dzt)
+        want_dx[e] = odx; want_dw += odw; want_db += odb
+    chk = assert_f32 if tdt == torch.float32 else assert_bf16
+    if nb:
+        chk(yg.reshape(nb, M, N), want_y, what="y"); chk(dxg.reshape(nb, M, K), want_dx, what="dx")
+    chk(dwg, want_dw, what="dw")
+    if tdt == torch.float32:
+        assert_f32(dbg, want_db, what="db")
+    else:
+        assert_bf16(dbg, want_db, stored_bf16=False, what="db")
+    # a batch axis on y that x does not have is a type error; nothing is written
+    bad = torch.full((M, N), 5.0, dtype=tdt, device=DEV)
+    if nb:
+        with pytest.raises(B.RelayError) as e:
+            B.relay_fused_dense_act(x.to(DEV), w.to(DEV), b.to(DEV), B.ACT_TANH, bad, None)
+        assert e.value.status_name == "ERR_RANK" and bool((bad == 5.0).all())
+
+
 def test_three_layer_mlp_chain_reduced_size_group_by_group():
     """Configuration 3's structure at width 256 / batch 192: every group is checked against the
     oracle fed with the GPU's stored inputs of that group (so relu masks are identical)."""
