@@ -387,6 +387,13 @@ relay_status_t relay_poll_status(void *stream);
  * It shows a caller that an expired wait in any kernel of this library is reported rather than hung on. */
 relay_status_t relay_debug_expire_wait(int32_t limit_us, void *stream);
 
+/* Host-only view of how the two-SM contraction kernel cuts an M x N output (contraction length K) into work units
+ * for `sms` SMs (no counterpart in the paper; touches no GPU): fills units[i] = row block (256 rows) |
+ * first 128-column chunk << 12 | width in chunks << 24, in the order the kernel hands them to its SM pairs
+ * (pair p takes units p, p + sms/2, ...).  Returns the number of units, -1 if the shape is too large for a list
+ * (the kernel then follows its fixed scheme), -2 for bad arguments or max_units too small.  For tests of the plan. */
+int32_t relay_debug_plan_units(int64_t M, int64_t N, int64_t K, int32_t sms, uint32_t *units, int32_t max_units);
+
 /* Number of kernels this library has launched on this process so far (monotonic counter). */
 int64_t relay_launch_count(void);
 

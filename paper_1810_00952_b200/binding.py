@@ -362,6 +362,18 @@ def relay_debug_expire_wait(limit_us: int = 1000):
     _check(lib().relay_debug_expire_wait(int(limit_us), _stream()))
 
 
+def relay_debug_plan_units(M: int, N: int, K: int, sms: int, max_units: int = 1024):
+    """Unit plan of the two-SM contraction kernel as (row block, first chunk, width in chunks) triples, or None
+    when the kernel would follow its fixed scheme."""
+    buf = (ctypes.c_uint32 * max_units)()
+    n = int(lib().relay_debug_plan_units(ctypes.c_int64(M), ctypes.c_int64(N), ctypes.c_int64(K), int(sms), buf, max_units))
+    if n == -1:
+        return None
+    if n < 0:
+        raise ValueError("relay_debug_plan_units: bad arguments")
+    return [(int(e) & 0xFFF, (int(e) >> 12) & 0xFFF, int(e) >> 24) for e in buf[:n]]
+
+
 def relay_launch_count() -> int:
     return int(lib().relay_launch_count())
 

@@ -492,3 +492,18 @@ relay_status_t launch_gemm_tc2(const GemmDesc &g, int sms, cudaStream_t st)
 }
 
 }  // namespace relay
+
+// Host-only view of the unit plan (no GPU is touched), so that its invariants can be tested for many shapes.
+extern "C" int32_t relay_debug_plan_units(int64_t M, int64_t N, int64_t K, int32_t sms, uint32_t *units, int32_t max_units)
+{
+    using namespace relay;
+    if (M < 1 || N < 1 || K < 1 || sms < 2 || !units || max_units < 0) return -2;
+    const int tiles_m = (int)((M + 255) / 256), tiles_n = (int)((N + BN - 1) / BN), k_blocks = (int)((K + BK - 1) / BK);
+    const int pairs = std::min(tiles_m * tiles_n, sms / 2);
+    static thread_local UnitTable tb;
+    tb.n = 0;
+    if (!plan_units(tiles_m, (int)((N + 127) / 128), pairs, k_blocks, &tb)) return -1;   // the fixed scheme would run
+    if (tb.n > max_units) return -2;
+    std::copy(tb.e, tb.e + tb.n, units);
+    return tb.n;
+}
