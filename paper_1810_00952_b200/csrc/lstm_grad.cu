@@ -33,25 +33,37 @@ __device__ __forceinline__ float sigm(float x) { return __fdividef(1.0f, 1.0f + 
 __device__ __forceinline__ float tanh_fast(float x) { return 1.0f - __fdividef(2.0f, 1.0f + __expf(2.0f * x)); }
 
 // a[t*B+b][0..I) = x[t,b,:],  a[t*B+b][I..I+H) = bf16(h_{t-1}[b,:])   (h_{-1} = h0)
+// VEC = 8: one thread moves 8 consecutive elements (I and H multiples of 8); VEC = 1: any shape
+template <int VEC>
 __global__ void __launch_bounds__(256) lstm_cat_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restrict__ h0,
                                                         const float *__restrict__ h_all, __nv_bfloat16 *__restrict__ a, int64_t T,
                                                         int64_t B, int64_t I, int64_t H)
 {
-    const int64_t W = I + H, total = T * B * W;
+    const int64_t W = I + H, total = T * B * W / VEC;
     pdl_wait();
-    for (int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x; e < total; e += (int64_t)gridDim.x * 256) {
+    for (int64_t v = (int64_t)blockIdx.x * 256 + threadIdx.x; v < total; v += (int64_t)gridDim.x * 256) {
+        const int64_t e = v * VEC;
         const int64_t row = e / W, col = e % W;
         if (col < I) {
-            a[e] = x[row * I + col];
+            if (VEC == 8) *reinterpret_cast<uint4 *>(a + e) = ld_stream(x + row * I + col);
+            else a[e] = x[row * I + col];
         } else {
             const int64_t t = row / B, b = row % B;
-            const float hv = t == 0 ? h0[b * H + (col - I)] : h_all[((t - 1) * B + b) * H + (col - I)];
-            a[e] = __float2bfloat16_rn(hv);
+            const float *src = (t == 0 ? h0 + b * H : h_all + ((t - 1) * B + b) * H) + (col - I);
+            if (VEC == 8) {
+                float f[8];
+                const float4 lo = *reinterpret_cast<const float4 *>(src), hi = *reinterpret_cast<const float4 *>(src + 4);
+                f[0] = lo.x; f[1] = lo.y; f[2] = lo.z; f[3] = lo.w; f[4] = hi.x; f[5] = hi.y; f[6] = hi.z; f[7] = hi.w;
+                *reinterpret_cast<uint4 *>(a + e) = pack(f);
+            } else {
+                a[e] = __float2bfloat16_rn(*src);
+            }
         }
     }
 }
 
-// one thread per (batch row, hidden unit): over time, z -> activated gates in place, c_all[t] = c_t
+// one thread per (batch row, hidden unit): over time, z -> activated gates in place, c_all[t] = c_t.
+// Only c carries from step to step: the loads of four steps are issued together so that their latency is paid once.
 __global__ void __launch_bounds__(256) lstm_cell_sweep_kernel(float *__restrict__ z, const float *__restrict__ c0,
                                                                float *__restrict__ c_all, int64_t T, int64_t B, int64_t H)
 {
@@ -60,12 +72,26 @@ __global__ void __launch_bounds__(256) lstm_cell_sweep_kernel(float *__restrict_
     if (idx >= B * H) return;
     const int64_t b = idx / H, u = idx % H;
     float c = c0[idx];
-    for (int64_t t = 0; t < T; ++t) {
-        float *zr = z + (t * B + b) * 4 * H + u;
-        const float ig = sigm(zr[0]), fg = sigm(zr[H]), gg = tanh_fast(zr[2 * H]), og = sigm(zr[3 * H]);
-        c = fmaf(fg, c, ig * gg);
-        zr[0] = ig; zr[H] = fg; zr[2 * H] = gg; zr[3 * H] = og;
-        c_all[(t * B + b) * H + u] = c;
+    constexpr int U = 4;
+    for (int64_t t0 = 0; t0 < T; t0 += U) {
+        float zi[U], zf[U], zg[U], zo[U];
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            if (t0 + k < T) {
+                const float *zr = z + ((t0 + k) * B + b) * 4 * H + u;
+                zi[k] = zr[0]; zf[k] = zr[H]; zg[k] = zr[2 * H]; zo[k] = zr[3 * H];
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            if (t0 + k < T) {
+                float *zr = z + ((t0 + k) * B + b) * 4 * H + u;
+                const float ig = sigm(zi[k]), fg = sigm(zf[k]), gg = tanh_fast(zg[k]), og = sigm(zo[k]);
+                c = fmaf(fg, c, ig * gg);
+                zr[0] = ig; zr[H] = fg; zr[2 * H] = gg; zr[3 * H] = og;
+                c_all[((t0 + k) * B + b) * H + u] = c;
+            }
+        }
     }
 }
 
@@ -532,9 +558,12 @@ extern "C" relay_status_t relay_lstm_cell_seq_grad(const relay_tensor_t *x, cons
 
     // (1) recompute the forward values the reverse sweep reads
     {
-        const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>((rows * W + 255) / 256, 148 * 32));
-        RELAY_CUDA(launch_pdl(lstm_cat_kernel, dim3(grid), dim3(256), 0, st, (const __nv_bfloat16 *)x->data, (const float *)h0->data,
-                              (const float *)h_all->data, a_cat, d.T, d.B, d.I, d.H));
+        const bool vec = d.I % 8 == 0 && d.H % 8 == 0;
+        const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>((rows * W / (vec ? 8 : 1) + 255) / 256, 148 * 32));
+        if (vec) RELAY_CUDA(launch_pdl(lstm_cat_kernel<8>, dim3(grid), dim3(256), 0, st, (const __nv_bfloat16 *)x->data, (const float *)h0->data,
+                                       (const float *)h_all->data, a_cat, d.T, d.B, d.I, d.H));
+        else RELAY_CUDA(launch_pdl(lstm_cat_kernel<1>, dim3(grid), dim3(256), 0, st, (const __nv_bfloat16 *)x->data, (const float *)h0->data,
+                                   (const float *)h_all->data, a_cat, d.T, d.B, d.I, d.H));
         RELAY_TRY(check_launch("lstm_cat"));
         RELAY_CUDA(cudaMemcpyAsync(w_cat, w_ih->data, (size_t)d.I * G * 2, cudaMemcpyDeviceToDevice, st));
         RELAY_CUDA(cudaMemcpyAsync(w_cat + (size_t)d.I * G, w_hh->data, (size_t)d.H * G * 2, cudaMemcpyDeviceToDevice, st));
