@@ -171,6 +171,7 @@ constexpr int TMEM_COLS = N_ISS * UNITS;
 struct GradParams {
     int T, B, H, n_blocks, k_blocks;
     int rows_per_group, n_epi;
+    int rows_per_warp;               // 32 (M = 128 MMAs), or 16 with M = 64 MMAs for groups of at most 64 rows (half the A rows read)
     int tile_stride, n_stages;       // bytes between the k-block tiles of the ring (a stage is N_ISS tiles); stages in the ring
     const float *gates;              // [T*B][4H] activated gates i | f | g | o
     const float *c_all, *c0;         // [T*B][H], [B][H]
@@ -240,8 +241,10 @@ lstm_grad_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __gr
     if (warp < 4) {
       if (warp < p.n_epi) {
         // ------------------------------ epilogue: one batch row per lane, 16 units ------------------------------
-        const int b = b_lo + warp * 32 + lane;
-        const bool live = warp * 32 + lane < nb;
+        // M = 128: accumulator row r sits in TMEM lane r.  M = 64: rows 16w .. 16w+15 sit in lanes 32w .. 32w+15, so warp w
+        // owns 16 rows in its first 16 lanes.
+        const int b = b_lo + warp * p.rows_per_warp + lane;
+        const bool live = lane < p.rows_per_warp && warp * p.rows_per_warp + lane < nb;
         float dc[UNITS], c_cur[UNITS];
 #pragma unroll
         for (int i = 0; i < UNITS; ++i) { dc[i] = 0.0f; c_cur[i] = 0.0f; }
@@ -357,7 +360,7 @@ lstm_grad_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __gr
                 for (int kb = 0; kb < p.k_blocks; ++kb) tc::tma_load_2d(w_s + (size_t)kb * W_KB, &tm_w, w_full, kb * BK, j0);
             }
             bool ok = tc::mbar_wait(w_full, 0, abort_flag, p.err, tc::ERR_WAIT_FULL);
-            const uint32_t idesc = tc::instr_desc_bf16(128, UNITS, false, false);
+            const uint32_t idesc = tc::instr_desc_bf16(p.rows_per_warp == 16 ? 64 : 128, UNITS, false, false);
             // descriptors differ from the first one only in the start-address field (16-byte units): one add per MMA
             const uint64_t desc_a0 = tc::smem_desc(tc::smem_u32(a_s) + (uint32_t)(iss * p.tile_stride), 16, 1024);
             const uint64_t desc_b0 = tc::smem_desc(tc::smem_u32(w_s) + (uint32_t)(iss * W_KB), 16, 1024);
@@ -442,7 +445,9 @@ relay_status_t run_steps_tc(const GradDims &d, const GradPlan &pl, char *ws, con
                                 (uint32_t)rows_per_group));
     GradParams p{};
     p.T = (int)d.T; p.B = (int)d.B; p.H = (int)d.H; p.n_blocks = n_blocks; p.k_blocks = (int)(4 * d.H / BK);
-    p.rows_per_group = rows_per_group; p.n_epi = (rows_per_group + 31) / 32;
+    p.rows_per_group = rows_per_group;
+    p.rows_per_warp = rows_per_group <= 64 ? 16 : 32;
+    p.n_epi = (rows_per_group + p.rows_per_warp - 1) / p.rows_per_warp;
     p.gates = (const float *)(ws + pl.gates); p.c_all = (const float *)(ws + pl.c_all); p.c0 = c0;
     p.dh_all = dh_all; p.dc_final = dc_final; p.dz = (__nv_bfloat16 *)(ws + pl.dz); p.dh0 = dh0; p.dc0 = dc0;
     p.counter = counter;

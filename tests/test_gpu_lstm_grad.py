@@ -62,7 +62,7 @@ def compare(got, want, keys=("dx", "dw_ih", "dw_hh", "db", "dh0", "dc0")):
 
 # persistent tensor-core route (H a multiple of 64), one or several batch groups; per-step route otherwise
 @pytest.mark.parametrize("T,Bn,In,H", [(1, 8, 64, 64), (3, 8, 64, 64), (5, 40, 96, 128), (4, 16, 32, 20), (6, 3, 24, 72), (3, 16, 64, 1024),
-                                       (2, 130, 64, 64)])
+                                       (2, 130, 64, 64), (2, 96, 64, 1024)])     # the last: 48 rows a group, all four lane quarters of M = 64
 def test_gradient_program(T, Bn, In, H):
     t, dh_all, dc_fin = case(T, Bn, In, H, salt=T * 100 + H)
     d = {k: v.to(DEV) for k, v in t.items()}
