@@ -162,7 +162,7 @@ constexpr int W_KB = UNITS * BK * 2;             // one k-block of the resident 
 // As in the forward kernel, ring stages are only as far apart as the rows a group really has: the MMA's rows
 // beyond the group's are whatever follows in shared memory, and the accumulator rows they produce are never read.
 constexpr int N_ISS = 4;                         // MMA-issuing threads (one lane each of warps 4, 6, 7, 8), one accumulator each
-constexpr int NUM_THREADS = 288;                 // warps 0-3 epilogue, warp 4 W loader + issuer 0, warp 5 dz loader, warps 6-8 issuers 1-3
+constexpr int NUM_THREADS = 320;                 // warps 0-3 epilogue, warp 4 W loader + issuer 0, warps 5 and 9 dz loaders, warps 6-8 issuers 1-3
 constexpr int TMEM_COLS = N_ISS * UNITS;
 // One thread issues a tcgen05.mma of N = 16 only every hundred cycles or so (descriptor arithmetic, barrier polling),
 // far slower than the tensor pipe runs it.  So a ring stage holds N_ISS k-blocks (one barrier round per stage), each
@@ -173,6 +173,7 @@ struct GradParams {
     int rows_per_group, n_epi;
     int rows_per_warp;               // 32 (M = 128 MMAs), or 16 with M = 64 MMAs for groups of at most 64 rows (half the A rows read)
     int tile_stride, n_stages;       // bytes between the k-block tiles of the ring (a stage is N_ISS tiles); stages in the ring
+    int n_load;                      // loader threads (1 or 2): they take the stages of a step in turn
     const float *gates;              // [T*B][4H] activated gates i | f | g | o
     const float *c_all, *c0;         // [T*B][H], [B][H]
     const float *dh_all;             // [T*B][H]
@@ -307,9 +308,9 @@ lstm_grad_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __gr
                     o[1] = make_uint4(pack2(dzv[g][8], dzv[g][9]), pack2(dzv[g][10], dzv[g][11]), pack2(dzv[g][12], dzv[g][13]), pack2(dzv[g][14], dzv[g][15]));
                 }
             }
-            // dZ[t] is read by TMA (async proxy) in the other blocks: fence the generic stores for it, then release
+            // dZ[t] is read by TMA (async proxy) in the other blocks: fence the generic stores for it; the warp barrier orders
+            // the warp's stores before lane 0's release, which is cumulative
             asm volatile("fence.proxy.async.global;" ::: "memory");
-            __threadfence();
             __syncwarp();
             if (lane == 0) red_release_add(counter, 1u);
         }
@@ -319,10 +320,12 @@ lstm_grad_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __gr
             for (int i = 0; i < UNITS; i += 4) o[i / 4] = make_float4(dc[i], dc[i + 1], dc[i + 2], dc[i + 3]);
         }
       }
-    } else if (warp == 5) {
-        // ------------------------------ dz loader: dZ[T-s] rows of the group -> ring, by TMA ------------------------------
-        if (lane == 0) {
-            int st = 0;
+    } else if (warp == 5 || warp == 9) {
+        // ------------------------------ dz loaders: dZ[T-s] rows of the group -> ring, by TMA ------------------------------
+        // (one thread needs several hundred cycles per stage; two threads take the stages of a step in turn)
+        const int ld = warp == 5 ? 0 : 1;
+        if (lane == 0 && ld < p.n_load) {
+            int st = ld;
             uint32_t phase = 0;
             bool ok = true;
             const uint32_t stage_bytes = (uint32_t)(N_ISS * p.rows_per_group * 128);
@@ -341,13 +344,14 @@ lstm_grad_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __gr
                 if (!ok) break;
                 asm volatile("fence.proxy.async.global;" ::: "memory");
                 const int row0 = (p.T - s) * p.B + b_lo;
-                for (int kb = 0; kb < p.k_blocks; kb += N_ISS) {
+                for (int kb = ld * N_ISS; kb < p.k_blocks; kb += p.n_load * N_ISS) {
                     if (!tc::mbar_wait(&empty[st], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
                     tc::mbar_expect_tx(&full[st], stage_bytes);
                     uint8_t *dst = a_s + (size_t)st * N_ISS * p.tile_stride;
 #pragma unroll
                     for (int i = 0; i < N_ISS; ++i) tc::tma_load_2d(dst + (size_t)i * p.tile_stride, &tm_dz, &full[st], (kb + i) * BK, row0);
-                    if (++st == p.n_stages) { st = 0; phase ^= 1; }
+                    st += p.n_load;
+                    if (st >= p.n_stages) { st -= p.n_stages; phase ^= 1; }
                 }
             }
         }
@@ -455,6 +459,8 @@ relay_status_t run_steps_tc(const GradDims &d, const GradPlan &pl, char *ws, con
     if (!p.err) return fail(RELAY_ERR_CUDA, "no device error word");
     p.tile_stride = (int)align_up((size_t)rows_per_group * 128, 1024);
     p.n_stages = std::min(MAX_STAGES, RING_BYTES / (N_ISS * p.tile_stride));
+    // two loaders when the stages of a step split evenly between them (each then walks the ring in steps of two)
+    p.n_load = ((p.k_blocks / N_ISS) % 2 == 0 && p.n_stages % 2 == 0) ? 2 : 1;
     // what follows the ring is at least one A tile long, so the rows an MMA reads past the last stage stay inside the allocation
     const size_t smem = 1024 + (size_t)RING_BYTES + std::max<size_t>((size_t)p.k_blocks * W_KB, A_TILE) + 1024;
     RELAY_CUDA(cudaFuncSetAttribute(lstm_grad_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));

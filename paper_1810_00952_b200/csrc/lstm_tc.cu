@@ -37,7 +37,7 @@ constexpr int W_KB = NCOL * BK * 2;              // one k-block of the resident 
 // memory (later stages, then the W slice).  Row r of the product depends on row r of A alone, and the epilogue
 // reads only the group's rows, so those accumulator rows are never looked at; the ring holds four times as many
 // bytes in flight as it would with zero-padded 128-row stages.
-constexpr int NUM_THREADS = 224;                 // warps 0-3 epilogue, warp 4 W loader + MMA issuer 0, warp 5 h loader, warp 6 issuer 1
+constexpr int NUM_THREADS = 256;                 // warps 0-3 epilogue, warp 4 W loader + MMA issuer 0, warps 5 and 7 h loaders, warp 6 issuer 1
 constexpr int MAX_ISS = 2;
 // One thread issues a tcgen05.mma only every hundred cycles or so (descriptor arithmetic, barrier polling), slower
 // than the tensor pipe runs an N = 64 one.  With an even number of k-blocks a ring stage therefore holds two of
@@ -49,6 +49,7 @@ struct Params {
     int rows_per_group, n_epi;       // batch rows per block group; epilogue warps that own rows (ceil(rows_per_group / 32))
     int tile_stride, n_stages;       // bytes between the k-block tiles of the ring (a stage is n_iss tiles); stages in the ring
     int n_iss;                       // MMA issuers = k-blocks per stage = accumulators (1 or 2)
+    int n_load;                      // loader threads (1 or 2): they take the stages of a step in turn
     const float *zx;                 // [T*B][4H] input projection + bias
     const float *h0, *c0;            // [B][H]
     float *h_all, *c_final;          // [T][B][H], [B][H]
@@ -187,8 +188,8 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
                 hq[0] = make_uint4(pack2(hn[0], hn[1]), pack2(hn[2], hn[3]), pack2(hn[4], hn[5]), pack2(hn[6], hn[7]));
                 hq[1] = make_uint4(pack2(hn[8], hn[9]), pack2(hn[10], hn[11]), pack2(hn[12], hn[13]), pack2(hn[14], hn[15]));
             }
+            // the warp's stores are ordered before lane 0's release by the warp barrier; the release is cumulative
             asm volatile("fence.proxy.async.global;" ::: "memory");
-            __threadfence();
             __syncwarp();
             if (lane == 0) red_release_add(counter, 1u);
             if (live) {   // the fp32 copy for the caller is off the critical path
@@ -202,10 +203,12 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
             for (int i = 0; i < UNITS; ++i) p.c_final[(size_t)b * p.H + j0 + i] = c[i];
         }
       }
-    } else if (warp == 5) {
-        // ------------------------------ h loader: bf16(h_{t-1}) -> ring, by TMA ------------------------------
-        if (lane == 0) {
-            int s = 0;
+    } else if (warp == 5 || warp == 7) {
+        // ------------------------------ h loaders: bf16(h_{t-1}) -> ring, by TMA ------------------------------
+        // (one thread needs several hundred cycles per stage; two threads take the stages of a step in turn)
+        const int ld = warp == 5 ? 0 : 1;
+        if (lane == 0 && ld < p.n_load) {
+            int s = ld;
             uint32_t phase = 0;
             bool ok = true;
             const uint32_t stage_bytes = (uint32_t)(p.n_iss * p.rows_per_group * 128);
@@ -224,13 +227,14 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
                 if (!ok) break;
                 asm volatile("fence.proxy.async.global;" ::: "memory");
                 const CUtensorMap *tm_h = (t & 1) ? &tm_h1 : &tm_h0;
-                for (int kb = 0; kb < p.k_blocks; kb += p.n_iss) {
+                for (int kb = ld * p.n_iss; kb < p.k_blocks; kb += p.n_load * p.n_iss) {
                     if (!tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
                     tc::mbar_expect_tx(&full[s], stage_bytes);
                     uint8_t *dst = a_s + (size_t)s * p.n_iss * p.tile_stride;
                     for (int i = 0; i < p.n_iss; ++i)
                         tc::tma_load_2d(dst + (size_t)i * p.tile_stride, tm_h, &full[s], (kb + i) * BK, b_lo);   // the group's rows only
-                    if (++s == p.n_stages) { s = 0; phase ^= 1; }
+                    s += p.n_load;
+                    if (s >= p.n_stages) { s -= p.n_stages; phase ^= 1; }
                 }
             }
         }
@@ -338,6 +342,8 @@ relay_status_t launch_lstm_tc(int64_t T, int64_t B, int64_t H, const float *zx, 
     p.n_iss = p.k_blocks % 2 == 0 ? 2 : 1;
     p.tile_stride = (int)align_up((size_t)rows_per_group * 128, 1024);
     p.n_stages = std::min(MAX_STAGES, RING_BYTES / (p.n_iss * p.tile_stride));
+    // two loaders when the stages of a step split evenly between them (each then walks the ring in steps of two)
+    p.n_load = ((p.k_blocks / p.n_iss) % 2 == 0 && p.n_stages % 2 == 0) ? 2 : 1;
     // what follows the ring is at least one A tile long, so the rows an MMA reads past the last stage stay inside the allocation
     const size_t smem = 1024 + (size_t)RING_BYTES + std::max<size_t>((size_t)p.k_blocks * W_KB, A_TILE) + 1024;
     RELAY_CUDA(cudaFuncSetAttribute(lstm_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
