@@ -215,7 +215,7 @@ lstm_grad_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __gr
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * MAX_STAGES + 2);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // provably warp-uniform
     const int blk = blockIdx.x % p.n_blocks, grp = blockIdx.x / p.n_blocks;
     const int j0 = blk * UNITS;
     const int b_lo = grp * p.rows_per_group;
@@ -357,13 +357,15 @@ lstm_grad_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __gr
         }
     } else {
         // ------------------------------ MMA issuers (warp 4 also loads the W slice) ------------------------------
-        if (lane == 0) {
+        // The whole warp runs the loop with warp-uniform values and one elected lane issues (mma_bf16_elect).
+        {
             const int iss = warp == 4 ? 0 : warp - 5;                 // warps 4, 6, 7, 8 -> issuers 0..3
-            if (iss == 0) {
+            if (iss == 0 && lane == 0) {
                 tc::mbar_expect_tx(w_full, (uint32_t)(p.k_blocks * W_KB));
                 for (int kb = 0; kb < p.k_blocks; ++kb) tc::tma_load_2d(w_s + (size_t)kb * W_KB, &tm_w, w_full, kb * BK, j0);
             }
-            bool ok = tc::mbar_wait(w_full, 0, abort_flag, p.err, tc::ERR_WAIT_FULL);
+            __syncwarp();
+            bool ok = __all_sync(0xffffffffu, tc::mbar_wait(w_full, 0, abort_flag, p.err, tc::ERR_WAIT_FULL));
             const uint32_t idesc = tc::instr_desc_bf16(p.rows_per_warp == 16 ? 64 : 128, UNITS, false, false);
             // descriptors differ from the first one only in the start-address field (16-byte units): one add per MMA
             const uint64_t desc_a0 = tc::smem_desc(tc::smem_u32(a_s) + (uint32_t)(iss * p.tile_stride), 16, 1024);
@@ -375,17 +377,19 @@ lstm_grad_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __gr
             for (int s = 1; s <= p.T && ok; ++s) {
                 uint32_t b_off = 0;
                 for (int kb = 0; kb < p.k_blocks; kb += N_ISS) {       // this issuer's k-block of the stage: kb + iss
-                    if (!tc::mbar_wait(&full[st], phase, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
+                    // every lane waits; the vote reconverges the warp (the lanes leave the wait at different times)
+                    ok = __all_sync(0xffffffffu, tc::mbar_wait(&full[st], phase, abort_flag, p.err, tc::ERR_WAIT_FULL));
+                    if (!ok) break;
                     tc::tc_fence_after_sync();
                     const uint64_t da = desc_a0 + a_off, db = desc_b0 + b_off;
                     const uint32_t acc = kb != 0;
 #pragma unroll
-                    for (int kk = 0; kk < BK / 16; ++kk) tc::mma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, acc | (kk != 0));
-                    tc::mma_commit(&empty[st]);
+                    for (int kk = 0; kk < BK / 16; ++kk) tc::mma_bf16_elect(d_tmem, da + 2 * kk, db + 2 * kk, idesc, acc | (kk != 0));
+                    tc::mma_commit_elect(&empty[st]);
                     a_off += a_stage; b_off += b_stage;
                     if (++st == p.n_stages) { st = 0; phase ^= 1; a_off = 0; }
                 }
-                if (ok) tc::mma_commit(tmem_full);
+                if (ok) tc::mma_commit_elect(tmem_full);
             }
         }
     }
