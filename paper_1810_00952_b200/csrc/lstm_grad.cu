@@ -324,32 +324,39 @@ lstm_grad_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __gr
         // ------------------------------ dz loaders: dZ[T-s] rows of the group -> ring, by TMA ------------------------------
         // (one thread needs several hundred cycles per stage; two threads take the stages of a step in turn)
         const int ld = warp == 5 ? 0 : 1;
-        if (lane == 0 && ld < p.n_load) {
+        if (ld < p.n_load) {                                           // warp-uniform loop, an elected lane issues
             int st = ld;
             uint32_t phase = 0;
             bool ok = true;
             const uint32_t stage_bytes = (uint32_t)(N_ISS * p.rows_per_group * 128);
             for (int s = 1; s <= p.T && ok; ++s) {
-                // grid barrier: every block of the group has written its columns of dZ[T-s]
+                // grid barrier: every block of the group has written its columns of dZ[T-s] (lane 0 polls, the warp follows)
                 const unsigned int target = (unsigned int)(p.n_epi * p.n_blocks) * (unsigned int)s;
-                const long long t0 = clock64();
-                unsigned spins = 0;
-                while (ld_acquire(counter) < target) {
-                    if ((++spins & 255u) == 0 && (*abort_flag || clock64() - t0 > tc::kWaitLimitCycles)) {
-                        if (!*abort_flag) { *abort_flag = 1; atomicCAS(p.err, 0, tc::ERR_WAIT_STEP); }
-                        ok = false;
-                        break;
+                if (lane == 0) {
+                    const long long t0 = clock64();
+                    unsigned spins = 0;
+                    while (ld_acquire(counter) < target) {
+                        if ((++spins & 255u) == 0 && (*abort_flag || clock64() - t0 > tc::kWaitLimitCycles)) {
+                            if (!*abort_flag) { *abort_flag = 1; atomicCAS(p.err, 0, tc::ERR_WAIT_STEP); }
+                            ok = false;
+                            break;
+                        }
                     }
+                    asm volatile("fence.proxy.async.global;" ::: "memory");
                 }
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
-                asm volatile("fence.proxy.async.global;" ::: "memory");
                 const int row0 = (p.T - s) * p.B + b_lo;
                 for (int kb = ld * N_ISS; kb < p.k_blocks; kb += p.n_load * N_ISS) {
-                    if (!tc::mbar_wait(&empty[st], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
-                    tc::mbar_expect_tx(&full[st], stage_bytes);
+                    ok = __all_sync(0xffffffffu, tc::mbar_wait(&empty[st], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY));
+                    if (!ok) break;
                     uint8_t *dst = a_s + (size_t)st * N_ISS * p.tile_stride;
+                    if (tc::elect_one()) {
+                        tc::mbar_expect_tx(&full[st], stage_bytes);
 #pragma unroll
-                    for (int i = 0; i < N_ISS; ++i) tc::tma_load_2d(dst + (size_t)i * p.tile_stride, &tm_dz, &full[st], (kb + i) * BK, row0);
+                        for (int i = 0; i < N_ISS; ++i) tc::tma_load_2d(dst + (size_t)i * p.tile_stride, &tm_dz, &full[st], (kb + i) * BK, row0);
+                    }
+                    __syncwarp();
                     st += p.n_load;
                     if (st >= p.n_stages) { st -= p.n_stages; phase ^= 1; }
                 }

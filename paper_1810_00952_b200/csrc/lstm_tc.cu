@@ -84,7 +84,7 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * MAX_STAGES + 2);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // provably warp-uniform
     const int blk = blockIdx.x % p.n_blocks, grp = blockIdx.x / p.n_blocks;
     const int j0 = blk * UNITS;
     const int b_lo = grp * p.rows_per_group;                      // first batch row of this block's group
@@ -205,34 +205,43 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
       }
     } else if (warp == 5 || warp == 7) {
         // ------------------------------ h loaders: bf16(h_{t-1}) -> ring, by TMA ------------------------------
-        // (one thread needs several hundred cycles per stage; two threads take the stages of a step in turn)
+        // Two warps take the stages of a step in turn.  Each runs its loop warp-uniform and an elected lane issues:
+        // addresses and coordinates then stay in uniform registers, which costs far fewer cycles per copy than one
+        // divergent lane does.
         const int ld = warp == 5 ? 0 : 1;
-        if (lane == 0 && ld < p.n_load) {
+        if (ld < p.n_load) {
             int s = ld;
             uint32_t phase = 0;
             bool ok = true;
             const uint32_t stage_bytes = (uint32_t)(p.n_iss * p.rows_per_group * 128);
             for (int t = 0; t < p.T && ok; ++t) {
-                // grid barrier: every block has published its part of h_{t-1}
+                // grid barrier: every block has published its part of h_{t-1} (lane 0 polls, the warp follows)
                 const unsigned int target = (unsigned int)(p.n_epi * p.n_blocks) * (unsigned int)(t + 1);   // n_epi arrivals per block
-                const long long t0 = clock64();
-                unsigned spins = 0;
-                while (ld_acquire(counter) < target) {
-                    if ((++spins & 255u) == 0 && (*abort_flag || clock64() - t0 > tc::kWaitLimitCycles)) {
-                        if (!*abort_flag) { *abort_flag = 1; atomicCAS(p.err, 0, tc::ERR_WAIT_STEP); }
-                        ok = false;
-                        break;
+                if (lane == 0) {
+                    const long long t0 = clock64();
+                    unsigned spins = 0;
+                    while (ld_acquire(counter) < target) {
+                        if ((++spins & 255u) == 0 && (*abort_flag || clock64() - t0 > tc::kWaitLimitCycles)) {
+                            if (!*abort_flag) { *abort_flag = 1; atomicCAS(p.err, 0, tc::ERR_WAIT_STEP); }
+                            ok = false;
+                            break;
+                        }
                     }
+                    asm volatile("fence.proxy.async.global;" ::: "memory");
                 }
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
-                asm volatile("fence.proxy.async.global;" ::: "memory");
                 const CUtensorMap *tm_h = (t & 1) ? &tm_h1 : &tm_h0;
                 for (int kb = ld * p.n_iss; kb < p.k_blocks; kb += p.n_load * p.n_iss) {
-                    if (!tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
-                    tc::mbar_expect_tx(&full[s], stage_bytes);
+                    ok = __all_sync(0xffffffffu, tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY));
+                    if (!ok) break;
                     uint8_t *dst = a_s + (size_t)s * p.n_iss * p.tile_stride;
-                    for (int i = 0; i < p.n_iss; ++i)
-                        tc::tma_load_2d(dst + (size_t)i * p.tile_stride, tm_h, &full[s], (kb + i) * BK, b_lo);   // the group's rows only
+                    if (tc::elect_one()) {
+                        tc::mbar_expect_tx(&full[s], stage_bytes);
+                        for (int i = 0; i < p.n_iss; ++i)
+                            tc::tma_load_2d(dst + (size_t)i * p.tile_stride, tm_h, &full[s], (kb + i) * BK, b_lo);   // the group's rows only
+                    }
+                    __syncwarp();
                     s += p.n_load;
                     if (s >= p.n_stages) { s -= p.n_stages; phase ^= 1; }
                 }
@@ -240,13 +249,15 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
         }
     } else {
         // ------------------------------ MMA issuers (warp 4 also loads the W slice) ------------------------------
+        // The whole warp runs the loop with warp-uniform values and one elected lane issues (mma_bf16_elect).
         const int iss = warp == 4 ? 0 : 1;
-        if (lane == 0 && iss < p.n_iss) {
-            if (iss == 0) {
+        if (iss < p.n_iss) {
+            if (iss == 0 && lane == 0) {
                 tc::mbar_expect_tx(w_full, (uint32_t)(p.k_blocks * W_KB));
                 for (int kb = 0; kb < p.k_blocks; ++kb) tc::tma_load_2d(w_s + (size_t)kb * W_KB, &tm_w, w_full, kb * BK, blk * NCOL);
             }
-            bool ok = tc::mbar_wait(w_full, 0, abort_flag, p.err, tc::ERR_WAIT_FULL);
+            __syncwarp();
+            bool ok = __all_sync(0xffffffffu, tc::mbar_wait(w_full, 0, abort_flag, p.err, tc::ERR_WAIT_FULL));
             const uint32_t idesc = tc::instr_desc_bf16(128, NCOL, false, false);
             // descriptors differ from the first one only in the start-address field (16-byte units): one add per MMA
             const uint64_t desc_a0 = tc::smem_desc(tc::smem_u32(a_s) + (uint32_t)(iss * p.tile_stride), 16, 1024);
@@ -258,17 +269,19 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
             for (int t = 0; t < p.T && ok; ++t) {
                 uint32_t b_off = 0;
                 for (int kb = 0; kb < p.k_blocks; kb += p.n_iss) {     // this issuer's k-block of the stage: kb + iss
-                    if (!tc::mbar_wait(&full[s], phase, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
+                    // every lane waits; the vote reconverges the warp (the lanes leave the wait at different times)
+                    ok = __all_sync(0xffffffffu, tc::mbar_wait(&full[s], phase, abort_flag, p.err, tc::ERR_WAIT_FULL));
+                    if (!ok) break;
                     tc::tc_fence_after_sync();
                     const uint64_t da = desc_a0 + a_off, db = desc_b0 + b_off;
                     const uint32_t acc = kb != 0;
 #pragma unroll
-                    for (int kk = 0; kk < BK / 16; ++kk) tc::mma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, acc | (kk != 0));
-                    tc::mma_commit(&empty[s]);
+                    for (int kk = 0; kk < BK / 16; ++kk) tc::mma_bf16_elect(d_tmem, da + 2 * kk, db + 2 * kk, idesc, acc | (kk != 0));
+                    tc::mma_commit_elect(&empty[s]);
                     a_off += a_stage; b_off += b_stage;
                     if (++s == p.n_stages) { s = 0; phase ^= 1; a_off = 0; }
                 }
-                if (ok) tc::mma_commit(tmem_full);
+                if (ok) tc::mma_commit_elect(tmem_full);
             }
         }
     }
