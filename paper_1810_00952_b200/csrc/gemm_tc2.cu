@@ -210,7 +210,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + BAR_TMEM + 4);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // provably warp-uniform
     const uint32_t rank = tc::cluster_ctarank();          // 0 = leader
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     const int n_units = tb.n > 0 ? tb.n
@@ -293,7 +293,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer (leader only) ----------------
-        if (lane == 0 && rank == 0) {
+        // The whole warp runs the loop with warp-uniform values and one elected lane issues: the descriptors then stay
+        // in uniform registers and an MMA costs the issuing warp far fewer cycles than from a single divergent lane.
+        if (rank == 0) {
             constexpr uint32_t idesc_256 = tc::instr_desc_bf16(256, 256, A_MN, B_MN);
             constexpr uint32_t idesc_128 = tc::instr_desc_bf16(256, 128, A_MN, B_MN);
             constexpr uint32_t a_lbo = A_MN ? MN_BOX_BYTES : 16, b_lbo = B_MN ? MN_BOX_BYTES : 16;
@@ -316,34 +318,36 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                 const bool both = c >= 3;                 // the unit owns both accumulator halves (t_local is even: such units come first)
                 const int buf = t_local & 1;
                 const uint32_t par = ((t_local >> 1) & 1) ^ 1;
-                if (!tc::mbar_wait(&tmem_empty[buf], par, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) break;
-                if (both && !tc::mbar_wait(&tmem_empty[1], par, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) break;
+                // every lane waits; the votes reconverge the warp (the lanes leave a wait at different times)
+                if (!__all_sync(0xffffffffu, tc::mbar_wait(&tmem_empty[buf], par, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY))) break;
+                if (both && !__all_sync(0xffffffffu, tc::mbar_wait(&tmem_empty[1], par, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY))) break;
                 tc::tc_fence_after_sync();
                 const uint32_t d0 = tmem_base + buf * BN, d1 = tmem_base + BN;
                 const uint32_t idesc0 = c == 1 ? idesc_128 : idesc_256, idesc1 = c == 3 ? idesc_128 : idesc_256;
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
-                    if (!tc::mbar_wait(&full[s], phase, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
+                    ok = __all_sync(0xffffffffu, tc::mbar_wait(&full[s], phase, abort_flag, p.err, tc::ERR_WAIT_FULL));
+                    if (!ok) break;
                     tc::tc_fence_after_sync();
                     const uint64_t da = desc_a0 + stage_off, db = desc_b0 + stage_off;
                     const uint32_t acc = kb != 0;
                     if (both) {
 #pragma unroll
                         for (int kk = 0; kk < BK / 16; ++kk) {
-                            tc::mma_bf16_pair(d0, da + ((kk * a_step) >> 4), db + ((kk * b_step) >> 4), idesc0, acc | (kk != 0));
-                            tc::mma_bf16_pair(d1, da + ((kk * a_step) >> 4), db + b1_off + ((kk * b_step) >> 4), idesc1, acc | (kk != 0));
+                            tc::mma_bf16_pair_elect(d0, da + ((kk * a_step) >> 4), db + ((kk * b_step) >> 4), idesc0, acc | (kk != 0));
+                            tc::mma_bf16_pair_elect(d1, da + ((kk * a_step) >> 4), db + b1_off + ((kk * b_step) >> 4), idesc1, acc | (kk != 0));
                         }
                     } else {
 #pragma unroll
                         for (int kk = 0; kk < BK / 16; ++kk)
-                            tc::mma_bf16_pair(d0, da + ((kk * a_step) >> 4), db + ((kk * b_step) >> 4), idesc0, acc | (kk != 0));
+                            tc::mma_bf16_pair_elect(d0, da + ((kk * a_step) >> 4), db + ((kk * b_step) >> 4), idesc0, acc | (kk != 0));
                     }
-                    tc::mma_commit_pair(&empty[s]);
+                    tc::mma_commit_pair_elect(&empty[s]);
                     stage_off += (uint32_t)st_bytes >> 4;
                     if (++s == n_st) { s = 0; phase ^= 1; stage_off = 0; }
                 }
                 if (!ok) break;
-                tc::mma_commit_pair(&tmem_full[buf]);
-                if (both) tc::mma_commit_pair(&tmem_full[1]);
+                tc::mma_commit_pair_elect(&tmem_full[buf]);
+                if (both) tc::mma_commit_pair_elect(&tmem_full[1]);
                 t_local += both ? 2 : 1;
             }
         }
