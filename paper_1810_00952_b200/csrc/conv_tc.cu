@@ -369,7 +369,7 @@ conv_fprop_tc2_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
     uint64_t *full = bars, *empty = bars + STAGES, *tmem_full = bars + 2 * STAGES, *tmem_empty = bars + 2 * STAGES + 2;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 4);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // provably warp-uniform
     const uint32_t rank = tc::cluster_ctarank();
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     const int cblocks = p.Cin / BK, half_rows = p.rows_per_tile / 2;
@@ -418,7 +418,9 @@ conv_fprop_tc2_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
             }
         }
     } else if (warp == 1) {
-        if (lane == 0 && rank == 0) {
+        // the whole warp runs the issue loop with warp-uniform values, an elected lane issues (descriptors stay in
+        // uniform registers: an MMA costs the issuing warp far fewer cycles than from one divergent lane)
+        if (rank == 0) {
             const uint32_t idesc = tc::instr_desc_bf16(256, p.nt, false, false);
             const uint64_t desc_a0 = tc::smem_desc(tc::smem_u32(smem), 16, 1024), desc_b0 = tc::smem_desc(tc::smem_u32(smem) + a_bytes, 16, 1024);
             uint32_t t_local = 0, phase = 0, stage_off = 0;
@@ -426,21 +428,22 @@ conv_fprop_tc2_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
             bool ok = true;
             for (int item = pair; item < p.n_items && ok; item += n_pairs, ++t_local) {
                 const int buf = t_local & 1;
-                if (!tc::mbar_wait(&tmem_empty[buf], ((t_local >> 1) & 1) ^ 1, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) break;
+                if (!__all_sync(0xffffffffu, tc::mbar_wait(&tmem_empty[buf], ((t_local >> 1) & 1) ^ 1, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY))) break;
                 tc::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * 256;
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
-                    if (!tc::mbar_wait(&full[s], phase, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
+                    ok = __all_sync(0xffffffffu, tc::mbar_wait(&full[s], phase, abort_flag, p.err, tc::ERR_WAIT_FULL));
+                    if (!ok) break;
                     tc::tc_fence_after_sync();
                     const uint64_t da = desc_a0 + stage_off, db = desc_b0 + stage_off;
                     const uint32_t acc = kb != 0;
 #pragma unroll
-                    for (int kk = 0; kk < BK / 16; ++kk) tc::mma_bf16_pair(d_tmem, da + kk * 2, db + kk * 2, idesc, acc | (kk != 0));
-                    tc::mma_commit_pair(&empty[s]);
+                    for (int kk = 0; kk < BK / 16; ++kk) tc::mma_bf16_pair_elect(d_tmem, da + kk * 2, db + kk * 2, idesc, acc | (kk != 0));
+                    tc::mma_commit_pair_elect(&empty[s]);
                     stage_off += (uint32_t)stage_bytes >> 4;
                     if (++s == STAGES) { s = 0; phase ^= 1; stage_off = 0; }
                 }
-                if (ok) tc::mma_commit_pair(&tmem_full[buf]);
+                if (ok) tc::mma_commit_pair_elect(&tmem_full[buf]);
             }
         }
     } else {
@@ -655,7 +658,7 @@ conv_wgrad_tc2_kernel(const __grid_constant__ CUtensorMap tm_dz, const __grid_co
     uint64_t *full = bars, *empty = bars + STAGES, *tmem_full = bars + 2 * STAGES;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 2);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // provably warp-uniform
     const uint32_t rank = tc::cluster_ctarank();
 
     int u = blockIdx.x >> 1;                           // unit of the pair
@@ -707,22 +710,24 @@ conv_wgrad_tc2_kernel(const __grid_constant__ CUtensorMap tm_dz, const __grid_co
             }
         }
     } else if (warp == 1) {
-        if (lane == 0 && rank == 0) {
+        // warp-uniform issue loop, an elected lane issues
+        if (rank == 0) {
             const uint32_t idesc = tc::instr_desc_bf16(256, 256, true, true);
             int s = 0;
             uint32_t phase = 0;
             bool ok = true;
             for (int kb = 0; kb < k_blocks; ++kb) {
-                if (!tc::mbar_wait(&full[s], phase, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
+                ok = __all_sync(0xffffffffu, tc::mbar_wait(&full[s], phase, abort_flag, p.err, tc::ERR_WAIT_FULL));
+                if (!ok) break;
                 tc::tc_fence_after_sync();
                 const uint32_t sa = tc::smem_u32(smem + (size_t)s * stage_bytes), sb = sa + a_bytes;
                 const uint64_t da = tc::smem_desc(sa, box_bytes, 1024), db = tc::smem_desc(sb, box_bytes, 1024);
                 const uint32_t acc = kb != 0;
-                for (int kk = 0; kk < p.kpix / 16; ++kk) tc::mma_bf16_pair(tmem_base, da + kk * 128, db + kk * 128, idesc, acc | (kk != 0));
-                tc::mma_commit_pair(&empty[s]);
+                for (int kk = 0; kk < p.kpix / 16; ++kk) tc::mma_bf16_pair_elect(tmem_base, da + kk * 128, db + kk * 128, idesc, acc | (kk != 0));
+                tc::mma_commit_pair_elect(&empty[s]);
                 if (++s == STAGES) { s = 0; phase ^= 1; }
             }
-            if (ok) tc::mma_commit_pair(&tmem_full[0]);
+            if (ok) tc::mma_commit_pair_elect(&tmem_full[0]);
         }
     } else {
         const int quarter = warp & 3;
