@@ -395,7 +395,7 @@ conv_fprop_tc2_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
     pdl_wait();   // set-up done; from here on the kernel touches global memory
 
     if (warp == 0) {
-        if (lane == 0) {
+        {   // warp-uniform loop, an elected lane issues the copies
             int s = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -407,12 +407,16 @@ conv_fprop_tc2_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
                 for (int r = 0; r < p.taps_r && ok; ++r)
                     for (int sft = 0; sft < p.taps_s && ok; ++sft)
                         for (int cb = 0; cb < cblocks; ++cb, ++kb) {
-                            if (!tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
+                            ok = __all_sync(0xffffffffu, tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY));
+                            if (!ok) break;
                             uint8_t *sa = smem + (size_t)s * stage_bytes, *sb = sa + a_bytes;
                             const uint32_t bar = tc::mapa(tc::smem_u32(&full[s]), 0);
-                            if (rank == 0) tc::mbar_expect_tx_cluster(bar, 2 * (a_bytes + bh_bytes));
-                            tc::tma_load_2d_pair(sa, &tm_w, bar, kb * BK, m0);
-                            tc::tma_load_4d_pair(sb, &tm_x, bar, cb * BK, sft - p.pad, h0 + r - p.pad, img);
+                            if (tc::elect_one()) {
+                                if (rank == 0) tc::mbar_expect_tx_cluster(bar, 2 * (a_bytes + bh_bytes));
+                                tc::tma_load_2d_pair(sa, &tm_w, bar, kb * BK, m0);
+                                tc::tma_load_4d_pair(sb, &tm_x, bar, cb * BK, sft - p.pad, h0 + r - p.pad, img);
+                            }
+                            __syncwarp();
                             if (++s == STAGES) { s = 0; phase ^= 1; }
                         }
             }
@@ -693,19 +697,22 @@ conv_wgrad_tc2_kernel(const __grid_constant__ CUtensorMap tm_dz, const __grid_co
     pdl_wait();   // set-up done; from here on the kernel touches global memory
 
     if (warp == 0) {
-        if (lane == 0) {
+        {   // warp-uniform loop, an elected lane issues the copies
             int s = 0;
             uint32_t phase = 0;
             for (int kb = 0; kb < k_blocks; ++kb) {
-                if (!tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) break;
+                if (!__all_sync(0xffffffffu, tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY))) break;
                 uint8_t *sa = smem + (size_t)s * stage_bytes, *sb = sa + a_bytes;
                 const uint32_t bar = tc::mapa(tc::smem_u32(&full[s]), 0);
-                if (rank == 0) tc::mbar_expect_tx_cluster(bar, 2 * stage_bytes);
                 const int img = img0 + kb / kb_per_img, h0 = (kb % kb_per_img) * p.rows_per_kblock;
+                if (tc::elect_one()) {
+                    if (rank == 0) tc::mbar_expect_tx_cluster(bar, 2 * stage_bytes);
 #pragma unroll
-                for (int i = 0; i < 2; ++i) tc::tma_load_4d_pair(sa + i * box_bytes, &tm_dz, bar, o0 + i * 64, 0, h0, img);
+                    for (int i = 0; i < 2; ++i) tc::tma_load_4d_pair(sa + i * box_bytes, &tm_dz, bar, o0 + i * 64, 0, h0, img);
 #pragma unroll
-                for (int j = 0; j < 2; ++j) tc::tma_load_4d_pair(sb + j * box_bytes, &tm_x, bar, c0 + j * 64, sft - p.pad, h0 + r - p.pad, img);
+                    for (int j = 0; j < 2; ++j) tc::tma_load_4d_pair(sb + j * box_bytes, &tm_x, bar, c0 + j * 64, sft - p.pad, h0 + r - p.pad, img);
+                }
+                __syncwarp();
                 if (++s == STAGES) { s = 0; phase ^= 1; }
             }
         }
