@@ -240,7 +240,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         // ---------------- TMA producers (both blocks): warp 0 loads A and posts the byte count, warp 18 loads B ----------------
         // (one thread issues only a few instructions per hundred cycles; two threads keep the ring fed)
         const bool load_a = warp == 0;
-        if (lane == 0) {
+        {   // warp-uniform loop, an elected lane issues the copies
             int cur = 0, s = 0, n_st = 0, st_bytes = 0;
             uint32_t phase = 0;
             uint64_t *full = bars, *empty = bars;
@@ -251,7 +251,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                 if (c != cur) {
                     // the new class's stages lie over the old one's: every old stage must have been released
                     for (int i = 0; i < n_st && ok; ++i) {
-                        if (!tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) ok = false;
+                        ok = __all_sync(0xffffffffu, tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY));
                         if (++s == n_st) { s = 0; phase ^= 1; }
                     }
                     if (!ok) break;
@@ -266,27 +266,31 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                 const int boxes0 = h0 >> 6, boxes = (h0 + h1) >> 6;
                 const uint32_t tx = 2u * (uint32_t)st_bytes;                        // bytes of both blocks
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
-                    if (!tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
+                    ok = __all_sync(0xffffffffu, tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY));
+                    if (!ok) break;
                     uint8_t *sa = smem + (size_t)s * st_bytes, *sb = sa + A_BYTES;
                     const uint32_t bar = tc::mapa(tc::smem_u32(&full[s]), 0);       // the leader's barrier
                     const int k0 = kb * BK;
-                    if (load_a) {
-                        if (rank == 0) tc::mbar_expect_tx_cluster(bar, tx);
-                        if (A_MN) {
+                    if (tc::elect_one()) {
+                        if (load_a) {
+                            if (rank == 0) tc::mbar_expect_tx_cluster(bar, tx);
+                            if (A_MN) {
 #pragma unroll
-                            for (int i = 0; i < 2; ++i) tc::tma_load_2d_pair(sa + i * MN_BOX_BYTES, &tm_a, bar, m0 + i * 64, k0);
+                                for (int i = 0; i < 2; ++i) tc::tma_load_2d_pair(sa + i * MN_BOX_BYTES, &tm_a, bar, m0 + i * 64, k0);
+                            } else {
+                                tc::tma_load_2d_pair(sa, &tm_a, bar, k0, m0);
+                            }
                         } else {
-                            tc::tma_load_2d_pair(sa, &tm_a, bar, k0, m0);
-                        }
-                    } else {
-                        // B in boxes of 64 columns: MN-major boxes are 64 x 64 k anyway; K-major boxes of 64 rows stack
-                        // to the same shared-memory image as one taller box
-                        for (int i = 0; i < boxes; ++i) {
-                            const int n = i < boxes0 ? na + i * 64 : nb + (i - boxes0) * 64;
-                            if (B_MN) tc::tma_load_2d_pair(sb + i * MN_BOX_BYTES, &tm_b, bar, n, k0);
-                            else tc::tma_load_2d_pair(sb + i * MN_BOX_BYTES, &tm_b, bar, k0, n);
+                            // B in boxes of 64 columns: MN-major boxes are 64 x 64 k anyway; K-major boxes of 64 rows stack
+                            // to the same shared-memory image as one taller box
+                            for (int i = 0; i < boxes; ++i) {
+                                const int n = i < boxes0 ? na + i * 64 : nb + (i - boxes0) * 64;
+                                if (B_MN) tc::tma_load_2d_pair(sb + i * MN_BOX_BYTES, &tm_b, bar, n, k0);
+                                else tc::tma_load_2d_pair(sb + i * MN_BOX_BYTES, &tm_b, bar, k0, n);
+                            }
                         }
                     }
+                    __syncwarp();
                     if (++s == n_st) { s = 0; phase ^= 1; }
                 }
             }
