@@ -195,7 +195,7 @@ conv_fprop_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
     uint64_t *full = bars, *empty = bars + STAGES, *tmem_full = bars + 2 * STAGES, *tmem_empty = bars + 2 * STAGES + 2;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 4);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // provably warp-uniform
     const int cblocks = p.Cin / BK;
 
     if (threadIdx.x == 0) {
@@ -237,7 +237,7 @@ conv_fprop_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
+        {   // warp-uniform issue loop, an elected lane issues
             const uint32_t idesc = tc::instr_desc_bf16(BM, p.nt, false, false);
             const uint64_t desc_a0 = tc::smem_desc(tc::smem_u32(smem), 16, 1024), desc_b0 = tc::smem_desc(tc::smem_u32(smem) + a_bytes, 16, 1024);
             uint32_t t_local = 0, phase = 0, stage_off = 0;   // stage_off = s * stage_bytes in 16-byte units
@@ -247,12 +247,13 @@ conv_fprop_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
                 const FpropItem wi = fprop_item<MH>(p, item);
                 const int buf = MH == 1 ? (t_local & 1) : 0;
                 const uint32_t empty_parity = MH == 1 ? (((t_local >> 1) & 1) ^ 1) : ((t_local & 1) ^ 1);
-                if (!tc::mbar_wait(&tmem_empty[buf], empty_parity, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) break;
-                if (MH == 2 && !tc::mbar_wait(&tmem_empty[1], empty_parity, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) break;
+                if (!__all_sync(0xffffffffu, tc::mbar_wait(&tmem_empty[buf], empty_parity, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY))) break;
+                if (MH == 2 && !__all_sync(0xffffffffu, tc::mbar_wait(&tmem_empty[1], empty_parity, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY))) break;
                 tc::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * 256;
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
-                    if (!tc::mbar_wait(&full[s], phase, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
+                    ok = __all_sync(0xffffffffu, tc::mbar_wait(&full[s], phase, abort_flag, p.err, tc::ERR_WAIT_FULL));
+                    if (!ok) break;
                     tc::tc_fence_after_sync();
                     // descriptors differ from the stage-0 ones only in the start address field (16-byte units),
                     // so the issuing thread spends one add per MMA instead of rebuilding them
@@ -261,18 +262,18 @@ conv_fprop_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
                     if (MH == 2 && wi.mh == 2) {
 #pragma unroll
                         for (int kk = 0; kk < BK / 16; ++kk) {
-                            tc::mma_bf16(d_tmem, da + kk * 2, db + kk * 2, idesc, acc | (kk != 0));
-                            tc::mma_bf16(d_tmem + 256, da + (BM * BK * 2 >> 4) + kk * 2, db + kk * 2, idesc, acc | (kk != 0));
+                            tc::mma_bf16_elect(d_tmem, da + kk * 2, db + kk * 2, idesc, acc | (kk != 0));
+                            tc::mma_bf16_elect(d_tmem + 256, da + (BM * BK * 2 >> 4) + kk * 2, db + kk * 2, idesc, acc | (kk != 0));
                         }
                     } else {
 #pragma unroll
-                        for (int kk = 0; kk < BK / 16; ++kk) tc::mma_bf16(d_tmem, da + kk * 2, db + kk * 2, idesc, acc | (kk != 0));
+                        for (int kk = 0; kk < BK / 16; ++kk) tc::mma_bf16_elect(d_tmem, da + kk * 2, db + kk * 2, idesc, acc | (kk != 0));
                     }
-                    tc::mma_commit(&empty[s]);
+                    tc::mma_commit_elect(&empty[s]);
                     stage_off += (uint32_t)stage_bytes >> 4;
                     if (++s == STAGES) { s = 0; phase ^= 1; stage_off = 0; }
                 }
-                if (ok) tc::mma_commit(&tmem_full[buf]);
+                if (ok) tc::mma_commit_elect(&tmem_full[buf]);
             }
         }
     } else {

@@ -55,7 +55,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 4);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // provably warp-uniform
     const int n_tiles = p.tiles_m * p.tiles_n;
 
     if (threadIdx.x == 0) {
@@ -79,17 +79,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
-        if (lane == 0) {
+        {   // warp-uniform loop, an elected lane issues the copies (addresses stay in uniform registers)
             int s = 0;
             uint32_t phase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
                 const int m0 = (tile % p.tiles_m) * BM, n0 = (tile / p.tiles_m) * BN;
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
-                    if (!tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY)) { ok = false; break; }
+                    ok = __all_sync(0xffffffffu, tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY));
+                    if (!ok) break;
                     uint8_t *sa = smem + (size_t)s * STAGE_BYTES, *sb = sa + A_BYTES;
-                    tc::mbar_expect_tx(&full[s], STAGE_BYTES);
                     const int k0 = kb * BK;
+                    if (tc::elect_one()) {
+                    tc::mbar_expect_tx(&full[s], STAGE_BYTES);
                     if (A_MN) {
 #pragma unroll
                         for (int i = 0; i < BM / 64; ++i) tc::tma_load_2d(sa + i * MN_BOX_BYTES, &tm_a, &full[s], m0 + i * 64, k0);
@@ -102,13 +104,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     } else {
                         tc::tma_load_2d(sb, &tm_b, &full[s], k0, n0);
                     }
+                    }
+                    __syncwarp();
                     if (++s == STAGES) { s = 0; phase ^= 1; }
                 }
             }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        if (lane == 0) {
+        {   // warp-uniform loop, an elected lane issues (descriptors stay in uniform registers)
             constexpr uint32_t idesc = tc::instr_desc_bf16(128, BN, A_MN, B_MN);
             // K-major: 8-row atoms 1024 B apart, one MMA (16 k) = 32 bytes along the swizzled row;
             // MN-major: 64-wide M/N groups one TMA box apart, 8-k atoms 1024 B apart, one MMA = 2 atoms.
@@ -125,12 +129,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 // MH = 1: accumulator t_local & 1;  MH = 2: accumulator h for half h, both used by every tile
                 const int buf = MH == 1 ? (t_local & 1) : 0;
                 const uint32_t empty_parity = MH == 1 ? (((t_local >> 1) & 1) ^ 1) : ((t_local & 1) ^ 1);
-                if (!tc::mbar_wait(&tmem_empty[buf], empty_parity, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) break;
-                if (MH == 2 && !tc::mbar_wait(&tmem_empty[1], empty_parity, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY)) break;
+                if (!__all_sync(0xffffffffu, tc::mbar_wait(&tmem_empty[buf], empty_parity, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY))) break;
+                if (MH == 2 && !__all_sync(0xffffffffu, tc::mbar_wait(&tmem_empty[1], empty_parity, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY))) break;
                 tc::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * BN;
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
-                    if (!tc::mbar_wait(&full[s], phase, abort_flag, p.err, tc::ERR_WAIT_FULL)) { ok = false; break; }
+                    ok = __all_sync(0xffffffffu, tc::mbar_wait(&full[s], phase, abort_flag, p.err, tc::ERR_WAIT_FULL));
+                    if (!ok) break;
                     tc::tc_fence_after_sync();
                     const uint64_t da = desc_a0 + stage_off, db = desc_b0 + stage_off;
                     const uint32_t acc = kb != 0;
@@ -138,14 +143,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     for (int kk = 0; kk < BK / 16; ++kk) {
 #pragma unroll
                         for (int h = 0; h < MH; ++h)
-                            tc::mma_bf16(d_tmem + h * BN, da + ((h * (128 * BK * 2) + kk * a_step) >> 4), db + ((kk * b_step) >> 4), idesc,
+                            tc::mma_bf16_elect(d_tmem + h * BN, da + ((h * (128 * BK * 2) + kk * a_step) >> 4), db + ((kk * b_step) >> 4), idesc,
                                          acc | (kk != 0));
                     }
-                    tc::mma_commit(&empty[s]);          // the stage is free once these MMAs have read it
+                    tc::mma_commit_elect(&empty[s]);          // the stage is free once these MMAs have read it
                     stage_off += STAGE_BYTES >> 4;
                     if (++s == STAGES) { s = 0; phase ^= 1; stage_off = 0; }
                 }
-                if (ok) tc::mma_commit(&tmem_full[buf]);  // the accumulator(s) are complete
+                if (ok) tc::mma_commit_elect(&tmem_full[buf]);  // the accumulator(s) are complete
             }
         }
     } else {
