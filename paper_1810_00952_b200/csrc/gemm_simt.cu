@@ -41,6 +41,9 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmDesc g)
             Bs[kk][nn] = (n < g.N && k < g.K) ? to_f<TIN>(B[k * g.b_sk + n * g.b_sn]) : 0.0f;
         }
         __syncthreads();
+        // threads whose 4 x 4 outputs all lie outside the problem skip the arithmetic (a tiny M or N would
+        // otherwise fill the fp64 pipe with products nobody stores)
+        if (m0 + tm < g.M && n0 + tn < g.N)
 #pragma unroll
         for (int kk = 0; kk < BK; ++kk) {
             float av[4], bv[4];
