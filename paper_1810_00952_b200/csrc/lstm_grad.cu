@@ -162,7 +162,7 @@ constexpr int W_KB = UNITS * BK * 2;             // one k-block of the resident 
 // As in the forward kernel, ring stages are only as far apart as the rows a group really has: the MMA's rows
 // beyond the group's are whatever follows in shared memory, and the accumulator rows they produce are never read.
 constexpr int N_ISS = 4;                         // MMA-issuing threads (one lane each of warps 4, 6, 7, 8), one accumulator each
-constexpr int NUM_THREADS = 320;                 // warps 0-3 epilogue, warp 4 W loader + issuer 0, warps 5 and 9 dz loaders, warps 6-8 issuers 1-3
+constexpr int NUM_THREADS = 512;                 // warps 0-3 and 12-15 epilogue, warp 4 W loader + issuer 0, warps 5 and 9 dz loaders, warps 6-8 issuers 1-3
 constexpr int TMEM_COLS = N_ISS * UNITS;
 // One thread issues a tcgen05.mma of N = 16 only every hundred cycles or so (descriptor arithmetic, barrier polling),
 // far slower than the tensor pipe runs it.  So a ring stage holds N_ISS k-blocks (one barrier round per stage), each
@@ -193,6 +193,14 @@ __device__ __forceinline__ unsigned int ld_acquire(const unsigned int *p)
 __device__ __forceinline__ void red_release_add(unsigned int *p, unsigned int v)
 {
     asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void load8(const float *p, float (&v)[UNITS / 2])
+{
+#pragma unroll
+    for (int i = 0; i < UNITS / 2; i += 4) {
+        const float4 q = *reinterpret_cast<const float4 *>(p + i);
+        v[i] = q.x; v[i + 1] = q.y; v[i + 2] = q.z; v[i + 3] = q.w;
+    }
 }
 __device__ __forceinline__ void load16(const float *p, float (&v)[UNITS])
 {
@@ -239,30 +247,35 @@ lstm_grad_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __gr
     tc::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp < 4) {
-      if (warp < p.n_epi) {
-        // ------------------------------ epilogue: one batch row per lane, 16 units ------------------------------
+    if (warp < 4 || warp >= 12) {
+      const int ew = warp & 3, half = warp >= 12 ? 1 : 0;
+      if (ew < p.n_epi) {
+        // ------------------------------ epilogue: one batch row per lane, 8 of the block's 16 units per warp ------------------------------
+        // Two warps share a TMEM lane quarter (warps w and 12 + w) and take 8 units each: one warp alone issues its
+        // instructions only every few cycles, and this part is on the critical path of every step.
         // M = 128: accumulator row r sits in TMEM lane r.  M = 64: rows 16w .. 16w+15 sit in lanes 32w .. 32w+15, so warp w
         // owns 16 rows in its first 16 lanes.
-        const int b = b_lo + warp * p.rows_per_warp + lane;
-        const bool live = lane < p.rows_per_warp && warp * p.rows_per_warp + lane < nb;
-        float dc[UNITS], c_cur[UNITS];
+        constexpr int HU = UNITS / 2;
+        const int u0 = j0 + half * HU;
+        const int b = b_lo + ew * p.rows_per_warp + lane;
+        const bool live = lane < p.rows_per_warp && ew * p.rows_per_warp + lane < nb;
+        float dc[HU], c_cur[HU];
 #pragma unroll
-        for (int i = 0; i < UNITS; ++i) { dc[i] = 0.0f; c_cur[i] = 0.0f; }
+        for (int i = 0; i < HU; ++i) { dc[i] = 0.0f; c_cur[i] = 0.0f; }
         if (live) {
-            if (p.dc_final) load16(p.dc_final + (size_t)b * p.H + j0, dc);
-            load16(p.c_all + ((size_t)(p.T - 1) * p.B + b) * p.H + j0, c_cur);
+            if (p.dc_final) load8(p.dc_final + (size_t)b * p.H + u0, dc);
+            load8(p.c_all + ((size_t)(p.T - 1) * p.B + b) * p.H + u0, c_cur);
         }
         for (int s = 0; s <= p.T; ++s) {
             const int t = p.T - 1 - s;
             // what does not depend on the recurrent product is fetched while it runs
-            float gt[4][UNITS], c_prev[UNITS], dh[UNITS];
+            float gt[4][HU], c_prev[HU], dh[HU];
             if (live && s < p.T) {
-                const float *grow = p.gates + ((size_t)t * p.B + b) * 4 * p.H + j0;
+                const float *grow = p.gates + ((size_t)t * p.B + b) * 4 * p.H + u0;
 #pragma unroll
-                for (int g = 0; g < 4; ++g) load16(grow + (size_t)g * p.H, gt[g]);
-                load16(t > 0 ? p.c_all + ((size_t)(t - 1) * p.B + b) * p.H + j0 : p.c0 + (size_t)b * p.H + j0, c_prev);
-                load16(p.dh_all + ((size_t)t * p.B + b) * p.H + j0, dh);
+                for (int g = 0; g < 4; ++g) load8(grow + (size_t)g * p.H, gt[g]);
+                load8(t > 0 ? p.c_all + ((size_t)(t - 1) * p.B + b) * p.H + u0 : p.c0 + (size_t)b * p.H + u0, c_prev);
+                load8(p.dh_all + ((size_t)t * p.B + b) * p.H + u0, dh);
             }
             if (s > 0) {
                 int ok = 1;
@@ -270,43 +283,41 @@ lstm_grad_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __gr
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) break;
                 tc::tc_fence_after_sync();
-                uint32_t d[32], d2[32];                                               // the four issuers' partial sums, 16 columns each
-                tc::tmem_ld_32x32(tmem_base + ((uint32_t)(warp * 32) << 16), d);
-                tc::tmem_ld_32x32(tmem_base + ((uint32_t)(warp * 32) << 16) + 32, d2);
+                uint32_t d[N_ISS][HU];                                                // the four issuers' partial sums of this warp's units
+                const uint32_t taddr = tmem_base + ((uint32_t)(ew * 32) << 16) + half * HU;
+#pragma unroll
+                for (int a = 0; a < N_ISS; ++a) tc::tmem_ld_32x8(taddr + a * UNITS, d[a]);
                 tc::tmem_ld_wait();
                 tc::tc_fence_before_sync();
+                float rec[HU];
 #pragma unroll
-                for (int i = 0; i < UNITS; ++i)
-                    d[i] = __float_as_uint((__uint_as_float(d[i]) + __uint_as_float(d[UNITS + i])) +
-                                           (__uint_as_float(d2[i]) + __uint_as_float(d2[UNITS + i])));
+                for (int i = 0; i < HU; ++i)
+                    rec[i] = (__uint_as_float(d[0][i]) + __uint_as_float(d[1][i])) + (__uint_as_float(d[2][i]) + __uint_as_float(d[3][i]));
                 if (s == p.T) {
                     if (live && p.dh0) {
-                        float4 *o = reinterpret_cast<float4 *>(p.dh0 + (size_t)b * p.H + j0);
+                        float4 *o = reinterpret_cast<float4 *>(p.dh0 + (size_t)b * p.H + u0);
 #pragma unroll
-                        for (int i = 0; i < UNITS; i += 4)
-                            o[i / 4] = make_float4(__uint_as_float(d[i]), __uint_as_float(d[i + 1]), __uint_as_float(d[i + 2]), __uint_as_float(d[i + 3]));
+                        for (int i = 0; i < HU; i += 4) o[i / 4] = make_float4(rec[i], rec[i + 1], rec[i + 2], rec[i + 3]);
                     }
                     break;
                 }
 #pragma unroll
-                for (int i = 0; i < UNITS; ++i) dh[i] += __uint_as_float(d[i]);
+                for (int i = 0; i < HU; ++i) dh[i] += rec[i];
             }
             if (live) {
-                float dzv[4][UNITS];
+                float dzv[4][HU];
 #pragma unroll
-                for (int i = 0; i < UNITS; ++i) {
+                for (int i = 0; i < HU; ++i) {
                     float q[4];
                     gate_grads(gt[0][i], gt[1][i], gt[2][i], gt[3][i], c_cur[i], c_prev[i], dh[i], dc[i], q);
                     dzv[0][i] = q[0]; dzv[1][i] = q[1]; dzv[2][i] = q[2]; dzv[3][i] = q[3];
                     c_cur[i] = c_prev[i];
                 }
-                __nv_bfloat16 *drow = p.dz + ((size_t)t * p.B + b) * 4 * p.H + j0;
+                __nv_bfloat16 *drow = p.dz + ((size_t)t * p.B + b) * 4 * p.H + u0;
 #pragma unroll
-                for (int g = 0; g < 4; ++g) {
-                    uint4 *o = reinterpret_cast<uint4 *>(drow + (size_t)g * p.H);
-                    o[0] = make_uint4(pack2(dzv[g][0], dzv[g][1]), pack2(dzv[g][2], dzv[g][3]), pack2(dzv[g][4], dzv[g][5]), pack2(dzv[g][6], dzv[g][7]));
-                    o[1] = make_uint4(pack2(dzv[g][8], dzv[g][9]), pack2(dzv[g][10], dzv[g][11]), pack2(dzv[g][12], dzv[g][13]), pack2(dzv[g][14], dzv[g][15]));
-                }
+                for (int g = 0; g < 4; ++g)
+                    *reinterpret_cast<uint4 *>(drow + (size_t)g * p.H) =
+                        make_uint4(pack2(dzv[g][0], dzv[g][1]), pack2(dzv[g][2], dzv[g][3]), pack2(dzv[g][4], dzv[g][5]), pack2(dzv[g][6], dzv[g][7]));
             }
             // dZ[t] is read by TMA (async proxy) in the other blocks: fence the generic stores for it; the warp barrier orders
             // the warp's stores before lane 0's release, which is cumulative
@@ -315,9 +326,9 @@ lstm_grad_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __gr
             if (lane == 0) red_release_add(counter, 1u);
         }
         if (live && p.dc0) {
-            float4 *o = reinterpret_cast<float4 *>(p.dc0 + (size_t)b * p.H + j0);
+            float4 *o = reinterpret_cast<float4 *>(p.dc0 + (size_t)b * p.H + u0);
 #pragma unroll
-            for (int i = 0; i < UNITS; i += 4) o[i / 4] = make_float4(dc[i], dc[i + 1], dc[i + 2], dc[i + 3]);
+            for (int i = 0; i < HU; i += 4) o[i / 4] = make_float4(dc[i], dc[i + 1], dc[i + 2], dc[i + 3]);
         }
       }
     } else if (warp == 5 || warp == 9) {
@@ -331,7 +342,7 @@ lstm_grad_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __gr
             const uint32_t stage_bytes = (uint32_t)(N_ISS * p.rows_per_group * 128);
             for (int s = 1; s <= p.T && ok; ++s) {
                 // grid barrier: every block of the group has written its columns of dZ[T-s] (lane 0 polls, the warp follows)
-                const unsigned int target = (unsigned int)(p.n_epi * p.n_blocks) * (unsigned int)s;
+                const unsigned int target = (unsigned int)(2 * p.n_epi * p.n_blocks) * (unsigned int)s;   // two epilogue warps per 16 or 32 rows
                 if (lane == 0) {
                     const long long t0 = clock64();
                     unsigned spins = 0;
@@ -362,7 +373,7 @@ lstm_grad_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __gr
                 }
             }
         }
-    } else {
+    } else if (warp == 4 || (warp >= 6 && warp <= 8)) {
         // ------------------------------ MMA issuers (warp 4 also loads the W slice) ------------------------------
         // The whole warp runs the loop with warp-uniform values and one elected lane issues (mma_bf16_elect).
         {
