@@ -155,7 +155,7 @@ __device__ __forceinline__ void finish_group(const Params &p, const CUtensorMap 
     const int sw = (lane >> 1) & 3;
 #pragma unroll
     for (int h = 0; h < (OUT_F32 ? 2 : 1); ++h) {        // 64 bytes of every row at a time
-        if (lane == 0) tc::tma_store_wait_read<0>();     // the previous store has read the buffer
+        if (tc::elect_one()) tc::tma_store_wait_read<0>();   // the previous store (same elected lane) has read the buffer
         __syncwarp();
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
@@ -168,7 +168,7 @@ __device__ __forceinline__ void finish_group(const Params &p, const CUtensorMap 
         }
         tc::fence_proxy_async();
         __syncwarp();
-        if (lane == 0) {
+        if (tc::elect_one()) {                           // the election is deterministic: always the same lane of the warp
             tc::tma_store_2d(tm_c, stage, nc + h * (OUT_F32 ? 16 : 0), row0);
             tc::tma_store_commit();
         }
@@ -388,7 +388,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                 if (lane == 0) tc::mbar_arrive_cluster(tc::mapa(tc::smem_u32(&tmem_empty[buf]), 0));
             }
         }
-        if (lane == 0) tc::tma_store_wait_all<0>();
+        __syncwarp();
+        if (tc::elect_one()) tc::tma_store_wait_all<0>();
     }
 
     tc::tc_fence_before_sync();
