@@ -28,6 +28,8 @@ relay_status_t make_tmap_nhwc_bf16(CUtensorMap *m, const void *base, uint64_t C,
                                    uint32_t box_c, uint32_t box_w, uint32_t box_h);
 relay_status_t make_tmap_2d(CUtensorMap *m, bool f32, const void *base, uint64_t inner, uint64_t outer, uint64_t row_stride,
                             uint32_t box_inner, uint32_t box_outer, bool swizzle128);
+relay_status_t make_tmap_2d_sw64(CUtensorMap *m, bool f32, const void *base, uint64_t inner, uint64_t outer, uint64_t row_stride,
+                                 uint32_t box_outer);
 
 namespace {
 
@@ -495,16 +497,18 @@ conv_fprop_tc2_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
                 default: break;
                 }
                 uint8_t *st = my_stage + (blk_count & 1) * 2048;
-                if (lane == 0) tc::tma_store_wait_read<1>();
+                if (tc::elect_one()) tc::tma_store_wait_read<1>();   // always the same lane of the warp
                 __syncwarp();
+                // 32 rows x 64 bytes in the 64-byte swizzle pattern of the output tensor map (16-byte piece q of row r at
+                // piece q ^ ((r >> 1) & 3)): conflict-free stores
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
-                    *reinterpret_cast<uint4 *>(st + lane * 64 + q * 16) =
+                    *reinterpret_cast<uint4 *>(st + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4)) =
                         make_uint4(pack2(v[8 * q], v[8 * q + 1]), pack2(v[8 * q + 2], v[8 * q + 3]), pack2(v[8 * q + 4], v[8 * q + 5]),
                                    pack2(v[8 * q + 6], v[8 * q + 7]));
                 tc::fence_proxy_async();
                 __syncwarp();
-                if (lane == 0) {
+                if (tc::elect_one()) {
                     tc::tma_store_2d(&tm_y, st, h0 * p.W + c * 32, img * p.Cout + o0);
                     tc::tma_store_commit();
                 }
@@ -513,7 +517,7 @@ conv_fprop_tc2_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
             __syncwarp();
             if (lane == 0) tc::mbar_arrive_cluster(tc::mapa(tc::smem_u32(&tmem_empty[buf]), 0));
         }
-        if (lane == 0) tc::tma_store_wait_all<0>();
+        if (tc::elect_one()) tc::tma_store_wait_all<0>();
     }
     tc::tc_fence_before_sync();
     __syncthreads();
@@ -863,15 +867,17 @@ relay_status_t launch_fprop(const ConvDims &d, const TcPlan &pl, const void *act
     // two-SM form: every tile is computed by a pair of blocks, each loading half of the activation tile
     if (Cout % 256 == 0 && pl.rows_per_tile % 2 == 0 && ((p.nt / 2) * 128) % 1024 == 0 && sms >= 2 &&
         (int64_t)p.n_tiles_total * (Cout / 256) >= sms / 2) {
-        CUtensorMap tm_xh;
+        CUtensorMap tm_xh, tm_y2;
         RELAY_TRY(make_tmap_nhwc_bf16(&tm_xh, act_nhwc, Cin, d.W, d.H, d.Nb, BK, (uint32_t)d.W, pl.rows_per_tile / 2));
+        // output boxes of 32 channels x 32 pixels, rows of 64 bytes in the 64-byte swizzle pattern
+        RELAY_TRY(make_tmap_2d_sw64(&tm_y2, false, out_nchw, (uint64_t)(d.H * d.W), (uint64_t)d.Nb * Cout, (uint64_t)(d.H * d.W), 32));
         const size_t stage2 = (size_t)BM * BK * 2 + (size_t)(p.nt / 2) * 128;
         p.stages = (int)std::min<size_t>(8, (kSmemLimit - 1024 - 4 * 4096) / stage2);
         p.pairs_per_ntile = Cout / 256;
         p.n_pairs = p.n_items = p.n_tiles_total * p.pairs_per_ntile;
         const size_t smem2 = 1024 + (size_t)p.stages * stage2 + 4 * 4096 + 256;
         RELAY_CUDA(cudaFuncSetAttribute(conv_fprop_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2));
-        RELAY_CUDA(launch_pdl(conv_fprop_tc2_kernel, dim3(2 * std::min(p.n_items, sms / 2)), dim3(NUM_THREADS), smem2, st, tm_w, tm_xh, tm_y, p));
+        RELAY_CUDA(launch_pdl(conv_fprop_tc2_kernel, dim3(2 * std::min(p.n_items, sms / 2)), dim3(NUM_THREADS), smem2, st, tm_w, tm_xh, tm_y2, p));
         return check_launch("conv_fprop_tc2");
     }
     // one-SM form: pairs fill whole rounds over the SMs; the remainder runs as singles
