@@ -238,7 +238,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
 
     if (warp == 0 || warp == 18) {
         // ---------------- TMA producers (both blocks): warp 0 loads A and posts the byte count, warp 18 loads B ----------------
-        // (one thread issues only a few instructions per hundred cycles; two threads keep the ring fed)
+        // (two producer warps keep the ring fed)
         const bool load_a = warp == 0;
         {   // warp-uniform loop, an elected lane issues the copies
             int cur = 0, s = 0, n_st = 0, st_bytes = 0;

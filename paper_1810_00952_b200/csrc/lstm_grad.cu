@@ -151,7 +151,7 @@ __global__ void __launch_bounds__(128) colsum_any_kernel(const __nv_bfloat16 *__
 // Block (grp, blk) owns 16 hidden units and the batch rows of group grp.  Per step s = 1 .. T it needs
 // dh_rec[row, unit] = sum_col dz_{T-s}[row, col] * W_hh[unit, col] over all 4H columns: its 16 rows of W_hh
 // (16 x 4H bf16, at most 128 KB) stay in shared memory, dz of the group's rows is streamed from the dZ array
-// (L2) through a ring by TMA, one thread issues tcgen05.mma (D[row, 16 units] in TMEM).  The epilogue warp
+// (L2) through a ring by TMA, issuer warps run tcgen05.mma (D[row, 16 units] in TMEM).  The epilogue warp
 // owning a row adds dh_all, applies the gate derivatives, writes bf16(dz_t) of its 64 gate columns into
 // dZ[t] and arrives on the group's grid barrier; the carried dc stays in registers.
 constexpr int UNITS = 16;
@@ -164,8 +164,8 @@ constexpr int W_KB = UNITS * BK * 2;             // one k-block of the resident 
 constexpr int N_ISS = 4;                         // MMA-issuing threads (one lane each of warps 4, 6, 7, 8), one accumulator each
 constexpr int NUM_THREADS = 512;                 // warps 0-3 and 12-15 epilogue, warp 4 W loader + issuer 0, warps 5 and 9 dz loaders, warps 6-8 issuers 1-3
 constexpr int TMEM_COLS = N_ISS * UNITS;
-// One thread issues a tcgen05.mma of N = 16 only every hundred cycles or so (descriptor arithmetic, barrier polling),
-// far slower than the tensor pipe runs it.  So a ring stage holds N_ISS k-blocks (one barrier round per stage), each
+// Issuing a tcgen05.mma of N = 16 costs the issuing warp tens of cycles even with warp-uniform operands (about 130
+// from a single divergent lane), far more than the tensor pipe needs for it.  So a ring stage holds N_ISS k-blocks (one barrier round per stage), each
 // issuer takes one k-block of every stage into its own accumulator, and the epilogue adds the accumulators up.
 
 struct GradParams {
@@ -333,7 +333,7 @@ lstm_grad_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __gr
       }
     } else if (warp == 5 || warp == 9) {
         // ------------------------------ dz loaders: dZ[T-s] rows of the group -> ring, by TMA ------------------------------
-        // (one thread needs several hundred cycles per stage; two threads take the stages of a step in turn)
+        // (two loader warps take the stages of a step in turn)
         const int ld = warp == 5 ? 0 : 1;
         if (ld < p.n_load) {                                           // warp-uniform loop, an elected lane issues
             int st = ld;

@@ -3,8 +3,8 @@
 // Block j owns 16 hidden units (64 gate columns: i, f, g, o of those units).  Its slice of W_hh
 // (64 columns x H, bf16) is loaded once by TMA and stays in shared memory for all T steps; the
 // running cell state of its units lives in registers.  Each step:
-//   one thread streams bf16(h_{t-1}) [B x H] from the exchange buffer in L2 through a shared memory
-//   ring by TMA (as many k-blocks in flight as the ring holds)  ->  one thread issues tcgen05.mma
+//   loader warps stream bf16(h_{t-1}) [B x H] from the exchange buffer in L2 through a shared memory
+//   ring by TMA (as many k-blocks in flight as the ring holds)  ->  issuer warps run tcgen05.mma
 //   (D[batch row, 64 gate columns] in TMEM)  ->  epilogue warps add the precomputed input projection,
 //   apply the gates, update c, write h_t (fp32 to h_all, bf16 to the exchange buffer)  ->  grid barrier.
 // Batch rows are independent, so the batch is split into groups of rows that run as separate sets of
@@ -39,10 +39,10 @@ constexpr int W_KB = NCOL * BK * 2;              // one k-block of the resident 
 // bytes in flight as it would with zero-padded 128-row stages.
 constexpr int NUM_THREADS = 256;                 // warps 0-3 epilogue, warp 4 W loader + MMA issuer 0, warps 5 and 7 h loaders, warp 6 issuer 1
 constexpr int MAX_ISS = 2;
-// One thread issues a tcgen05.mma only every hundred cycles or so (descriptor arithmetic, barrier polling), slower
-// than the tensor pipe runs an N = 64 one.  With an even number of k-blocks a ring stage therefore holds two of
-// them (one barrier round per stage), each of two issuers takes one into its own accumulator, and the epilogue
-// adds the two accumulators up.
+// Issuing a tcgen05.mma costs the issuing warp tens of cycles even with warp-uniform operands (and about 130 from a
+// single divergent lane), more than the tensor pipe needs for an N = 64 one.  With an even number of k-blocks a ring
+// stage therefore holds two of them (one barrier round per stage), each of two issuer warps takes one into its own
+// accumulator, and the epilogue adds the two accumulators up.
 
 struct Params {
     int T, B, H, n_blocks, k_blocks;
