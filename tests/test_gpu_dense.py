@@ -217,3 +217,19 @@ def test_two_sm_kernel_ragged_edges_and_half_width_tail_units():
     _, odw, odb = oracle.dense_act_grad(xo[:, krows], wo[krows], yo, dyo, act, F64, F64, F64, want_dx=False, dz_dtype=oracle.BF16)
     assert_bf16(dw[krows], odw, what="dw")
     assert_bf16(db, odb, stored_bf16=False, what="db")
+
+
+def test_two_sm_kernel_fixed_unit_scheme_on_a_large_ragged_output():
+    """An output too large for the kernel's unit list (40 row blocks x 129 column chunks): the fixed scheme runs, whole
+    rounds of 256 x 512 units and then 256 x 256 tiles with a split tail.  One sampled row in EVERY 256-row block (all
+    columns), so that a unit that is skipped or computed twice with other data shows."""
+    M, K, N = 10000, 2048, 16392
+    assert B.relay_debug_plan_units(M, N, K, 148) is None
+    t = I.cfg1_tiny_mlp(M, K, N, salt=91)
+    x, b = t["x"].bfloat16(), t["b"].bfloat16()
+    w = (t["w"] / np.sqrt(K)).bfloat16()
+    y = run_fwd(x, w, b, B.ACT_RELU)
+    rng = np.random.default_rng(13)
+    rows = np.unique(np.concatenate([np.arange(0, M, 256) + rng.integers(0, 16, (M + 255) // 256), [255, 256, M - 1]]))
+    want = oracle.dense_act(x[rows].double().numpy(), w.double().numpy(), b.double().numpy(), B.ACT_RELU, F64)
+    assert_bf16(y[rows], want, what="y")
