@@ -353,10 +353,11 @@ lstm_grad_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __gr
                             break;
                         }
                     }
-                    asm volatile("fence.proxy.async.global;" ::: "memory");
                 }
+                __syncwarp();                                           // lane 0's acquire is ordered before the other lanes' accesses
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
+                asm volatile("fence.proxy.async.global;" ::: "memory");   // every lane: whichever lane is elected issues the copies
                 const int row0 = (p.T - s) * p.B + b_lo;
                 for (int kb = ld * N_ISS; kb < p.k_blocks; kb += p.n_load * N_ISS) {
                     ok = __all_sync(0xffffffffu, tc::mbar_wait(&empty[st], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY));

@@ -227,10 +227,11 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
                             break;
                         }
                     }
-                    asm volatile("fence.proxy.async.global;" ::: "memory");
                 }
+                __syncwarp();                                           // lane 0's acquire is ordered before the other lanes' accesses
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
+                asm volatile("fence.proxy.async.global;" ::: "memory");   // every lane: whichever lane is elected issues the copies
                 const CUtensorMap *tm_h = (t & 1) ? &tm_h1 : &tm_h0;
                 for (int kb = ld * p.n_iss; kb < p.k_blocks; kb += p.n_load * p.n_iss) {
                     ok = __all_sync(0xffffffffu, tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY));
