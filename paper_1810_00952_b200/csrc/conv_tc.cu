@@ -966,22 +966,34 @@ relay_status_t launch_conv_fwd_tc(const ConvDims &d, const void *x, bool x_is_nh
     return launch_fprop(d, pl, x_nhwc, (int)d.C, wf, (int)d.O, b, b_dt, act, y, st);
 }
 
+relay_status_t launch_nchw_to_nhwc_bf16(const void *in, void *out, int64_t Nb, int64_t C, int64_t HW, cudaStream_t st)
+{
+    return launch_transpose(false, in, nullptr, out, Nb, C, HW, 0, nullptr, st);
+}
+
 relay_status_t launch_conv_grad_tc(const ConvDims &d, const void *x, const void *w, const void *y, const void *dy, int act, void *dx,
-                                   void *dw, float *db, void *ws, cudaStream_t st)
+                                   void *dw, float *db, void *ws, cudaStream_t st, bool nhwc_in, float *nhwc_partials)
 {
     TcPlan pl = plan(d);
     char *base = (char *)ws;
-    void *x_nhwc = base;
+    const void *x_nhwc = base;
     void *dz_nhwc = base + pl.x_nhwc;
     void *wb = base + pl.x_nhwc + pl.dz_nhwc;
     float *part = (float *)(base + pl.x_nhwc + pl.dz_nhwc + pl.wpack);
     float *db_part = (float *)(base + pl.x_nhwc + pl.dz_nhwc + pl.wpack + pl.part);
     const int64_t HW = d.H * d.W;
-    // dZ = dy (.) act'(y), written straight into NHWC; x into NHWC
-    // (the same pass leaves per-block partial sums of dZ over pixels for the bias gradient)
-    RELAY_TRY(launch_transpose(true, dy, y, dz_nhwc, d.Nb, d.O, HW, act, db ? db_part : nullptr, st));
-    RELAY_TRY(launch_transpose(false, x, nullptr, x_nhwc, d.Nb, d.C, HW, 0, nullptr, st));
-    if (db) RELAY_TRY(launch_colsum_finalize(db_part, (int)(d.Nb * ((HW + 63) / 64)), d.O, 1.0f, db, st));
+    if (nhwc_in) {
+        // x, y, dy are NHWC already: dZ = dy (.) act'(y) is one elementwise pass over [N*H*W, O] whose column sums are db;
+        // x is read where it lies
+        RELAY_TRY(launch_act_grad(RELAY_BF16, dy, y, dz_nhwc, db, nhwc_partials, d.Nb * HW, d.O, act, st));
+        x_nhwc = x;
+    } else {
+        // dZ = dy (.) act'(y), written straight into NHWC; x into NHWC
+        // (the same pass leaves per-block partial sums of dZ over pixels for the bias gradient)
+        RELAY_TRY(launch_transpose(true, dy, y, dz_nhwc, d.Nb, d.O, HW, act, db ? db_part : nullptr, st));
+        RELAY_TRY(launch_transpose(false, x, nullptr, base, d.Nb, d.C, HW, 0, nullptr, st));
+        if (db) RELAY_TRY(launch_colsum_finalize(db_part, (int)(d.Nb * ((HW + 63) / 64)), d.O, 1.0f, db, st));
+    }
     if (dx) {
         RELAY_CUDA(launch_pdl(pack_weights_kernel, dim3((unsigned)((d.O * d.C * 9 + 255) / 256)), dim3(256), 0, st, (const __nv_bfloat16 *)w, (__nv_bfloat16 *)nullptr, (__nv_bfloat16 *)wb, (int)d.O, (int)d.C, 3, 3));
         RELAY_TRY(check_launch("pack_weights"));
