@@ -56,7 +56,7 @@ class ClockSampler:
         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap"
 
     def __init__(self, index: int):
-        self.index, self.rows, self.proc = index, [], None
+        self.index, self.rows, self.proc, self.t0 = index, [], None, None
 
     def start(self):
         try:
@@ -69,7 +69,12 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
+            self.rows.append((time.monotonic(), [c.strip() for c in line.split(",")]))
+
+    def begin(self):
+        """Marks the start of the timed region: only samples that arrive from here on are reported (the tool is
+        started earlier, during the warm-up, because it needs a few hundred milliseconds to deliver its first row)."""
+        self.t0 = time.monotonic()
 
     def stop(self):
         if not self.proc:
@@ -80,7 +85,8 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
         sm, mx, reasons = [], None, set()
-        for r in self.rows:
+        rows = [r for t, r in self.rows if self.t0 is None or t >= self.t0]
+        for r in rows:
             try:
                 sm.append(float(r[0])); mx = float(r[1])
             except Exception:
@@ -195,6 +201,15 @@ class Workload:
             ps_ = (shp[0], shp[1], shp[2] // 2, shp[3] // 2)
             self.pool_y, self.pool_idx = E(*ps_), E(*ps_, dt=torch.int32)
             self.pool_dy, self.pool_dx = I.normal(8, 1, ps_, 1.0, torch.bfloat16).to(dev), torch.empty_like(self.pool_x)
+            # the conv configuration's tensors tagged NHWC (device-resident, permuted once): the layout-tagged calls
+            c4 = self.devt["cfg4"] if "cfg4" in groups else {k: v.to(dev) for k, v in
+                                                             I.cfg4_conv(*((2, 32, 14, 14, 32) if small else (32, 256, 56, 56, 256))).items()}
+            nhwc = lambda a: a.permute(0, 2, 3, 1).contiguous()
+            self.nhwc = dict(x=nhwc(c4["x"]), dy=nhwc(c4["dy"]), w=c4["w"], b=c4["b"])
+            self.nhwc.update(y=torch.empty_like(self.nhwc["dy"]), dx=torch.empty_like(self.nhwc["x"]), dw=torch.empty_like(c4["w"]),
+                             db=E(c4["w"].shape[0], dt=f32))
+            ws_bytes = max(ws_bytes, B.relay_workspace_bytes_conv2d_act(self.nhwc["x"], c4["w"], 1, 1, layout=B.NHWC),
+                           B.relay_workspace_bytes_conv2d_act_grad(self.nhwc["x"], c4["w"], 1, 1, layout=B.NHWC))
         self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
         self.flush_buf = torch.zeros(1024 * 1024 * 1024, dtype=torch.uint8, device=dev)
         self.pinned_out = {g: {k: torch.empty_like(v, device="cpu").pin_memory() for k, v in o.items()} for g, o in self.out.items()}
@@ -288,6 +303,12 @@ class Workload:
             self.flush_l2()
             with tm.region("next.pool_grad"):
                 B.relay_max_pool2d_grad(self.pool_idx, self.pool_dy, 2, 2, 2, 2, self.pool_dx)
+            h = self.nhwc
+            self.flush_l2()
+            with tm.region("next.conv_nhwc"):
+                B.relay_fused_conv2d_act(h["x"], h["w"], h["b"], 1, 1, B.ACT_RELU, h["y"], ws, layout=B.NHWC)
+            with tm.region("next.conv_nhwc_grad"):
+                B.relay_fused_conv2d_act_grad(h["x"], h["w"], h["y"], h["dy"], 1, 1, B.ACT_RELU, h["dx"], h["dw"], h["db"], ws, layout=B.NHWC)
 
     # -- algorithmic work per step -------------------------------------------------------------------------
     def work(self):
@@ -320,6 +341,9 @@ class Workload:
             w["next.sgd"] = dict(bytes=sum(3 * p.numel() * 2 for p in self.sgd_params))
             pool_bytes = self.pool_x.numel() * 2 + self.pool_y.numel() * (2 + 4)
             w["next.pool"] = dict(bytes=pool_bytes); w["next.pool_grad"] = dict(bytes=pool_bytes)
+            n, h, wd, c = self.nhwc["x"].shape
+            f = 2 * n * h * wd * self.nhwc["w"].shape[0] * c * 9
+            w["next.conv_nhwc"] = dict(flop=f); w["next.conv_nhwc_grad"] = dict(flop=2 * f)
         return w
 
 
@@ -421,13 +445,14 @@ def main():
         torch.cuda.synchronize()
 
     tm = Timer()
+    sampler = ClockSampler(local); sampler.start()
     for _ in range(args.warmup):
         wl.step(tm)
     tm.collect(); tm.ms = {}
     B.relay_poll_status()
 
-    sampler = ClockSampler(local); sampler.start()
     barrier()
+    sampler.begin()
     n0 = B.relay_launch_count()
     t_all0 = torch.cuda.Event(enable_timing=True); t_all1 = torch.cuda.Event(enable_timing=True)
     t_all0.record()

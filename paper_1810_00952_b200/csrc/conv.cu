@@ -112,8 +112,8 @@ extern "C" relay_status_t relay_fused_conv2d_act(const relay_tensor_t *x, const 
     char *base = (char *)ws;
     void *y_nchw = base;
     if (tc) {
-        RELAY_TRY(launch_conv_fwd_tc(d, x->data, true, w->data, bp, b_dt, act, y_nchw, base + y_bytes(d), st));
-        return launch_nchw_to_nhwc_bf16(y_nchw, y->data, d.Nb, d.O, d.P * d.Q, st);
+        // the tensor-core instance reads NHWC itself and, in its two-SM form, stores NHWC tiles
+        return launch_conv_fwd_tc(d, x->data, true, w->data, bp, b_dt, act, y_nchw, base + y_bytes(d), st, y->data);
     } else {
         void *x_nchw = base + y_bytes(d);
         RELAY_TRY(launch_layout_change(d.dt, x->data, x_nchw, d.Nb, d.H * d.W, d.C, st));
@@ -174,15 +174,14 @@ extern "C" relay_status_t relay_fused_conv2d_act_grad(const relay_tensor_t *x, c
     void *dxp = dx ? dx->data : nullptr;
     char *inner = (char *)ws;
     if (d.nhwc && conv_tc_eligible(d)) {
-        // the tensor-core instance works on NHWC itself: no copies of x, y, dy; only dx comes back through a layout change
+        // the tensor-core instance works on NHWC itself: no copies of x, y, dy; dx passes through an NCHW temporary only
+        // where the one-SM kernel computes it
         char *base = (char *)ws;
         void *dx_nchw = base + x_bytes(d);
         float *partials = (float *)(base + 2 * x_bytes(d));            // at most N*H*W*O/8 bytes: fits the y-sized region
         inner = base + 2 * x_bytes(d) + 2 * y_bytes(d);
-        RELAY_TRY(launch_conv_grad_tc(d, x->data, w->data, y->data, dy->data, act, dx ? dx_nchw : nullptr, dw->data,
-                                      db ? (float *)db->data : nullptr, inner, st, true, partials));
-        if (dx) RELAY_TRY(launch_nchw_to_nhwc_bf16(dx_nchw, dx->data, d.Nb, d.C, d.H * d.W, st));
-        return RELAY_OK;
+        return launch_conv_grad_tc(d, x->data, w->data, y->data, dy->data, act, dx ? dx_nchw : nullptr, dw->data,
+                                   db ? (float *)db->data : nullptr, inner, st, true, partials, dx ? dx->data : nullptr);
     }
     if (d.nhwc) {
         char *base = (char *)ws;

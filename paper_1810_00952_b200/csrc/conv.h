@@ -26,14 +26,14 @@ bool conv_tc_eligible(const ConvDims &d);
 size_t conv_tc_fwd_workspace(const ConvDims &d);
 size_t conv_tc_grad_workspace(const ConvDims &d);
 // `x_is_nhwc`: x is already in the kernel's own activation layout, the repack pass is skipped (y is NCHW either way)
+// `y_nhwc` (optional): the result is wanted as [Nb][H][W][O]; `y` is then an NCHW temporary that the call may or may not use
 relay_status_t launch_conv_fwd_tc(const ConvDims &d, const void *x, bool x_is_nhwc, const void *w, const void *b, int32_t b_dt, int act,
-                                  void *y, void *ws, cudaStream_t st);
+                                  void *y, void *ws, cudaStream_t st, void *y_nhwc = nullptr);
 // whole gradient group: dZ = dy (.) act'(y) (kept in NHWC), db, dx (if wanted), dw
-// `nhwc_in`: x, y, dy are NHWC already (no repack passes; `nhwc_partials` holds the column-sum partials of db);
-// dx is written NCHW either way
+// `nhwc_in`: x, y, dy are NHWC already (no repack passes; `nhwc_partials` holds the column-sum partials of db) and the
+// input gradient is wanted in `dx_nhwc`; `dx` is then an NCHW temporary that the call may or may not use
 relay_status_t launch_conv_grad_tc(const ConvDims &d, const void *x, const void *w, const void *y, const void *dy, int act, void *dx,
-                                   void *dw, float *db, void *ws, cudaStream_t st, bool nhwc_in = false, float *nhwc_partials = nullptr);
-// vectorised layout change of a bf16 NCHW tensor (C and H*W multiples of 8) to NHWC
-relay_status_t launch_nchw_to_nhwc_bf16(const void *in, void *out, int64_t Nb, int64_t C, int64_t HW, cudaStream_t st);
+                                   void *dw, float *db, void *ws, cudaStream_t st, bool nhwc_in = false, float *nhwc_partials = nullptr,
+                                   void *dx_nhwc = nullptr);
 
 }  // namespace relay

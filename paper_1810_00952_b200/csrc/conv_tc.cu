@@ -154,6 +154,7 @@ struct FpropParams {
     int n_pairs, pairs_per_ntile, n_items;   // items [0, n_pairs) are pairs, the rest singles (MH = 2); MH = 1: all singles
     const void *bias;           // per output channel, or null
     int bias_bf16, act;
+    int out_nhwc;               // two-SM kernel: the output tensor map is [Nb*H*W pixels][Cout], tiles are stored pixel-major
     int *err;
 };
 
@@ -501,15 +502,25 @@ conv_fprop_tc2_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
                 __syncwarp();
                 // 32 rows x 64 bytes in the 64-byte swizzle pattern of the output tensor map (16-byte piece q of row r at
                 // piece q ^ ((r >> 1) & 3)): conflict-free stores
+                if (p.out_nhwc) {
+                    // pixel-major block: row j = pixel j, this lane's channel is element `lane` of the row (the 32 lanes of
+                    // a store fill one 64-byte row, so the 2-byte stores are conflict-free as well)
+                    uint8_t *col = st + ((lane & 7) << 1);
 #pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    *reinterpret_cast<uint4 *>(st + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4)) =
-                        make_uint4(pack2(v[8 * q], v[8 * q + 1]), pack2(v[8 * q + 2], v[8 * q + 3]), pack2(v[8 * q + 4], v[8 * q + 5]),
-                                   pack2(v[8 * q + 6], v[8 * q + 7]));
+                    for (int j = 0; j < 32; ++j)
+                        *reinterpret_cast<__nv_bfloat16 *>(col + j * 64 + (((lane >> 3) ^ ((j >> 1) & 3)) << 4)) = __float2bfloat16_rn(v[j]);
+                } else {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        *reinterpret_cast<uint4 *>(st + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4)) =
+                            make_uint4(pack2(v[8 * q], v[8 * q + 1]), pack2(v[8 * q + 2], v[8 * q + 3]), pack2(v[8 * q + 4], v[8 * q + 5]),
+                                       pack2(v[8 * q + 6], v[8 * q + 7]));
+                }
                 tc::fence_proxy_async();
                 __syncwarp();
                 if (tc::elect_one()) {
-                    tc::tma_store_2d(&tm_y, st, h0 * p.W + c * 32, img * p.Cout + o0);
+                    if (p.out_nhwc) tc::tma_store_2d(&tm_y, st, o0, (img * p.H + h0) * p.W + c * 32);
+                    else tc::tma_store_2d(&tm_y, st, h0 * p.W + c * 32, img * p.Cout + o0);
                     tc::tma_store_commit();
                 }
             }
@@ -845,17 +856,31 @@ TcPlan plan(const ConvDims &d)
     return pl;
 }
 
+// the two-SM form takes every tile as a pair of blocks; it is the form that can also store pixel-major (NHWC) tiles
+bool fprop_pair_form(const ConvDims &d, const TcPlan &pl, int Cout, int sms)
+{
+    const int nt = pl.rows_per_tile * (int)d.W;
+    return Cout % 256 == 0 && pl.rows_per_tile % 2 == 0 && ((nt / 2) * 128) % 1024 == 0 && sms >= 2 &&
+           (int64_t)d.Nb * (d.H / pl.rows_per_tile) * (Cout / 256) >= sms / 2;
+}
+
+int sm_count()
+{
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 148;
+    return sms;
+}
+
+// `out_nhwc` (only where fprop_pair_form holds): `out` is [Nb][H][W][Cout] instead of [Nb][Cout][H][W]
 relay_status_t launch_fprop(const ConvDims &d, const TcPlan &pl, const void *act_nhwc, int Cin, const void *wpacked, int Cout,
-                            const void *bias, int32_t b_dt, int act, void *out_nchw, cudaStream_t st)
+                            const void *bias, int32_t b_dt, int act, void *out_nchw, cudaStream_t st, bool out_nhwc = false)
 {
     CUtensorMap tm_w, tm_x, tm_y;
     RELAY_TRY(make_tmap_2d_bf16(&tm_w, wpacked, (uint64_t)9 * Cin, Cout, (uint64_t)9 * Cin, BK, BM));
     RELAY_TRY(make_tmap_nhwc_bf16(&tm_x, act_nhwc, Cin, d.W, d.H, d.Nb, BK, (uint32_t)d.W, pl.rows_per_tile));
     // output NCHW as [Nb * Cout rows][H * W columns]; 32 x 32 boxes, rows of 64 bytes, no swizzle
     RELAY_TRY(make_tmap_2d(&tm_y, false, out_nchw, (uint64_t)(d.H * d.W), (uint64_t)d.Nb * Cout, (uint64_t)(d.H * d.W), 32, 32, false));
-    int dev = 0, sms = 148;
-    RELAY_CUDA(cudaGetDevice(&dev));
-    RELAY_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const int sms = sm_count();
     FpropParams p{};
     p.Cin = Cin; p.Cout = Cout; p.H = (int)d.H; p.W = (int)d.W; p.Nb = (int)d.Nb; p.taps_r = 3; p.taps_s = 3; p.pad = 1;
     p.rows_per_tile = pl.rows_per_tile; p.nt = pl.rows_per_tile * (int)d.W;
@@ -865,12 +890,14 @@ relay_status_t launch_fprop(const ConvDims &d, const TcPlan &pl, const void *act
     p.err = device_error_word();
     if (!p.err) return fail(RELAY_ERR_CUDA, "no device error word");
     // two-SM form: every tile is computed by a pair of blocks, each loading half of the activation tile
-    if (Cout % 256 == 0 && pl.rows_per_tile % 2 == 0 && ((p.nt / 2) * 128) % 1024 == 0 && sms >= 2 &&
-        (int64_t)p.n_tiles_total * (Cout / 256) >= sms / 2) {
+    if (out_nhwc && !fprop_pair_form(d, pl, Cout, sms)) return fail(RELAY_ERR_UNSUPPORTED, "conv2d: no pixel-major store in the one-SM kernel");
+    if (fprop_pair_form(d, pl, Cout, sms)) {
         CUtensorMap tm_xh, tm_y2;
         RELAY_TRY(make_tmap_nhwc_bf16(&tm_xh, act_nhwc, Cin, d.W, d.H, d.Nb, BK, (uint32_t)d.W, pl.rows_per_tile / 2));
-        // output boxes of 32 channels x 32 pixels, rows of 64 bytes in the 64-byte swizzle pattern
-        RELAY_TRY(make_tmap_2d_sw64(&tm_y2, false, out_nchw, (uint64_t)(d.H * d.W), (uint64_t)d.Nb * Cout, (uint64_t)(d.H * d.W), 32));
+        // output boxes of 32 channels x 32 pixels (NHWC: 32 pixels x 32 channels), rows of 64 bytes in the 64-byte swizzle pattern
+        if (out_nhwc) RELAY_TRY(make_tmap_2d_sw64(&tm_y2, false, out_nchw, (uint64_t)Cout, (uint64_t)(d.Nb * d.H * d.W), (uint64_t)Cout, 32));
+        else RELAY_TRY(make_tmap_2d_sw64(&tm_y2, false, out_nchw, (uint64_t)(d.H * d.W), (uint64_t)d.Nb * Cout, (uint64_t)(d.H * d.W), 32));
+        p.out_nhwc = out_nhwc ? 1 : 0;
         const size_t stage2 = (size_t)BM * BK * 2 + (size_t)(p.nt / 2) * 128;
         p.stages = (int)std::min<size_t>(8, (kSmemLimit - 1024 - 4 * 4096) / stage2);
         p.pairs_per_ntile = Cout / 256;
@@ -951,7 +978,7 @@ size_t conv_tc_grad_workspace(const ConvDims &d)
 }
 
 relay_status_t launch_conv_fwd_tc(const ConvDims &d, const void *x, bool x_is_nhwc, const void *w, const void *b, int32_t b_dt, int act,
-                                  void *y, void *ws, cudaStream_t st)
+                                  void *y, void *ws, cudaStream_t st, void *y_nhwc)
 {
     TcPlan pl = plan(d);
     char *base = (char *)ws;
@@ -963,16 +990,14 @@ relay_status_t launch_conv_fwd_tc(const ConvDims &d, const void *x, bool x_is_nh
     }
     RELAY_CUDA(launch_pdl(pack_weights_kernel, dim3((unsigned)((d.O * d.C * 9 + 255) / 256)), dim3(256), 0, st, (const __nv_bfloat16 *)w, (__nv_bfloat16 *)wf, (__nv_bfloat16 *)nullptr, (int)d.O, (int)d.C, 3, 3));
     RELAY_TRY(check_launch("pack_weights"));
-    return launch_fprop(d, pl, x_nhwc, (int)d.C, wf, (int)d.O, b, b_dt, act, y, st);
-}
-
-relay_status_t launch_nchw_to_nhwc_bf16(const void *in, void *out, int64_t Nb, int64_t C, int64_t HW, cudaStream_t st)
-{
-    return launch_transpose(false, in, nullptr, out, Nb, C, HW, 0, nullptr, st);
+    if (!y_nhwc) return launch_fprop(d, pl, x_nhwc, (int)d.C, wf, (int)d.O, b, b_dt, act, y, st);
+    if (fprop_pair_form(d, pl, (int)d.O, sm_count())) return launch_fprop(d, pl, x_nhwc, (int)d.C, wf, (int)d.O, b, b_dt, act, y_nhwc, st, true);
+    RELAY_TRY(launch_fprop(d, pl, x_nhwc, (int)d.C, wf, (int)d.O, b, b_dt, act, y, st));
+    return launch_transpose(false, y, nullptr, y_nhwc, d.Nb, d.O, d.H * d.W, 0, nullptr, st);
 }
 
 relay_status_t launch_conv_grad_tc(const ConvDims &d, const void *x, const void *w, const void *y, const void *dy, int act, void *dx,
-                                   void *dw, float *db, void *ws, cudaStream_t st, bool nhwc_in, float *nhwc_partials)
+                                   void *dw, float *db, void *ws, cudaStream_t st, bool nhwc_in, float *nhwc_partials, void *dx_nhwc)
 {
     TcPlan pl = plan(d);
     char *base = (char *)ws;
@@ -997,7 +1022,12 @@ relay_status_t launch_conv_grad_tc(const ConvDims &d, const void *x, const void 
     if (dx) {
         RELAY_CUDA(launch_pdl(pack_weights_kernel, dim3((unsigned)((d.O * d.C * 9 + 255) / 256)), dim3(256), 0, st, (const __nv_bfloat16 *)w, (__nv_bfloat16 *)nullptr, (__nv_bfloat16 *)wb, (int)d.O, (int)d.C, 3, 3));
         RELAY_TRY(check_launch("pack_weights"));
-        RELAY_TRY(launch_fprop(d, pl, dz_nhwc, (int)d.O, wb, (int)d.C, nullptr, RELAY_F32, RELAY_ACT_NONE, dx, st));
+        if (dx_nhwc && fprop_pair_form(d, pl, (int)d.C, sm_count())) {
+            RELAY_TRY(launch_fprop(d, pl, dz_nhwc, (int)d.O, wb, (int)d.C, nullptr, RELAY_F32, RELAY_ACT_NONE, dx_nhwc, st, true));
+        } else {
+            RELAY_TRY(launch_fprop(d, pl, dz_nhwc, (int)d.O, wb, (int)d.C, nullptr, RELAY_F32, RELAY_ACT_NONE, dx, st));
+            if (dx_nhwc) RELAY_TRY(launch_transpose(false, dx, nullptr, dx_nhwc, d.Nb, d.C, HW, 0, nullptr, st));
+        }
     }
     CUtensorMap tm_dz, tm_x;
     RELAY_TRY(make_tmap_nhwc_bf16(&tm_dz, dz_nhwc, d.O, d.W, d.H, d.Nb, 64, (uint32_t)d.W, pl.rows_per_kblock));

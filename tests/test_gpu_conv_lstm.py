@@ -79,7 +79,10 @@ def test_conv_reduced_config_bf16_3x3(N, C, H, W, O):
 
 @pytest.mark.parametrize("N,C,H,W,O,R,stride,pad,tdt", [(2, 3, 7, 6, 4, 3, 1, 1, torch.float32), (1, 5, 9, 9, 3, 3, 2, 1, torch.bfloat16),
                                                          (2, 128, 16, 16, 128, 3, 1, 1, torch.bfloat16),      # tensor-core instance
-                                                         (3, 128, 12, 24, 256, 3, 1, 1, torch.bfloat16)])
+                                                         (3, 128, 12, 24, 256, 3, 1, 1, torch.bfloat16),
+                                                         # two-SM kernel storing NHWC tiles itself: 3 and 1 blocks of 32 pixels
+                                                         (76, 256, 12, 8, 256, 3, 1, 1, torch.bfloat16),
+                                                         (80, 256, 4, 8, 256, 3, 1, 1, torch.bfloat16)])
 def test_conv_nhwc_tagged_activations(N, C, H, W, O, R, stride, pad, tdt):
     """Layout-tagged activations: x, y, dy, dx are NHWC tensors of shape (N,H,W,C); the values are those of the NCHW
     definition (the oracle is given the same tensors permuted on the host)."""
@@ -152,6 +155,23 @@ def test_conv_full_size_sampled():
                                          B.ACT_RELU, F64, F64, F64, want_dx=False)
     assert_bf16(dw[oc, ic], odw, what="dw")
     assert_bf16(db[oc], odb, stored_bf16=False, what="db")
+    # the same tensors tagged NHWC: the kernels store pixel-major tiles of the same accumulators, so y, dx and dw agree
+    # bit for bit with the NCHW call; db is summed in another order
+    nhwc = lambda a: a.permute(0, 2, 3, 1).contiguous().to(DEV)
+    xh, dyh = nhwc(t["x"]), nhwc(t["dy"])
+    wd, bd = t["w"].to(DEV), t["b"].to(DEV)
+    yh = Guarded(tuple(dyh.shape), torch.bfloat16, DEV)
+    B.relay_fused_conv2d_act(xh, wd, bd, 1, 1, B.ACT_RELU, yh.t, workspace(B.relay_workspace_bytes_conv2d_act(xh, wd, 1, 1, layout=B.NHWC), DEV),
+                             layout=B.NHWC)
+    torch.cuda.synchronize()
+    assert torch.equal(yh.check().permute(0, 3, 1, 2), y)
+    dxh, dwh, dbh = Guarded(tuple(xh.shape), torch.bfloat16, DEV), Guarded(tuple(wd.shape), torch.bfloat16, DEV), Guarded((wd.shape[0],), torch.float32, DEV)
+    B.relay_fused_conv2d_act_grad(xh, wd, yh.t, dyh, 1, 1, B.ACT_RELU, dxh.t, dwh.t, dbh.t,
+                                  workspace(B.relay_workspace_bytes_conv2d_act_grad(xh, wd, 1, 1, layout=B.NHWC), DEV), layout=B.NHWC)
+    torch.cuda.synchronize()
+    B.relay_poll_status()
+    assert torch.equal(dxh.check().permute(0, 3, 1, 2), dx) and torch.equal(dwh.check(), dw)
+    assert_bf16(dbh.check()[oc], odb, stored_bf16=False, what="db nhwc")
 
 
 # ---- LSTM -------------------------------------------------------------------------------------------
