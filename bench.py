@@ -232,6 +232,14 @@ class Workload:
                 n += v.numel() * v.element_size()
         return n
 
+    def make_alternate(self):
+        """Second set of device input and result buffers for the pipelined end-to-end loop."""
+        self.alt = ({g: {k: torch.empty_like(v) for k, v in d.items()} for g, d in self.devt.items()},
+                    {g: {k: torch.empty_like(v) for k, v in o.items()} for g, o in self.out.items()})
+
+    def swap(self):
+        (self.devt, self.out), self.alt = self.alt, (self.devt, self.out)
+
     def flush_l2(self):
         # 1 GiB read (a max-reduction): evicts the 126 MB L2 with CLEAN lines, so no write-back of the
         # flush itself overlaps the timed kernels, and keeps the GPU busy while the host queues the group
@@ -546,39 +554,52 @@ def main():
     # end to end: pinned host inputs -> device, the step, results -> pinned host, all inside the timed region
     e2e = None
     if not args.no_e2e:
-        # Every step uploads its inputs from pinned host memory and reads all of its results back.  The read-back of
-        # step i runs on a second stream and overlaps the upload of step i+1 (opposite directions of the link); the
-        # compute of step i+1 waits for it, since it overwrites the buffers being read.
+        # Every step uploads its inputs from pinned host memory and reads all of its results back.  Three streams and two
+        # sets of device buffers: while step i computes, the inputs of step i+1 upload into the other set and the results
+        # of step i-1 are read back from it (the two directions of the link run concurrently).  A set's inputs are not
+        # overwritten before the compute that read them has ended, nor its results before their read-back has.
         tm2 = Timer()
         h2d = d2h = 0
         main_s = torch.cuda.current_stream()
-        d2h_s = torch.cuda.Stream()
+        up_s, d2h_s = torch.cuda.Stream(), torch.cuda.Stream()
+        wl.make_alternate()
+        comp_done, dl_done = [None, None], [None, None]
 
-        def e2e_step(prev_done):
+        def e2e_step(i):
             nonlocal h2d, d2h
-            h2d = wl.upload()
-            if prev_done is not None:
-                main_s.wait_event(prev_done)
+            k = i & 1
+            wl.swap()
+            with torch.cuda.stream(up_s):
+                if comp_done[k] is not None:
+                    up_s.wait_event(comp_done[k])
+                h2d = wl.upload()
+                up_done = torch.cuda.Event(); up_done.record(up_s)
+            main_s.wait_event(up_done)
+            if dl_done[k] is not None:
+                main_s.wait_event(dl_done[k])
             wl.step(tm2)
-            computed = torch.cuda.Event(); computed.record(main_s)
+            comp_done[k] = torch.cuda.Event(); comp_done[k].record(main_s)
             with torch.cuda.stream(d2h_s):
-                d2h_s.wait_event(computed)
+                d2h_s.wait_event(comp_done[k])
                 d2h = wl.download()
-                done = torch.cuda.Event(); done.record(d2h_s)
-            return done
+                dl_done[k] = torch.cuda.Event(); dl_done[k].record(d2h_s)
 
-        done = None
-        for _ in range(2):
-            done = e2e_step(done)
-        main_s.wait_event(done)
+        def drain():
+            for e in dl_done:
+                if e is not None:
+                    main_s.wait_event(e)
+
+        for i in range(2):
+            e2e_step(i)
+        drain()
         barrier()
         a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
-        n_e2e = max(2, min(args.steps, 5))
+        n_e2e = 2 * max(1, min(args.steps, 20) // 2)
         a.record()
-        done = None
-        for _ in range(n_e2e):
-            done = e2e_step(done)
-        main_s.wait_event(done)
+        up_s.wait_event(a)
+        for i in range(n_e2e):
+            e2e_step(i)
+        drain()
         b.record()
         barrier()
         e_ms = max_over_ranks(a.elapsed_time(b) / n_e2e, dist, dev)
@@ -586,7 +607,8 @@ def main():
         e2e = {"value": world * flop_all / (e_ms * 1e-3) / 1e12 if flop_all else None, "unit": "TFLOP/s", "ms_per_step": e_ms,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "note": "whole step incl. L2 flushes and all groups, inputs uploaded and all results read back every step "
-                       "(read-back of a step overlaps the next step's upload); dense+conv FLOPs over that time"}
+                       "(pipelined over two buffer sets: upload of the next step and read-back of the previous one overlap the compute); "
+                       "dense+conv FLOPs over that time"}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
