@@ -1,5 +1,6 @@
 // Direct conv2d kernels (SIMT): one result element per thread, fp32 accumulation in a fixed
-// loop order.  They take every stride / padding / window size and both float types, and are
+// loop order.  The fp32 instances sum short runs (one window, or 16 terms) in fp32 and add the run
+// sums in fp64, so the rounding error does not grow with the number of terms.  They take every stride / padding / window size and both float types, and are
 // the path for instances the implicit-GEMM tensor-core kernels do not cover.
 #include "conv.h"
 #include "ewise_kernels.cuh"
@@ -17,6 +18,8 @@ template <typename T> __device__ __forceinline__ void stf(T *p, int64_t i, float
     else p[i] = v;
 }
 
+template <typename T> constexpr bool kWideSum = sizeof(T) == 4;
+
 template <typename T, bool FAST>
 __global__ void __launch_bounds__(256) conv_fwd_direct_kernel(const ConvDims d, const T *__restrict__ x, const T *__restrict__ w,
                                                                const void *__restrict__ b, int b_dt, int act, T *__restrict__ y)
@@ -27,7 +30,8 @@ __global__ void __launch_bounds__(256) conv_fwd_direct_kernel(const ConvDims d, 
         int64_t p = t % d.P; t /= d.P;
         int64_t o = t % d.O, n = t / d.O;
         float acc = 0.0f;
-        for (int64_t c = 0; c < d.C; ++c)
+        double wide = 0.0;
+        for (int64_t c = 0; c < d.C; ++c) {
             for (int64_t r = 0; r < d.R; ++r) {
                 int64_t i = p * d.stride - d.pad + r;
                 if (i < 0 || i >= d.H) continue;
@@ -37,6 +41,9 @@ __global__ void __launch_bounds__(256) conv_fwd_direct_kernel(const ConvDims d, 
                     acc = fmaf(ldf(x, ((n * d.C + c) * d.H + i) * d.W + j), ldf(w, ((o * d.C + c) * d.R + r) * d.S + s), acc);
                 }
             }
+            if constexpr (kWideSum<T>) { wide += (double)acc; acc = 0.0f; }
+        }
+        if constexpr (kWideSum<T>) acc = (float)wide;
         if (b) acc += b_dt == RELAY_BF16 ? __bfloat162float(((const __nv_bfloat16 *)b)[o]) : ((const float *)b)[o];
         stf(y, lin, act_fwd<FAST>(acc, act));
     }
@@ -52,7 +59,8 @@ __global__ void __launch_bounds__(256) conv_dx_direct_kernel(const ConvDims d, c
         int64_t i = t % d.H; t /= d.H;
         int64_t c = t % d.C, n = t / d.C;
         float acc = 0.0f;
-        for (int64_t o = 0; o < d.O; ++o)
+        double wide = 0.0;
+        for (int64_t o = 0; o < d.O; ++o) {
             for (int64_t r = 0; r < d.R; ++r) {
                 int64_t pn = i + d.pad - r;
                 if (pn < 0 || pn % d.stride) continue;
@@ -66,6 +74,9 @@ __global__ void __launch_bounds__(256) conv_dx_direct_kernel(const ConvDims d, c
                     acc = fmaf(ldf(dz, ((n * d.O + o) * d.P + p) * d.Q + q), ldf(w, ((o * d.C + c) * d.R + r) * d.S + s), acc);
                 }
             }
+            if constexpr (kWideSum<T>) { wide += (double)acc; acc = 0.0f; }
+        }
+        if constexpr (kWideSum<T>) acc = (float)wide;
         stf(dx, lin, acc);
     }
 }
@@ -84,15 +95,25 @@ __global__ void __launch_bounds__(256) conv_dw_direct_kernel(const ConvDims d, c
     int64_t c = t % d.C, o = t / d.C;
     const int64_t npq = d.Nb * d.P * d.Q;
     float acc = 0.0f;
+    double wide = 0.0;
+    int run = 0;
     for (int64_t l = lane; l < npq; l += 32) {
         int64_t q = l % d.Q, u = l / d.Q;
         int64_t p = u % d.P, n = u / d.P;
         int64_t i = p * d.stride - d.pad + r, j = q * d.stride - d.pad + s;
         if (i < 0 || i >= d.H || j < 0 || j >= d.W) continue;
         acc = fmaf(ldf(dz, ((n * d.O + o) * d.P + p) * d.Q + q), ldf(x, ((n * d.C + c) * d.H + i) * d.W + j), acc);
+        if constexpr (kWideSum<T>) if (++run == 16) { wide += (double)acc; acc = 0.0f; run = 0; }
     }
+    if constexpr (kWideSum<T>) {
+        wide += (double)acc;
 #pragma unroll
-    for (int k = 16; k > 0; k >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, k);
+        for (int k = 16; k > 0; k >>= 1) wide += __shfl_xor_sync(0xffffffffu, wide, k);
+        acc = (float)wide;
+    } else {
+#pragma unroll
+        for (int k = 16; k > 0; k >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, k);
+    }
     if (lane == 0) stf(dw, e, acc);
 }
 

@@ -1,7 +1,10 @@
 // SIMT contraction kernel, sums in k order.  It is the fp32 path of the dense groups (tensor cores
 // would round the operands to tf32) and the path for shapes the tensor-core kernel does not take.
-// fp32 operands are accumulated in fp64 and rounded once on the store, so that results that suffer
-// cancellation still meet the fp32 tolerance; bf16 operands are accumulated in fp32.
+// fp32 operands: runs of 16 products are summed in fp32 (exact products, one rounding per
+// fused multiply-add, on a partial sum that stays small) and the run sums are added in fp64 and
+// rounded once on the store.  The rounding error is then about 1e-7 of the output's RMS whatever K is,
+// so outputs that suffer cancellation still meet the fp32 tolerance, while the fp64 pipe (1/16 of the
+// fp32 rate) sees one addition per 16 products.  bf16 operands are accumulated in fp32.
 #include <type_traits>
 
 #include "ewise_kernels.cuh"
@@ -9,58 +12,97 @@
 
 namespace relay {
 
-constexpr int BM = 64, BN = 64, BK = 16;
+constexpr int BN = 64, BK = 32, KSUB = 16;
 
 template <typename T> __device__ __forceinline__ float to_f(T v);
 template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
 
-template <typename TIN, typename TOUT, bool FAST>
-__global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmDesc g)
+// block tile (16 * TM) x 64, thread tile TM x 4: TM = 4 in general, TM = 1 for outputs of at most 16 rows
+// (all 256 threads then hold live outputs instead of one warp's worth).  The loads of k-block i+1 are issued
+// into registers before the arithmetic of k-block i, all of a thread's loads back to back, so that one
+// memory round trip per k-block is exposed at most.
+template <typename TIN, typename TOUT, bool FAST, int TM>
+__global__ void __launch_bounds__(256, 2) gemm_simt_kernel(const GemmDesc g)
 {
+    constexpr int BM = 16 * TM;
+    constexpr int A_LD = BM * BK / 256, B_LD = BN * BK / 256;
     __shared__ float As[BK][BM + 1];
     __shared__ float Bs[BK][BN + 1];
     const TIN *A = (const TIN *)g.a;
     const TIN *B = (const TIN *)g.b;
     const int tid = threadIdx.x;
     const int64_t m0 = (int64_t)blockIdx.x * BM, n0 = (int64_t)blockIdx.y * BN;
-    const int tm = (tid / 16) * 4, tn = (tid % 16) * 4;
-    using Acc = typename std::conditional<sizeof(TIN) == 4, double, float>::type;
-    Acc acc[4][4] = {};
+    const int tm = (tid / 16) * TM, tn = (tid % 16) * 4;
+    constexpr bool F64 = sizeof(TIN) == 4;
+    using Acc = typename std::conditional<F64, double, float>::type;
+    Acc acc[TM][4] = {};
     // loader index order follows the unit stride of each operand so that loads coalesce
     const bool a_k_fast = g.a_sk == 1, b_n_fast = g.b_sn == 1;
-    for (int64_t k0 = 0; k0 < g.K; k0 += BK) {
-        for (int e = tid; e < BM * BK; e += 256) {
-            int mm = a_k_fast ? e / BK : e % BM, kk = a_k_fast ? e % BK : e / BM;
-            int64_t m = m0 + mm, k = k0 + kk;
-            As[kk][mm] = (m < g.M && k < g.K) ? to_f<TIN>(A[m * g.a_sm + k * g.a_sk]) : 0.0f;
+    float ra[A_LD], rb[B_LD];
+    auto load_tiles = [&](int64_t k0) {
+#pragma unroll
+        for (int i = 0; i < A_LD; ++i) {
+            const int e = tid + i * 256;
+            const int mm = a_k_fast ? e / BK : e % BM, kk = a_k_fast ? e % BK : e / BM;
+            const int64_t m = m0 + mm, k = k0 + kk;
+            ra[i] = (m < g.M && k < g.K) ? to_f<TIN>(A[m * g.a_sm + k * g.a_sk]) : 0.0f;
         }
-        for (int e = tid; e < BN * BK; e += 256) {
-            int nn = b_n_fast ? e % BN : e / BK, kk = b_n_fast ? e / BN : e % BK;
-            int64_t n = n0 + nn, k = k0 + kk;
-            Bs[kk][nn] = (n < g.N && k < g.K) ? to_f<TIN>(B[k * g.b_sk + n * g.b_sn]) : 0.0f;
+#pragma unroll
+        for (int i = 0; i < B_LD; ++i) {
+            const int e = tid + i * 256;
+            const int nn = b_n_fast ? e % BN : e / BK, kk = b_n_fast ? e / BN : e % BK;
+            const int64_t n = n0 + nn, k = k0 + kk;
+            rb[i] = (n < g.N && k < g.K) ? to_f<TIN>(B[k * g.b_sk + n * g.b_sn]) : 0.0f;
+        }
+    };
+    load_tiles(0);
+    for (int64_t k0 = 0; k0 < g.K; k0 += BK) {
+#pragma unroll
+        for (int i = 0; i < A_LD; ++i) {
+            const int e = tid + i * 256;
+            As[a_k_fast ? e % BK : e / BM][a_k_fast ? e / BK : e % BM] = ra[i];
+        }
+#pragma unroll
+        for (int i = 0; i < B_LD; ++i) {
+            const int e = tid + i * 256;
+            Bs[b_n_fast ? e / BN : e % BK][b_n_fast ? e % BN : e / BK] = rb[i];
         }
         __syncthreads();
-        // threads whose 4 x 4 outputs all lie outside the problem skip the arithmetic (a tiny M or N would
-        // otherwise fill the fp64 pipe with products nobody stores)
-        if (m0 + tm < g.M && n0 + tn < g.N)
+        if (k0 + BK < g.K) load_tiles(k0 + BK);
+        // threads whose outputs all lie outside the problem skip the arithmetic
+        if (m0 + tm < g.M && n0 + tn < g.N) {
+#pragma unroll 1
+            for (int ks = 0; ks < BK; ks += KSUB) {
+                float part[TM][4] = {};
 #pragma unroll
-        for (int kk = 0; kk < BK; ++kk) {
-            float av[4], bv[4];
+                for (int kk = ks; kk < ks + KSUB; ++kk) {
+                    float av[TM], bv[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) av[i] = As[kk][tm + i];
+                    for (int i = 0; i < TM; ++i) av[i] = As[kk][tm + i];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) bv[j] = Bs[kk][tn + j];
+                    for (int j = 0; j < 4; ++j) bv[j] = Bs[kk][tn + j];
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+                    for (int i = 0; i < TM; ++i)
 #pragma unroll
-                for (int j = 0; j < 4; ++j) acc[i][j] = fma((Acc)av[i], (Acc)bv[j], acc[i][j]);
+                        for (int j = 0; j < 4; ++j) {
+                            if constexpr (F64) part[i][j] = fmaf(av[i], bv[j], part[i][j]);
+                            else acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+                        }
+                }
+                if constexpr (F64) {
+#pragma unroll
+                    for (int i = 0; i < TM; ++i)
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) acc[i][j] += (double)part[i][j];
+                }
+            }
         }
         __syncthreads();
     }
     TOUT *C = (TOUT *)g.c;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < TM; ++i) {
         int64_t m = m0 + tm + i;
         if (m >= g.M) continue;
 #pragma unroll
@@ -77,16 +119,23 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmDesc g)
     }
 }
 
+template <int TM>
+static relay_status_t launch_tm(const GemmDesc &g, cudaStream_t st)
+{
+    constexpr int BM = 16 * TM;
+    dim3 grid((unsigned)((g.M + BM - 1) / BM), (unsigned)((g.N + BN - 1) / BN));
+    if (grid.y > 65535) return fail(RELAY_ERR_UNSUPPORTED, "SIMT contraction: N = %lld exceeds the grid limit", (long long)g.N);
+    if (g.in_dtype == RELAY_F32 && g.out_dtype == RELAY_F32) gemm_simt_kernel<float, float, false, TM><<<grid, 256, 0, st>>>(g);
+    else if (g.in_dtype == RELAY_BF16 && g.out_dtype == RELAY_BF16) gemm_simt_kernel<__nv_bfloat16, __nv_bfloat16, true, TM><<<grid, 256, 0, st>>>(g);
+    else if (g.in_dtype == RELAY_BF16 && g.out_dtype == RELAY_F32) gemm_simt_kernel<__nv_bfloat16, float, false, TM><<<grid, 256, 0, st>>>(g);
+    else return fail(RELAY_ERR_UNSUPPORTED, "SIMT contraction: %s -> %s has no instance", dtype_name(g.in_dtype), dtype_name(g.out_dtype));
+    return check_launch("gemm_simt");
+}
+
 relay_status_t launch_gemm_simt(const GemmDesc &g, cudaStream_t st)
 {
     if (g.M == 0 || g.N == 0) return RELAY_OK;
-    dim3 grid((unsigned)((g.M + BM - 1) / BM), (unsigned)((g.N + BN - 1) / BN));
-    if (grid.y > 65535) return fail(RELAY_ERR_UNSUPPORTED, "SIMT contraction: N = %lld exceeds the grid limit", (long long)g.N);
-    if (g.in_dtype == RELAY_F32 && g.out_dtype == RELAY_F32) gemm_simt_kernel<float, float, false><<<grid, 256, 0, st>>>(g);
-    else if (g.in_dtype == RELAY_BF16 && g.out_dtype == RELAY_BF16) gemm_simt_kernel<__nv_bfloat16, __nv_bfloat16, true><<<grid, 256, 0, st>>>(g);
-    else if (g.in_dtype == RELAY_BF16 && g.out_dtype == RELAY_F32) gemm_simt_kernel<__nv_bfloat16, float, false><<<grid, 256, 0, st>>>(g);
-    else return fail(RELAY_ERR_UNSUPPORTED, "SIMT contraction: %s -> %s has no instance", dtype_name(g.in_dtype), dtype_name(g.out_dtype));
-    return check_launch("gemm_simt");
+    return g.M <= 16 ? launch_tm<1>(g, st) : launch_tm<4>(g, st);
 }
 
 }  // namespace relay
