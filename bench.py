@@ -126,6 +126,65 @@ class Timer:
         self.pending = []
 
 
+class LeNetStep:
+    """One training step of the LeNet-shaped model of the paper's listing (Fig. 3), fp32: conv 5x5 + tanh, max_pool 2x2,
+    conv 5x5 + tanh, max_pool 2x2, flatten, linear + tanh, linear, softmax_cross_entropy; the gradient program back to
+    every parameter; one SGD update of the eight parameters.  All buffers are allocated once; `run` only enqueues."""
+
+    def __init__(self, B, I, dev, N):
+        self.B, self.N = B, N
+        self.t = t = {k: v.to(dev) for k, v in I.lenet_batch(N).items()}
+        self.p0 = {k: t[k].clone() for k in ("w1", "b1", "w2", "b2", "w3", "b3", "w4", "b4")}
+        E = lambda *s, dt=torch.float32: torch.empty(*s, dtype=dt, device=dev)
+        i32 = torch.int32
+        self.c1, self.p1, self.i1 = E(N, 20, 24, 24), E(N, 20, 12, 12), E(N, 20, 12, 12, dt=i32)
+        self.c2, self.p2, self.i2 = E(N, 50, 8, 8), E(N, 50, 4, 4), E(N, 50, 4, 4, dt=i32)
+        self.f1, self.f2, self.loss, self.dscores = E(N, 500), E(N, 10), E(N), E(N, 10)
+        self.dloss = torch.full((N,), 1.0 / N, device=dev)
+        self.g = {k: torch.empty_like(v) for k, v in self.p0.items()}
+        self.d_f1, self.d_flat, self.d_c2, self.d_p1, self.d_c1 = E(N, 500), E(N, 800), E(N, 50, 8, 8), E(N, 20, 12, 12), E(N, 20, 24, 24)
+        flat = self.p2.view(N, 800)
+        self.ws = torch.empty(max(16, B.relay_workspace_bytes_conv2d_act(t["x"], t["w1"], 1, 0), B.relay_workspace_bytes_conv2d_act(self.p1, t["w2"], 1, 0),
+                                  B.relay_workspace_bytes_dense_act_grad(self.f1, t["w4"]), B.relay_workspace_bytes_dense_act_grad(flat, t["w3"]),
+                                  B.relay_workspace_bytes_conv2d_act_grad(self.p1, t["w2"], 1, 0),
+                                  B.relay_workspace_bytes_conv2d_act_grad(t["x"], t["w1"], 1, 0)), dtype=torch.uint8, device=dev)
+        self.graph = None
+
+    def flop(self):
+        N = self.N
+        conv1, conv2, fc1, fc2 = 2 * N * 20 * 24 * 24 * 25, 2 * N * 50 * 8 * 8 * 20 * 25, 2 * N * 800 * 500, 2 * N * 500 * 10
+        return 3 * (conv2 + fc1 + fc2) + 2 * conv1        # forward + (dx, dW) of every layer; the first layer has no dx
+
+    def run(self):
+        B, t, g, ws, N = self.B, self.t, self.g, self.ws, self.N
+        TANH, NONE, K = B.ACT_TANH, B.ACT_NONE, (2, 2, 2, 2)
+        for k, v in self.p0.items():                       # every run starts from the same parameters
+            t[k].copy_(v)
+        B.relay_fused_conv2d_act(t["x"], t["w1"], t["b1"], 1, 0, TANH, self.c1, ws)
+        B.relay_max_pool2d(self.c1, *K, self.p1, self.i1)
+        B.relay_fused_conv2d_act(self.p1, t["w2"], t["b2"], 1, 0, TANH, self.c2, ws)
+        B.relay_max_pool2d(self.c2, *K, self.p2, self.i2)
+        flat = self.p2.view(N, 800)
+        B.relay_fused_dense_act(flat, t["w3"], t["b3"], TANH, self.f1, ws)
+        B.relay_fused_dense_act(self.f1, t["w4"], t["b4"], NONE, self.f2, ws)
+        B.relay_softmax_xent_grad(self.f2, t["labels"], self.dloss, self.loss, self.dscores)
+        B.relay_fused_dense_act_grad(self.f1, t["w4"], self.f2, self.dscores, NONE, self.d_f1, g["w4"], g["b4"], ws)
+        B.relay_fused_dense_act_grad(flat, t["w3"], self.f1, self.d_f1, TANH, self.d_flat, g["w3"], g["b3"], ws)
+        B.relay_max_pool2d_grad(self.i2, self.d_flat.view(N, 50, 4, 4), *K, self.d_c2)
+        B.relay_fused_conv2d_act_grad(self.p1, t["w2"], self.c2, self.d_c2, 1, 0, TANH, self.d_p1, g["w2"], g["b2"], ws)
+        B.relay_max_pool2d_grad(self.i1, self.d_p1, *K, self.d_c1)
+        B.relay_fused_conv2d_act_grad(t["x"], t["w1"], self.c1, self.d_c1, 1, 0, TANH, None, g["w1"], g["b1"], ws)
+        names = list(g)
+        B.relay_sgd_update([t[k] for k in names], [g[k] for k in names], 0.002)
+
+    def capture(self):
+        self.graph, s = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+        s.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.graph(self.graph, stream=s):
+            self.run()
+        torch.cuda.current_stream().wait_stream(s)
+
+
 class Workload:
     def __init__(self, dev, groups, small=False):
         from paper_1810_00952_b200 import binding as B
@@ -201,6 +260,7 @@ class Workload:
             ps_ = (shp[0], shp[1], shp[2] // 2, shp[3] // 2)
             self.pool_y, self.pool_idx = E(*ps_), E(*ps_, dt=torch.int32)
             self.pool_dy, self.pool_dx = I.normal(8, 1, ps_, 1.0, torch.bfloat16).to(dev), torch.empty_like(self.pool_x)
+            self.lenet = LeNetStep(B, I, dev, 4 if small else 64)
             # the conv configuration's tensors tagged NHWC (device-resident, permuted once): the layout-tagged calls
             c4 = self.devt["cfg4"] if "cfg4" in groups else {k: v.to(dev) for k, v in
                                                              I.cfg4_conv(*((2, 32, 14, 14, 32) if small else (32, 256, 56, 56, 256))).items()}
@@ -232,6 +292,25 @@ class Workload:
                 n += v.numel() * v.element_size()
         return n
 
+    def capture_cfg1(self):
+        """Captures the tiny layer's forward + gradient group (five small launches, launch-bound when issued one by
+        one) into a CUDA graph; `step` replays it as the group `cfg1.graph` while the captured buffers are current."""
+        if "cfg1" not in self.groups:
+            return
+        B, d, o, ws = self.B, self.devt["cfg1"], self.out["cfg1"], self.ws
+        g, s = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+        s.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.graph(g, stream=s):
+            B.relay_fused_dense_act(d["x"], d["w"], d["b"], B.ACT_RELU, o["y"], ws)
+            B.relay_fused_dense_act_grad(d["x"], d["w"], o["y"], d["dy"], B.ACT_RELU, o["dx"], o["dw"], o["db"], ws)
+        torch.cuda.current_stream().wait_stream(s)
+        self.cfg1_graph, self.cfg1_graph_bufs = g, d
+
+    def capture_graphs(self):
+        self.capture_cfg1()
+        if "next" in self.groups:
+            self.lenet.capture()
+
     def make_alternate(self):
         """Second set of device input and result buffers for the pipelined end-to-end loop."""
         self.alt = ({g: {k: torch.empty_like(v) for k, v in d.items()} for g, d in self.devt.items()},
@@ -254,6 +333,9 @@ class Workload:
                 B.relay_fused_dense_act(d["x"], d["w"], d["b"], B.ACT_RELU, o["y"], ws)
             with tm.region("cfg1.grad"):
                 B.relay_fused_dense_act_grad(d["x"], d["w"], o["y"], d["dy"], B.ACT_RELU, o["dx"], o["dw"], o["db"], ws)
+            if getattr(self, "cfg1_graph", None) is not None and self.cfg1_graph_bufs is d:
+                with tm.region("cfg1.graph"):
+                    self.cfg1_graph.replay()
         if "cfg2" in self.groups:
             d, o = self.devt["cfg2"], self.out["cfg2"]
             self.flush_l2()
@@ -311,6 +393,11 @@ class Workload:
             self.flush_l2()
             with tm.region("next.pool_grad"):
                 B.relay_max_pool2d_grad(self.pool_idx, self.pool_dy, 2, 2, 2, 2, self.pool_dx)
+            with tm.region("next.lenet"):
+                self.lenet.run()
+            if self.lenet.graph is not None:
+                with tm.region("next.lenet_graph"):
+                    self.lenet.graph.replay()
             h = self.nhwc
             self.flush_l2()
             with tm.region("next.conv_nhwc"):
@@ -323,6 +410,7 @@ class Workload:
         w = {}
         if "cfg1" in self.groups:
             w["cfg1.fwd"] = dict(flop=2 * 8 * 64 * 32); w["cfg1.grad"] = dict(flop=2 * 2 * 8 * 64 * 32 + 8 * 32 * 2)
+            w["cfg1.graph"] = dict(flop=w["cfg1.fwd"]["flop"] + w["cfg1.grad"]["flop"])
         if "cfg2" in self.groups:
             r, c = self.host["cfg2"]["x"].shape
             w["cfg2.fwd"] = dict(bytes=2 * r * c * 2 + 2 * c * 2)
@@ -352,6 +440,7 @@ class Workload:
             n, h, wd, c = self.nhwc["x"].shape
             f = 2 * n * h * wd * self.nhwc["w"].shape[0] * c * 9
             w["next.conv_nhwc"] = dict(flop=f); w["next.conv_nhwc_grad"] = dict(flop=2 * f)
+            w["next.lenet"] = dict(flop=self.lenet.flop()); w["next.lenet_graph"] = dict(flop=self.lenet.flop())
         return w
 
 
@@ -454,6 +543,9 @@ def main():
 
     tm = Timer()
     sampler = ClockSampler(local); sampler.start()
+    wl.step(tm)                      # first use of every kernel, outside the capture
+    torch.cuda.synchronize()
+    wl.capture_graphs()
     for _ in range(args.warmup):
         wl.step(tm)
     tm.collect(); tm.ms = {}

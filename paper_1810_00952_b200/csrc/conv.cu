@@ -51,7 +51,7 @@ static size_t conv_grad_ws(const ConvDims &d, size_t *dz_bytes)
 {
     *dz_bytes = align_up((size_t)(d.Nb * d.O * d.P * d.Q) * dtype_size(d.dt), 256);
     if (conv_tc_eligible(d)) return conv_tc_grad_workspace(d);   // the tensor-core tier keeps dZ in its own layout
-    return *dz_bytes;
+    return *dz_bytes + conv_dw_partial_bytes(d);                 // dZ, then the split sums of the weight gradient
 }
 
 }  // namespace relay
@@ -202,7 +202,7 @@ extern "C" relay_status_t relay_fused_conv2d_act_grad(const relay_tensor_t *x, c
         RELAY_TRY(act_grad_any(d.dt, dyp, yp, dz, nullptr, nullptr, rows, cols, act, st));
         if (db) RELAY_TRY(launch_conv_db(d, dz, (float *)db->data, st));
         if (dx) RELAY_TRY(launch_conv_dx_direct(d, dz, w->data, dxp, st));
-        RELAY_TRY(launch_conv_dw_direct(d, dz, xp, dw->data, st));
+        RELAY_TRY(launch_conv_dw_direct(d, dz, xp, dw->data, (float *)(inner + dz_bytes), st));
     }
     if (d.nhwc && dx) RELAY_TRY(launch_layout_change(d.dt, dxp, dx->data, d.Nb, d.C, d.H * d.W, st));
     return RELAY_OK;

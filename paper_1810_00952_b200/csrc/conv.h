@@ -14,11 +14,13 @@ struct ConvDims {
 // (NCHW -> NHWC: R = C, S = H*W;  NHWC -> NCHW: R = H*W, S = C)
 relay_status_t launch_layout_change(int32_t dt, const void *in, void *out, int64_t batch, int64_t R, int64_t S, cudaStream_t st);
 
-// direct (SIMT) tier: any stride / pad / window, fp32 accumulation in a fixed order
+// general (SIMT) tier: any stride / pad / window, implicit GEMM with gathers in the tile loaders (conv_igemm.cu);
+// the weight gradient is split along its sum and needs conv_dw_partial_bytes(d) of fp32 partials
 relay_status_t launch_conv_fwd_direct(const ConvDims &d, const void *x, const void *w, const void *b, int32_t b_dt, int act,
                                       void *y, cudaStream_t st);
 relay_status_t launch_conv_dx_direct(const ConvDims &d, const void *dz, const void *w, void *dx, cudaStream_t st);
-relay_status_t launch_conv_dw_direct(const ConvDims &d, const void *dz, const void *x, void *dw, cudaStream_t st);
+size_t conv_dw_partial_bytes(const ConvDims &d);
+relay_status_t launch_conv_dw_direct(const ConvDims &d, const void *dz, const void *x, void *dw, float *partials, cudaStream_t st);
 relay_status_t launch_conv_db(const ConvDims &d, const void *dz, float *db, cudaStream_t st);
 
 // implicit-GEMM tensor-core tier (3x3, stride 1, pad 1, bf16)

@@ -1,14 +1,13 @@
 // SIMT contraction kernel, sums in k order.  It is the fp32 path of the dense groups (tensor cores
 // would round the operands to tf32) and the path for shapes the tensor-core kernel does not take.
-// fp32 operands: runs of 16 products are summed in fp32 (exact products, one rounding per
-// fused multiply-add, on a partial sum that stays small) and the run sums are added in fp64 and
-// rounded once on the store.  The rounding error is then about 1e-7 of the output's RMS whatever K is,
-// so outputs that suffer cancellation still meet the fp32 tolerance, while the fp64 pipe (1/16 of the
-// fp32 rate) sees one addition per 16 products.  bf16 operands are accumulated in fp32.
+// fp32 operands: runs of 16 products are summed in fp32 and the run sums are added into a pair of floats
+// (simt_acc.cuh); the rounding error is then about 1e-7 of the output's RMS whatever K is, so outputs that suffer
+// cancellation still meet the fp32 tolerance.  bf16 operands are accumulated in fp32.
 #include <type_traits>
 
 #include "ewise_kernels.cuh"
 #include "gemm.h"
+#include "simt_acc.cuh"
 
 namespace relay {
 
@@ -35,7 +34,7 @@ __global__ void __launch_bounds__(256, 2) gemm_simt_kernel(const GemmDesc g)
     const int64_t m0 = (int64_t)blockIdx.x * BM, n0 = (int64_t)blockIdx.y * BN;
     const int tm = (tid / 16) * TM, tn = (tid % 16) * 4;
     constexpr bool F64 = sizeof(TIN) == 4;
-    using Acc = typename std::conditional<F64, double, float>::type;
+    using Acc = typename std::conditional<F64, PairSum, float>::type;
     Acc acc[TM][4] = {};
     // loader index order follows the unit stride of each operand so that loads coalesce
     const bool a_k_fast = g.a_sk == 1, b_n_fast = g.b_sn == 1;
@@ -94,7 +93,7 @@ __global__ void __launch_bounds__(256, 2) gemm_simt_kernel(const GemmDesc g)
 #pragma unroll
                     for (int i = 0; i < TM; ++i)
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) acc[i][j] += (double)part[i][j];
+                        for (int j = 0; j < 4; ++j) acc[i][j].add(part[i][j]);
                 }
             }
         }
@@ -109,9 +108,10 @@ __global__ void __launch_bounds__(256, 2) gemm_simt_kernel(const GemmDesc g)
         for (int j = 0; j < 4; ++j) {
             int64_t n = n0 + tn + j;
             if (n >= g.N) continue;
-            Acc zz = acc[i][j];
-            if (g.bias) zz += (Acc)(g.bias_dtype == RELAY_BF16 ? __bfloat162float(((const __nv_bfloat16 *)g.bias)[n]) : ((const float *)g.bias)[n]);
-            const float z = (float)zz;
+            float z;
+            const float bv = !g.bias ? 0.0f : g.bias_dtype == RELAY_BF16 ? __bfloat162float(((const __nv_bfloat16 *)g.bias)[n]) : ((const float *)g.bias)[n];
+            if constexpr (F64) z = (float)(acc[i][j].value() + (double)bv);
+            else z = acc[i][j] + bv;
             float y = act_fwd<FAST>(z, g.act);
             if constexpr (sizeof(TOUT) == 2) C[m * g.ldc + n] = __float2bfloat16_rn(y);
             else C[m * g.ldc + n] = y;

@@ -60,7 +60,7 @@ def test_conv_small_shapes_forward_and_gradient(N, C, H, W, O, R, stride, pad, t
 def test_conv_reduced_config_bf16_3x3(N, C, H, W, O):
     """Configuration 4's structure (3x3, stride 1, pad 1, NCHW/OIHW, bf16) at reduced sizes; the shapes
     with C and O multiples of 128 take the implicit-GEMM tensor-core kernels (several tiles, batch
-    slices of unequal size), the first one the direct kernels."""
+    slices of unequal size), the first one the general SIMT tier."""
     t = I.cfg4_conv(N, C, H, W, O, salt=C + W)
     y = conv_fwd(t["x"], t["w"], t["b"], 1, 1, B.ACT_RELU)
     xo, wo, bo, dyo = (I.as_f64(t[k]) for k in ("x", "w", "b", "dy"))
