@@ -47,11 +47,28 @@ struct IgemmArgs {
     int bias_bf16, act;
 };
 
-template <typename T, int MODE, bool FAST>
+// (c, r, s) of a flattened window index moved on by `step`: carries, a division only when a carry happens
+__device__ __forceinline__ void advance(int &c, int &r, int &s, int step, int R, int S)
+{
+    s += step;
+    if (s >= S) {
+        const int q = s / S;
+        s -= q * S;
+        r += q;
+        if (r >= R) {
+            const int q2 = r / R;
+            r -= q2 * R;
+            c += q2;
+        }
+    }
+}
+
+template <typename T, int MODE, bool FAST, bool STRIDE1>
 __global__ void __launch_bounds__(256, 2) conv_igemm_kernel(const IgemmArgs g)
 {
-    __shared__ float As[BK][BM + 1];
-    __shared__ float Bs[BK][BN + 1];
+    // the operand whose four values per thread are the same across a half-warp is read as one 16-byte vector
+    __shared__ __align__(16) float As[BK][BM + 4];
+    __shared__ __align__(16) float Bs[BK][BN + 4];
     const T *A = (const T *)g.a;
     const T *B = (const T *)g.b;
     const int tid = threadIdx.x;
@@ -59,6 +76,7 @@ __global__ void __launch_bounds__(256, 2) conv_igemm_kernel(const IgemmArgs g)
     const int64_t k_begin = (int64_t)blockIdx.z * g.k_per_slice;
     const int64_t k_end = min(g.Kg, k_begin + (int64_t)g.k_per_slice);
     const int RS = g.R * g.S, PQ = g.P * g.Q, HW = g.H * g.W;
+    const int stride = STRIDE1 ? 1 : g.stride;
     constexpr bool WIDE = sizeof(T) == 4;
     using Acc = typename std::conditional<WIDE, PairSum, float>::type;
     Acc acc[4][4] = {};
@@ -80,7 +98,7 @@ __global__ void __launch_bounds__(256, 2) conv_igemm_kernel(const IgemmArgs g)
             a_img = (int)(m / per);
             const int rem = (int)(m % per);
             a_y = rem / wdt; a_x = rem % wdt;
-            if (MODE == FWD) { a_y = a_y * g.stride - g.pad; a_x = a_x * g.stride - g.pad; }
+            if (MODE == FWD) { a_y = a_y * stride - g.pad; a_x = a_x * stride - g.pad; }
             else { a_y += g.pad; a_x += g.pad; }
         }
     }
@@ -102,16 +120,19 @@ __global__ void __launch_bounds__(256, 2) conv_igemm_kernel(const IgemmArgs g)
     float ra[LD], rb[LD];
     auto load_tiles = [&](int64_t k0) {
         if (MODE == FWD) {
+            // slot 0's k is decomposed by division, the other slots follow by carries
+            const int64_t kf = k0 + tid / BM;
+            int c = (int)(kf / RS), r, sx;
+            { const int rs = (int)(kf % RS); r = rs / g.S; sx = rs % g.S; }
 #pragma unroll
             for (int i = 0; i < LD; ++i) {
-                const int64_t k = k0 + tid / BM + 4 * i;
                 float v = 0.0f;
-                if (a_row_ok && k < k_end) {
-                    const int c = (int)(k / RS), rs = (int)(k % RS);
-                    const int yy = a_y + rs / g.S, xx = a_x + rs % g.S;
+                if (a_row_ok && kf + 4 * i < k_end) {
+                    const int yy = a_y + r, xx = a_x + sx;
                     if (yy >= 0 && yy < g.H && xx >= 0 && xx < g.W) v = ldf(A, (((int64_t)a_img * g.C + c) * g.H + yy) * g.W + xx);
                 }
                 ra[i] = v;
+                advance(c, r, sx, 4, g.R, g.S);
             }
             const int64_t k = k0 + tid % BK;
 #pragma unroll
@@ -120,26 +141,30 @@ __global__ void __launch_bounds__(256, 2) conv_igemm_kernel(const IgemmArgs g)
                 rb[i] = (n < g.Ng && k < k_end) ? ldf(B, n * g.Kg + k) : 0.0f;
             }
         } else if (MODE == DX) {
+            const int64_t kf = k0 + tid / BM;
+            int o = (int)(kf / RS), r, sx;
+            { const int rs = (int)(kf % RS); r = rs / g.S; sx = rs % g.S; }
 #pragma unroll
             for (int i = 0; i < LD; ++i) {
-                const int64_t k = k0 + tid / BM + 4 * i;
                 float v = 0.0f;
-                if (a_row_ok && k < k_end) {
-                    const int o = (int)(k / RS), rs = (int)(k % RS);
-                    const int yn = a_y - rs / g.S, xn = a_x - rs % g.S;
-                    if (yn >= 0 && xn >= 0 && yn % g.stride == 0 && xn % g.stride == 0) {
-                        const int p = yn / g.stride, q = xn / g.stride;
+                if (a_row_ok && kf + 4 * i < k_end) {
+                    const int yn = a_y - r, xn = a_x - sx;
+                    if (STRIDE1) {
+                        if (yn >= 0 && xn >= 0 && yn < g.P && xn < g.Q) v = ldf(A, (((int64_t)a_img * g.O + o) * g.P + yn) * g.Q + xn);
+                    } else if (yn >= 0 && xn >= 0 && yn % stride == 0 && xn % stride == 0) {
+                        const int p = yn / stride, q = xn / stride;
                         if (p < g.P && q < g.Q) v = ldf(A, (((int64_t)a_img * g.O + o) * g.P + p) * g.Q + q);
                     }
                 }
                 ra[i] = v;
+                advance(o, r, sx, 4, g.R, g.S);
             }
             const int64_t k = k0 + tid % BK;
-            const int o = (int)(k / RS), rs = (int)(k % RS);
+            const int ob = (int)(k / RS), rsb = (int)(k % RS);
 #pragma unroll
             for (int i = 0; i < LD; ++i) {
                 const int64_t c = n0 + tid / BK + 16 * i;
-                rb[i] = (c < g.Ng && k < k_end) ? ldf(B, ((int64_t)o * g.C + c) * RS + rs) : 0.0f;
+                rb[i] = (c < g.Ng && k < k_end) ? ldf(B, ((int64_t)ob * g.C + c) * RS + rsb) : 0.0f;
             }
         } else {
             const int64_t k = k0 + tid % BK;
@@ -155,7 +180,7 @@ __global__ void __launch_bounds__(256, 2) conv_igemm_kernel(const IgemmArgs g)
                 const int64_t o = m0 + tid / BK + 16 * i;
                 ra[i] = (k_ok && o < g.Mg) ? ldf(A, ((int64_t)img * g.O + o) * PQ + (int64_t)p * g.Q + q) : 0.0f;
             }
-            const int y0 = p * g.stride, x0 = q * g.stride;
+            const int y0 = p * stride, x0 = q * stride;
             const int64_t base = (int64_t)img * g.C * HW + (int64_t)y0 * g.W + x0;
 #pragma unroll
             for (int i = 0; i < LD; ++i) {
@@ -182,10 +207,17 @@ __global__ void __launch_bounds__(256, 2) conv_igemm_kernel(const IgemmArgs g)
 #pragma unroll
         for (int kk = 0; kk < BK; ++kk) {
             float av[4], bv[4];
+            if (MODE == DW) {
+                const float4 a4 = *reinterpret_cast<const float4 *>(&As[kk][4 * lane_m]);
+                av[0] = a4.x; av[1] = a4.y; av[2] = a4.z; av[3] = a4.w;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) av[i] = As[kk][lane_m + 16 * i];
+                for (int j = 0; j < 4; ++j) bv[j] = Bs[kk][lane_n + 16 * j];
+            } else {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) bv[j] = Bs[kk][lane_n + 16 * j];
+                for (int i = 0; i < 4; ++i) av[i] = As[kk][lane_m + 16 * i];
+                const float4 b4 = *reinterpret_cast<const float4 *>(&Bs[kk][4 * lane_n]);
+                bv[0] = b4.x; bv[1] = b4.y; bv[2] = b4.z; bv[3] = b4.w;
+            }
 #pragma unroll
             for (int i = 0; i < 4; ++i)
 #pragma unroll
@@ -206,14 +238,14 @@ __global__ void __launch_bounds__(256, 2) conv_igemm_kernel(const IgemmArgs g)
     // ---- store ---------------------------------------------------------------------------------------------
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        const int64_t m = m0 + lane_m + 16 * i;
+        const int64_t m = m0 + (MODE == DW ? 4 * lane_m + i : lane_m + 16 * i);
         if (m >= g.Mg) continue;
         int64_t row_base = 0;      // FWD: offset of y[n, 0, p, q];  DX: offset of dx[n, 0, i, j]
         if (MODE == FWD) row_base = (m / PQ) * (int64_t)g.O * PQ + m % PQ;
         if (MODE == DX) row_base = (m / HW) * (int64_t)g.C * HW + m % HW;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int64_t n = n0 + lane_n + 16 * j;
+            const int64_t n = n0 + (MODE == DW ? lane_n + 16 * j : 4 * lane_n + j);
             if (n >= g.Ng) continue;
             float bv = 0.0f;
             if (MODE == FWD && g.bias) bv = g.bias_bf16 ? __bfloat162float(((const __nv_bfloat16 *)g.bias)[n]) : ((const float *)g.bias)[n];
@@ -270,6 +302,16 @@ int dw_slices(const ConvDims &d)
     return (int)std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(by_work, 4096), (2 * 148 + tiles - 1) / tiles));
 }
 
+template <int MODE>
+void launch_mode(const ConvDims &d, const IgemmArgs &g, dim3 grid, cudaStream_t st)
+{
+    const bool bf = d.dt == RELAY_BF16, s1 = d.stride == 1;
+    if (bf && s1) conv_igemm_kernel<__nv_bfloat16, MODE, true, true><<<grid, 256, 0, st>>>(g);
+    else if (bf) conv_igemm_kernel<__nv_bfloat16, MODE, true, false><<<grid, 256, 0, st>>>(g);
+    else if (s1) conv_igemm_kernel<float, MODE, false, true><<<grid, 256, 0, st>>>(g);
+    else conv_igemm_kernel<float, MODE, false, false><<<grid, 256, 0, st>>>(g);
+}
+
 }  // namespace
 
 size_t conv_dw_partial_bytes(const ConvDims &d)
@@ -288,8 +330,7 @@ relay_status_t launch_conv_fwd_direct(const ConvDims &d, const void *x, const vo
     g.a = x; g.b = w; g.out = y; g.bias = b; g.bias_bf16 = b_dt == RELAY_BF16; g.act = act;
     dim3 grid;
     RELAY_TRY(grid_of(g, 1, &grid));
-    if (d.dt == RELAY_BF16) conv_igemm_kernel<__nv_bfloat16, FWD, true><<<grid, 256, 0, st>>>(g);
-    else conv_igemm_kernel<float, FWD, false><<<grid, 256, 0, st>>>(g);
+    launch_mode<FWD>(d, g, grid, st);
     return check_launch("conv_igemm_fwd");
 }
 
@@ -303,8 +344,7 @@ relay_status_t launch_conv_dx_direct(const ConvDims &d, const void *dz, const vo
     g.a = dz; g.b = w; g.out = dx;
     dim3 grid;
     RELAY_TRY(grid_of(g, 1, &grid));
-    if (d.dt == RELAY_BF16) conv_igemm_kernel<__nv_bfloat16, DX, true><<<grid, 256, 0, st>>>(g);
-    else conv_igemm_kernel<float, DX, false><<<grid, 256, 0, st>>>(g);
+    launch_mode<DX>(d, g, grid, st);
     return check_launch("conv_igemm_dx");
 }
 
@@ -321,8 +361,7 @@ relay_status_t launch_conv_dw_direct(const ConvDims &d, const void *dz, const vo
     g.a = dz; g.b = x; g.out = partials;
     dim3 grid;
     RELAY_TRY(grid_of(g, slices, &grid));
-    if (d.dt == RELAY_BF16) conv_igemm_kernel<__nv_bfloat16, DW, true><<<grid, 256, 0, st>>>(g);
-    else conv_igemm_kernel<float, DW, false><<<grid, 256, 0, st>>>(g);
+    launch_mode<DW>(d, g, grid, st);
     RELAY_TRY(check_launch("conv_igemm_dw"));
     const unsigned rb = (unsigned)((total + 255) / 256);
     if (d.dt == RELAY_BF16) conv_dw_reduce_kernel<<<rb, 256, 0, st>>>(partials, slices, total, (__nv_bfloat16 *)dw);

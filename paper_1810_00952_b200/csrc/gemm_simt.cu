@@ -17,17 +17,17 @@ template <typename T> __device__ __forceinline__ float to_f(T v);
 template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
 
-// block tile (16 * TM) x 64, thread tile TM x 4: TM = 4 in general, TM = 1 for outputs of at most 16 rows
-// (all 256 threads then hold live outputs instead of one warp's worth).  The loads of k-block i+1 are issued
+// block tile (16 * TM) x 64, thread tile TM x 4: TM = 4 for large outputs, TM = 1 for outputs of at most 16 rows
+// (all 256 threads then hold live outputs instead of one warp's worth) and for grids that would not fill the SMs.  The loads of k-block i+1 are issued
 // into registers before the arithmetic of k-block i, all of a thread's loads back to back, so that one
 // memory round trip per k-block is exposed at most.
 template <typename TIN, typename TOUT, bool FAST, int TM>
-__global__ void __launch_bounds__(256, 2) gemm_simt_kernel(const GemmDesc g)
+__global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmDesc g)
 {
     constexpr int BM = 16 * TM;
     constexpr int A_LD = BM * BK / 256, B_LD = BN * BK / 256;
-    __shared__ float As[BK][BM + 1];
-    __shared__ float Bs[BK][BN + 1];
+    __shared__ __align__(16) float As[BK][BM + 4];     // rows of whole 16-byte vectors: a thread's four values are one load
+    __shared__ __align__(16) float Bs[BK][BN + 4];
     const TIN *A = (const TIN *)g.a;
     const TIN *B = (const TIN *)g.b;
     const int tid = threadIdx.x;
@@ -77,10 +77,15 @@ __global__ void __launch_bounds__(256, 2) gemm_simt_kernel(const GemmDesc g)
 #pragma unroll
                 for (int kk = ks; kk < ks + KSUB; ++kk) {
                     float av[TM], bv[4];
+                    if constexpr (TM == 4) {
+                        const float4 a4 = *reinterpret_cast<const float4 *>(&As[kk][tm]);
+                        av[0] = a4.x; av[1] = a4.y; av[2] = a4.z; av[3] = a4.w;
+                    } else {
 #pragma unroll
-                    for (int i = 0; i < TM; ++i) av[i] = As[kk][tm + i];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) bv[j] = Bs[kk][tn + j];
+                        for (int i = 0; i < TM; ++i) av[i] = As[kk][tm + i];
+                    }
+                    const float4 b4 = *reinterpret_cast<const float4 *>(&Bs[kk][tn]);
+                    bv[0] = b4.x; bv[1] = b4.y; bv[2] = b4.z; bv[3] = b4.w;
 #pragma unroll
                     for (int i = 0; i < TM; ++i)
 #pragma unroll
@@ -135,7 +140,10 @@ static relay_status_t launch_tm(const GemmDesc &g, cudaStream_t st)
 relay_status_t launch_gemm_simt(const GemmDesc &g, cudaStream_t st)
 {
     if (g.M == 0 || g.N == 0) return RELAY_OK;
-    return g.M <= 16 ? launch_tm<1>(g, st) : launch_tm<4>(g, st);
+    // 16-row tiles while 64-row tiles would leave SMs without a block: a block of the small tile spends a k-block
+    // mostly waiting for its loads, so more and lighter blocks finish sooner
+    const int64_t big_tiles = ((g.M + 63) / 64) * ((g.N + BN - 1) / BN);
+    return (g.M <= 16 || big_tiles < 2 * 148) ? launch_tm<1>(g, st) : launch_tm<4>(g, st);
 }
 
 }  // namespace relay
