@@ -15,24 +15,31 @@ template <typename T> __device__ __forceinline__ void stf(T *p, int64_t i, float
     else p[i] = v;
 }
 
-// db[o] = sum over n, p, q of dz[n,o,p,q]: one block per channel, fixed-order combine
+// db[o] = sum over n, p, q of dz[n,o,p,q]: one block of 32 warps per channel; warp w takes the images w, w + 32, ...,
+// its lanes run along the contiguous pixels (four independent loads in flight per lane); fixed-order combine
 template <typename T>
-__global__ void __launch_bounds__(256) conv_db_kernel(const ConvDims d, const T *__restrict__ dz, float *__restrict__ db)
+__global__ void __launch_bounds__(1024) conv_db_kernel(const ConvDims d, const T *__restrict__ dz, float *__restrict__ db)
 {
-    __shared__ float sm[8];
+    __shared__ float sm[32];
     const int64_t o = blockIdx.x, pq = d.P * d.Q;
-    float acc = 0.0f;
-    for (int64_t l = threadIdx.x; l < d.Nb * pq; l += blockDim.x) {
-        int64_t n = l / pq, r = l % pq;
-        acc += ldf(dz, (n * d.O + o) * pq + r);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
+    for (int64_t n = warp; n < d.Nb; n += 32) {
+        const T *row = dz + (n * d.O + o) * pq;
+        int64_t r = lane;
+        for (; r + 96 < pq; r += 128) {
+            a0 += ldf(row, r); a1 += ldf(row, r + 32); a2 += ldf(row, r + 64); a3 += ldf(row, r + 96);
+        }
+        for (; r < pq; r += 32) a0 += ldf(row, r);
     }
+    float acc = (a0 + a1) + (a2 + a3);
 #pragma unroll
     for (int k = 16; k > 0; k >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, k);
-    if ((threadIdx.x & 31) == 0) sm[threadIdx.x >> 5] = acc;
+    if (lane == 0) sm[warp] = acc;
     __syncthreads();
     if (threadIdx.x == 0) {
         float s = 0.0f;
-        for (int k = 0; k < 8; ++k) s += sm[k];
+        for (int k = 0; k < 32; ++k) s += sm[k];
         db[o] = s;
     }
 }
@@ -40,8 +47,8 @@ __global__ void __launch_bounds__(256) conv_db_kernel(const ConvDims d, const T 
 relay_status_t launch_conv_db(const ConvDims &d, const void *dz, float *db, cudaStream_t st)
 {
     if (d.O == 0) return RELAY_OK;
-    if (d.dt == RELAY_BF16) conv_db_kernel<<<(unsigned)d.O, 256, 0, st>>>(d, (const __nv_bfloat16 *)dz, db);
-    else conv_db_kernel<<<(unsigned)d.O, 256, 0, st>>>(d, (const float *)dz, db);
+    if (d.dt == RELAY_BF16) conv_db_kernel<<<(unsigned)d.O, 1024, 0, st>>>(d, (const __nv_bfloat16 *)dz, db);
+    else conv_db_kernel<<<(unsigned)d.O, 1024, 0, st>>>(d, (const float *)dz, db);
     return check_launch("conv_db");
 }
 
