@@ -25,6 +25,12 @@
  *     relay_last_error() returns a thread-local description of the last failure.
  *   - Kernels that wait on hardware barriers give up after a bounded number of polls and set a
  *     device-side error word instead of hanging; relay_poll_status() reads (and clears) it.
+ *   - Stream capture: a compute entry point may be called while `stream` is being captured into a
+ *     CUDA graph (it enqueues kernels on `stream` only, allocates nothing and does not synchronise),
+ *     provided an entry point of the same kind was called once on this device before the capture
+ *     (module loading and one-time address look-ups happen on first use).  The graph holds the
+ *     pointers of the captured call: replaying it recomputes into the same buffers.
+ *     relay_poll_status() synchronises and must stay outside a capture.
  */
 #ifndef RELAY_B200_H_
 #define RELAY_B200_H_
