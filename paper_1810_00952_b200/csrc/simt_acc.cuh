@@ -3,8 +3,8 @@
 // bf16 operands: a plain fp32 accumulator, products added in k order.
 // fp32 operands: runs of products are summed in fp32 (exact products, one rounding per fused multiply-add, on a
 // partial sum that stays small) and the run sums are added into an unevaluated pair of floats (hi + lo) with the
-// error-free two-sum, so the total carries about 48 bits whatever the number of terms.  The fp64 pipe, which runs
-// at 1/16 of the fp32 rate on this part, is not used.
+// error-free two-sum, so the total carries about 48 bits whatever the number of terms.  The fp64 pipe, far narrower
+// than the fp32 one on this part, is not used in the loop.
 #pragma once
 
 namespace relay {
