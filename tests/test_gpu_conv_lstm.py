@@ -37,7 +37,12 @@ def conv_grad(x, w, y, dy, stride, pad, act, want_dx=True, want_db=True):
 
 
 @pytest.mark.parametrize("N,C,H,W,O,R,stride,pad", [(2, 3, 7, 6, 4, 3, 1, 1), (1, 5, 9, 9, 3, 3, 2, 1), (2, 2, 8, 5, 6, 5, 1, 0),
-                                                     (1, 4, 6, 6, 2, 1, 1, 0), (3, 8, 10, 12, 16, 3, 2, 2), (1, 1, 1, 1, 1, 3, 1, 1)])
+                                                     (1, 4, 6, 6, 2, 1, 1, 0), (3, 8, 10, 12, 16, 3, 2, 2), (1, 1, 1, 1, 1, 3, 1, 1),
+                                                     # several tiles of the general tier along every GEMM axis, ragged tails, a split
+                                                     # weight-gradient sum with a short last slice: 70 output channels (two tiles),
+                                                     # LeNet's second conv (N*P*Q = 4096 over 37 slices), a 7x7 window at stride 3
+                                                     (3, 7, 11, 13, 70, 3, 2, 1), (64, 20, 12, 12, 50, 5, 1, 0), (2, 4, 23, 19, 3, 7, 3, 3),
+                                                     (5, 3, 33, 17, 5, 1, 1, 0)])
 @pytest.mark.parametrize("tdt", [torch.float32, torch.bfloat16])
 def test_conv_small_shapes_forward_and_gradient(N, C, H, W, O, R, stride, pad, tdt):
     t = I.cfg4_conv(N, C, H, W, O, R, R, dtype=tdt, salt=H)
