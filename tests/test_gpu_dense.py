@@ -52,7 +52,8 @@ def test_tiny_mlp_layer_fp32_forward_and_gradient(act):
 
 
 @pytest.mark.parametrize("M,K,N", [(1, 1, 1), (37, 53, 29), (130, 70, 200), (64, 64, 64), (5, 300, 8),
-                                   (128, 64, 256), (200, 136, 264), (384, 512, 320), (72, 1032, 520)])
+                                   (128, 64, 256), (200, 136, 264), (384, 512, 320), (72, 1032, 520),
+                                   (1100, 24, 1100)])      # SIMT kernel with its 64-row tile (a grid that fills the SMs)
 @pytest.mark.parametrize("tdt", [torch.float32, torch.bfloat16])
 def test_odd_shapes_forward_and_gradient(M, K, N, tdt):
     t = I.cfg1_tiny_mlp(M, K, N, salt=M)
