@@ -716,7 +716,8 @@ def main():
                 "config": {"workload": ("reduced shapes" if args.small else "all five configurations at full size")
                            + ": step = cfg1 fwd+grad, cfg2 fwd+grad, cfg3 3-layer fwd+bwd, cfg4 conv fwd+dX+dW+db, cfg5 LSTM forward + gradient program"
                            + ", then softmax cross-entropy loss / loss+partial on 8192x8192 bf16, SGD on three 4096^2 bf16 matrices and 2x2 max pooling"
-                           + " forward + gradient on 32x256x56x56 bf16",
+                           + " forward + gradient on 32x256x56x56 bf16, one fp32 LeNet training step (batch 64) eager and replayed from a"
+                           + " CUDA graph, the cfg4 conv with NHWC-tagged tensors; cfg1 is also replayed from a CUDA graph",
                            "value_covers": "dense + conv2d groups (cfg3 + cfg4) FLOPs / their device time; hbm_gbs covers cfg2",
                            "groups": groups, "l2": "1 GiB streamed through L2 between groups (flush with clean lines); cfg2 inputs also exceed L2",
                            "replicas": world},
