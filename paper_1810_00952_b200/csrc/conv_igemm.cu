@@ -1,6 +1,6 @@
 // General conv2d tier (SIMT): every stride / padding / window size, both float types.  The three
 // contractions of a conv2d group are run as implicit GEMMs on 64 x 64 output tiles, k-blocks of 16, with the
-// operand gathers done by the tile loaders (no im2col buffer):
+// operand gathers done by the tile loaders (no im2col buffer; smaller tiles for small grids and few channels):
 //
 //   forward          Y[(n,p,q), o]   = sum over (c,r,s) of  X[n, c, p*st-pad+r, q*st-pad+s] * W[o, (c,r,s)]
 //   input gradient   dX[(n,i,j), c]  = sum over (o,r,s) of  dZ[n, o, (i+pad-r)/st, (j+pad-s)/st] * W[o, c, r, s]
@@ -23,7 +23,7 @@ namespace relay {
 
 namespace {
 
-constexpr int BM = 64, BN = 64, BK = 16, LD = BM * BK / 256;   // LD loader slots per thread and operand
+constexpr int BK = 16;       // k-block depth; a block tile is (16 * TMR) x (16 * TN), a thread tile TMR x TN
 enum { FWD = 0, DX = 1, DW = 2 };
 
 template <typename T> __device__ __forceinline__ float ldf(const T *p, int64_t i)
@@ -63,10 +63,16 @@ __device__ __forceinline__ void advance(int &c, int &r, int &s, int step, int R,
     }
 }
 
-template <typename T, int MODE, bool FAST, bool STRIDE1>
+// TMR x TN outputs per thread: 4 x 4 in general; FWD and DX also come with 2 rows (twice the blocks when the grid
+// would leave SMs idle) and with 2 columns (few output channels: less arithmetic on padding)
+template <typename T, int MODE, bool FAST, bool STRIDE1, int TMR, int TN>
 __global__ void __launch_bounds__(256, 2) conv_igemm_kernel(const IgemmArgs g)
 {
-    // the operand whose four values per thread are the same across a half-warp is read as one 16-byte vector
+    static_assert(MODE != DW || (TMR == 4 && TN == 4), "the weight gradient uses the 64 x 64 tile");
+    constexpr int BM = 16 * TMR, BN = 16 * TN;
+    constexpr int LDA = TMR, LDB = TN;                  // loader slots per thread: BM * BK / 256, BN * BK / 256
+    constexpr int KSTEP = 256 / BM;                     // FWD, DX: k distance between a thread's A slots
+    // the operand whose values per thread are the same across a half-warp is read as one vector
     __shared__ __align__(16) float As[BK][BM + 4];
     __shared__ __align__(16) float Bs[BK][BN + 4];
     const T *A = (const T *)g.a;
@@ -79,13 +85,13 @@ __global__ void __launch_bounds__(256, 2) conv_igemm_kernel(const IgemmArgs g)
     const int stride = STRIDE1 ? 1 : g.stride;
     constexpr bool WIDE = sizeof(T) == 4;
     using Acc = typename std::conditional<WIDE, PairSum, float>::type;
-    Acc acc[4][4] = {};
+    Acc acc[TMR][TN] = {};
     // output rows / columns of this thread: lanes run along the axis that is contiguous in memory
     // (pixels for FWD and DX, the flattened (c,r,s) index for DW)
     const int lane_m = MODE == DW ? tid / 16 : tid % 16, lane_n = MODE == DW ? tid % 16 : tid / 16;
 
     // ---- loader state that does not depend on the k-block ---------------------------------------------
-    // FWD, DX: A slot i holds (row mm = tid % 64, k-offset kk = tid / 64 + 4 i): the row's pixel is decomposed once.
+    // FWD, DX: A slot i holds (row mm = tid % BM, k-offset kk = tid / BM + KSTEP i): the row's pixel is decomposed once.
     // DW:      A and B slot i hold (k-offset kk = tid % 16, row / column tid / 16 + 16 i): k is decomposed once per
     //          k-block, the B column's (c,r,s) once per slot.
     int a_img = 0, a_y = 0, a_x = 0;          // FWD: (n, p*st-pad, q*st-pad);  DX: (n, i+pad, j+pad)
@@ -102,11 +108,11 @@ __global__ void __launch_bounds__(256, 2) conv_igemm_kernel(const IgemmArgs g)
             else { a_y += g.pad; a_x += g.pad; }
         }
     }
-    int64_t b_off[LD];                          // DW: (c*H + r - pad)*W + s - pad of the slot's column
-    int b_dy[LD], b_dx[LD];                     // DW: r - pad, s - pad (negative dy marks a column out of range)
+    int64_t b_off[LDB];                         // DW: (c*H + r - pad)*W + s - pad of the slot's column
+    int b_dy[LDB], b_dx[LDB];                   // DW: r - pad, s - pad (INT_MIN marks a column out of range)
     if (MODE == DW) {
 #pragma unroll
-        for (int i = 0; i < LD; ++i) {
+        for (int i = 0; i < LDB; ++i) {
             const int64_t n = n0 + tid / BK + 16 * i;
             b_dy[i] = INT_MIN; b_dx[i] = 0; b_off[i] = 0;
             if (n < g.Ng) {
@@ -117,7 +123,7 @@ __global__ void __launch_bounds__(256, 2) conv_igemm_kernel(const IgemmArgs g)
         }
     }
 
-    float ra[LD], rb[LD];
+    float ra[LDA], rb[LDB];
     auto load_tiles = [&](int64_t k0) {
         if (MODE == FWD) {
             // slot 0's k is decomposed by division, the other slots follow by carries
@@ -125,18 +131,18 @@ __global__ void __launch_bounds__(256, 2) conv_igemm_kernel(const IgemmArgs g)
             int c = (int)(kf / RS), r, sx;
             { const int rs = (int)(kf % RS); r = rs / g.S; sx = rs % g.S; }
 #pragma unroll
-            for (int i = 0; i < LD; ++i) {
+            for (int i = 0; i < LDA; ++i) {
                 float v = 0.0f;
-                if (a_row_ok && kf + 4 * i < k_end) {
+                if (a_row_ok && kf + KSTEP * i < k_end) {
                     const int yy = a_y + r, xx = a_x + sx;
                     if (yy >= 0 && yy < g.H && xx >= 0 && xx < g.W) v = ldf(A, (((int64_t)a_img * g.C + c) * g.H + yy) * g.W + xx);
                 }
                 ra[i] = v;
-                advance(c, r, sx, 4, g.R, g.S);
+                advance(c, r, sx, KSTEP, g.R, g.S);
             }
             const int64_t k = k0 + tid % BK;
 #pragma unroll
-            for (int i = 0; i < LD; ++i) {
+            for (int i = 0; i < LDB; ++i) {
                 const int64_t n = n0 + tid / BK + 16 * i;
                 rb[i] = (n < g.Ng && k < k_end) ? ldf(B, n * g.Kg + k) : 0.0f;
             }
@@ -145,9 +151,9 @@ __global__ void __launch_bounds__(256, 2) conv_igemm_kernel(const IgemmArgs g)
             int o = (int)(kf / RS), r, sx;
             { const int rs = (int)(kf % RS); r = rs / g.S; sx = rs % g.S; }
 #pragma unroll
-            for (int i = 0; i < LD; ++i) {
+            for (int i = 0; i < LDA; ++i) {
                 float v = 0.0f;
-                if (a_row_ok && kf + 4 * i < k_end) {
+                if (a_row_ok && kf + KSTEP * i < k_end) {
                     const int yn = a_y - r, xn = a_x - sx;
                     if (STRIDE1) {
                         if (yn >= 0 && xn >= 0 && yn < g.P && xn < g.Q) v = ldf(A, (((int64_t)a_img * g.O + o) * g.P + yn) * g.Q + xn);
@@ -157,12 +163,12 @@ __global__ void __launch_bounds__(256, 2) conv_igemm_kernel(const IgemmArgs g)
                     }
                 }
                 ra[i] = v;
-                advance(o, r, sx, 4, g.R, g.S);
+                advance(o, r, sx, KSTEP, g.R, g.S);
             }
             const int64_t k = k0 + tid % BK;
             const int ob = (int)(k / RS), rsb = (int)(k % RS);
 #pragma unroll
-            for (int i = 0; i < LD; ++i) {
+            for (int i = 0; i < LDB; ++i) {
                 const int64_t c = n0 + tid / BK + 16 * i;
                 rb[i] = (c < g.Ng && k < k_end) ? ldf(B, ((int64_t)ob * g.C + c) * RS + rsb) : 0.0f;
             }
@@ -176,14 +182,14 @@ __global__ void __launch_bounds__(256, 2) conv_igemm_kernel(const IgemmArgs g)
                 p = pq / g.Q; q = pq % g.Q;
             }
 #pragma unroll
-            for (int i = 0; i < LD; ++i) {
+            for (int i = 0; i < LDA; ++i) {
                 const int64_t o = m0 + tid / BK + 16 * i;
                 ra[i] = (k_ok && o < g.Mg) ? ldf(A, ((int64_t)img * g.O + o) * PQ + (int64_t)p * g.Q + q) : 0.0f;
             }
             const int y0 = p * stride, x0 = q * stride;
             const int64_t base = (int64_t)img * g.C * HW + (int64_t)y0 * g.W + x0;
 #pragma unroll
-            for (int i = 0; i < LD; ++i) {
+            for (int i = 0; i < LDB; ++i) {
                 float v = 0.0f;
                 if (k_ok && b_dy[i] != INT_MIN) {
                     const int yy = y0 + b_dy[i], xx = x0 + b_dx[i];
@@ -197,55 +203,62 @@ __global__ void __launch_bounds__(256, 2) conv_igemm_kernel(const IgemmArgs g)
     if (k_begin < k_end) load_tiles(k_begin);
     for (int64_t k0 = k_begin; k0 < k_end; k0 += BK) {
 #pragma unroll
-        for (int i = 0; i < LD; ++i) {
-            if (MODE == DW) { As[tid % BK][tid / BK + 16 * i] = ra[i]; Bs[tid % BK][tid / BK + 16 * i] = rb[i]; }
-            else { As[tid / BM + 4 * i][tid % BM] = ra[i]; Bs[tid % BK][tid / BK + 16 * i] = rb[i]; }
+        for (int i = 0; i < LDA; ++i) {
+            if (MODE == DW) As[tid % BK][tid / BK + 16 * i] = ra[i];
+            else As[tid / BM + KSTEP * i][tid % BM] = ra[i];
         }
+#pragma unroll
+        for (int i = 0; i < LDB; ++i) Bs[tid % BK][tid / BK + 16 * i] = rb[i];
         __syncthreads();
         if (k0 + BK < k_end) load_tiles(k0 + BK);
-        float part[4][4] = {};
+        float part[TMR][TN] = {};
 #pragma unroll
         for (int kk = 0; kk < BK; ++kk) {
-            float av[4], bv[4];
+            float av[TMR], bv[TN];
             if (MODE == DW) {
                 const float4 a4 = *reinterpret_cast<const float4 *>(&As[kk][4 * lane_m]);
                 av[0] = a4.x; av[1] = a4.y; av[2] = a4.z; av[3] = a4.w;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) bv[j] = Bs[kk][lane_n + 16 * j];
+                for (int j = 0; j < TN; ++j) bv[j] = Bs[kk][lane_n + 16 * j];
             } else {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) av[i] = As[kk][lane_m + 16 * i];
-                const float4 b4 = *reinterpret_cast<const float4 *>(&Bs[kk][4 * lane_n]);
-                bv[0] = b4.x; bv[1] = b4.y; bv[2] = b4.z; bv[3] = b4.w;
+                for (int i = 0; i < TMR; ++i) av[i] = As[kk][lane_m + 16 * i];
+                if constexpr (TN == 4) {
+                    const float4 b4 = *reinterpret_cast<const float4 *>(&Bs[kk][4 * lane_n]);
+                    bv[0] = b4.x; bv[1] = b4.y; bv[2] = b4.z; bv[3] = b4.w;
+                } else {
+                    const float2 b2 = *reinterpret_cast<const float2 *>(&Bs[kk][2 * lane_n]);
+                    bv[0] = b2.x; bv[1] = b2.y;
+                }
             }
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+            for (int i = 0; i < TMR; ++i)
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                for (int j = 0; j < TN; ++j) {
                     if constexpr (WIDE) part[i][j] = fmaf(av[i], bv[j], part[i][j]);
                     else acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
                 }
         }
         if constexpr (WIDE) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+            for (int i = 0; i < TMR; ++i)
 #pragma unroll
-                for (int j = 0; j < 4; ++j) acc[i][j].add(part[i][j]);
+                for (int j = 0; j < TN; ++j) acc[i][j].add(part[i][j]);
         }
         __syncthreads();
     }
 
     // ---- store ---------------------------------------------------------------------------------------------
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < TMR; ++i) {
         const int64_t m = m0 + (MODE == DW ? 4 * lane_m + i : lane_m + 16 * i);
         if (m >= g.Mg) continue;
         int64_t row_base = 0;      // FWD: offset of y[n, 0, p, q];  DX: offset of dx[n, 0, i, j]
         if (MODE == FWD) row_base = (m / PQ) * (int64_t)g.O * PQ + m % PQ;
         if (MODE == DX) row_base = (m / HW) * (int64_t)g.C * HW + m % HW;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int64_t n = n0 + (MODE == DW ? lane_n + 16 * j : 4 * lane_n + j);
+        for (int j = 0; j < TN; ++j) {
+            const int64_t n = n0 + (MODE == DW ? lane_n + 16 * j : TN * lane_n + j);
             if (n >= g.Ng) continue;
             float bv = 0.0f;
             if (MODE == FWD && g.bias) bv = g.bias_bf16 ? __bfloat162float(((const __nv_bfloat16 *)g.bias)[n]) : ((const float *)g.bias)[n];
@@ -285,9 +298,9 @@ bool fits_int(const ConvDims &d)
            d.O * d.R * d.S <= lim && d.Nb * d.P * d.Q <= (1ll << 40) && d.Nb * d.H * d.W <= (1ll << 40);
 }
 
-relay_status_t grid_of(const IgemmArgs &g, int slices, dim3 *grid)
+relay_status_t grid_of(const IgemmArgs &g, int bm, int bn, int slices, dim3 *grid)
 {
-    const int64_t gx = (g.Mg + BM - 1) / BM, gy = (g.Ng + BN - 1) / BN;
+    const int64_t gx = (g.Mg + bm - 1) / bm, gy = (g.Ng + bn - 1) / bn;
     if (gx > 2147483647ll || gy > 65535 || slices > 65535) return fail(RELAY_ERR_UNSUPPORTED, "conv2d: extent exceeds the grid limit");
     *grid = dim3((unsigned)gx, (unsigned)gy, (unsigned)slices);
     return RELAY_OK;
@@ -296,20 +309,37 @@ relay_status_t grid_of(const IgemmArgs &g, int slices, dim3 *grid)
 // slices of the weight gradient's sum: enough blocks for two per SM, at least four k-blocks per slice
 int dw_slices(const ConvDims &d)
 {
-    const int64_t tiles = ((d.O + BM - 1) / BM) * ((d.C * d.R * d.S + BN - 1) / BN);
+    const int64_t tiles = ((d.O + 63) / 64) * ((d.C * d.R * d.S + 63) / 64);
     const int64_t Kg = d.Nb * d.P * d.Q;
     const int64_t by_work = std::max<int64_t>(1, Kg / (4 * BK));
     return (int)std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(by_work, 4096), (2 * 148 + tiles - 1) / tiles));
 }
 
-template <int MODE>
-void launch_mode(const ConvDims &d, const IgemmArgs &g, dim3 grid, cudaStream_t st)
+template <int MODE, int TMR, int TN>
+void launch_tile(const ConvDims &d, const IgemmArgs &g, dim3 grid, cudaStream_t st)
 {
     const bool bf = d.dt == RELAY_BF16, s1 = d.stride == 1;
-    if (bf && s1) conv_igemm_kernel<__nv_bfloat16, MODE, true, true><<<grid, 256, 0, st>>>(g);
-    else if (bf) conv_igemm_kernel<__nv_bfloat16, MODE, true, false><<<grid, 256, 0, st>>>(g);
-    else if (s1) conv_igemm_kernel<float, MODE, false, true><<<grid, 256, 0, st>>>(g);
-    else conv_igemm_kernel<float, MODE, false, false><<<grid, 256, 0, st>>>(g);
+    if (bf && s1) conv_igemm_kernel<__nv_bfloat16, MODE, true, true, TMR, TN><<<grid, 256, 0, st>>>(g);
+    else if (bf) conv_igemm_kernel<__nv_bfloat16, MODE, true, false, TMR, TN><<<grid, 256, 0, st>>>(g);
+    else if (s1) conv_igemm_kernel<float, MODE, false, true, TMR, TN><<<grid, 256, 0, st>>>(g);
+    else conv_igemm_kernel<float, MODE, false, false, TMR, TN><<<grid, 256, 0, st>>>(g);
+}
+
+// FWD and DX: 32 columns per tile when the output has at most 32 channels, 32 rows per tile while 64-row tiles
+// would leave SMs without two blocks
+template <int MODE>
+relay_status_t launch_rows_cols(const ConvDims &d, const IgemmArgs &g, cudaStream_t st)
+{
+    const bool narrow = g.Ng <= 32;
+    const int bn = narrow ? 32 : 64;
+    const bool low = ((g.Mg + 63) / 64) * ((g.Ng + bn - 1) / bn) < 2 * 148;
+    dim3 grid;
+    RELAY_TRY(grid_of(g, low ? 32 : 64, bn, 1, &grid));
+    if (low && narrow) launch_tile<MODE, 2, 2>(d, g, grid, st);
+    else if (low) launch_tile<MODE, 2, 4>(d, g, grid, st);
+    else if (narrow) launch_tile<MODE, 4, 2>(d, g, grid, st);
+    else launch_tile<MODE, 4, 4>(d, g, grid, st);
+    return RELAY_OK;
 }
 
 }  // namespace
@@ -328,9 +358,7 @@ relay_status_t launch_conv_fwd_direct(const ConvDims &d, const void *x, const vo
     g.Mg = d.Nb * d.P * d.Q; g.Ng = d.O; g.Kg = d.C * d.R * d.S;
     g.k_per_slice = (int)((g.Kg + BK - 1) / BK * BK);
     g.a = x; g.b = w; g.out = y; g.bias = b; g.bias_bf16 = b_dt == RELAY_BF16; g.act = act;
-    dim3 grid;
-    RELAY_TRY(grid_of(g, 1, &grid));
-    launch_mode<FWD>(d, g, grid, st);
+    RELAY_TRY(launch_rows_cols<FWD>(d, g, st));
     return check_launch("conv_igemm_fwd");
 }
 
@@ -342,9 +370,7 @@ relay_status_t launch_conv_dx_direct(const ConvDims &d, const void *dz, const vo
     g.Mg = d.Nb * d.H * d.W; g.Ng = d.C; g.Kg = d.O * d.R * d.S;
     g.k_per_slice = (int)((g.Kg + BK - 1) / BK * BK);
     g.a = dz; g.b = w; g.out = dx;
-    dim3 grid;
-    RELAY_TRY(grid_of(g, 1, &grid));
-    launch_mode<DX>(d, g, grid, st);
+    RELAY_TRY(launch_rows_cols<DX>(d, g, st));
     return check_launch("conv_igemm_dx");
 }
 
@@ -360,8 +386,8 @@ relay_status_t launch_conv_dw_direct(const ConvDims &d, const void *dz, const vo
     const int slices = g.Kg == 0 ? 1 : (int)((g.Kg + g.k_per_slice - 1) / g.k_per_slice);     // <= want
     g.a = dz; g.b = x; g.out = partials;
     dim3 grid;
-    RELAY_TRY(grid_of(g, slices, &grid));
-    launch_mode<DW>(d, g, grid, st);
+    RELAY_TRY(grid_of(g, 64, 64, slices, &grid));
+    launch_tile<DW, 4, 4>(d, g, grid, st);
     RELAY_TRY(check_launch("conv_igemm_dw"));
     const unsigned rb = (unsigned)((total + 255) / 256);
     if (d.dt == RELAY_BF16) conv_dw_reduce_kernel<<<rb, 256, 0, st>>>(partials, slices, total, (__nv_bfloat16 *)dw);
