@@ -272,15 +272,23 @@ __global__ void __launch_bounds__(256, 2) conv_igemm_kernel(const IgemmArgs g)
     }
 }
 
-// dw[e] = sum over slices of part[slice][e], in slice order
+// dw[e] = sum over slices of part[slice][e], in a fixed order: one warp per element, lane l adds the slices
+// l, l + 32, ... (independent loads, one round trip), then the lanes are combined by a fixed shuffle tree
 template <typename T>
 __global__ void __launch_bounds__(256) conv_dw_reduce_kernel(const float *__restrict__ part, int n_slices, int64_t total, T *__restrict__ dw)
 {
-    const int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    const int lane = threadIdx.x & 31;
+    const int64_t e = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     if (e >= total) return;
     PairSum s;
-    for (int z = 0; z < n_slices; ++z) s.add(part[(int64_t)z * total + e]);
-    stf(dw, e, (float)s.value());
+    for (int z = lane; z < n_slices; z += 32) s.add(part[(int64_t)z * total + e]);
+#pragma unroll
+    for (int k = 16; k > 0; k >>= 1) {
+        const float oh = __shfl_down_sync(0xffffffffu, s.hi, k), ol = __shfl_down_sync(0xffffffffu, s.lo, k);
+        s.add(oh);
+        s.lo += ol;
+    }
+    if (lane == 0) stf(dw, e, (float)s.value());
 }
 
 IgemmArgs base_args(const ConvDims &d)
@@ -389,7 +397,7 @@ relay_status_t launch_conv_dw_direct(const ConvDims &d, const void *dz, const vo
     RELAY_TRY(grid_of(g, 64, 64, slices, &grid));
     launch_tile<DW, 4, 4>(d, g, grid, st);
     RELAY_TRY(check_launch("conv_igemm_dw"));
-    const unsigned rb = (unsigned)((total + 255) / 256);
+    const unsigned rb = (unsigned)((total + 7) / 8);
     if (d.dt == RELAY_BF16) conv_dw_reduce_kernel<<<rb, 256, 0, st>>>(partials, slices, total, (__nv_bfloat16 *)dw);
     else conv_dw_reduce_kernel<<<rb, 256, 0, st>>>(partials, slices, total, (float *)dw);
     return check_launch("conv_dw_reduce");
