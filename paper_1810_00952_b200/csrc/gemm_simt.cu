@@ -11,20 +11,21 @@
 
 namespace relay {
 
-constexpr int BN = 64, BK = 32, KSUB = 16;
+constexpr int BK = 32, KSUB = 16;
 
 template <typename T> __device__ __forceinline__ float to_f(T v);
 template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
 
-// block tile (16 * TM) x 64, thread tile TM x 4: TM = 4 for large outputs, TM = 1 for outputs of at most 16 rows
-// (all 256 threads then hold live outputs instead of one warp's worth) and for grids that would not fill the SMs.  The loads of k-block i+1 are issued
+// block tile (16 * TM) x (16 * TN), thread tile TM x TN: 64 x 64 for large outputs; 16 x 64, 16 x 32 or 16 x 16
+// for outputs whose grid of larger tiles would not give every SM a block.  The loads of k-block i+1 are issued
 // into registers before the arithmetic of k-block i, all of a thread's loads back to back, so that one
 // memory round trip per k-block is exposed at most.
-template <typename TIN, typename TOUT, bool FAST, int TM>
+template <typename TIN, typename TOUT, bool FAST, int TM, int TN>
 __global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmDesc g)
 {
-    constexpr int BM = 16 * TM;
+    static_assert(TM == 1 || TN == 4, "the large tile is 64 x 64");
+    constexpr int BM = 16 * TM, BN = 16 * TN;
     constexpr int A_LD = BM * BK / 256, B_LD = BN * BK / 256;
     __shared__ __align__(16) float As[BK][BM + 4];     // rows of whole 16-byte vectors: a thread's four values are one load
     __shared__ __align__(16) float Bs[BK][BN + 4];
@@ -32,10 +33,10 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmDesc g)
     const TIN *B = (const TIN *)g.b;
     const int tid = threadIdx.x;
     const int64_t m0 = (int64_t)blockIdx.x * BM, n0 = (int64_t)blockIdx.y * BN;
-    const int tm = (tid / 16) * TM, tn = (tid % 16) * 4;
+    const int tm = (tid / 16) * TM, tn = (tid % 16) * TN;
     constexpr bool F64 = sizeof(TIN) == 4;
     using Acc = typename std::conditional<F64, PairSum, float>::type;
-    Acc acc[TM][4] = {};
+    Acc acc[TM][TN] = {};
     // loader index order follows the unit stride of each operand so that loads coalesce
     const bool a_k_fast = g.a_sk == 1, b_n_fast = g.b_sn == 1;
     float ra[A_LD], rb[B_LD];
@@ -73,10 +74,10 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmDesc g)
         if (m0 + tm < g.M && n0 + tn < g.N) {
 #pragma unroll 1
             for (int ks = 0; ks < BK; ks += KSUB) {
-                float part[TM][4] = {};
+                float part[TM][TN] = {};
 #pragma unroll
                 for (int kk = ks; kk < ks + KSUB; ++kk) {
-                    float av[TM], bv[4];
+                    float av[TM], bv[TN];
                     if constexpr (TM == 4) {
                         const float4 a4 = *reinterpret_cast<const float4 *>(&As[kk][tm]);
                         av[0] = a4.x; av[1] = a4.y; av[2] = a4.z; av[3] = a4.w;
@@ -84,12 +85,19 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmDesc g)
 #pragma unroll
                         for (int i = 0; i < TM; ++i) av[i] = As[kk][tm + i];
                     }
-                    const float4 b4 = *reinterpret_cast<const float4 *>(&Bs[kk][tn]);
-                    bv[0] = b4.x; bv[1] = b4.y; bv[2] = b4.z; bv[3] = b4.w;
+                    if constexpr (TN == 4) {
+                        const float4 b4 = *reinterpret_cast<const float4 *>(&Bs[kk][tn]);
+                        bv[0] = b4.x; bv[1] = b4.y; bv[2] = b4.z; bv[3] = b4.w;
+                    } else if constexpr (TN == 2) {
+                        const float2 b2 = *reinterpret_cast<const float2 *>(&Bs[kk][tn]);
+                        bv[0] = b2.x; bv[1] = b2.y;
+                    } else {
+                        bv[0] = Bs[kk][tn];
+                    }
 #pragma unroll
                     for (int i = 0; i < TM; ++i)
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
+                        for (int j = 0; j < TN; ++j) {
                             if constexpr (F64) part[i][j] = fmaf(av[i], bv[j], part[i][j]);
                             else acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
                         }
@@ -98,7 +106,7 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmDesc g)
 #pragma unroll
                     for (int i = 0; i < TM; ++i)
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) acc[i][j].add(part[i][j]);
+                        for (int j = 0; j < TN; ++j) acc[i][j].add(part[i][j]);
                 }
             }
         }
@@ -110,7 +118,7 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmDesc g)
         int64_t m = m0 + tm + i;
         if (m >= g.M) continue;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < TN; ++j) {
             int64_t n = n0 + tn + j;
             if (n >= g.N) continue;
             float z;
@@ -124,15 +132,15 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmDesc g)
     }
 }
 
-template <int TM>
-static relay_status_t launch_tm(const GemmDesc &g, cudaStream_t st)
+template <int TM, int TN>
+static relay_status_t launch_tile(const GemmDesc &g, cudaStream_t st)
 {
-    constexpr int BM = 16 * TM;
+    constexpr int BM = 16 * TM, BN = 16 * TN;
     dim3 grid((unsigned)((g.M + BM - 1) / BM), (unsigned)((g.N + BN - 1) / BN));
     if (grid.y > 65535) return fail(RELAY_ERR_UNSUPPORTED, "SIMT contraction: N = %lld exceeds the grid limit", (long long)g.N);
-    if (g.in_dtype == RELAY_F32 && g.out_dtype == RELAY_F32) gemm_simt_kernel<float, float, false, TM><<<grid, 256, 0, st>>>(g);
-    else if (g.in_dtype == RELAY_BF16 && g.out_dtype == RELAY_BF16) gemm_simt_kernel<__nv_bfloat16, __nv_bfloat16, true, TM><<<grid, 256, 0, st>>>(g);
-    else if (g.in_dtype == RELAY_BF16 && g.out_dtype == RELAY_F32) gemm_simt_kernel<__nv_bfloat16, float, false, TM><<<grid, 256, 0, st>>>(g);
+    if (g.in_dtype == RELAY_F32 && g.out_dtype == RELAY_F32) gemm_simt_kernel<float, float, false, TM, TN><<<grid, 256, 0, st>>>(g);
+    else if (g.in_dtype == RELAY_BF16 && g.out_dtype == RELAY_BF16) gemm_simt_kernel<__nv_bfloat16, __nv_bfloat16, true, TM, TN><<<grid, 256, 0, st>>>(g);
+    else if (g.in_dtype == RELAY_BF16 && g.out_dtype == RELAY_F32) gemm_simt_kernel<__nv_bfloat16, float, false, TM, TN><<<grid, 256, 0, st>>>(g);
     else return fail(RELAY_ERR_UNSUPPORTED, "SIMT contraction: %s -> %s has no instance", dtype_name(g.in_dtype), dtype_name(g.out_dtype));
     return check_launch("gemm_simt");
 }
@@ -140,10 +148,13 @@ static relay_status_t launch_tm(const GemmDesc &g, cudaStream_t st)
 relay_status_t launch_gemm_simt(const GemmDesc &g, cudaStream_t st)
 {
     if (g.M == 0 || g.N == 0) return RELAY_OK;
-    // 16-row tiles while 64-row tiles would leave SMs without a block: a block of the small tile spends a k-block
-    // mostly waiting for its loads, so more and lighter blocks finish sooner
-    const int64_t big_tiles = ((g.M + 63) / 64) * ((g.N + BN - 1) / BN);
-    return (g.M <= 16 || big_tiles < 2 * 148) ? launch_tm<1>(g, st) : launch_tm<4>(g, st);
+    // The largest tile whose grid still gives every SM a block: with few warps on an SM a block's time goes to waiting
+    // for its own shared-memory reads, so while SMs are idle more and lighter blocks finish sooner.
+    auto tiles = [&](int bm, int bn) { return ((g.M + bm - 1) / bm) * ((g.N + bn - 1) / bn); };
+    if (g.M > 16 && tiles(64, 64) >= 2 * 148) return launch_tile<4, 4>(g, st);
+    if (tiles(16, 64) >= 148) return launch_tile<1, 4>(g, st);
+    if (tiles(16, 32) >= 148) return launch_tile<1, 2>(g, st);
+    return launch_tile<1, 1>(g, st);
 }
 
 }  // namespace relay
