@@ -63,8 +63,8 @@ __device__ __forceinline__ void advance(int &c, int &r, int &s, int step, int R,
     }
 }
 
-// TMR x TN outputs per thread: 4 x 4 in general; FWD and DX also come with 2 rows (twice the blocks when the grid
-// would leave SMs idle) and with 2 columns (few output channels: less arithmetic on padding)
+// TMR x TN outputs per thread: 4 x 4 in general; FWD and DX also come with 2 or 1 rows (more blocks when the grid
+// would leave SMs idle) and with 2 or 1 columns (few output channels: less arithmetic on padding)
 template <typename T, int MODE, bool FAST, bool STRIDE1, int TMR, int TN>
 __global__ void __launch_bounds__(256, 2) conv_igemm_kernel(const IgemmArgs g)
 {
@@ -226,9 +226,11 @@ __global__ void __launch_bounds__(256, 2) conv_igemm_kernel(const IgemmArgs g)
                 if constexpr (TN == 4) {
                     const float4 b4 = *reinterpret_cast<const float4 *>(&Bs[kk][4 * lane_n]);
                     bv[0] = b4.x; bv[1] = b4.y; bv[2] = b4.z; bv[3] = b4.w;
-                } else {
+                } else if constexpr (TN == 2) {
                     const float2 b2 = *reinterpret_cast<const float2 *>(&Bs[kk][2 * lane_n]);
                     bv[0] = b2.x; bv[1] = b2.y;
+                } else {
+                    bv[0] = Bs[kk][lane_n];
                 }
             }
 #pragma unroll
@@ -333,21 +335,27 @@ void launch_tile(const ConvDims &d, const IgemmArgs &g, dim3 grid, cudaStream_t 
     else conv_igemm_kernel<float, MODE, false, false, TMR, TN><<<grid, 256, 0, st>>>(g);
 }
 
-// FWD and DX: 32 columns per tile when the output has at most 32 channels, 32 rows per tile while 64-row tiles
-// would leave SMs without two blocks
+// FWD and DX: the tile is as wide as the output channels need (16, 32 or 64 columns) and as tall (64, 32 or 16 rows)
+// as still gives every SM a block: with few warps on an SM a block's time goes to waiting for its own
+// shared-memory reads, so while SMs are idle more and lighter blocks finish sooner
+template <int MODE, int TN>
+relay_status_t launch_rows(const ConvDims &d, const IgemmArgs &g, cudaStream_t st)
+{
+    const int64_t cols = (g.Ng + 16 * TN - 1) / (16 * TN);
+    auto blocks = [&](int bm) { return ((g.Mg + bm - 1) / bm) * cols; };
+    dim3 grid;
+    if (blocks(64) >= 148) { RELAY_TRY(grid_of(g, 64, 16 * TN, 1, &grid)); launch_tile<MODE, 4, TN>(d, g, grid, st); }
+    else if (blocks(32) >= 148) { RELAY_TRY(grid_of(g, 32, 16 * TN, 1, &grid)); launch_tile<MODE, 2, TN>(d, g, grid, st); }
+    else { RELAY_TRY(grid_of(g, 16, 16 * TN, 1, &grid)); launch_tile<MODE, 1, TN>(d, g, grid, st); }
+    return RELAY_OK;
+}
+
 template <int MODE>
 relay_status_t launch_rows_cols(const ConvDims &d, const IgemmArgs &g, cudaStream_t st)
 {
-    const bool narrow = g.Ng <= 32;
-    const int bn = narrow ? 32 : 64;
-    const bool low = ((g.Mg + 63) / 64) * ((g.Ng + bn - 1) / bn) < 2 * 148;
-    dim3 grid;
-    RELAY_TRY(grid_of(g, low ? 32 : 64, bn, 1, &grid));
-    if (low && narrow) launch_tile<MODE, 2, 2>(d, g, grid, st);
-    else if (low) launch_tile<MODE, 2, 4>(d, g, grid, st);
-    else if (narrow) launch_tile<MODE, 4, 2>(d, g, grid, st);
-    else launch_tile<MODE, 4, 4>(d, g, grid, st);
-    return RELAY_OK;
+    if (g.Ng <= 16) return launch_rows<MODE, 1>(d, g, st);
+    if (g.Ng <= 32) return launch_rows<MODE, 2>(d, g, st);
+    return launch_rows<MODE, 4>(d, g, st);
 }
 
 }  // namespace
