@@ -618,6 +618,13 @@ def main():
         rooflines["conv2d forward group (repack + conv_fprop_tc_kernel)"] = {
             "bound": "tensor", "achieved": a, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": a / peaks["bf16_tflops"],
             "traffic": traffic_of("conv_fprop_tc2_kernel"), "peak_source": peaks["source"] + " (burst, of measured)"}
+    for key, name in (("cfg4.grad", "conv2d gradient group (repacks + conv_fprop_tc_kernel on dZ + conv_wgrad_tc_kernel + reduce)"),
+                      ("next.conv_nhwc", "conv2d forward group, NHWC-tagged tensors (conv_fprop_tc_kernel storing NHWC tiles)"),
+                      ("next.conv_nhwc_grad", "conv2d gradient group, NHWC-tagged tensors")):
+        if key in table:
+            a = table[key]["tflops"]
+            rooflines[name] = {"bound": "tensor", "achieved": a, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": a / peaks["bf16_tflops"],
+                               "traffic": None, "peak_source": peaks["source"] + " (burst, of measured)"}
     for key, name in (("cfg2.fwd", "ewise2d_kernel<tanh_affine_residual_fwd>"), ("cfg2.grad", "ewise2d_kernel<tanh_affine_residual_grad> + finalize")):
         if key in table:
             a = table[key]["gbs"]
