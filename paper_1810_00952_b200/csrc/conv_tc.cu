@@ -44,11 +44,39 @@ constexpr int TMEM_COLS = 512;
 // 64 channels x 64 pixels per block, 16-byte global accesses on both sides (HW % 8 == 0, C % 8 == 0).
 // GRAD with db_part != null also writes, per block, the sums over its 64 pixels of the stored (rounded) dZ
 // of each of its 64 channels to db_part[(n * gridDim.x + blockIdx.x) * C + c]: the bias gradient's partials.
+// Weight packing that rides along with a repack launch: the z-slices of the grid beyond `n_img` pack the weights
+// (one output element per thread, as pack_weights_kernel below), so the 1 MB job costs no launch of its own.
+struct PackJob {
+    const __nv_bfloat16 *w;    // null: nothing to pack
+    __nv_bfloat16 *wf, *wb;    // wf[o][tap][c], wb[c][mirror(tap)][o]; either may be null
+    int O, C, taps, n_img;
+};
+
+__device__ __forceinline__ void pack_one(const PackJob &j, unsigned i)
+{
+    const unsigned taps = j.taps, total = (unsigned)j.O * j.C * taps;
+    if (i >= total) return;
+    if (j.wf) {
+        const unsigned c = i % j.C, t = i / j.C, tap = t % taps, o = t / taps;
+        j.wf[i] = j.w[(o * j.C + c) * taps + tap];
+    }
+    if (j.wb) {
+        const unsigned o = i % j.O, t = i / j.O, tap2 = t % taps, c = t / taps;
+        j.wb[i] = j.w[(o * j.C + c) * taps + (taps - 1 - tap2)];
+    }
+}
+
 template <bool GRAD>
 __global__ void __launch_bounds__(256) nchw_to_nhwc_kernel(const __nv_bfloat16 *__restrict__ in, const __nv_bfloat16 *__restrict__ y,
                                                             __nv_bfloat16 *__restrict__ out, int C, int HW, int act,
-                                                            float *__restrict__ db_part)
+                                                            float *__restrict__ db_part, const PackJob job)
 {
+    if (job.w != nullptr && (int)blockIdx.z >= job.n_img) {        // whole blocks: no barrier is skipped by part of a block
+        pdl_wait();
+        const unsigned blk = (((unsigned)blockIdx.z - job.n_img) * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
+        pack_one(job, blk * 256u + threadIdx.x);
+        return;
+    }
     // [pixel][channel]; 33 words per row: the scattered 2-byte stores below are at most 2-way conflicted and
     // the 4-byte reads of the write phase are conflict-free
     __shared__ __align__(16) __nv_bfloat16 tile[64][66];
@@ -931,12 +959,21 @@ relay_status_t launch_fprop(const ConvDims &d, const TcPlan &pl, const void *act
     return check_launch("conv_fprop_tc");
 }
 
+// `w` (optional): the same launch also packs the O x Cw x 3 x 3 weights into wf and / or wb
 relay_status_t launch_transpose(bool grad, const void *in, const void *y, void *out, int64_t Nb, int64_t C, int64_t HW, int act,
-                                float *db_part, cudaStream_t st)
+                                float *db_part, cudaStream_t st, const void *w = nullptr, void *wf = nullptr, void *wb = nullptr,
+                                int64_t O = 0, int64_t Cw = 0)
 {
     dim3 grid((unsigned)((HW + 63) / 64), (unsigned)((C + 63) / 64), (unsigned)Nb);
-    if (grad) RELAY_CUDA(launch_pdl(nchw_to_nhwc_kernel<true>, grid, dim3(256), 0, st, (const __nv_bfloat16 *)in, (const __nv_bfloat16 *)y, (__nv_bfloat16 *)out, (int)C, (int)HW, act, db_part));
-    else RELAY_CUDA(launch_pdl(nchw_to_nhwc_kernel<false>, grid, dim3(256), 0, st, (const __nv_bfloat16 *)in, (const __nv_bfloat16 *)nullptr, (__nv_bfloat16 *)out, (int)C, (int)HW, act, (float *)nullptr));
+    PackJob job{};
+    if (w != nullptr) {
+        job.w = (const __nv_bfloat16 *)w; job.wf = (__nv_bfloat16 *)wf; job.wb = (__nv_bfloat16 *)wb;
+        job.O = (int)O; job.C = (int)Cw; job.taps = 9; job.n_img = (int)Nb;
+        const int64_t per_slice = (int64_t)grid.x * grid.y * 256;
+        grid.z += (unsigned)((O * Cw * 9 + per_slice - 1) / per_slice);
+    }
+    if (grad) RELAY_CUDA(launch_pdl(nchw_to_nhwc_kernel<true>, grid, dim3(256), 0, st, (const __nv_bfloat16 *)in, (const __nv_bfloat16 *)y, (__nv_bfloat16 *)out, (int)C, (int)HW, act, db_part, job));
+    else RELAY_CUDA(launch_pdl(nchw_to_nhwc_kernel<false>, grid, dim3(256), 0, st, (const __nv_bfloat16 *)in, (const __nv_bfloat16 *)nullptr, (__nv_bfloat16 *)out, (int)C, (int)HW, act, (float *)nullptr, job));
     return check_launch("nchw_to_nhwc");
 }
 
@@ -985,11 +1022,13 @@ relay_status_t launch_conv_fwd_tc(const ConvDims &d, const void *x, bool x_is_nh
     void *wf = base + pl.x_nhwc;
     const void *x_nhwc = x;
     if (!x_is_nhwc) {
-        RELAY_TRY(launch_transpose(false, x, nullptr, base, d.Nb, d.C, d.H * d.W, 0, nullptr, st));
+        // the repack launch packs the weights as well
+        RELAY_TRY(launch_transpose(false, x, nullptr, base, d.Nb, d.C, d.H * d.W, 0, nullptr, st, w, wf, nullptr, d.O, d.C));
         x_nhwc = base;
+    } else {
+        RELAY_CUDA(launch_pdl(pack_weights_kernel, dim3((unsigned)((d.O * d.C * 9 + 255) / 256)), dim3(256), 0, st, (const __nv_bfloat16 *)w, (__nv_bfloat16 *)wf, (__nv_bfloat16 *)nullptr, (int)d.O, (int)d.C, 3, 3));
+        RELAY_TRY(check_launch("pack_weights"));
     }
-    RELAY_CUDA(launch_pdl(pack_weights_kernel, dim3((unsigned)((d.O * d.C * 9 + 255) / 256)), dim3(256), 0, st, (const __nv_bfloat16 *)w, (__nv_bfloat16 *)wf, (__nv_bfloat16 *)nullptr, (int)d.O, (int)d.C, 3, 3));
-    RELAY_TRY(check_launch("pack_weights"));
     if (!y_nhwc) return launch_fprop(d, pl, x_nhwc, (int)d.C, wf, (int)d.O, b, b_dt, act, y, st);
     if (fprop_pair_form(d, pl, (int)d.O, sm_count())) return launch_fprop(d, pl, x_nhwc, (int)d.C, wf, (int)d.O, b, b_dt, act, y_nhwc, st, true);
     RELAY_TRY(launch_fprop(d, pl, x_nhwc, (int)d.C, wf, (int)d.O, b, b_dt, act, y, st));
@@ -1015,13 +1054,16 @@ relay_status_t launch_conv_grad_tc(const ConvDims &d, const void *x, const void 
     } else {
         // dZ = dy (.) act'(y), written straight into NHWC; x into NHWC
         // (the same pass leaves per-block partial sums of dZ over pixels for the bias gradient)
-        RELAY_TRY(launch_transpose(true, dy, y, dz_nhwc, d.Nb, d.O, HW, act, db ? db_part : nullptr, st));
+        // (the same launch packs the mirrored weights that the input gradient needs)
+        RELAY_TRY(launch_transpose(true, dy, y, dz_nhwc, d.Nb, d.O, HW, act, db ? db_part : nullptr, st, dx ? w : nullptr, nullptr, wb, d.O, d.C));
         RELAY_TRY(launch_transpose(false, x, nullptr, base, d.Nb, d.C, HW, 0, nullptr, st));
         if (db) RELAY_TRY(launch_colsum_finalize(db_part, (int)(d.Nb * ((HW + 63) / 64)), d.O, 1.0f, db, st));
     }
     if (dx) {
-        RELAY_CUDA(launch_pdl(pack_weights_kernel, dim3((unsigned)((d.O * d.C * 9 + 255) / 256)), dim3(256), 0, st, (const __nv_bfloat16 *)w, (__nv_bfloat16 *)nullptr, (__nv_bfloat16 *)wb, (int)d.O, (int)d.C, 3, 3));
-        RELAY_TRY(check_launch("pack_weights"));
+        if (nhwc_in) {
+            RELAY_CUDA(launch_pdl(pack_weights_kernel, dim3((unsigned)((d.O * d.C * 9 + 255) / 256)), dim3(256), 0, st, (const __nv_bfloat16 *)w, (__nv_bfloat16 *)nullptr, (__nv_bfloat16 *)wb, (int)d.O, (int)d.C, 3, 3));
+            RELAY_TRY(check_launch("pack_weights"));
+        }
         if (dx_nhwc && fprop_pair_form(d, pl, (int)d.C, sm_count())) {
             RELAY_TRY(launch_fprop(d, pl, dz_nhwc, (int)d.O, wb, (int)d.C, nullptr, RELAY_F32, RELAY_ACT_NONE, dx_nhwc, st, true));
         } else {
