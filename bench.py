@@ -34,6 +34,7 @@ import torch  # noqa: E402
 
 METRIC = "fused-group TFLOP/s (dense/conv) and HBM GB/s (ewise/reduce) on 1 B200 vs roofline"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL_PEAKS = {"hbm_gbs": 7700.0, "bf16_tflops": 2250.0}      # data-sheet figures (HGX B200, dense bf16), for context
 ALL_GROUPS = ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "next"]
 
 
@@ -221,6 +222,14 @@ class Workload:
             self.grad_specs = [(ids[0], B.RED_NONE, 0, 0), (ids[1], B.RED_SUM, 1, 0), (ids[2], B.RED_SUM, 1, 1)]
             d = self.devt["cfg2"]
             ws_bytes = max(ws_bytes, B.relay_workspace_bytes_reduce([d["dout"], d["x"], d["a"], d["b"]], self.grad_specs))
+        if "cfg2" in groups:
+            # standalone reductions of the same [rows, cols] bf16 tensor: over the last axis (sum, max, argmax) and over axis 0
+            r, c = self.host["cfg2"]["x"].shape
+            self.red_prog = P.Program([P.BF16])
+            self.red_out = dict(sum1=E(r, dt=f32), max1=E(r, dt=f32), arg1=E(r, dt=torch.int64), sum0=E(c, dt=f32))
+            self.red_specs = dict(sum1=[(0, B.RED_SUM, 2, 0)], max1=[(0, B.RED_MAX, 2, 0)], arg1=[(0, B.RED_ARGMAX, 2, 0)],
+                                  sum0=[(0, B.RED_SUM, 1, 0)])
+            ws_bytes = max(ws_bytes, B.relay_workspace_bytes_reduce([self.devt["cfg2"]["x"]], self.red_specs["sum0"]))
         if "cfg3" in groups:
             m, k = self.host["cfg3"]["x"].shape
             o = dict()
@@ -244,6 +253,7 @@ class Workload:
             # upstream partials of the gradient program (device-resident, generated once)
             self.lstm_dh_all = I.normal(5, 8, (T, Bn, H), 1.0, f32).to(dev)
             self.lstm_dc_fin = I.normal(5, 9, (Bn, H), 1.0, f32).to(dev)
+            self.lstm_zx = E(T * Bn, 4 * H, dt=f32)       # the batched input contraction alone (not a result of the step)
             ws_bytes = max(ws_bytes, B.relay_workspace_bytes_lstm(d["x"], d["w_ih"], d["w_hh"]),
                            B.relay_workspace_bytes_lstm_grad(d["x"], d["w_ih"], d["w_hh"]))
         if "next" in groups:
@@ -345,6 +355,11 @@ class Workload:
             with tm.region("cfg2.grad"):
                 B.relay_fused_reduce(self.grad_prog.arrays(), [d["dout"], d["x"], d["a"], d["b"]], self.grad_specs,
                                      [o["dx"], o["da"], o["db"]], ws)
+            ra = self.red_prog.arrays()
+            for key in ("sum1", "max1", "arg1", "sum0"):
+                self.flush_l2()
+                with tm.region("a8." + key):
+                    B.relay_fused_reduce(ra, [d["x"]], self.red_specs[key], [self.red_out[key]], ws)
         if "cfg3" in self.groups:
             d, o = self.devt["cfg3"], self.out["cfg3"]
             self.flush_l2()
@@ -359,11 +374,17 @@ class Workload:
                     B.relay_fused_dense_act_grad(acts[l], d[f"w{l}"], acts[l + 1], g, B.ACT_RELU, o[f"dx{l}"], o[f"dw{l}"],
                                                  o[f"db{l}"], ws)
                     g = o[f"dx{l}"]
+            # the two gradient contractions of one layer alone, each with its operand read transposed in place
+            with tm.region("cfg3.bwd.gemm_dx"):
+                B.relay_contract_act(d["dy"], 0, d["w2"], 1, None, B.ACT_NONE, o["dx2"])
+            with tm.region("cfg3.bwd.gemm_dw"):
+                B.relay_contract_act(acts[2], 1, d["dy"], 0, None, B.ACT_NONE, o["dw2"])
         if "cfg4" in self.groups:
             d, o = self.devt["cfg4"], self.out["cfg4"]
             self.flush_l2()
             with tm.region("cfg4.fwd"):
                 B.relay_fused_conv2d_act(d["x"], d["w"], d["b"], 1, 1, B.ACT_RELU, o["y"], ws)
+            self.flush_l2()
             with tm.region("cfg4.grad"):
                 B.relay_fused_conv2d_act_grad(d["x"], d["w"], o["y"], d["dy"], 1, 1, B.ACT_RELU, o["dx"], o["dw"], o["db"], ws)
         if "cfg5" in self.groups:
@@ -371,6 +392,10 @@ class Workload:
             self.flush_l2()
             with tm.region("cfg5.lstm"):
                 B.relay_lstm_cell_seq(d["x"], d["w_ih"], d["w_hh"], d["b"], d["h0"], d["c0"], o["h_all"], o["c"], ws)
+            T_, Bn_, In_ = d["x"].shape
+            self.flush_l2()
+            with tm.region("cfg5.lstm.zx_gemm"):
+                B.relay_contract_act(d["x"].view(T_ * Bn_, In_), 0, d["w_ih"], 0, d["b"], B.ACT_NONE, self.lstm_zx)
             self.flush_l2()
             with tm.region("cfg5.lstm_grad"):
                 B.relay_lstm_cell_seq_grad(d["x"], d["w_ih"], d["w_hh"], d["b"], d["h0"], d["c0"], o["h_all"], self.lstm_dh_all,
@@ -402,6 +427,7 @@ class Workload:
             self.flush_l2()
             with tm.region("next.conv_nhwc"):
                 B.relay_fused_conv2d_act(h["x"], h["w"], h["b"], 1, 1, B.ACT_RELU, h["y"], ws, layout=B.NHWC)
+            self.flush_l2()
             with tm.region("next.conv_nhwc_grad"):
                 B.relay_fused_conv2d_act_grad(h["x"], h["w"], h["y"], h["dy"], 1, 1, B.ACT_RELU, h["dx"], h["dw"], h["db"], ws, layout=B.NHWC)
 
@@ -415,10 +441,13 @@ class Workload:
             r, c = self.host["cfg2"]["x"].shape
             w["cfg2.fwd"] = dict(bytes=2 * r * c * 2 + 2 * c * 2)
             w["cfg2.grad"] = dict(bytes=3 * r * c * 2 + 2 * c * 2 + 2 * c * 4)
+            w["a8.sum1"] = dict(bytes=r * c * 2 + r * 4); w["a8.max1"] = dict(bytes=r * c * 2 + r * 4)
+            w["a8.arg1"] = dict(bytes=r * c * 2 + r * 8); w["a8.sum0"] = dict(bytes=r * c * 2 + c * 4)
         if "cfg3" in self.groups:
             m, k = self.host["cfg3"]["x"].shape
             w["cfg3.fwd"] = dict(flop=3 * 2 * m * k * k); w["cfg3.bwd"] = dict(flop=6 * 2 * m * k * k)
             w["cfg3.fwd.layer"] = dict(flop=2 * m * k * k)
+            w["cfg3.bwd.gemm_dx"] = dict(flop=2 * m * k * k); w["cfg3.bwd.gemm_dw"] = dict(flop=2 * m * k * k)
         if "cfg4" in self.groups:
             n, c, h, wd = self.host["cfg4"]["x"].shape
             o = self.host["cfg4"]["w"].shape[0]
@@ -428,6 +457,7 @@ class Workload:
             T, Bn, In = self.host["cfg5"]["x"].shape
             H = self.host["cfg5"]["w_hh"].shape[0]
             w["cfg5.lstm"] = dict(flop=2 * T * Bn * (In + H) * 4 * H)
+            w["cfg5.lstm.zx_gemm"] = dict(flop=2 * T * Bn * In * 4 * H)
             # gradient program: gate recomputation (one forward's worth), dz w_hh^T per step, dx, dw_ih, dw_hh
             w["cfg5.lstm_grad"] = dict(flop=2 * T * Bn * (In + H) * 4 * H + 2 * T * Bn * 4 * H * (H + In) + 2 * T * Bn * 4 * H * (In + H))
         if "next" in self.groups:
@@ -447,29 +477,76 @@ class Workload:
 # ---------------------------------------------------------------------------------------------------
 # CPU oracle on a bounded sample (single thread); also the `--impl reference` arm
 # ---------------------------------------------------------------------------------------------------
-def oracle_sample(rows3=192, rows2=1024):
-    """Times the fp64 oracle, as it stands, on slices of the same workload along the independent
-    dimension.  Returns (tflops, gbs, seconds, description)."""
+def oracle_sample(rows3=192, rows2=1024, imgs4=1, rows5=2, reps1=200):
+    """Times the fp64 oracle, as it stands, single-threaded, on slices of all five configurations along their
+    independent dimension (batch rows / images; configuration 1 at full size).  Returns a dict: the aggregate rates
+    over the sampled work (TFLOP/s over the dense + conv samples, GB/s of algorithmic bytes over the elementwise
+    sample), the seconds spent, a description, and per configuration the sampled time with the full-size time it
+    extrapolates to (linear in the sliced dimension)."""
     import oracle
     from relay_workloads import inputs as I
     from relay_workloads import program as P
-    t3 = I.cfg3_mlp(batch=rows3)
+    per = {}
+    # configuration 1: full size, forward + gradient group, repeated (a single pass is microseconds)
+    t1 = I.cfg1_tiny_mlp()
+    x, w, b, dy = (I.as_f64(t1[k]) for k in ("x", "w", "b", "dy"))
+    t0 = time.perf_counter()
+    for _ in range(reps1):
+        y = oracle.dense_act(x, w, b, oracle.ACT_RELU, oracle.F32)
+        oracle.dense_act_grad(x, w, y, dy, oracle.ACT_RELU, oracle.F32, oracle.F32, oracle.F32)
+    s1 = (time.perf_counter() - t0) / reps1
+    per["cfg1"] = {"sample": "full size, forward + gradient group", "us_per_pass": s1 * 1e6, "flop": 3 * 2 * 8 * 64 * 32}
+    # configuration 2: forward and gradient group on the first rows2 rows
+    t2 = I.cfg2_ewise(rows=rows2)
+    prog, outs = P.tanh_affine_residual_fwd(P.BF16)
+    gprog, gids = P.tanh_affine_residual_grad(P.BF16)
+    ins = [I.as_f64(t2[k]) for k in ("x", "a", "b")]
+    gins = [I.as_f64(t2[k]) for k in ("dout", "x", "a", "b")]
+    t0 = time.perf_counter()
+    oracle.ewise(prog.arrays(), ins, outs)
+    s2f = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    oracle.reduce(gprog.arrays(), gins, [(gids[0], 0, (), False, oracle.BF16), (gids[1], 1, (0,), False, oracle.F32),
+                                         (gids[2], 1, (0,), True, oracle.F32)])
+    s2g = time.perf_counter() - t0
+    bytes2 = (2 + 3) * rows2 * 8192 * 2
+    per["cfg2"] = {"sample": f"first {rows2} of 8192 rows, forward + gradient group", "seconds": s2f + s2g,
+                   "full_size_seconds_extrapolated": (s2f + s2g) * 8192 / rows2, "bytes": bytes2}
+    # configuration 3: one layer forward + gradient group on the first rows3 batch rows
+    t3 = I.cfg3_mlp(batch=rows3, layers=1)
     x, w, b, dy = (I.as_f64(t3[k]) for k in ("x", "w0", "b0", "dy"))
     t0 = time.perf_counter()
     y = oracle.dense_act(x, w, b, oracle.ACT_RELU, oracle.BF16)
     oracle.dense_act_grad(x, w, y, dy, oracle.ACT_RELU, oracle.BF16, oracle.BF16, oracle.F32)
     s3 = time.perf_counter() - t0
     flop3 = 3 * 2 * rows3 * 4096 * 4096
-    t2 = I.cfg2_ewise(rows=rows2)
-    prog, outs = P.tanh_affine_residual_fwd(P.BF16)
-    ins = [I.as_f64(t2[k]) for k in ("x", "a", "b")]
+    per["cfg3"] = {"sample": f"one layer forward + gradient group on the first {rows3} of 4096 batch rows", "seconds": s3,
+                   "full_size_seconds_extrapolated": s3 * 3 * 4096 / rows3, "flop": flop3}
+    # configuration 4: forward + gradient group on the first imgs4 images
+    t4 = I.cfg4_conv(N=imgs4)
+    x, w, b, dy = (I.as_f64(t4[k]) for k in ("x", "w", "b", "dy"))
     t0 = time.perf_counter()
-    oracle.ewise(prog.arrays(), ins, outs)
-    s2 = time.perf_counter() - t0
-    bytes2 = 2 * rows2 * 8192 * 2
-    desc = (f"cfg3 layer forward+gradient on the first {rows3} batch rows ({flop3 / 1e9:.1f} GFLOP, {s3:.1f} s) and "
-            f"cfg2 forward on the first {rows2} rows ({bytes2 / 1e6:.1f} MB, {s2:.1f} s)")
-    return flop3 / s3 / 1e12, bytes2 / s2 / 1e9, s3 + s2, desc
+    y = oracle.conv2d_act(x, w, b, 1, 1, oracle.ACT_RELU, oracle.BF16)
+    oracle.conv2d_act_grad(x, w, y, dy, 1, 1, oracle.ACT_RELU, oracle.BF16, oracle.BF16, oracle.F32)
+    s4 = time.perf_counter() - t0
+    flop4 = 3 * 2 * imgs4 * 56 * 56 * 256 * 256 * 9
+    per["cfg4"] = {"sample": f"forward + dX + dW + db on the first {imgs4} of 32 images", "seconds": s4,
+                   "full_size_seconds_extrapolated": s4 * 32 / imgs4, "flop": flop4}
+    # configuration 5: the whole sequence (128 steps) for the first rows5 batch rows
+    t5 = I.cfg5_lstm(B=rows5)
+    a5 = [I.as_f64(t5[k]) for k in ("x", "w_ih", "w_hh", "b", "h0", "c0")]
+    t0 = time.perf_counter()
+    oracle.lstm_cell_seq(*a5)
+    s5 = time.perf_counter() - t0
+    flop5 = 2 * 128 * rows5 * 2048 * 4096
+    per["cfg5"] = {"sample": f"all 128 steps for the first {rows5} of 64 batch rows (forward)", "seconds": s5,
+                   "full_size_seconds_extrapolated": s5 * 64 / rows5, "flop": flop5}
+    sec = s1 * reps1 + s2f + s2g + s3 + s4 + s5
+    desc = (f"cfg1 full size x{reps1} ({s1 * 1e6:.0f} us per pass); cfg2 forward+gradient on the first {rows2} rows ({bytes2 / 1e6:.1f} MB, "
+            f"{s2f + s2g:.1f} s); cfg3 one layer forward+gradient on the first {rows3} batch rows ({flop3 / 1e9:.1f} GFLOP, {s3:.1f} s); "
+            f"cfg4 forward+gradient on the first {imgs4} image(s) ({flop4 / 1e9:.1f} GFLOP, {s4:.1f} s); cfg5 forward, 128 steps, "
+            f"first {rows5} batch rows ({flop5 / 1e9:.1f} GFLOP, {s5:.1f} s); full-size times are extrapolated linearly")
+    return {"tflops": (flop3 + flop4) / (s3 + s4) / 1e12, "gbs": bytes2 / (s2f + s2g) / 1e9, "seconds": sec, "desc": desc, "per_config": per}
 
 
 def run_reference(args, rank, world):
@@ -477,10 +554,11 @@ def run_reference(args, rank, world):
         return
     vals = []
     for i in range(args.warmup + args.steps):
-        tf, gb, sec, desc = oracle_sample(rows3=16, rows2=64)
+        r = oracle_sample(rows3=16, rows2=64, imgs4=1, rows5=1, reps1=20)
         if i >= args.warmup:
-            vals.append((tf, gb, sec))
-    tf = float(np.mean([v[0] for v in vals])); gb = float(np.mean([v[1] for v in vals])); sec = float(np.mean([v[2] for v in vals]))
+            vals.append(r)
+    tf = float(np.mean([v["tflops"] for v in vals])); gb = float(np.mean([v["gbs"] for v in vals])); sec = float(np.mean([v["seconds"] for v in vals]))
+    desc = vals[-1]["desc"] if vals else ""
     line = {"impl": "reference", "metric": METRIC, "value": tf, "unit": "TFLOP/s", "hbm_gbs": gb, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
@@ -572,7 +650,7 @@ def main():
     step_ms_max = max_over_ranks(step_ms, dist, dev)
 
     tensor_keys = [k for k in top if k.startswith(("cfg3", "cfg4"))]
-    hbm_keys = [k for k in top if k.startswith("cfg2")]
+    hbm_keys = [k for k in top if k.startswith(("cfg2", "a8"))]
     t_ms = max_over_ranks(sum(float(np.mean(tm.ms[k])) for k in tensor_keys), dist, dev)
     h_ms = max_over_ranks(sum(float(np.mean(tm.ms[k])) for k in hbm_keys), dist, dev)
     tflops = whole_job(sum(work[k]["flop"] for k in tensor_keys), world, t_ms) / 1e12 if t_ms else None
@@ -585,9 +663,11 @@ def main():
         if "flop" in work.get(k, {}):
             e["tflops"] = work[k]["flop"] / (ms * 1e-3) / 1e12
             e["frac_of_measured_bf16_peak"] = e["tflops"] / peaks["bf16_tflops"]
+            e["frac_of_nominal_bf16_peak"] = e["tflops"] / NOMINAL_PEAKS["bf16_tflops"]
         if "bytes" in work.get(k, {}):
             e["gbs"] = work[k]["bytes"] / (ms * 1e-3) / 1e9
             e["frac_of_measured_hbm"] = e["gbs"] / peaks["hbm_gbs"]
+            e["frac_of_nominal_hbm"] = e["gbs"] / NOMINAL_PEAKS["hbm_gbs"]
         table[k] = e
 
     # roofline of the dominant roofline-bound kernel: the tensor-core contraction (its three operand
@@ -613,6 +693,13 @@ def main():
             "us_per_launch": table["cfg3.fwd"]["ms"] * 1e3 / 3,
             # the launches run inside a step of several milliseconds of device work: the sustained figure for context
             "frac_of_sustained_peak": a / peaks["bf16_tflops_sustained"] if peaks.get("bf16_tflops_sustained") else None}
+    for key, name in (("cfg3.bwd.gemm_dx", "gemm_tc2_kernel, dx = dZ w^T (both operands K-major), one 4096^3 launch"),
+                      ("cfg3.bwd.gemm_dw", "gemm_tc2_kernel, dw = x^T dZ (both operands MN-major), one 4096^3 launch"),
+                      ("cfg5.lstm.zx_gemm", "gemm_tc2_kernel, zx = x W_ih + b for all T*B rows (8192 x 4096 x 1024, fp32 result)")):
+        if key in table:
+            a = table[key]["tflops"]
+            rooflines[name] = {"bound": "tensor", "achieved": a, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": a / peaks["bf16_tflops"],
+                               "traffic": None, "peak_source": peaks["source"] + " (burst, of measured)", "us_per_launch": table[key]["ms"] * 1e3}
     if "cfg4.fwd" in table:
         a = table["cfg4.fwd"]["tflops"]
         rooflines["conv2d forward group (repack + conv_fprop_tc_kernel)"] = {
@@ -626,6 +713,14 @@ def main():
             rooflines[name] = {"bound": "tensor", "achieved": a, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": a / peaks["bf16_tflops"],
                                "traffic": None, "peak_source": peaks["source"] + " (burst, of measured)"}
     for key, name in (("cfg2.fwd", "ewise2d_kernel<tanh_affine_residual_fwd>"), ("cfg2.grad", "ewise2d_kernel<tanh_affine_residual_grad> + finalize")):
+        if key in table:
+            a = table[key]["gbs"]
+            rooflines[name] = {"bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": a / peaks["hbm_gbs"],
+                               "traffic": traffic_of(key), "peak_source": peaks["source"] + " (of measured)"}
+    for key, name in (("a8.sum1", "rowreduce_kernel<sum> (8192x8192 bf16 over the last axis)"),
+                      ("a8.max1", "rowreduce_kernel<max> (8192x8192 bf16 over the last axis)"),
+                      ("a8.arg1", "rowreduce_kernel<argmax> (8192x8192 bf16 over the last axis, int64 indices)"),
+                      ("a8.sum0", "ewise2d_kernel<identity_colsum> + finalize (8192x8192 bf16 over axis 0)")):
         if key in table:
             a = table[key]["gbs"]
             rooflines[name] = {"bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": a / peaks["hbm_gbs"],
@@ -646,6 +741,8 @@ def main():
             rooflines[name] = {"bound": "tensor", "achieved": a, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": a / peaks["bf16_tflops"],
                                "traffic": None, "peak_source": peaks["source"] + " (burst, of measured)",
                                "us_per_step": table[key]["ms"] * 1e3 / 128, "note": "latency chain of dependent steps"}
+    for r_ in rooflines.values():
+        r_["frac_of_nominal"] = r_["achieved"] / NOMINAL_PEAKS["bf16_tflops" if r_["unit"] == "TFLOP/s" else "hbm_gbs"]
     if rooflines:
         first = next(iter(rooflines))
         roofline = dict(rooflines[first], kernel=first)
@@ -711,9 +808,9 @@ def main():
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        tf, gb, sec, desc = oracle_sample()
-        cpu = {"value": tf, "unit": "TFLOP/s", "hbm_gbs": gb, "cores": 1, "kind": "oracle", "sample": desc,
-               "host_cores_available": os.cpu_count()}
+        r = oracle_sample()
+        cpu = {"value": r["tflops"], "unit": "TFLOP/s", "hbm_gbs": r["gbs"], "cores": 1, "kind": "oracle", "sample": r["desc"],
+               "per_config": r["per_config"], "seconds": r["seconds"], "host_cores_available": os.cpu_count()}
 
     if rank == 0:
         line = {"metric": METRIC, "value": tflops if tflops is not None else gbs, "unit": "TFLOP/s" if tflops is not None else "GB/s",
@@ -721,15 +818,15 @@ def main():
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 (fp32 accumulate); cfg1 f32",
                 "data": "synthetic",
                 "config": {"workload": ("reduced shapes" if args.small else "all five configurations at full size")
-                           + ": step = cfg1 fwd+grad, cfg2 fwd+grad, cfg3 3-layer fwd+bwd, cfg4 conv fwd+dX+dW+db, cfg5 LSTM forward + gradient program"
+                           + ": step = cfg1 fwd+grad, cfg2 fwd+grad, four standalone reductions of the cfg2 tensor (sum / max / argmax over the last axis, sum over axis 0), cfg3 3-layer fwd+bwd, cfg4 conv fwd+dX+dW+db, cfg5 LSTM forward + gradient program"
                            + ", then softmax cross-entropy loss / loss+partial on 8192x8192 bf16, SGD on three 4096^2 bf16 matrices and 2x2 max pooling"
                            + " forward + gradient on 32x256x56x56 bf16, one fp32 LeNet training step (batch 64) eager and replayed from a"
                            + " CUDA graph, the cfg4 conv with NHWC-tagged tensors; cfg1 is also replayed from a CUDA graph",
-                           "value_covers": "dense + conv2d groups (cfg3 + cfg4) FLOPs / their device time; hbm_gbs covers cfg2",
+                           "value_covers": "dense + conv2d groups (cfg3 + cfg4) FLOPs / their device time; hbm_gbs covers cfg2 and the standalone reductions (a8.*)",
                            "groups": groups, "l2": "1 GiB streamed through L2 between groups (flush with clean lines); cfg2 inputs also exceed L2",
                            "replicas": world},
                 "groups": table, "roofline": roofline, "rooflines": rooflines, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
-                "clocks": clocks, "peaks": {k: peaks.get(k) for k in ("hbm_gbs", "bf16_tflops", "bf16_tflops_sustained", "source")}}
+                "clocks": clocks, "peaks": dict({k: peaks.get(k) for k in ("hbm_gbs", "bf16_tflops", "bf16_tflops_sustained", "source")}, nominal=NOMINAL_PEAKS)}
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

@@ -381,6 +381,18 @@ relay_status_t relay_sgd_update(const relay_tensor_t *const *params, const relay
 /* Thread-local text describing the last non-OK status returned on this thread ("" if none). */
 const char *relay_last_error(void);
 
+/* The contraction that the dense groups are built from, as a primitive operator of its own (Fig. 3 relay.linear without
+ * its hidden parameters; the adjoints that Section 4.2's reverse mode needs are the same product with one operand
+ * transposed):   c[m,n] = act( sum_k A(m,k) * B(k,n) + bias[n] ),  A = a or a^T, B = b or b^T (trans_* != 0), the
+ * transposed operand being READ in place, never materialised.
+ *   a:(M,K) or (K,M)  b:(K,N) or (N,K)  bias:(N) or NULL  ->  c:(M,N); a and b share one dtype t in {f32, bf16};
+ *   c has dtype t or f32 (the fp32 accumulator stored unrounded); bias has dtype t or f32.
+ *   trans_a = trans_b = 0 is relay_fused_dense_act; (0,1) computes dx = dZ w^T and (1,0) dw = x^T dZ of its gradient
+ *   group.  Device pointers, caller-owned; needs no workspace; K = 0 gives act(bias).  Errors as everywhere
+ *   (null -> rank -> dtype -> layout -> shape -> attr -> alignment/overlap), detected before any launch. */
+relay_status_t relay_contract_act(const relay_tensor_t *a, int32_t trans_a, const relay_tensor_t *b, int32_t trans_b,
+                                  const relay_tensor_t *bias, int32_t act, const relay_tensor_t *c, void *stream);
+
 /* Synchronises `stream`, then reads and clears the device-side error word of the current
  * device: RELAY_ERR_TIMEOUT if a bounded wait expired in any kernel since the last poll,
  * RELAY_ERR_CUDA if the stream reports an error, else RELAY_OK. */

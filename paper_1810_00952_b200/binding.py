@@ -258,6 +258,11 @@ def relay_fused_dense_act_grad(x, w, y, dy, act, dx, dw, db, ws=None):
                                             _ref(desc(dx)), _ref(desc(dw)), _ref(desc(db)), wp, wb, _stream()))
 
 
+def relay_contract_act(a, trans_a, b, trans_b, bias, act, c):
+    _check(lib().relay_contract_act(_ref(desc(a)), int(bool(trans_a)), _ref(desc(b)), int(bool(trans_b)), _ref(desc(bias)), int(act),
+                                    _ref(desc(c)), _stream()))
+
+
 def relay_fused_conv2d_act(x, w, b, stride, pad, act, y, ws=None, layout=NCHW):
     """`layout` tags x and y: NCHW tensors of shape (N,C,H,W) or NHWC tensors of shape (N,H,W,C)."""
     wp, wb = _ws(ws)

@@ -200,3 +200,48 @@ extern "C" relay_status_t relay_fused_dense_act_grad(const relay_tensor_t *x, co
     g.c = dw->data; g.ldc = d.N;
     return launch_gemm(g, st);
 }
+
+// The contraction under the dense groups as a call of its own: c = act(op(a) op(b) + bias) with either operand read
+// transposed where it lies (the forward product, dx = dZ w^T and dw = x^T dZ are its three forms).
+extern "C" relay_status_t relay_contract_act(const relay_tensor_t *a, int32_t trans_a, const relay_tensor_t *b, int32_t trans_b,
+                                             const relay_tensor_t *bias, int32_t act, const relay_tensor_t *c, void *stream)
+{
+    clear_error();
+    RELAY_TRY(check_not_null(a, "a"));
+    RELAY_TRY(check_not_null(b, "b"));
+    RELAY_TRY(check_not_null(c, "c"));
+    const relay_tensor_t *t3[3] = {a, b, c};
+    const char *names[3] = {"a", "b", "c"};
+    for (int i = 0; i < 3; ++i) { RELAY_TRY(check_type(t3[i], names[i])); RELAY_TRY(check_rank(t3[i], 2, names[i])); }
+    if (bias) { RELAY_TRY(check_type(bias, "bias")); RELAY_TRY(check_rank(bias, 1, "bias")); }
+    if (!is_float(a->dtype)) return fail(RELAY_ERR_DTYPE, "a: base type %s, needs f32 or bf16", dtype_name(a->dtype));
+    RELAY_TRY(check_dtype(b, a->dtype, "b"));
+    if (c->dtype != a->dtype && c->dtype != RELAY_F32) return fail(RELAY_ERR_DTYPE, "c: base type %s, needs %s or f32", dtype_name(c->dtype), dtype_name(a->dtype));
+    if (bias && bias->dtype != a->dtype && bias->dtype != RELAY_F32)
+        return fail(RELAY_ERR_DTYPE, "bias: base type %s, needs %s or f32", dtype_name(bias->dtype), dtype_name(a->dtype));
+    for (int i = 0; i < 3; ++i) RELAY_TRY(check_layout(t3[i], RELAY_ROWMAJOR, RELAY_ROWMAJOR, names[i]));
+    const int64_t M = trans_a ? a->shape[1] : a->shape[0], K = trans_a ? a->shape[0] : a->shape[1];
+    const int64_t Kb = trans_b ? b->shape[1] : b->shape[0], N = trans_b ? b->shape[0] : b->shape[1];
+    if (K != Kb) return fail(RELAY_ERR_SHAPE, "contraction lengths differ: op(a) has %lld columns, op(b) has %lld rows", (long long)K, (long long)Kb);
+    RELAY_TRY(check_shape(c, {M, N}, "c"));
+    if (bias) RELAY_TRY(check_shape(bias, {N}, "bias"));
+    if (act < RELAY_ACT_NONE || act > RELAY_ACT_SIGMOID) return fail(RELAY_ERR_ATTR, "unknown activation %d", act);
+    RELAY_TRY(check_data(a, "a"));
+    RELAY_TRY(check_data(b, "b"));
+    if (bias) RELAY_TRY(check_data(bias, "bias"));
+    RELAY_TRY(check_data(c, "c"));
+    const relay_tensor_t *outs[1] = {c}, *ins[3] = {a, b, bias};
+    RELAY_TRY(check_no_overlap(outs, 1, ins, 3));
+    cudaStream_t st = (cudaStream_t)stream;
+    if (M == 0 || N == 0) return RELAY_OK;
+    if (K == 0 && !bias && act == RELAY_ACT_NONE) { RELAY_CUDA(cudaMemsetAsync(c->data, 0, nbytes(c), st)); return RELAY_OK; }
+    GemmDesc g;
+    g.M = M; g.N = N; g.K = K;
+    g.a = a->data; g.a_sm = trans_a ? 1 : a->shape[1]; g.a_sk = trans_a ? a->shape[1] : 1;
+    g.b = b->data; g.b_sk = trans_b ? 1 : b->shape[1]; g.b_sn = trans_b ? b->shape[1] : 1;
+    g.c = c->data; g.ldc = N;
+    g.in_dtype = a->dtype; g.out_dtype = c->dtype;
+    g.bias = bias ? bias->data : nullptr; g.bias_dtype = bias ? bias->dtype : RELAY_F32;
+    g.act = act;
+    return launch_gemm(g, st);
+}

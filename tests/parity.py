@@ -49,7 +49,9 @@ def assert_bf16(got, want, stored_bf16=True, what=""):
 
 
 class Guarded:
-    """Output buffer with sentinel-filled margins on both sides to catch out-of-range writes."""
+    """Output buffer with sentinel-filled margins on both sides to catch out-of-range writes.  The view itself starts
+    out holding a value no result can take (NaN for floating types, the most negative integer for signed ones, 255 for bytes), and
+    `check` asserts that none of it survives: an output element that no work unit wrote shows at any size."""
 
     def __init__(self, shape, dtype, device, margin=256):
         n = int(np.prod(shape)) if len(shape) else 1
@@ -58,9 +60,15 @@ class Guarded:
         self.full = torch.full((n + 2 * m,), 7, dtype=dtype, device=device)
         self.m, self.n = m, n
         self.t = self.full[m:m + n].view(tuple(shape))
+        self.unwritten = float("nan") if dtype.is_floating_point else (0 if dtype == torch.bool else 255 if dtype == torch.uint8 else torch.iinfo(dtype).min)
+        if dtype != torch.bool:
+            self.t.fill_(self.unwritten)
 
-    def check(self):
+    def check(self, all_written=True):
         assert bool((self.full[:self.m] == 7).all()) and bool((self.full[self.m + self.n:] == 7).all()), "out-of-range write"
+        if all_written and self.n and self.t.dtype != torch.bool:
+            left = torch.isnan(self.t) if self.t.dtype.is_floating_point else (self.t == self.unwritten)
+            assert not bool(left.any()), ("elements never written", int(left.sum()), left.nonzero()[:4].tolist())
         return self.t
 
 

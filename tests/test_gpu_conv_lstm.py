@@ -143,23 +143,42 @@ def test_conv_rejections():
 
 
 def test_conv_full_size_sampled():
-    """Configuration 4 at full size: the oracle recomputes one whole image of y and dx, and a block
-    of dW (8 output x 8 input channels, all taps, all 32 images), from the GPU's stored y."""
+    """Configuration 4 at full size.  The forward / dX kernels walk (image, band of rows) tiles in rounds over the SM
+    pairs, the last round in another item shape, a schedule that exists only at this size: the oracle recomputes two
+    random output rows (all channels) of EVERY image of y and dx plus images 0 and 31 whole, four 8 x 8 channel
+    blocks of dW at the corners of its (o, c) range (all taps, all 32 images) and db of those channels, from the
+    GPU's stored y; every output is also screened for elements that no tile wrote (Guarded)."""
     t = I.cfg4_conv()
     y = conv_fwd(t["x"], t["w"], t["b"], 1, 1, B.ACT_RELU)
     dx, dw, db = conv_grad(t["x"], t["w"], y, t["dy"], 1, 1, B.ACT_RELU)
     wo, bo = I.as_f64(t["w"]), I.as_f64(t["b"])
-    n = 17
-    xo = I.as_f64(t["x"][n:n + 1])
-    assert_bf16(y[n:n + 1], oracle.conv2d_act(xo, wo, bo, 1, 1, B.ACT_RELU, F64), what="y")
-    odx, _, _ = oracle.conv2d_act_grad(xo, wo, to_np(y[n:n + 1]), I.as_f64(t["dy"][n:n + 1]), 1, 1, B.ACT_RELU, F64, F64, F64,
-                                       want_dw=False, want_db=False)
-    assert_bf16(dx[n:n + 1], odx, what="dx")
-    oc, ic = slice(120, 128), slice(248, 256)
-    _, odw, odb = oracle.conv2d_act_grad(I.as_f64(t["x"][:, ic]), wo[oc, ic], to_np(y[:, oc]), I.as_f64(t["dy"][:, oc]), 1, 1,
-                                         B.ACT_RELU, F64, F64, F64, want_dx=False)
-    assert_bf16(dw[oc, ic], odw, what="dw")
-    assert_bf16(db[oc], odb, stored_bf16=False, what="db")
+    for n in (0, 31):
+        xo = I.as_f64(t["x"][n:n + 1])
+        assert_bf16(y[n:n + 1], oracle.conv2d_act(xo, wo, bo, 1, 1, B.ACT_RELU, F64), what=f"y image {n}")
+        odx, _, _ = oracle.conv2d_act_grad(xo, wo, to_np(y[n:n + 1]), I.as_f64(t["dy"][n:n + 1]), 1, 1, B.ACT_RELU, F64, F64, F64,
+                                           want_dw=False, want_db=False)
+        assert_bf16(dx[n:n + 1], odx, what=f"dx image {n}")
+    # an output row depends on the three input rows around it: the oracle is run on that band (its zero padding is the
+    # real one at the image's edge, elsewhere the band's outer rows are not used)
+    rng = np.random.default_rng(17)
+    H = t["x"].shape[2]
+    got_y, want_y, got_dx, want_dx = [], [], [], []
+    for n in range(t["x"].shape[0]):
+        for h in {int(v) for v in rng.choice(H, 2, replace=False)} | ({0, H - 1} if n == 7 else set()):
+            lo, hi = max(h - 1, 0), min(h + 2, H)
+            xo = I.as_f64(t["x"][n:n + 1, :, lo:hi])
+            want_y.append(oracle.conv2d_act(xo, wo, bo, 1, 1, B.ACT_RELU, F64)[0, :, h - lo]); got_y.append(to_np(y[n, :, h]))
+            odx, _, _ = oracle.conv2d_act_grad(xo, wo, to_np(y[n:n + 1, :, lo:hi]), I.as_f64(t["dy"][n:n + 1, :, lo:hi]), 1, 1,
+                                               B.ACT_RELU, F64, F64, F64, want_dw=False, want_db=False)
+            want_dx.append(odx[0, :, h - lo]); got_dx.append(to_np(dx[n, :, h]))
+    assert_bf16(np.stack(got_y), np.stack(want_y), what="y rows of every image")
+    assert_bf16(np.stack(got_dx), np.stack(want_dx), what="dx rows of every image")
+    for oc, ic in [(slice(0, 8), slice(0, 8)), (slice(0, 8), slice(248, 256)), (slice(248, 256), slice(0, 8)),
+                   (slice(248, 256), slice(248, 256)), (slice(120, 128), slice(128, 136))]:
+        _, odw, odb = oracle.conv2d_act_grad(I.as_f64(t["x"][:, ic]), wo[oc, ic], to_np(y[:, oc]), I.as_f64(t["dy"][:, oc]), 1, 1,
+                                             B.ACT_RELU, F64, F64, F64, want_dx=False)
+        assert_bf16(dw[oc, ic], odw, what=f"dw {oc} {ic}")
+        assert_bf16(db[oc], odb, stored_bf16=False, what="db")
     # the same tensors tagged NHWC: the kernels store pixel-major tiles of the same accumulators, so y, dx and dw agree
     # bit for bit with the NCHW call; db is summed in another order
     nhwc = lambda a: a.permute(0, 2, 3, 1).contiguous().to(DEV)

@@ -171,11 +171,15 @@ def test_dense_rejections_leave_outputs_untouched():
 
 def test_full_size_mlp_layer_sampled_rows_and_columns():
     """Configuration 3 at full size (4096^3 per contraction, bf16, fp32 accumulate), all three
-    layers forward and backward; the oracle recomputes sampled rows of y / dx (all columns) and
-    sampled rows of dW (all columns) plus db, each from the GPU's stored inputs of that group."""
+    layers forward and backward.  The work units of the contraction kernels are 256-row blocks cut into
+    column ranges, a schedule that exists only at this size, so the oracle recomputes one row (all columns) in
+    EVERY 128-row block of y and dx, one k-row (all columns) in every 128-row block of dW, the block-edge rows,
+    and all of db, each from the GPU's stored inputs of that group; every output is also screened for
+    elements that no unit wrote (Guarded)."""
     t = I.cfg3_mlp()
     rng = np.random.default_rng(5)
-    rows = np.unique(np.concatenate([[0, 127, 128, 4095], rng.integers(0, 4096, 8)]))
+    rows = np.unique(np.concatenate([[0, 127, 128, 255, 256, 4095], np.arange(0, 4096, 128) + rng.integers(0, 128, 32)]))
+    assert len(np.unique(rows // 128)) == 32
     acts = [t["x"].to(DEV)]
     for l in range(3):
         acts.append(run_fwd(acts[-1], t[f"w{l}"], t[f"b{l}"], B.ACT_RELU))
@@ -188,10 +192,11 @@ def test_full_size_mlp_layer_sampled_rows_and_columns():
         odx, _, _ = oracle.dense_act_grad(to_np(acts[l][rows]), wo, to_np(acts[l + 1][rows]), to_np(g[rows]), B.ACT_RELU, F64, F64, F64,
                                           want_dw=False, want_db=False)
         assert_bf16(dx[rows], odx, what=f"dx{l}")
-        # dW rows k in `rows`: needs x[:, rows] over the whole batch
-        _, odw, odb = oracle.dense_act_grad(to_np(acts[l][:, rows]), wo[rows], to_np(acts[l + 1]), to_np(g), B.ACT_RELU, F64, F64, F64,
+        # dW rows k in `krows`: needs x[:, krows] over the whole batch
+        krows = np.unique(np.concatenate([[0, 127, 128, 4095], np.arange(0, 4096, 128) + rng.integers(0, 128, 32)]))
+        _, odw, odb = oracle.dense_act_grad(to_np(acts[l][:, krows]), wo[krows], to_np(acts[l + 1]), to_np(g), B.ACT_RELU, F64, F64, F64,
                                             want_dx=False)
-        assert_bf16(dw[rows], odw, what=f"dw{l}")
+        assert_bf16(dw[krows], odw, what=f"dw{l}")
         assert_bf16(db, odb, stored_bf16=False, what=f"db{l}")
         g = dx
 
@@ -207,14 +212,15 @@ def test_two_sm_kernel_ragged_edges_and_half_width_tail_units():
     y = run_fwd(x, w, b, act)
     xo, wo, bo, dyo = (v.double().numpy() for v in (x, w, b, dy))
     rng = np.random.default_rng(11)
-    rows = np.unique(np.concatenate([[0, 127, 128, 255, 256, 2559, 2560, M - 1], rng.integers(0, M, 12)]))
+    rows = np.unique(np.concatenate([[0, 127, 128, 255, 256, 2559, 2560, M - 1],
+                                     np.minimum(np.arange(0, M, 128) + rng.integers(0, 128, (M + 127) // 128), M - 1)]))
     assert_bf16(y[rows], oracle.dense_act(xo[rows], wo, bo, act, F64), what="y")
     dx, dw, db = run_grad(x, w, y, dy, act)
     yo = to_np(y)
     odx, _, _ = oracle.dense_act_grad(xo[rows], wo, yo[rows], dyo[rows], act, F64, F64, F64, want_dw=False, want_db=False,
                                       dz_dtype=oracle.BF16)
     assert_bf16(dx[rows], odx, what="dx")
-    krows = np.unique(np.concatenate([[0, 63, 64, K - 1], rng.integers(0, K, 6)]))
+    krows = np.unique(np.concatenate([[0, 63, 64, 127, 128, K - 1], rng.integers(0, K, 6)]))
     _, odw, odb = oracle.dense_act_grad(xo[:, krows], wo[krows], yo, dyo, act, F64, F64, F64, want_dx=False, dz_dtype=oracle.BF16)
     assert_bf16(dw[krows], odw, what="dw")
     assert_bf16(db, odb, stored_bf16=False, what="db")
@@ -225,7 +231,7 @@ def test_two_sm_kernel_fixed_unit_scheme_on_a_large_ragged_output():
     rounds of 256 x 512 units and then 256 x 256 tiles with a split tail.  One sampled row in EVERY 256-row block (all
     columns), so that a unit that is skipped or computed twice with other data shows."""
     M, K, N = 10000, 2048, 16392
-    assert B.relay_debug_plan_units(M, N, K, 148) is None
+    assert B.relay_debug_plan_units(M, N, K, torch.cuda.get_device_properties(0).multi_processor_count) is None
     t = I.cfg1_tiny_mlp(M, K, N, salt=91)
     x, b = t["x"].bfloat16(), t["b"].bfloat16()
     w = (t["w"] / np.sqrt(K)).bfloat16()
@@ -234,3 +240,43 @@ def test_two_sm_kernel_fixed_unit_scheme_on_a_large_ragged_output():
     rows = np.unique(np.concatenate([np.arange(0, M, 256) + rng.integers(0, 16, (M + 255) // 256), [255, 256, M - 1]]))
     want = oracle.dense_act(x[rows].double().numpy(), w.double().numpy(), b.double().numpy(), B.ACT_RELU, F64)
     assert_bf16(y[rows], want, what="y")
+
+
+@pytest.mark.parametrize("M,K,N", [(37, 53, 29), (256, 512, 384), (520, 264, 1032), (8, 64, 32)])
+@pytest.mark.parametrize("tdt", [torch.float32, torch.bfloat16])
+def test_contraction_with_operands_read_transposed(M, K, N, tdt):
+    """The contraction as a call of its own, in the three forms the dense groups use (plain, b transposed as in
+    dx = dZ w^T, a transposed as in dw = x^T dZ) and with both transposed; results in the operand type and as the
+    unrounded fp32 accumulator.  The oracle gets the transposed matrices materialised on the host."""
+    t = I.cfg1_tiny_mlp(M, K, N, salt=K)
+    a = t["x"].to(tdt)                                   # (M, K)
+    b = (t["w"] / np.sqrt(K)).to(tdt)                    # (K, N)
+    bias = t["b"].to(tdt)
+    ao, bo, biaso = a.double().numpy(), b.double().numpy(), bias.double().numpy()
+    chk = assert_f32 if tdt == torch.float32 else assert_bf16
+    for ta, tb in ((0, 0), (0, 1), (1, 0), (1, 1)):
+        ad = (a.t().contiguous() if ta else a).to(DEV)
+        bd = (b.t().contiguous() if tb else b).to(DEV)
+        for cdt, act, bb in ((tdt, B.ACT_TANH, bias), (torch.float32, B.ACT_NONE, None)):
+            c = Guarded((M, N), cdt, DEV)
+            B.relay_contract_act(ad, ta, bd, tb, None if bb is None else bb.to(DEV), act, c.t)
+            torch.cuda.synchronize()
+            want = oracle.dense_act(ao, bo, None if bb is None else biaso, act, F64)
+            if cdt == torch.float32 and tdt == torch.bfloat16:
+                assert_bf16(c.check(), want, stored_bf16=False, what=f"c f32 {ta}{tb}")
+            else:
+                chk(c.check(), want, what=f"c {ta}{tb}")
+    # type errors: contraction lengths differ, operand types differ, result of a third type
+    n0 = B.relay_launch_count()
+    c = torch.full((M, N), 5.0, dtype=tdt, device=DEV)
+    for args, status in [((a.to(DEV), 1, b.to(DEV), 0, None, B.ACT_NONE, c), "ERR_SHAPE" if M != K else None),
+                         ((a.to(DEV), 0, b.to(DEV).to(torch.float32 if tdt == torch.bfloat16 else torch.bfloat16), 0, None, B.ACT_NONE, c), "ERR_DTYPE"),
+                         ((a.to(DEV), 0, b.to(DEV), 0, None, 7, c), "ERR_ATTR"),
+                         ((a.to(DEV), 0, b.to(DEV), 0, None, B.ACT_NONE, torch.empty(M, N, dtype=torch.int32, device=DEV)), "ERR_DTYPE")]:
+        if status is None:
+            continue
+        with pytest.raises(B.RelayError) as e:
+            B.relay_contract_act(*args)
+        assert e.value.status_name == status, str(e.value)
+    torch.cuda.synchronize()
+    assert B.relay_launch_count() == n0 and bool((c == 5.0).all())

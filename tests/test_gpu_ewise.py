@@ -223,12 +223,15 @@ def test_empty_tensors_are_accepted():
 
 def test_full_size_forward_and_gradient_sampled_columns():
     """Configuration 2 at full size (8192 x 8192, bf16) in the launch shape the benchmark times;
-    the oracle recomputes 48 whole columns (all 8192 rows each, so column sums are covered)."""
+    the oracle recomputes whole columns (all 8192 rows each, so column sums are covered): at least one in
+    every 256-column slab of the launch grid, the slab edges, and random ones."""
     t = I.cfg2_ewise()
     prog, outs, got = _fwd(t, P.BF16, 8192, 8192)
     dx, da, db = _grad(t, P.BF16)
     rng = np.random.default_rng(3)
-    cols = np.unique(np.concatenate([[0, 7, 8, 255, 256, 8191], rng.integers(0, 8192, 42)]))
+    cols = np.unique(np.concatenate([[0, 7, 8, 255, 256, 8191], np.arange(0, 8192, 256) + rng.integers(0, 256, 32),
+                                     rng.integers(0, 8192, 16)]))
+    assert len(np.unique(cols // 256)) == 32
     sub = {k: t[k][..., cols] for k in ("x", "a", "b", "dout")}
     fp, fo = P.tanh_affine_residual_fwd(5, 5)
     (want,) = oracle.ewise(fp.arrays(), [I.as_f64(sub[k]) for k in ("x", "a", "b")], fo)

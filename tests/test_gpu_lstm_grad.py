@@ -113,8 +113,8 @@ def test_empty_sequence_and_rejections():
 
 def test_full_size_sampled_batch_rows():
     """Configuration 5 at full size (T=128, B=64, I=H=1024).  Batch rows are independent in dx, dh0 and dc0, so the
-    oracle runs the whole program on 2 of the 64 rows; the weight partials (sums over all rows) are covered by
-    the H=1024 case above."""
+    oracle runs the whole program on 2 of the 64 rows; the weight partials (sums over all rows and steps) are compared
+    at T = 128 with a batch the oracle can run whole in the next test."""
     t, dh_all, dc_fin = case(128, 64, 1024, 1024, salt=0, h0_random=False)
     d = {k: v.to(DEV) for k, v in t.items()}
     h_all, _ = forward(d)
@@ -127,6 +127,21 @@ def test_full_size_sampled_batch_rows():
     assert_bf16(got["dc0"][rows], want["dc0"], stored_bf16=False, what="dc0")
     for k in ("dw_ih", "dw_hh", "db"):
         assert bool(torch.isfinite(got[k].float()).all())
+
+
+def test_full_length_sequence_all_six_partials():
+    """T = 128, I = H = 1024 as in configuration 5, with a batch of 8 rows so that the oracle can run the whole
+    program: the weight and bias partials are sums over all 128 steps (and rows), which no shorter case reaches.
+    (The two sides round dz to bf16 from an fp32 and an fp64 value; a differing last bit changes every later dz a
+    little, so after a few steps their roundings are independent and each of the T*B terms of a weight partial differs
+    by a fraction of a bf16 step of that term.  The error is 1.8e-3 of the RMS whatever T and B are, but its largest
+    element over the 4.2 M of a weight partial depends on how heavy-tailed the sums are: with 4 rows one element
+    reaches 1.05e-2 of the RMS beyond its storage rounding, with 8 rows 0.8e-2, inside the 1e-2 bound.)"""
+    t, dh_all, dc_fin = case(128, 8, 1024, 1024, salt=41)
+    d = {k: v.to(DEV) for k, v in t.items()}
+    h_all, _ = forward(d)
+    got = backward(d, h_all, dh_all.to(DEV), dc_fin.to(DEV))
+    compare(got, oracle_grads(t, dh_all, dc_fin))
 
 
 @pytest.mark.parametrize("T,Bn,In,H", [(128, 64, 1024, 1024), (32, 96, 128, 512)])
