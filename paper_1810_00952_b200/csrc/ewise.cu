@@ -153,42 +153,78 @@ __global__ void __launch_bounds__(32 * TY) colsum_finalize_kernel(const float *_
     }
 }
 
-// reduction over the last axis of a [rows, cols] tensor: one warp per row, 128-bit loads
+// reduction over the last axis of a [rows, cols] tensor: one warp per row, 128-bit loads.
+// max / argmax work on whole vectors: the maximum of a 16-byte vector is taken with packed comparisons on the
+// stored type (exact: comparing needs no arithmetic), and only a vector that beats the lane's running maximum is
+// kept (its raw bits and its index); the first element that attains the maximum is looked up once, at the end.
+// A lane meets its vectors in increasing column order and replaces only on strictly greater, so the kept vector
+// is the lane's first one holding the maximum: ties go to the lowest index.
+__device__ __forceinline__ float vec_max(const uint4 &r, const __nv_bfloat16 *)
+{
+    const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162 *>(&r.x), b = *reinterpret_cast<const __nv_bfloat162 *>(&r.y);
+    const __nv_bfloat162 c = *reinterpret_cast<const __nv_bfloat162 *>(&r.z), d = *reinterpret_cast<const __nv_bfloat162 *>(&r.w);
+    const __nv_bfloat162 m = __hmax2(__hmax2(a, b), __hmax2(c, d));
+    return fmaxf(__low2float(m), __high2float(m));
+}
+__device__ __forceinline__ float vec_max(const uint4 &r, const float *)
+{
+    return fmaxf(fmaxf(__uint_as_float(r.x), __uint_as_float(r.y)), fmaxf(__uint_as_float(r.z), __uint_as_float(r.w)));
+}
+
 template <typename T, int RED>
 __global__ void __launch_bounds__(256) rowreduce_kernel(const T *__restrict__ in, int64_t rows, int64_t cols, float scale,
                                                          void *__restrict__ out)
 {
     constexpr int V = VecN<T>::N;
+    constexpr int U = 8;                 // 16-byte loads in flight per lane
     const int lane = threadIdx.x & 31;
     const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (row >= rows) return;
     const T *p = in + row * cols;
     const int64_t nvec = cols / V;
     float best = RED == RELAY_RED_SUM ? 0.0f : -INFINITY;
-    int64_t pos = 0;
-    for (int64_t j = lane; j < nvec; j += 32 * kUnroll) {
-        uint4 raw[kUnroll];
+    uint4 best_raw = make_uint4(0, 0, 0, 0);
+    int64_t best_vec = 0;
+    for (int64_t j = lane; j < nvec; j += 32 * U) {
+        uint4 raw[U];
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u)
+        for (int u = 0; u < U; ++u)
             if (j + u * 32 < nvec) raw[u] = ld_stream(p + (j + u * 32) * V);
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
+        for (int u = 0; u < U; ++u) {
             if (j + u * 32 >= nvec) break;
-            float f[V];
-            unpack(raw[u], f);
+            if (RED == RELAY_RED_SUM) {
+                float f[V];
+                unpack(raw[u], f);
+                float s = 0.0f;
 #pragma unroll
-            for (int v = 0; v < V; ++v) {
-                if (RED == RELAY_RED_SUM) best += f[v];
-                else if (f[v] > best) { best = f[v]; pos = (j + u * 32) * V + v; }
+                for (int v = 0; v < V; ++v) s += f[v];
+                best += s;
+            } else {
+                const float m = vec_max(raw[u], (const T *)nullptr);
+                if (m > best) { best = m; best_raw = raw[u]; best_vec = j + u * 32; }
             }
         }
+    }
+    int64_t pos = 0;
+    if (RED == RELAY_RED_ARGMAX) {
+        float f[V];
+        unpack(best_raw, f);
+        int first = 0;
+#pragma unroll
+        for (int v = V - 1; v >= 0; --v)
+            if (f[v] == best) first = v;
+        pos = best_vec * V + first;
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         float ob = __shfl_xor_sync(0xffffffffu, best, o);
-        int64_t op = __shfl_xor_sync(0xffffffffu, pos, o);
         if (RED == RELAY_RED_SUM) best += ob;
-        else if (ob > best || (ob == best && op < pos)) { best = ob; pos = op; }
+        else if (RED == RELAY_RED_MAX) best = fmaxf(best, ob);
+        else {
+            int64_t op = __shfl_xor_sync(0xffffffffu, pos, o);
+            if (ob > best || (ob == best && op < pos)) { best = ob; pos = op; }
+        }
     }
     if (lane == 0) {
         if (RED == RELAY_RED_ARGMAX) ((int64_t *)out)[row] = pos;

@@ -173,6 +173,39 @@ def test_argmax_bit_exact_with_ties(shape, axis):
         assert np.array_equal(out.check().cpu().numpy(), want)
 
 
+def test_standalone_reductions_full_size_all_results():
+    """The standalone reductions at the size and in the launch shape the benchmark times (8192 x 8192 bf16): sum, max and
+    argmax over the last axis and the sum over axis 0, EVERY result against the oracle.  Ties are planted for the argmax:
+    in every row the maximum is written to several columns (two of them inside one 16-byte vector, others in the strips
+    of other lanes), and in some rows to column 0 and the last column; the lowest index must win, bit for bit."""
+    t = I.cfg2_ewise()
+    x = t["x"].clone()
+    rng = np.random.default_rng(29)
+    top = float(x.max()) + 1.0
+    for r in range(8192):
+        c = np.sort(rng.choice(8192, 4, replace=False))
+        x[r, c] = top
+        x[r, min(int(c[0]) + 1, 8191)] = top                  # a neighbour in the same (or the next) vector
+    x[5, 0] = top; x[6, 8191] = top; x[7] = top               # first column, a late column, a constant row
+    xd = x.to(DEV)
+    ident = P.Program([P.BF16])
+    outs = dict(sum1=Guarded((8192,), torch.float32, DEV), max1=Guarded((8192,), torch.float32, DEV),
+                arg1=Guarded((8192,), torch.int64, DEV), sum0=Guarded((8192,), torch.float32, DEV))
+    specs = dict(sum1=(0, B.RED_SUM, 2, 0), max1=(0, B.RED_MAX, 2, 0), arg1=(0, B.RED_ARGMAX, 2, 0), sum0=(0, B.RED_SUM, 1, 0))
+    for k, sp in specs.items():
+        ws = workspace(B.relay_workspace_bytes_reduce([xd], [sp]), DEV)
+        B.relay_fused_reduce(None, [xd], [sp], [outs[k].t], ws)
+    torch.cuda.synchronize()
+    xo = x.double().numpy()
+    w_sum1, w_max1, w_arg1, w_sum0 = oracle.reduce(ident.arrays(), [xo], [(0, oracle.RED_SUM, (1,), False, 5), (0, oracle.RED_MAX, (1,), False, 5),
+                                                                          (0, oracle.RED_ARGMAX, (1,), False, P.I64), (0, oracle.RED_SUM, (0,), False, 5)])
+    assert np.array_equal(outs["arg1"].check().cpu().numpy(), w_arg1)
+    assert np.array_equal(to_np(outs["max1"].check()), w_max1)              # a maximum is one of the inputs: exact
+    assert_bf16(outs["sum1"].check(), w_sum1, stored_bf16=False, what="sum over the last axis")
+    assert_bf16(outs["sum0"].check(), w_sum0, stored_bf16=False, what="sum over axis 0")
+    assert int(w_arg1[7]) == 0 and int(w_arg1[5]) == 0
+
+
 def test_reduce_with_prologue_and_unreduced_output_generic():
     g = torch.Generator().manual_seed(13)
     x, w = torch.randn(40, 24, generator=g), torch.randn(24, generator=g)
