@@ -131,6 +131,130 @@ __global__ void __launch_bounds__(256) nchw_to_nhwc_kernel(const __nv_bfloat16 *
     }
 }
 
+// ---------------------------------------------------------------------------------------------------
+// The same repack as a PERSISTENT kernel that runs beside the tensor-core kernel which consumes it.  Two blocks per SM
+// (little shared memory, and at most a third of the registers, so that the consumer's one large block per SM still fits) walk a list of units: first the
+// weight-packing units, then (image, 64-pixel block) units of up to two activation tensors, image by image.  A unit's
+// loads for four channel blocks are all in flight before the first is transposed, so two blocks per SM keep enough
+// bytes in flight.  Finished units are counted with release semantics: flags[0] counts packing units, flags[1 + n] the
+// units of image n of the FIRST tensor; the consumer (launched behind this kernel with programmatic stream
+// serialisation, and therefore started once every block here is resident and past its own wait for the stream's
+// earlier work) polls them before it loads a tile.  This kernel never waits for the consumer.
+struct RepackJob {
+    const __nv_bfloat16 *in, *y;   // y: saved forward output (grad != 0: out = in * act'(y))
+    __nv_bfloat16 *out;
+    float *db_part;                // grad: per-unit sums over the 64 pixels, [n][pixel block][C], or null
+    int C, grad, act, flagged;
+};
+struct RepackStream {
+    RepackJob job[2];
+    int n_jobs, Nb, HW, pbx;       // pbx: 64-pixel blocks per image
+    PackJob pack;
+    int pack_units;                // units of kPackPerUnit weight elements
+    unsigned int *flags;
+};
+constexpr int kPackPerUnit = 4096;
+
+template <bool GRAD>
+__device__ __forceinline__ void repack_unit(const RepackJob &j, int HW, int pbx, int n, int pb, __nv_bfloat16 (*tile)[66])
+{
+    // channel blocks whose loads are in flight together: 8 loads of 16 bytes per thread either way
+    constexpr int NT = GRAD ? 2 : 4;
+    const int p0 = pb * 64, tid = threadIdx.x;
+    const size_t img = (size_t)n * j.C * HW;
+    for (int cg = 0; cg < j.C; cg += 64 * NT) {
+        uint4 v[NT][2], yy[GRAD ? NT : 1][2];
+#pragma unroll
+        for (int t = 0; t < NT; ++t)
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const int idx = tid + i * 256, cl = idx >> 3, chunk = idx & 7;
+                const int c = cg + t * 64 + cl, p = p0 + chunk * 8;
+                v[t][i] = make_uint4(0, 0, 0, 0);
+                if (GRAD) yy[t][i] = make_uint4(0, 0, 0, 0);
+                if (c < j.C && p < HW) {
+                    const size_t off = img + (size_t)c * HW + p;
+                    v[t][i] = ld_stream(j.in + off);
+                    if (GRAD) yy[t][i] = ld_stream(j.y + off);
+                }
+            }
+#pragma unroll
+        for (int t = 0; t < NT; ++t) {
+            const int c0 = cg + t * 64;
+            if (c0 >= j.C) break;
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const int idx = tid + i * 256, cl = idx >> 3, chunk = idx & 7;
+                uint4 val = v[t][i];
+                if (GRAD) {
+                    float a[8], b[8];
+                    unpack(val, a);
+                    unpack(yy[GRAD ? t : 0][i], b);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) a[q] *= act_grad_from_output(b[q], j.act);
+                    val = pack(a);
+                }
+                const uint32_t w[4] = {val.x, val.y, val.z, val.w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    tile[chunk * 8 + 2 * q][cl] = __ushort_as_bfloat16((unsigned short)(w[q] & 0xffffu));
+                    tile[chunk * 8 + 2 * q + 1][cl] = __ushort_as_bfloat16((unsigned short)(w[q] >> 16));
+                }
+                if (GRAD && j.db_part != nullptr) {      // the 8 lanes that share a channel row combine in a fixed order
+                    float r[8];
+                    unpack(val, r);
+                    float sum = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
+                    sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+                    sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+                    sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+                    if (chunk == 0 && c0 + cl < j.C) j.db_part[((size_t)n * pbx + pb) * j.C + c0 + cl] = sum;
+                }
+            }
+            __syncthreads();
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const int idx = tid + i * 256, pl = idx >> 3, cchunk = idx & 7;
+                const int c = c0 + cchunk * 8, p = p0 + pl;
+                if (c < j.C && p < HW) {
+                    const uint32_t *row = reinterpret_cast<const uint32_t *>(&tile[pl][cchunk * 8]);
+                    *reinterpret_cast<uint4 *>(j.out + ((size_t)n * HW + p) * j.C + c) = make_uint4(row[0], row[1], row[2], row[3]);
+                }
+            }
+            __syncthreads();
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256, 3) repack_stream_kernel(const RepackStream S)
+{
+    __shared__ __align__(16) __nv_bfloat16 tile[64][66];
+    // first the stream's earlier work must be complete (this kernel overwrites scratch that it may still read); only
+    // then may the consumer start: whatever it reads that this kernel does not produce is then final as well
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int act_units = S.Nb * S.pbx, total = S.pack_units + S.n_jobs * act_units;
+    for (int u = blockIdx.x; u < total; u += gridDim.x) {
+        unsigned int *flag = nullptr;
+        if (u < S.pack_units) {
+#pragma unroll 1
+            for (int k = 0; k < kPackPerUnit / 256; ++k) pack_one(S.pack, (unsigned)u * kPackPerUnit + k * 256 + threadIdx.x);
+            flag = S.flags;
+        } else {
+            const int v = u - S.pack_units, ji = v / act_units, w = v - ji * act_units, n = w / S.pbx, pb = w - n * S.pbx;
+            const RepackJob &j = S.job[ji];
+            if (j.grad) repack_unit<true>(j, S.HW, S.pbx, n, pb, tile);
+            else repack_unit<false>(j, S.HW, S.pbx, n, pb, tile);
+            if (j.flagged) flag = S.flags + 1 + n;
+        }
+        if (flag != nullptr) {             // block-uniform
+            tc::fence_proxy_async_global();   // the consumer reads these stores through TMA
+            __threadfence();
+            __syncthreads();
+            if (threadIdx.x == 0) tc::red_release_add_u32(flag, 1u);
+        }
+    }
+}
+
 // wf[o][tap][c] = w[o][c][tap];   wb[c][mirror(tap)][o] = w[o][c][tap]   (either may be null); one thread
 // per OUTPUT element so that the stores coalesce (the 1 MB source stays in L2)
 __global__ void pack_weights_kernel(const __nv_bfloat16 *__restrict__ w, __nv_bfloat16 *__restrict__ wf,
@@ -150,17 +274,20 @@ __global__ void pack_weights_kernel(const __nv_bfloat16 *__restrict__ w, __nv_bf
     }
 }
 
-// dw[o][c][tap] = bf16( sum over slices, in slice order, of part[slice][tap][o][c] ); one thread per
-// (tap, o, c) with (o, c) fastest so that the partial reads coalesce (the 2-byte stores scatter, 1.2 MB)
+// dw[o][c][tap] = bf16( sum over slices, in slice order, of part[slice][tap][o][c] ); one thread per (o, c) adds up all
+// its taps: the partial reads coalesce over (o, c) for every tap, and a warp's stores cover one contiguous run of
+// 32 * taps output elements
 __global__ void wgrad_reduce_kernel(const float *__restrict__ part, int n_slices, __nv_bfloat16 *__restrict__ dw, int O, int C, int taps)
 {
-    const unsigned oc_total = (unsigned)O * C, total = oc_total * (unsigned)taps;
+    const unsigned oc_total = (unsigned)O * C;
+    const size_t total = (size_t)oc_total * taps;
     pdl_wait();
-    for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
-        const unsigned tap = i / oc_total, oc = i - tap * oc_total;
-        float s = 0.0f;
-        for (int j = 0; j < n_slices; ++j) s += part[(size_t)j * total + i];
-        dw[(size_t)oc * taps + tap] = __float2bfloat16_rn(s);
+    for (unsigned oc = blockIdx.x * blockDim.x + threadIdx.x; oc < oc_total; oc += gridDim.x * blockDim.x) {
+        for (int tap = 0; tap < taps; ++tap) {
+            float s = 0.0f;
+            for (int j = 0; j < n_slices; ++j) s += part[(size_t)j * total + (size_t)tap * oc_total + oc];
+            dw[(size_t)oc * taps + tap] = __float2bfloat16_rn(s);
+        }
     }
 }
 
@@ -180,6 +307,9 @@ struct FpropParams {
     int rows_per_tile, nt;      // nt = rows_per_tile * W = UMMA N
     int tiles_per_img, n_tiles_total, k_blocks, stages;
     int n_pairs, pairs_per_ntile, n_items;   // items [0, n_pairs) are pairs, the rest singles (MH = 2); MH = 1: all singles
+    const unsigned int *flags;  // two-SM kernel running beside the repack that feeds it (else null): flags[0] counts packed weight
+    int pack_units, units_per_img;   // units, flags[1 + n] the repacked units of image n; a tile is loaded once both are complete
+    int n_full;                 // two-SM kernel: items [0, n_full) are whole tiles, items beyond are HALF tiles (rows_per_tile / 2 rows)
     const void *bias;           // per output channel, or null
     int bias_bf16, act;
     int out_nhwc;               // two-SM kernel: the output tensor map is [Nb*H*W pixels][Cout], tiles are stored pixel-major
@@ -386,9 +516,30 @@ conv_fprop_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
 // activation tile (rows_per_tile / 2 image rows), 30 KB per k-block at cfg4, so six stages fit and the two
 // TMEM accumulators alternate between tiles (the epilogue overlaps the next main loop).
 // ---------------------------------------------------------------------------------------------------
+// Work items of the two-SM kernel.  Whole rounds over the SM pairs are made of whole tiles; the tiles that would start
+// one more, mostly empty round are cut into two half tiles each (half as many image rows, N halved), so that this last
+// round is about half as long and twice as many pairs share it.
+struct PairItem { int m0, img, h0, rows; bool half; };
+__device__ __forceinline__ PairItem pair_item(const FpropParams &p, int item)
+{
+    PairItem it;
+    int t = item, sub = 0;
+    it.half = item >= p.n_full;
+    if (it.half) { const int j = item - p.n_full; t = p.n_full + (j >> 1); sub = j & 1; }
+    const int nt_idx = t / p.pairs_per_ntile;
+    it.m0 = (t % p.pairs_per_ntile) * 256;
+    it.rows = it.half ? p.rows_per_tile >> 1 : p.rows_per_tile;
+    it.img = nt_idx / p.tiles_per_img;
+    it.h0 = (nt_idx % p.tiles_per_img) * p.rows_per_tile + sub * it.rows;
+    return it;
+}
+
+// tm_xh: activation boxes of rows_per_tile / 2 image rows (a block's half of a whole tile); tm_xq: of rows_per_tile / 4 rows (its
+// half of a half tile); tm_y: 32-pixel x 32-channel output boxes; tm_yt: 16-pixel boxes, unswizzled, for the half tiles
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 conv_fprop_tc2_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x,
-                      const __grid_constant__ CUtensorMap tm_y, const FpropParams p)
+                      const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_xq,
+                      const __grid_constant__ CUtensorMap tm_yt, const FpropParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -404,7 +555,7 @@ conv_fprop_tc2_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
     const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // provably warp-uniform
     const uint32_t rank = tc::cluster_ctarank();
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-    const int cblocks = p.Cin / BK, half_rows = p.rows_per_tile / 2;
+    const int cblocks = p.Cin / BK;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
@@ -414,6 +565,8 @@ conv_fprop_tc2_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
         tc::prefetch_tmap(&tm_w);
         tc::prefetch_tmap(&tm_x);
         tc::prefetch_tmap(&tm_y);
+        tc::prefetch_tmap(&tm_xq);
+        tc::prefetch_tmap(&tm_yt);
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc::smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
@@ -424,17 +577,51 @@ conv_fprop_tc2_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
     tc::cluster_sync();
     tc::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    pdl_wait();   // set-up done; from here on the kernel touches global memory
+    // Beside a repack kernel (p.flags): that kernel has already waited for the stream's earlier work, and what it
+    // produces is handed over through its counters, so this kernel starts at once and waits for the repack kernel's
+    // completion only at its very end (completion of this kernel then still implies completion of all earlier ones).
+    if (p.flags != nullptr) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    else pdl_wait();   // set-up done; from here on the kernel touches global memory
 
     if (warp == 0) {
         {   // warp-uniform loop, an elected lane issues the copies
             int s = 0;
             uint32_t phase = 0;
             bool ok = true;
+            // bounded poll of one of the repack kernel's counters (lane 0 polls, the warp follows)
+            auto wait_count = [&](const unsigned int *counter, unsigned int target) -> bool {
+                int good = 1;
+                if (lane == 0) {
+                    const long long t0 = clock64();
+                    unsigned spins = 0;
+                    while (tc::ld_acquire_u32(counter) < target) {
+                        __nanosleep(100);
+                        if ((++spins & 255u) == 0 && (*abort_flag || clock64() - t0 > tc::kWaitLimitCycles)) {
+                            if (!*abort_flag) { *abort_flag = 1; atomicCAS(p.err, 0, tc::ERR_WAIT_STEP); }
+                            good = 0;
+                            break;
+                        }
+                    }
+                }
+                __syncwarp();                                  // lane 0's acquire is ordered before the other lanes' accesses
+                good = __shfl_sync(0xffffffffu, good, 0);
+                tc::fence_proxy_async_global();                // every lane: whichever lane is elected issues the copies
+                return good != 0;
+            };
+            int ready_img = -1;
+            if (p.flags != nullptr) ok = wait_count(p.flags, (unsigned)p.pack_units);
             for (int item = pair; item < p.n_items && ok; item += n_pairs) {
-                const int m0 = (item % p.pairs_per_ntile) * 256 + (int)rank * BM;
-                const int nt_idx = item / p.pairs_per_ntile;
-                const int img = nt_idx / p.tiles_per_img, h0 = (nt_idx % p.tiles_per_img) * p.rows_per_tile + (int)rank * half_rows;
+                const PairItem it = pair_item(p, item);
+                if (p.flags != nullptr && it.img != ready_img) {
+                    ok = wait_count(p.flags + 1 + it.img, (unsigned)p.units_per_img);
+                    if (!ok) break;
+                    ready_img = it.img;
+                }
+                const int m0 = it.m0 + (int)rank * BM;
+                const int rows_cta = it.rows >> 1;                       // this block's image rows of the tile
+                const int img = it.img, h0 = it.h0 + (int)rank * rows_cta;
+                const uint32_t tx_bytes = 2u * (uint32_t)(a_bytes + rows_cta * p.W * 128);
+                const CUtensorMap *mx = it.half ? &tm_xq : &tm_x;
                 int kb = 0;
                 for (int r = 0; r < p.taps_r && ok; ++r)
                     for (int sft = 0; sft < p.taps_s && ok; ++sft)
@@ -444,9 +631,9 @@ conv_fprop_tc2_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
                             uint8_t *sa = smem + (size_t)s * stage_bytes, *sb = sa + a_bytes;
                             const uint32_t bar = tc::mapa(tc::smem_u32(&full[s]), 0);
                             if (tc::elect_one()) {
-                                if (rank == 0) tc::mbar_expect_tx_cluster(bar, 2 * (a_bytes + bh_bytes));
+                                if (rank == 0) tc::mbar_expect_tx_cluster(bar, tx_bytes);
                                 tc::tma_load_2d_pair(sa, &tm_w, bar, kb * BK, m0);
-                                tc::tma_load_4d_pair(sb, &tm_x, bar, cb * BK, sft - p.pad, h0 + r - p.pad, img);
+                                tc::tma_load_4d_pair(sb, mx, bar, cb * BK, sft - p.pad, h0 + r - p.pad, img);
                             }
                             __syncwarp();
                             if (++s == STAGES) { s = 0; phase ^= 1; }
@@ -457,13 +644,14 @@ conv_fprop_tc2_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
         // the whole warp runs the issue loop with warp-uniform values, an elected lane issues (descriptors stay in
         // uniform registers: an MMA costs the issuing warp far fewer cycles than from one divergent lane)
         if (rank == 0) {
-            const uint32_t idesc = tc::instr_desc_bf16(256, p.nt, false, false);
+            const uint32_t idesc_full = tc::instr_desc_bf16(256, p.nt, false, false), idesc_half = tc::instr_desc_bf16(256, p.nt >> 1, false, false);
             const uint64_t desc_a0 = tc::smem_desc(tc::smem_u32(smem), 16, 1024), desc_b0 = tc::smem_desc(tc::smem_u32(smem) + a_bytes, 16, 1024);
             uint32_t t_local = 0, phase = 0, stage_off = 0;
             int s = 0;
             bool ok = true;
             for (int item = pair; item < p.n_items && ok; item += n_pairs, ++t_local) {
                 const int buf = t_local & 1;
+                const uint32_t idesc = item >= p.n_full ? idesc_half : idesc_full;
                 if (!__all_sync(0xffffffffu, tc::mbar_wait(&tmem_empty[buf], ((t_local >> 1) & 1) ^ 1, abort_flag, p.err, tc::ERR_WAIT_TMEM_EMPTY))) break;
                 tc::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * 256;
@@ -488,9 +676,9 @@ conv_fprop_tc2_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
         uint32_t t_local = 0, blk_count = 0;
         for (int item = pair; item < p.n_items; item += n_pairs, ++t_local) {
             const int buf = t_local & 1;
-            const int m0 = (item % p.pairs_per_ntile) * 256 + (int)rank * BM;
-            const int nt_idx = item / p.pairs_per_ntile;
-            const int img = nt_idx / p.tiles_per_img, h0 = (nt_idx % p.tiles_per_img) * p.rows_per_tile;
+            const PairItem it = pair_item(p, item);
+            const int m0 = it.m0 + (int)rank * BM;
+            const int img = it.img, h0 = it.h0;
             int ok = 1;
             if (lane == 0) ok = tc::mbar_wait(&tmem_full[buf], (t_local >> 1) & 1, abort_flag, p.err, tc::ERR_WAIT_TMEM_FULL) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -502,54 +690,88 @@ conv_fprop_tc2_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
             if (p.bias != nullptr && o < p.Cout)
                 bias = p.bias_bf16 ? __bfloat162float(((const __nv_bfloat16 *)p.bias)[o]) : ((const float *)p.bias)[o];
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * 256;
+            if (!it.half) {
 #pragma unroll 1
-            for (int c = 0; c < p.nt / 32; ++c, ++blk_count) {
-                uint32_t r[32];
-                tc::tmem_ld_32x32(taddr + c * 32, r);
-                tc::tmem_ld_wait();
-                float v[32];
+                for (int c = 0; c < p.nt / 32; ++c, ++blk_count) {
+                    uint32_t r[32];
+                    tc::tmem_ld_32x32(taddr + c * 32, r);
+                    tc::tmem_ld_wait();
+                    float v[32];
 #pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) + bias;
-                switch (p.act) {
-                case RELAY_ACT_RELU:
+                    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) + bias;
+                    switch (p.act) {
+                    case RELAY_ACT_RELU:
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.0f);
-                    break;
-                case RELAY_ACT_TANH:
+                        for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.0f);
+                        break;
+                    case RELAY_ACT_TANH:
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = tanh_<true>(v[j]);
-                    break;
-                case RELAY_ACT_SIGMOID:
+                        for (int j = 0; j < 32; ++j) v[j] = tanh_<true>(v[j]);
+                        break;
+                    case RELAY_ACT_SIGMOID:
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = sigmoid_<true>(v[j]);
-                    break;
-                default: break;
+                        for (int j = 0; j < 32; ++j) v[j] = sigmoid_<true>(v[j]);
+                        break;
+                    default: break;
+                    }
+                    uint8_t *st = my_stage + (blk_count & 1) * 2048;
+                    if (tc::elect_one()) tc::tma_store_wait_read<1>();   // always the same lane of the warp
+                    __syncwarp();
+                    // 32 rows x 64 bytes in the 64-byte swizzle pattern of the output tensor map (16-byte piece q of row r at
+                    // piece q ^ ((r >> 1) & 3)): conflict-free stores
+                    if (p.out_nhwc) {
+                        // pixel-major block: row j = pixel j, this lane's channel is element `lane` of the row (the 32 lanes of
+                        // a store fill one 64-byte row, so the 2-byte stores are conflict-free as well)
+                        uint8_t *col = st + ((lane & 7) << 1);
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            *reinterpret_cast<__nv_bfloat16 *>(col + j * 64 + (((lane >> 3) ^ ((j >> 1) & 3)) << 4)) = __float2bfloat16_rn(v[j]);
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+                            *reinterpret_cast<uint4 *>(st + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4)) =
+                                make_uint4(pack2(v[8 * q], v[8 * q + 1]), pack2(v[8 * q + 2], v[8 * q + 3]), pack2(v[8 * q + 4], v[8 * q + 5]),
+                                           pack2(v[8 * q + 6], v[8 * q + 7]));
+                    }
+                    tc::fence_proxy_async();
+                    __syncwarp();
+                    if (tc::elect_one()) {
+                        if (p.out_nhwc) tc::tma_store_2d(&tm_y, st, o0, (img * p.H + h0) * p.W + c * 32);
+                        else tc::tma_store_2d(&tm_y, st, h0 * p.W + c * 32, img * p.Cout + o0);
+                        tc::tma_store_commit();
+                    }
                 }
-                uint8_t *st = my_stage + (blk_count & 1) * 2048;
-                if (tc::elect_one()) tc::tma_store_wait_read<1>();   // always the same lane of the warp
-                __syncwarp();
-                // 32 rows x 64 bytes in the 64-byte swizzle pattern of the output tensor map (16-byte piece q of row r at
-                // piece q ^ ((r >> 1) & 3)): conflict-free stores
-                if (p.out_nhwc) {
-                    // pixel-major block: row j = pixel j, this lane's channel is element `lane` of the row (the 32 lanes of
-                    // a store fill one 64-byte row, so the 2-byte stores are conflict-free as well)
-                    uint8_t *col = st + ((lane & 7) << 1);
+            } else {
+                // half tile: nt / 2 pixels in chunks of 16 (nt / 2 is a multiple of 16, not always of 32); unswizzled staging:
+                // NCHW 32 channel rows of 32 bytes, NHWC 16 pixel rows of 64 bytes
+#pragma unroll 1
+                for (int c = 0; c < (p.nt >> 1) / 16; ++c, ++blk_count) {
+                    uint32_t r[16];
+                    tc::tmem_ld_32x16(taddr + c * 16, r);
+                    tc::tmem_ld_wait();
+                    float v[16];
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        *reinterpret_cast<__nv_bfloat16 *>(col + j * 64 + (((lane >> 3) ^ ((j >> 1) & 3)) << 4)) = __float2bfloat16_rn(v[j]);
-                } else {
+                    for (int j = 0; j < 16; ++j) v[j] = act_fwd<true>(__uint_as_float(r[j]) + bias, p.act);
+                    uint8_t *st = my_stage + (blk_count & 1) * 2048;
+                    if (tc::elect_one()) tc::tma_store_wait_read<1>();
+                    __syncwarp();
+                    if (p.out_nhwc) {
 #pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        *reinterpret_cast<uint4 *>(st + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4)) =
-                            make_uint4(pack2(v[8 * q], v[8 * q + 1]), pack2(v[8 * q + 2], v[8 * q + 3]), pack2(v[8 * q + 4], v[8 * q + 5]),
-                                       pack2(v[8 * q + 6], v[8 * q + 7]));
-                }
-                tc::fence_proxy_async();
-                __syncwarp();
-                if (tc::elect_one()) {
-                    if (p.out_nhwc) tc::tma_store_2d(&tm_y, st, o0, (img * p.H + h0) * p.W + c * 32);
-                    else tc::tma_store_2d(&tm_y, st, h0 * p.W + c * 32, img * p.Cout + o0);
-                    tc::tma_store_commit();
+                        for (int j = 0; j < 16; ++j) *reinterpret_cast<__nv_bfloat16 *>(st + j * 64 + lane * 2) = __float2bfloat16_rn(v[j]);
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < 2; ++q)
+                            *reinterpret_cast<uint4 *>(st + lane * 32 + q * 16) =
+                                make_uint4(pack2(v[8 * q], v[8 * q + 1]), pack2(v[8 * q + 2], v[8 * q + 3]), pack2(v[8 * q + 4], v[8 * q + 5]),
+                                           pack2(v[8 * q + 6], v[8 * q + 7]));
+                    }
+                    tc::fence_proxy_async();
+                    __syncwarp();
+                    if (tc::elect_one()) {
+                        if (p.out_nhwc) tc::tma_store_2d(&tm_yt, st, o0, (img * p.H + h0) * p.W + c * 16);
+                        else tc::tma_store_2d(&tm_yt, st, h0 * p.W + c * 16, img * p.Cout + o0);
+                        tc::tma_store_commit();
+                    }
                 }
             }
             tc::tc_fence_before_sync();
@@ -565,6 +787,7 @@ conv_fprop_tc2_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
         tc::tc_fence_after_sync();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
+    if (p.flags != nullptr && threadIdx.x == 0) asm volatile("griddepcontrol.wait;" ::: "memory");   // see the start of the kernel
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -830,7 +1053,7 @@ struct TcPlan {
     int wg_nt = 0, wg_c_tiles = 0, wg_m_tiles = 0, wg_slices = 0, wg_imgs_per_slice = 0, wg_stages = 0;
     bool wg_pair = false;    // two-SM wgrad: units of 256 output x 256 input channels computed by pairs of blocks
     int fp_stages = 0;
-    size_t x_nhwc = 0, dz_nhwc = 0, wpack = 0, part = 0, db_part = 0;
+    size_t x_nhwc = 0, dz_nhwc = 0, wpack = 0, part = 0, db_part = 0, flags = 0;
 };
 
 constexpr size_t kSmemLimit = 227 * 1024 - 2048;
@@ -880,6 +1103,7 @@ TcPlan plan(const ConvDims &d)
     pl.wpack = align_up((size_t)d.O * d.C * 9 * 2, 1024);
     pl.part = align_up((size_t)pl.wg_slices * 9 * d.O * d.C * sizeof(float), 1024);
     pl.db_part = align_up((size_t)d.Nb * ((d.H * d.W + 63) / 64) * d.O * sizeof(float), 1024);   // one partial row per repack block
+    pl.flags = align_up((size_t)(1 + d.Nb) * sizeof(unsigned int), 1024);                          // counters of the repack kernel that runs beside a conv
     pl.ok = true;
     return pl;
 }
@@ -900,8 +1124,11 @@ int sm_count()
 }
 
 // `out_nhwc` (only where fprop_pair_form holds): `out` is [Nb][H][W][Cout] instead of [Nb][Cout][H][W]
+// `flags` (only where fprop_pair_form holds): the activations and packed weights are being produced by a repack_stream_kernel
+// launched just before on the same stream; see there
 relay_status_t launch_fprop(const ConvDims &d, const TcPlan &pl, const void *act_nhwc, int Cin, const void *wpacked, int Cout,
-                            const void *bias, int32_t b_dt, int act, void *out_nchw, cudaStream_t st, bool out_nhwc = false)
+                            const void *bias, int32_t b_dt, int act, void *out_nchw, cudaStream_t st, bool out_nhwc = false,
+                            const unsigned int *flags = nullptr, int pack_units = 0)
 {
     CUtensorMap tm_w, tm_x, tm_y;
     RELAY_TRY(make_tmap_2d_bf16(&tm_w, wpacked, (uint64_t)9 * Cin, Cout, (uint64_t)9 * Cin, BK, BM));
@@ -918,9 +1145,10 @@ relay_status_t launch_fprop(const ConvDims &d, const TcPlan &pl, const void *act
     p.err = device_error_word();
     if (!p.err) return fail(RELAY_ERR_CUDA, "no device error word");
     // two-SM form: every tile is computed by a pair of blocks, each loading half of the activation tile
-    if (out_nhwc && !fprop_pair_form(d, pl, Cout, sms)) return fail(RELAY_ERR_UNSUPPORTED, "conv2d: no pixel-major store in the one-SM kernel");
+    if ((out_nhwc || flags) && !fprop_pair_form(d, pl, Cout, sms)) return fail(RELAY_ERR_UNSUPPORTED, "conv2d: not in the one-SM kernel");
+    p.flags = flags; p.pack_units = pack_units; p.units_per_img = (int)((d.H * d.W + 63) / 64);
     if (fprop_pair_form(d, pl, Cout, sms)) {
-        CUtensorMap tm_xh, tm_y2;
+        CUtensorMap tm_xh, tm_y2, tm_xq, tm_yt;
         RELAY_TRY(make_tmap_nhwc_bf16(&tm_xh, act_nhwc, Cin, d.W, d.H, d.Nb, BK, (uint32_t)d.W, pl.rows_per_tile / 2));
         // output boxes of 32 channels x 32 pixels (NHWC: 32 pixels x 32 channels), rows of 64 bytes in the 64-byte swizzle pattern
         if (out_nhwc) RELAY_TRY(make_tmap_2d_sw64(&tm_y2, false, out_nchw, (uint64_t)Cout, (uint64_t)(d.Nb * d.H * d.W), (uint64_t)Cout, 32));
@@ -929,10 +1157,21 @@ relay_status_t launch_fprop(const ConvDims &d, const TcPlan &pl, const void *act
         const size_t stage2 = (size_t)BM * BK * 2 + (size_t)(p.nt / 2) * 128;
         p.stages = (int)std::min<size_t>(8, (kSmemLimit - 1024 - 4 * 4096) / stage2);
         p.pairs_per_ntile = Cout / 256;
-        p.n_pairs = p.n_items = p.n_tiles_total * p.pairs_per_ntile;
+        p.n_pairs = p.n_items = p.n_full = p.n_tiles_total * p.pairs_per_ntile;
+        // the items that would start one more round over the pairs, if they are at most half a round, run as half tiles
+        const int pairs = std::min(p.n_items, sms / 2), rest = p.n_items % pairs;
+        const bool can_halve = pl.rows_per_tile % 4 == 0 && ((p.nt / 4) * 128) % 1024 == 0 && (p.nt / 2) % 16 == 0;
+        tm_xq = tm_xh; tm_yt = tm_y2;
+        if (can_halve && p.n_items > pairs && rest != 0 && 2 * rest <= pairs) {
+            p.n_full = p.n_items - rest;
+            p.n_items = p.n_full + 2 * rest;
+            RELAY_TRY(make_tmap_nhwc_bf16(&tm_xq, act_nhwc, Cin, d.W, d.H, d.Nb, BK, (uint32_t)d.W, pl.rows_per_tile / 4));
+            if (out_nhwc) RELAY_TRY(make_tmap_2d(&tm_yt, false, out_nchw, (uint64_t)Cout, (uint64_t)(d.Nb * d.H * d.W), (uint64_t)Cout, 32, 16, false));
+            else RELAY_TRY(make_tmap_2d(&tm_yt, false, out_nchw, (uint64_t)(d.H * d.W), (uint64_t)d.Nb * Cout, (uint64_t)(d.H * d.W), 16, 32, false));
+        }
         const size_t smem2 = 1024 + (size_t)p.stages * stage2 + 4 * 4096 + 256;
         RELAY_CUDA(cudaFuncSetAttribute(conv_fprop_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2));
-        RELAY_CUDA(launch_pdl(conv_fprop_tc2_kernel, dim3(2 * std::min(p.n_items, sms / 2)), dim3(NUM_THREADS), smem2, st, tm_w, tm_xh, tm_y2, p));
+        RELAY_CUDA(launch_pdl(conv_fprop_tc2_kernel, dim3(2 * pairs), dim3(NUM_THREADS), smem2, st, tm_w, tm_xh, tm_y2, tm_xq, tm_yt, p));
         return check_launch("conv_fprop_tc2");
     }
     // one-SM form: pairs fill whole rounds over the SMs; the remainder runs as singles
@@ -977,6 +1216,32 @@ relay_status_t launch_transpose(bool grad, const void *in, const void *y, void *
     return check_launch("nchw_to_nhwc");
 }
 
+// Launches the persistent repack beside which the next kernel of the stream (a two-SM conv given `flags`) runs.
+// job0 is the tensor that conv consumes (counted per image); job1 (optional) only has to be complete when that conv ends.
+relay_status_t launch_repack_stream(const ConvDims &d, const RepackJob &job0, const RepackJob *job1, const void *w, void *wf, void *wb,
+                                    unsigned int *flags, int *pack_units, cudaStream_t st)
+{
+    RepackStream S{};
+    S.job[0] = job0; S.n_jobs = 1;
+    if (job1) { S.job[1] = *job1; S.n_jobs = 2; }
+    S.Nb = (int)d.Nb; S.HW = (int)(d.H * d.W); S.pbx = (S.HW + 63) / 64;
+    S.pack.w = (const __nv_bfloat16 *)w; S.pack.wf = (__nv_bfloat16 *)wf; S.pack.wb = (__nv_bfloat16 *)wb;
+    S.pack.O = (int)d.O; S.pack.C = (int)d.C; S.pack.taps = 9; S.pack.n_img = 0;
+    S.pack_units = (int)((d.O * d.C * 9 + kPackPerUnit - 1) / kPackPerUnit);
+    S.flags = flags;
+    *pack_units = S.pack_units;
+    RELAY_CUDA(cudaMemsetAsync(flags, 0, (size_t)(1 + d.Nb) * sizeof(unsigned int), st));
+    // the SMs must already be split for the most shared memory while this kernel runs: a consumer block that needed another
+    // split could only start on an SM once it had drained
+    RELAY_CUDA(cudaFuncSetAttribute(repack_stream_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared));
+    int per_sm = 0;
+    RELAY_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, repack_stream_kernel, 256, 0));
+    const int64_t total = S.pack_units + (int64_t)S.n_jobs * S.Nb * S.pbx;
+    const int grid = (int)std::min<int64_t>(total, (int64_t)sm_count() * std::max(1, std::min(per_sm, 2)));
+    RELAY_CUDA(launch_pdl(repack_stream_kernel, dim3((unsigned)grid), dim3(256), 0, st, S));
+    return check_launch("repack_stream");
+}
+
 }  // namespace
 
 relay_status_t make_tmap_nhwc_bf16(CUtensorMap *m, const void *base, uint64_t C, uint64_t W, uint64_t H, uint64_t N,
@@ -1011,7 +1276,7 @@ size_t conv_tc_fwd_workspace(const ConvDims &d)
 size_t conv_tc_grad_workspace(const ConvDims &d)
 {
     TcPlan pl = plan(d);
-    return pl.ok ? pl.x_nhwc + pl.dz_nhwc + pl.wpack + pl.part + pl.db_part : 0;
+    return pl.ok ? pl.x_nhwc + pl.dz_nhwc + pl.wpack + pl.part + pl.db_part + pl.flags : 0;
 }
 
 relay_status_t launch_conv_fwd_tc(const ConvDims &d, const void *x, bool x_is_nhwc, const void *w, const void *b, int32_t b_dt, int act,
@@ -1046,7 +1311,21 @@ relay_status_t launch_conv_grad_tc(const ConvDims &d, const void *x, const void 
     float *part = (float *)(base + pl.x_nhwc + pl.dz_nhwc + pl.wpack);
     float *db_part = (float *)(base + pl.x_nhwc + pl.dz_nhwc + pl.wpack + pl.part);
     const int64_t HW = d.H * d.W;
-    if (nhwc_in) {
+    const bool beside = !nhwc_in && dx && !dx_nhwc && fprop_pair_form(d, pl, (int)d.C, sm_count());
+    if (beside) {
+        // One persistent repack kernel writes dZ = dy (.) act'(y) in NHWC (with the bias-gradient partials), then x in NHWC, and
+        // packs the mirrored weights; the input-gradient conv runs BESIDE it, taking each image of dZ as soon as it is complete.
+        // That conv ends only after the repack kernel has, so the weight-gradient kernel behind it finds x complete.
+        unsigned int *flags = (unsigned int *)(base + pl.x_nhwc + pl.dz_nhwc + pl.wpack + pl.part + pl.db_part);
+        RepackJob jz{}, jx{};
+        jz.in = (const __nv_bfloat16 *)dy; jz.y = (const __nv_bfloat16 *)y; jz.out = (__nv_bfloat16 *)dz_nhwc; jz.db_part = db ? db_part : nullptr;
+        jz.C = (int)d.O; jz.grad = 1; jz.act = act; jz.flagged = 1;
+        jx.in = (const __nv_bfloat16 *)x; jx.out = (__nv_bfloat16 *)base; jx.C = (int)d.C;
+        int pack_units = 0;
+        RELAY_TRY(launch_repack_stream(d, jz, &jx, w, nullptr, wb, flags, &pack_units, st));
+        RELAY_TRY(launch_fprop(d, pl, dz_nhwc, (int)d.O, wb, (int)d.C, nullptr, RELAY_F32, RELAY_ACT_NONE, dx, st, false, flags, pack_units));
+        if (db) RELAY_TRY(launch_colsum_finalize(db_part, (int)(d.Nb * ((HW + 63) / 64)), d.O, 1.0f, db, st));
+    } else if (nhwc_in) {
         // x, y, dy are NHWC already: dZ = dy (.) act'(y) is one elementwise pass over [N*H*W, O] whose column sums are db;
         // x is read where it lies
         RELAY_TRY(launch_act_grad(RELAY_BF16, dy, y, dz_nhwc, db, nhwc_partials, d.Nb * HW, d.O, act, st));
@@ -1059,7 +1338,7 @@ relay_status_t launch_conv_grad_tc(const ConvDims &d, const void *x, const void 
         RELAY_TRY(launch_transpose(false, x, nullptr, base, d.Nb, d.C, HW, 0, nullptr, st));
         if (db) RELAY_TRY(launch_colsum_finalize(db_part, (int)(d.Nb * ((HW + 63) / 64)), d.O, 1.0f, db, st));
     }
-    if (dx) {
+    if (dx && !beside) {
         if (nhwc_in) {
             RELAY_CUDA(launch_pdl(pack_weights_kernel, dim3((unsigned)((d.O * d.C * 9 + 255) / 256)), dim3(256), 0, st, (const __nv_bfloat16 *)w, (__nv_bfloat16 *)nullptr, (__nv_bfloat16 *)wb, (int)d.O, (int)d.C, 3, 3));
             RELAY_TRY(check_launch("pack_weights"));
@@ -1094,7 +1373,7 @@ relay_status_t launch_conv_grad_tc(const ConvDims &d, const void *x, const void 
         RELAY_CUDA(launch_pdl(conv_wgrad_tc_kernel, dim3(grid), dim3(NUM_THREADS), smem, st, tm_dz, tm_x, tm_part, p));
     }
     RELAY_TRY(check_launch("conv_wgrad_tc"));
-    RELAY_CUDA(launch_pdl(wgrad_reduce_kernel, dim3((unsigned)((9 * d.O * d.C + 255) / 256)), dim3(256), 0, st, (const float *)part, p.n_slices, (__nv_bfloat16 *)dw, (int)d.O, (int)d.C, 9));
+    RELAY_CUDA(launch_pdl(wgrad_reduce_kernel, dim3((unsigned)((d.O * d.C + 127) / 128)), dim3(128), 0, st, (const float *)part, p.n_slices, (__nv_bfloat16 *)dw, (int)d.O, (int)d.C, 9));
     return check_launch("wgrad_reduce");
 }
 
