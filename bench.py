@@ -230,6 +230,14 @@ class Workload:
             self.red_specs = dict(sum1=[(0, B.RED_SUM, 2, 0)], max1=[(0, B.RED_MAX, 2, 0)], arg1=[(0, B.RED_ARGMAX, 2, 0)],
                                   sum0=[(0, B.RED_SUM, 1, 0)])
             ws_bytes = max(ws_bytes, B.relay_workspace_bytes_reduce([self.devt["cfg2"]["x"]], self.red_specs["sum0"]))
+            # two programs that have no pre-compiled body (they run on the vectorised evaluator): out = sigmoid(x*y) + relu(z)
+            # with z constant down the rows, and its gradient group (dx, dy unreduced, dz summed over the rows)
+            self.vm_fwd, self.vm_fwd_outs = P.sigmoid_product_relu_fwd(P.BF16)
+            self.vm_grad, ids = P.sigmoid_product_relu_grad(P.BF16)
+            self.vm_grad_specs = [(ids[0], B.RED_NONE, 0, 0), (ids[1], B.RED_NONE, 0, 0), (ids[2], B.RED_SUM, 1, 0)]
+            self.vm_out = dict(out=E(r, c), dx=E(r, c), dy=E(r, c), dz=E(c, dt=f32))
+            d = self.devt["cfg2"]
+            ws_bytes = max(ws_bytes, B.relay_workspace_bytes_reduce([d["dout"], d["x"], d["dout"], d["a"]], self.vm_grad_specs))
         if "cfg3" in groups:
             m, k = self.host["cfg3"]["x"].shape
             o = dict()
@@ -355,6 +363,13 @@ class Workload:
             with tm.region("cfg2.grad"):
                 B.relay_fused_reduce(self.grad_prog.arrays(), [d["dout"], d["x"], d["a"], d["b"]], self.grad_specs,
                                      [o["dx"], o["da"], o["db"]], ws)
+            self.flush_l2()
+            with tm.region("a6.vm_fwd"):
+                B.relay_fused_ewise(self.vm_fwd.arrays(), [d["x"], d["dout"], d["a"]], self.vm_fwd_outs, [self.vm_out["out"]], ws)
+            self.flush_l2()
+            with tm.region("a7.vm_grad"):
+                B.relay_fused_reduce(self.vm_grad.arrays(), [d["dout"], d["x"], o["out"], d["a"]], self.vm_grad_specs,
+                                     [self.vm_out["dx"], self.vm_out["dy"], self.vm_out["dz"]], ws)
             ra = self.red_prog.arrays()
             for key in ("sum1", "max1", "arg1", "sum0"):
                 self.flush_l2()
@@ -441,6 +456,7 @@ class Workload:
             r, c = self.host["cfg2"]["x"].shape
             w["cfg2.fwd"] = dict(bytes=2 * r * c * 2 + 2 * c * 2)
             w["cfg2.grad"] = dict(bytes=3 * r * c * 2 + 2 * c * 2 + 2 * c * 4)
+            w["a6.vm_fwd"] = dict(bytes=3 * r * c * 2 + c * 2); w["a7.vm_grad"] = dict(bytes=5 * r * c * 2 + c * 2 + c * 4)
             w["a8.sum1"] = dict(bytes=r * c * 2 + r * 4); w["a8.max1"] = dict(bytes=r * c * 2 + r * 4)
             w["a8.arg1"] = dict(bytes=r * c * 2 + r * 8); w["a8.sum0"] = dict(bytes=r * c * 2 + c * 4)
         if "cfg3" in self.groups:
@@ -650,7 +666,7 @@ def main():
     step_ms_max = max_over_ranks(step_ms, dist, dev)
 
     tensor_keys = [k for k in top if k.startswith(("cfg3", "cfg4"))]
-    hbm_keys = [k for k in top if k.startswith(("cfg2", "a8"))]
+    hbm_keys = [k for k in top if k.startswith(("cfg2", "a6", "a7", "a8"))]
     t_ms = max_over_ranks(sum(float(np.mean(tm.ms[k])) for k in tensor_keys), dist, dev)
     h_ms = max_over_ranks(sum(float(np.mean(tm.ms[k])) for k in hbm_keys), dist, dev)
     tflops = whole_job(sum(work[k]["flop"] for k in tensor_keys), world, t_ms) / 1e12 if t_ms else None
@@ -717,7 +733,9 @@ def main():
             a = table[key]["gbs"]
             rooflines[name] = {"bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": a / peaks["hbm_gbs"],
                                "traffic": traffic_of(key), "peak_source": peaks["source"] + " (of measured)"}
-    for key, name in (("a8.sum1", "rowreduce_kernel<sum> (8192x8192 bf16 over the last axis)"),
+    for key, name in (("a6.vm_fwd", "ewise_vm_kernel, out = sigmoid(x*y) + relu(z) (8192x8192 bf16, interpreted stack program)"),
+                      ("a7.vm_grad", "ewise_vm_kernel + finalize, gradient group of the same (dx, dy, column sum dz)"),
+                      ("a8.sum1", "rowreduce_kernel<sum> (8192x8192 bf16 over the last axis)"),
                       ("a8.max1", "rowreduce_kernel<max> (8192x8192 bf16 over the last axis)"),
                       ("a8.arg1", "rowreduce_kernel<argmax> (8192x8192 bf16 over the last axis, int64 indices)"),
                       ("a8.sum0", "ewise2d_kernel<identity_colsum> + finalize (8192x8192 bf16 over axis 0)")):
@@ -818,11 +836,11 @@ def main():
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 (fp32 accumulate); cfg1 f32",
                 "data": "synthetic",
                 "config": {"workload": ("reduced shapes" if args.small else "all five configurations at full size")
-                           + ": step = cfg1 fwd+grad, cfg2 fwd+grad, four standalone reductions of the cfg2 tensor (sum / max / argmax over the last axis, sum over axis 0), cfg3 3-layer fwd+bwd, cfg4 conv fwd+dX+dW+db, cfg5 LSTM forward + gradient program"
+                           + ": step = cfg1 fwd+grad, cfg2 fwd+grad, an elementwise program and its gradient group on the vectorised evaluator, four standalone reductions of the cfg2 tensor (sum / max / argmax over the last axis, sum over axis 0), cfg3 3-layer fwd+bwd, cfg4 conv fwd+dX+dW+db, cfg5 LSTM forward + gradient program"
                            + ", then softmax cross-entropy loss / loss+partial on 8192x8192 bf16, SGD on three 4096^2 bf16 matrices and 2x2 max pooling"
                            + " forward + gradient on 32x256x56x56 bf16, one fp32 LeNet training step (batch 64) eager and replayed from a"
                            + " CUDA graph, the cfg4 conv with NHWC-tagged tensors; cfg1 is also replayed from a CUDA graph",
-                           "value_covers": "dense + conv2d groups (cfg3 + cfg4) FLOPs / their device time; hbm_gbs covers cfg2 and the standalone reductions (a8.*)",
+                           "value_covers": "dense + conv2d groups (cfg3 + cfg4) FLOPs / their device time; hbm_gbs covers cfg2, two programs on the vectorised evaluator (a6.vm_fwd, a7.vm_grad) and the standalone reductions (a8.*)",
                            "groups": groups, "l2": "1 GiB streamed through L2 between groups (flush with clean lines); cfg2 inputs also exceed L2",
                            "replicas": world},
                 "groups": table, "roofline": roofline, "rooflines": rooflines, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),

@@ -393,9 +393,10 @@ const char *relay_last_error(void);
 relay_status_t relay_contract_act(const relay_tensor_t *a, int32_t trans_a, const relay_tensor_t *b, int32_t trans_b,
                                   const relay_tensor_t *bias, int32_t act, const relay_tensor_t *c, void *stream);
 
-/* Synchronises `stream`, then reads and clears the device-side error word of the current
- * device: RELAY_ERR_TIMEOUT if a bounded wait expired in any kernel since the last poll,
- * RELAY_ERR_CUDA if the stream reports an error, else RELAY_OK. */
+/* Synchronises `stream`, then reads and clears (in one atomic step, enqueued on `stream`) the device-side error word
+ * of the current device: RELAY_ERR_TIMEOUT if a bounded wait expired in any kernel since the last poll,
+ * RELAY_ERR_CUDA if the stream reports an error, else RELAY_OK.  The word belongs to the device, not to a stream:
+ * a poll also reports, and consumes, a time-out raised by work of another stream. */
 relay_status_t relay_poll_status(void *stream);
 
 /* Self-test of the time-out path (no counterpart in the paper): enqueues a one-block kernel that
@@ -411,6 +412,15 @@ relay_status_t relay_debug_expire_wait(int32_t limit_us, void *stream);
  * (pair p takes units p, p + sms/2, ...).  Returns the number of units, -1 if the shape is too large for a list
  * (the kernel then follows its fixed scheme), -2 for bad arguments or max_units too small.  For tests of the plan. */
 int32_t relay_debug_plan_units(int64_t M, int64_t N, int64_t K, int32_t sms, uint32_t *units, int32_t max_units);
+
+/* Host-only view of which kernel tier relay_fused_ewise / relay_fused_reduce would run a group on (no counterpart in the
+ * paper; touches no GPU; arguments as for relay_fused_reduce, all-RELAY_RED_NONE specs describe a relay_fused_ewise call):
+ * 0 a pre-compiled body, 1 the vectorised evaluator (16-byte accesses, the program interpreted on 8 elements at a
+ * time), 2 the scalar evaluator (any rank, broadcast pattern, axes mask and base type), 3 the row-reduction kernel;
+ * -1 if the group does not type-check (relay_last_error() says why).  For tests and for callers that want to know
+ * whether a program takes the fast route. */
+int32_t relay_debug_group_route(const relay_ewise_prog_t *prog, const relay_tensor_t *const *inputs, int32_t n_in,
+                                const relay_out_spec_t *specs, int32_t n_out);
 
 /* Number of kernels this library has launched on this process so far (monotonic counter). */
 int64_t relay_launch_count(void);

@@ -299,6 +299,18 @@ def relay_fused_reduce(prog: Optional[dict], inputs, specs, outputs, ws=None):
                                     _desc_array(outs), len(outs), wp, wb, _stream()))
 
 
+def relay_debug_group_route(prog: Optional[dict], inputs, specs) -> int:
+    """Kernel tier a group would run on: 0 pre-compiled body, 1 vectorised evaluator, 2 scalar evaluator, 3 row reduction.
+    specs as for relay_fused_reduce; (value, RED_NONE, 0, 0) entries describe a relay_fused_ewise call.  Host only."""
+    p = make_prog(prog) if prog is not None else None
+    ins = [desc(t) for t in inputs]
+    sp = (OutSpec * max(len(specs), 1))(*[OutSpec(*s) for s in specs])
+    r = int(lib().relay_debug_group_route(ctypes.byref(p) if p is not None else None, _desc_array(ins), len(ins), sp, len(specs)))
+    if r < 0:
+        raise RelayError(1, lib().relay_last_error().decode())
+    return r
+
+
 STATIC_SCRATCH_BYTES = 8 << 20
 
 

@@ -131,7 +131,11 @@ relay_status_t check_no_overlap(const relay_tensor_t *const *outs, int n_out, co
     return RELAY_OK;
 }
 
-__device__ int g_error_word = 0;
+// [0]: the error word that kernels set; [1]: where relay_poll_status has it exchanged to.  One pair per device, shared by
+// all streams: a poll reports (and clears) a time-out of any stream's kernel.
+__device__ int g_error_word[2] = {0, 0};
+
+__global__ void poll_exchange_kernel(int *word, int *result) { *result = atomicExch(word, 0); }
 
 int *device_error_word()
 {
@@ -141,7 +145,7 @@ int *device_error_word()
     std::lock_guard<std::mutex> lk(g_mu);
     if (!addr[dev]) {
         void *p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_error_word) != cudaSuccess) return nullptr;
+        if (cudaGetSymbolAddress(&p, g_error_word) != cudaSuccess) return nullptr;   // address of element [0]
         addr[dev] = (int *)p;
     }
     return addr[dev];
@@ -188,13 +192,14 @@ relay_status_t relay_poll_status(void *stream)
     if (e != cudaSuccess) return fail(RELAY_ERR_CUDA, "stream reports: %s", cudaGetErrorString(e));
     int *w = device_error_word();
     if (!w) return fail(RELAY_ERR_CUDA, "no device error word (no CUDA device?)");
+    // read and clear in one step (a kernel of another stream may set the word at any time): atomic exchange on the
+    // device, result through a second word
     int v = 0;
-    RELAY_CUDA(cudaMemcpy(&v, w, sizeof(int), cudaMemcpyDeviceToHost));
-    if (v != 0) {
-        int zero = 0;
-        RELAY_CUDA(cudaMemcpy(w, &zero, sizeof(int), cudaMemcpyHostToDevice));
-        return fail(RELAY_ERR_TIMEOUT, "a bounded device-side wait expired (code %d)", v);
-    }
+    poll_exchange_kernel<<<1, 1, 0, (cudaStream_t)stream>>>(w, w + 1);
+    RELAY_TRY(check_launch("poll_exchange"));
+    RELAY_CUDA(cudaMemcpyAsync(&v, w + 1, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    RELAY_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    if (v != 0) return fail(RELAY_ERR_TIMEOUT, "a bounded device-side wait expired (code %d)", v);
     return RELAY_OK;
 }
 
@@ -278,6 +283,8 @@ relay_status_t relay_infer_broadcast(const relay_tensor_t *a, const relay_tensor
     RELAY_TRY(check_not_null(out, "out"));
     RELAY_TRY(check_type(a, "a"));
     RELAY_TRY(check_type(b, "b"));
+    // the operator that follows the broadcast step needs one base type (Fig. 5, Type-Noncomp-BinaryOp)
+    if (a->dtype != b->dtype) return fail(RELAY_ERR_DTYPE, "broadcast: base types %s and %s differ", dtype_name(a->dtype), dtype_name(b->dtype));
     int r = a->rank > b->rank ? a->rank : b->rank;
     int64_t s[RELAY_MAX_RANK];
     for (int d = 0; d < r; ++d) {

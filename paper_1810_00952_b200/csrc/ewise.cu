@@ -130,9 +130,9 @@ __global__ void __launch_bounds__(kTX *kTY, Body::NIN >= 4 ? 2 : 3) ewise2d_kern
 // second pass of a column sum: thread (tx, ty) adds the partials of slices ty, ty+TY, ... of its column in
 // slice order, then the TY row-threads are combined in ty order (fixed order, so reruns are bit-identical).
 // grid.y indexes the summed result k: partials at partial + k * n_slices * cols, output out[k].
-struct FinalizeOuts { float *out[RELAY_MAX_OUTPUTS]; };
+struct FinalizeOuts { float *out[RELAY_MAX_OUTPUTS]; float scale[RELAY_MAX_OUTPUTS]; };
 template <int TY>
-__global__ void __launch_bounds__(32 * TY) colsum_finalize_kernel(const float *__restrict__ partial, int n_slices, int64_t cols, float scale,
+__global__ void __launch_bounds__(32 * TY) colsum_finalize_kernel(const float *__restrict__ partial, int n_slices, int64_t cols,
                                                                   const FinalizeOuts outs)
 {
     __shared__ float sm[TY][33];
@@ -149,7 +149,7 @@ __global__ void __launch_bounds__(32 * TY) colsum_finalize_kernel(const float *_
         float t = 0.0f;
 #pragma unroll
         for (int j = 0; j < TY; ++j) t += sm[j][tx];
-        outs.out[blockIdx.y][c] = t * scale;
+        outs.out[blockIdx.y][c] = t * outs.scale[blockIdx.y];
     }
 }
 
@@ -241,12 +241,12 @@ struct DevOutputs {
 
 __global__ void __launch_bounds__(256) ewise_generic_kernel(const DevProgram P, const DevOutputs O, int64_t total)
 {
-    float vals[kDevMaxValues];
+    Val vals[kDevMaxValues];
     int64_t idx[RELAY_MAX_RANK];
     for (int64_t lin = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; lin < total; lin += (int64_t)gridDim.x * blockDim.x) {
         unravel(lin, P.rank, P.shape, idx);
         eval_program(P, idx, vals);
-        for (int k = 0; k < O.n_out; ++k) store_from_float(O.ptr[k], lin, O.dtype[k], vals[O.value[k]]);
+        for (int k = 0; k < O.n_out; ++k) store_value(O.ptr[k], lin, O.dtype[k], vals[O.value[k]]);
     }
 }
 
@@ -270,7 +270,7 @@ __global__ void __launch_bounds__(256) reduce_generic_kernel(const DevProgram P,
 {
     __shared__ float sbest[8];
     __shared__ long long spos[8];
-    float vals[kDevMaxValues];
+    Val vals[kDevMaxValues];
     int64_t idx[RELAY_MAX_RANK];
     const int lane_in_group = threadIdx.x % R.group;
     const int groups_per_block = blockDim.x / R.group;
@@ -294,7 +294,7 @@ __global__ void __launch_bounds__(256) reduce_generic_kernel(const DevProgram P,
                 rj /= P.shape[ax];
             }
             eval_program(P, idx, vals);
-            float v = vals[R.value];
+            float v = vals[R.value].f;
             if (is_sum) best += v;
             else if (v > best) { best = v; pos = j; }
         }
@@ -412,15 +412,11 @@ static void fill_dev_program(const TypedProgram &tp, const relay_tensor_t *const
     }
     for (int j = 0; j < tp.n_instr; ++j) {
         P->op[j] = (int8_t)tp.instr[j].op; P->a[j] = (int8_t)tp.instr[j].a; P->b[j] = (int8_t)tp.instr[j].b;
-        P->c[j] = (int8_t)tp.instr[j].c; P->dt[j] = (int8_t)tp.instr[j].dtype; P->imm[j] = (float)tp.instr[j].imm;
+        P->c[j] = (int8_t)tp.instr[j].c; P->dt[j] = (int8_t)tp.instr[j].dtype; P->imm[j] = tp.instr[j].imm;
     }
 }
 
-// 2-D view: is every input either full-shape, constant down the rows, or a scalar, all in one
-// float storage type, with whole 16-byte vectors per row?
-struct View2D { bool ok; int64_t rows, cols; int kind[RELAY_MAX_INPUTS]; int32_t storage; };
-
-static View2D view2d(const TypedProgram &tp)
+View2D view2d(const TypedProgram &tp)
 {
     View2D v{};
     v.ok = false;
@@ -479,22 +475,21 @@ relay_status_t launch_body2d(int32_t storage, const Args2D<Body::NIN, Body::NOUT
     return check_launch(what);
 }
 
-// finalises n_out column sums whose partials lie one after another ([k][n_slices][cols])
-relay_status_t launch_colsum_finalize_n(const float *partial, int n_slices, int64_t cols, float scale, float *const *out, int n_out,
+relay_status_t launch_colsum_finalize_n(const float *partial, int n_slices, int64_t cols, const float *scale, float *const *out, int n_out,
                                         cudaStream_t st)
 {
     FinalizeOuts fo{};
-    for (int k = 0; k < n_out; ++k) fo.out[k] = out[k];
+    for (int k = 0; k < n_out; ++k) { fo.out[k] = out[k]; fo.scale[k] = scale ? scale[k] : 1.0f; }
     const dim3 grid((unsigned)((cols + 31) / 32), (unsigned)n_out);
-    if (n_slices > 256) RELAY_CUDA(launch_pdl(colsum_finalize_kernel<32>, grid, dim3(32, 32), 0, st, partial, n_slices, cols, scale, fo));
-    else RELAY_CUDA(launch_pdl(colsum_finalize_kernel<8>, grid, dim3(32, 8), 0, st, partial, n_slices, cols, scale, fo));
+    if (n_slices > 256) RELAY_CUDA(launch_pdl(colsum_finalize_kernel<32>, grid, dim3(32, 32), 0, st, partial, n_slices, cols, fo));
+    else RELAY_CUDA(launch_pdl(colsum_finalize_kernel<8>, grid, dim3(32, 8), 0, st, partial, n_slices, cols, fo));
     return check_launch("colsum_finalize");
 }
 
 relay_status_t launch_colsum_finalize(const float *partial, int n_slices, int64_t cols, float scale, float *out,
                                       cudaStream_t st)
 {
-    return launch_colsum_finalize_n(partial, n_slices, cols, scale, &out, 1, st);
+    return launch_colsum_finalize_n(partial, n_slices, cols, &scale, &out, 1, st);
 }
 
 // dZ = dy (.) act'(y) stored to dz, and (if db) db = column sums of dZ; used by the dense gradient group
@@ -583,6 +578,17 @@ extern "C" relay_status_t relay_fused_ewise(const relay_ewise_prog_t *prog, cons
         return launch_body2d<BodyTanhAffineResidualFwd>(v.storage, A, ns, st, "ewise2d<tanh_affine_residual_fwd>");
     }
 
+    // any other program over the 2-D view: the vectorised evaluator
+    if (v.ok) {
+        VmPlan vp;
+        const bool no_sums[RELAY_MAX_OUTPUTS] = {false};
+        if (vm_plan(tp, v, out_values, no_sums, n_out, &vp)) {
+            const int64_t gx = (v.cols + 255) / 256;
+            const int ns = (int)std::max<int64_t>(1, std::min<int64_t>((148 * 8) / gx, v.rows / 32));
+            return vm_launch(vp, v, inputs, n_in, outputs, n_out, nullptr, ns, st);
+        }
+    }
+
     DevProgram P;
     fill_dev_program(tp, inputs, &P);
     DevOutputs O{};
@@ -601,6 +607,9 @@ struct ReducePlan {
     bool fast_grad = false;     // pre-compiled tanh-affine gradient group
     bool fast_colsum = false;   // identity column sum / mean over all leading axes
     bool fast_row = false;      // identity reduction over the last axis
+    bool vm = false;            // vectorised evaluator: unreduced results and sums / means over all leading axes
+    VmPlan vmp;
+    int32_t vm_values[RELAY_MAX_OUTPUTS];
     int n_slices = 1;
     size_t ws_need = 0;
     int64_t red_shape[RELAY_MAX_OUTPUTS][RELAY_MAX_RANK];
@@ -651,6 +660,19 @@ static relay_status_t plan_reduce(const relay_ewise_prog_t *prog, const relay_te
     if (pl->fast_grad || pl->fast_colsum) {
         pl->n_slices = colsum_slices(v.rows, v.cols, v.storage);
         pl->ws_need = (size_t)(pl->fast_grad ? 2 : 1) * pl->n_slices * (size_t)v.cols * sizeof(float);
+    } else if (!pl->fast_row && v.ok && tp.rank >= 2) {
+        bool sums[RELAY_MAX_OUTPUTS], fits = true;
+        for (int k = 0; k < n_out; ++k) {
+            const bool colsum = (specs[k].red_op == RELAY_RED_SUM || specs[k].red_op == RELAY_RED_MEAN) && specs[k].axes_mask == lead_mask;
+            if (specs[k].red_op != RELAY_RED_NONE && !colsum) fits = false;
+            sums[k] = colsum;
+            pl->vm_values[k] = specs[k].value;
+        }
+        if (fits && vm_plan(tp, v, pl->vm_values, sums, n_out, &pl->vmp)) {
+            pl->vm = true;
+            pl->n_slices = vm_grid_slices(v, colsum_slices(v.rows, v.cols, v.storage));
+            pl->ws_need = (size_t)pl->vmp.n_sum * pl->n_slices * (size_t)v.cols * sizeof(float);
+        }
     }
     return RELAY_OK;
 }
@@ -703,7 +725,7 @@ extern "C" relay_status_t relay_fused_reduce(const relay_ewise_prog_t *prog, con
         A.rows = v.rows; A.cols = v.cols; A.aux = 0;
         RELAY_TRY(launch_body2d<BodyTanhAffineResidualGrad>(v.storage, A, pl.n_slices, st, "ewise2d<tanh_affine_residual_grad>"));
         float *sums[2] = {(float *)outputs[1]->data, (float *)outputs[2]->data};
-        return launch_colsum_finalize_n(A.partial[1], pl.n_slices, v.cols, 1.0f, sums, 2, st);
+        return launch_colsum_finalize_n(A.partial[1], pl.n_slices, v.cols, nullptr, sums, 2, st);
     }
     if (pl.fast_colsum) {
         Args2D<1, 1> A{};
@@ -729,6 +751,19 @@ extern "C" relay_status_t relay_fused_reduce(const relay_ewise_prog_t *prog, con
         }
 #undef ROWRED
         return check_launch("rowreduce");
+    }
+
+    if (pl.vm) {
+        RELAY_TRY(vm_launch(pl.vmp, v, inputs, n_in, outputs, n_out, (float *)ws, pl.n_slices, st));
+        float *sums[RELAY_MAX_OUTPUTS];
+        float scale[RELAY_MAX_OUTPUTS];
+        int n_sum = 0;
+        for (int k = 0; k < n_out; ++k)
+            if (specs[k].red_op != RELAY_RED_NONE) {
+                sums[n_sum] = (float *)outputs[k]->data;
+                scale[n_sum++] = specs[k].red_op == RELAY_RED_MEAN ? 1.0f / (float)v.rows : 1.0f;
+            }
+        return n_sum ? launch_colsum_finalize_n((const float *)ws, pl.n_slices, v.cols, scale, sums, n_sum, st) : RELAY_OK;
     }
 
     // generic: one evaluator pass for the unreduced results, one reduction launch per reduced result
@@ -760,4 +795,26 @@ extern "C" relay_status_t relay_fused_reduce(const relay_ewise_prog_t *prog, con
         RELAY_TRY(check_launch("reduce_generic"));
     }
     return RELAY_OK;
+}
+
+// Which kernel tier a group would run on (host only, launches nothing): 0 a pre-compiled body, 1 the vectorised
+// evaluator, 2 the scalar evaluator, 3 the row-reduction kernel; -1 if the group does not type-check.
+extern "C" int32_t relay_debug_group_route(const relay_ewise_prog_t *prog, const relay_tensor_t *const *inputs, int32_t n_in,
+                                           const relay_out_spec_t *specs, int32_t n_out)
+{
+    clear_error();
+    ReducePlan pl;
+    if (plan_reduce(prog, inputs, n_in, specs, n_out, &pl) != RELAY_OK) return -1;
+    bool all_unreduced = true;
+    for (int k = 0; k < n_out; ++k) all_unreduced = all_unreduced && specs[k].red_op == RELAY_RED_NONE;
+    if (!all_unreduced) return (pl.fast_grad || pl.fast_colsum) ? 0 : pl.fast_row ? 3 : pl.vm ? 1 : 2;
+    const View2D &v = pl.v;
+    if (v.ok && n_out == 1 && n_in == 3 && kinds_match<BodyTanhAffineResidualFwd>(v) && pl.tp.dtype[specs[0].value] == v.storage &&
+        canon(pl.tp, specs[0].value) == known_tanh_affine_fwd(v.storage).out)
+        return 0;
+    VmPlan vp;
+    int32_t values[RELAY_MAX_OUTPUTS];
+    const bool no_sums[RELAY_MAX_OUTPUTS] = {false};
+    for (int k = 0; k < n_out; ++k) values[k] = specs[k].value;
+    return v.ok && vm_plan(pl.tp, v, values, no_sums, n_out, &vp) ? 1 : 2;
 }

@@ -5,6 +5,23 @@
 
 namespace relay {
 
+struct TypedProgram;
+
+// Collapsed 2-D view [rows, cols] of a group: every input is full-shape, constant down the rows, or a scalar, all in one
+// float storage type, with whole 16-byte vectors per row (ok = false otherwise).
+struct View2D { bool ok; int64_t rows, cols; int kind[RELAY_MAX_INPUTS]; int32_t storage; };
+View2D view2d(const TypedProgram &tp);
+
+// Vectorised evaluator for programs without a pre-compiled body (ewise_vm.cu): plan on the host, then launch.
+struct VmPlan { bool ok = false; int n_sum = 0; alignas(8) unsigned char storage[1024]; };
+bool vm_plan(const TypedProgram &tp, const View2D &v, const int32_t *out_values, const bool *colsum, int n_out, VmPlan *plan);
+int vm_grid_slices(const View2D &v, int n_slices_wanted);
+relay_status_t vm_launch(const VmPlan &plan, const View2D &v, const relay_tensor_t *const *inputs, int n_in, const relay_tensor_t *const *outputs,
+                         int n_out, float *partials, int n_slices, cudaStream_t st);
+// finalises n_out column sums whose partials lie one after another ([k][n_slices][cols]); scale[k] multiplies sum k (null: 1)
+relay_status_t launch_colsum_finalize_n(const float *partial, int n_slices, int64_t cols, const float *scale, float *const *out, int n_out,
+                                        cudaStream_t st);
+
 // number of row slices (and therefore of partial rows) a column sum over [rows, cols] uses
 int colsum_slices(int64_t rows, int64_t cols, int32_t storage);
 

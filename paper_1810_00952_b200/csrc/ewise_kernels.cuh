@@ -98,24 +98,32 @@ __device__ __forceinline__ void st_stream(void *p, const uint4 &r)
 }
 
 // ---- scalar typed access (generic evaluator) ----------------------------------------------------
-__device__ __forceinline__ float load_as_float(const void *p, int64_t i, int dt)
+// A program value is held in the lane of its base type: floats (and Bool, as 0 / 1) in `f`, IntType values in `i`
+// as a 64-bit integer, so that integers are exact over their whole range whatever casts they pass through.
+union Val { float f; long long i; };
+__device__ __forceinline__ bool is_int_type(int dt) { return dt == RELAY_I32 || dt == RELAY_I64; }
+
+__device__ __forceinline__ Val load_value(const void *p, int64_t i, int dt)
 {
+    Val v;
+    v.i = 0;
     switch (dt) {
-    case RELAY_F32: return ((const float *)p)[i];
-    case RELAY_BF16: return __bfloat162float(((const __nv_bfloat16 *)p)[i]);
-    case RELAY_I32: return (float)((const int32_t *)p)[i];
-    case RELAY_I64: return (float)((const int64_t *)p)[i];
-    default: return ((const uint8_t *)p)[i] ? 1.0f : 0.0f;
+    case RELAY_F32: v.f = ((const float *)p)[i]; break;
+    case RELAY_BF16: v.f = __bfloat162float(((const __nv_bfloat16 *)p)[i]); break;
+    case RELAY_I32: v.i = ((const int32_t *)p)[i]; break;
+    case RELAY_I64: v.i = ((const int64_t *)p)[i]; break;
+    default: v.f = ((const uint8_t *)p)[i] ? 1.0f : 0.0f; break;
     }
+    return v;
 }
-__device__ __forceinline__ void store_from_float(void *p, int64_t i, int dt, float v)
+__device__ __forceinline__ void store_value(void *p, int64_t i, int dt, Val v)
 {
     switch (dt) {
-    case RELAY_F32: ((float *)p)[i] = v; break;
-    case RELAY_BF16: ((__nv_bfloat16 *)p)[i] = __float2bfloat16_rn(v); break;
-    case RELAY_I32: ((int32_t *)p)[i] = (int32_t)v; break;
-    case RELAY_I64: ((int64_t *)p)[i] = (int64_t)v; break;
-    default: ((uint8_t *)p)[i] = v != 0.0f ? 1 : 0; break;
+    case RELAY_F32: ((float *)p)[i] = v.f; break;
+    case RELAY_BF16: ((__nv_bfloat16 *)p)[i] = __float2bfloat16_rn(v.f); break;
+    case RELAY_I32: ((int32_t *)p)[i] = (int32_t)v.i; break;
+    case RELAY_I64: ((int64_t *)p)[i] = v.i; break;
+    default: ((uint8_t *)p)[i] = v.f != 0.0f ? 1 : 0; break;
     }
 }
 
@@ -127,59 +135,85 @@ struct DevProgram {
     const void *in_ptr[RELAY_MAX_INPUTS];
     int8_t in_dtype[RELAY_MAX_INPUTS];
     int8_t op[RELAY_MAX_INSTR], a[RELAY_MAX_INSTR], b[RELAY_MAX_INSTR], c[RELAY_MAX_INSTR], dt[RELAY_MAX_INSTR];
-    float imm[RELAY_MAX_INSTR];
+    double imm[RELAY_MAX_INSTR];
 };
 
 constexpr int kDevMaxValues = RELAY_MAX_INPUTS + RELAY_MAX_INSTR;
 
-__device__ __forceinline__ float cast_value(float v, int dt)
+// cast (Fig. 1): float -> int truncates toward zero (saturating at the ends of the integer type), int -> float rounds
+// once to nearest even, int -> int keeps the low bits, anything -> Bool is "!= 0"
+__device__ __forceinline__ Val cast_value(Val x, int from, int to)
 {
-    switch (dt) {
-    case RELAY_BF16: return round_bf16(v);
-    case RELAY_I32: case RELAY_I64: return truncf(v);
-    case RELAY_BOOL: return v != 0.0f ? 1.0f : 0.0f;
-    default: return v;
+    Val r;
+    r.i = 0;
+    if (is_int_type(from)) {
+        switch (to) {
+        case RELAY_I32: r.i = (int32_t)x.i; break;
+        case RELAY_I64: r.i = x.i; break;
+        case RELAY_F32: r.f = __ll2float_rn(x.i); break;
+        case RELAY_BF16: r.f = __bfloat162float(__ll2bfloat16_rn(x.i)); break;
+        default: r.f = x.i != 0 ? 1.0f : 0.0f; break;
+        }
+    } else {
+        switch (to) {
+        case RELAY_I32: r.i = __float2int_rz(x.f); break;
+        case RELAY_I64: r.i = __float2ll_rz(x.f); break;
+        case RELAY_BF16: r.f = round_bf16(x.f); break;
+        case RELAY_BOOL: r.f = x.f != 0.0f ? 1.0f : 0.0f; break;
+        default: r.f = x.f; break;
+        }
     }
+    return r;
 }
 
 // evaluates every value of the program at the output multi-index idx[]
-__device__ __forceinline__ void eval_program(const DevProgram &P, const int64_t *idx, float *vals)
+__device__ __forceinline__ void eval_program(const DevProgram &P, const int64_t *idx, Val *vals)
 {
     for (int i = 0; i < P.n_in; ++i) {
         int64_t off = 0;
         for (int d = 0; d < P.rank; ++d) off += idx[d] * P.in_stride[i][d];
-        vals[i] = load_as_float(P.in_ptr[i], off, P.in_dtype[i]);
+        vals[i] = load_value(P.in_ptr[i], off, P.in_dtype[i]);
     }
     for (int j = 0; j < P.n_instr; ++j) {
-        float x = P.a[j] >= 0 ? vals[P.a[j]] : 0.0f;
-        float y = P.b[j] >= 0 ? vals[P.b[j]] : 0.0f;
-        float z = P.c[j] >= 0 ? vals[P.c[j]] : 0.0f;
-        float r;
-        switch (P.op[j]) {
-        case RELAY_OP_ADD: r = x + y; break;
-        case RELAY_OP_SUB: r = x - y; break;
-        case RELAY_OP_MUL: r = x * y; break;
-        case RELAY_OP_DIV: r = x / y; break;
-        case RELAY_OP_NEG: r = -x; break;
-        case RELAY_OP_SQ: r = x * x; break;
-        case RELAY_OP_NE: r = x != y ? 1.0f : 0.0f; break;
-        case RELAY_OP_EQ: r = x == y ? 1.0f : 0.0f; break;
-        case RELAY_OP_LT: r = x < y ? 1.0f : 0.0f; break;
-        case RELAY_OP_LE: r = x <= y ? 1.0f : 0.0f; break;
-        case RELAY_OP_GT: r = x > y ? 1.0f : 0.0f; break;
-        case RELAY_OP_GE: r = x >= y ? 1.0f : 0.0f; break;
-        case RELAY_OP_SELECT: r = x != 0.0f ? y : z; break;
-        case RELAY_OP_RELU: r = fmaxf(x, 0.0f); break;
-        case RELAY_OP_TANH: r = tanhf(x); break;
-        case RELAY_OP_SIGMOID: r = 1.0f / (1.0f + expf(-x)); break;
-        case RELAY_OP_CAST: r = x; break;
-        case RELAY_OP_CONST: r = P.imm[j]; break;
-        case RELAY_OP_EXP: r = expf(x); break;
-        case RELAY_OP_LOG: r = logf(x); break;
-        case RELAY_OP_MAX: r = fmaxf(x, y); break;
-        default: r = fminf(x, y); break;
+        const int op = P.op[j], dt = P.dt[j];
+        Val out;
+        out.i = 0;
+        if (op == RELAY_OP_CAST) {
+            const int src = P.a[j];
+            out = cast_value(vals[src], src < P.n_in ? P.in_dtype[src] : P.dt[src - P.n_in], dt);
+        } else if (op == RELAY_OP_CONST) {
+            if (is_int_type(dt)) out.i = (long long)P.imm[j];
+            else { out.f = (float)P.imm[j]; out = cast_value(out, RELAY_F32, dt); }
+        } else if (op == RELAY_OP_SELECT) {
+            out = vals[P.a[j]].f != 0.0f ? vals[P.b[j]] : vals[P.c[j]];
+        } else {
+            const float x = P.a[j] >= 0 ? vals[P.a[j]].f : 0.0f;
+            const float y = P.b[j] >= 0 ? vals[P.b[j]].f : 0.0f;
+            float r;
+            switch (op) {
+            case RELAY_OP_ADD: r = x + y; break;
+            case RELAY_OP_SUB: r = x - y; break;
+            case RELAY_OP_MUL: r = x * y; break;
+            case RELAY_OP_DIV: r = x / y; break;
+            case RELAY_OP_NEG: r = -x; break;
+            case RELAY_OP_SQ: r = x * x; break;
+            case RELAY_OP_NE: r = x != y ? 1.0f : 0.0f; break;
+            case RELAY_OP_EQ: r = x == y ? 1.0f : 0.0f; break;
+            case RELAY_OP_LT: r = x < y ? 1.0f : 0.0f; break;
+            case RELAY_OP_LE: r = x <= y ? 1.0f : 0.0f; break;
+            case RELAY_OP_GT: r = x > y ? 1.0f : 0.0f; break;
+            case RELAY_OP_GE: r = x >= y ? 1.0f : 0.0f; break;
+            case RELAY_OP_RELU: r = fmaxf(x, 0.0f); break;
+            case RELAY_OP_TANH: r = tanhf(x); break;
+            case RELAY_OP_SIGMOID: r = 1.0f / (1.0f + expf(-x)); break;
+            case RELAY_OP_EXP: r = expf(x); break;
+            case RELAY_OP_LOG: r = logf(x); break;
+            case RELAY_OP_MAX: r = fmaxf(x, y); break;
+            default: r = fminf(x, y); break;
+            }
+            out.f = dt == RELAY_BF16 ? round_bf16(r) : r;   // a value of type bf16 holds a bf16 number
         }
-        vals[P.n_in + j] = cast_value(r, P.dt[j]);  // a value of type bf16 holds a bf16 number
+        vals[P.n_in + j] = out;
     }
 }
 

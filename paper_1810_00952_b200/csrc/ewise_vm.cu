@@ -3,19 +3,22 @@
 // [rows, cols] whose inputs are full-shape tensors, tensors constant down the rows, or scalars of one float storage
 // type, with unreduced results and column sums.
 //
-// Host: the let-list is turned into a small STACK program.  Values used once are evaluated in place as expression
-// trees; values used several times are computed once, stay on the stack, and are copied to the top where needed.
-// Operands of a stack instruction are implicit (the top of the stack), so the device code can keep the stack in
-// REGISTERS: the interpreter dispatches on (stack height, opcode) and every case indexes the stack with constants.
+// Host: the let-list is turned into code for a small ACCUMULATOR machine.  The accumulator holds 16 elements per
+// thread in registers; every instruction combines it with at most one operand that is fetched from shared memory: an
+// input (the TMA-filled tile ring, or the row of an input that is constant down the rows), a temporary (a
+// thread-private slot that an earlier instruction stored the accumulator to) or a literal.  Expression trees are
+// evaluated deeper operand first, so that the other operand is a leaf wherever possible; values used several times are
+// computed once and kept in a temporary.  With one accumulator there is no register state that depends on where
+// in the program the interpreter is: it branches once per instruction on the opcode, and the branch tree is shallow.
 //
-// Device: a block owns 256 columns x a slice of rows.  One producer thread streams 8-row tiles of every full-shape
-// input into a shared-memory ring with TMA (the bytes in flight live in shared memory, not in registers); 256
-// consumer threads each interpret the program once per tile on 8 elements (a 16-byte vector of bf16, two of f32),
-// taking operands from shared memory; operands that are constant down the rows sit in shared memory as one row.
-// Column sums: per-thread accumulators -> fixed-order combine in shared memory -> one partial per row slice ->
+// Device: a block owns 256 columns x a slice of rows.  16-row tiles of every full-shape input stream into a
+// shared-memory ring by TMA, issued by one lane of warp 0 ahead of use (the bytes in flight live in shared memory,
+// not in registers); the 256 threads each interpret the program once per tile on 2 rows x 8 columns.  Column sums:
+// per-thread accumulators -> fixed-order combine in shared memory -> one partial per row slice ->
 // colsum_finalize_kernel (no float atomics: reruns are bit-identical).
 #include <algorithm>
 #include <cstring>
+#include <new>
 
 #include "ewise_host.h"
 #include "ewise_kernels.cuh"
@@ -29,19 +32,32 @@ relay_status_t make_tmap_2d(CUtensorMap *m, bool f32, const void *base, uint64_t
 
 namespace {
 
-constexpr int VM_TX = 32, VM_TY = 8, VM_E = 8;           // 256 consumer threads, 8 elements each per tile
-constexpr int VM_COLS = VM_TX * VM_E;                    // columns per block
-constexpr int VM_STAGES = 4;
-constexpr int VM_MAXSP = 8, VM_MAXCODE = 96, VM_MAXFULL = 4, VM_MAXFIXED = 4, VM_MAXSUM = 3;
-constexpr int VM_THREADS = VM_TX * VM_TY + 32;           // + the producer warp
+constexpr int VM_TX = 32, VM_TY = 8, VM_V = 8, VM_R = 2;   // 256 threads; a thread owns 8 columns of rows ty and ty + 8 of a tile
+constexpr int VM_E = VM_V * VM_R;                          // elements in the accumulator
+constexpr int VM_COLS = VM_TX * VM_V;                      // columns per block
+constexpr int VM_TILE_ROWS = VM_TY * VM_R;
+constexpr int VM_THREADS = VM_TX * VM_TY;
+constexpr int VM_MAXCODE = 96, VM_MAXFULL = 4, VM_MAXFIXED = 4, VM_MAXSUM = 2, VM_MAXTEMP = 4, VM_MAXCONST = 6;
+constexpr int VM_RING_BYTES = 96 * 1024;                   // budget of the tile ring
 
-// stack opcodes: 0 .. RELAY_OP_COUNT_-1 are the program's own operators (operands on top of the stack)
-enum : int { S_PUSH_IN = 32, S_PUSH_CONST, S_PICK, S_STORE, S_COLSUM, S_ROUND_BF16, S_TO_BOOL, S_POP };
+// opcodes: 0 .. RELAY_OP_COUNT_-1 are the program's own operators, acc = acc (op) operand for the binary ones
+enum : int {
+    A_LOAD = 22,        // acc = operand
+    A_RSUB, A_RDIV,     // acc = operand - acc, operand / acc (the deeper operand of a tree is evaluated first)
+    A_STASH,            // temporary[operand] = acc
+    A_STORE,            // output[operand] = acc
+    A_COLSUM0, A_COLSUM1,
+    A_ROUND_BF16, A_TO_BOOL,
+    A_NOPS
+};
+static_assert(RELAY_OP_COUNT_ == 22, "the machine's own opcodes start after the program's operators");
+
+// operand of an instruction: 0..7 input i; 8.. slot (temporaries first, then literals); SELECT packs two temporaries
+constexpr int OPD_SLOT = 8;
 
 struct VmCode {
     int32_t n;
-    uint8_t op[VM_MAXCODE], arg[VM_MAXCODE], sp[VM_MAXCODE];   // sp: stack height BEFORE the instruction
-    float imm[VM_MAXCODE];
+    uint8_t op[VM_MAXCODE], opd[VM_MAXCODE];
 };
 
 struct VmArgs {
@@ -51,9 +67,10 @@ struct VmArgs {
     void *out[RELAY_MAX_OUTPUTS];
     int8_t out_dt[RELAY_MAX_OUTPUTS];
     float *partial[VM_MAXSUM];
+    float literal[VM_MAXCONST];
     int64_t rows, cols;
-    int32_t rows_per_slice, n_full, n_fixed, n_sum;
-    int32_t box_cols, box_rows;        // TMA box (min(256, cols) x min(8, rows))
+    int32_t rows_per_slice, n_full, n_fixed, n_sum, n_temp, n_const, stages;
+    int32_t box_cols, box_rows;        // TMA box (min(256, cols) x min(16, rows))
     int *err;
     VmCode code;
 };
@@ -66,21 +83,23 @@ template <typename T> __device__ __forceinline__ int vm_col(int tx, int v)
     else return (v < 4 ? 0 : 128) + tx * 4 + (v & 3);
 }
 
-template <typename T> __device__ __forceinline__ void vm_load(const char *row, int tx, float (&f)[VM_E])
+// (register arrays are only ever indexed with constants and never passed as pointers: a pointer into one would move it
+// to local memory)
+template <typename T> __device__ __forceinline__ void vm_load_row(const char *row, int tx, bool hi_live, float (&f)[VM_V])
 {
     if constexpr (sizeof(T) == 2) {
         unpack(*reinterpret_cast<const uint4 *>(row + tx * 16), f);
     } else {
-        float lo[4], hi[4];
+        float lo[4], hi[4] = {0.0f, 0.0f, 0.0f, 0.0f};
         unpack(*reinterpret_cast<const uint4 *>(row + tx * 16), lo);
-        unpack(*reinterpret_cast<const uint4 *>(row + 512 + tx * 16), hi);
+        if (hi_live) unpack(*reinterpret_cast<const uint4 *>(row + 512 + tx * 16), hi);
 #pragma unroll
         for (int v = 0; v < 4; ++v) { f[v] = lo[v]; f[4 + v] = hi[v]; }
     }
 }
 
-// stores `n` consecutive result elements (n = 8 or 4) starting at element index `at` of an output of type `dt`
-template <int N> __device__ __forceinline__ void vm_store_run(void *out, int dt, int64_t at, const float *f)
+// stores N consecutive result elements (N = 8 or 4) starting at element index `at` of an output of type `dt`
+template <int N> __device__ __forceinline__ void vm_store_run(void *out, int dt, int64_t at, const float (&f)[N])
 {
     if (dt == RELAY_F32) {
 #pragma unroll
@@ -107,106 +126,43 @@ template <int N> __device__ __forceinline__ void vm_store_run(void *out, int dt,
 struct VmThread {
     const char *stage;      // ring stage of the current tile
     const char *fixed;      // rows of the operands that are constant down the rows
-    int tx, ty;
-    int tile_bytes, row_bytes;
-    int64_t row, col0;      // this thread's row of the tile and the block's first column
+    char *slots;            // temporaries: [slot][4 pieces of 16 bytes][256 threads]; literals behind them: 16 bytes each
+    int tx, ty, tid;
+    bool hi_live;           // f32: the thread's second run of 4 columns lies inside the tensor
+    bool row_live[VM_R];
+    int tile_bytes, row_bytes, n_temp;
+    int64_t row0, col0;     // first row of the tile and the block's first column
 };
 
-template <typename T, bool FAST>
-__device__ __forceinline__ float vm_unary(int op, float x)
+// fetches the operand of an instruction into o[16]
+template <typename T>
+__device__ __forceinline__ void vm_fetch(int opd, float (&o)[VM_E], const VmArgs &A, const VmThread &th)
 {
-    switch (op) {
-    case RELAY_OP_NEG: return -x;
-    case RELAY_OP_SQ: return x * x;
-    case RELAY_OP_RELU: return fmaxf(x, 0.0f);
-    case RELAY_OP_TANH: return tanh_<FAST>(x);
-    case RELAY_OP_SIGMOID: return sigmoid_<FAST>(x);
-    case RELAY_OP_EXP: return FAST ? __expf(x) : expf(x);
-    case RELAY_OP_LOG: return FAST ? __logf(x) : logf(x);
-    case S_ROUND_BF16: return round_bf16(x);
-    default: return x != 0.0f ? 1.0f : 0.0f;   // S_TO_BOOL
-    }
-}
-template <bool FAST>
-__device__ __forceinline__ float vm_binary(int op, float x, float y)
-{
-    switch (op) {
-    case RELAY_OP_ADD: return x + y;
-    case RELAY_OP_SUB: return x - y;
-    case RELAY_OP_MUL: return x * y;
-    case RELAY_OP_DIV: return FAST ? __fdividef(x, y) : x / y;
-    case RELAY_OP_NE: return x != y ? 1.0f : 0.0f;
-    case RELAY_OP_EQ: return x == y ? 1.0f : 0.0f;
-    case RELAY_OP_LT: return x < y ? 1.0f : 0.0f;
-    case RELAY_OP_LE: return x <= y ? 1.0f : 0.0f;
-    case RELAY_OP_GT: return x > y ? 1.0f : 0.0f;
-    case RELAY_OP_GE: return x >= y ? 1.0f : 0.0f;
-    case RELAY_OP_MAX: return fmaxf(x, y);
-    default: return fminf(x, y);               // RELAY_OP_MIN
-    }
-}
-
-// one stack instruction at stack height SP (every index into `s` is a compile-time constant)
-template <int SP, typename T, bool FAST>
-__device__ __forceinline__ void vm_exec(int op, int arg, float imm, float (&s)[VM_MAXSP][VM_E], float (&acc)[VM_MAXSUM][VM_E],
-                                        const VmArgs &A, const VmThread &th)
-{
-    if (op == S_PUSH_IN) {
-        if constexpr (SP < VM_MAXSP) {
-            const int slot = A.in_slot[arg];
-            const char *row = A.in_kind[arg] == 0 ? th.stage + slot * th.tile_bytes + th.ty * th.row_bytes : th.fixed + slot * th.row_bytes;
-            vm_load<T>(row, th.tx, s[SP]);
-        }
-    } else if (op == S_PUSH_CONST) {
-        if constexpr (SP < VM_MAXSP) {
+    if (opd < OPD_SLOT) {
+        const int slot = A.in_slot[opd];
+        if (A.in_kind[opd] == 0) {
+            const char *row = th.stage + slot * th.tile_bytes + th.ty * th.row_bytes;
+            float r0[VM_V], r1[VM_V];
+            vm_load_row<T>(row, th.tx, th.hi_live, r0);
+            vm_load_row<T>(row + VM_TY * th.row_bytes, th.tx, th.hi_live, r1);
 #pragma unroll
-            for (int v = 0; v < VM_E; ++v) s[SP][v] = imm;
-        }
-    } else if (op == S_PICK) {
-        if constexpr (SP >= 1 && SP < VM_MAXSP) {
+            for (int v = 0; v < VM_V; ++v) { o[v] = r0[v]; o[VM_V + v] = r1[v]; }
+        } else {
+            float r0[VM_V];
+            vm_load_row<T>(th.fixed + slot * (VM_COLS * (int)sizeof(T)), th.tx, th.hi_live, r0);
 #pragma unroll
-            for (int q = 0; q < SP; ++q)
-                if (arg == q) {
-#pragma unroll
-                    for (int v = 0; v < VM_E; ++v) s[SP][v] = s[SP - 1 - q][v];
-                }
-        }
-    } else if (op == S_STORE) {
-        if constexpr (SP >= 1) {
-            void *out = A.out[arg];
-            const int dt = A.out_dt[arg];
-            if constexpr (sizeof(T) == 2) {
-                if (th.col0 + th.tx * 8 < A.cols) vm_store_run<8>(out, dt, th.row * A.cols + th.col0 + th.tx * 8, s[SP - 1]);
-            } else {
-                if (th.col0 + th.tx * 4 < A.cols) vm_store_run<4>(out, dt, th.row * A.cols + th.col0 + th.tx * 4, s[SP - 1]);
-                if (th.col0 + 128 + th.tx * 4 < A.cols) vm_store_run<4>(out, dt, th.row * A.cols + th.col0 + 128 + th.tx * 4, s[SP - 1] + 4);
-            }
-        }
-    } else if (op == S_COLSUM) {
-        if constexpr (SP >= 1) {
-#pragma unroll
-            for (int k = 0; k < VM_MAXSUM; ++k)
-                if (arg == k) {
-#pragma unroll
-                    for (int v = 0; v < VM_E; ++v) acc[k][v] += s[SP - 1][v];
-                }
-        }
-    } else if (op == S_POP) {
-    } else if (op == RELAY_OP_SELECT) {
-        if constexpr (SP >= 3) {
-#pragma unroll
-            for (int v = 0; v < VM_E; ++v) s[SP - 3][v] = s[SP - 3][v] != 0.0f ? s[SP - 2][v] : s[SP - 1][v];
-        }
-    } else if (op == RELAY_OP_NEG || op == RELAY_OP_SQ || op == RELAY_OP_RELU || op == RELAY_OP_TANH || op == RELAY_OP_SIGMOID ||
-               op == RELAY_OP_EXP || op == RELAY_OP_LOG || op == S_ROUND_BF16 || op == S_TO_BOOL) {
-        if constexpr (SP >= 1) {
-#pragma unroll
-            for (int v = 0; v < VM_E; ++v) s[SP - 1][v] = vm_unary<T, FAST>(op, s[SP - 1][v]);
+            for (int v = 0; v < VM_V; ++v) { o[v] = r0[v]; o[VM_V + v] = r0[v]; }
         }
     } else {
-        if constexpr (SP >= 2) {
+        // a temporary (one 64-byte value per thread, in four pieces) or a literal (one 16-byte piece for everybody)
+        const int k = opd - OPD_SLOT;
+        const bool temp = k < th.n_temp;
+        const char *p = temp ? th.slots + (k * 4 * VM_THREADS + th.tid) * 16 : th.slots + (th.n_temp * 4 * VM_THREADS + (k - th.n_temp)) * 16;
+        const int step = temp ? VM_THREADS * 16 : 0;
 #pragma unroll
-            for (int v = 0; v < VM_E; ++v) s[SP - 2][v] = vm_binary<FAST>(op, s[SP - 2][v], s[SP - 1][v]);
+        for (int q = 0; q < 4; ++q) {
+            const uint4 w = *reinterpret_cast<const uint4 *>(p + q * step);
+            o[4 * q] = __uint_as_float(w.x); o[4 * q + 1] = __uint_as_float(w.y); o[4 * q + 2] = __uint_as_float(w.z); o[4 * q + 3] = __uint_as_float(w.w);
         }
     }
 }
@@ -219,47 +175,49 @@ ewise_vm_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constant__
     extern __shared__ uint8_t vm_smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(vm_smem_raw) + 1023) & ~uintptr_t(1023));
     const int row_bytes = A.box_cols * (int)sizeof(T), tile_bytes = ((A.box_rows * row_bytes + 127) / 128) * 128;
-    const int stage_bytes = A.n_full * tile_bytes;
-    uint8_t *fixed = smem + VM_STAGES * stage_bytes;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(fixed + ((A.n_fixed * VM_COLS * (int)sizeof(T) + 127) / 128) * 128);
-    uint64_t *full = bars, *empty = bars + VM_STAGES;
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 2 * VM_STAGES);
+    const int stage_bytes = A.n_full * tile_bytes, STAGES = A.stages;
+    const int ring_bytes = max(STAGES * stage_bytes, VM_TY * (VM_COLS + 1) * (int)sizeof(float));   // the ring's start doubles as the combine buffer
+    uint8_t *fixed = smem + ((ring_bytes + 127) / 128) * 128;
+    uint8_t *slots = fixed + ((A.n_fixed * VM_COLS * (int)sizeof(T) + 127) / 128) * 128;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(slots + ((A.n_temp * 4 * VM_THREADS + A.n_const) * 16 + 127) / 128 * 128);
+    uint64_t *full = bars, *empty = bars + 4;
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 8);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int64_t col0 = (int64_t)blockIdx.x * VM_COLS;
     const int64_t r0 = (int64_t)blockIdx.y * A.rows_per_slice, r1 = min(A.rows, r0 + (int64_t)A.rows_per_slice);
     const int n_tiles = r1 > r0 ? (int)((r1 - r0 + A.box_rows - 1) / A.box_rows) : 0;
 
     if (tid == 0) {
-        for (int s = 0; s < VM_STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], VM_TY); }
+        for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], VM_TY); }
         *abort_flag = 0;
         tc::fence_barrier_init();
         tc::prefetch_tmap(&tm0);
     }
     pdl_wait();
-    // operands that are constant down the rows: one row of this block's columns each (a scalar fills the row)
-    if (tid < VM_COLS) {
-        for (int g = 0; g < A.n_fixed; ++g) {
-            const T *p = (const T *)A.fixed_ptr[g];
-            T val = T(0.0f);
-            if (A.fixed_scalar[g]) val = p[0];
-            else if (col0 + tid < A.cols) val = p[col0 + tid];
-            reinterpret_cast<T *>(fixed)[g * VM_COLS + tid] = val;
-        }
+    // operands that are constant down the rows: one row of this block's columns each (a scalar fills the row); literals
+    for (int g = 0; g < A.n_fixed; ++g) {
+        const T *p = (const T *)A.fixed_ptr[g];
+        T val = T(0.0f);
+        if (A.fixed_scalar[g]) val = p[0];
+        else if (col0 + tid < A.cols) val = p[col0 + tid];
+        reinterpret_cast<T *>(fixed)[g * VM_COLS + tid] = val;
     }
+    if (tid < A.n_const * 4) reinterpret_cast<float *>(slots + A.n_temp * 4 * VM_THREADS * 16)[tid] = A.literal[tid >> 2];
     __syncthreads();
 
-    float acc[VM_MAXSUM][VM_E];
+    float sum[VM_MAXSUM][VM_V];
 #pragma unroll
     for (int k = 0; k < VM_MAXSUM; ++k)
 #pragma unroll
-        for (int v = 0; v < VM_E; ++v) acc[k][v] = 0.0f;
+        for (int v = 0; v < VM_V; ++v) sum[k][v] = 0.0f;
 
-    if (warp == VM_TY) {
-        // producer: every lane runs the loop, one elected lane issues
+    {
+        // Warp 0 is also the producer: before it interprets tile t it refills the ring with tile t + STAGES - 1, whose
+        // stage the other warps released when they finished tile t - 1 (they run at most a tile or two behind).
         const CUtensorMap *tms[VM_MAXFULL] = {&tm0, &tm1, &tm2, &tm3};
-        for (int t = 0; t < n_tiles; ++t) {
-            const int s = t % VM_STAGES;
-            if (!__all_sync(0xffffffffu, tc::mbar_wait(&empty[s], ((t / VM_STAGES) & 1) ^ 1, abort_flag, A.err, tc::ERR_WAIT_EMPTY))) break;
+        auto issue = [&](int t) -> bool {        // whole warp 0; false when a wait gave up
+            const int s = t % STAGES;
+            if (!__all_sync(0xffffffffu, tc::mbar_wait(&empty[s], ((t / STAGES) & 1) ^ 1, abort_flag, A.err, tc::ERR_WAIT_EMPTY))) return false;
             if (tc::elect_one()) {
                 tc::mbar_expect_tx(&full[s], (uint32_t)(A.n_full * A.box_rows * row_bytes));
 #pragma unroll
@@ -267,38 +225,132 @@ ewise_vm_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constant__
                     if (f < A.n_full) tc::tma_load_2d(smem + s * stage_bytes + f * tile_bytes, tms[f], &full[s], (int)col0, (int)(r0 + (int64_t)t * A.box_rows));
             }
             __syncwarp();
-        }
-    } else {
+            return true;
+        };
+        bool ok_issue = true;
+        if (warp == 0)
+            for (int t = 0; t < STAGES - 1 && t < n_tiles && ok_issue; ++t) ok_issue = issue(t);
         VmThread th;
         th.fixed = reinterpret_cast<const char *>(fixed);
-        th.tx = lane; th.ty = warp;
-        th.tile_bytes = tile_bytes; th.row_bytes = row_bytes;
+        th.slots = reinterpret_cast<char *>(slots);
+        th.tx = lane; th.ty = warp; th.tid = tid;
+        th.tile_bytes = tile_bytes; th.row_bytes = row_bytes; th.n_temp = A.n_temp;
         th.col0 = col0;
+        th.hi_live = sizeof(T) == 4 && col0 + 128 + lane * 4 < A.cols;
         const bool col_live = col0 + vm_col<T>(lane, 0) < A.cols;     // a thread's first column decides (its second run is checked at the store)
-        float s[VM_MAXSP][VM_E];
+        float acc[VM_E];
+#pragma unroll
+        for (int e = 0; e < VM_E; ++e) acc[e] = 0.0f;
         for (int t = 0; t < n_tiles; ++t) {
-            const int st = t % VM_STAGES;
+            if (warp == 0 && t + STAGES - 1 < n_tiles && ok_issue) ok_issue = issue(t + STAGES - 1);
+            const int st = t % STAGES;
             int ok = 1;
-            if (lane == 0) ok = tc::mbar_wait(&full[st], (t / VM_STAGES) & 1, abort_flag, A.err, tc::ERR_WAIT_FULL) ? 1 : 0;
+            if (lane == 0) ok = tc::mbar_wait(&full[st], (t / STAGES) & 1, abort_flag, A.err, tc::ERR_WAIT_FULL) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
             th.stage = reinterpret_cast<const char *>(smem + st * stage_bytes);
-            th.row = r0 + (int64_t)t * A.box_rows + warp;
-            if (warp < A.box_rows && th.row < r1 && col_live) {
+            th.row0 = r0 + (int64_t)t * A.box_rows;
+#pragma unroll
+            for (int r = 0; r < VM_R; ++r) th.row_live[r] = warp + VM_TY * r < A.box_rows && th.row0 + warp + VM_TY * r < r1;
+            if (th.row_live[0] && col_live) {
 #pragma unroll 1
                 for (int pc = 0; pc < A.code.n; ++pc) {
-                    const int op = A.code.op[pc], arg = A.code.arg[pc];
-                    const float imm = A.code.imm[pc];
-                    switch (A.code.sp[pc]) {
-                    case 0: vm_exec<0, T, FAST>(op, arg, imm, s, acc, A, th); break;
-                    case 1: vm_exec<1, T, FAST>(op, arg, imm, s, acc, A, th); break;
-                    case 2: vm_exec<2, T, FAST>(op, arg, imm, s, acc, A, th); break;
-                    case 3: vm_exec<3, T, FAST>(op, arg, imm, s, acc, A, th); break;
-                    case 4: vm_exec<4, T, FAST>(op, arg, imm, s, acc, A, th); break;
-                    case 5: vm_exec<5, T, FAST>(op, arg, imm, s, acc, A, th); break;
-                    case 6: vm_exec<6, T, FAST>(op, arg, imm, s, acc, A, th); break;
-                    case 7: vm_exec<7, T, FAST>(op, arg, imm, s, acc, A, th); break;
-                    default: vm_exec<8, T, FAST>(op, arg, imm, s, acc, A, th); break;
+                    const int op = A.code.op[pc], opd = A.code.opd[pc];
+                    if (op <= A_RDIV && op != RELAY_OP_NEG && op != RELAY_OP_SQ && op != RELAY_OP_RELU && op != RELAY_OP_TANH && op != RELAY_OP_SIGMOID &&
+                        op != RELAY_OP_EXP && op != RELAY_OP_LOG && op != RELAY_OP_SELECT) {
+                        float o[VM_E];
+                        vm_fetch<T>(opd, o, A, th);
+#define VM_BIN(OP, EXPR)                                                         \
+    case OP:                                                                     \
+        _Pragma("unroll") for (int e = 0; e < VM_E; ++e) { const float x = acc[e], y = o[e]; acc[e] = (EXPR); } \
+        break;
+                        switch (op) {
+                            VM_BIN(RELAY_OP_ADD, x + y)
+                            VM_BIN(RELAY_OP_SUB, x - y)
+                            VM_BIN(RELAY_OP_MUL, x * y)
+                            VM_BIN(RELAY_OP_DIV, FAST ? __fdividef(x, y) : x / y)
+                            VM_BIN(RELAY_OP_NE, x != y ? 1.0f : 0.0f)
+                            VM_BIN(RELAY_OP_EQ, x == y ? 1.0f : 0.0f)
+                            VM_BIN(RELAY_OP_LT, x < y ? 1.0f : 0.0f)
+                            VM_BIN(RELAY_OP_LE, x <= y ? 1.0f : 0.0f)
+                            VM_BIN(RELAY_OP_GT, x > y ? 1.0f : 0.0f)
+                            VM_BIN(RELAY_OP_GE, x >= y ? 1.0f : 0.0f)
+                            VM_BIN(RELAY_OP_MAX, fmaxf(x, y))
+                            VM_BIN(RELAY_OP_MIN, fminf(x, y))
+                            VM_BIN(A_RSUB, y - x)
+                            VM_BIN(A_RDIV, FAST ? __fdividef(y, x) : y / x)
+                        default:      // A_LOAD
+#pragma unroll
+                            for (int e = 0; e < VM_E; ++e) acc[e] = o[e];
+                            break;
+                        }
+#undef VM_BIN
+                    } else {
+#define VM_UN(OP, EXPR)                                                          \
+    case OP:                                                                     \
+        _Pragma("unroll") for (int e = 0; e < VM_E; ++e) { const float x = acc[e]; acc[e] = (EXPR); } \
+        break;
+                        switch (op) {
+                            VM_UN(RELAY_OP_NEG, -x)
+                            VM_UN(RELAY_OP_SQ, x * x)
+                            VM_UN(RELAY_OP_RELU, fmaxf(x, 0.0f))
+                            // bf16 storage: exp2 / reciprocal approximations (absolute error about 1e-7).  The one-instruction
+                            // tanh.approx of the pre-compiled bodies (relative error 2^-11) is not used here: a program may
+                            // multiply the result by anything.
+                            VM_UN(RELAY_OP_TANH, FAST ? 1.0f - __fdividef(2.0f, 1.0f + __expf(2.0f * x)) : tanhf(x))
+                            VM_UN(RELAY_OP_SIGMOID, FAST ? __fdividef(1.0f, 1.0f + __expf(-x)) : 1.0f / (1.0f + expf(-x)))
+                            VM_UN(RELAY_OP_EXP, FAST ? __expf(x) : expf(x))
+                            VM_UN(RELAY_OP_LOG, FAST ? __logf(x) : logf(x))
+                            VM_UN(A_ROUND_BF16, round_bf16(x))
+                            VM_UN(A_TO_BOOL, x != 0.0f ? 1.0f : 0.0f)
+                        case RELAY_OP_SELECT: {      // acc = acc ? temporary (opd & 15) : temporary (opd >> 4)
+                            float a[VM_E], b[VM_E];
+                            vm_fetch<T>(OPD_SLOT + (opd & 15), a, A, th);
+                            vm_fetch<T>(OPD_SLOT + (opd >> 4), b, A, th);
+#pragma unroll
+                            for (int e = 0; e < VM_E; ++e) acc[e] = acc[e] != 0.0f ? a[e] : b[e];
+                            break;
+                        }
+                        case A_STASH: {
+                            char *p = th.slots + ((opd - OPD_SLOT) * 4 * VM_THREADS + tid) * 16;
+#pragma unroll
+                            for (int q = 0; q < 4; ++q)
+                                *reinterpret_cast<uint4 *>(p + q * VM_THREADS * 16) = make_uint4(__float_as_uint(acc[4 * q]), __float_as_uint(acc[4 * q + 1]),
+                                                                                                 __float_as_uint(acc[4 * q + 2]), __float_as_uint(acc[4 * q + 3]));
+                            break;
+                        }
+                        case A_STORE: {
+                            void *out = A.out[opd];
+                            const int dt = A.out_dt[opd];
+#pragma unroll
+                            for (int r = 0; r < VM_R; ++r) {
+                                if (!th.row_live[r]) continue;
+                                const int64_t at = (th.row0 + warp + VM_TY * r) * A.cols + col0;
+                                if constexpr (sizeof(T) == 2) {
+                                    float w[8];
+#pragma unroll
+                                    for (int v = 0; v < 8; ++v) w[v] = acc[VM_V * r + v];
+                                    vm_store_run<8>(out, dt, at + lane * 8, w);
+                                } else {
+                                    float lo[4], hi[4];
+#pragma unroll
+                                    for (int v = 0; v < 4; ++v) { lo[v] = acc[VM_V * r + v]; hi[v] = acc[VM_V * r + 4 + v]; }
+                                    vm_store_run<4>(out, dt, at + lane * 4, lo);
+                                    if (th.hi_live) vm_store_run<4>(out, dt, at + 128 + lane * 4, hi);
+                                }
+                            }
+                            break;
+                        }
+                        case A_COLSUM0:
+#pragma unroll
+                            for (int v = 0; v < VM_V; ++v) sum[0][v] += acc[v] + (th.row_live[1] ? acc[VM_V + v] : 0.0f);
+                            break;
+                        default:      // A_COLSUM1
+#pragma unroll
+                            for (int v = 0; v < VM_V; ++v) sum[1][v] += acc[v] + (th.row_live[1] ? acc[VM_V + v] : 0.0f);
+                            break;
+                        }
+#undef VM_UN
                     }
                 }
             }
@@ -312,12 +364,10 @@ ewise_vm_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constant__
         __syncthreads();                                    // the ring is no longer read: its first bytes hold the combine buffer
         float(*sm)[VM_COLS + 1] = reinterpret_cast<float(*)[VM_COLS + 1]>(smem);
         for (int k = 0; k < A.n_sum; ++k) {
-            if (warp < VM_TY) {
 #pragma unroll
-                for (int v = 0; v < VM_E; ++v) sm[warp][vm_col<T>(lane, v)] = acc[k][v];
-            }
+            for (int v = 0; v < VM_V; ++v) sm[warp][vm_col<T>(lane, v)] = sum[k][v];
             __syncthreads();
-            if (tid < VM_COLS && col0 + tid < A.cols) {
+            if (col0 + tid < A.cols) {
                 float t = 0.0f;
 #pragma unroll
                 for (int j = 0; j < VM_TY; ++j) t += sm[j][tid];
@@ -328,69 +378,138 @@ ewise_vm_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constant__
     }
 }
 
-}  // namespace
-
 // =================================================================================================
-// host: let-list -> stack program
+// host: let-list -> accumulator code
 // =================================================================================================
-namespace {
-
 struct Compiler {
     const TypedProgram &tp;
     VmCode &code;
     int alias[kMaxValues];       // value this one is a plain copy of (casts that change nothing), or itself
     int uses[kMaxValues];
-    int pos[kMaxValues];         // stack position of a value kept on the stack, -1 otherwise
-    int sp = 0, max_sp = 0;
+    int home[kMaxValues];        // temporary that holds the value, -1 if none
+    bool temp_used[VM_MAXTEMP] = {false};
+    int n_temp = 0;              // highest temporary in use + 1
+    float literal[VM_MAXCONST];
+    int n_const = 0;
+    int acc_holds = -1;          // value currently in the accumulator, if known
+    int last_op = -1;
     bool ok = true;
 
     Compiler(const TypedProgram &t, VmCode &c) : tp(t), code(c) { code.n = 0; }
 
-    void emit(int op, int arg, float imm, int delta)
+    void emit(int op, int opd)
     {
         if (code.n >= VM_MAXCODE) { ok = false; return; }
-        code.op[code.n] = (uint8_t)op; code.arg[code.n] = (uint8_t)arg; code.sp[code.n] = (uint8_t)sp; code.imm[code.n] = imm;
+        code.op[code.n] = (uint8_t)op; code.opd[code.n] = (uint8_t)opd;
         ++code.n;
-        sp += delta;
-        max_sp = std::max(max_sp, sp);
-        if (sp > VM_MAXSP || sp < 0) ok = false;
+        last_op = op;
+        if (op != A_STASH && op != A_STORE && op != A_COLSUM0 && op != A_COLSUM1) acc_holds = -1;
     }
-    static bool floatlike(int32_t dt) { return dt == RELAY_F32 || dt == RELAY_BF16 || dt == RELAY_BOOL; }
+    int alloc_temp()
+    {
+        for (int k = 0; k < VM_MAXTEMP; ++k)
+            if (!temp_used[k]) { temp_used[k] = true; n_temp = std::max(n_temp, k + 1); return k; }
+        ok = false;
+        return 0;
+    }
+    float literal_of(const relay_instr_t &in) const
+    {
+        float c = (float)in.imm;
+        if (in.dtype == RELAY_BF16) c = __bfloat162float(__float2bfloat16_rn(c));
+        else if (in.dtype == RELAY_BOOL) c = in.imm != 0.0 ? 1.0f : 0.0f;
+        return c;
+    }
+    int const_slot(float c)
+    {
+        for (int i = 0; i < n_const; ++i)
+            if (memcmp(&literal[i], &c, sizeof c) == 0) return i;
+        if (n_const == VM_MAXCONST) { ok = false; return 0; }
+        literal[n_const] = c;
+        return n_const++;
+    }
+    bool is_const(int v) const { return v >= tp.n_in && tp.instr[v - tp.n_in].op == RELAY_OP_CONST; }
+    // operands that an instruction can take straight from shared memory
+    bool is_leaf(int v) const { v = alias[v]; return v < tp.n_in || home[v] >= 0 || is_const(v); }
+    // operand code of a leaf; literals are numbered behind the temporaries once their count is known, so they are
+    // recorded as 128 + index here and renumbered by finish()
+    int operand(int v)
+    {
+        v = alias[v];
+        if (v < tp.n_in) return v;
+        if (home[v] >= 0) return OPD_SLOT + home[v];
+        return 128 + const_slot(literal_of(tp.instr[v - tp.n_in]));
+    }
+    static int mirrored(int op)      // x op y == y mirrored(op) x
+    {
+        switch (op) {
+        case RELAY_OP_SUB: return A_RSUB;
+        case RELAY_OP_DIV: return A_RDIV;
+        case RELAY_OP_LT: return RELAY_OP_GT;
+        case RELAY_OP_LE: return RELAY_OP_GE;
+        case RELAY_OP_GT: return RELAY_OP_LT;
+        case RELAY_OP_GE: return RELAY_OP_LE;
+        default: return op;          // commutative
+        }
+    }
+    // a temporary that holds v, for SELECT (an input, a literal or an expression is copied into one first)
+    int as_temp(int v, int depth, bool *owned)
+    {
+        v = alias[v];
+        *owned = false;
+        if (v >= tp.n_in && home[v] >= 0) return home[v];
+        gen(v, depth + 1);
+        const int t = alloc_temp();
+        emit(A_STASH, OPD_SLOT + t);
+        *owned = true;
+        return t;
+    }
 
-    // pushes value v
-    void push(int v, int depth = 0)
+    // evaluates value v into the accumulator
+    void gen(int v, int depth = 0)
     {
         if (!ok || depth > 40) { ok = false; return; }
         v = alias[v];
-        if (v < tp.n_in) { emit(S_PUSH_IN, v, 0.0f, +1); return; }
-        if (pos[v] >= 0) { emit(S_PICK, sp - 1 - pos[v], 0.0f, +1); return; }
-        compute(v, depth);
-    }
-    // evaluates instruction value v onto the top of the stack
-    void compute(int v, int depth)
-    {
+        if (acc_holds == v) return;
+        if (is_leaf(v)) { emit(A_LOAD, operand(v)); acc_holds = v; return; }
         const relay_instr_t &in = tp.instr[v - tp.n_in];
-        if (in.op == RELAY_OP_CONST) {
-            float c = (float)in.imm;
-            if (in.dtype == RELAY_BF16) c = __bfloat162float(__float2bfloat16_rn(c));
-            else if (in.dtype == RELAY_BOOL) c = in.imm != 0.0 ? 1.0f : 0.0f;
-            emit(S_PUSH_CONST, 0, c, +1);
-            return;
-        }
         if (in.op == RELAY_OP_CAST) {       // a cast that is not a plain copy
-            push(in.a, depth + 1);
-            emit(in.dtype == RELAY_BF16 ? S_ROUND_BF16 : S_TO_BOOL, 0, 0.0f, 0);
-            return;
+            gen(in.a, depth + 1);
+            emit(in.dtype == RELAY_BF16 ? A_ROUND_BF16 : A_TO_BOOL, 0);
+        } else if (in.op == RELAY_OP_SELECT) {
+            bool own_b, own_c;
+            const int tb = as_temp(in.b, depth, &own_b), tc_ = as_temp(in.c, depth, &own_c);
+            gen(in.a, depth + 1);
+            emit(RELAY_OP_SELECT, tb | (tc_ << 4));
+            if (own_b) temp_used[tb] = false;
+            if (own_c) temp_used[tc_] = false;
+        } else if (in.b < 0) {              // unary
+            gen(in.a, depth + 1);
+            emit(in.op, 0);
+        } else if (is_leaf(in.b)) {
+            gen(in.a, depth + 1);
+            emit(in.op, operand(in.b));
+        } else if (is_leaf(in.a)) {
+            gen(in.b, depth + 1);
+            emit(mirrored(in.op), operand(in.a));
+        } else {
+            gen(in.a, depth + 1);
+            const int t = alloc_temp();
+            emit(A_STASH, OPD_SLOT + t);
+            gen(in.b, depth + 1);
+            emit(mirrored(in.op), OPD_SLOT + t);
+            temp_used[t] = false;
         }
-        if (in.a >= 0) push(in.a, depth + 1);
-        if (in.b >= 0) push(in.b, depth + 1);
-        if (in.c >= 0) push(in.c, depth + 1);
-        const int ar = (in.a >= 0) + (in.b >= 0) + (in.c >= 0);
-        emit(in.op, 0, 0.0f, 1 - ar);
-        // a value of type bf16 holds a bf16 number (comparisons and select of already rounded values need no rounding)
-        if (in.dtype == RELAY_BF16 && in.op != RELAY_OP_SELECT && in.op != RELAY_OP_MAX && in.op != RELAY_OP_MIN && in.op != RELAY_OP_NEG &&
-            in.op != RELAY_OP_RELU)
-            emit(S_ROUND_BF16, 0, 0.0f, 0);
+        // a value of type bf16 holds a bf16 number (operators that only pick one of their operands need no rounding)
+        if (in.dtype == RELAY_BF16 && in.op != RELAY_OP_CAST && in.op != RELAY_OP_SELECT && in.op != RELAY_OP_MAX && in.op != RELAY_OP_MIN &&
+            in.op != RELAY_OP_NEG && in.op != RELAY_OP_RELU)
+            emit(A_ROUND_BF16, 0);
+        acc_holds = v;
+    }
+    // literals live behind the temporaries
+    void finish()
+    {
+        for (int i = 0; i < code.n; ++i)
+            if (code.opd[i] >= 128 && code.op[i] != RELAY_OP_SELECT) code.opd[i] = (uint8_t)(OPD_SLOT + n_temp + (code.opd[i] - 128));
     }
 };
 
@@ -399,7 +518,8 @@ struct Compiler {
 struct VmPlanImpl {
     VmCode code;
     int in_kind[RELAY_MAX_INPUTS], in_slot[RELAY_MAX_INPUTS];
-    int n_full = 0, n_fixed = 0, n_sum = 0;
+    int n_full = 0, n_fixed = 0, n_sum = 0, n_temp = 0, n_const = 0;
+    float literal[VM_MAXCONST];
     int sum_of_out[RELAY_MAX_OUTPUTS];     // index of the accumulator of output k, or -1
 };
 
@@ -417,6 +537,9 @@ bool vm_plan(const TypedProgram &tp, const View2D &v, const int32_t *out_values,
         else { if (P.n_fixed == VM_MAXFIXED) return false; P.in_kind[i] = 1; P.in_slot[i] = P.n_fixed++; }
     }
     if (P.n_full < 1) return false;
+    // at least two ring stages of 16-row tiles must fit
+    const int64_t tile = std::min<int64_t>(VM_COLS, v.cols) * (v.storage == RELAY_F32 ? 4 : 2) * std::min<int64_t>(VM_TILE_ROWS, v.rows);
+    if (2 * P.n_full * ((tile + 127) / 128 * 128) > VM_RING_BYTES) return false;
     Compiler C(tp, P.code);
     // which values are needed, and which are plain copies of another value
     bool needed[kMaxValues] = {false};
@@ -429,8 +552,8 @@ bool vm_plan(const TypedProgram &tp, const View2D &v, const int32_t *out_values,
         if (in.c >= 0) needed[in.c] = true;
     }
     for (int x = 0; x < tp.n_values; ++x) {
-        C.alias[x] = x; C.uses[x] = 0; C.pos[x] = -1;
-        if (needed[x] && !Compiler::floatlike(tp.dtype[x])) return false;           // integer lanes: scalar evaluator
+        C.alias[x] = x; C.uses[x] = 0; C.home[x] = -1;
+        if (needed[x] && !(tp.dtype[x] == RELAY_F32 || tp.dtype[x] == RELAY_BF16 || tp.dtype[x] == RELAY_BOOL)) return false;   // integer lanes: scalar evaluator
         if (x >= tp.n_in && needed[x]) {
             const relay_instr_t &in = tp.instr[x - tp.n_in];
             if (in.op == RELAY_OP_CAST) {
@@ -449,24 +572,32 @@ bool vm_plan(const TypedProgram &tp, const View2D &v, const int32_t *out_values,
         if (in.c >= 0) ++C.uses[C.alias[in.c]];
     }
     for (int k = 0; k < n_out; ++k) ++C.uses[C.alias[out_values[k]]];
-    // values used more than once are computed in let order and stay on the stack
+    // values used more than once are computed in let order and kept in a temporary
     for (int x = tp.n_in; x < tp.n_values && C.ok; ++x) {
-        if (!needed[x] || C.alias[x] != x || C.uses[x] < 2 || tp.instr[x - tp.n_in].op == RELAY_OP_CONST) continue;
-        C.compute(x, 0);
-        C.pos[x] = C.sp - 1;
+        if (!needed[x] || C.alias[x] != x || C.uses[x] < 2 || C.is_const(x)) continue;
+        C.gen(x);
+        const int t = C.alloc_temp();
+        C.emit(A_STASH, OPD_SLOT + t);
+        C.home[x] = t;
+        C.acc_holds = x;
     }
     for (int k = 0; k < n_out && C.ok; ++k) {
-        C.push(out_values[k]);
+        C.gen(out_values[k]);
         P.sum_of_out[k] = -1;
         if (colsum[k]) {
             if (P.n_sum == VM_MAXSUM) return false;
             P.sum_of_out[k] = P.n_sum;
-            C.emit(S_COLSUM, P.n_sum++, 0.0f, -1);
+            C.emit(A_COLSUM0 + P.n_sum++, 0);
         } else {
-            C.emit(S_STORE, k, 0.0f, -1);
+            // the store of a bf16 result rounds by itself: a rounding that was emitted just for it is dropped
+            if (C.last_op == A_ROUND_BF16 && tp.dtype[out_values[k]] == RELAY_BF16 && C.ok) { --P.code.n; C.acc_holds = -1; }
+            C.emit(A_STORE, k);
         }
     }
     if (!C.ok) return false;
+    C.finish();
+    P.n_temp = C.n_temp; P.n_const = C.n_const;
+    memcpy(P.literal, C.literal, sizeof P.literal);
     plan->ok = true;
     plan->n_sum = P.n_sum;
     return true;
@@ -480,9 +611,10 @@ relay_status_t vm_launch(const VmPlan &plan, const View2D &v, const relay_tensor
     const int esize = f32 ? 4 : 2;
     VmArgs A{};
     A.rows = v.rows; A.cols = v.cols;
-    A.n_full = P.n_full; A.n_fixed = P.n_fixed; A.n_sum = P.n_sum;
+    A.n_full = P.n_full; A.n_fixed = P.n_fixed; A.n_sum = P.n_sum; A.n_temp = P.n_temp; A.n_const = P.n_const;
+    memcpy(A.literal, P.literal, sizeof A.literal);
     A.box_cols = (int)std::min<int64_t>(VM_COLS, v.cols);
-    A.box_rows = (int)std::min<int64_t>(VM_TY, v.rows);
+    A.box_rows = (int)std::min<int64_t>(VM_TILE_ROWS, v.rows);
     A.rows_per_slice = (int)((v.rows + n_slices - 1) / n_slices);
     A.rows_per_slice = (A.rows_per_slice + A.box_rows - 1) / A.box_rows * A.box_rows;      // slices start on tile boundaries
     A.code = P.code;
@@ -506,8 +638,11 @@ relay_status_t vm_launch(const VmPlan &plan, const View2D &v, const relay_tensor
         if (P.sum_of_out[k] >= 0) A.partial[P.sum_of_out[k]] = partials + (size_t)P.sum_of_out[k] * n_slices * v.cols;
     }
     const int row_bytes = A.box_cols * esize, tile_bytes = ((A.box_rows * row_bytes + 127) / 128) * 128;
-    const size_t ring = (size_t)VM_STAGES * P.n_full * tile_bytes;
-    const size_t smem = 1024 + std::max(ring, (size_t)VM_TY * (VM_COLS + 1) * sizeof(float)) + ((size_t)P.n_fixed * VM_COLS * esize + 127) / 128 * 128 + 256;
+    const int stage_bytes = P.n_full * tile_bytes;
+    A.stages = std::max(2, std::min(4, VM_RING_BYTES / 2 / stage_bytes));     // as many as half the budget holds (two blocks per SM), at least two
+    const size_t ring = std::max((size_t)A.stages * stage_bytes, (size_t)VM_TY * (VM_COLS + 1) * sizeof(float));
+    const size_t smem = 1024 + (ring + 127) / 128 * 128 + ((size_t)P.n_fixed * VM_COLS * esize + 127) / 128 * 128 +
+                        ((size_t)(P.n_temp * 4 * VM_THREADS + P.n_const) * 16 + 127) / 128 * 128 + 256;
     const dim3 grid((unsigned)((v.cols + VM_COLS - 1) / VM_COLS), (unsigned)((v.rows + A.rows_per_slice - 1) / A.rows_per_slice));
     if (f32) {
         RELAY_CUDA(cudaFuncSetAttribute(ewise_vm_kernel<float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -522,7 +657,7 @@ relay_status_t vm_launch(const VmPlan &plan, const View2D &v, const relay_tensor
 int vm_grid_slices(const View2D &v, int n_slices_wanted)
 {
     // the slices the launch really makes (whole tiles per slice)
-    const int box_rows = (int)std::min<int64_t>(VM_TY, v.rows);
+    const int box_rows = (int)std::min<int64_t>(VM_TILE_ROWS, v.rows);
     int rps = (int)((v.rows + n_slices_wanted - 1) / n_slices_wanted);
     rps = (rps + box_rows - 1) / box_rows * box_rows;
     return (int)((v.rows + rps - 1) / rps);

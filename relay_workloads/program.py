@@ -127,3 +127,29 @@ def tanh_affine_residual_grad(storage=BF16, math=F32):
     ds = p.mul(d, s)
     dae = p.mul(ds, x)
     return p, [dx, dae, ds]
+
+
+def sigmoid_product_relu_fwd(storage=BF16, math=F32):
+    """out = sigmoid(x * y) + relu(z); inputs (x, y, z) in `storage` (z may be constant down the rows), arithmetic in
+    `math`, out in `storage`."""
+    p = Program([storage, storage, storage])
+    x, y, z = (p.cast(i, math) for i in range(3))
+    out = p.cast(p.add(p.sigmoid(p.mul(x, y)), p.relu(z)), storage)
+    return p, [out]
+
+
+def sigmoid_product_relu_grad(storage=BF16, math=F32):
+    """Gradient program of out = sigmoid(x*y) + relu(z) for upstream dout; inputs (dout, x, y, z).
+    With s = sigmoid(x*y), ds = dout * s * (1 - s):  dx = ds * y,  dy = ds * x,  dz = dout where z > 0 else 0.
+    Returns (program, [dx_id, dy_id, dz_elem_id]); when z is constant down the rows its partial is the sum of the last
+    value over the rows (a value used by every row collects every row's contribution)."""
+    p = Program([storage] * 4)
+    d, x, y, z = (p.cast(i, math) for i in range(4))
+    s = p.sigmoid(p.mul(x, y))
+    one = p.const(1.0, math)
+    ds = p.mul(d, p.mul(s, p.sub(one, s)))
+    dx = p.cast(p.mul(ds, y), storage)
+    dy = p.cast(p.mul(ds, x), storage)
+    zero = p.const(0.0, math)
+    dz = p.select(p.cmp(OP_GT, z, zero), d, zero)
+    return p, [dx, dy, dz]

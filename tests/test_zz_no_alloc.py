@@ -23,7 +23,9 @@ def _outputs(rows, cols):
 def test_static_scratch_matches_workspace_entry_point_twice_in_a_row():
     prog, ids = P.tanh_affine_residual_grad(P.BF16)
     specs = [(ids[0], B.RED_NONE, 0, 0), (ids[1], B.RED_SUM, 1, 0), (ids[2], B.RED_SUM, 1, 1)]
-    for call, (rows, cols) in enumerate([(517, 1024), (2048, 4096)]):      # two calls in a row, the second larger
+    # calls in a row on the shared array: a larger one after a smaller one, then a smaller one again (fewer row slices
+    # than the array still holds from the call before: stale partials must not be read)
+    for call, (rows, cols) in enumerate([(517, 1024), (2048, 4096), (96, 1024)]):
         t = I.cfg2_ewise(rows, cols, salt=call)
         ins = [t[k].to(DEV) for k in ("dout", "x", "a", "b")]
         need = B.relay_workspace_bytes_reduce(ins, specs)
