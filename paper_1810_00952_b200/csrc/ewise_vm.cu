@@ -52,12 +52,12 @@ enum : int {
 };
 static_assert(RELAY_OP_COUNT_ == 22, "the machine's own opcodes start after the program's operators");
 
-// operand of an instruction: 0..7 input i; 8.. slot (temporaries first, then literals); SELECT packs two temporaries
+// operand of an instruction: 0..7 input i; 8.. slot (temporaries first, then literals)
 constexpr int OPD_SLOT = 8;
 
 struct VmCode {
     int32_t n;
-    uint8_t op[VM_MAXCODE], opd[VM_MAXCODE];
+    uint8_t op[VM_MAXCODE], opd[VM_MAXCODE], opd2[VM_MAXCODE];   // opd2: SELECT's second operand
 };
 
 struct VmArgs {
@@ -83,16 +83,27 @@ template <typename T> __device__ __forceinline__ int vm_col(int tx, int v)
     else return (v < 4 ? 0 : 128) + tx * 4 + (v & 3);
 }
 
+__device__ __forceinline__ uint4 lds128(uint32_t addr)
+{
+    uint4 r;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
+    return r;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, const uint4 &r)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(r.x), "r"(r.y), "r"(r.z), "r"(r.w) : "memory");
+}
+
 // (register arrays are only ever indexed with constants and never passed as pointers: a pointer into one would move it
 // to local memory)
-template <typename T> __device__ __forceinline__ void vm_load_row(const char *row, int tx, bool hi_live, float (&f)[VM_V])
+template <typename T> __device__ __forceinline__ void vm_load_row(uint32_t row, bool hi_live, float (&f)[VM_V])
 {
     if constexpr (sizeof(T) == 2) {
-        unpack(*reinterpret_cast<const uint4 *>(row + tx * 16), f);
+        unpack(lds128(row), f);
     } else {
         float lo[4], hi[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        unpack(*reinterpret_cast<const uint4 *>(row + tx * 16), lo);
-        if (hi_live) unpack(*reinterpret_cast<const uint4 *>(row + 512 + tx * 16), hi);
+        unpack(lds128(row), lo);
+        if (hi_live) unpack(lds128(row + 512), hi);
 #pragma unroll
         for (int v = 0; v < 4; ++v) { f[v] = lo[v]; f[4 + v] = hi[v]; }
     }
@@ -123,10 +134,11 @@ template <int N> __device__ __forceinline__ void vm_store_run(void *out, int dt,
     }
 }
 
-struct VmThread {
-    const char *stage;      // ring stage of the current tile
-    const char *fixed;      // rows of the operands that are constant down the rows
-    char *slots;            // temporaries: [slot][4 pieces of 16 bytes][256 threads]; literals behind them: 16 bytes each
+struct VmThread {             // shared-memory addresses are 32-bit shared-window addresses, already offset by this thread's lane
+    uint32_t stage;         // ring stage of the current tile + ty * row_bytes + tx * 16
+    uint32_t fixed;         // rows of the operands that are constant down the rows + tx * 16
+    uint32_t temps;         // temporaries: [slot][4 pieces of 16 bytes][256 threads] + tid * 16
+    uint32_t literals;      // 16 bytes each, behind the temporaries
     int tx, ty, tid;
     bool hi_live;           // f32: the thread's second run of 4 columns lies inside the tensor
     bool row_live[VM_R];
@@ -141,15 +153,15 @@ __device__ __forceinline__ void vm_fetch(int opd, float (&o)[VM_E], const VmArgs
     if (opd < OPD_SLOT) {
         const int slot = A.in_slot[opd];
         if (A.in_kind[opd] == 0) {
-            const char *row = th.stage + slot * th.tile_bytes + th.ty * th.row_bytes;
+            const uint32_t row = th.stage + slot * th.tile_bytes;
             float r0[VM_V], r1[VM_V];
-            vm_load_row<T>(row, th.tx, th.hi_live, r0);
-            vm_load_row<T>(row + VM_TY * th.row_bytes, th.tx, th.hi_live, r1);
+            vm_load_row<T>(row, th.hi_live, r0);
+            vm_load_row<T>(row + VM_TY * th.row_bytes, th.hi_live, r1);
 #pragma unroll
             for (int v = 0; v < VM_V; ++v) { o[v] = r0[v]; o[VM_V + v] = r1[v]; }
         } else {
             float r0[VM_V];
-            vm_load_row<T>(th.fixed + slot * (VM_COLS * (int)sizeof(T)), th.tx, th.hi_live, r0);
+            vm_load_row<T>(th.fixed + slot * (VM_COLS * (int)sizeof(T)), th.hi_live, r0);
 #pragma unroll
             for (int v = 0; v < VM_V; ++v) { o[v] = r0[v]; o[VM_V + v] = r0[v]; }
         }
@@ -157,18 +169,18 @@ __device__ __forceinline__ void vm_fetch(int opd, float (&o)[VM_E], const VmArgs
         // a temporary (one 64-byte value per thread, in four pieces) or a literal (one 16-byte piece for everybody)
         const int k = opd - OPD_SLOT;
         const bool temp = k < th.n_temp;
-        const char *p = temp ? th.slots + (k * 4 * VM_THREADS + th.tid) * 16 : th.slots + (th.n_temp * 4 * VM_THREADS + (k - th.n_temp)) * 16;
-        const int step = temp ? VM_THREADS * 16 : 0;
+        const uint32_t p = temp ? th.temps + k * (4 * VM_THREADS * 16) : th.literals + (k - th.n_temp) * 16;
+        const uint32_t step = temp ? VM_THREADS * 16 : 0;
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-            const uint4 w = *reinterpret_cast<const uint4 *>(p + q * step);
+            const uint4 w = lds128(p + q * step);
             o[4 * q] = __uint_as_float(w.x); o[4 * q + 1] = __uint_as_float(w.y); o[4 * q + 2] = __uint_as_float(w.z); o[4 * q + 3] = __uint_as_float(w.w);
         }
     }
 }
 
 template <typename T, bool FAST>
-__global__ void __launch_bounds__(VM_THREADS, 2)
+__global__ void __launch_bounds__(VM_THREADS, 3)
 ewise_vm_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constant__ CUtensorMap tm1, const __grid_constant__ CUtensorMap tm2,
                 const __grid_constant__ CUtensorMap tm3, const __grid_constant__ VmArgs A)
 {
@@ -231,8 +243,9 @@ ewise_vm_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constant__
         if (warp == 0)
             for (int t = 0; t < STAGES - 1 && t < n_tiles && ok_issue; ++t) ok_issue = issue(t);
         VmThread th;
-        th.fixed = reinterpret_cast<const char *>(fixed);
-        th.slots = reinterpret_cast<char *>(slots);
+        th.fixed = tc::smem_u32(fixed) + lane * 16;
+        th.temps = tc::smem_u32(slots) + tid * 16;
+        th.literals = tc::smem_u32(slots) + A.n_temp * 4 * VM_THREADS * 16;
         th.tx = lane; th.ty = warp; th.tid = tid;
         th.tile_bytes = tile_bytes; th.row_bytes = row_bytes; th.n_temp = A.n_temp;
         th.col0 = col0;
@@ -248,7 +261,7 @@ ewise_vm_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constant__
             if (lane == 0) ok = tc::mbar_wait(&full[st], (t / STAGES) & 1, abort_flag, A.err, tc::ERR_WAIT_FULL) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
-            th.stage = reinterpret_cast<const char *>(smem + st * stage_bytes);
+            th.stage = tc::smem_u32(smem + st * stage_bytes) + warp * row_bytes + lane * 16;
             th.row0 = r0 + (int64_t)t * A.box_rows;
 #pragma unroll
             for (int r = 0; r < VM_R; ++r) th.row_live[r] = warp + VM_TY * r < A.box_rows && th.row0 + warp + VM_TY * r < r1;
@@ -303,20 +316,20 @@ ewise_vm_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constant__
                             VM_UN(RELAY_OP_LOG, FAST ? __logf(x) : logf(x))
                             VM_UN(A_ROUND_BF16, round_bf16(x))
                             VM_UN(A_TO_BOOL, x != 0.0f ? 1.0f : 0.0f)
-                        case RELAY_OP_SELECT: {      // acc = acc ? temporary (opd & 15) : temporary (opd >> 4)
+                        case RELAY_OP_SELECT: {      // acc = acc ? operand : second operand
                             float a[VM_E], b[VM_E];
-                            vm_fetch<T>(OPD_SLOT + (opd & 15), a, A, th);
-                            vm_fetch<T>(OPD_SLOT + (opd >> 4), b, A, th);
+                            vm_fetch<T>(opd, a, A, th);
+                            vm_fetch<T>(A.code.opd2[pc], b, A, th);
 #pragma unroll
                             for (int e = 0; e < VM_E; ++e) acc[e] = acc[e] != 0.0f ? a[e] : b[e];
                             break;
                         }
                         case A_STASH: {
-                            char *p = th.slots + ((opd - OPD_SLOT) * 4 * VM_THREADS + tid) * 16;
+                            const uint32_t p = th.temps + (opd - OPD_SLOT) * (4 * VM_THREADS * 16);
 #pragma unroll
                             for (int q = 0; q < 4; ++q)
-                                *reinterpret_cast<uint4 *>(p + q * VM_THREADS * 16) = make_uint4(__float_as_uint(acc[4 * q]), __float_as_uint(acc[4 * q + 1]),
-                                                                                                 __float_as_uint(acc[4 * q + 2]), __float_as_uint(acc[4 * q + 3]));
+                                sts128(p + q * VM_THREADS * 16, make_uint4(__float_as_uint(acc[4 * q]), __float_as_uint(acc[4 * q + 1]), __float_as_uint(acc[4 * q + 2]),
+                                                                           __float_as_uint(acc[4 * q + 3])));
                             break;
                         }
                         case A_STORE: {
@@ -397,10 +410,10 @@ struct Compiler {
 
     Compiler(const TypedProgram &t, VmCode &c) : tp(t), code(c) { code.n = 0; }
 
-    void emit(int op, int opd)
+    void emit(int op, int opd, int opd2 = 0)
     {
         if (code.n >= VM_MAXCODE) { ok = false; return; }
-        code.op[code.n] = (uint8_t)op; code.opd[code.n] = (uint8_t)opd;
+        code.op[code.n] = (uint8_t)op; code.opd[code.n] = (uint8_t)opd; code.opd2[code.n] = (uint8_t)opd2;
         ++code.n;
         last_op = op;
         if (op != A_STASH && op != A_STORE && op != A_COLSUM0 && op != A_COLSUM1) acc_holds = -1;
@@ -451,17 +464,16 @@ struct Compiler {
         default: return op;          // commutative
         }
     }
-    // a temporary that holds v, for SELECT (an input, a literal or an expression is copied into one first)
-    int as_temp(int v, int depth, bool *owned)
+    // operand code of v for SELECT: a leaf as it is, anything else through a temporary
+    int as_operand(int v, int depth, int *owned_temp)
     {
-        v = alias[v];
-        *owned = false;
-        if (v >= tp.n_in && home[v] >= 0) return home[v];
+        *owned_temp = -1;
+        if (is_leaf(v)) return operand(v);
         gen(v, depth + 1);
         const int t = alloc_temp();
         emit(A_STASH, OPD_SLOT + t);
-        *owned = true;
-        return t;
+        *owned_temp = t;
+        return OPD_SLOT + t;
     }
 
     // evaluates value v into the accumulator
@@ -476,12 +488,12 @@ struct Compiler {
             gen(in.a, depth + 1);
             emit(in.dtype == RELAY_BF16 ? A_ROUND_BF16 : A_TO_BOOL, 0);
         } else if (in.op == RELAY_OP_SELECT) {
-            bool own_b, own_c;
-            const int tb = as_temp(in.b, depth, &own_b), tc_ = as_temp(in.c, depth, &own_c);
+            int own_b, own_c;
+            const int ob = as_operand(in.b, depth, &own_b), oc = as_operand(in.c, depth, &own_c);
             gen(in.a, depth + 1);
-            emit(RELAY_OP_SELECT, tb | (tc_ << 4));
-            if (own_b) temp_used[tb] = false;
-            if (own_c) temp_used[tc_] = false;
+            emit(RELAY_OP_SELECT, ob, oc);
+            if (own_b >= 0) temp_used[own_b] = false;
+            if (own_c >= 0) temp_used[own_c] = false;
         } else if (in.b < 0) {              // unary
             gen(in.a, depth + 1);
             emit(in.op, 0);
@@ -508,8 +520,10 @@ struct Compiler {
     // literals live behind the temporaries
     void finish()
     {
-        for (int i = 0; i < code.n; ++i)
-            if (code.opd[i] >= 128 && code.op[i] != RELAY_OP_SELECT) code.opd[i] = (uint8_t)(OPD_SLOT + n_temp + (code.opd[i] - 128));
+        for (int i = 0; i < code.n; ++i) {
+            if (code.opd[i] >= 128) code.opd[i] = (uint8_t)(OPD_SLOT + n_temp + (code.opd[i] - 128));
+            if (code.opd2[i] >= 128) code.opd2[i] = (uint8_t)(OPD_SLOT + n_temp + (code.opd2[i] - 128));
+        }
     }
 };
 
