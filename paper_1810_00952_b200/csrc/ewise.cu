@@ -23,7 +23,14 @@ namespace relay {
 // =================================================================================================
 constexpr int kTX = 32, kTY = 8, kUnroll = 4;
 
-template <typename Body, typename T, bool FAST>
+// CL > 1: the kernel is launched in clusters of CL blocks along y, the row slices of one column strip.  The slices'
+// partial column sums then never leave the chip: every block leaves its partials in its own shared memory, and after a
+// cluster barrier block r of the cluster adds up, in slice order, the CL partials of its share of the strip's columns
+// through distributed shared memory and writes the final sums (A.final[k], times A.scale[k]).  No second launch and no
+// scratch memory; the order is fixed, so reruns are bit-identical.
+constexpr int kColsumCluster = 8;
+
+template <typename Body, typename T, bool FAST, int CL = 1>
 __global__ void __launch_bounds__(kTX *kTY, Body::NIN >= 4 ? 2 : 3) ewise2d_kernel(const Args2D<Body::NIN, Body::NOUT> A)
 {
     constexpr int V = VecN<T>::N, NIN = Body::NIN, NOUT = Body::NOUT;
@@ -107,22 +114,51 @@ __global__ void __launch_bounds__(kTX *kTY, Body::NIN >= 4 ? 2 : 3) ewise2d_kern
     constexpr bool any_sum = []() { bool s = false; for (int k = 0; k < NOUT; ++k) s = s || Body::col_sum(k); return s; }();
     if constexpr (any_sum) {
         __shared__ float sm[kTY][kTX * V + 1];
+        __shared__ float mine[CL > 1 ? NOUT : 1][kTX * V];      // CL > 1: this block's partials, read by its cluster
 #pragma unroll
         for (int k = 0; k < NOUT; ++k) {
             if (!Body::col_sum(k)) continue;
 #pragma unroll
             for (int v = 0; v < V; ++v) sm[ty][tx * V + v] = acc[k][v];
             __syncthreads();
-            if (ty == 0 && active && A.partial[k] != nullptr) {
+            if (ty == 0) {
 #pragma unroll
                 for (int v = 0; v < V; ++v) {
                     float s = 0.0f;
 #pragma unroll
                     for (int j = 0; j < kTY; ++j) s += sm[j][tx * V + v];
-                    A.partial[k][(int64_t)blockIdx.y * A.cols + col0 + v] = s;
+                    if constexpr (CL > 1) mine[k][tx * V + v] = active ? s : 0.0f;
+                    else if (active && A.partial[k] != nullptr) A.partial[k][(int64_t)blockIdx.y * A.cols + col0 + v] = s;
                 }
             }
             __syncthreads();
+        }
+        if constexpr (CL > 1) {
+            asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+            uint32_t rank;
+            asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+            constexpr int share = kTX * V / CL;                     // columns of the strip that this block finishes
+            const int t = ty * kTX + tx;
+            if (t < share) {
+                const int c = (int)rank * share + t;
+                const int64_t col = (int64_t)blockIdx.x * (kTX * V) + c;
+#pragma unroll
+                for (int k = 0; k < NOUT; ++k) {
+                    if (!Body::col_sum(k) || A.final[k] == nullptr) continue;
+                    float s = 0.0f;
+#pragma unroll
+                    for (int j = 0; j < CL; ++j) {
+                        uint32_t remote;
+                        float v;
+                        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"((uint32_t)__cvta_generic_to_shared(&mine[k][c])), "r"(j));
+                        asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+                        s += v;
+                    }
+                    if (col < A.cols) A.final[k][col] = s * A.scale[k];
+                }
+            }
+            // no block may exit (and give up its shared memory) while another still reads it
+            asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
         }
     }
 }
@@ -475,6 +511,29 @@ relay_status_t launch_body2d(int32_t storage, const Args2D<Body::NIN, Body::NOUT
     return check_launch(what);
 }
 
+// Column sums finished inside the kernel by clusters of kColsumCluster row slices (no partials, no second launch):
+// taken when that many slices per column strip give every SM a block.  A.final / A.scale name the results.  Used for the
+// bodies with three or more streamed inputs; with one or two inputs 8 blocks per strip measured slower than the many
+// short slices of the two-pass form (8192 x 8192 bf16 column sum: 41 us against 30 us).
+static bool cluster_sums(int64_t rows, int64_t cols, int32_t storage)
+{
+    const int vec = storage == RELAY_BF16 ? 8 : 4;
+    const int64_t gx = (cols + (int64_t)kTX * vec - 1) / (kTX * vec);
+    return gx * kColsumCluster >= 148 && rows >= 32 * kColsumCluster;
+}
+template <typename Body>
+relay_status_t launch_body2d_cluster(int32_t storage, const Args2D<Body::NIN, Body::NOUT> &A0, cudaStream_t st, const char *what)
+{
+    Args2D<Body::NIN, Body::NOUT> A = A0;
+    const int vec = storage == RELAY_BF16 ? 8 : 4;
+    const dim3 block(kTX, kTY), cluster(1, kColsumCluster, 1);
+    const dim3 grid((unsigned)((A.cols + (int64_t)kTX * vec - 1) / (kTX * vec)), kColsumCluster);
+    A.rows_per_slice = (int)((A.rows + kColsumCluster - 1) / kColsumCluster);
+    if (storage == RELAY_BF16) RELAY_CUDA(launch_pdl_cluster(ewise2d_kernel<Body, __nv_bfloat16, true, kColsumCluster>, grid, block, cluster, 0, st, A));
+    else RELAY_CUDA(launch_pdl_cluster(ewise2d_kernel<Body, float, false, kColsumCluster>, grid, block, cluster, 0, st, A));
+    return check_launch(what);
+}
+
 relay_status_t launch_colsum_finalize_n(const float *partial, int n_slices, int64_t cols, const float *scale, float *const *out, int n_out,
                                         cudaStream_t st)
 {
@@ -723,6 +782,11 @@ extern "C" relay_status_t relay_fused_reduce(const relay_ewise_prog_t *prog, con
         A.out[0] = outputs[0]->data; A.out[1] = A.out[2] = nullptr;
         A.partial[0] = nullptr; A.partial[1] = part; A.partial[2] = part + (size_t)pl.n_slices * v.cols;
         A.rows = v.rows; A.cols = v.cols; A.aux = 0;
+        if (cluster_sums(v.rows, v.cols, v.storage)) {
+            A.partial[1] = A.partial[2] = nullptr;
+            A.final[1] = (float *)outputs[1]->data; A.final[2] = (float *)outputs[2]->data; A.scale[1] = A.scale[2] = 1.0f;
+            return launch_body2d_cluster<BodyTanhAffineResidualGrad>(v.storage, A, st, "ewise2d<tanh_affine_residual_grad>");
+        }
         RELAY_TRY(launch_body2d<BodyTanhAffineResidualGrad>(v.storage, A, pl.n_slices, st, "ewise2d<tanh_affine_residual_grad>"));
         float *sums[2] = {(float *)outputs[1]->data, (float *)outputs[2]->data};
         return launch_colsum_finalize_n(A.partial[1], pl.n_slices, v.cols, nullptr, sums, 2, st);
@@ -731,8 +795,8 @@ extern "C" relay_status_t relay_fused_reduce(const relay_ewise_prog_t *prog, con
         Args2D<1, 1> A{};
         A.in[0] = inputs[0]->data; A.out[0] = nullptr; A.partial[0] = (float *)ws;
         A.rows = v.rows; A.cols = v.cols; A.aux = 0;
-        RELAY_TRY(launch_body2d<BodyIdentityColSum>(v.storage, A, pl.n_slices, st, "ewise2d<identity_colsum>"));
         const float scale = specs[0].red_op == RELAY_RED_MEAN ? 1.0f / (float)v.rows : 1.0f;
+        RELAY_TRY(launch_body2d<BodyIdentityColSum>(v.storage, A, pl.n_slices, st, "ewise2d<identity_colsum>"));
         return launch_colsum_finalize(A.partial[0], pl.n_slices, v.cols, scale, (float *)outputs[0]->data, st);
     }
     if (pl.fast_row) {

@@ -294,7 +294,9 @@ template <int NIN, int NOUT>
 struct Args2D {
     const void *in[NIN];
     void *out[NOUT];        // unreduced results (storage type T); unused for summed results
-    float *partial[NOUT];   // [n_slices][cols] fp32 partial column sums for summed results
+    float *partial[NOUT];   // [n_slices][cols] fp32 partial column sums for summed results (launches without clusters)
+    float *final[NOUT];     // cluster launches: the finished column sums, [cols] fp32 ...
+    float scale[NOUT];      // ... times this factor
     int64_t rows, cols;
     int rows_per_slice;
     int aux;                // body-specific run-time attribute (e.g. activation code)
