@@ -105,10 +105,14 @@ class Timer:
     """CUDA-event timing of labelled regions on the current stream."""
 
     def __init__(self):
-        self.pending, self.ms = [], {}
+        self.pending, self.ms, self.div = [], {}, {}
 
-    def region(self, label):
+    def region(self, label, launches=1):
+        """`launches` > 1: the region holds that many back-to-back launches of one kernel on DIFFERENT tensors (nothing a launch
+        reads was touched by the launches before it); the recorded time is the region's divided by `launches`, i.e. the
+        kernel's average duration without the few microseconds of event and launch latency that a lone short kernel carries."""
         t = self
+        t.div[label] = launches
 
         class R:
             def __enter__(self_inner):
@@ -123,7 +127,7 @@ class Timer:
     def collect(self):
         torch.cuda.synchronize()
         for label, a, b in self.pending:
-            self.ms.setdefault(label, []).append(a.elapsed_time(b))
+            self.ms.setdefault(label, []).append(a.elapsed_time(b) / self.div.get(label, 1))
         self.pending = []
 
 
@@ -278,6 +282,10 @@ class Workload:
             ps_ = (shp[0], shp[1], shp[2] // 2, shp[3] // 2)
             self.pool_y, self.pool_idx = E(*ps_), E(*ps_, dt=torch.int32)
             self.pool_dy, self.pool_dx = I.normal(8, 1, ps_, 1.0, torch.bfloat16).to(dev), torch.empty_like(self.pool_x)
+            # four sets of tensors for four back-to-back launches (a launch's 90 MB are then not in L2 from the one before)
+            self.pool_sets = [dict(x=self.pool_x, y=self.pool_y, idx=self.pool_idx, dy=self.pool_dy, dx=self.pool_dx)]
+            for _ in range(0 if small else 3):
+                self.pool_sets.append({k: v.clone() for k, v in self.pool_sets[0].items()})
             self.lenet = LeNetStep(B, I, dev, 4 if small else 64)
             # the conv configuration's tensors tagged NHWC (device-resident, permuted once): the layout-tagged calls
             c4 = self.devt["cfg4"] if "cfg4" in groups else {k: v.to(dev) for k, v in
@@ -371,10 +379,13 @@ class Workload:
                 B.relay_fused_reduce(self.vm_grad.arrays(), [d["dout"], d["x"], o["out"], d["a"]], self.vm_grad_specs,
                                      [self.vm_out["dx"], self.vm_out["dy"], self.vm_out["dz"]], ws)
             ra = self.red_prog.arrays()
+            # four launches back to back, each on another 8192 x 8192 tensor (134 MB each, so none is still in L2)
+            red_ins = [d["x"], d["dout"], o["out"], o["dx"]]
             for key in ("sum1", "max1", "arg1", "sum0"):
                 self.flush_l2()
-                with tm.region("a8." + key):
-                    B.relay_fused_reduce(ra, [d["x"]], self.red_specs[key], [self.red_out[key]], ws)
+                with tm.region("a8." + key, launches=len(red_ins)):
+                    for xin in red_ins:
+                        B.relay_fused_reduce(ra, [xin], self.red_specs[key], [self.red_out[key]], ws)
         if "cfg3" in self.groups:
             d, o = self.devt["cfg3"], self.out["cfg3"]
             self.flush_l2()
@@ -428,11 +439,13 @@ class Workload:
             with tm.region("next.sgd"):
                 B.relay_sgd_update(self.sgd_params, self.sgd_grads, 1e-3)
             self.flush_l2()
-            with tm.region("next.pool"):
-                B.relay_max_pool2d(self.pool_x, 2, 2, 2, 2, self.pool_y, self.pool_idx)
+            with tm.region("next.pool", launches=len(self.pool_sets)):
+                for ps in self.pool_sets:
+                    B.relay_max_pool2d(ps["x"], 2, 2, 2, 2, ps["y"], ps["idx"])
             self.flush_l2()
-            with tm.region("next.pool_grad"):
-                B.relay_max_pool2d_grad(self.pool_idx, self.pool_dy, 2, 2, 2, 2, self.pool_dx)
+            with tm.region("next.pool_grad", launches=len(self.pool_sets)):
+                for ps in self.pool_sets:
+                    B.relay_max_pool2d_grad(ps["idx"], ps["dy"], 2, 2, 2, 2, ps["dx"])
             with tm.region("next.lenet"):
                 self.lenet.run()
             if self.lenet.graph is not None:
@@ -824,6 +837,25 @@ def main():
                        "(pipelined over two buffer sets: upload of the next step and read-back of the previous one overlap the compute); "
                        "dense+conv FLOPs over that time"}
 
+    # cfg5: where a step of the persistent kernel spends its time (one extra call, outside every timed region)
+    lstm_phases = None
+    if "cfg5" in groups and not args.small:
+        try:
+            d, o = wl.devt["cfg5"], wl.out["cfg5"]
+            cyc = torch.zeros(8, dtype=torch.int64, device=dev)
+            B.relay_debug_lstm_phase_cycles(d["x"], d["w_ih"], d["w_hh"], d["b"], d["h0"], d["c0"], o["h_all"], o["c"], wl.ws, cyc)
+            torch.cuda.synchronize()
+            c = [int(v) for v in cyc.cpu()]
+            mhz = clocks.get("sm_mhz") or 1965.0
+            T_ = max(c[7], 1)
+            us = lambda v: v / T_ / mhz
+            lstm_phases = {"us_per_step": us(c[0]), "loader_waits_for_grid_barrier_us": us(c[3]), "loader_issues_copies_us": us(c[4]),
+                           "issuer_waits_for_first_stage_us": us(c[5]), "issuer_first_stage_to_last_commit_us": us(c[6]),
+                           "epilogue_waits_for_product_us": us(c[1]), "epilogue_gates_and_publish_us": us(c[2]),
+                           "note": "cycle counts of block 0 summed over the steps / T / sampled SM clock; the phases of the three warp roles overlap"}
+        except Exception as e:      # the breakdown is a report, not a gate
+            lstm_phases = {"error": str(e)}
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         r = oracle_sample()
@@ -841,9 +873,10 @@ def main():
                            + " forward + gradient on 32x256x56x56 bf16, one fp32 LeNet training step (batch 64) eager and replayed from a"
                            + " CUDA graph, the cfg4 conv with NHWC-tagged tensors; cfg1 is also replayed from a CUDA graph",
                            "value_covers": "dense + conv2d groups (cfg3 + cfg4) FLOPs / their device time; hbm_gbs covers cfg2, two programs on the vectorised evaluator (a6.vm_fwd, a7.vm_grad) and the standalone reductions (a8.*)",
-                           "groups": groups, "l2": "1 GiB streamed through L2 between groups (flush with clean lines); cfg2 inputs also exceed L2",
+                           "groups": groups, "l2": "1 GiB streamed through L2 between groups (flush with clean lines); cfg2 inputs also exceed L2; the standalone reductions and "
+                                 "the pooling kernels are timed as four back-to-back launches on four different sets of tensors (per-launch time = region / 4)",
                            "replicas": world},
-                "groups": table, "roofline": roofline, "rooflines": rooflines, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
+                "groups": table, "roofline": roofline, "rooflines": rooflines, "cfg5_step_phases": lstm_phases, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
                 "clocks": clocks, "peaks": dict({k: peaks.get(k) for k in ("hbm_gbs", "bf16_tflops", "bf16_tflops_sustained", "source")}, nominal=NOMINAL_PEAKS)}
         print(json.dumps(line))
     if dist is not None:

@@ -413,6 +413,18 @@ relay_status_t relay_debug_expire_wait(int32_t limit_us, void *stream);
  * (the kernel then follows its fixed scheme), -2 for bad arguments or max_units too small.  For tests of the plan. */
 int32_t relay_debug_plan_units(int64_t M, int64_t N, int64_t K, int32_t sms, uint32_t *units, int32_t max_units);
 
+/* relay_lstm_cell_seq with a per-phase cycle count of its dependent steps (no counterpart in the paper; same arguments and
+ * results).  `cycles` is a DEVICE pointer to 8 int64 that one block of the persistent kernel fills with SM-clock cycle
+ * counts summed over the T steps: [0] the whole step loop, [1] the epilogue warp waiting for the recurrent product,
+ * [2] the epilogue (accumulator read, gates, publishing bf16(h_t)), [3] the loader waiting on the grid barrier for
+ * h_{t-1} of all blocks, [4] the loader issuing the step's copies, [5] the MMA issuer waiting for the step's first
+ * operand stage, [6] the issuer from there to the step's last commit, [7] T.  RELAY_ERR_UNSUPPORTED for shapes that run
+ * one launch per step instead of the persistent kernel. */
+relay_status_t relay_debug_lstm_phase_cycles(const relay_tensor_t *x, const relay_tensor_t *w_ih, const relay_tensor_t *w_hh,
+                                             const relay_tensor_t *b, const relay_tensor_t *h0, const relay_tensor_t *c0,
+                                             const relay_tensor_t *h_all, const relay_tensor_t *c_final, void *ws, size_t ws_bytes,
+                                             int64_t *cycles, void *stream);
+
 /* Host-only view of which kernel tier relay_fused_ewise / relay_fused_reduce would run a group on (no counterpart in the
  * paper; touches no GPU; arguments as for relay_fused_reduce, all-RELAY_RED_NONE specs describe a relay_fused_ewise call):
  * 0 a pre-compiled body, 1 the vectorised evaluator (16-byte accesses, the program interpreted on 8 elements at a

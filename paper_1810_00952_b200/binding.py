@@ -326,6 +326,13 @@ def relay_fused_reduce_static_scratch(prog: Optional[dict], inputs, specs, outpu
                                                    _desc_array(outs), len(outs), _stream()))
 
 
+def relay_debug_lstm_phase_cycles(x, w_ih, w_hh, b, h0, c0, h_all, c_final, ws, cycles):
+    """relay_lstm_cell_seq that also fills `cycles` (device int64[8]) with per-phase cycle counts of the step loop."""
+    wp, wb = _ws(ws)
+    _check(lib().relay_debug_lstm_phase_cycles(_ref(desc(x)), _ref(desc(w_ih)), _ref(desc(w_hh)), _ref(desc(b)), _ref(desc(h0)), _ref(desc(c0)),
+                                               _ref(desc(h_all)), _ref(desc(c_final)), wp, wb, ctypes.c_void_p(cycles.data_ptr()), _stream()))
+
+
 def relay_lstm_cell_seq(x, w_ih, w_hh, b, h0, c0, h_all, c_final, ws=None):
     wp, wb = _ws(ws)
     _check(lib().relay_lstm_cell_seq(_ref(desc(x)), _ref(desc(w_ih)), _ref(desc(w_hh)), _ref(desc(b)), _ref(desc(h0)),

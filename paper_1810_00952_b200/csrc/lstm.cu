@@ -98,10 +98,9 @@ extern "C" size_t relay_workspace_bytes_lstm(const relay_tensor_t *x, const rela
     return lstm_ws(d);
 }
 
-extern "C" relay_status_t relay_lstm_cell_seq(const relay_tensor_t *x, const relay_tensor_t *w_ih, const relay_tensor_t *w_hh,
-                                              const relay_tensor_t *b, const relay_tensor_t *h0, const relay_tensor_t *c0,
-                                              const relay_tensor_t *h_all, const relay_tensor_t *c_final, void *ws, size_t ws_bytes,
-                                              void *stream)
+static relay_status_t lstm_seq(const relay_tensor_t *x, const relay_tensor_t *w_ih, const relay_tensor_t *w_hh, const relay_tensor_t *b,
+                               const relay_tensor_t *h0, const relay_tensor_t *c0, const relay_tensor_t *h_all, const relay_tensor_t *c_final,
+                               void *ws, size_t ws_bytes, void *stream, long long *timing)
 {
     clear_error();
     const relay_tensor_t *all[8] = {x, w_ih, w_hh, b, h0, c0, h_all, c_final};
@@ -144,7 +143,8 @@ extern "C" relay_status_t relay_lstm_cell_seq(const relay_tensor_t *x, const rel
     // (2) the dependent steps: one persistent kernel when the shape fits it, else one launch per step
     if (lstm_tc_eligible(d.T, d.B, d.H))
         return launch_lstm_tc(d.T, d.B, d.H, zx, w_hh->data, (const float *)h0->data, (const float *)c0->data, (float *)h_all->data,
-                              (float *)c_final->data, (char *)ws + lstm_zx_bytes(d), st);
+                              (float *)c_final->data, (char *)ws + lstm_zx_bytes(d), st, timing);
+    if (timing) return fail(RELAY_ERR_UNSUPPORTED, "phase cycles are counted by the persistent kernel only; this shape runs one launch per step");
     dim3 grid((unsigned)((d.H + 255) / 256), (unsigned)((d.B + kRowsPerBlock - 1) / kRowsPerBlock));
     float *hall = (float *)h_all->data;
     for (int64_t t = 0; t < d.T; ++t) {
@@ -154,4 +154,24 @@ extern "C" relay_status_t relay_lstm_cell_seq(const relay_tensor_t *x, const rel
         RELAY_TRY(check_launch("lstm_step"));
     }
     return RELAY_OK;
+}
+
+extern "C" relay_status_t relay_lstm_cell_seq(const relay_tensor_t *x, const relay_tensor_t *w_ih, const relay_tensor_t *w_hh,
+                                              const relay_tensor_t *b, const relay_tensor_t *h0, const relay_tensor_t *c0,
+                                              const relay_tensor_t *h_all, const relay_tensor_t *c_final, void *ws, size_t ws_bytes,
+                                              void *stream)
+{
+    return lstm_seq(x, w_ih, w_hh, b, h0, c0, h_all, c_final, ws, ws_bytes, stream, nullptr);
+}
+
+extern "C" relay_status_t relay_debug_lstm_phase_cycles(const relay_tensor_t *x, const relay_tensor_t *w_ih, const relay_tensor_t *w_hh,
+                                                        const relay_tensor_t *b, const relay_tensor_t *h0, const relay_tensor_t *c0,
+                                                        const relay_tensor_t *h_all, const relay_tensor_t *c_final, void *ws, size_t ws_bytes,
+                                                        int64_t *cycles, void *stream)
+{
+    clear_error();
+    RELAY_TRY(check_not_null(cycles, "cycles"));
+    if (((uintptr_t)cycles & 7) != 0) return fail(RELAY_ERR_ALIGN, "cycles: not 8-byte aligned");
+    RELAY_CUDA(cudaMemsetAsync(cycles, 0, 8 * sizeof(int64_t), (cudaStream_t)stream));
+    return lstm_seq(x, w_ih, w_hh, b, h0, c0, h_all, c_final, ws, ws_bytes, stream, (long long *)cycles);
 }

@@ -56,6 +56,7 @@ struct Params {
     __nv_bfloat16 *hq;               // [2][B][H] exchange buffer for bf16(h)
     unsigned int *counter;           // grid barrier
     int *err;
+    long long *timing;               // null, or 8 cycle counts that block 0 leaves (see relay_debug_lstm_phase_cycles)
 };
 
 __device__ __forceinline__ unsigned int ld_acquire(const unsigned int *p)
@@ -68,8 +69,11 @@ __device__ __forceinline__ void red_release_add(unsigned int *p, unsigned int v)
 {
     asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
-__device__ __forceinline__ float fast_sigmoid(float x) { return __fdividef(1.0f, 1.0f + __expf(-x)); }
-__device__ __forceinline__ float fast_tanh(float x) { return 1.0f - __fdividef(2.0f, 1.0f + __expf(2.0f * x)); }
+// The gate math of a step sits on the chain of dependent steps, 80 activations per lane: one MUFU instruction each
+// (tanh.approx, relative error 2^-11, far inside the bf16-operand tolerance of this path) instead of an exp2 and a
+// reciprocal.
+__device__ __forceinline__ float fast_tanh(float x) { return tanh_<true>(x); }
+__device__ __forceinline__ float fast_sigmoid(float x) { return fmaf(0.5f, tanh_<true>(0.5f * x), 0.5f); }
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_h0,
@@ -135,6 +139,9 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
         __syncwarp();
         if (lane == 0) red_release_add(counter, 1u);
 
+        const bool timed = p.timing != nullptr && blockIdx.x == 0 && warp == 0;
+        long long t_loop = 0, t_wait = 0, t_work = 0;
+        if (timed) t_loop = clock64();
         for (int t = 0; t < p.T; ++t) {
             // the input projection does not depend on h: fetch it while the recurrent product runs
             float zx[4][UNITS];
@@ -149,9 +156,11 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
                     }
             }
             int ok = 1;
+            const long long tw0 = timed ? clock64() : 0;
             if (lane == 0) ok = tc::mbar_wait(tmem_full, t & 1, abort_flag, p.err, tc::ERR_WAIT_TMEM_FULL) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
+            const long long tw1 = timed ? clock64() : 0;
             tc::tc_fence_after_sync();
             uint32_t d0[32], d1[32];
             const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16);
@@ -192,12 +201,14 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
             asm volatile("fence.proxy.async.global;" ::: "memory");
             __syncwarp();
             if (lane == 0) red_release_add(counter, 1u);
+            if (timed) { t_wait += tw1 - tw0; t_work += clock64() - tw1; }
             if (live) {   // the fp32 copy for the caller is off the critical path
                 float4 *ho = reinterpret_cast<float4 *>(p.h_all + ((size_t)t * p.B + b) * p.H + j0);
 #pragma unroll
                 for (int i = 0; i < UNITS; i += 4) ho[i / 4] = make_float4(hn[i], hn[i + 1], hn[i + 2], hn[i + 3]);
             }
         }
+        if (timed && lane == 0) { p.timing[0] = clock64() - t_loop; p.timing[1] = t_wait; p.timing[2] = t_work; p.timing[7] = p.T; }
         if (live) {
 #pragma unroll
             for (int i = 0; i < UNITS; ++i) p.c_final[(size_t)b * p.H + j0 + i] = c[i];
@@ -214,7 +225,10 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
             uint32_t phase = 0;
             bool ok = true;
             const uint32_t stage_bytes = (uint32_t)(p.n_iss * p.rows_per_group * 128);
+            const bool timed = p.timing != nullptr && blockIdx.x == 0 && ld == 0 && lane == 0;
+            long long t_bar = 0, t_iss = 0;
             for (int t = 0; t < p.T && ok; ++t) {
+                const long long tb0 = timed ? clock64() : 0;
                 // grid barrier: every block has published its part of h_{t-1} (lane 0 polls, the warp follows)
                 const unsigned int target = (unsigned int)(p.n_epi * p.n_blocks) * (unsigned int)(t + 1);   // n_epi arrivals per block
                 if (lane == 0) {
@@ -232,6 +246,7 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
                 asm volatile("fence.proxy.async.global;" ::: "memory");   // every lane: whichever lane is elected issues the copies
+                const long long tb1 = timed ? clock64() : 0;
                 const CUtensorMap *tm_h = (t & 1) ? &tm_h1 : &tm_h0;
                 for (int kb = ld * p.n_iss; kb < p.k_blocks; kb += p.n_load * p.n_iss) {
                     ok = __all_sync(0xffffffffu, tc::mbar_wait(&empty[s], phase ^ 1, abort_flag, p.err, tc::ERR_WAIT_EMPTY));
@@ -246,7 +261,9 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
                     s += p.n_load;
                     if (s >= p.n_stages) { s -= p.n_stages; phase ^= 1; }
                 }
+                if (timed) { t_bar += tb1 - tb0; t_iss += clock64() - tb1; }
             }
+            if (timed) { p.timing[3] = t_bar; p.timing[4] = t_iss; }
         }
     } else {
         // ------------------------------ MMA issuers (warp 4 also loads the W slice) ------------------------------
@@ -267,12 +284,17 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
             const uint32_t d_tmem = tmem_base + iss * NCOL;
             int s = 0;
             uint32_t phase = 0, a_off = 0;
+            const bool timed = p.timing != nullptr && blockIdx.x == 0 && iss == 0 && lane == 0;
+            long long t_first = 0, t_rest = 0;          // wait for the step's first stage (barrier + first copy); first stage -> last commit
             for (int t = 0; t < p.T && ok; ++t) {
                 uint32_t b_off = 0;
+                const long long tm0 = timed ? clock64() : 0;
+                long long tm1 = 0;
                 for (int kb = 0; kb < p.k_blocks; kb += p.n_iss) {     // this issuer's k-block of the stage: kb + iss
                     // every lane waits; the vote reconverges the warp (the lanes leave the wait at different times)
                     ok = __all_sync(0xffffffffu, tc::mbar_wait(&full[s], phase, abort_flag, p.err, tc::ERR_WAIT_FULL));
                     if (!ok) break;
+                    if (timed && kb == 0) tm1 = clock64();
                     tc::tc_fence_after_sync();
                     const uint64_t da = desc_a0 + a_off, db = desc_b0 + b_off;
                     const uint32_t acc = kb != 0;
@@ -283,7 +305,9 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
                     if (++s == p.n_stages) { s = 0; phase ^= 1; a_off = 0; }
                 }
                 if (ok) tc::mma_commit_elect(tmem_full);
+                if (timed) { t_first += tm1 - tm0; t_rest += clock64() - tm1; }
             }
+            if (timed) { p.timing[5] = t_first; p.timing[6] = t_rest; }
         }
     }
     tc::tc_fence_before_sync();
@@ -326,7 +350,7 @@ size_t lstm_tc_workspace(int64_t B, int64_t H)
 }
 
 relay_status_t launch_lstm_tc(int64_t T, int64_t B, int64_t H, const float *zx, const void *w_hh, const float *h0, const float *c0,
-                              float *h_all, float *c_final, void *ws, cudaStream_t st)
+                              float *h_all, float *c_final, void *ws, cudaStream_t st, long long *timing)
 {
     char *base = (char *)ws;
     __nv_bfloat16 *wp = (__nv_bfloat16 *)base;
@@ -352,6 +376,7 @@ relay_status_t launch_lstm_tc(int64_t T, int64_t B, int64_t H, const float *zx, 
     p.rows_per_group = rows_per_group; p.n_epi = (rows_per_group + 31) / 32;
     p.zx = zx; p.h0 = h0; p.c0 = c0; p.h_all = h_all; p.c_final = c_final; p.hq = hq; p.counter = counter;
     p.err = device_error_word();
+    p.timing = timing;
     if (!p.err) return fail(RELAY_ERR_CUDA, "no device error word");
     p.n_iss = p.k_blocks % 2 == 0 ? 2 : 1;
     p.tile_stride = (int)align_up((size_t)rows_per_group * 128, 1024);

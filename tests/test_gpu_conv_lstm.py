@@ -248,3 +248,18 @@ def test_lstm_rejections():
     with pytest.raises(B.RelayError) as e:
         B.relay_lstm_cell_seq(t["x"], t["w_ih"], t["w_hh"], t["b"], t["h0"], t["c0"], h_all, c, None)
     assert e.value.status_name == "ERR_WORKSPACE"
+
+
+def test_lstm_phase_cycle_report_leaves_results_unchanged():
+    """The instrumented call returns the same h_all / c_final bit for bit and plausible counts (phases within the loop)."""
+    t = I.cfg5_lstm(6, 16, 128, 256, salt=3)
+    d = {k: v.to(DEV) for k, v in t.items()}
+    h1, c1 = lstm(t)
+    h2, c2 = torch.empty_like(h1), torch.empty_like(c1)
+    ws = workspace(B.relay_workspace_bytes_lstm(d["x"], d["w_ih"], d["w_hh"]), DEV)
+    cyc = torch.full((8,), -1, dtype=torch.int64, device=DEV)
+    B.relay_debug_lstm_phase_cycles(d["x"], d["w_ih"], d["w_hh"], d["b"], d["h0"], d["c0"], h2, c2, ws, cyc)
+    B.relay_poll_status()
+    assert torch.equal(h1, h2) and torch.equal(c1, c2)
+    c = cyc.cpu().tolist()
+    assert c[7] == 6 and c[0] > 0 and all(0 <= v <= c[0] for v in c[1:7])
