@@ -125,6 +125,9 @@ extern "C" relay_status_t relay_fused_dense_act(const relay_tensor_t *x, const r
     RELAY_TRY(check_data(y, "y"));
     const relay_tensor_t *outs[1] = {y}, *ins[3] = {x, w, b};
     RELAY_TRY(check_no_overlap(outs, 1, ins, 3));
+    if (dense_small_eligible(d.M, d.K, d.N, d.dt))
+        return launch_dense_small_fwd(d.dt, x->data, w->data, b ? b->data : nullptr, b ? b->dtype : RELAY_F32, y->data, d.M, d.K, d.N, act,
+                                      (cudaStream_t)stream);
     GemmDesc g;
     g.M = d.M; g.N = d.N; g.K = d.K;
     g.a = x->data; g.a_sm = d.K; g.a_sk = 1;
@@ -180,6 +183,9 @@ extern "C" relay_status_t relay_fused_dense_act_grad(const relay_tensor_t *x, co
         return RELAY_OK;
     }
 
+    if (dense_small_eligible(d.M, d.K, d.N, d.dt))
+        return launch_dense_small_grad(d.dt, x->data, w->data, y->data, dy->data, dx ? dx->data : nullptr, dw->data, db ? (float *)db->data : nullptr,
+                                       d.M, d.K, d.N, act, st);
     void *dz = ws;
     float *partials = (float *)((char *)ws + dz_bytes);
     RELAY_TRY(act_grad_any(d.dt, dy->data, y->data, dz, db ? (float *)db->data : nullptr, partials, d.M, d.N, act, st));

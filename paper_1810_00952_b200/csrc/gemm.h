@@ -30,4 +30,11 @@ relay_status_t launch_gemm_tc(const GemmDesc &g, cudaStream_t st);
 bool gemm_tc2_eligible(const GemmDesc &g, int sms);
 relay_status_t launch_gemm_tc2(const GemmDesc &g, int sms, cudaStream_t st);
 
+// dense anchor / gradient group of a problem that fits one thread block: a single launch each (dense_small.cu)
+bool dense_small_eligible(int64_t M, int64_t K, int64_t N, int32_t dt);
+relay_status_t launch_dense_small_fwd(int32_t dt, const void *x, const void *w, const void *bias, int32_t bias_dt, void *y, int64_t M, int64_t K,
+                                      int64_t N, int act, cudaStream_t st);
+relay_status_t launch_dense_small_grad(int32_t dt, const void *x, const void *w, const void *y, const void *dy, void *dx, void *dw, float *db,
+                                       int64_t M, int64_t K, int64_t N, int act, cudaStream_t st);
+
 }  // namespace relay
