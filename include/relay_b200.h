@@ -406,6 +406,15 @@ relay_status_t relay_poll_status(void *stream);
  * It shows a caller that an expired wait in any kernel of this library is reported rather than hung on. */
 relay_status_t relay_debug_expire_wait(int32_t limit_us, void *stream);
 
+/* Self-test of the bounds-check build (no counterpart in the paper).  The library can be built with
+ * -DRELAY_BOUNDS_CHECK (librelay_b200_check.so): the memory-bound and SIMT kernels then look every global address they
+ * compute up in the ranges of the call's tensors and workspace, skip an access that lies outside and record it in the
+ * device error word, so that relay_poll_status() returns RELAY_ERR_CUDA ("bounds check failed") instead of the kernel
+ * faulting.  This call registers one 16-byte range and has a kernel look up (not access) the address just behind it:
+ * in the check build the next relay_poll_status() reports the failed check; in the ordinary build the call returns
+ * RELAY_ERR_UNSUPPORTED. */
+relay_status_t relay_debug_bounds_probe(void *stream);
+
 /* Host-only view of how the two-SM contraction kernel cuts an M x N output (contraction length K) into work units
  * for `sms` SMs (no counterpart in the paper; touches no GPU): fills units[i] = row block (256 rows) |
  * first 128-column chunk << 12 | width in chunks << 24, in the order the kernel hands them to its SM pairs

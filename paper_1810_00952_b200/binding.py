@@ -13,7 +13,9 @@ from typing import Optional, Sequence
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "librelay_b200.so")
+# RELAY_B200_LIB names another build of the same library (the bounds-check variant librelay_b200_check.so)
+LIB_PATH = os.environ.get("RELAY_B200_LIB") or os.path.join(_HERE, "librelay_b200.so")
+CHECK_LIB_PATH = os.path.join(_HERE, "librelay_b200_check.so")
 
 MAX_RANK = 6
 F32, BF16, I32, I64, BOOL = 0, 1, 2, 3, 4
@@ -380,6 +382,10 @@ def relay_last_error() -> str:
 
 def relay_poll_status():
     _check(lib().relay_poll_status(_stream()))
+
+
+def relay_debug_bounds_probe():
+    _check(lib().relay_debug_bounds_probe(_stream()))
 
 
 def relay_debug_expire_wait(limit_us: int = 1000):

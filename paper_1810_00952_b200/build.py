@@ -26,21 +26,28 @@ def _deps_mtime() -> float:
     return max(os.path.getmtime(f) for f in files)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    os.makedirs(OBJ, exist_ok=True)
+CHECK_LIB = os.path.join(HERE, "librelay_b200_check.so")
+
+
+def build(force: bool = False, verbose: bool = False, check: bool = False) -> str:
+    """check=True builds the bounds-check variant (-DRELAY_BOUNDS_CHECK, see csrc/common.h) as librelay_b200_check.so."""
+    obj_dir = OBJ + ("_check" if check else "")
+    lib = CHECK_LIB if check else LIB
+    flags = FLAGS + (["-DRELAY_BOUNDS_CHECK"] if check else [])
+    os.makedirs(obj_dir, exist_ok=True)
     srcs = sorted(glob.glob(os.path.join(CSRC, "*.cu")))
     hdr_time = _deps_mtime()
     jobs = []
     objs = []
     for src in srcs:
-        obj = os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
+        obj = os.path.join(obj_dir, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
         if force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), hdr_time):
             jobs.append((src, obj))
 
     def compile_one(job):
         src, obj = job
-        cmd = [NVCC, *FLAGS, "-c", src, "-o", obj]
+        cmd = [NVCC, *flags, "-c", src, "-o", obj]
         r = subprocess.run(cmd, capture_output=True, text=True)
         log = obj[:-2] + ".log"
         with open(log, "w") as f:
@@ -53,13 +60,13 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if jobs:
         with ThreadPoolExecutor(max_workers=min(8, len(jobs))) as ex:
             list(ex.map(compile_one, jobs))
-    if jobs or force or not os.path.exists(LIB):
-        tmp = LIB + f".tmp{os.getpid()}"
+    if jobs or force or not os.path.exists(lib):
+        tmp = lib + f".tmp{os.getpid()}"
         cmd = [NVCC, "-shared", "-o", tmp, *objs, "-cudart", "static"]
         subprocess.check_call(cmd)
-        os.replace(tmp, LIB)
-    return LIB
+        os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose=True))
+    print(build(force="--force" in sys.argv, verbose=True, check="--check" in sys.argv))

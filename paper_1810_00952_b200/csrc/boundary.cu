@@ -199,8 +199,30 @@ relay_status_t relay_poll_status(void *stream)
     RELAY_TRY(check_launch("poll_exchange"));
     RELAY_CUDA(cudaMemcpyAsync(&v, w + 1, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
     RELAY_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    if (v == kErrBounds) return fail(RELAY_ERR_CUDA, "a device-side bounds check failed: a kernel computed an address outside the call's tensors (the access was skipped)");
     if (v != 0) return fail(RELAY_ERR_TIMEOUT, "a bounded device-side wait expired (code %d)", v);
     return RELAY_OK;
+}
+
+#ifdef RELAY_BOUNDS_CHECK
+__global__ void bounds_probe_kernel(const char *base) { (void)relay_in_bounds(base + 16, 16); }   // looks an address up; touches nothing
+#endif
+
+relay_status_t relay_debug_bounds_probe(void *stream)
+{
+    clear_error();
+#ifdef RELAY_BOUNDS_CHECK
+    int *w = device_error_word();
+    if (!w) return fail(RELAY_ERR_CUDA, "no device error word (no CUDA device?)");
+    BoundsReg br;
+    br.add(w, 16);                         // a 16-byte range; the probe asks for the 16 bytes behind it
+    RELAY_TRY(br.commit((cudaStream_t)stream));
+    bounds_probe_kernel<<<1, 1, 0, (cudaStream_t)stream>>>((const char *)w);
+    return check_launch("bounds_probe");
+#else
+    (void)stream;
+    return fail(RELAY_ERR_UNSUPPORTED, "this build of the library carries no bounds checks");
+#endif
 }
 
 relay_status_t relay_debug_expire_wait(int32_t limit_us, void *stream)

@@ -134,4 +134,52 @@ __device__ __forceinline__ void pdl_wait()
 // device-side error word (set by kernels whose bounded waits expire)
 int *device_error_word();  // device address of the word on the current device (nullptr on failure)
 
+// ---- bounds-check build (-DRELAY_BOUNDS_CHECK) -----------------------------------------------------
+// A debugging variant of the library.  A launch function registers the address ranges its kernel may touch (every
+// tensor of the call and the workspace); the kernels' global-memory access helpers look every address up, and an
+// access outside all ranges is SKIPPED (loads return zero) and recorded in the device error word, which
+// relay_poll_status reports.  Nothing traps.  The table is one __constant__ object per translation unit and is
+// rewritten by every registering launch, so calls that overlap on one device confuse it: the variant is for
+// single-stream test runs.  In the ordinary build all of this compiles to nothing.
+constexpr int kErrBounds = 6;
+#ifdef RELAY_BOUNDS_CHECK
+struct BoundsTable { int n; int *err; unsigned long long lo[16], hi[16]; };
+#ifdef __CUDACC__
+static __constant__ BoundsTable c_bounds;
+__device__ __forceinline__ bool relay_in_bounds(const void *p, size_t bytes)
+{
+    if (c_bounds.n == 0) return true;                    // this launch registered nothing
+    const unsigned long long a = (unsigned long long)p;
+    for (int i = 0; i < c_bounds.n; ++i)
+        if (a >= c_bounds.lo[i] && a + bytes <= c_bounds.hi[i]) return true;
+    if (c_bounds.err) atomicCAS(c_bounds.err, 0, kErrBounds);
+    return false;
+}
+struct BoundsReg {
+    BoundsTable t{};
+    void add(const void *p, size_t bytes)
+    {
+        if (!p || !bytes || t.n >= 16) return;
+        t.lo[t.n] = (unsigned long long)p; t.hi[t.n] = (unsigned long long)p + bytes; ++t.n;
+    }
+    void add(const relay_tensor_t *x) { if (x) add(x->data, nbytes(x)); }
+    relay_status_t commit(cudaStream_t st)
+    {
+        t.err = device_error_word();
+        RELAY_CUDA(cudaMemcpyToSymbolAsync(c_bounds, &t, sizeof t, 0, cudaMemcpyHostToDevice, st));
+        return RELAY_OK;
+    }
+};
+#endif
+#else
+#ifdef __CUDACC__
+__device__ __forceinline__ constexpr bool relay_in_bounds(const void *, size_t) { return true; }
+#endif
+struct BoundsReg {
+    void add(const void *, size_t) {}
+    void add(const relay_tensor_t *) {}
+    relay_status_t commit(cudaStream_t) { return RELAY_OK; }
+};
+#endif
+
 }  // namespace relay

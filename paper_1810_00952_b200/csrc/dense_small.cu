@@ -15,11 +15,13 @@ namespace {
 
 template <typename T> __device__ __forceinline__ float ld_f(const T *p, int64_t i)
 {
+    if (!relay_in_bounds(p + i, sizeof(T))) return 0.0f;
     if constexpr (sizeof(T) == 2) return __bfloat162float(p[i]);
     else return p[i];
 }
 template <typename T> __device__ __forceinline__ void st_f(T *p, int64_t i, float v)
 {
+    if (!relay_in_bounds(p + i, sizeof(T))) return;
     if constexpr (sizeof(T) == 2) p[i] = __float2bfloat16_rn(v);
     else p[i] = v;
 }
@@ -36,7 +38,8 @@ __device__ __forceinline__ void stage(const T *__restrict__ src, float *dst, int
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const int i4 = base + u * 256 + threadIdx.x;
-                if (i4 < n4) v[u] = reinterpret_cast<const float4 *>(src)[i4];
+                if (i4 < n4 && relay_in_bounds(reinterpret_cast<const float4 *>(src) + i4, 16)) v[u] = reinterpret_cast<const float4 *>(src)[i4];
+                else v[u] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
@@ -44,7 +47,7 @@ __device__ __forceinline__ void stage(const T *__restrict__ src, float *dst, int
                 if (i4 < n4) { dst[perm(4 * i4)] = v[u].x; dst[perm(4 * i4 + 1)] = v[u].y; dst[perm(4 * i4 + 2)] = v[u].z; dst[perm(4 * i4 + 3)] = v[u].w; }
             }
         }
-        for (int i = 4 * n4 + threadIdx.x; i < n; i += 256) dst[perm(i)] = src[i];
+        for (int i = 4 * n4 + threadIdx.x; i < n; i += 256) dst[perm(i)] = ld_f(src, i);
     } else {
         for (int i = threadIdx.x; i < n; i += 256) dst[perm(i)] = ld_f(src, i);
     }
@@ -77,7 +80,7 @@ __global__ void __launch_bounds__(256) dense_small_fwd_kernel(const T *__restric
     for (int o = threadIdx.x; o < M * N; o += 256) {
         const int m = o / N, n = o - m * N;
         float z = dot_runs(xs + m * K, 1, ws + n, N, K);
-        if (bias) z += bias_bf16 ? __bfloat162float(((const __nv_bfloat16 *)bias)[n]) : ((const float *)bias)[n];
+        if (bias) z += bias_bf16 ? ld_f((const __nv_bfloat16 *)bias, n) : ld_f((const float *)bias, n);
         st_f(y, o, act_fwd<FAST>(z, act));
     }
 }
@@ -120,7 +123,7 @@ __global__ void __launch_bounds__(256) dense_small_grad_kernel(const T *__restri
                 for (int m = m0; m < min(M, m0 + 16); ++m) part += dz[m * N + n];
                 acc.add(part);
             }
-            db[n] = (float)acc.value();
+            if (relay_in_bounds(db + n, 4)) db[n] = (float)acc.value();
         }
 }
 
@@ -138,7 +141,10 @@ bool dense_small_eligible(int64_t M, int64_t K, int64_t N, int32_t dt)
 relay_status_t launch_dense_small_fwd(int32_t dt, const void *x, const void *w, const void *bias, int32_t bias_dt, void *y, int64_t M, int64_t K,
                                       int64_t N, int act, cudaStream_t st)
 {
-    const size_t smem = (size_t)(M * K + K * N) * 4;
+    const size_t smem = (size_t)(M * K + K * N) * 4, es = dtype_size(dt);
+    BoundsReg br;
+    br.add(x, (size_t)M * K * es); br.add(w, (size_t)K * N * es); br.add(y, (size_t)M * N * es); br.add(bias, (size_t)N * dtype_size(bias_dt));
+    RELAY_TRY(br.commit(st));
     if (dt == RELAY_F32)
         RELAY_CUDA(launch_pdl(dense_small_fwd_kernel<float, false>, dim3(1), dim3(256), smem, st, (const float *)x, (const float *)w, bias,
                               (int)(bias_dt == RELAY_BF16), (float *)y, (int)M, (int)K, (int)N, act));
@@ -151,7 +157,11 @@ relay_status_t launch_dense_small_fwd(int32_t dt, const void *x, const void *w, 
 relay_status_t launch_dense_small_grad(int32_t dt, const void *x, const void *w, const void *y, const void *dy, void *dx, void *dw, float *db,
                                        int64_t M, int64_t K, int64_t N, int act, cudaStream_t st)
 {
-    const size_t smem = (size_t)(M * K + K * (N + 1) + 2 * M * N) * 4;
+    const size_t smem = (size_t)(M * K + K * (N + 1) + 2 * M * N) * 4, es = dtype_size(dt);
+    BoundsReg br;
+    br.add(x, (size_t)M * K * es); br.add(w, (size_t)K * N * es); br.add(y, (size_t)M * N * es); br.add(dy, (size_t)M * N * es);
+    br.add(dx, (size_t)M * K * es); br.add(dw, (size_t)K * N * es); br.add(db, (size_t)N * 4);
+    RELAY_TRY(br.commit(st));
     if (dt == RELAY_F32)
         RELAY_CUDA(launch_pdl(dense_small_grad_kernel<float>, dim3(1), dim3(256), smem, st, (const float *)x, (const float *)w, (const float *)y,
                               (const float *)dy, (float *)dx, (float *)dw, db, (int)M, (int)K, (int)N, act));

@@ -128,7 +128,8 @@ __global__ void __launch_bounds__(kTX *kTY, Body::NIN >= 4 ? 2 : 3) ewise2d_kern
 #pragma unroll
                     for (int j = 0; j < kTY; ++j) s += sm[j][tx * V + v];
                     if constexpr (CL > 1) mine[k][tx * V + v] = active ? s : 0.0f;
-                    else if (active && A.partial[k] != nullptr) A.partial[k][(int64_t)blockIdx.y * A.cols + col0 + v] = s;
+                    else if (active && A.partial[k] != nullptr && relay_in_bounds(&A.partial[k][(int64_t)blockIdx.y * A.cols + col0 + v], 4))
+                        A.partial[k][(int64_t)blockIdx.y * A.cols + col0 + v] = s;
                 }
             }
             __syncthreads();
@@ -154,7 +155,7 @@ __global__ void __launch_bounds__(kTX *kTY, Body::NIN >= 4 ? 2 : 3) ewise2d_kern
                         asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
                         s += v;
                     }
-                    if (col < A.cols) A.final[k][col] = s * A.scale[k];
+                    if (col < A.cols && relay_in_bounds(&A.final[k][col], 4)) A.final[k][col] = s * A.scale[k];
                 }
             }
             // no block may exit (and give up its shared memory) while another still reads it
@@ -178,14 +179,15 @@ __global__ void __launch_bounds__(32 * TY) colsum_finalize_kernel(const float *_
     const float *p = partial + (size_t)blockIdx.y * n_slices * cols;
     float s = 0.0f;
     if (c < cols)
-        for (int j = ty; j < n_slices; j += TY) s += p[(int64_t)j * cols + c];
+        for (int j = ty; j < n_slices; j += TY)
+            if (relay_in_bounds(&p[(int64_t)j * cols + c], 4)) s += p[(int64_t)j * cols + c];
     sm[ty][tx] = s;
     __syncthreads();
     if (ty == 0 && c < cols) {
         float t = 0.0f;
 #pragma unroll
         for (int j = 0; j < TY; ++j) t += sm[j][tx];
-        outs.out[blockIdx.y][c] = t * outs.scale[blockIdx.y];
+        if (relay_in_bounds(&outs.out[blockIdx.y][c], 4)) outs.out[blockIdx.y][c] = t * outs.scale[blockIdx.y];
     }
 }
 
@@ -263,8 +265,8 @@ __global__ void __launch_bounds__(256) rowreduce_kernel(const T *__restrict__ in
         }
     }
     if (lane == 0) {
-        if (RED == RELAY_RED_ARGMAX) ((int64_t *)out)[row] = pos;
-        else ((float *)out)[row] = best * scale;
+        if (RED == RELAY_RED_ARGMAX) { if (relay_in_bounds((int64_t *)out + row, 8)) ((int64_t *)out)[row] = pos; }
+        else if (relay_in_bounds((float *)out + row, 4)) ((float *)out)[row] = best * scale;
     }
 }
 
@@ -351,8 +353,8 @@ __global__ void __launch_bounds__(256) reduce_generic_kernel(const DevProgram P,
         }
     }
     if (live && lane_in_group == 0) {
-        if (R.red_op == RELAY_RED_ARGMAX) ((int64_t *)R.out)[kept] = pos;
-        else ((float *)R.out)[kept] = best * R.scale;
+        if (R.red_op == RELAY_RED_ARGMAX) { if (relay_in_bounds((int64_t *)R.out + kept, 8)) ((int64_t *)R.out)[kept] = pos; }
+        else if (relay_in_bounds((float *)R.out + kept, 4)) ((float *)R.out)[kept] = best * R.scale;
     }
 }
 
@@ -539,6 +541,10 @@ relay_status_t launch_colsum_finalize_n(const float *partial, int n_slices, int6
 {
     FinalizeOuts fo{};
     for (int k = 0; k < n_out; ++k) { fo.out[k] = out[k]; fo.scale[k] = scale ? scale[k] : 1.0f; }
+    BoundsReg br;
+    br.add(partial, (size_t)n_out * n_slices * cols * sizeof(float));
+    for (int k = 0; k < n_out; ++k) br.add(out[k], (size_t)cols * sizeof(float));
+    RELAY_TRY(br.commit(st));
     const dim3 grid((unsigned)((cols + 31) / 32), (unsigned)n_out);
     if (n_slices > 256) RELAY_CUDA(launch_pdl(colsum_finalize_kernel<32>, grid, dim3(32, 32), 0, st, partial, n_slices, cols, fo));
     else RELAY_CUDA(launch_pdl(colsum_finalize_kernel<8>, grid, dim3(32, 8), 0, st, partial, n_slices, cols, fo));
@@ -555,6 +561,11 @@ relay_status_t launch_colsum_finalize(const float *partial, int n_slices, int64_
 relay_status_t launch_act_grad(int32_t storage, const void *dy, const void *y, void *dz, float *db, float *partials,
                                int64_t rows, int64_t cols, int act, cudaStream_t st)
 {
+    const size_t esz = storage == RELAY_BF16 ? 2 : 4;
+    BoundsReg br;
+    br.add(dy, (size_t)rows * cols * esz); br.add(y, (size_t)rows * cols * esz); br.add(dz, (size_t)rows * cols * esz);
+    br.add(db, (size_t)cols * 4); br.add(partials, db ? (size_t)colsum_slices(rows, cols, storage) * cols * 4 : 0);
+    RELAY_TRY(br.commit(st));
     Args2D<2, 2> A{};
     A.in[0] = dy; A.in[1] = y;
     A.out[0] = dz; A.out[1] = nullptr;
@@ -568,6 +579,9 @@ relay_status_t launch_act_grad(int32_t storage, const void *dy, const void *y, v
 
 relay_status_t launch_colsum_bf16(const void *in, int64_t rows, int64_t cols, float *partials, float *out, cudaStream_t st)
 {
+    BoundsReg br;
+    br.add(in, (size_t)rows * cols * 2); br.add(out, (size_t)cols * 4); br.add(partials, (size_t)colsum_slices(rows, cols, RELAY_BF16) * cols * 4);
+    RELAY_TRY(br.commit(st));
     Args2D<1, 1> A{};
     A.in[0] = in; A.out[0] = nullptr; A.partial[0] = partials;
     A.rows = rows; A.cols = cols; A.aux = 0;
@@ -622,6 +636,10 @@ extern "C" relay_status_t relay_fused_ewise(const relay_ewise_prog_t *prog, cons
     RELAY_TRY(check_no_overlap(outputs, n_out, inputs, n_in));
     if (tp.total == 0) return RELAY_OK;
     cudaStream_t st = (cudaStream_t)stream;
+    BoundsReg br;
+    for (int i = 0; i < n_in; ++i) br.add(inputs[i]);
+    for (int k = 0; k < n_out; ++k) br.add(outputs[k]);
+    RELAY_TRY(br.commit(st));
 
     // pre-compiled body?
     View2D v = view2d(tp);
@@ -774,6 +792,11 @@ extern "C" relay_status_t relay_fused_reduce(const relay_ewise_prog_t *prog, con
     if (tp.total == 0) return RELAY_OK;
     cudaStream_t st = (cudaStream_t)stream;
     const View2D &v = pl.v;
+    BoundsReg br;
+    for (int i = 0; i < n_in; ++i) br.add(inputs[i]);
+    for (int k = 0; k < n_out; ++k) br.add(outputs[k]);
+    br.add(ws, pl.ws_need);
+    RELAY_TRY(br.commit(st));
 
     if (pl.fast_grad) {
         Args2D<4, 3> A{};

@@ -8,6 +8,7 @@
 #include <cstdint>
 
 #include "../../include/relay_b200.h"
+#include "common.h"
 
 namespace relay {
 
@@ -89,11 +90,13 @@ __device__ __forceinline__ uint4 pack(const float (&f)[4])
 __device__ __forceinline__ uint4 ld_stream(const void *p)
 {
     uint4 r;
+    if (!relay_in_bounds(p, 16)) return make_uint4(0, 0, 0, 0);
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
     return r;
 }
 __device__ __forceinline__ void st_stream(void *p, const uint4 &r)
 {
+    if (!relay_in_bounds(p, 16)) return;
     asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(r.x), "r"(r.y), "r"(r.z), "r"(r.w) : "memory");
 }
 
@@ -107,6 +110,8 @@ __device__ __forceinline__ Val load_value(const void *p, int64_t i, int dt)
 {
     Val v;
     v.i = 0;
+    const size_t esz = dt == RELAY_BF16 ? 2 : dt == RELAY_I64 ? 8 : dt == RELAY_BOOL ? 1 : 4;
+    if (!relay_in_bounds((const char *)p + i * esz, esz)) return v;
     switch (dt) {
     case RELAY_F32: v.f = ((const float *)p)[i]; break;
     case RELAY_BF16: v.f = __bfloat162float(((const __nv_bfloat16 *)p)[i]); break;
@@ -118,6 +123,8 @@ __device__ __forceinline__ Val load_value(const void *p, int64_t i, int dt)
 }
 __device__ __forceinline__ void store_value(void *p, int64_t i, int dt, Val v)
 {
+    const size_t esz = dt == RELAY_BF16 ? 2 : dt == RELAY_I64 ? 8 : dt == RELAY_BOOL ? 1 : 4;
+    if (!relay_in_bounds((const char *)p + i * esz, esz)) return;
     switch (dt) {
     case RELAY_F32: ((float *)p)[i] = v.f; break;
     case RELAY_BF16: ((__nv_bfloat16 *)p)[i] = __float2bfloat16_rn(v.f); break;

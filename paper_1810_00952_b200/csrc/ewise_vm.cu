@@ -121,7 +121,7 @@ template <int N> __device__ __forceinline__ void vm_store_run(void *out, int dt,
         if constexpr (N == 8) {
             st_stream((__nv_bfloat16 *)out + at, make_uint4(pack2(f[0], f[1]), pack2(f[2], f[3]), pack2(f[4], f[5]), pack2(f[6], f[7])));
         } else {
-            *reinterpret_cast<uint2 *>((__nv_bfloat16 *)out + at) = make_uint2(pack2(f[0], f[1]), pack2(f[2], f[3]));
+            if (relay_in_bounds((__nv_bfloat16 *)out + at, 8)) *reinterpret_cast<uint2 *>((__nv_bfloat16 *)out + at) = make_uint2(pack2(f[0], f[1]), pack2(f[2], f[3]));
         }
     } else {   // bool: one byte per element
         uint32_t w[N / 4];
@@ -129,6 +129,7 @@ template <int N> __device__ __forceinline__ void vm_store_run(void *out, int dt,
         for (int q = 0; q < N / 4; ++q)
             w[q] = (f[4 * q] != 0.0f ? 1u : 0u) | (f[4 * q + 1] != 0.0f ? 0x100u : 0u) | (f[4 * q + 2] != 0.0f ? 0x10000u : 0u) |
                    (f[4 * q + 3] != 0.0f ? 0x1000000u : 0u);
+        if (!relay_in_bounds((uint8_t *)out + at, N)) return;
         if constexpr (N == 8) *reinterpret_cast<uint2 *>((uint8_t *)out + at) = make_uint2(w[0], w[1]);
         else *reinterpret_cast<uint32_t *>((uint8_t *)out + at) = w[0];
     }
@@ -210,8 +211,8 @@ ewise_vm_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constant__
     for (int g = 0; g < A.n_fixed; ++g) {
         const T *p = (const T *)A.fixed_ptr[g];
         T val = T(0.0f);
-        if (A.fixed_scalar[g]) val = p[0];
-        else if (col0 + tid < A.cols) val = p[col0 + tid];
+        if (A.fixed_scalar[g]) { if (relay_in_bounds(p, sizeof(T))) val = p[0]; }
+        else if (col0 + tid < A.cols && relay_in_bounds(p + col0 + tid, sizeof(T))) val = p[col0 + tid];
         reinterpret_cast<T *>(fixed)[g * VM_COLS + tid] = val;
     }
     if (tid < A.n_const * 4) reinterpret_cast<float *>(slots + A.n_temp * 4 * VM_THREADS * 16)[tid] = A.literal[tid >> 2];
@@ -384,7 +385,7 @@ ewise_vm_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constant__
                 float t = 0.0f;
 #pragma unroll
                 for (int j = 0; j < VM_TY; ++j) t += sm[j][tid];
-                A.partial[k][(int64_t)blockIdx.y * A.cols + col0 + tid] = t;
+                if (relay_in_bounds(&A.partial[k][(int64_t)blockIdx.y * A.cols + col0 + tid], 4)) A.partial[k][(int64_t)blockIdx.y * A.cols + col0 + tid] = t;
             }
             __syncthreads();
         }
@@ -634,6 +635,11 @@ relay_status_t vm_launch(const VmPlan &plan, const View2D &v, const relay_tensor
     A.code = P.code;
     A.err = device_error_word();
     if (!A.err) return fail(RELAY_ERR_CUDA, "no device error word");
+    BoundsReg br;
+    for (int i = 0; i < n_in; ++i) br.add(inputs[i]);
+    for (int k = 0; k < n_out; ++k) br.add(outputs[k]);
+    br.add(partials, (size_t)P.n_sum * n_slices * v.cols * sizeof(float));
+    RELAY_TRY(br.commit(st));
     CUtensorMap tm[VM_MAXFULL];
     memset(tm, 0, sizeof tm);
     for (int i = 0; i < n_in; ++i) {

@@ -46,14 +46,14 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmDesc g)
             const int e = tid + i * 256;
             const int mm = a_k_fast ? e / BK : e % BM, kk = a_k_fast ? e % BK : e / BM;
             const int64_t m = m0 + mm, k = k0 + kk;
-            ra[i] = (m < g.M && k < g.K) ? to_f<TIN>(A[m * g.a_sm + k * g.a_sk]) : 0.0f;
+            ra[i] = (m < g.M && k < g.K && relay_in_bounds(&A[m * g.a_sm + k * g.a_sk], sizeof(TIN))) ? to_f<TIN>(A[m * g.a_sm + k * g.a_sk]) : 0.0f;
         }
 #pragma unroll
         for (int i = 0; i < B_LD; ++i) {
             const int e = tid + i * 256;
             const int nn = b_n_fast ? e % BN : e / BK, kk = b_n_fast ? e / BN : e % BK;
             const int64_t n = n0 + nn, k = k0 + kk;
-            rb[i] = (n < g.N && k < g.K) ? to_f<TIN>(B[k * g.b_sk + n * g.b_sn]) : 0.0f;
+            rb[i] = (n < g.N && k < g.K && relay_in_bounds(&B[k * g.b_sk + n * g.b_sn], sizeof(TIN))) ? to_f<TIN>(B[k * g.b_sk + n * g.b_sn]) : 0.0f;
         }
     };
     load_tiles(0);
@@ -120,7 +120,7 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmDesc g)
 #pragma unroll
         for (int j = 0; j < TN; ++j) {
             int64_t n = n0 + tn + j;
-            if (n >= g.N) continue;
+            if (n >= g.N || !relay_in_bounds(&C[m * g.ldc + n], sizeof(TOUT))) continue;
             float z;
             const float bv = !g.bias ? 0.0f : g.bias_dtype == RELAY_BF16 ? __bfloat162float(((const __nv_bfloat16 *)g.bias)[n]) : ((const float *)g.bias)[n];
             if constexpr (F64) z = (float)(acc[i][j].value() + (double)bv);
@@ -148,6 +148,17 @@ static relay_status_t launch_tile(const GemmDesc &g, cudaStream_t st)
 relay_status_t launch_gemm_simt(const GemmDesc &g, cudaStream_t st)
 {
     if (g.M == 0 || g.N == 0) return RELAY_OK;
+    {
+        const size_t ein = dtype_size(g.in_dtype), eout = dtype_size(g.out_dtype);
+        BoundsReg br;
+        if (g.K > 0) {
+            br.add(g.a, (size_t)((g.M - 1) * g.a_sm + (g.K - 1) * g.a_sk + 1) * ein);
+            br.add(g.b, (size_t)((g.K - 1) * g.b_sk + (g.N - 1) * g.b_sn + 1) * ein);
+        }
+        br.add(g.c, (size_t)((g.M - 1) * g.ldc + g.N) * eout);
+        br.add(g.bias, (size_t)g.N * dtype_size(g.bias_dtype));
+        RELAY_TRY(br.commit(st));
+    }
     // The largest tile whose grid still gives every SM a block: with few warps on an SM a block's time goes to waiting
     // for its own shared-memory reads, so while SMs are idle more and lighter blocks finish sooner.
     auto tiles = [&](int bm, int bn) { return ((g.M + bm - 1) / bm) * ((g.N + bn - 1) / bn); };

@@ -24,3 +24,10 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_runtest_teardown(item, nextitem):
+    """Against the bounds-check build (RELAY_B200_LIB set) every GPU test ends with a poll of the device error word."""
+    if os.environ.get("RELAY_B200_LIB") and "gpu" in item.keywords:
+        from paper_1810_00952_b200 import binding as B
+        B.relay_poll_status()
