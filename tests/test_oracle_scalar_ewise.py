@@ -249,6 +249,40 @@ def test_cfg2_gradient_program_against_finite_differences():
     assert np.all(np.abs(dx) >= np.abs(dout) - 1e-15) and np.all(np.abs(dx) <= 2.5 * np.abs(dout))
 
 
+def test_sigmoid_product_relu_programs_against_numpy_and_finite_differences():
+    """The second pair of benchmark programs (out = sigmoid(x*y) + relu(z), z constant down the rows): the forward program
+    against its closed form, the gradient program (dx, dy unreduced, dz as a column sum) against central differences of
+    L = sum(dout * out) through the forward program, away from the kink of relu."""
+    rng = np.random.default_rng(16)
+    R, C = 5, 4
+    x, y = rng.standard_normal((R, C)), rng.standard_normal((R, C))
+    z = rng.standard_normal(C); z[np.abs(z) < 1e-2] = 0.5
+    dout = rng.standard_normal((R, C))
+    F64 = 5
+    fwd, fo = P.sigmoid_product_relu_fwd(F64, F64)
+    grd, (dx_id, dy_id, dz_id) = P.sigmoid_product_relu_grad(F64, F64)
+    (o,) = oracle.ewise(fwd.arrays(), [x, y, z], fo)
+    assert np.allclose(o, 1.0 / (1.0 + np.exp(-x * y)) + np.maximum(z, 0.0)[None, :], rtol=0, atol=1e-15)
+
+    def loss(x_, y_, z_):
+        (o_,) = oracle.ewise(fwd.arrays(), [x_, y_, z_], fo)
+        return float(np.sum(dout * o_))
+
+    dx, dy, dz = oracle.reduce(grd.arrays(), [dout, x, y, z], [
+        (dx_id, oracle.RED_NONE, (), False, F64), (dy_id, oracle.RED_NONE, (), False, F64), (dz_id, oracle.RED_SUM, (0,), False, F64)])
+    assert dx.shape == (R, C) and dy.shape == (R, C) and dz.shape == (C,)
+    h = 1e-5
+    for arr, grad in ((x, dx), (y, dy), (z, dz)):
+        for idx in np.ndindex(arr.shape):
+            keep = arr[idx]
+            arr[idx] = keep + h; lp = loss(x, y, z)
+            arr[idx] = keep - h; lm = loss(x, y, z)
+            arr[idx] = keep
+            fd = (lp - lm) / (2 * h)
+            assert abs(fd - grad[idx]) <= 1e-7 * max(1.0, abs(fd)), (idx, fd, grad[idx])
+    assert np.all(dz[z < 0] == 0.0)                       # relu'(z) = 0 below the kink
+
+
 # ---------------------------------------------------------------------------------------------
 # reduce group
 # ---------------------------------------------------------------------------------------------
