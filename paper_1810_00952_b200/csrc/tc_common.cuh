@@ -12,7 +12,7 @@ namespace relay {
 namespace tc {
 
 // ---- error codes written to the device error word when a bounded wait expires ---------------------
-enum : int { ERR_WAIT_FULL = 1, ERR_WAIT_EMPTY = 2, ERR_WAIT_TMEM_FULL = 3, ERR_WAIT_TMEM_EMPTY = 4, ERR_WAIT_STEP = 5 };
+enum : int { ERR_WAIT_FULL = 1, ERR_WAIT_EMPTY = 2, ERR_WAIT_TMEM_FULL = 3, ERR_WAIT_TMEM_EMPTY = 4, ERR_WAIT_STEP = 5, ERR_WAIT_EXCHANGE = 7 };   // 6: a failed bounds check (common.h)
 
 constexpr long long kWaitLimitCycles = 4000000000LL;  // about two seconds at the boost clock
 

@@ -60,9 +60,13 @@ def compare(got, want, keys=("dx", "dw_ih", "dw_hh", "db", "dh0", "dc0")):
             assert_bf16(got[k], want[k], stored_bf16=k in ("dx", "dw_ih", "dw_hh"), what=k)
 
 
-# persistent tensor-core route (H a multiple of 64), one or several batch groups; per-step route otherwise
+# cluster kernel (H a multiple of 64, B <= 128), per-step kernels otherwise.  The cluster kernel's variants: one, two or four
+# MMA issuers (H / 64 odd, even, a multiple of four); a stage in one copy (rows of a group a multiple of 8) or tile by tile;
+# 16 to 64 accumulator columns (rows of a group rounded up to 16), one or two (row, unit) pairs per thread; a last group
+# with fewer rows than the others
 @pytest.mark.parametrize("T,Bn,In,H", [(1, 8, 64, 64), (3, 8, 64, 64), (5, 40, 96, 128), (4, 16, 32, 20), (6, 3, 24, 72), (3, 16, 64, 1024),
-                                       (2, 130, 64, 64), (2, 96, 64, 1024)])     # the last: 48 rows a group, all four lane quarters of M = 64
+                                       (2, 130, 64, 64), (2, 96, 64, 1024), (3, 20, 32, 128), (3, 24, 64, 192), (2, 100, 64, 1024),
+                                       (2, 128, 32, 1024), (3, 44, 64, 256), (4, 20, 64, 512)])
 def test_gradient_program(T, Bn, In, H):
     t, dh_all, dc_fin = case(T, Bn, In, H, salt=T * 100 + H)
     d = {k: v.to(DEV) for k, v in t.items()}
