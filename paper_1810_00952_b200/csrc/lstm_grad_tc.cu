@@ -96,12 +96,6 @@ __device__ __forceinline__ void st_async_v4(uint32_t addr, uint32_t bar, float a
     asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];"
                  ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d), "r"(bar) : "memory");
 }
-__device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *m, uint64_t *bar, int c0, int c1, int c2)
-{
-    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-                 ::"r"(tc::smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(tc::smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
-                 : "memory");
-}
 __device__ __forceinline__ void tmem_ld_32x4(uint32_t taddr, uint32_t (&r)[4])
 {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(taddr) : "memory");
@@ -302,7 +296,7 @@ lstm_grad_cluster_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                 uint8_t *dst = a_s + (size_t)st * p.n_iss * p.tile_stride;
                 if (tc::elect_one()) {
                     tc::mbar_expect_tx(&full[st], stage_bytes);
-                    for (int i = 0; i < p.n_iss; i += p.box_kb) tma_load_3d(dst + (size_t)i * p.tile_stride, &tm_dz, &full[st], 0, row0, kb0 + kb + i);
+                    for (int i = 0; i < p.n_iss; i += p.box_kb) tc::tma_load_3d(dst + (size_t)i * p.tile_stride, &tm_dz, &full[st], 0, row0, kb0 + kb + i);
                 }
                 __syncwarp();
                 if (++st == p.n_stages) { st = 0; phase ^= 1; }
