@@ -380,13 +380,20 @@ class Workload:
             with tm.region("cfg2.grad"):
                 B.relay_fused_reduce(self.grad_prog.arrays(), [d["dout"], d["x"], d["a"], d["b"]], self.grad_specs,
                                      [o["dx"], o["da"], o["db"]], ws)
-            self.flush_l2()
-            with tm.region("a6.vm_fwd"):
-                B.relay_fused_ewise(self.vm_fwd.arrays(), [d["x"], d["dout"], d["a"]], self.vm_fwd_outs, [self.vm_out["out"]], ws)
-            self.flush_l2()
-            with tm.region("a7.vm_grad"):
-                B.relay_fused_reduce(self.vm_grad.arrays(), [d["dout"], d["x"], o["out"], d["a"]], self.vm_grad_specs,
-                                     [self.vm_out["dx"], self.vm_out["dy"], self.vm_out["dz"]], ws)
+            # a program without a pre-compiled body: as the library runs it (a body compiled at run time where the compiler
+            # library is present), then on the in-kernel interpreter (the route without that library)
+            for tag, compiled in (("jit", True), ("vm", False)):
+                if compiled and B.relay_debug_jit_compiled() < 0:
+                    continue
+                before = B.relay_debug_set_jit(compiled)
+                self.flush_l2()
+                with tm.region(f"a6.{tag}_fwd"):
+                    B.relay_fused_ewise(self.vm_fwd.arrays(), [d["x"], d["dout"], d["a"]], self.vm_fwd_outs, [self.vm_out["out"]], ws)
+                self.flush_l2()
+                with tm.region(f"a7.{tag}_grad"):
+                    B.relay_fused_reduce(self.vm_grad.arrays(), [d["dout"], d["x"], o["out"], d["a"]], self.vm_grad_specs,
+                                         [self.vm_out["dx"], self.vm_out["dy"], self.vm_out["dz"]], ws)
+                B.relay_debug_set_jit(before)
             ra = self.red_prog.arrays()
             # four launches back to back, each on another 8192 x 8192 tensor (134 MB each, so none is still in L2)
             red_ins = [d["x"], d["dout"], o["out"], o["dx"]]
@@ -479,7 +486,8 @@ class Workload:
             r, c = self.host["cfg2"]["x"].shape
             w["cfg2.fwd"] = dict(bytes=2 * r * c * 2 + 2 * c * 2)
             w["cfg2.grad"] = dict(bytes=3 * r * c * 2 + 2 * c * 2 + 2 * c * 4)
-            w["a6.vm_fwd"] = dict(bytes=3 * r * c * 2 + c * 2); w["a7.vm_grad"] = dict(bytes=5 * r * c * 2 + c * 2 + c * 4)
+            for tag in ("jit", "vm"):
+                w[f"a6.{tag}_fwd"] = dict(bytes=3 * r * c * 2 + c * 2); w[f"a7.{tag}_grad"] = dict(bytes=5 * r * c * 2 + c * 2 + c * 4)
             w["a8.sum1"] = dict(bytes=r * c * 2 + r * 4); w["a8.max1"] = dict(bytes=r * c * 2 + r * 4)
             w["a8.arg1"] = dict(bytes=r * c * 2 + r * 8); w["a8.sum0"] = dict(bytes=r * c * 2 + c * 4)
         if "cfg3" in self.groups:
@@ -756,8 +764,10 @@ def main():
             a = table[key]["gbs"]
             rooflines[name] = {"bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": a / peaks["hbm_gbs"],
                                "traffic": traffic_of(key), "peak_source": peaks["source"] + " (of measured)"}
-    for key, name in (("a6.vm_fwd", "ewise_vm_kernel, out = sigmoid(x*y) + relu(z) (8192x8192 bf16, interpreted stack program)"),
-                      ("a7.vm_grad", "ewise_vm_kernel + finalize, gradient group of the same (dx, dy, column sum dz)"),
+    for key, name in (("a6.jit_fwd", "relay_jit_kernel, out = sigmoid(x*y) + relu(z) (8192x8192 bf16, body compiled at run time)"),
+                      ("a7.jit_grad", "relay_jit_kernel + finalize, gradient group of the same (dx, dy, column sum dz)"),
+                      ("a6.vm_fwd", "ewise_vm_kernel, the same forward program on the in-kernel interpreter (run-time compiler switched off)"),
+                      ("a7.vm_grad", "ewise_vm_kernel + finalize, the same gradient group on the interpreter"),
                       ("a8.sum1", "rowreduce_kernel<sum> (8192x8192 bf16 over the last axis)"),
                       ("a8.max1", "rowreduce_kernel<max> (8192x8192 bf16 over the last axis)"),
                       ("a8.arg1", "rowreduce_kernel<argmax> (8192x8192 bf16 over the last axis, int64 indices)"),
@@ -893,7 +903,7 @@ def main():
                            + ", then softmax cross-entropy loss / loss+partial on 8192x8192 bf16, SGD on three 4096^2 bf16 matrices and 2x2 max pooling"
                            + " forward + gradient on 32x256x56x56 bf16, one fp32 LeNet training step (batch 64) eager and replayed from a"
                            + " CUDA graph, the cfg4 conv with NHWC-tagged tensors; cfg1 is also replayed from a CUDA graph",
-                           "value_covers": "dense + conv2d groups (cfg3 + cfg4) FLOPs / their device time; hbm_gbs covers cfg2 (the configuration's own two groups); the programs on the vectorised evaluator (a6.vm_fwd, a7.vm_grad) and the standalone reductions (a8.*) are reported per group",
+                           "value_covers": "dense + conv2d groups (cfg3 + cfg4) FLOPs / their device time; hbm_gbs covers cfg2 (the configuration's own two groups); a program without a pre-compiled body (a6.jit_fwd, a7.jit_grad: compiled at run time; a6.vm_fwd, a7.vm_grad: interpreted) and the standalone reductions (a8.*) are reported per group",
                            "groups": groups, "l2": "1 GiB streamed through L2 between groups (flush with clean lines); cfg2 inputs also exceed L2; the standalone reductions and "
                                  "the pooling kernels are timed as four back-to-back launches on four different sets of tensors (per-launch time = region / 4)",
                            "replicas": world},

@@ -415,6 +415,23 @@ relay_status_t relay_debug_expire_wait(int32_t limit_us, void *stream);
  * RELAY_ERR_UNSUPPORTED. */
 relay_status_t relay_debug_bounds_probe(void *stream);
 
+/* Run-time compiled bodies (Section 4.1: an operator group is fused into ONE kernel generated for that group).  A fused
+ * elementwise or elementwise + column-sum group over the collapsed 2-D view that has no pre-compiled body is written out
+ * as the per-element body of a kernel, compiled for this GPU by the NVRTC library when that library can be loaded at run
+ * time, cached for the life of the process (first call of a new program: some hundred milliseconds on the host), and
+ * launched like any other kernel; without the library, in the bounds-check build, or when switched off here, the same
+ * groups run on the library's in-kernel interpreter.  relay_debug_set_jit switches the compiled bodies on (non-zero,
+ * the default) or off for the process and returns the previous setting; relay_debug_jit_compiled returns how many
+ * bodies have been compiled so far, -1 when no run-time compiler is available.  Neither touches the GPU. */
+int32_t relay_debug_set_jit(int32_t enabled);
+int32_t relay_debug_jit_compiled(void);
+/* Host only (needs no GPU): generates the source of the body that would be compiled at run time for this group and
+ * compiles it for sm_100a.  Returns 1 if it compiled (its text, NUL-terminated and cut to `cap` bytes, is copied to `src`
+ * when that is not NULL), 0 if the group does not run on that tier, -1 without a run-time compiler, -2 if the source did
+ * not compile (relay_last_error() has the compiler's messages), -3 if the group does not type-check. */
+int32_t relay_debug_jit_compile(const relay_ewise_prog_t *prog, const relay_tensor_t *const *inputs, int32_t n_in,
+                                const relay_out_spec_t *specs, int32_t n_out, char *src, size_t cap);
+
 /* Host-only view of how the two-SM contraction kernel cuts an M x N output (contraction length K) into work units
  * for `sms` SMs (no counterpart in the paper; touches no GPU): fills units[i] = row block (256 rows) |
  * first 128-column chunk << 12 | width in chunks << 24, in the order the kernel hands them to its SM pairs

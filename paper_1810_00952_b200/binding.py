@@ -313,6 +313,22 @@ def relay_debug_group_route(prog: Optional[dict], inputs, specs) -> int:
     return r
 
 
+def relay_debug_jit_compile(prog: Optional[dict], inputs, specs, want_source: bool = False):
+    """Host only: generates the body that would be compiled at run time for this group and compiles it for sm_100a.
+    Returns the library's code (1 compiled, 0 not on that tier, -1 no run-time compiler), with the source text if asked;
+    raises on a compile error or an ill-typed group."""
+    p = make_prog(prog) if prog is not None else None
+    ins = [desc(t) for t in inputs]
+    sp = (OutSpec * max(len(specs), 1))(*[OutSpec(*s) for s in specs])
+    cap = 1 << 16
+    buf = ctypes.create_string_buffer(cap) if want_source else None
+    r = int(lib().relay_debug_jit_compile(ctypes.byref(p) if p is not None else None, _desc_array(ins), len(ins), sp, len(specs), buf,
+                                          ctypes.c_size_t(cap if want_source else 0)))
+    if r <= -2:
+        raise RelayError(1, lib().relay_last_error().decode())
+    return (r, buf.value.decode()) if want_source else r
+
+
 STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -382,6 +398,16 @@ def relay_last_error() -> str:
 
 def relay_poll_status():
     _check(lib().relay_poll_status(_stream()))
+
+
+def relay_debug_set_jit(enabled: bool) -> bool:
+    """Switches the run-time compiled elementwise bodies on or off for this process; returns the previous setting."""
+    return bool(lib().relay_debug_set_jit(1 if enabled else 0))
+
+
+def relay_debug_jit_compiled() -> int:
+    """Bodies compiled at run time so far; -1 when no run-time compiler library is available."""
+    return int(lib().relay_debug_jit_compiled())
 
 
 def relay_debug_bounds_probe():

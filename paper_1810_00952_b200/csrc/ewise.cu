@@ -660,6 +660,11 @@ extern "C" relay_status_t relay_fused_ewise(const relay_ewise_prog_t *prog, cons
         VmPlan vp;
         const bool no_sums[RELAY_MAX_OUTPUTS] = {false};
         if (vm_plan(tp, v, out_values, no_sums, n_out, &vp)) {
+            // a body compiled for this program where a run-time compiler is present, else the interpreter
+            int32_t odt[RELAY_MAX_OUTPUTS];
+            for (int k = 0; k < n_out; ++k) odt[k] = outputs[k]->dtype;
+            if (const void *jk = jit_get(tp, v, out_values, odt, no_sums, n_out))
+                return jit_launch(jk, v, inputs, n_in, outputs, n_out, nullptr, jit_n_slices(v, false), st);
             const int64_t gx = (v.cols + 255) / 256;
             const int ns = (int)std::max<int64_t>(1, std::min<int64_t>((148 * 8) / gx, v.rows / 32));
             return vm_launch(vp, v, inputs, n_in, outputs, n_out, nullptr, ns, st);
@@ -686,6 +691,7 @@ struct ReducePlan {
     bool fast_row = false;      // identity reduction over the last axis
     bool vm = false;            // vectorised evaluator: unreduced results and sums / means over all leading axes
     VmPlan vmp;
+    int jit_slices = 1;
     int32_t vm_values[RELAY_MAX_OUTPUTS];
     int n_slices = 1;
     size_t ws_need = 0;
@@ -748,7 +754,9 @@ static relay_status_t plan_reduce(const relay_ewise_prog_t *prog, const relay_te
         if (fits && vm_plan(tp, v, pl->vm_values, sums, n_out, &pl->vmp)) {
             pl->vm = true;
             pl->n_slices = vm_grid_slices(v, colsum_slices(v.rows, v.cols, v.storage));
-            pl->ws_need = (size_t)pl->vmp.n_sum * pl->n_slices * (size_t)v.cols * sizeof(float);
+            pl->jit_slices = jit_n_slices(v, true);
+            // room for either route: which one runs is decided at the launch (is a run-time compiler present?)
+            pl->ws_need = (size_t)pl->vmp.n_sum * std::max(pl->n_slices, pl->jit_slices) * (size_t)v.cols * sizeof(float);
         }
     }
     return RELAY_OK;
@@ -841,7 +849,16 @@ extern "C" relay_status_t relay_fused_reduce(const relay_ewise_prog_t *prog, con
     }
 
     if (pl.vm) {
-        RELAY_TRY(vm_launch(pl.vmp, v, inputs, n_in, outputs, n_out, (float *)ws, pl.n_slices, st));
+        int32_t odt[RELAY_MAX_OUTPUTS];
+        bool is_sum[RELAY_MAX_OUTPUTS];
+        for (int k = 0; k < n_out; ++k) { odt[k] = outputs[k]->dtype; is_sum[k] = specs[k].red_op != RELAY_RED_NONE; }
+        int slices = pl.n_slices;
+        if (const void *jk = jit_get(tp, v, pl.vm_values, odt, is_sum, n_out)) {
+            slices = pl.jit_slices;
+            RELAY_TRY(jit_launch(jk, v, inputs, n_in, outputs, n_out, (float *)ws, slices, st));
+        } else {
+            RELAY_TRY(vm_launch(pl.vmp, v, inputs, n_in, outputs, n_out, (float *)ws, slices, st));
+        }
         float *sums[RELAY_MAX_OUTPUTS];
         float scale[RELAY_MAX_OUTPUTS];
         int n_sum = 0;
@@ -850,7 +867,7 @@ extern "C" relay_status_t relay_fused_reduce(const relay_ewise_prog_t *prog, con
                 sums[n_sum] = (float *)outputs[k]->data;
                 scale[n_sum++] = specs[k].red_op == RELAY_RED_MEAN ? 1.0f / (float)v.rows : 1.0f;
             }
-        return n_sum ? launch_colsum_finalize_n((const float *)ws, pl.n_slices, v.cols, scale, sums, n_sum, st) : RELAY_OK;
+        return n_sum ? launch_colsum_finalize_n((const float *)ws, slices, v.cols, scale, sums, n_sum, st) : RELAY_OK;
     }
 
     // generic: one evaluator pass for the unreduced results, one reduction launch per reduced result
@@ -904,4 +921,32 @@ extern "C" int32_t relay_debug_group_route(const relay_ewise_prog_t *prog, const
     const bool no_sums[RELAY_MAX_OUTPUTS] = {false};
     for (int k = 0; k < n_out; ++k) values[k] = specs[k].value;
     return v.ok && vm_plan(pl.tp, v, values, no_sums, n_out, &vp) ? 1 : 2;
+}
+
+// Host only: the source of the body that would be compiled at run time for this group, and whether it compiles for sm_100a.
+// 1: compiled (the source, NUL-terminated and cut to `cap` bytes, is in `src` if that is not null); 0: the group does not
+// run on the vectorised tier; -1: no run-time compiler on this machine; -2: it did not compile (relay_last_error has the
+// compiler's messages); -3: the group does not type-check.
+extern "C" int32_t relay_debug_jit_compile(const relay_ewise_prog_t *prog, const relay_tensor_t *const *inputs, int32_t n_in,
+                                           const relay_out_spec_t *specs, int32_t n_out, char *src, size_t cap)
+{
+    clear_error();
+    ReducePlan pl;
+    if (plan_reduce(prog, inputs, n_in, specs, n_out, &pl) != RELAY_OK) return -3;
+    bool all_unreduced = true;
+    for (int k = 0; k < n_out; ++k) all_unreduced = all_unreduced && specs[k].red_op == RELAY_RED_NONE;
+    int32_t values[RELAY_MAX_OUTPUTS], odt[RELAY_MAX_OUTPUTS];
+    bool sums[RELAY_MAX_OUTPUTS];
+    for (int k = 0; k < n_out; ++k) { values[k] = specs[k].value; sums[k] = specs[k].red_op != RELAY_RED_NONE; odt[k] = pl.tp.dtype[specs[k].value]; }
+    if (all_unreduced) {
+        VmPlan vp;
+        if (!pl.v.ok || !vm_plan(pl.tp, pl.v, values, sums, n_out, &vp)) return 0;
+    } else if (!pl.vm) {
+        return 0;
+    }
+    std::string text, log;
+    const int r = jit_compile_only(pl.tp, pl.v, values, odt, sums, n_out, &text, &log);
+    if (r == -2) fail(RELAY_ERR_CUDA, "run-time compilation failed: %s", log.c_str());
+    if (src && cap > 0) { snprintf(src, cap, "%s", text.c_str()); }
+    return r;
 }

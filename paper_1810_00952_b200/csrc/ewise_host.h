@@ -1,6 +1,8 @@
 // Host-side launch helpers of the memory-bound kernels that other groups reuse
 // (the dense / conv2d gradient groups need dZ = dy (.) act'(y) and its column sums).
 #pragma once
+#include <string>
+
 #include "common.h"
 
 namespace relay {
@@ -18,6 +20,16 @@ bool vm_plan(const TypedProgram &tp, const View2D &v, const int32_t *out_values,
 int vm_grid_slices(const View2D &v, int n_slices_wanted);
 relay_status_t vm_launch(const VmPlan &plan, const View2D &v, const relay_tensor_t *const *inputs, int n_in, const relay_tensor_t *const *outputs,
                          int n_out, float *partials, int n_slices, cudaStream_t st);
+// Bodies compiled at run time for the same class of groups (ewise_jit.cu).  jit_get: the kernel for this group (compiled on first
+// use, cached), or nullptr when there is no run-time compiler on this machine, it is switched off, or the group is outside the
+// class: the caller then takes the interpreter.  out_dtype[k]: storage type of result k; partials: [n_sum][n_slices][cols].
+bool jit_usable();
+const void *jit_get(const TypedProgram &tp, const View2D &v, const int32_t *out_values, const int32_t *out_dtype, const bool *colsum, int n_out);
+int jit_n_slices(const View2D &v, bool any_sum);
+int jit_compile_only(const TypedProgram &tp, const View2D &v, const int32_t *out_values, const int32_t *out_dtype, const bool *colsum, int n_out,
+                     std::string *src, std::string *log);
+relay_status_t jit_launch(const void *kernel, const View2D &v, const relay_tensor_t *const *inputs, int n_in, const relay_tensor_t *const *outputs,
+                          int n_out, float *partials, int n_slices, cudaStream_t st);
 // finalises n_out column sums whose partials lie one after another ([k][n_slices][cols]); scale[k] multiplies sum k (null: 1)
 relay_status_t launch_colsum_finalize_n(const float *partial, int n_slices, int64_t cols, const float *scale, float *const *out, int n_out,
                                         cudaStream_t st);

@@ -1,5 +1,5 @@
-"""GPU parity: programs without a pre-compiled body on the vectorised evaluator, and integer-typed values on the scalar
-evaluator, against the CPU oracle through the C-ABI."""
+"""GPU parity: programs without a pre-compiled body on the vectorised tier -- once as bodies compiled at run time, once on
+the in-kernel interpreter -- and integer-typed values on the scalar evaluator, against the CPU oracle through the C-ABI."""
 import numpy as np
 import pytest
 import torch
@@ -15,6 +15,16 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 TDT = {P.BF16: torch.bfloat16, P.F32: torch.float32, P.BOOL: torch.uint8}
 VEC = 1
+
+
+@pytest.fixture(autouse=True, params=["compiled", "interpreted"])
+def tier(request):
+    """Every test of this file runs twice: with the run-time compiled bodies and with them switched off."""
+    if request.param == "compiled" and B.relay_debug_jit_compiled() < 0:
+        pytest.skip("no run-time compiler library on this machine")
+    before = B.relay_debug_set_jit(request.param == "compiled")
+    yield request.param
+    B.relay_debug_set_jit(before)
 
 
 def rnd(shape, tdt, seed, scale=1.0):
@@ -198,3 +208,20 @@ def test_integer_values_are_exact_beyond_24_bits():
             assert np.array_equal(got.numpy().astype(np.int64), wv.astype(np.int64)), name
         else:
             assert np.array_equal(got.double().numpy(), wv), name      # one rounding to nearest even on both sides
+
+
+def test_a_body_is_compiled_once_per_program_and_only_when_switched_on(tier):
+    x, y = rnd((64, 264), torch.float32, 5), rnd((264,), torch.float32, 6)
+    p = P.Program([P.F32, P.F32]); v = p.add(p.mul(0, p.const(1.0 + 2.0 ** -20)), p.tanh(1))      # a program no other test uses
+    n0 = B.relay_debug_jit_compiled()
+    for _ in range(2):
+        (got,), (want,) = run_ewise(p, [x, y], [v])
+        assert_f32(got, want, "out")
+    n1 = B.relay_debug_jit_compiled()
+    if tier == "compiled":
+        assert n1 == n0 + 1                         # the second call found it in the cache
+        x2 = rnd((7, 520), torch.float32, 8)        # another shape: same body, same kernel
+        run_ewise(p, [x2, rnd((520,), torch.float32, 9)], [v])
+        assert B.relay_debug_jit_compiled() == n1
+    else:
+        assert n1 == n0 or n0 < 0
