@@ -422,7 +422,8 @@ relay_status_t relay_debug_bounds_probe(void *stream);
  * launched like any other kernel; without the library, in the bounds-check build, or when switched off here, the same
  * groups run on the library's in-kernel interpreter.  relay_debug_set_jit switches the compiled bodies on (non-zero,
  * the default) or off for the process and returns the previous setting; relay_debug_jit_compiled returns how many
- * bodies have been compiled so far, -1 when no run-time compiler is available.  Neither touches the GPU. */
+ * bodies have been compiled so far, -1 when compiled bodies cannot be used in this process (no run-time compiler
+ * library, no CUDA driver, the bounds-check build).  Neither touches the GPU. */
 int32_t relay_debug_set_jit(int32_t enabled);
 int32_t relay_debug_jit_compiled(void);
 /* Host only (needs no GPU): generates the source of the body that would be compiled at run time for this group and
@@ -453,8 +454,9 @@ relay_status_t relay_debug_lstm_phase_cycles(const relay_tensor_t *x, const rela
 
 /* Host-only view of which kernel tier relay_fused_ewise / relay_fused_reduce would run a group on (no counterpart in the
  * paper; touches no GPU; arguments as for relay_fused_reduce, all-RELAY_RED_NONE specs describe a relay_fused_ewise call):
- * 0 a pre-compiled body, 1 the vectorised evaluator (16-byte accesses, the program interpreted on 8 elements at a
- * time), 2 the scalar evaluator (any rank, broadcast pattern, axes mask and base type), 3 the row-reduction kernel;
+ * 0 a pre-compiled body, 1 the vectorised tier (16-byte accesses over the collapsed 2-D view: a body compiled at run
+ * time where that is available, else the program interpreted on 16 elements at a time), 2 the scalar evaluator (any
+ * rank, broadcast pattern, axes mask and base type), 3 the row-reduction kernel;
  * -1 if the group does not type-check (relay_last_error() says why).  For tests and for callers that want to know
  * whether a program takes the fast route. */
 int32_t relay_debug_group_route(const relay_ewise_prog_t *prog, const relay_tensor_t *const *inputs, int32_t n_in,

@@ -302,7 +302,8 @@ def relay_fused_reduce(prog: Optional[dict], inputs, specs, outputs, ws=None):
 
 
 def relay_debug_group_route(prog: Optional[dict], inputs, specs) -> int:
-    """Kernel tier a group would run on: 0 pre-compiled body, 1 vectorised evaluator, 2 scalar evaluator, 3 row reduction.
+    """Kernel tier a group would run on: 0 pre-compiled body, 1 vectorised tier (compiled at run time or interpreted), 2 scalar
+    evaluator, 3 row reduction.
     specs as for relay_fused_reduce; (value, RED_NONE, 0, 0) entries describe a relay_fused_ewise call.  Host only."""
     p = make_prog(prog) if prog is not None else None
     ins = [desc(t) for t in inputs]
@@ -406,7 +407,7 @@ def relay_debug_set_jit(enabled: bool) -> bool:
 
 
 def relay_debug_jit_compiled() -> int:
-    """Bodies compiled at run time so far; -1 when no run-time compiler library is available."""
+    """Bodies compiled at run time so far; -1 when compiled bodies cannot be used in this process (no compiler library, no driver)."""
     return int(lib().relay_debug_jit_compiled())
 
 

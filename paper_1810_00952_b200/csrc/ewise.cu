@@ -655,16 +655,16 @@ extern "C" relay_status_t relay_fused_ewise(const relay_ewise_prog_t *prog, cons
         return launch_body2d<BodyTanhAffineResidualFwd>(v.storage, A, ns, st, "ewise2d<tanh_affine_residual_fwd>");
     }
 
-    // any other program over the 2-D view: the vectorised evaluator
+    // any other program over the 2-D view: a body compiled for this program where a run-time compiler is present, else the
+    // in-kernel interpreter (which takes fewer programs: bounded temporaries and literals)
     if (v.ok) {
-        VmPlan vp;
         const bool no_sums[RELAY_MAX_OUTPUTS] = {false};
+        int32_t odt[RELAY_MAX_OUTPUTS];
+        for (int k = 0; k < n_out; ++k) odt[k] = outputs[k]->dtype;
+        if (const void *jk = jit_get(tp, v, out_values, odt, no_sums, n_out))
+            return jit_launch(jk, v, inputs, n_in, outputs, n_out, nullptr, jit_n_slices(v, false), st);
+        VmPlan vp;
         if (vm_plan(tp, v, out_values, no_sums, n_out, &vp)) {
-            // a body compiled for this program where a run-time compiler is present, else the interpreter
-            int32_t odt[RELAY_MAX_OUTPUTS];
-            for (int k = 0; k < n_out; ++k) odt[k] = outputs[k]->dtype;
-            if (const void *jk = jit_get(tp, v, out_values, odt, no_sums, n_out))
-                return jit_launch(jk, v, inputs, n_in, outputs, n_out, nullptr, jit_n_slices(v, false), st);
             const int64_t gx = (v.cols + 255) / 256;
             const int ns = (int)std::max<int64_t>(1, std::min<int64_t>((148 * 8) / gx, v.rows / 32));
             return vm_launch(vp, v, inputs, n_in, outputs, n_out, nullptr, ns, st);
@@ -690,6 +690,7 @@ struct ReducePlan {
     bool fast_colsum = false;   // identity column sum / mean over all leading axes
     bool fast_row = false;      // identity reduction over the last axis
     bool vm = false;            // vectorised evaluator: unreduced results and sums / means over all leading axes
+    bool jit = false;           // in the class a body can be compiled for at run time (a superset of `vm`)
     VmPlan vmp;
     int jit_slices = 1;
     int32_t vm_values[RELAY_MAX_OUTPUTS];
@@ -751,12 +752,15 @@ static relay_status_t plan_reduce(const relay_ewise_prog_t *prog, const relay_te
             sums[k] = colsum;
             pl->vm_values[k] = specs[k].value;
         }
-        if (fits && vm_plan(tp, v, pl->vm_values, sums, n_out, &pl->vmp)) {
-            pl->vm = true;
-            pl->n_slices = vm_grid_slices(v, colsum_slices(v.rows, v.cols, v.storage));
+        if (fits) {
+            int n_sum = 0;
+            for (int k = 0; k < n_out; ++k) n_sum += sums[k];
+            pl->jit = jit_in_class(tp, v, pl->vm_values, n_out);
+            pl->vm = vm_plan(tp, v, pl->vm_values, sums, n_out, &pl->vmp);
+            pl->n_slices = pl->vm ? vm_grid_slices(v, colsum_slices(v.rows, v.cols, v.storage)) : 1;
             pl->jit_slices = jit_n_slices(v, true);
             // room for either route: which one runs is decided at the launch (is a run-time compiler present?)
-            pl->ws_need = (size_t)pl->vmp.n_sum * std::max(pl->n_slices, pl->jit_slices) * (size_t)v.cols * sizeof(float);
+            if (pl->jit || pl->vm) pl->ws_need = (size_t)n_sum * std::max(pl->n_slices, pl->jit_slices) * (size_t)v.cols * sizeof(float);
         }
     }
     return RELAY_OK;
@@ -848,12 +852,13 @@ extern "C" relay_status_t relay_fused_reduce(const relay_ewise_prog_t *prog, con
         return check_launch("rowreduce");
     }
 
-    if (pl.vm) {
-        int32_t odt[RELAY_MAX_OUTPUTS];
-        bool is_sum[RELAY_MAX_OUTPUTS];
-        for (int k = 0; k < n_out; ++k) { odt[k] = outputs[k]->dtype; is_sum[k] = specs[k].red_op != RELAY_RED_NONE; }
+    int32_t odt[RELAY_MAX_OUTPUTS];
+    bool is_sum[RELAY_MAX_OUTPUTS];
+    for (int k = 0; k < n_out; ++k) { odt[k] = outputs[k]->dtype; is_sum[k] = specs[k].red_op != RELAY_RED_NONE; }
+    const void *jk = pl.jit ? jit_get(tp, v, pl.vm_values, odt, is_sum, n_out) : nullptr;
+    if (jk || pl.vm) {
         int slices = pl.n_slices;
-        if (const void *jk = jit_get(tp, v, pl.vm_values, odt, is_sum, n_out)) {
+        if (jk) {
             slices = pl.jit_slices;
             RELAY_TRY(jit_launch(jk, v, inputs, n_in, outputs, n_out, (float *)ws, slices, st));
         } else {
@@ -911,7 +916,7 @@ extern "C" int32_t relay_debug_group_route(const relay_ewise_prog_t *prog, const
     if (plan_reduce(prog, inputs, n_in, specs, n_out, &pl) != RELAY_OK) return -1;
     bool all_unreduced = true;
     for (int k = 0; k < n_out; ++k) all_unreduced = all_unreduced && specs[k].red_op == RELAY_RED_NONE;
-    if (!all_unreduced) return (pl.fast_grad || pl.fast_colsum) ? 0 : pl.fast_row ? 3 : pl.vm ? 1 : 2;
+    if (!all_unreduced) return (pl.fast_grad || pl.fast_colsum) ? 0 : pl.fast_row ? 3 : (pl.vm || (pl.jit && jit_usable())) ? 1 : 2;
     const View2D &v = pl.v;
     if (v.ok && n_out == 1 && n_in == 3 && kinds_match<BodyTanhAffineResidualFwd>(v) && pl.tp.dtype[specs[0].value] == v.storage &&
         canon(pl.tp, specs[0].value) == known_tanh_affine_fwd(v.storage).out)
@@ -920,7 +925,7 @@ extern "C" int32_t relay_debug_group_route(const relay_ewise_prog_t *prog, const
     int32_t values[RELAY_MAX_OUTPUTS];
     const bool no_sums[RELAY_MAX_OUTPUTS] = {false};
     for (int k = 0; k < n_out; ++k) values[k] = specs[k].value;
-    return v.ok && vm_plan(pl.tp, v, values, no_sums, n_out, &vp) ? 1 : 2;
+    return v.ok && (vm_plan(pl.tp, v, values, no_sums, n_out, &vp) || (jit_usable() && jit_in_class(pl.tp, v, values, n_out))) ? 1 : 2;
 }
 
 // Host only: the source of the body that would be compiled at run time for this group, and whether it compiles for sm_100a.
@@ -938,12 +943,8 @@ extern "C" int32_t relay_debug_jit_compile(const relay_ewise_prog_t *prog, const
     int32_t values[RELAY_MAX_OUTPUTS], odt[RELAY_MAX_OUTPUTS];
     bool sums[RELAY_MAX_OUTPUTS];
     for (int k = 0; k < n_out; ++k) { values[k] = specs[k].value; sums[k] = specs[k].red_op != RELAY_RED_NONE; odt[k] = pl.tp.dtype[specs[k].value]; }
-    if (all_unreduced) {
-        VmPlan vp;
-        if (!pl.v.ok || !vm_plan(pl.tp, pl.v, values, sums, n_out, &vp)) return 0;
-    } else if (!pl.vm) {
-        return 0;
-    }
+    if (all_unreduced ? !jit_in_class(pl.tp, pl.v, values, n_out) : !pl.jit) return 0;
+    if (!all_unreduced && (pl.fast_grad || pl.fast_colsum || pl.fast_row)) return 0;
     std::string text, log;
     const int r = jit_compile_only(pl.tp, pl.v, values, odt, sums, n_out, &text, &log);
     if (r == -2) fail(RELAY_ERR_CUDA, "run-time compilation failed: %s", log.c_str());

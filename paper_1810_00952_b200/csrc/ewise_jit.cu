@@ -135,13 +135,10 @@ struct Gen {
     bool ok = false;
 };
 
-// `out_dtype[k]`: storage type of result k (bf16, f32 or Bool as bytes); `colsum[k]`: result k is summed over the rows
-Gen generate(const TypedProgram &tp, const View2D &v, const int32_t *out_values, const int32_t *out_dtype, const bool *colsum, int n_out)
+// which values the results depend on; false if one of them is of a type the bodies do not carry (integer lanes)
+bool needed_values(const TypedProgram &tp, const int32_t *out_values, int n_out, bool (&needed)[kMaxValues])
 {
-    Gen G;
-    const bool bf = v.storage == RELAY_BF16;
-    const int V = bf ? 8 : 4;
-    bool needed[kMaxValues] = {false};
+    for (int x = 0; x < kMaxValues; ++x) needed[x] = false;
     for (int k = 0; k < n_out; ++k) needed[out_values[k]] = true;
     for (int x = tp.n_values - 1; x >= tp.n_in; --x) {
         if (!needed[x]) continue;
@@ -150,9 +147,20 @@ Gen generate(const TypedProgram &tp, const View2D &v, const int32_t *out_values,
         if (in.b >= 0) needed[in.b] = true;
         if (in.c >= 0) needed[in.c] = true;
     }
-    int n_full = 0;
     for (int x = 0; x < tp.n_values; ++x)
-        if (needed[x] && !(tp.dtype[x] == RELAY_F32 || tp.dtype[x] == RELAY_BF16 || tp.dtype[x] == RELAY_BOOL)) return G;   // integer lanes: not here
+        if (needed[x] && !(tp.dtype[x] == RELAY_F32 || tp.dtype[x] == RELAY_BF16 || tp.dtype[x] == RELAY_BOOL)) return false;
+    return true;
+}
+
+// `out_dtype[k]`: storage type of result k (bf16, f32 or Bool as bytes); `colsum[k]`: result k is summed over the rows
+Gen generate(const TypedProgram &tp, const View2D &v, const int32_t *out_values, const int32_t *out_dtype, const bool *colsum, int n_out)
+{
+    Gen G;
+    const bool bf = v.storage == RELAY_BF16;
+    const int V = bf ? 8 : 4;
+    bool needed[kMaxValues];
+    if (!needed_values(tp, out_values, n_out, needed)) return G;
+    int n_full = 0;
     for (int i = 0; i < tp.n_in; ++i) n_full += v.kind[i] == KIND_FULL;
     for (int k = 0; k < n_out; ++k) {
         G.sum_of_out[k] = colsum[k] ? G.n_sum++ : -1;
@@ -350,6 +358,14 @@ Kernel *compile(const Gen &G, int vec)
 
 }  // namespace
 
+// The class of groups a body can be generated for (whether or not a compiler is present): over the collapsed 2-D view,
+// float and Bool values only; the caller has checked that every result is unreduced or a sum over all leading axes.
+bool jit_in_class(const TypedProgram &tp, const View2D &v, const int32_t *out_values, int n_out)
+{
+    bool needed[kMaxValues];
+    return v.ok && n_out >= 1 && n_out <= RELAY_MAX_OUTPUTS && v.rows < (1ll << 31) && needed_values(tp, out_values, n_out, needed);
+}
+
 bool jit_usable()
 {
 #ifdef RELAY_BOUNDS_CHECK
@@ -442,12 +458,13 @@ using namespace relay;
 // returns the previous setting.
 extern "C" int32_t relay_debug_set_jit(int32_t enabled) { return g_enabled.exchange(enabled ? 1 : 0); }
 
-// Bodies compiled so far in this process; -1 when no run-time compiler is available here.
+// Bodies compiled so far in this process; -1 when compiled bodies cannot be used here (no run-time compiler library, or no
+// driver to load them with).
 extern "C" int32_t relay_debug_jit_compiled(void)
 {
 #ifdef RELAY_BOUNDS_CHECK
     return -1;
 #else
-    return nvrtc().ok ? g_compiled.load() : -1;
+    return nvrtc().ok && driver().ok ? g_compiled.load() : -1;
 #endif
 }

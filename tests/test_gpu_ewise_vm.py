@@ -225,3 +225,18 @@ def test_a_body_is_compiled_once_per_program_and_only_when_switched_on(tier):
         assert B.relay_debug_jit_compiled() == n1
     else:
         assert n1 == n0 or n0 < 0
+
+
+def test_a_program_beyond_the_interpreters_limits(tier):
+    """More values alive at once than the interpreter has temporaries for: a compiled body where the compiler is present, the
+    scalar evaluator otherwise -- the same results either way."""
+    x = rnd((37, 264), torch.float32, 11, 0.5)
+    p = P.Program([P.F32]); vals = [p.exp(0)]
+    for i in range(7):
+        vals.append(p.tanh(p.add(vals[-1], vals[0])))
+    acc = vals[0]
+    for t in vals[1:]:
+        acc = p.mul(acc, t)
+    total = p.add(acc, p.add(vals[1], p.add(vals[2], p.add(vals[3], p.add(vals[4], p.add(vals[5], p.add(vals[6], vals[7])))))))
+    (got,), (want,) = run_ewise(p, [x], [total], expect_route=VEC if tier == "compiled" else 2)
+    assert_f32(got, want, "total")

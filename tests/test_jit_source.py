@@ -7,11 +7,16 @@ from paper_1810_00952_b200 import binding as B
 from relay_workloads import program as P
 
 BF, F32 = torch.bfloat16, torch.float32
-pytestmark = pytest.mark.skipif(B.relay_debug_jit_compiled() < 0, reason="no run-time compiler library on this machine")
-
-
 def compile_group(prog, inputs, specs, want_source=False):
     return B.relay_debug_jit_compile(prog.arrays() if prog is not None else None, inputs, specs, want_source)
+
+
+def _no_compiler():
+    p = P.Program([P.F32]); v = p.neg(0)
+    return compile_group(p, [torch.empty(8, 64)], [(v, B.RED_NONE, 0, 0)]) == -1
+
+
+pytestmark = pytest.mark.skipif(_no_compiler(), reason="no run-time compiler library on this machine")
 
 
 @pytest.mark.parametrize("tdt,code", [(BF, P.BF16), (F32, P.F32)])
