@@ -276,9 +276,14 @@ relay_status_t relay_fused_reduce(const relay_ewise_prog_t *prog, const relay_te
  * allocation is forbidden.  They still pass inputs and outputs, but no workspace: the scratch for
  * the per-slice partial sums is a fixed array of RELAY_STATIC_SCRATCH_BYTES inside the library's
  * device image (each GPU that loads the library holds one copy until the process exits).
- *   - A group whose relay_workspace_bytes_reduce() exceeds RELAY_STATIC_SCRATCH_BYTES is rejected
- *     with RELAY_ERR_WORKSPACE before anything is launched; use relay_fused_reduce then.
- *   - The call allocates nothing, on the device or through any allocating library routine.
+ *   - A group whose kernels would use more scratch than RELAY_STATIC_SCRATCH_BYTES is rejected
+ *     with RELAY_ERR_WORKSPACE before anything is launched; use relay_fused_reduce then.  (What
+ *     counts is what the group really uses, which is at most relay_workspace_bytes_reduce():
+ *     a reduction over the last axis, for one, uses none and is never rejected.)
+ *   - The call allocates nothing, on the device or through any allocating library routine.  That
+ *     includes compiling a body for a program at run time: here a program uses a compiled body only
+ *     if an earlier relay_fused_reduce / relay_fused_ewise call already compiled it, and runs on
+ *     the library's built-in kernels otherwise (same results within the same tolerance).
  *   - The first call on each device looks up the array's device address (a one-time set-up with
  *     that device current); make that first call outside any stream capture.
  *   - All calls share the one array, and it keeps whatever the last call left there.  A call

@@ -295,6 +295,12 @@ struct DevReduce {
     void *out;
     float scale;
     int32_t group;  // threads that share one result: 32 (a warp) or 256 (the block)
+    // n_split > 1 (group 256 only): the reduced extent of every result is cut into n_split runs of `chunk` elements, one block
+    // each, which leave (value, position) in part_val / part_pos[result * n_split + run] for reduce_split_finish_kernel
+    int32_t n_split;
+    int64_t chunk;
+    float *part_val;
+    long long *part_pos;
 };
 
 __device__ __forceinline__ void combine(int red_op, float &best, int64_t &pos, float ob, int64_t op)
@@ -312,7 +318,10 @@ __global__ void __launch_bounds__(256) reduce_generic_kernel(const DevProgram P,
     int64_t idx[RELAY_MAX_RANK];
     const int lane_in_group = threadIdx.x % R.group;
     const int groups_per_block = blockDim.x / R.group;
-    const int64_t kept = (int64_t)blockIdx.x * groups_per_block + threadIdx.x / R.group;
+    const int64_t unit = (int64_t)blockIdx.x * groups_per_block + threadIdx.x / R.group;
+    const int64_t kept = R.n_split > 1 ? unit / R.n_split : unit;
+    const int64_t run = R.n_split > 1 ? unit % R.n_split : 0;
+    const int64_t j0 = run * R.chunk, j1 = R.n_split > 1 ? min(R.red_elems, j0 + R.chunk) : R.red_elems;
     const bool live = kept < R.kept_elems;
     const bool is_sum = R.red_op == RELAY_RED_SUM || R.red_op == RELAY_RED_MEAN;
     float best = is_sum ? 0.0f : -INFINITY;
@@ -324,7 +333,7 @@ __global__ void __launch_bounds__(256) reduce_generic_kernel(const DevProgram P,
             idx[ax] = rem % P.shape[ax];
             rem /= P.shape[ax];
         }
-        for (int64_t j = lane_in_group; j < R.red_elems; j += R.group) {
+        for (int64_t j = j0 + lane_in_group; j < j1; j += R.group) {
             int64_t rj = j;
             for (int i = R.n_red - 1; i >= 0; --i) {
                 int ax = R.red_axis[i];
@@ -353,9 +362,32 @@ __global__ void __launch_bounds__(256) reduce_generic_kernel(const DevProgram P,
         }
     }
     if (live && lane_in_group == 0) {
-        if (R.red_op == RELAY_RED_ARGMAX) { if (relay_in_bounds((int64_t *)R.out + kept, 8)) ((int64_t *)R.out)[kept] = pos; }
+        if (R.n_split > 1) {
+            if (relay_in_bounds(R.part_val + unit, 4)) R.part_val[unit] = best;
+            if (relay_in_bounds(R.part_pos + unit, 8)) R.part_pos[unit] = pos;
+        } else if (R.red_op == RELAY_RED_ARGMAX) { if (relay_in_bounds((int64_t *)R.out + kept, 8)) ((int64_t *)R.out)[kept] = pos; }
         else if (relay_in_bounds((float *)R.out + kept, 4)) ((float *)R.out)[kept] = best * R.scale;
     }
+}
+
+// second pass of a split reduction: one thread per result combines its runs in run order (sums in fp64: the runs are few)
+__global__ void __launch_bounds__(128) reduce_split_finish_kernel(const DevReduce R)
+{
+    const int64_t kept = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (kept >= R.kept_elems) return;
+    const bool is_sum = R.red_op == RELAY_RED_SUM || R.red_op == RELAY_RED_MEAN;
+    double sum = 0.0;
+    float best = -INFINITY;
+    int64_t pos = 0;
+    for (int s = 0; s < R.n_split; ++s) {
+        const int64_t u = kept * R.n_split + s;
+        if (!relay_in_bounds(R.part_val + u, 4) || !relay_in_bounds(R.part_pos + u, 8)) continue;
+        const float v = R.part_val[u];
+        if (is_sum) sum += (double)v;
+        else if (v > best) { best = v; pos = R.part_pos[u]; }      // runs are in index order: the first maximum stays
+    }
+    if (R.red_op == RELAY_RED_ARGMAX) { if (relay_in_bounds((int64_t *)R.out + kept, 8)) ((int64_t *)R.out)[kept] = pos; }
+    else if (relay_in_bounds((float *)R.out + kept, 4)) ((float *)R.out)[kept] = is_sum ? (float)(sum * (double)R.scale) : best;
 }
 
 // =================================================================================================
@@ -683,6 +715,17 @@ extern "C" relay_status_t relay_fused_ewise(const relay_ewise_prog_t *prog, cons
 // ---- reduce ----------------------------------------------------------------------------------------
 namespace relay {
 
+// Scalar-evaluator reductions with few results over a long reduced extent (a sum over all axes, say) are cut into runs
+// that separate blocks reduce; the runs' (value, position) pairs take at most this much of the workspace.
+constexpr int kSplitUnitsMax = 4096;
+constexpr size_t kSplitScratchBytes = (size_t)kSplitUnitsMax * (sizeof(float) + sizeof(long long));
+static int generic_split(int64_t kept_elems, int64_t red_elems)
+{
+    if (kept_elems > 64 || red_elems < 65536) return 1;
+    const int64_t n = std::min<int64_t>(kSplitUnitsMax / kept_elems, red_elems / 8192);
+    return n >= 2 ? (int)n : 1;
+}
+
 struct ReducePlan {
     TypedProgram tp;
     View2D v;
@@ -763,6 +806,27 @@ static relay_status_t plan_reduce(const relay_ewise_prog_t *prog, const relay_te
             if (pl->jit || pl->vm) pl->ws_need = (size_t)n_sum * std::max(pl->n_slices, pl->jit_slices) * (size_t)v.cols * sizeof(float);
         }
     }
+    if (!pl->fast_grad && !pl->fast_colsum && !pl->fast_row) {
+        // what is neither pre-compiled, compiled at run time nor interpreted 16 elements at a time runs on the scalar
+        // evaluator; whether a compiled body exists is only known at the launch, so the room for split runs is asked for
+        // whenever that evaluator may run
+        for (int k = 0; k < n_out; ++k) {
+            if (specs[k].red_op == RELAY_RED_NONE) continue;
+            int64_t kept = 1, red = 1;
+            for (int d = 0; d < tp.rank; ++d) (specs[k].axes_mask >> d & 1 ? red : kept) *= tp.shape[d];
+            if (generic_split(kept, red) > 1) pl->ws_need = std::max(pl->ws_need, kSplitScratchBytes);
+        }
+    }
+    return RELAY_OK;
+}
+
+// scratch that relay_fused_reduce will really use for this group (never more than relay_workspace_bytes_reduce's bound)
+relay_status_t reduce_planned_scratch(const relay_ewise_prog_t *prog, const relay_tensor_t *const *inputs, int32_t n_in,
+                                      const relay_out_spec_t *specs, int32_t n_out, size_t *need)
+{
+    ReducePlan pl;
+    RELAY_TRY(plan_reduce(prog, inputs, n_in, specs, n_out, &pl));
+    *need = pl.ws_need;
     return RELAY_OK;
 }
 
@@ -778,11 +842,13 @@ extern "C" size_t relay_workspace_bytes_reduce(const relay_tensor_t *const *inpu
     static const relay_ewise_prog_t empty = {0, 0, nullptr};
     TypedProgram tp;
     if (type_program(&empty, inputs, n_in, &tp) != RELAY_OK) return 0;
-    View2D v = view2d(tp);
-    if (!v.ok) return 0;
     int n_sum = 0;
     for (int k = 0; k < n_out; ++k) n_sum += specs[k].red_op != RELAY_RED_NONE;
-    return (size_t)n_sum * colsum_slices(v.rows, v.cols, v.storage) * (size_t)v.cols * sizeof(float);
+    // runs of a split reduction on the scalar evaluator (any shape and type), or per-slice partials of column sums
+    const size_t split = n_sum ? kSplitScratchBytes : 0;
+    View2D v = view2d(tp);
+    if (!v.ok) return split;
+    return std::max(split, (size_t)n_sum * colsum_slices(v.rows, v.cols, v.storage) * (size_t)v.cols * sizeof(float));
 }
 
 extern "C" relay_status_t relay_fused_reduce(const relay_ewise_prog_t *prog, const relay_tensor_t *const *inputs, int32_t n_in,
@@ -899,9 +965,22 @@ extern "C" relay_status_t relay_fused_reduce(const relay_ewise_prog_t *prog, con
         }
         R.scale = specs[k].red_op == RELAY_RED_MEAN ? 1.0f / (float)R.red_elems : 1.0f;
         R.group = (R.kept_elems < 148 * 8 && R.red_elems >= 1024) ? 256 : 32;
+        R.n_split = generic_split(R.kept_elems, R.red_elems);
+        int64_t units = R.kept_elems;
+        if (R.n_split > 1) {
+            R.group = 256;
+            R.chunk = (R.red_elems + R.n_split - 1) / R.n_split;
+            R.part_val = (float *)ws;
+            R.part_pos = (long long *)((char *)ws + (size_t)kSplitUnitsMax * sizeof(float));
+            units *= R.n_split;
+        }
         const int per_block = 256 / R.group;
-        reduce_generic_kernel<<<(unsigned)((R.kept_elems + per_block - 1) / per_block), 256, 0, st>>>(P, R);
+        reduce_generic_kernel<<<(unsigned)((units + per_block - 1) / per_block), 256, 0, st>>>(P, R);
         RELAY_TRY(check_launch("reduce_generic"));
+        if (R.n_split > 1) {
+            reduce_split_finish_kernel<<<(unsigned)((R.kept_elems + 127) / 128), 128, 0, st>>>(R);
+            RELAY_TRY(check_launch("reduce_split_finish"));
+        }
     }
     return RELAY_OK;
 }

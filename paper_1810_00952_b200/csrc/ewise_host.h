@@ -24,6 +24,7 @@ relay_status_t vm_launch(const VmPlan &plan, const View2D &v, const relay_tensor
 // use, cached), or nullptr when there is no run-time compiler on this machine, it is switched off, or the group is outside the
 // class: the caller then takes the interpreter.  out_dtype[k]: storage type of result k; partials: [n_sum][n_slices][cols].
 bool jit_usable();
+bool jit_set_cached_only(bool on);   // this thread: use only bodies compiled already (returns the previous setting)
 bool jit_in_class(const TypedProgram &tp, const View2D &v, const int32_t *out_values, int n_out);
 const void *jit_get(const TypedProgram &tp, const View2D &v, const int32_t *out_values, const int32_t *out_dtype, const bool *colsum, int n_out);
 int jit_n_slices(const View2D &v, bool any_sum);

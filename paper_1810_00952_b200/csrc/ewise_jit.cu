@@ -366,6 +366,16 @@ bool jit_in_class(const TypedProgram &tp, const View2D &v, const int32_t *out_va
     return v.ok && n_out >= 1 && n_out <= RELAY_MAX_OUTPUTS && v.rows < (1ll << 31) && needed_values(tp, out_values, n_out, needed);
 }
 
+// Set by callers that must not allocate (compiling and loading a module allocates host and device memory): on this thread
+// only bodies that are compiled already are used, any other group runs on the interpreter.
+static thread_local bool t_cached_only = false;
+bool jit_set_cached_only(bool on)
+{
+    const bool before = t_cached_only;
+    t_cached_only = on;
+    return before;
+}
+
 bool jit_usable()
 {
 #ifdef RELAY_BOUNDS_CHECK
@@ -388,6 +398,7 @@ const void *jit_get(const TypedProgram &tp, const View2D &v, const int32_t *out_
     std::lock_guard<std::mutex> lock(g_mu);
     auto it = g_cache.find(key);
     if (it != g_cache.end()) return it->second;
+    if (t_cached_only) return nullptr;
     Kernel *k = compile(G, v.storage == RELAY_BF16 ? 8 : 4);
     g_cache.emplace(key, k);
     return k;

@@ -35,12 +35,20 @@ relay_status_t static_scratch_of_current_device(void **out)
 
 }  // namespace
 
+namespace relay {
+relay_status_t reduce_planned_scratch(const relay_ewise_prog_t *prog, const relay_tensor_t *const *inputs, int32_t n_in,
+                                      const relay_out_spec_t *specs, int32_t n_out, size_t *need);
+bool jit_set_cached_only(bool on);
+}
+
 extern "C" relay_status_t relay_fused_reduce_static_scratch(const relay_ewise_prog_t *prog, const relay_tensor_t *const *inputs,
                                                             int32_t n_in, const relay_out_spec_t *specs,
                                                             const relay_tensor_t *const *outputs, int32_t n_out, void *stream)
 {
     relay::clear_error();
-    const size_t need = relay_workspace_bytes_reduce(inputs, n_in, specs, n_out);
+    // what this group's kernels will really use (a reduction over the last axis uses none), not the program-independent bound
+    size_t need = 0;
+    RELAY_TRY(relay::reduce_planned_scratch(prog, inputs, n_in, specs, n_out, &need));
     if (need > kStaticScratchBytes)
         return relay::fail(RELAY_ERR_WORKSPACE,
                            "this group needs %zu bytes of scratch but the built-in scratch holds %zu; use relay_fused_reduce "
@@ -50,5 +58,11 @@ extern "C" relay_status_t relay_fused_reduce_static_scratch(const relay_ewise_pr
     RELAY_TRY(static_scratch_of_current_device(&scratch));
     // Every partial that the second pass reads is written by the first pass of the same call, so
     // nothing in the array has to be cleared between calls.
-    return relay_fused_reduce(prog, inputs, n_in, specs, outputs, n_out, scratch, kStaticScratchBytes, stream);
+    // Compiling a body for a new program and loading it allocates (host memory, device memory for the code), so this call
+    // never does: a program whose body an earlier relay_fused_reduce / relay_fused_ewise call compiled uses it, any other
+    // runs on the library's built-in kernels.
+    const bool before = relay::jit_set_cached_only(true);
+    const relay_status_t r = relay_fused_reduce(prog, inputs, n_in, specs, outputs, n_out, scratch, kStaticScratchBytes, stream);
+    relay::jit_set_cached_only(before);
+    return r;
 }

@@ -31,3 +31,18 @@ def pytest_runtest_teardown(item, nextitem):
     if os.environ.get("RELAY_B200_LIB") and "gpu" in item.keywords:
         from paper_1810_00952_b200 import binding as B
         B.relay_poll_status()
+
+
+def pytest_terminal_summary(terminalreporter):
+    """fp32 parity: the plain (unfloored) relative error beside the gated one -- how many tests stay within 1e-4 on every
+    non-zero element, and the largest ones."""
+    try:
+        from parity import STRICT_REL
+    except Exception:
+        return
+    if not STRICT_REL:
+        return
+    within = sum(1 for v in STRICT_REL.values() if v <= 1e-4)
+    terminalreporter.write_line(f"fp32 parity, plain max relative error over non-zero elements: {within} of {len(STRICT_REL)} tests <= 1e-4")
+    for k, v in sorted(STRICT_REL.items(), key=lambda kv: -kv[1])[:8]:
+        terminalreporter.write_line(f"  {v:.3e}  {k}")

@@ -24,12 +24,24 @@ def bf16_ulp(v: np.ndarray) -> np.ndarray:
     return 2.0 ** (np.floor(np.log2(a)) - 7)
 
 
+# Per test: the largest PLAIN relative error |g - o| / |o| over the elements with o != 0 that assert_f32 has seen, i.e. the
+# criterion without the floor on the denominator.  It is not the gate (an element that is the difference of two nearly
+# equal terms can have any relative error in fp32) but it is reported at the end of the run (conftest.py), so that a reader
+# sees how far the plain criterion is met.
+STRICT_REL = {}
+
+
 def assert_f32(got, want, what=""):
     g, o = to_np(got), np.asarray(want, dtype=np.float64)
     assert g.shape == o.shape, (what, g.shape, o.shape)
     if o.size == 0:
         return
     assert np.all(np.isfinite(g)), what
+    nz = o != 0
+    if nz.any():
+        import os
+        key = os.environ.get("PYTEST_CURRENT_TEST", "?").split(" ")[0]
+        STRICT_REL[key] = max(STRICT_REL.get(key, 0.0), float((np.abs(g - o)[nz] / np.abs(o[nz])).max()))
     err = np.abs(g - o) / np.maximum(np.abs(o), 1e-2 * rms(o) + 1e-30)
     assert err.max() <= 1e-4, (what, float(err.max()), np.unravel_index(err.argmax(), err.shape))
 

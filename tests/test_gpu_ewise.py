@@ -206,6 +206,43 @@ def test_standalone_reductions_full_size_all_results():
     assert int(w_arg1[7]) == 0 and int(w_arg1[5]) == 0
 
 
+@pytest.mark.parametrize("shape,axes", [((1024, 2048), (0, 1)), ((3, 700, 301), (1, 2)), ((2, 517, 1031), (0, 1, 2)), ((262144, 2), (0,))])
+def test_few_results_over_a_long_extent_are_split_over_blocks(shape, axes):
+    """A reduction with a handful of results over a long reduced extent (a sum over all axes, say) is cut into runs that
+    separate blocks reduce and a second pass combines in run order: sum, mean, max and argmax (ties: the lowest position
+    wins across runs too), with and without a program in front, and a sum whose terms nearly cancel."""
+    g = torch.Generator().manual_seed(23)
+    x = torch.randn(*shape, generator=g)
+    mask = sum(1 << a for a in axes)
+    ident, sqp = P.Program([P.F32]), P.Program([P.F32])
+    sq = sqp.sq(0)
+    xo = x.double().numpy()
+    oshape = oracle.reduce_shape(shape, axes, False)
+    for red in (B.RED_SUM, B.RED_MEAN, B.RED_MAX):
+        for prog, val in ((None, 0), (sqp, sq)):
+            out = Guarded(oshape, torch.float32, DEV)
+            specs = [(val, red, mask, 0)]
+            B.relay_fused_reduce(prog.arrays() if prog else None, [x.to(DEV)], specs, [out.t],
+                                 workspace(B.relay_workspace_bytes_reduce([x], specs), DEV))
+            (want,) = oracle.reduce((prog or ident).arrays(), [xo], [(val, red, axes, False, 5)])
+            if red == B.RED_MAX and prog is None:
+                assert np.array_equal(to_np(out.check()), want)
+            elif prog is None and red != B.RED_MAX:
+                # a sum of zero-mean terms: bounded against the size of the terms, not of the (cancelled) result
+                n_red = int(np.prod([shape[a] for a in axes]))
+                scale = 1.0 if red == B.RED_SUM else 1.0 / n_red
+                assert np.all(np.abs(to_np(out.check()) - want) <= 1e-6 * scale * np.sqrt(n_red) * 8)
+            else:
+                assert_f32(out.check(), want, what=f"{red} {shape} {axes}")
+    xt = torch.randint(0, 7, shape, generator=g).float()          # many ties, in every run
+    out = Guarded(oshape, torch.int64, DEV)
+    specs = [(0, B.RED_ARGMAX, mask, 0)]
+    B.relay_fused_reduce(None, [xt.to(DEV)], specs, [out.t], workspace(B.relay_workspace_bytes_reduce([xt], specs), DEV))
+    (want,) = oracle.reduce(ident.arrays(), [xt.double().numpy()], [(0, oracle.RED_ARGMAX, axes, False, P.I64)])
+    assert np.array_equal(out.check().cpu().numpy(), want)
+    B.relay_poll_status()
+
+
 def test_reduce_with_prologue_and_unreduced_output_generic():
     g = torch.Generator().manual_seed(13)
     x, w = torch.randn(40, 24, generator=g), torch.randn(24, generator=g)

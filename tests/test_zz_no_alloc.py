@@ -61,3 +61,36 @@ def test_static_scratch_rejects_groups_beyond_its_size():
     assert e.value.status_name == "ERR_WORKSPACE" and "scratch" in str(e.value)
     torch.cuda.synchronize()
     assert B.relay_launch_count() == n0 and all(bool((o == 5.0).all()) for o in outs)
+
+
+def test_static_scratch_takes_groups_that_use_less_than_their_bound():
+    """What decides is the scratch a group's kernels really use: a reduction over the last axis uses none, so it is taken even
+    where the program-independent bound of relay_workspace_bytes_reduce lies beyond the built-in array."""
+    x = torch.randn(16, 2_400_000, device=DEV).to(torch.bfloat16)
+    sp = [(0, B.RED_SUM, 2, 0)]
+    assert B.relay_workspace_bytes_reduce([x], sp) > B.STATIC_SCRATCH_BYTES
+    got, want = torch.full((16,), 9.0, device=DEV), torch.full((16,), 9.0, device=DEV)
+    B.relay_fused_reduce(None, [x], sp, [want], torch.empty(B.relay_workspace_bytes_reduce([x], sp), dtype=torch.uint8, device=DEV))
+    B.relay_fused_reduce_static_scratch(None, [x], sp, [got])
+    torch.cuda.synchronize()
+    assert torch.equal(got, want)
+    assert torch.allclose(got, x.float().sum(1), rtol=1e-3, atol=1.0)
+
+
+def test_static_scratch_compiles_nothing():
+    """Compiling a body at run time allocates, so this entry point never does it: a program without a pre-compiled body
+    runs on the built-in kernels until relay_fused_reduce has compiled it, and gives the same sums either way."""
+    x = torch.randn(300, 512, device=DEV)
+    p = P.Program([P.F32]); v = p.tanh(p.sq(0))
+    sp = [(v, B.RED_SUM, 1, 0)]
+    n0 = B.relay_debug_jit_compiled()
+    a, b, c = (torch.full((512,), 9.0, device=DEV) for _ in range(3))
+    B.relay_fused_reduce_static_scratch(p.arrays(), [x], sp, [a])
+    assert B.relay_debug_jit_compiled() == n0
+    B.relay_fused_reduce(p.arrays(), [x], sp, [b], torch.empty(B.relay_workspace_bytes_reduce([x], sp), dtype=torch.uint8, device=DEV))
+    B.relay_fused_reduce_static_scratch(p.arrays(), [x], sp, [c])
+    torch.cuda.synchronize()
+    assert torch.equal(b, c)
+    want = torch.tanh(x.double() ** 2).sum(0)
+    for got in (a, b):
+        assert float((got.double() - want).abs().max()) <= 1e-4 * float(want.abs().max())
