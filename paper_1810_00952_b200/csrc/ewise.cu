@@ -21,7 +21,7 @@ namespace relay {
 // =================================================================================================
 // kernels
 // =================================================================================================
-constexpr int kTX = 32, kTY = 8, kUnroll = 4;
+constexpr int kTX = 32, kTY = 8;
 
 // CL > 1: the kernel is launched in clusters of CL blocks along y, the row slices of one column strip.  The slices'
 // partial column sums then never leave the chip: every block leaves its partials in its own shared memory, and after a
@@ -30,10 +30,13 @@ constexpr int kTX = 32, kTY = 8, kUnroll = 4;
 // scratch memory; the order is fixed, so reruns are bit-identical.
 constexpr int kColsumCluster = 8;
 
-template <typename Body, typename T, bool FAST, int CL = 1>
-__global__ void __launch_bounds__(kTX *kTY, Body::NIN >= 4 ? 2 : 3) ewise2d_kernel(const Args2D<Body::NIN, Body::NOUT> A)
+// TX lanes of 16 bytes side by side in a row (the block covers TX * V columns), 256 / TX rows per pass, UN passes of loads
+// in flight per thread.
+template <typename Body, typename T, bool FAST, int CL = 1, int TX = 32, int UN = 4>
+__global__ void __launch_bounds__(256, Body::NIN >= 4 ? 2 : 3) ewise2d_kernel(const Args2D<Body::NIN, Body::NOUT> A)
 {
     constexpr int V = VecN<T>::N, NIN = Body::NIN, NOUT = Body::NOUT;
+    constexpr int kTX = TX, kTY = 256 / TX, kUnroll = UN;
     const int tx = threadIdx.x, ty = threadIdx.y;
     const int64_t col0 = ((int64_t)blockIdx.x * kTX + tx) * V;
     pdl_wait();
@@ -547,8 +550,8 @@ relay_status_t launch_body2d(int32_t storage, const Args2D<Body::NIN, Body::NOUT
 
 // Column sums finished inside the kernel by clusters of kColsumCluster row slices (no partials, no second launch):
 // taken when that many slices per column strip give every SM a block.  A.final / A.scale name the results.  Used for the
-// bodies with three or more streamed inputs; with one or two inputs 8 blocks per strip measured slower than the many
-// short slices of the two-pass form (8192 x 8192 bf16 column sum: 41 us against 30 us).
+// cfg2 gradient body (strips of 32 lanes: two streamed inputs and one streamed result keep enough bytes in flight); the plain
+// column sum, with one streamed input, needs narrower strips and more blocks (launch_colsum_cluster below).
 static bool cluster_sums(int64_t rows, int64_t cols, int32_t storage)
 {
     const int vec = storage == RELAY_BF16 ? 8 : 4;
@@ -565,6 +568,31 @@ relay_status_t launch_body2d_cluster(int32_t storage, const Args2D<Body::NIN, Bo
     A.rows_per_slice = (int)((A.rows + kColsumCluster - 1) / kColsumCluster);
     if (storage == RELAY_BF16) RELAY_CUDA(launch_pdl_cluster(ewise2d_kernel<Body, __nv_bfloat16, true, kColsumCluster>, grid, block, cluster, 0, st, A));
     else RELAY_CUDA(launch_pdl_cluster(ewise2d_kernel<Body, float, false, kColsumCluster>, grid, block, cluster, 0, st, A));
+    return check_launch(what);
+}
+
+// Column sum of ONE streamed input finished in clusters: narrow strips (TX lanes of 16 bytes) so that CL slices per strip
+// still give every SM several blocks, and UN row passes of loads in flight per thread.  Measured on 8192 x 8192 bf16
+// (two-pass form with per-slice partials and a second launch: 29.1 us): strips of 16 lanes (256 bytes of a row), clusters
+// of 8 slices, 4 passes in flight 24.5 us; 8 passes in flight 36.8 us; 8 lanes 29.1 us; 32 lanes 33 us and more; clusters
+// of 4 slices 33.2 us (16 lanes) / 25.2 us (8 lanes).
+constexpr int kColsumStripLanes = 16;
+static bool colsum_in_clusters(int64_t rows, int64_t cols, int32_t storage)
+{
+    const int vec = storage == RELAY_BF16 ? 8 : 4;
+    const int64_t gx = (cols + (int64_t)kColsumStripLanes * vec - 1) / (kColsumStripLanes * vec);
+    return gx * kColsumCluster >= 148 * 2 && rows >= 1024;
+}
+template <typename Body, int CL, int TX, int UN>
+relay_status_t launch_colsum_cluster(int32_t storage, const Args2D<Body::NIN, Body::NOUT> &A0, cudaStream_t st, const char *what)
+{
+    Args2D<Body::NIN, Body::NOUT> A = A0;
+    const int vec = storage == RELAY_BF16 ? 8 : 4;
+    const dim3 block(TX, 256 / TX), cluster(1, CL, 1);
+    const dim3 grid((unsigned)((A.cols + (int64_t)TX * vec - 1) / (TX * vec)), CL);
+    A.rows_per_slice = (int)((A.rows + CL - 1) / CL);
+    if (storage == RELAY_BF16) RELAY_CUDA(launch_pdl_cluster(ewise2d_kernel<Body, __nv_bfloat16, true, CL, TX, UN>, grid, block, cluster, 0, st, A));
+    else RELAY_CUDA(launch_pdl_cluster(ewise2d_kernel<Body, float, false, CL, TX, UN>, grid, block, cluster, 0, st, A));
     return check_launch(what);
 }
 
@@ -683,7 +711,7 @@ extern "C" relay_status_t relay_fused_ewise(const relay_ewise_prog_t *prog, cons
         A.rows = v.rows; A.cols = v.cols; A.aux = 0;
         const int vec = v.storage == RELAY_BF16 ? 8 : 4;
         const int64_t gx = (v.cols + (int64_t)kTX * vec - 1) / (kTX * vec);
-        int ns = (int)std::max<int64_t>(1, std::min<int64_t>((148 * 16) / gx, (v.rows + kTY * kUnroll - 1) / (kTY * kUnroll)));
+        int ns = (int)std::max<int64_t>(1, std::min<int64_t>((148 * 16) / gx, (v.rows + kTY * 4 - 1) / (kTY * 4)));
         return launch_body2d<BodyTanhAffineResidualFwd>(v.storage, A, ns, st, "ewise2d<tanh_affine_residual_fwd>");
     }
 
@@ -897,6 +925,10 @@ extern "C" relay_status_t relay_fused_reduce(const relay_ewise_prog_t *prog, con
         A.in[0] = inputs[0]->data; A.out[0] = nullptr; A.partial[0] = (float *)ws;
         A.rows = v.rows; A.cols = v.cols; A.aux = 0;
         const float scale = specs[0].red_op == RELAY_RED_MEAN ? 1.0f / (float)v.rows : 1.0f;
+        if (colsum_in_clusters(v.rows, v.cols, v.storage)) {
+            A.partial[0] = nullptr; A.final[0] = (float *)outputs[0]->data; A.scale[0] = scale;
+            return launch_colsum_cluster<BodyIdentityColSum, kColsumCluster, kColsumStripLanes, 4>(v.storage, A, st, "ewise2d<identity_colsum>");
+        }
         RELAY_TRY(launch_body2d<BodyIdentityColSum>(v.storage, A, pl.n_slices, st, "ewise2d<identity_colsum>"));
         return launch_colsum_finalize(A.partial[0], pl.n_slices, v.cols, scale, (float *)outputs[0]->data, st);
     }

@@ -138,7 +138,7 @@ RED = {B.RED_SUM: "sum", B.RED_MAX: "max", B.RED_MEAN: "mean"}
 
 @pytest.mark.parametrize("shape,axes", [((300, 512), (0,)), ((300, 512), (1,)), ((37, 29), (0,)), ((37, 29), (1,)),
                                          ((5, 6, 64), (0, 1)), ((5, 6, 64), (2,)), ((5, 6, 7), (0, 2)), ((4, 3, 5, 6), (1, 3)),
-                                         ((3000,), (0,)), ((2, 4096), (0, 1))])
+                                         ((3000,), (0,)), ((2, 4096), (0, 1)), ((1100, 4872), (0,))])
 @pytest.mark.parametrize("tdt", [torch.bfloat16, torch.float32])
 def test_standalone_reduce_all_routes(shape, axes, tdt):
     g = torch.Generator().manual_seed(7)
