@@ -66,7 +66,9 @@ __device__ __forceinline__ void pack_one(const PackJob &j, unsigned i)
     }
 }
 
-template <bool GRAD>
+// NT: channel blocks of 64 that one thread block repacks; the loads of all of them are in flight before the first is
+// transposed (16 * NT KB per block with GRAD, 8 * NT KB without).
+template <bool GRAD, int NT>
 __global__ void __launch_bounds__(256) nchw_to_nhwc_kernel(const __nv_bfloat16 *__restrict__ in, const __nv_bfloat16 *__restrict__ y,
                                                             __nv_bfloat16 *__restrict__ out, int C, int HW, int act,
                                                             float *__restrict__ db_part, const PackJob job)
@@ -79,53 +81,67 @@ __global__ void __launch_bounds__(256) nchw_to_nhwc_kernel(const __nv_bfloat16 *
     }
     // [pixel][channel]; 33 words per row: the scattered 2-byte stores below are at most 2-way conflicted and
     // the 4-byte reads of the write phase are conflict-free
-    __shared__ __align__(16) __nv_bfloat16 tile[64][66];
-    const int n = blockIdx.z, c0 = blockIdx.y * 64, p0 = blockIdx.x * 64;
+    __shared__ __align__(16) __nv_bfloat16 tile[NT][64][66];
+    const int n = blockIdx.z, cb = blockIdx.y * (64 * NT), p0 = blockIdx.x * 64;
     const size_t img = (size_t)n * C * HW;
     pdl_wait();
+    uint4 v[NT][2], yy[GRAD ? NT : 1][2];
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        const int idx = threadIdx.x + i * 256;
-        const int cl = idx >> 3, chunk = idx & 7;
-        const int c = c0 + cl, p = p0 + chunk * 8;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (c < C && p < HW) {
-            const size_t off = img + (size_t)c * HW + p;
-            v = ld_stream(in + off);
-            if (GRAD) {
-                const uint4 yy = ld_stream(y + off);
-                float a[8], b[8];
-                unpack(v, a);
-                unpack(yy, b);
+    for (int t = 0; t < NT; ++t)
 #pragma unroll
-                for (int j = 0; j < 8; ++j) a[j] *= act_grad_from_output(b[j], act);
-                v = pack(a);
+        for (int i = 0; i < 2; ++i) {
+            const int idx = threadIdx.x + i * 256;
+            const int cl = idx >> 3, chunk = idx & 7;
+            const int c = cb + t * 64 + cl, p = p0 + chunk * 8;
+            v[t][i] = make_uint4(0, 0, 0, 0);
+            if (GRAD) yy[GRAD ? t : 0][i] = make_uint4(0, 0, 0, 0);
+            if (c < C && p < HW) {
+                const size_t off = img + (size_t)c * HW + p;
+                v[t][i] = ld_stream(in + off);
+                if (GRAD) yy[GRAD ? t : 0][i] = ld_stream(y + off);
             }
         }
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            tile[chunk * 8 + 2 * j][cl] = __ushort_as_bfloat16((unsigned short)(w[j] & 0xffffu));
-            tile[chunk * 8 + 2 * j + 1][cl] = __ushort_as_bfloat16((unsigned short)(w[j] >> 16));
+    for (int t = 0; t < NT; ++t)
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int idx = threadIdx.x + i * 256;
+            const int cl = idx >> 3, chunk = idx & 7;
+            const int c = cb + t * 64 + cl;
+            uint4 val = v[t][i];
+            if (GRAD) {
+                float a[8], b[8];
+                unpack(val, a);
+                unpack(yy[GRAD ? t : 0][i], b);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) a[j] *= act_grad_from_output(b[j], act);
+                val = pack(a);
+            }
+            const uint32_t w[4] = {val.x, val.y, val.z, val.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                tile[t][chunk * 8 + 2 * j][cl] = __ushort_as_bfloat16((unsigned short)(w[j] & 0xffffu));
+                tile[t][chunk * 8 + 2 * j + 1][cl] = __ushort_as_bfloat16((unsigned short)(w[j] >> 16));
+            }
+            if (GRAD && db_part != nullptr) {          // the 8 lanes that share a channel row combine in a fixed order
+                float r[8];
+                unpack(val, r);
+                float sum = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
+                sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+                sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+                sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+                if (chunk == 0 && c < C) db_part[((size_t)n * gridDim.x + blockIdx.x) * C + c] = sum;
+            }
         }
-        if (GRAD && db_part != nullptr) {          // the 8 lanes that share a channel row combine in a fixed order
-            float r[8];
-            unpack(v, r);
-            float sum = ((r[0] + r[1]) + (r[2] + r[3])) + ((r[4] + r[5]) + (r[6] + r[7]));
-            sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-            sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-            sum += __shfl_xor_sync(0xffffffffu, sum, 4);
-            if (chunk == 0 && c < C) db_part[((size_t)n * gridDim.x + blockIdx.x) * C + c] = sum;
-        }
-    }
     __syncthreads();
+    // 8 * NT lanes write the 128 * NT contiguous bytes of one pixel
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < 2 * NT; ++i) {
         const int idx = threadIdx.x + i * 256;
-        const int pl = idx >> 3, cchunk = idx & 7;           // 8 lanes write the 128 contiguous bytes of one pixel
-        const int c = c0 + cchunk * 8, p = p0 + pl;
+        const int pl = idx / (8 * NT), cchunk = idx % (8 * NT), t = cchunk >> 3;
+        const int c = cb + cchunk * 8, p = p0 + pl;
         if (c < C && p < HW) {
-            const uint32_t *row = reinterpret_cast<const uint32_t *>(&tile[pl][cchunk * 8]);
+            const uint32_t *row = reinterpret_cast<const uint32_t *>(&tile[t][pl][(cchunk & 7) * 8]);
             *reinterpret_cast<uint4 *>(out + ((size_t)n * HW + p) * C + c) = make_uint4(row[0], row[1], row[2], row[3]);
         }
     }
@@ -1203,7 +1219,9 @@ relay_status_t launch_transpose(bool grad, const void *in, const void *y, void *
                                 float *db_part, cudaStream_t st, const void *w = nullptr, void *wf = nullptr, void *wb = nullptr,
                                 int64_t O = 0, int64_t Cw = 0)
 {
-    dim3 grid((unsigned)((HW + 63) / 64), (unsigned)((C + 63) / 64), (unsigned)Nb);
+    static const int nt_env = getenv("RELAY_REPACK_NT") ? atoi(getenv("RELAY_REPACK_NT")) : 1;
+    const int NT = grad ? 1 : nt_env;
+    dim3 grid((unsigned)((HW + 63) / 64), (unsigned)((C + 64 * NT - 1) / (64 * NT)), (unsigned)Nb);
     PackJob job{};
     if (w != nullptr) {
         job.w = (const __nv_bfloat16 *)w; job.wf = (__nv_bfloat16 *)wf; job.wb = (__nv_bfloat16 *)wb;
@@ -1211,8 +1229,12 @@ relay_status_t launch_transpose(bool grad, const void *in, const void *y, void *
         const int64_t per_slice = (int64_t)grid.x * grid.y * 256;
         grid.z += (unsigned)((O * Cw * 9 + per_slice - 1) / per_slice);
     }
-    if (grad) RELAY_CUDA(launch_pdl(nchw_to_nhwc_kernel<true>, grid, dim3(256), 0, st, (const __nv_bfloat16 *)in, (const __nv_bfloat16 *)y, (__nv_bfloat16 *)out, (int)C, (int)HW, act, db_part, job));
-    else RELAY_CUDA(launch_pdl(nchw_to_nhwc_kernel<false>, grid, dim3(256), 0, st, (const __nv_bfloat16 *)in, (const __nv_bfloat16 *)nullptr, (__nv_bfloat16 *)out, (int)C, (int)HW, act, (float *)nullptr, job));
+#define RELAY_REPACK(G, N_) RELAY_CUDA(launch_pdl(nchw_to_nhwc_kernel<G, N_>, grid, dim3(256), 0, st, (const __nv_bfloat16 *)in, (const __nv_bfloat16 *)(G ? y : nullptr), (__nv_bfloat16 *)out, (int)C, (int)HW, act, G ? db_part : (float *)nullptr, job))
+    if (grad) RELAY_REPACK(true, 1);
+    else if (NT == 4) RELAY_REPACK(false, 4);
+    else if (NT == 2) RELAY_REPACK(false, 2);
+    else RELAY_REPACK(false, 1);
+#undef RELAY_REPACK
     return check_launch("nchw_to_nhwc");
 }
 

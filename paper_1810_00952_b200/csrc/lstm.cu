@@ -125,8 +125,11 @@ static relay_status_t lstm_seq(const relay_tensor_t *x, const relay_tensor_t *w_
     RELAY_TRY(check_workspace(ws, ws_bytes, lstm_ws(d)));
     cudaStream_t st = (cudaStream_t)stream;
     if (d.B == 0 || d.H == 0) return RELAY_OK;
-    RELAY_CUDA(cudaMemcpyAsync(c_final->data, c0->data, nbytes(c0), cudaMemcpyDeviceToDevice, st));
+    const bool tc = d.T > 0 && lstm_tc_eligible(d.T, d.B, d.H);
+    // the per-step kernels carry the cell state in c_final; the persistent kernel keeps it in registers and writes c_final itself
+    if (!tc) RELAY_CUDA(cudaMemcpyAsync(c_final->data, c0->data, nbytes(c0), cudaMemcpyDeviceToDevice, st));
     if (d.T == 0) return RELAY_OK;
+    if (tc) RELAY_TRY(launch_lstm_tc_prepare(d.B, d.H, w_hh->data, (char *)ws + lstm_zx_bytes(d), st));
 
     // (1) zx = x W_ih + b for all T*B rows
     float *zx = (float *)ws;
@@ -141,7 +144,7 @@ static relay_status_t lstm_seq(const relay_tensor_t *x, const relay_tensor_t *w_
     RELAY_TRY(launch_gemm(g, st));
 
     // (2) the dependent steps: one persistent kernel when the shape fits it, else one launch per step
-    if (lstm_tc_eligible(d.T, d.B, d.H))
+    if (tc)
         return launch_lstm_tc(d.T, d.B, d.H, zx, w_hh->data, (const float *)h0->data, (const float *)c0->data, (float *)h_all->data,
                               (float *)c_final->data, (char *)ws + lstm_zx_bytes(d), st, timing);
     if (timing) return fail(RELAY_ERR_UNSUPPORTED, "phase cycles are counted by the persistent kernel only; this shape runs one launch per step");

@@ -10,6 +10,9 @@ namespace relay {
 // H / 16 blocks co-resident on the device
 bool lstm_tc_eligible(int64_t T, int64_t B, int64_t H);
 size_t lstm_tc_workspace(int64_t B, int64_t H);
+// launch_lstm_tc_prepare packs W_hh into the blocks' slices and clears the step counters (both in `ws`); it reads nothing that
+// the input projection writes, so the caller enqueues it BEFORE that contraction, whose set-up then overlaps its tail.
+relay_status_t launch_lstm_tc_prepare(int64_t B, int64_t H, const void *w_hh, void *ws, cudaStream_t st);
 // zx: [T*B][4H] fp32 (input projection + bias); runs all T steps.  `timing` (optional, device, 8 entries): block 0 leaves
 // cycle counts summed over the steps: [0] step loop, [1] epilogue warp waiting for the accumulator, [2] epilogue (TMEM
 // read, gates, publish), [3] loader waiting on the grid barrier, [4] loader issuing the step's copies, [5] issuer

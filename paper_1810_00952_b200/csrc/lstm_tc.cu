@@ -315,20 +315,38 @@ lstm_persistent_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_co
     if (warp == 4) { tc::tc_fence_after_sync(); tc::tmem_dealloc(tmem_base, MAX_ISS * NCOL); }
 }
 
-// wp[blk][g*16 + i][k] = w_hh[k][g*H + blk*16 + i]
-__global__ void __launch_bounds__(256) pack_whh_kernel(const __nv_bfloat16 *__restrict__ w_hh, __nv_bfloat16 *__restrict__ wp, int H)
+// wp[blk][g*16 + i][k] = w_hh[k][g*H + blk*16 + i]: block (blk, k-block of 64) moves a 64 x 64 tile with 16-byte accesses on
+// both sides (a source row holds four runs of 16 columns, one per gate block; a packed row is 64 consecutive k).  Block
+// (0, 0) also clears the step counters, so the call needs no memset of its own.
+__global__ void __launch_bounds__(256) pack_whh_kernel(const __nv_bfloat16 *__restrict__ w_hh, __nv_bfloat16 *__restrict__ wp, int H,
+                                                        unsigned int *__restrict__ counter, int n_counter)
 {
-    __shared__ __nv_bfloat16 tile[64][66];     // [k local][column local]
+    __shared__ __align__(16) __nv_bfloat16 tile[64][66];     // [column local n][k local]; 33 words per row
     const int blk = blockIdx.x, k0 = blockIdx.y * 64;
-    for (int e = threadIdx.x; e < 64 * 64; e += 256) {
-        const int kl = e >> 6, n = e & 63;
-        const int g = n >> 4, i = n & 15;
-        tile[kl][n] = w_hh[(size_t)(k0 + kl) * 4 * H + (size_t)g * H + blk * 16 + i];
+    if (blk == 0 && k0 == 0)
+        for (int e = threadIdx.x; e < n_counter; e += 256) counter[e] = 0u;
+    uint4 v[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const int idx = threadIdx.x + r * 256, kl = idx >> 3, g = (idx >> 1) & 3, half = idx & 1;
+        v[r] = *reinterpret_cast<const uint4 *>(w_hh + (size_t)(k0 + kl) * 4 * H + (size_t)g * H + blk * 16 + half * 8);
+    }
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const int idx = threadIdx.x + r * 256, kl = idx >> 3, g = (idx >> 1) & 3, half = idx & 1;
+        const uint32_t w[4] = {v[r].x, v[r].y, v[r].z, v[r].w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            tile[g * 16 + half * 8 + 2 * q][kl] = __ushort_as_bfloat16((unsigned short)(w[q] & 0xffffu));
+            tile[g * 16 + half * 8 + 2 * q + 1][kl] = __ushort_as_bfloat16((unsigned short)(w[q] >> 16));
+        }
     }
     __syncthreads();
-    for (int e = threadIdx.x; e < 64 * 64; e += 256) {
-        const int n = e >> 6, kl = e & 63;
-        wp[((size_t)blk * 64 + n) * H + k0 + kl] = tile[kl][n];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const int idx = threadIdx.x + r * 256, n = idx >> 3, kc = idx & 7;
+        const uint32_t *row = reinterpret_cast<const uint32_t *>(&tile[n][kc * 8]);
+        *reinterpret_cast<uint4 *>(wp + ((size_t)blk * 64 + n) * H + k0 + kc * 8) = make_uint4(row[0], row[1], row[2], row[3]);
     }
 }
 
@@ -349,6 +367,15 @@ size_t lstm_tc_workspace(int64_t B, int64_t H)
     return align_up((size_t)H * 4 * H * 2, 1024) /* packed W_hh */ + align_up((size_t)2 * B * H * 2, 1024) /* exchange */ + 1024 /* counters */;
 }
 
+relay_status_t launch_lstm_tc_prepare(int64_t B, int64_t H, const void *w_hh, void *ws, cudaStream_t st)
+{
+    char *base = (char *)ws;
+    __nv_bfloat16 *wp = (__nv_bfloat16 *)base;
+    unsigned int *counter = (unsigned int *)(base + align_up((size_t)H * 4 * H * 2, 1024) + align_up((size_t)2 * B * H * 2, 1024));
+    pack_whh_kernel<<<dim3((unsigned)(H / UNITS), (unsigned)(H / 64)), 256, 0, st>>>((const __nv_bfloat16 *)w_hh, wp, (int)H, counter, 256);
+    return check_launch("pack_whh");
+}
+
 relay_status_t launch_lstm_tc(int64_t T, int64_t B, int64_t H, const float *zx, const void *w_hh, const float *h0, const float *c0,
                               float *h_all, float *c_final, void *ws, cudaStream_t st, long long *timing)
 {
@@ -357,9 +384,6 @@ relay_status_t launch_lstm_tc(int64_t T, int64_t B, int64_t H, const float *zx, 
     __nv_bfloat16 *hq = (__nv_bfloat16 *)(base + align_up((size_t)H * 4 * H * 2, 1024));
     unsigned int *counter = (unsigned int *)((char *)hq + align_up((size_t)2 * B * H * 2, 1024));
     const int n_blocks = (int)(H / UNITS);
-    pack_whh_kernel<<<dim3(n_blocks, (unsigned)(H / 64)), 256, 0, st>>>((const __nv_bfloat16 *)w_hh, wp, (int)H);
-    RELAY_TRY(check_launch("pack_whh"));
-    RELAY_CUDA(cudaMemsetAsync(counter, 0, 1024, st));
     CUtensorMap tm_w, tm_h0, tm_h1;
     RELAY_TRY(make_tmap_2d_bf16(&tm_w, wp, (uint64_t)H, (uint64_t)n_blocks * NCOL, (uint64_t)H, BK, NCOL));
     // split the batch into groups of rows while every block still fits on its own SM (at least 8 rows a group)
