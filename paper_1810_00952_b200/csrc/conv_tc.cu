@@ -66,6 +66,34 @@ __device__ __forceinline__ void pack_one(const PackJob &j, unsigned i)
     }
 }
 
+// Transposition tile of the repack kernels: 64 pixels x 64 channels as [pixel][channel pair] 32-bit words, 33 words per row.
+// A thread arrives with 16 bytes = 8 pixels (chunk * 8 ..) of channel `cl`; the lane 8 further on holds the same pixels of
+// channel cl ^ 1.  The two exchange half of their words, so that each ends up with four (even channel, odd channel) words
+// -- the even-channel lane for the chunk's first four pixels, the odd-channel lane for the last four -- and stores 4 words
+// instead of 8 half-words.  Column index XOR 2 for the upper half of the pixels: with it the 32 lanes of a store hit 32
+// different banks (without it pixels 32 apart collide), and the reader undoes it by swapping the halves of its 16 bytes.
+// Every lane of the warp must call tile_put together.
+__device__ __forceinline__ void tile_put(uint32_t (*tile)[33], int cl, int chunk, const uint4 &val)
+{
+    const bool odd = cl & 1;
+    const uint32_t r0 = __shfl_xor_sync(0xffffffffu, odd ? val.x : val.z, 8);
+    const uint32_t r1 = __shfl_xor_sync(0xffffffffu, odd ? val.y : val.w, 8);
+    const uint32_t e0 = odd ? r0 : val.x, e1 = odd ? r1 : val.y;      // even channel's two words (pixels 0,1 | 2,3 of this lane's four)
+    const uint32_t o0 = odd ? val.z : r0, o1 = odd ? val.w : r1;      // odd channel's
+    const int px = chunk * 8 + (odd ? 4 : 0), col = (cl >> 1) ^ ((chunk >> 2) << 1);
+    tile[px + 0][col] = __byte_perm(e0, o0, 0x5410);
+    tile[px + 1][col] = __byte_perm(e0, o0, 0x7632);
+    tile[px + 2][col] = __byte_perm(e1, o1, 0x5410);
+    tile[px + 3][col] = __byte_perm(e1, o1, 0x7632);
+}
+// the 8 channels cchunk * 8 .. of pixel pl
+__device__ __forceinline__ uint4 tile_get(const uint32_t (*tile)[33], int pl, int cchunk)
+{
+    const uint32_t *row = &tile[pl][cchunk * 4];
+    const uint32_t a = row[0], b = row[1], c = row[2], d = row[3];
+    return (pl & 32) ? make_uint4(c, d, a, b) : make_uint4(a, b, c, d);
+}
+
 // NT: channel blocks of 64 that one thread block repacks; the loads of all of them are in flight before the first is
 // transposed (16 * NT KB per block with GRAD, 8 * NT KB without).
 template <bool GRAD, int NT>
@@ -79,9 +107,7 @@ __global__ void __launch_bounds__(256) nchw_to_nhwc_kernel(const __nv_bfloat16 *
         pack_one(job, blk * 256u + threadIdx.x);
         return;
     }
-    // [pixel][channel]; 33 words per row: the scattered 2-byte stores below are at most 2-way conflicted and
-    // the 4-byte reads of the write phase are conflict-free
-    __shared__ __align__(16) __nv_bfloat16 tile[NT][64][66];
+    __shared__ uint32_t tile[NT][64][33];
     const int n = blockIdx.z, cb = blockIdx.y * (64 * NT), p0 = blockIdx.x * 64;
     const size_t img = (size_t)n * C * HW;
     pdl_wait();
@@ -117,12 +143,7 @@ __global__ void __launch_bounds__(256) nchw_to_nhwc_kernel(const __nv_bfloat16 *
                 for (int j = 0; j < 8; ++j) a[j] *= act_grad_from_output(b[j], act);
                 val = pack(a);
             }
-            const uint32_t w[4] = {val.x, val.y, val.z, val.w};
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                tile[t][chunk * 8 + 2 * j][cl] = __ushort_as_bfloat16((unsigned short)(w[j] & 0xffffu));
-                tile[t][chunk * 8 + 2 * j + 1][cl] = __ushort_as_bfloat16((unsigned short)(w[j] >> 16));
-            }
+            tile_put(tile[t], cl, chunk, val);
             if (GRAD && db_part != nullptr) {          // the 8 lanes that share a channel row combine in a fixed order
                 float r[8];
                 unpack(val, r);
@@ -140,10 +161,7 @@ __global__ void __launch_bounds__(256) nchw_to_nhwc_kernel(const __nv_bfloat16 *
         const int idx = threadIdx.x + i * 256;
         const int pl = idx / (8 * NT), cchunk = idx % (8 * NT), t = cchunk >> 3;
         const int c = cb + cchunk * 8, p = p0 + pl;
-        if (c < C && p < HW) {
-            const uint32_t *row = reinterpret_cast<const uint32_t *>(&tile[t][pl][(cchunk & 7) * 8]);
-            *reinterpret_cast<uint4 *>(out + ((size_t)n * HW + p) * C + c) = make_uint4(row[0], row[1], row[2], row[3]);
-        }
+        if (c < C && p < HW) *reinterpret_cast<uint4 *>(out + ((size_t)n * HW + p) * C + c) = tile_get(tile[t], pl, cchunk & 7);
     }
 }
 
@@ -172,7 +190,7 @@ struct RepackStream {
 constexpr int kPackPerUnit = 4096;
 
 template <bool GRAD>
-__device__ __forceinline__ void repack_unit(const RepackJob &j, int HW, int pbx, int n, int pb, __nv_bfloat16 (*tile)[66])
+__device__ __forceinline__ void repack_unit(const RepackJob &j, int HW, int pbx, int n, int pb, uint32_t (*tile)[33])
 {
     // channel blocks whose loads are in flight together: 8 loads of 16 bytes per thread either way
     constexpr int NT = GRAD ? 2 : 4;
@@ -210,12 +228,7 @@ __device__ __forceinline__ void repack_unit(const RepackJob &j, int HW, int pbx,
                     for (int q = 0; q < 8; ++q) a[q] *= act_grad_from_output(b[q], j.act);
                     val = pack(a);
                 }
-                const uint32_t w[4] = {val.x, val.y, val.z, val.w};
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    tile[chunk * 8 + 2 * q][cl] = __ushort_as_bfloat16((unsigned short)(w[q] & 0xffffu));
-                    tile[chunk * 8 + 2 * q + 1][cl] = __ushort_as_bfloat16((unsigned short)(w[q] >> 16));
-                }
+                tile_put(tile, cl, chunk, val);
                 if (GRAD && j.db_part != nullptr) {      // the 8 lanes that share a channel row combine in a fixed order
                     float r[8];
                     unpack(val, r);
@@ -231,10 +244,7 @@ __device__ __forceinline__ void repack_unit(const RepackJob &j, int HW, int pbx,
             for (int i = 0; i < 2; ++i) {
                 const int idx = tid + i * 256, pl = idx >> 3, cchunk = idx & 7;
                 const int c = c0 + cchunk * 8, p = p0 + pl;
-                if (c < j.C && p < HW) {
-                    const uint32_t *row = reinterpret_cast<const uint32_t *>(&tile[pl][cchunk * 8]);
-                    *reinterpret_cast<uint4 *>(j.out + ((size_t)n * HW + p) * j.C + c) = make_uint4(row[0], row[1], row[2], row[3]);
-                }
+                if (c < j.C && p < HW) *reinterpret_cast<uint4 *>(j.out + ((size_t)n * HW + p) * j.C + c) = tile_get(tile, pl, cchunk);
             }
             __syncthreads();
         }
@@ -243,7 +253,7 @@ __device__ __forceinline__ void repack_unit(const RepackJob &j, int HW, int pbx,
 
 __global__ void __launch_bounds__(256, 3) repack_stream_kernel(const RepackStream S)
 {
-    __shared__ __align__(16) __nv_bfloat16 tile[64][66];
+    __shared__ uint32_t tile[64][33];
     // first the stream's earlier work must be complete (this kernel overwrites scratch that it may still read); only
     // then may the consumer start: whatever it reads that this kernel does not produce is then final as well
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -1219,8 +1229,9 @@ relay_status_t launch_transpose(bool grad, const void *in, const void *y, void *
                                 float *db_part, cudaStream_t st, const void *w = nullptr, void *wf = nullptr, void *wb = nullptr,
                                 int64_t O = 0, int64_t Cw = 0)
 {
-    static const int nt_env = getenv("RELAY_REPACK_NT") ? atoi(getenv("RELAY_REPACK_NT")) : 1;
-    const int NT = grad ? 1 : nt_env;
+    // one channel block per thread block: two per block measured the same (97.4 us for the forward group of cfg4 either
+    // way), four slower (102.6 us: fewer blocks fit an SM)
+    constexpr int NT = 1;
     dim3 grid((unsigned)((HW + 63) / 64), (unsigned)((C + 64 * NT - 1) / (64 * NT)), (unsigned)Nb);
     PackJob job{};
     if (w != nullptr) {
@@ -1230,10 +1241,8 @@ relay_status_t launch_transpose(bool grad, const void *in, const void *y, void *
         grid.z += (unsigned)((O * Cw * 9 + per_slice - 1) / per_slice);
     }
 #define RELAY_REPACK(G, N_) RELAY_CUDA(launch_pdl(nchw_to_nhwc_kernel<G, N_>, grid, dim3(256), 0, st, (const __nv_bfloat16 *)in, (const __nv_bfloat16 *)(G ? y : nullptr), (__nv_bfloat16 *)out, (int)C, (int)HW, act, G ? db_part : (float *)nullptr, job))
-    if (grad) RELAY_REPACK(true, 1);
-    else if (NT == 4) RELAY_REPACK(false, 4);
-    else if (NT == 2) RELAY_REPACK(false, 2);
-    else RELAY_REPACK(false, 1);
+    if (grad) RELAY_REPACK(true, NT);
+    else RELAY_REPACK(false, NT);
 #undef RELAY_REPACK
     return check_launch("nchw_to_nhwc");
 }
