@@ -24,7 +24,7 @@ template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v
 template <typename TIN, typename TOUT, bool FAST, int TM, int TN>
 __global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmDesc g)
 {
-    static_assert(TM == 1 || TN == 4, "the large tile is 64 x 64");
+    static_assert(TM == 1 || TN == 4, "the large tiles are 64 x 64 and 128 x 64");
     constexpr int BM = 16 * TM, BN = 16 * TN;
     constexpr int A_LD = BM * BK / 256, B_LD = BN * BK / 256;
     __shared__ __align__(16) float As[BK][BM + 4];     // rows of whole 16-byte vectors: a thread's four values are one load
@@ -37,23 +37,33 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmDesc g)
     constexpr bool F64 = sizeof(TIN) == 4;
     using Acc = typename std::conditional<F64, PairSum, float>::type;
     Acc acc[TM][TN] = {};
-    // loader index order follows the unit stride of each operand so that loads coalesce
+    // loader index order follows the unit stride of each operand so that loads coalesce.  A thread's loads of one operand
+    // are a fixed distance apart (element e = tid + 256 i), so one base offset per operand and a constant step address them;
+    // only the k-range test changes from k-block to k-block.
     const bool a_k_fast = g.a_sk == 1, b_n_fast = g.b_sn == 1;
+    const int a_m = a_k_fast ? tid / BK : tid % BM, a_k = a_k_fast ? tid % BK : tid / BM;          // element 0 of this thread
+    const int b_n = b_n_fast ? tid % BN : tid / BK, b_k = b_n_fast ? tid / BN : tid % BK;
+    constexpr int A_STEP_M = 256 / BK, A_STEP_K = 256 / BM;                                         // per i, k-fast / m-fast order
+    constexpr int B_STEP_K = 256 / BN, B_STEP_N = 256 / BK;
+    static_assert(256 % BK == 0 && 256 % BM == 0 && 256 % BN == 0, "loader steps");
+    const TIN *a_base = A + (m0 + a_m) * g.a_sm + (int64_t)a_k * g.a_sk;
+    const TIN *b_base = B + (int64_t)b_k * g.b_sk + (n0 + b_n) * g.b_sn;
+    const int64_t a_step = a_k_fast ? (int64_t)A_STEP_M * g.a_sm : (int64_t)A_STEP_K * g.a_sk;
+    const int64_t b_step = b_n_fast ? (int64_t)B_STEP_K * g.b_sk : (int64_t)B_STEP_N * g.b_sn;
     float ra[A_LD], rb[B_LD];
     auto load_tiles = [&](int64_t k0) {
+        const TIN *pa = a_base + k0 * g.a_sk, *pb = b_base + k0 * g.b_sk;
 #pragma unroll
         for (int i = 0; i < A_LD; ++i) {
-            const int e = tid + i * 256;
-            const int mm = a_k_fast ? e / BK : e % BM, kk = a_k_fast ? e % BK : e / BM;
-            const int64_t m = m0 + mm, k = k0 + kk;
-            ra[i] = (m < g.M && k < g.K && relay_in_bounds(&A[m * g.a_sm + k * g.a_sk], sizeof(TIN))) ? to_f<TIN>(A[m * g.a_sm + k * g.a_sk]) : 0.0f;
+            const int mm = a_k_fast ? a_m + i * A_STEP_M : a_m, kk = a_k_fast ? a_k : a_k + i * A_STEP_K;
+            const TIN *q = pa + i * a_step;
+            ra[i] = (m0 + mm < g.M && k0 + kk < g.K && relay_in_bounds(q, sizeof(TIN))) ? to_f<TIN>(*q) : 0.0f;
         }
 #pragma unroll
         for (int i = 0; i < B_LD; ++i) {
-            const int e = tid + i * 256;
-            const int nn = b_n_fast ? e % BN : e / BK, kk = b_n_fast ? e / BN : e % BK;
-            const int64_t n = n0 + nn, k = k0 + kk;
-            rb[i] = (n < g.N && k < g.K && relay_in_bounds(&B[k * g.b_sk + n * g.b_sn], sizeof(TIN))) ? to_f<TIN>(B[k * g.b_sk + n * g.b_sn]) : 0.0f;
+            const int nn = b_n_fast ? b_n : b_n + i * B_STEP_N, kk = b_n_fast ? b_k + i * B_STEP_K : b_k;
+            const TIN *q = pb + i * b_step;
+            rb[i] = (n0 + nn < g.N && k0 + kk < g.K && relay_in_bounds(q, sizeof(TIN))) ? to_f<TIN>(*q) : 0.0f;
         }
     };
     load_tiles(0);
@@ -78,9 +88,12 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const GemmDesc g)
 #pragma unroll
                 for (int kk = ks; kk < ks + KSUB; ++kk) {
                     float av[TM], bv[TN];
-                    if constexpr (TM == 4) {
-                        const float4 a4 = *reinterpret_cast<const float4 *>(&As[kk][tm]);
-                        av[0] = a4.x; av[1] = a4.y; av[2] = a4.z; av[3] = a4.w;
+                    if constexpr (TM % 4 == 0) {
+#pragma unroll
+                        for (int q = 0; q < TM / 4; ++q) {
+                            const float4 a4 = *reinterpret_cast<const float4 *>(&As[kk][tm + 4 * q]);
+                            av[4 * q] = a4.x; av[4 * q + 1] = a4.y; av[4 * q + 2] = a4.z; av[4 * q + 3] = a4.w;
+                        }
                     } else {
 #pragma unroll
                         for (int i = 0; i < TM; ++i) av[i] = As[kk][tm + i];
@@ -162,7 +175,10 @@ relay_status_t launch_gemm_simt(const GemmDesc &g, cudaStream_t st)
     // The largest tile whose grid still gives every SM a block: with few warps on an SM a block's time goes to waiting
     // for its own shared-memory reads, so while SMs are idle more and lighter blocks finish sooner.
     auto tiles = [&](int bm, int bn) { return ((g.M + bm - 1) / bm) * ((g.N + bn - 1) / bn); };
-    if (g.M > 16 && tiles(64, 64) >= 2 * 148) return launch_tile<4, 4>(g, st);
+    // 64 x 64 as soon as its grid gives every SM a block (two fit an SM): 1024^3 fp32 runs at 17 TFLOP/s on it against 10 on
+    // 16 x 64 tiles.  A 128 x 64 tile (8 x 4 per thread) was measured too: 19 TFLOP/s at 1024^3, no gain at 2048^3 (its 235
+    // registers leave one block per SM) and far slower on small outputs, so it is not used.
+    if (g.M > 16 && tiles(64, 64) >= 148) return launch_tile<4, 4>(g, st);
     if (tiles(16, 64) >= 148) return launch_tile<1, 4>(g, st);
     if (tiles(16, 32) >= 148) return launch_tile<1, 2>(g, st);
     return launch_tile<1, 1>(g, st);
