@@ -806,7 +806,7 @@ def main():
     # LSTM sequence and its gradient program: tensor-core work on a chain of T dependent steps; the fraction of the
     # tensor peak is reported for the record (the chain, not the tensor pipe, bounds them)
     for key, name in (("cfg5.lstm", "relay_lstm_cell_seq (zx contraction + lstm_persistent_kernel, T=128 dependent steps)"),
-                      ("cfg5.lstm_grad", "relay_lstm_cell_seq_grad (recompute + lstm_grad_persistent_kernel + dx/dW contractions)")):
+                      ("cfg5.lstm_grad", "relay_lstm_cell_seq_grad (recompute + lstm_grad_cluster_kernel + dx/dW contractions)")):
         if key in table:
             a = table[key]["tflops"]
             rooflines[name] = {"bound": "tensor", "achieved": a, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": a / peaks["bf16_tflops"],
