@@ -26,32 +26,46 @@ template <typename T> __device__ __forceinline__ void st_f(T *p, int64_t i, floa
     else p[i] = v;
 }
 
-// Copies n elements of a 16-byte aligned global array into shared memory as floats, dst[perm(i)] = src[i], with a
-// thread's loads all in flight before its first store (up to 16 elements per thread in one round trip).
-template <typename T, typename Perm>
-__device__ __forceinline__ void stage(const T *__restrict__ src, float *dst, int n, Perm perm)
-{
-    if constexpr (sizeof(T) == 4) {
-        const int n4 = n >> 2;
-        for (int base = 0; base < n4; base += 4 * 256) {
-            float4 v[4];
+// Copies n elements of a 16-byte aligned global array into shared memory as floats, dst[perm(i)] = src[i], in two
+// phases so that the loads of SEVERAL operands are in flight together: `begin` issues a thread's loads of the first
+// 4 * 256 vectors (4096 fp32 elements, enough for every operand of the tiny layer), `end` stores them and copies whatever
+// is left the plain way.  A kernel calls begin for all its operands, then end for all: one memory round trip in all.
+template <typename T>
+struct Stage {
+    float4 v[4];
+    __device__ __forceinline__ void begin(const T *__restrict__ src, int n)
+    {
+        if constexpr (sizeof(T) == 4) {
+            const int n4 = n >> 2;
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                const int i4 = base + u * 256 + threadIdx.x;
+                const int i4 = u * 256 + threadIdx.x;
                 if (i4 < n4 && relay_in_bounds(reinterpret_cast<const float4 *>(src) + i4, 16)) v[u] = reinterpret_cast<const float4 *>(src)[i4];
                 else v[u] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
             }
+        }
+    }
+    template <typename Perm>
+    __device__ __forceinline__ void end(const T *__restrict__ src, float *dst, int n, Perm perm)
+    {
+        if constexpr (sizeof(T) == 4) {
+            const int n4 = n >> 2;
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                const int i4 = base + u * 256 + threadIdx.x;
+                const int i4 = u * 256 + threadIdx.x;
                 if (i4 < n4) { dst[perm(4 * i4)] = v[u].x; dst[perm(4 * i4 + 1)] = v[u].y; dst[perm(4 * i4 + 2)] = v[u].z; dst[perm(4 * i4 + 3)] = v[u].w; }
             }
+            for (int i4 = 4 * 256 + threadIdx.x; i4 < n4; i4 += 256) {
+                float4 r = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                if (relay_in_bounds(reinterpret_cast<const float4 *>(src) + i4, 16)) r = reinterpret_cast<const float4 *>(src)[i4];
+                dst[perm(4 * i4)] = r.x; dst[perm(4 * i4 + 1)] = r.y; dst[perm(4 * i4 + 2)] = r.z; dst[perm(4 * i4 + 3)] = r.w;
+            }
+            for (int i = 4 * n4 + threadIdx.x; i < n; i += 256) dst[perm(i)] = ld_f(src, i);
+        } else {
+            for (int i = threadIdx.x; i < n; i += 256) dst[perm(i)] = ld_f(src, i);
         }
-        for (int i = 4 * n4 + threadIdx.x; i < n; i += 256) dst[perm(i)] = ld_f(src, i);
-    } else {
-        for (int i = threadIdx.x; i < n; i += 256) dst[perm(i)] = ld_f(src, i);
     }
-}
+};
 
 // sum over j < n of a[j * sa] * b[j * sb]
 __device__ __forceinline__ float dot_runs(const float *a, int sa, const float *b, int sb, int n)
@@ -74,13 +88,19 @@ __global__ void __launch_bounds__(256) dense_small_fwd_kernel(const T *__restric
     float *xs = sm, *ws = sm + M * K;                 // xs[m][k], ws[k][n]
     pdl_wait();
     auto same = [](int i) { return i; };
-    stage(x, xs, M * K, same);
-    stage(w, ws, K * N, same);
+    Stage<T> sx, sw;
+    sx.begin(x, M * K);
+    sw.begin(w, K * N);
+    // the bias of this thread's first output travels with the operands
+    float b0 = 0.0f;
+    if (bias && (int)threadIdx.x < M * N) b0 = bias_bf16 ? ld_f((const __nv_bfloat16 *)bias, threadIdx.x % N) : ld_f((const float *)bias, threadIdx.x % N);
+    sx.end(x, xs, M * K, same);
+    sw.end(w, ws, K * N, same);
     __syncthreads();
     for (int o = threadIdx.x; o < M * N; o += 256) {
         const int m = o / N, n = o - m * N;
         float z = dot_runs(xs + m * K, 1, ws + n, N, K);
-        if (bias) z += bias_bf16 ? ld_f((const __nv_bfloat16 *)bias, n) : ld_f((const float *)bias, n);
+        if (bias) z += o == (int)threadIdx.x ? b0 : bias_bf16 ? ld_f((const __nv_bfloat16 *)bias, n) : ld_f((const float *)bias, n);
         st_f(y, o, act_fwd<FAST>(z, act));
     }
 }
@@ -95,10 +115,12 @@ __global__ void __launch_bounds__(256) dense_small_grad_kernel(const T *__restri
     float *xs = sm, *ws = xs + M * K, *dz = ws + K * NP;   // xs[m][k], ws[k][n], dz[m][n]
     pdl_wait();
     float *ys = dz + M * N;                             // the saved output, until dZ is formed
-    stage(x, xs, M * K, [](int i) { return i; });
-    stage(w, ws, K * N, [N, NP](int i) { return (i / N) * NP + i % N; });
-    stage(dy, dz, M * N, [](int i) { return i; });
-    stage(y, ys, M * N, [](int i) { return i; });
+    Stage<T> sx, sw, sdy, sy;
+    sx.begin(x, M * K); sw.begin(w, K * N); sdy.begin(dy, M * N); sy.begin(y, M * N);
+    sx.end(x, xs, M * K, [](int i) { return i; });
+    sw.end(w, ws, K * N, [N, NP](int i) { return (i / N) * NP + i % N; });
+    sdy.end(dy, dz, M * N, [](int i) { return i; });
+    sy.end(y, ys, M * N, [](int i) { return i; });
     __syncthreads();
     for (int i = threadIdx.x; i < M * N; i += 256) {
         float v = dz[i] * act_grad_from_output(ys[i], act);
