@@ -16,6 +16,10 @@ struct GemmDesc {
     int32_t out_dtype = RELAY_F32;                  // dtype of C
     const void *bias = nullptr; int32_t bias_dtype = RELAY_F32;  // per column n, or nullptr
     int32_t act = RELAY_ACT_NONE;
+    // > 0: the N columns are the pre-activations of an LSTM cell in four blocks of this many columns [ i | f | g | o ] and the
+    // epilogue stores the activated gates (tanh for g, logistic for the others).  Only launch_gemm_tc2 implements it; the
+    // caller checks gemm_tc_eligible && gemm_tc2_eligible first and calls it directly.
+    int64_t gate_block = 0;
 };
 
 // Picks the tensor-core kernel when the description fits it, else the SIMT kernel (both on the

@@ -141,7 +141,15 @@ __device__ __forceinline__ void finish_group(const Params &p, const CUtensorMap 
         for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
     }
     if (TRANSC) {                                        // tanh / sigmoid: their own instantiation (they need many registers)
-        if (p.act == RELAY_ACT_TANH) {
+        if (p.gate_block > 0) {                          // LSTM gates: a 32-column group lies inside one gate block (warp-uniform)
+            if (nc / p.gate_block == 2) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = 1.0f - __fdividef(2.0f, 1.0f + __expf(2.0f * v[j]));
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = __fdividef(1.0f, 1.0f + __expf(-v[j]));
+            }
+        } else if (p.act == RELAY_ACT_TANH) {
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = OUT_F32 ? tanh_<false>(v[j]) : tanh_<true>(v[j]);
         } else {
@@ -460,6 +468,7 @@ relay_status_t launch_gemm_tc2(const GemmDesc &g, int sms, cudaStream_t st)
     p.M = (int)g.M; p.N = (int)g.N; p.K = (int)g.K;
     p.c = g.c; p.ldc = g.ldc;
     p.bias = g.bias; p.bias_bf16 = g.bias_dtype == RELAY_BF16; p.act = g.act; p.out_f32 = f32;
+    p.gate_block = (int)g.gate_block;
     p.tiles_m = (int)((g.M + 255) / 256); p.tiles_n = (int)((g.N + BN - 1) / BN); p.k_blocks = (int)((g.K + BK - 1) / BK);
     p.err = device_error_word();
     if (!p.err) return fail(RELAY_ERR_CUDA, "no device error word");
@@ -480,7 +489,9 @@ relay_status_t launch_gemm_tc2(const GemmDesc &g, int sms, cudaStream_t st)
         p.tail_split = (rem > 0 && 2 * rem <= pairs) ? 2 : 1;
         p.full_tiles = p.tail_split == 2 ? narrow - rem : narrow;
     }
-    const bool transc = g.act == RELAY_ACT_TANH || g.act == RELAY_ACT_SIGMOID;
+    if (g.gate_block > 0 && (g.gate_block % 32 != 0 || g.N != 4 * g.gate_block))
+        return fail(RELAY_ERR_UNSUPPORTED, "gate blocks of %lld columns over N = %lld", (long long)g.gate_block, (long long)g.N);
+    const bool transc = g.act == RELAY_ACT_TANH || g.act == RELAY_ACT_SIGMOID || g.gate_block > 0;
 #define LAUNCH3(AMN, BMN, TR)                                                                                               \
     do {                                                                                                                    \
         RELAY_CUDA(cudaFuncSetAttribute(gemm_tc2_kernel<AMN, BMN, TR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES)); \

@@ -22,6 +22,9 @@ struct Params {
     // are cut into tail_split column parts
     int wide_units, full_tiles, tail_split;
     int *err;
+    // > 0 (two-SM kernel only): the columns are LSTM pre-activations in blocks of this many columns [ i | f | g | o ]; the
+    // epilogue applies tanh to block 2 and the logistic function to the others (`act` is ignored)
+    int gate_block;
 };
 
 // Bias values of up to 256 columns starting at n0, one 32-column group per register: lane j holds the bias of
