@@ -123,7 +123,6 @@ lstm_grad_cluster_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
              *xfull = bars + 2 * MAX_STAGES + 2;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * MAX_STAGES + 3);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
-    unsigned int *arrived = tmem_slot + 2;                        // worker warps through with the current step (running count)
 
     const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // provably warp-uniform
     const int ks = (int)tc::cluster_ctarank();                    // = blockIdx.x % KS
@@ -140,7 +139,6 @@ lstm_grad_cluster_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
         tc::mbar_init(tmem_full, p.n_iss);
         tc::mbar_init(xfull, 1);                                  // armed once per step with the bytes the four blocks send
         *abort_flag = 0;
-        *arrived = 0;
         tc::fence_barrier_init();
         tc::prefetch_tmap(&tm_w);
         tc::prefetch_tmap(&tm_dz);
@@ -197,8 +195,8 @@ lstm_grad_cluster_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                     }
                 }
             }
+            int ok = 1;                                    // a warp whose wait gave up skips the step's work but still meets the others
             if (s > 0) {
-                int ok = 1;
                 if (lane == 0) ok = tc::mbar_wait(tmem_full, (s - 1) & 1, abort_flag, p.err, tc::ERR_WAIT_TMEM_FULL) ? 1 : 0;
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (ok) {
@@ -222,11 +220,10 @@ lstm_grad_cluster_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                     if (lane == 0) ok = mbar_wait_cluster(xfull, (s - 1) & 1, abort_flag, p.err, tc::ERR_WAIT_EXCHANGE) ? 1 : 0;
                     ok = __shfl_sync(0xffffffffu, ok, 0);
                 }
-                if (!ok) break;
                 __syncwarp();
 #pragma unroll
                 for (int i = 0; i < MAX_PAIRS; ++i) {
-                    if (live[i]) {
+                    if (ok && live[i]) {
                         const float *xs = xbuf + slot_index(threadIdx.x & (QU - 1), row[i], p.n_pad);
                         const int qs = QU * p.n_pad;
                         const float rec = (xs[0] + xs[qs]) + (xs[2 * qs] + xs[3 * qs]);
@@ -234,12 +231,12 @@ lstm_grad_cluster_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                         else dh[i] += rec;
                     }
                 }
-                if (s == p.T) break;
-                if (threadIdx.x == 0) tc::mbar_expect_tx(xfull, x_bytes);   // the phase just seen complete is over: arm the next one
+                if (s == p.T) break;                        // the last pass only produces dh0: every warp leaves here
+                if (ok && threadIdx.x == 0) tc::mbar_expect_tx(xfull, x_bytes);   // the phase just seen complete is over: arm the next one
             }
 #pragma unroll
             for (int i = 0; i < MAX_PAIRS; ++i) {
-                if (live[i]) {
+                if (ok && live[i]) {
                     float dzv[4];
                     lstm_gate_grads(gt[i][0], gt[i][1], gt[i][2], gt[i][3], c_cur[i], c_prev[i], dh[i], dc[i], dzv);
                     c_cur[i] = c_prev[i];
@@ -248,18 +245,18 @@ lstm_grad_cluster_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                     for (int g = 0; g < 4; ++g) drow[(size_t)g * p.H] = __float2bfloat16_rn(dzv[g]);
                 }
             }
-            // dZ[t] is read by TMA (async proxy) in the other blocks: fence the generic stores for it.  The warp barrier orders the
-            // warp's stores (and its reads of the exchange slots, which the next step overwrites) before lane 0's count in shared
-            // memory; the counts form a release sequence, so the warp that comes last has all sixteen warps' stores before its
-            // ONE release on the group's counter (arrivals on one address are served one after the other: sixteen per block
-            // cost more than the product itself)
+            // dZ[t] is read by TMA (async proxy) in the other blocks: every thread fences its generic stores for it.  Then the
+            // sixteen warps meet at a barrier (which also orders their reads of the exchange slots, overwritten in the next
+            // step, before the arrival) and ONE thread releases the group's counter: the release is cumulative over what the
+            // barrier ordered before it.  Arrivals on one address are served one after the other (sixteen per block cost more
+            // than the product itself), and a running count in shared memory whose last arrival does the release was slower
+            // still.  The barrier doubles as the vote on giving up: all warps leave together if any wait ran out.
             asm volatile("fence.proxy.async.global;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) {
-                unsigned int old;
-                asm volatile("atom.acq_rel.cta.shared::cta.add.u32 %0, [%1], 1;" : "=r"(old) : "r"(tc::smem_u32(arrived)) : "memory");
-                if (old == (unsigned int)(N_WORK * (s + 1) - 1)) tc::red_release_add_u32(counter, 1u);
-            }
+            unsigned int any_bad;
+            asm volatile("{\n\t.reg .pred p, q;\n\tsetp.eq.u32 p, %1, 0;\n\tbar.red.or.pred q, 1, %2, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+                         : "=r"(any_bad) : "r"((unsigned int)ok), "n"(N_WORK * 32) : "memory");
+            if (any_bad) break;
+            if (threadIdx.x == 0) tc::red_release_add_u32(counter, 1u);
         }
 #pragma unroll
         for (int i = 0; i < MAX_PAIRS; ++i)
