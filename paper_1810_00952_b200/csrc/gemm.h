@@ -28,6 +28,9 @@ relay_status_t launch_gemm(const GemmDesc &g, cudaStream_t st);
 
 // the two tiers, callable directly
 relay_status_t launch_gemm_simt(const GemmDesc &g, cudaStream_t st);
+// fp32 problems large enough to give every SM a 128 x 64 tile (gemm_simt_big.cu); launch_gemm_simt picks it itself
+bool gemm_simt_big_eligible(const GemmDesc &g);
+relay_status_t launch_gemm_simt_big(const GemmDesc &g, cudaStream_t st);
 bool gemm_tc_eligible(const GemmDesc &g);
 relay_status_t launch_gemm_tc(const GemmDesc &g, cudaStream_t st);
 // two-SM (cta_group::2) variant: 256 x 256 tiles computed by pairs of blocks

@@ -172,6 +172,7 @@ relay_status_t launch_gemm_simt(const GemmDesc &g, cudaStream_t st)
         br.add(g.bias, (size_t)g.N * dtype_size(g.bias_dtype));
         RELAY_TRY(br.commit(st));
     }
+    if (gemm_simt_big_eligible(g)) return launch_gemm_simt_big(g, st);
     // The largest tile whose grid still gives every SM a block: with few warps on an SM a block's time goes to waiting
     // for its own shared-memory reads, so while SMs are idle more and lighter blocks finish sooner.
     auto tiles = [&](int bm, int bn) { return ((g.M + bm - 1) / bm) * ((g.N + bn - 1) / bn); };

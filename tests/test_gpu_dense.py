@@ -242,7 +242,7 @@ def test_two_sm_kernel_fixed_unit_scheme_on_a_large_ragged_output():
     assert_bf16(y[rows], want, what="y")
 
 
-@pytest.mark.parametrize("M,K,N", [(37, 53, 29), (256, 512, 384), (520, 264, 1032), (8, 64, 32)])
+@pytest.mark.parametrize("M,K,N", [(37, 53, 29), (256, 512, 384), (520, 264, 1032), (8, 64, 32), (1100, 40, 1090)])
 @pytest.mark.parametrize("tdt", [torch.float32, torch.bfloat16])
 def test_contraction_with_operands_read_transposed(M, K, N, tdt):
     """The contraction as a call of its own, in the three forms the dense groups use (plain, b transposed as in
