@@ -818,7 +818,7 @@ def main():
         mhz = clocks.get("sm_mhz") or 1965.0
         peak_alu = sms * 128 * 2 * mhz * 1e6 / 1e12
         a = table["cfg1.fp32_mid.fwd"]["tflops"]
-        rooflines["gemm_simt_kernel (fp32 1024^3, true fp32 FMA with compensated run sums)"] = {
+        rooflines["gemm_simt_big_kernel (fp32 1024^3, true fp32 FMA with compensated run sums)"] = {
             "bound": "alu", "achieved": a, "peak": peak_alu, "unit": "TFLOP/s", "frac": a / peak_alu, "traffic": None,
             "peak_source": f"derived: {sms} SMs x 128 FMA lanes x 2 FLOP x {mhz:.0f} MHz (SM clock sampled during the run)"}
     for r_ in rooflines.values():
